@@ -1,0 +1,329 @@
+"""CPU oracle for SwiftKV prefill -- TEST INFRASTRUCTURE, not part of the product path.
+
+A plain, slow, fp64 numpy restatement of (1) the unmodified Llama-style decoder prefill (Sec. 3.1) and
+(2) the SwiftKV prefill (Sec. 3.2 Eq. 2, Sec. 3.3, Sec. 3.5), one step per line, no blocking, no fusion.
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this module; it shares no code
+with the CUDA library and never imports it.
+
+Pins (see tests/test_oracle_pins.py): brute-force attention, RoPE/RMSNorm/softmax identities, the
+identity-residual and constant-prompt special cases, l = L equals the baseline, g = 1 equals a separately
+written per-layer Eq. 2 loop, the folded fused projection equals norm-then-project, Table 1's FLOP rows,
+the KV-cache reduction percentages of Sec. 4, and library routines (torch fp64) on the tiny configuration.
+The paper prints no worked numerical example of a forward pass, so K/V/logit VALUES are pinned by these
+structural facts and library cross-checks only.
+
+Conventions.  Row vectors: a projection is  h @ W.T  with W stored [out_features, in_features] (the paper
+writes W x, Eq. 2).  `l` (swift_layer) is a COUNT: layers 1..l (0-based 0..l-1) run on every prompt token;
+s = output of layer l = the paper's x_{l+1}.  `g` = AcrossKV group size; groups are consecutive, aligned at
+layer l+1, the first layer of a group projects K/V for the whole group; a short last group is allowed.
+RoPE is the rotate-half form (pairs (i, i + hd/2)), positions restart at 0 for each prompt, K is cached
+after RoPE, V as projected.  RMSNorm eps as configured; softmax scale 1/sqrt(head_dim); no biases; untied
+embedding / lm_head.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import Callable, Dict, List, Sequence
+
+import numpy as np
+
+F64 = np.float64
+
+
+@dataclass
+class Config:
+    vocab: int
+    hidden: int
+    n_layers: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    rope_theta: float
+    rms_eps: float = 1e-5
+
+    @property
+    def d_q(self) -> int:
+        return self.n_q_heads * self.head_dim
+
+    @property
+    def d_kv(self) -> int:
+        return self.n_kv_heads * self.head_dim
+
+
+class Weights:
+    """Weight container.  `layer(j)` (0-based) returns a dict with in_norm, wq, wk, wv, wo, post_norm,
+    w_gate, w_up, w_down as fp64 arrays; it may build them lazily so that very large models never have to
+    be resident all at once.  `embed_rows(ids)` returns the embedding rows of the given token ids."""
+
+    def __init__(self, embed_rows: Callable[[np.ndarray], np.ndarray], final_norm: np.ndarray,
+                 lm_head: Callable[[], np.ndarray], layer: Callable[[int], Dict[str, np.ndarray]]):
+        self.embed_rows = embed_rows
+        self.final_norm = np.asarray(final_norm, dtype=F64)
+        self._lm_head = lm_head
+        self.layer = layer
+
+    def lm_head(self) -> np.ndarray:
+        return np.asarray(self._lm_head(), dtype=F64)
+
+    @staticmethod
+    def from_arrays(embed, final_norm, lm_head, layers: Sequence[Dict[str, np.ndarray]]) -> "Weights":
+        embed = np.asarray(embed, dtype=F64)
+        lm = np.asarray(lm_head, dtype=F64)
+        layers = [{k: np.asarray(v, dtype=F64) for k, v in w.items()} for w in layers]
+        return Weights(lambda ids: embed[np.asarray(ids, dtype=np.int64)], final_norm, lambda: lm,
+                       lambda j: layers[j])
+
+
+# ---------------------------------------------------------------------------------------------------
+# operators (Sec. 3.1)
+# ---------------------------------------------------------------------------------------------------
+def rmsnorm(x: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
+    """y = x / sqrt(mean(x^2) + eps) * gamma, over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gamma
+
+
+def unit_rms(x: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps): the statistic shared by every later layer's input norm of s."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps)
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary embedding, rotate-half pairing.  x: [n, heads, hd]; pos: [n] integer positions."""
+    n, _, hd = x.shape
+    half = hd // 2
+    i = np.arange(half, dtype=F64)
+    inv_freq = theta ** (-2.0 * i / hd)                       # [half]
+    ang = np.asarray(pos, dtype=F64)[:, None] * inv_freq[None, :]   # [n, half]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    a = x[..., :half]
+    b = x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def softmax_rows(z: np.ndarray) -> np.ndarray:
+    z = z - np.max(z, axis=-1, keepdims=True)
+    e = np.exp(z)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def causal_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """Causal grouped-query attention of one prompt against its own keys.
+    q: [n, n_q, hd]; K, V: [n, n_kv, hd]; query head h reads KV head h // (n_q / n_kv).  Returns [n, n_q*hd]."""
+    n, n_q, hd = q.shape
+    n_kv = K.shape[1]
+    rep = n_q // n_kv
+    out = np.empty((n, n_q, hd), dtype=F64)
+    allowed = np.tril(np.ones((n, n), dtype=bool))            # key t <= query p
+    for h in range(n_q):
+        kv = h // rep
+        scores = q[:, h, :] @ K[:, kv, :].T / math.sqrt(hd)   # [n, n]
+        scores = np.where(allowed, scores, -np.inf)
+        out[:, h, :] = softmax_rows(scores) @ V[:, kv, :]
+    return out.reshape(n, n_q * hd)
+
+
+def single_query_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """One query token (the last of its prompt) against every cached key of that prompt, itself included.
+    q: [n_q, hd]; K, V: [m, n_kv, hd].  Returns [n_q*hd]."""
+    n_q, hd = q.shape
+    rep = n_q // K.shape[1]
+    out = np.empty((n_q, hd), dtype=F64)
+    for h in range(n_q):
+        kv = h // rep
+        scores = K[:, kv, :] @ q[h] / math.sqrt(hd)           # [m]
+        out[h] = softmax_rows(scores[None, :])[0] @ V[:, kv, :]
+    return out.reshape(n_q * hd)
+
+
+def mlp(m: np.ndarray, w: Dict[str, np.ndarray]) -> np.ndarray:
+    return (silu(m @ w["w_gate"].T) * (m @ w["w_up"].T)) @ w["w_down"].T
+
+
+def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.ndarray):
+    """One unmodified decoder layer on all rows of one prompt.  Returns (X_out, K, V) with K after RoPE."""
+    n = X.shape[0]
+    h = rmsnorm(X, w["in_norm"], cfg.rms_eps)
+    q = (h @ w["wq"].T).reshape(n, cfg.n_q_heads, cfg.head_dim)
+    k = (h @ w["wk"].T).reshape(n, cfg.n_kv_heads, cfg.head_dim)
+    v = (h @ w["wv"].T).reshape(n, cfg.n_kv_heads, cfg.head_dim)
+    q = rope(q, pos, cfg.rope_theta)
+    k = rope(k, pos, cfg.rope_theta)
+    a = causal_attention(q, k, v)
+    X = X + a @ w["wo"].T
+    m = rmsnorm(X, w["post_norm"], cfg.rms_eps)
+    X = X + mlp(m, w)
+    return X, k, v
+
+
+def tail_layer(cfg: Config, w: Dict[str, np.ndarray], y: np.ndarray, p: int, K: np.ndarray, V: np.ndarray):
+    """A later layer (> l) applied to the one continuing token of a prompt (position p).  No K/V projection
+    happens here: the layer attends to the cache K, V[0..p] that the SwiftKV projection filled."""
+    h = rmsnorm(y, w["in_norm"], cfg.rms_eps)
+    q = (h @ w["wq"].T).reshape(1, cfg.n_q_heads, cfg.head_dim)
+    q = rope(q, np.array([p]), cfg.rope_theta)[0]
+    a = single_query_attention(q, K[: p + 1], V[: p + 1])
+    y = y + a @ w["wo"].T
+    m = rmsnorm(y, w["post_norm"], cfg.rms_eps)
+    return y + mlp(m, w)
+
+
+def _offsets(seq_lens: Sequence[int]) -> List[int]:
+    off = [0]
+    for n in seq_lens:
+        off.append(off[-1] + int(n))
+    return off
+
+
+# ---------------------------------------------------------------------------------------------------
+# the two models
+# ---------------------------------------------------------------------------------------------------
+def baseline(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]):
+    """Unmodified prefill (Sec. 3.1): every prompt token through all L layers.
+    Returns {"K": [L] x [T, n_kv, hd], "V": same, "logits": [B, vocab]} in packed prompt-major token order."""
+    return swiftkv(cfg, W, tokens, seq_lens, cfg.n_layers, 1)
+
+
+def group_leader(l: int, g: int, j: int) -> int:
+    """1-based layer j > l -> the 1-based layer whose K/V projection its AcrossKV group shares (Sec. 3.3)."""
+    return l + 1 + g * ((j - l - 1) // g)
+
+
+def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int], l: int, g: int = 1):
+    """SwiftKV prefill.  Layers 1..l as in the unmodified model; s = x_{l+1}; for every later layer j the
+    cache is  K_j = rope(rmsnorm(s, gamma_in[r]) @ W_K[r].T),  V_j = rmsnorm(s, gamma_in[r]) @ W_V[r].T
+    with r the leader of j's AcrossKV group (Eq. 2, Sec. 3.3); only the last token of each prompt runs
+    layers l+1..L (footnote in Sec. 3.2; Sec. 3.5), attending to those caches."""
+    L = cfg.n_layers
+    assert 1 <= l <= L and g >= 1
+    tokens = np.asarray(tokens, dtype=np.int64)
+    off = _offsets(seq_lens)
+    T, B = off[-1], len(seq_lens)
+    assert tokens.shape[0] == T
+    pos = np.concatenate([np.arange(n) for n in seq_lens]) if B else np.zeros(0, dtype=np.int64)
+
+    X = np.asarray(W.embed_rows(tokens), dtype=F64)            # x_1
+    K = [None] * L
+    V = [None] * L
+    for j in range(l):                                         # layers 1..l, all tokens
+        w = W.layer(j)
+        Kj = np.empty((T, cfg.n_kv_heads, cfg.head_dim), dtype=F64)
+        Vj = np.empty_like(Kj)
+        Xn = np.empty_like(X)
+        for b in range(B):
+            a, e = off[b], off[b + 1]
+            Xn[a:e], Kj[a:e], Vj[a:e] = decoder_layer(cfg, w, X[a:e], pos[a:e])
+        X, K[j], V[j] = Xn, Kj, Vj
+    s = X                                                      # x_{l+1}
+
+    for j1 in range(l + 1, L + 1):                             # 1-based later layers
+        r1 = group_leader(l, g, j1)
+        if j1 == r1:
+            w = W.layer(r1 - 1)
+            h = rmsnorm(s, w["in_norm"], cfg.rms_eps)
+            k = (h @ w["wk"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+            K[j1 - 1] = rope(k, pos, cfg.rope_theta)
+            V[j1 - 1] = (h @ w["wv"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+        else:
+            K[j1 - 1] = K[r1 - 1]                              # alias: one cache per group
+            V[j1 - 1] = V[r1 - 1]
+
+    last = [off[b + 1] - 1 for b in range(B)]
+    Y = s[last].copy()                                         # the continuing tokens
+    for j in range(l, L):
+        w = W.layer(j)
+        for b in range(B):
+            a, e = off[b], off[b + 1]
+            Y[b] = tail_layer(cfg, w, Y[b], e - a - 1, K[j][a:e], V[j][a:e])
+    logits = rmsnorm(Y, W.final_norm, cfg.rms_eps) @ W.lm_head().T
+    return {"K": K, "V": V, "logits": logits}
+
+
+def swiftkv_eq2_ungrouped(cfg: Config, W: Weights, s: np.ndarray, pos: np.ndarray, l: int):
+    """Eq. 2 written out with no grouping code at all: KV_j = W_KV^j applied to the normed s, for all j > l.
+    Used to pin swiftkv(l, g=1).  Returns ({j: K_j}, {j: V_j}) with 0-based j."""
+    Ks, Vs = {}, {}
+    T = s.shape[0]
+    for j in range(l, cfg.n_layers):
+        w = W.layer(j)
+        h = rmsnorm(s, w["in_norm"], cfg.rms_eps)
+        Ks[j] = rope((h @ w["wk"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim), pos, cfg.rope_theta)
+        Vs[j] = (h @ w["wv"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    return Ks, Vs
+
+
+def hidden_after(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int], n: int) -> np.ndarray:
+    """Residual stream after n unmodified layers (x_{n+1}), all tokens."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    off = _offsets(seq_lens)
+    pos = np.concatenate([np.arange(m) for m in seq_lens])
+    X = np.asarray(W.embed_rows(tokens), dtype=F64)
+    for j in range(n):
+        w = W.layer(j)
+        Xn = np.empty_like(X)
+        for b in range(len(seq_lens)):
+            a, e = off[b], off[b + 1]
+            Xn[a:e], _, _ = decoder_layer(cfg, w, X[a:e], pos[a:e])
+        X = Xn
+    return X
+
+
+# ---------------------------------------------------------------------------------------------------
+# the fused, gain-folded SingleInputKV projection (Sec. 3.5; one GEMM for all later layers)
+# ---------------------------------------------------------------------------------------------------
+def folded_kv_weight(cfg: Config, W: Weights, l: int, g: int) -> np.ndarray:
+    """Concatenate, over AcrossKV group leaders r, [diag(gamma_in[r]) folded into W_K[r] ; same for W_V[r]].
+    Returns [n_groups * 2 * d_kv, hidden]; rows of leader number i occupy [i*2*d_kv, (i+1)*2*d_kv), K first."""
+    blocks = []
+    for r1 in range(l + 1, cfg.n_layers + 1, g):
+        w = W.layer(r1 - 1)
+        blocks.append(w["wk"] * w["in_norm"][None, :])
+        blocks.append(w["wv"] * w["in_norm"][None, :])
+    return np.concatenate(blocks, axis=0)
+
+
+def fused_single_input_kv(cfg: Config, Wt: np.ndarray, s: np.ndarray, pos: np.ndarray):
+    """One projection of the unit-rms s through the folded weight; K blocks get RoPE.
+    Returns lists (K_i, V_i) per group leader i."""
+    T = s.shape[0]
+    out = unit_rms(s, cfg.rms_eps) @ Wt.T
+    n_groups = Wt.shape[0] // (2 * cfg.d_kv)
+    Ks, Vs = [], []
+    for i in range(n_groups):
+        blk = out[:, i * 2 * cfg.d_kv:(i + 1) * 2 * cfg.d_kv]
+        Ks.append(rope(blk[:, :cfg.d_kv].reshape(T, cfg.n_kv_heads, cfg.head_dim), pos, cfg.rope_theta))
+        Vs.append(blk[:, cfg.d_kv:].reshape(T, cfg.n_kv_heads, cfg.head_dim))
+    return Ks, Vs
+
+
+# ---------------------------------------------------------------------------------------------------
+# closed forms the paper prints: Table 1 (GFLOPs per prefill token) and the KV-cache reduction of Sec. 4
+# ---------------------------------------------------------------------------------------------------
+def table1_gflops_per_token(cfg: Config, l: int, g: int, context: float) -> Dict[str, float]:
+    """Per-prefill-token GFLOPs in the paper's Table 1 convention: 2 FLOPs per multiply-add; "Vocab" counts
+    the embedding and the lm_head both as matmuls; K,V is projected for every layer <= l and once per
+    AcrossKV group after it; Q,O / MLP / attention only for the l layers that prompt tokens run;
+    attention = QK^T and PV against an average of context/2 keys (causal)."""
+    L, d = cfg.n_layers, cfg.hidden
+    n_groups = -(-(L - l) // g)
+    vocab = 2 * (2 * d * cfg.vocab)
+    kv = (l + n_groups) * 2 * d * (2 * cfg.d_kv)
+    qo = l * (2 * d * cfg.d_q + 2 * cfg.d_q * d)
+    mlp_f = l * 3 * 2 * d * cfg.ffn
+    attn = l * 4 * cfg.d_q * (context / 2.0)
+    tot = vocab + kv + qo + mlp_f + attn
+    return {k: v / 1e9 for k, v in dict(vocab=vocab, kv=kv, qo=qo, mlp=mlp_f, attn=attn, total=tot).items()}
+
+
+def kv_cache_reduction(n_layers: int, l: int, g: int) -> float:
+    """Fraction of KV-cache memory saved: layers > l keep one cache per AcrossKV group."""
+    n_groups = -(-(n_layers - l) // g)
+    return 1.0 - (l + n_groups) / n_layers

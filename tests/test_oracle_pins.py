@@ -1,0 +1,351 @@
+"""Pins for the CPU oracle: facts the paper and the mathematics fix, independent of the oracle itself.
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a wrong sign or index, a
+transposed operand, a wrong mask) fails at least one of them.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as S
+from oracle import swiftkv_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _cfg(shape: S.ModelShape) -> O.Config:
+    return O.Config(shape.vocab, shape.hidden, shape.n_layers, shape.n_q_heads, shape.n_kv_heads,
+                    shape.head_dim, shape.ffn, shape.rope_theta, shape.rms_eps)
+
+
+def _weights(shape: S.ModelShape, seed=0, dtype=torch.float32, zero_out=False) -> O.Weights:
+    w = S.make_weights(shape, seed, dtype)
+    layers = []
+    for lw in w.layers:
+        d = {k: v.double().numpy() for k, v in lw.items()}
+        if zero_out:
+            d["wo"] = np.zeros_like(d["wo"])
+            d["w_down"] = np.zeros_like(d["w_down"])
+        layers.append(d)
+    return O.Weights.from_arrays(w.embed.double().numpy(), w.final_norm.double().numpy(),
+                                 w.lm_head.double().numpy(), layers)
+
+
+SMALL = S.ModelShape(96, 64, 6, 4, 2, 16, 80, 10000.0, 1e-5, "small")
+LENS = [13, 1, 7]
+
+
+@pytest.fixture(scope="module")
+def small():
+    cfg = _cfg(SMALL)
+    W = _weights(SMALL, seed=5)
+    tok = S.make_prompts(5, LENS, SMALL.vocab).numpy()
+    return cfg, W, tok
+
+
+def rel_l2(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+# ------------------------------------------------------------------ operators ---------------------
+def test_attention_against_brute_force():
+    """Explicit n x n scores, explicit mask, explicit loops -- on tiny inputs, including n = 1."""
+    rng = np.random.default_rng(0)
+    for n, nq, nkv, hd in [(1, 4, 2, 8), (5, 4, 1, 4), (17, 6, 3, 8), (33, 2, 2, 16)]:
+        q = rng.standard_normal((n, nq, hd))
+        K = rng.standard_normal((n, nkv, hd))
+        V = rng.standard_normal((n, nkv, hd))
+        got = O.causal_attention(q, K, V).reshape(n, nq, hd)
+        for p in range(n):
+            for h in range(nq):
+                kv = h // (nq // nkv)
+                w = [math.exp(sum(q[p, h, c] * K[t, kv, c] for c in range(hd)) / math.sqrt(hd)) for t in range(p + 1)]
+                z = sum(w)
+                ref = [sum(w[t] * V[t, kv, c] for t in range(p + 1)) / z for c in range(hd)]
+                assert np.allclose(got[p, h], ref, rtol=1e-10, atol=1e-12)
+        if n == 1:
+            assert np.allclose(got[0], np.repeat(V[0], nq // nkv, axis=0))
+        # the single-query form equals the last row of the causal form
+        sq = O.single_query_attention(q[-1], K, V)
+        assert np.allclose(sq, got[-1].reshape(-1), rtol=1e-12, atol=1e-14)
+
+
+def test_attention_against_torch_sdpa():
+    rng = np.random.default_rng(1)
+    n, nq, nkv, hd = 40, 8, 2, 32
+    q, K, V = (rng.standard_normal((n, h, hd)) for h in (nq, nkv, nkv))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q).transpose(0, 1)[None], torch.from_numpy(K).transpose(0, 1)[None],
+        torch.from_numpy(V).transpose(0, 1)[None], is_causal=True, enable_gqa=True)[0].transpose(0, 1)
+    assert np.allclose(O.causal_attention(q, K, V), ref.reshape(n, -1).numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_rope_identities():
+    rng = np.random.default_rng(2)
+    hd, theta = 16, 10000.0
+    q = rng.standard_normal((1, 3, hd))
+    k = rng.standard_normal((1, 3, hd))
+    assert np.array_equal(O.rope(q, np.array([0]), theta), q)                    # position 0 is the identity
+    for m, n in [(5, 3), (100, 7), (65535, 65000)]:
+        qm = O.rope(q, np.array([m]), theta)
+        kn = O.rope(k, np.array([n]), theta)
+        assert np.allclose(np.linalg.norm(qm, axis=-1), np.linalg.norm(q, axis=-1))   # a rotation
+        lhs = np.sum(qm * kn, axis=-1)
+        rhs = np.sum(O.rope(q, np.array([m - n]), theta) * k, axis=-1)           # depends on m - n only
+        assert np.allclose(lhs, rhs, rtol=1e-9, atol=1e-9)
+    # complex-number formulation: pair (i, i + hd/2) times exp(i * p * theta^(-2i/hd))
+    p = 11
+    x = rng.standard_normal((1, 1, hd))
+    z = (x[0, 0, :hd // 2] + 1j * x[0, 0, hd // 2:]) * np.exp(1j * p * theta ** (-2.0 * np.arange(hd // 2) / hd))
+    assert np.allclose(O.rope(x, np.array([p]), theta)[0, 0], np.concatenate([z.real, z.imag]))
+    # a hand-computed value: hd = 2, theta irrelevant (single frequency 1), 90-degree turn
+    out = O.rope(np.array([[[1.0, 0.0]]]), np.array([1]), 10000.0)
+    assert np.allclose(out[0, 0], [math.cos(1.0), math.sin(1.0)])
+
+
+def test_rmsnorm_silu_softmax():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((5, 32)) * 3
+    g = rng.standard_normal(32)
+    eps = 1e-5
+    y = O.rmsnorm(x, np.ones(32), eps)
+    ms = np.mean(x * x, -1)
+    assert np.allclose(np.mean(y * y, -1), ms / (ms + eps))
+    assert np.allclose(O.rmsnorm(1000 * x, g, eps), O.rmsnorm(x, g, eps), rtol=1e-4)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x), (32,), torch.from_numpy(g), eps).numpy()
+    assert np.allclose(O.rmsnorm(x, g, eps), ref, rtol=1e-12)
+    assert np.allclose(O.unit_rms(x, eps) * g, O.rmsnorm(x, g, eps))
+    assert O.silu(np.array([0.0]))[0] == 0.0
+    assert np.allclose(O.silu(np.array([30.0, -30.0])), [30.0, 0.0], atol=1e-11)
+    assert np.allclose(O.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy())
+    sm = O.softmax_rows(x)
+    assert np.allclose(sm.sum(-1), 1.0) and np.allclose(sm, torch.softmax(torch.from_numpy(x), -1).numpy())
+
+
+# ------------------------------------------------------------------ library cross-check -----------
+def _torch_llama_forward(shape, w, tokens, seq_lens):
+    """An independent fp64 forward of the unmodified model from torch library routines
+    (rms_norm, linear, scaled_dot_product_attention with GQA, silu) and complex-number RoPE."""
+    F = torch.nn.functional
+    dt = torch.float64
+    hd, half = shape.head_dim, shape.head_dim // 2
+    Ks, Vs, logits = [[] for _ in range(shape.n_layers)], [[] for _ in range(shape.n_layers)], []
+    off = 0
+    for n in seq_lens:
+        ids = torch.as_tensor(tokens[off:off + n]).long()
+        off += n
+        x = w.embed.to(dt)[ids]
+        rot = torch.polar(torch.ones(n, half, dtype=dt),
+                          torch.arange(n, dtype=dt)[:, None] * shape.rope_theta ** (-2.0 * torch.arange(half, dtype=dt) / hd))
+
+        def rope(t):
+            z = torch.complex(t[..., :half], t[..., half:]) * rot[:, None, :]
+            return torch.cat([z.real, z.imag], -1)
+        for j, lw in enumerate(w.layers):
+            lw = {k: v.to(dt) for k, v in lw.items()}
+            h = F.rms_norm(x, (shape.hidden,), lw["in_norm"], shape.rms_eps)
+            q = rope(F.linear(h, lw["wq"]).view(n, shape.n_q_heads, hd))
+            k = rope(F.linear(h, lw["wk"]).view(n, shape.n_kv_heads, hd))
+            v = F.linear(h, lw["wv"]).view(n, shape.n_kv_heads, hd)
+            Ks[j].append(k)
+            Vs[j].append(v)
+            a = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None],
+                                               v.transpose(0, 1)[None], is_causal=True, enable_gqa=True)
+            x = x + F.linear(a[0].transpose(0, 1).reshape(n, -1), lw["wo"])
+            m = F.rms_norm(x, (shape.hidden,), lw["post_norm"], shape.rms_eps)
+            x = x + F.linear(F.silu(F.linear(m, lw["w_gate"])) * F.linear(m, lw["w_up"]), lw["w_down"])
+        logits.append(F.linear(F.rms_norm(x[-1], (shape.hidden,), w.final_norm.to(dt), shape.rms_eps), w.lm_head.to(dt)))
+    return [torch.cat(k).numpy() for k in Ks], [torch.cat(v).numpy() for v in Vs], torch.stack(logits).numpy()
+
+
+def test_baseline_against_torch_library_forward_on_config1():
+    """Config 1 (tiny Llama-style decoder, prompts of 128 and 96 tokens): the oracle's unmodified model
+    against a forward pass assembled from torch library routines."""
+    shape = S.TINY
+    lens = [128, 96]
+    w = S.make_weights(shape, 0, torch.float32)
+    tok = S.make_prompts(0, lens, shape.vocab).numpy()
+    Kt, Vt, lt = _torch_llama_forward(shape, w, tok, lens)
+    out = O.baseline(_cfg(shape), _weights(shape, 0), tok, lens)
+    for j in range(shape.n_layers):
+        assert rel_l2(out["K"][j], Kt[j]) < 1e-12 and rel_l2(out["V"][j], Vt[j]) < 1e-12
+    assert rel_l2(out["logits"], lt) < 1e-12
+    # and the SwiftKV model agrees with it on everything that does not depend on the re-wiring
+    sk = O.swiftkv(_cfg(shape), _weights(shape, 0), tok, lens, 2, 1)
+    for j in range(2):
+        assert np.array_equal(sk["K"][j], out["K"][j]) and np.array_equal(sk["V"][j], out["V"][j])
+    assert rel_l2(sk["logits"], out["logits"]) > 1e-3          # it IS a different model
+
+
+# ------------------------------------------------------------------ SwiftKV structure -------------
+def test_layers_up_to_l_untouched_and_l_equal_L_is_baseline(small):
+    cfg, W, tok = small
+    base = O.baseline(cfg, W, tok, LENS)
+    for l in (1, 3, 5):
+        sk = O.swiftkv(cfg, W, tok, LENS, l, 2)
+        for j in range(l):
+            assert np.array_equal(sk["K"][j], base["K"][j]) and np.array_equal(sk["V"][j], base["V"][j])
+    full = O.swiftkv(cfg, W, tok, LENS, cfg.n_layers, 3)
+    for j in range(cfg.n_layers):
+        assert np.array_equal(full["K"][j], base["K"][j]) and np.array_equal(full["V"][j], base["V"][j])
+    assert np.array_equal(full["logits"], base["logits"])
+
+
+def test_group1_equals_ungrouped_eq2(small):
+    """AcrossKV with group 1 is SingleInputKV: compare with Eq. 2 written with no grouping code, fed with the
+    hidden state after l unmodified layers."""
+    cfg, W, tok = small
+    l = 2
+    s = O.hidden_after(cfg, W, tok, LENS, l)
+    pos = np.concatenate([np.arange(n) for n in LENS])
+    Ks, Vs = O.swiftkv_eq2_ungrouped(cfg, W, s, pos, l)
+    sk = O.swiftkv(cfg, W, tok, LENS, l, 1)
+    for j in range(l, cfg.n_layers):
+        assert np.allclose(sk["K"][j], Ks[j], rtol=1e-13, atol=1e-15)
+        assert np.allclose(sk["V"][j], Vs[j], rtol=1e-13, atol=1e-15)
+    # Eq. 2 on V needs no RoPE: V_j = rmsnorm(s) W_V^T, re-derived here from library calls
+    j = 4
+    w = W.layer(j)
+    v = torch.nn.functional.linear(
+        torch.nn.functional.rms_norm(torch.from_numpy(s), (cfg.hidden,), torch.from_numpy(w["in_norm"]), cfg.rms_eps),
+        torch.from_numpy(w["wv"])).numpy().reshape(-1, cfg.n_kv_heads, cfg.head_dim)
+    assert np.allclose(sk["V"][j], v, rtol=1e-12, atol=1e-14)
+
+
+def test_acrosskv_grouping(small):
+    """Fig. 1's example: L = 8, l = 4, 2-way AcrossKV -> layers 5,6 share layer 5's projection, 7,8 layer 7's."""
+    assert [O.group_leader(4, 2, j) for j in (5, 6, 7, 8)] == [5, 5, 7, 7]
+    assert [O.group_leader(2, 4, j) for j in (3, 4, 5, 6, 7)] == [3, 3, 3, 3, 7]
+    cfg, W, tok = small
+    l = 2
+    one = O.swiftkv(cfg, W, tok, LENS, l, 1)
+    for g in (2, 3, 4):
+        sk = O.swiftkv(cfg, W, tok, LENS, l, g)
+        distinct = {id(k) for k in sk["K"]}
+        assert len(distinct) == l + -(-(cfg.n_layers - l) // g)
+        for j1 in range(l + 1, cfg.n_layers + 1):
+            r1 = O.group_leader(l, g, j1)
+            assert sk["K"][j1 - 1] is sk["K"][r1 - 1] and sk["V"][j1 - 1] is sk["V"][r1 - 1]
+            # the projection of s does not depend on g
+            assert np.array_equal(sk["K"][r1 - 1], one["K"][r1 - 1])
+            assert np.array_equal(sk["V"][r1 - 1], one["V"][r1 - 1])
+        assert rel_l2(sk["logits"], one["logits"]) > 1e-6       # sharing changes the model
+
+
+def test_folded_fused_projection_equals_norm_then_project(small):
+    cfg, W, tok = small
+    pos = np.concatenate([np.arange(n) for n in LENS])
+    for l, g in [(2, 1), (2, 2), (1, 3)]:
+        s = O.hidden_after(cfg, W, tok, LENS, l)
+        Wt = O.folded_kv_weight(cfg, W, l, g)
+        n_groups = -(-(cfg.n_layers - l) // g)
+        assert Wt.shape == (n_groups * 2 * cfg.d_kv, cfg.hidden)
+        Ks, Vs = O.fused_single_input_kv(cfg, Wt, s, pos)
+        sk = O.swiftkv(cfg, W, tok, LENS, l, g)
+        for i in range(n_groups):
+            r = l + i * g
+            assert rel_l2(Ks[i], sk["K"][r]) < 1e-12 and rel_l2(Vs[i], sk["V"][r]) < 1e-12
+
+
+def test_identity_residual_special_case():
+    """W_O = W_down = 0 makes every layer the identity on the residual stream, so x_j = x_1 for all j and the
+    SwiftKV model (any l, g = 1) must reproduce the unmodified model exactly: the paper's premise
+    x_j ~ x_{l+1} made exact."""
+    cfg = _cfg(SMALL)
+    W = _weights(SMALL, seed=9, zero_out=True)
+    tok = S.make_prompts(9, LENS, SMALL.vocab).numpy()
+    base = O.baseline(cfg, W, tok, LENS)
+    for l in (1, 2, 4, 5):
+        sk = O.swiftkv(cfg, W, tok, LENS, l, 1)
+        for j in range(cfg.n_layers):
+            assert np.allclose(sk["K"][j], base["K"][j], rtol=1e-12, atol=1e-14)
+            assert np.allclose(sk["V"][j], base["V"][j], rtol=1e-12, atol=1e-14)
+        assert np.allclose(sk["logits"], base["logits"], rtol=1e-11, atol=1e-13)
+
+
+def test_constant_prompt_special_case():
+    """All tokens of a prompt identical -> all V rows identical -> attention output is V whatever the scores ->
+    hidden states are position-independent: logits(length n) = logits(length 1), K_j[p] = rope(K_j[0], p)."""
+    cfg = _cfg(SMALL)
+    W = _weights(SMALL, seed=3)
+    for fn in (lambda t, ln: O.baseline(cfg, W, t, ln), lambda t, ln: O.swiftkv(cfg, W, t, ln, 3, 2)):
+        a = fn(np.full(9, 17), [9])
+        b = fn(np.full(1, 17), [1])
+        assert np.allclose(a["logits"], b["logits"], rtol=1e-10, atol=1e-13)
+        for j in range(cfg.n_layers):
+            assert np.allclose(a["V"][j], np.broadcast_to(a["V"][j][0], a["V"][j].shape), rtol=1e-10, atol=1e-13)
+            k0 = np.repeat(b["K"][j], 9, axis=0)
+            assert np.allclose(a["K"][j], O.rope(k0, np.arange(9), cfg.rope_theta), rtol=1e-10, atol=1e-13)
+
+
+def test_causality_and_batch_independence(small):
+    cfg, W, tok = small
+    for l, g in [(cfg.n_layers, 1), (3, 2)]:
+        full = O.swiftkv(cfg, W, tok, LENS, l, g)
+        # a prompt alone gives the same caches and logits as inside the batch
+        off = 0
+        for b, n in enumerate(LENS):
+            alone = O.swiftkv(cfg, W, tok[off:off + n], [n], l, g)
+            for j in range(cfg.n_layers):
+                # (equal up to BLAS blocking: a [T, d] and an [n, d] product round in different orders)
+                assert np.allclose(alone["K"][j], full["K"][j][off:off + n], rtol=1e-12, atol=1e-14)
+                assert np.allclose(alone["V"][j], full["V"][j][off:off + n], rtol=1e-12, atol=1e-14)
+            assert np.allclose(alone["logits"][0], full["logits"][b], rtol=1e-12, atol=1e-14)   # BLAS blocks [B,d] and [1,d] differently
+            off += n
+        # changing later tokens leaves earlier cache rows untouched
+        t2 = tok.copy()
+        t2[8:13] = (t2[8:13] + 1) % cfg.vocab
+        ch = O.swiftkv(cfg, W, t2, LENS, l, g)
+        for j in range(cfg.n_layers):
+            assert np.array_equal(ch["K"][j][:8], full["K"][j][:8]) and np.array_equal(ch["V"][j][:8], full["V"][j][:8])
+            assert not np.array_equal(ch["V"][j][8:13], full["V"][j][8:13])
+        # a truncated prompt is a causal prefix
+        tr = O.swiftkv(cfg, W, tok[:6], [6], l, g)
+        for j in range(cfg.n_layers):
+            assert np.allclose(tr["K"][j], full["K"][j][:6], rtol=1e-12, atol=1e-14)
+            assert np.allclose(tr["V"][j], full["V"][j][:6], rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------------------ closed forms the paper prints --
+def _rows(name):
+    with open(os.path.join(GOLD, name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_table1_flop_breakdown():
+    cfg = _cfg(S.LLAMA31_70B)
+    rows = _rows("table1_gflops_per_token.txt")
+    # the context length behind the attention column is not printed; fix it from the baseline row only
+    base_attn = float(rows[0][6])
+    context = base_attn * 1e9 / (cfg.n_layers * 4 * cfg.d_q) * 2
+    base_total = None
+    for frac, g, vocab, kv, qo, mlp, attn, total, rel in rows:
+        l = round(cfg.n_layers * (1 - float(frac)))
+        got = O.table1_gflops_per_token(cfg, l, int(g), context)
+        assert abs(got["vocab"] - float(vocab)) < 0.11
+        assert abs(got["kv"] - float(kv)) < 0.1
+        assert abs(got["qo"] - float(qo)) < 0.6
+        assert abs(got["mlp"] - float(mlp)) < 0.6
+        assert abs(got["attn"] - float(attn)) < 0.6
+        assert abs(got["total"] - float(total)) < 1.5
+        base_total = base_total or got["total"]
+        assert abs(100 * got["total"] / base_total - float(rel)) < 0.15
+
+
+def test_kv_cache_reduction_percentages():
+    for g, pct in _rows("kv_cache_reduction.txt"):
+        assert abs(100 * O.kv_cache_reduction(32, 16, int(g)) - float(pct)) < 1e-9
+        if 40 % int(g) == 0:      # the printed figures assume whole groups; a short last group saves less
+            assert abs(100 * O.kv_cache_reduction(80, 40, int(g)) - float(pct)) < 1e-9
+    assert O.kv_cache_reduction(32, 32, 4) == 0.0 and O.kv_cache_reduction(32, 16, 1) == 0.0
+
+
+def test_normalized_throughput_arithmetic():
+    """tokens/s x 2 x parameter count of the baseline model reproduces the paper's TFLOPS/GPU figures."""
+    shapes = {"llama-3.1-70b": S.LLAMA31_70B, "llama-3.1-8b": S.LLAMA31_8B}
+    for name, tps, n_gpus, tflops in _rows("normalized_throughput.txt"):
+        got = float(tps) * 2 * shapes[name].n_params() / int(n_gpus) / 1e12
+        assert abs(got - float(tflops)) / float(tflops) < 0.01
