@@ -1,0 +1,207 @@
+/*
+ * swiftkv.h -- C ABI of the SwiftKV prefill library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the prefill of a Llama-style decoder (RMSNorm, rotary embedding, causal grouped-query
+ * attention, SwiGLU MLP; paper Sec. 3.1) re-wired by SwiftKV:
+ *   - SingleInputKV (Sec. 3.2, Eq. 2): layers 1..l run unchanged on every prompt token; the output of
+ *     layer l (the paper's x_{l+1}) is projected ONCE through the K/V projections of every later layer,
+ *     which fills their KV caches; prompt tokens skip every other operation of layers l+1..L.
+ *   - AcrossKV (Sec. 3.3): groups of g consecutive later layers share the K/V computed by the first layer of
+ *     the group and one cache allocation.
+ *   - The last token of each prompt continues through layers l+1..L to give the first output token's
+ *     logits (footnote of Sec. 3.2; Sec. 3.5: only the tokens that must produce output are propagated).
+ *   - The K/V projections of all later layers run as a single fused GEMM over a concatenated weight with
+ *     each layer's input-norm gain folded in (Sec. 3.5).
+ *
+ * Conventions
+ *   - Every function returns an int32 status (SWIFTKV_OK = 0, errors < 0), never throws, never aborts.
+ *     swiftkv_last_error() returns a thread-local description of the last failure in this thread.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are ordinary host
+ *     memory.  All buffers are CALLER-OWNED; the library allocates no device memory.  Device buffers must be
+ *     256-byte aligned unless stated.
+ *   - Weight matrices are [out_features, in_features] row-major in the model dtype (bf16 or fp32), gains
+ *     are vectors in the model dtype.  They must outlive the model and are never written by the library.
+ *   - swift_layer l is a COUNT: layers 1..l (0-based 0..l-1) run on all tokens; l = n_layers is the
+ *     unmodified model.  acrosskv_group g >= 1; groups are aligned at layer l+1; a short last group is allowed.
+ *   - Work is queued on the CUDA stream passed to swiftkv_prefill and is not synchronised by the library
+ *     unless stated; results are ordered after that stream.
+ */
+#ifndef SWIFTKV_H_
+#define SWIFTKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SWIFTKV_OK                    0
+#define SWIFTKV_ERR_INVALID_ARG      -1
+#define SWIFTKV_ERR_WORKSPACE_SMALL  -2
+#define SWIFTKV_ERR_NOT_READY        -3
+#define SWIFTKV_ERR_CUDA             -4
+#define SWIFTKV_ERR_DEVICE_TIMEOUT   -5   /* a bounded wait inside a kernel ran out                      */
+#define SWIFTKV_ERR_BAD_TOKEN        -6   /* a token id outside [0, vocab) was met on the device         */
+#define SWIFTKV_ERR_UNSUPPORTED      -7
+
+#define SWIFTKV_DTYPE_F32  0
+#define SWIFTKV_DTYPE_BF16 1
+
+typedef struct swiftkv_model swiftkv_model;   /* opaque, library-owned host object */
+
+typedef struct {
+  int32_t vocab, hidden, n_layers, n_q_heads, n_kv_heads, head_dim, ffn;
+  float   rope_theta, rms_eps;
+  int32_t dtype;                               /* SWIFTKV_DTYPE_*: storage type of weights, activations, KV cache */
+} swiftkv_config;
+
+typedef struct {                               /* one decoder layer; all device pointers                */
+  const void *in_norm;                         /* [hidden]                 gain of the input RMSNorm    */
+  const void *wq, *wk, *wv;                    /* [n_q*hd, hidden], [n_kv*hd, hidden] x 2               */
+  const void *wo;                              /* [hidden, n_q*hd]                                      */
+  const void *post_norm;                       /* [hidden]                 gain of the post-attention RMSNorm */
+  const void *w_gate, *w_up;                   /* [ffn, hidden] x 2                                     */
+  const void *w_down;                          /* [hidden, ffn]                                         */
+} swiftkv_layer_weights;
+
+typedef struct {
+  const void *embed;                           /* device [vocab, hidden]                                */
+  const void *final_norm;                      /* device [hidden]                                       */
+  const void *lm_head;                         /* device [vocab, hidden]                                */
+  const swiftkv_layer_weights *layers;         /* HOST array of n_layers entries (copied by model_load) */
+} swiftkv_weights;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int32_t swiftkv_version(void);
+
+/* Thread-local text of the last error raised in the calling thread ("" if none). */
+const char *swiftkv_last_error(void);
+
+/*
+ * Bytes the caller must provide for a model that will prefill at most max_tokens packed prompt tokens in at
+ * most max_seqs prompts with (swift_layer, acrosskv_group).
+ *   workspace_bytes : activations, metadata, the RoPE table, the folded SingleInputKV weight (Sec. 3.5).
+ *   kv_cache_bytes  : (l + ceil((L-l)/g)) cache slots of 2 * max_tokens * n_kv*hd elements: layers of one
+ *                     AcrossKV group share one slot, which is how the memory saving of Sec. 3.3 is realised
+ *                     ((L-l)/L * (1-1/g) of the unmodified model's cache when g divides L-l).
+ * A model loaded with these sizes also accepts any later (l', g') whose needs do not exceed them.
+ * Errors: INVALID_ARG (null pointers, non-positive sizes, l outside [1, L], g < 1, n_q % n_kv != 0, odd head_dim).
+ */
+int32_t swiftkv_workspace_bytes(const swiftkv_config *cfg, int32_t max_tokens, int32_t max_seqs,
+                                int32_t swift_layer, int32_t acrosskv_group,
+                                size_t *workspace_bytes, size_t *kv_cache_bytes);
+
+/*
+ * Create a model over caller-owned device buffers.  Records the (borrowed) weight pointers, builds the TMA
+ * descriptors of the weight matrices and fills the RoPE table (cos/sin of p * theta^(-2i/hd), evaluated in
+ * double precision, rotate-half pairing (i, i + hd/2)) on the current device's default stream, then
+ * synchronises that stream.  The device current at this call is the model's device.
+ * Errors: INVALID_ARG (as above, or a null / misaligned pointer), WORKSPACE_SMALL, CUDA.
+ */
+int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_weights *weights,
+                           void *workspace, size_t workspace_bytes,
+                           void *kv_cache, size_t kv_cache_bytes,
+                           int32_t max_tokens, int32_t max_seqs, swiftkv_model **out);
+
+/*
+ * SwiftKV prefill of a packed batch (Sec. 3.2 Eq. 2, Sec. 3.3, Sec. 3.5).
+ *   tokens   : HOST int32 [sum(seq_lens)], prompt-major; ids in [0, vocab)
+ *   seq_lens : HOST int32 [n_seqs], each >= 1
+ * Copies the ids to the device on `cuda_stream` (a cudaStream_t, may be 0), then queues every kernel of the
+ * path on that stream and returns without synchronising.  After the stream completes, the KV cache of every
+ * layer holds K (after RoPE) and V of every prompt token and the first-token logits are available.
+ * The first call with a new (swift_layer, acrosskv_group) also folds and concatenates the later layers' K/V
+ * weights (once; cached until another pair is used).
+ * Errors: INVALID_ARG (l, g, n_seqs, lengths, token range, totals beyond max_tokens / max_seqs),
+ *         WORKSPACE_SMALL ((l, g) needs more than the model was sized for), CUDA.
+ */
+int32_t swiftkv_prefill(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                        int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream);
+
+/*
+ * Same, with the token ids already resident on the device (DEVICE int32 [sum(seq_lens)]); seq_lens stays a
+ * HOST array.  Ids cannot be range-checked on the host: a bad id is clamped, recorded in the device status
+ * word and reported by swiftkv_status() as SWIFTKV_ERR_BAD_TOKEN.
+ */
+int32_t swiftkv_prefill_device_tokens(swiftkv_model *m, const int32_t *tokens_dev, const int32_t *seq_lens,
+                                      int32_t n_seqs, int32_t swift_layer, int32_t acrosskv_group,
+                                      void *cuda_stream);
+
+typedef struct {
+  const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype, AFTER RoPE            */
+  const void *v;            /* device, same shape                                                           */
+  int64_t token_stride;     /* elements between consecutive tokens (= n_kv_heads * head_dim)               */
+  int64_t head_stride;      /* elements between consecutive KV heads (= head_dim)                          */
+  int32_t n_tokens;         /* packed prompt tokens of the last prefill, prompt-major order                */
+  int32_t dtype;            /* SWIFTKV_DTYPE_*                                                              */
+  int32_t owner_layer;      /* 0-based layer whose projection produced this cache (the AcrossKV group's
+                               first layer for layers >= l; the layer itself otherwise)                    */
+} swiftkv_kv_view;
+
+/*
+ * Borrowed view of one layer's cache after the last prefill (layer is 0-based).  Layers of one AcrossKV
+ * group return the SAME pointers.  Valid until the next prefill or free; only ordered after the stream given
+ * to that prefill.  Errors: INVALID_ARG, NOT_READY (no prefill yet).
+ */
+int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out);
+
+/*
+ * Borrowed pointer to the first-token logits of the last prefill: DEVICE fp32 [n_seqs][vocab]
+ * (final RMSNorm then lm_head on the last token of each prompt).  Errors: INVALID_ARG, NOT_READY.
+ */
+int32_t swiftkv_first_logits(const swiftkv_model *m, const float **logits, int32_t *n_seqs);
+
+/*
+ * Synchronises `cuda_stream` and returns the device status word latched by the kernels of earlier calls:
+ * OK, DEVICE_TIMEOUT (a bounded in-kernel wait gave up; results are invalid), BAD_TOKEN, or CUDA.
+ * Clears the word.
+ */
+int32_t swiftkv_status(swiftkv_model *m, void *cuda_stream);
+
+/*
+ * Kernel-class timing.  With profiling enabled, each prefill brackets every launch with CUDA events on the
+ * prefill's stream; swiftkv_profile_read synchronises the stream and returns the device time (ms) and launch
+ * count accumulated per class since the last read, then resets them.  Classes are SWIFTKV_KC_*.
+ */
+#define SWIFTKV_KC_GEMM      0   /* projection / MLP / SingleInputKV GEMMs (M = all prompt tokens)       */
+#define SWIFTKV_KC_ATTENTION 1   /* causal varlen GQA prefill attention                                   */
+#define SWIFTKV_KC_ELEMWISE  2   /* embedding gather, RMSNorm, RoPE, SwiGLU, gathers, weight fold         */
+#define SWIFTKV_KC_TAIL      3   /* last-token path of layers > l and the lm_head                         */
+#define SWIFTKV_KC_COUNT     4
+int32_t swiftkv_profile_enable(swiftkv_model *m, int32_t on);
+int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, float *ms_per_class /*[KC_COUNT]*/,
+                             int32_t *launches_per_class /*[KC_COUNT]*/);
+
+/* Number of kernels the last prefill launched. */
+int32_t swiftkv_last_launch_count(const swiftkv_model *m);
+
+/* Select kernel families (debug / comparison): bit 0 = tensor-core GEMMs, bit 1 = tensor-core attention.
+ * Default: all that the model's shape and dtype support.  Returns the mask in effect. */
+int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
+
+/* Destroys the host object (never the caller's buffers).  Null is allowed. */
+void swiftkv_model_free(swiftkv_model *m);
+
+/*
+ * Stand-alone operator entry points (the same kernels the prefill uses), for unit tests and profiling.
+ * All pointers are DEVICE memory; all run on `cuda_stream` without synchronising.
+ */
+
+/* C[M,N] = A[M,K] * B[N,K]^T, bf16 in, fp32 accumulate on the tensor cores (tcgen05), bf16 out, row-major,
+ * ldc = N.  Needs K % 64 == 0, N % 128 == 0, 16-byte aligned pointers.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
+                          void *cuda_stream);
+
+/* Causal varlen grouped-query attention (Sec. 3.1) on packed prompts.  q [T, n_q, hd], k, v [T, n_kv, hd],
+ * out [T, n_q*hd] in `dtype`; cu_seqlens DEVICE int32 [n_seqs+1]; softmax scale 1/sqrt(hd).
+ * max_seq_len bounds the longest prompt (grid sizing). */
+int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, void *out,
+                                  const int32_t *cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                                  int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                  int32_t dtype, int32_t use_tensor_cores, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWIFTKV_H_ */

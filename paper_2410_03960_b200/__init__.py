@@ -1,0 +1,16 @@
+"""SwiftKV prefill for NVIDIA B200: a thin Python binding over the C-ABI CUDA library (libswiftkv.so).
+
+Every step of the prefill runs in the library's kernels; this package only marshals arguments.
+PyTorch is used for device memory and streams.
+"""
+from .binding import (  # noqa: F401
+    KC_NAMES,
+    SwiftKVError,
+    SwiftKVModel,
+    attention_prefill,
+    gemm_bf16,
+    library_path,
+    load_library,
+    workspace_bytes,
+)
+from .flops import prefill_flops  # noqa: F401

@@ -1,0 +1,238 @@
+"""ctypes binding of libswiftkv.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB: Optional[C.CDLL] = None
+
+DTYPE_F32, DTYPE_BF16 = 0, 1
+KC_NAMES = ("gemm", "attention", "elementwise", "tail")
+
+# every symbol include/swiftkv.h declares
+EXPORTS = (
+    "swiftkv_version", "swiftkv_last_error", "swiftkv_workspace_bytes", "swiftkv_model_load", "swiftkv_prefill",
+    "swiftkv_prefill_device_tokens", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
+    "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
+    "swiftkv_model_free", "swiftkv_gemm_bf16", "swiftkv_attention_prefill",
+)
+
+
+class SwiftKVError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"swiftkv error {code}: {msg}")
+        self.code = code
+
+
+class _Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("vocab", "hidden", "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "ffn")] + \
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32)]
+
+
+class _LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("in_norm", "wq", "wk", "wv", "wo", "post_norm", "w_gate", "w_up", "w_down")]
+
+
+class _Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p),
+                ("layers", C.POINTER(_LayerWeights))]
+
+
+class _KVView(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("token_stride", C.c_int64), ("head_stride", C.c_int64),
+                ("n_tokens", C.c_int32), ("dtype", C.c_int32), ("owner_layer", C.c_int32)]
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libswiftkv.so")
+
+
+def load_library() -> C.CDLL:
+    """Loads libswiftkv.so.  There is no fallback: without the built CUDA library nothing in this package runs."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2410_03960_b200.build` "
+                           "(the SwiftKV prefill path has no CPU or PyTorch fallback)")
+    lib = C.CDLL(path)
+    lib.swiftkv_last_error.restype = C.c_char_p
+    lib.swiftkv_workspace_bytes.argtypes = [C.POINTER(_Config), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                            C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    lib.swiftkv_model_load.argtypes = [C.POINTER(_Config), C.POINTER(_Weights), C.c_void_p, C.c_size_t, C.c_void_p,
+                                       C.c_size_t, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]
+    lib.swiftkv_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+    lib.swiftkv_prefill_device_tokens.argtypes = lib.swiftkv_prefill.argtypes
+    lib.swiftkv_kv_cache_view.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_KVView)]
+    lib.swiftkv_first_logits.argtypes = [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)]
+    lib.swiftkv_status.argtypes = [C.c_void_p, C.c_void_p]
+    lib.swiftkv_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+    lib.swiftkv_last_launch_count.argtypes = [C.c_void_p]
+    lib.swiftkv_set_kernel_mask.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_model_free.argtypes = [C.c_void_p]
+    lib.swiftkv_model_free.restype = None
+    lib.swiftkv_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+    lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 8 + [C.c_void_p]
+    _LIB = lib
+    return lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise SwiftKVError(rc, load_library().swiftkv_last_error().decode())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _make_config(shape, dtype: torch.dtype) -> _Config:
+    code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[dtype]
+    return _Config(shape.vocab, shape.hidden, shape.n_layers, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                   shape.ffn, float(shape.rope_theta), float(shape.rms_eps), code)
+
+
+def workspace_bytes(shape, dtype: torch.dtype, max_tokens: int, max_seqs: int, swift_layer: int,
+                    acrosskv_group: int) -> Tuple[int, int]:
+    """swiftkv_workspace_bytes -> (workspace_bytes, kv_cache_bytes)."""
+    cfg = _make_config(shape, dtype)
+    ws, kv = C.c_size_t(0), C.c_size_t(0)
+    _check(load_library().swiftkv_workspace_bytes(C.byref(cfg), max_tokens, max_seqs, swift_layer, acrosskv_group,
+                                                  C.byref(ws), C.byref(kv)))
+    return ws.value, kv.value
+
+
+class SwiftKVModel:
+    """swiftkv_model_load / swiftkv_prefill / swiftkv_kv_cache_view / swiftkv_first_logits over torch CUDA tensors.
+
+    `weights` needs .embed, .final_norm, .lm_head and .layers (a list of dicts with in_norm, wq, wk, wv, wo,
+    post_norm, w_gate, w_up, w_down) as contiguous CUDA tensors of `dtype`, [out_features, in_features].
+    The workspace and the KV cache are torch tensors owned by this object.
+    """
+
+    def __init__(self, shape, weights, dtype: torch.dtype, max_tokens: int, max_seqs: int, swift_layer: int,
+                 acrosskv_group: int = 1, device: str = "cuda:0"):
+        self.lib = load_library()
+        self.shape, self.dtype, self.device = shape, dtype, torch.device(device)
+        self.max_tokens, self.max_seqs = max_tokens, max_seqs
+        self._weights = weights           # keep the tensors alive: the library borrows their memory
+        ws_b, kv_b = workspace_bytes(shape, dtype, max_tokens, max_seqs, swift_layer, acrosskv_group)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(ws_b, dtype=torch.uint8, device=self.device)
+            self.kv_cache = torch.empty(kv_b, dtype=torch.uint8, device=self.device)
+            cfg = _make_config(shape, dtype)
+            arr = (_LayerWeights * shape.n_layers)()
+            for j, lw in enumerate(weights.layers):
+                for name, _ in _LayerWeights._fields_:
+                    t = lw[name]
+                    assert t.is_cuda and t.is_contiguous() and t.dtype == dtype, name
+                    setattr(arr[j], name, t.data_ptr())
+            for t in (weights.embed, weights.final_norm, weights.lm_head):
+                assert t.is_cuda and t.is_contiguous() and t.dtype == dtype
+            w = _Weights(weights.embed.data_ptr(), weights.final_norm.data_ptr(), weights.lm_head.data_ptr(), arr)
+            handle = C.c_void_p()
+            _check(self.lib.swiftkv_model_load(C.byref(cfg), C.byref(w), self.workspace.data_ptr(), ws_b,
+                                               self.kv_cache.data_ptr(), kv_b, max_tokens, max_seqs, C.byref(handle)))
+        self._h = handle
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self.lib.swiftkv_model_free(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def prefill(self, tokens, seq_lens: Sequence[int], swift_layer: int, acrosskv_group: int = 1,
+                stream: Optional[torch.cuda.Stream] = None) -> None:
+        """swiftkv_prefill: `tokens` is a HOST int32 tensor (packed, prompt-major)."""
+        tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous()
+        assert not tokens.is_cuda
+        lens = (C.c_int32 * len(seq_lens))(*[int(n) for n in seq_lens])
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_prefill(self._h, tokens.data_ptr(), lens, len(seq_lens), swift_layer, acrosskv_group,
+                                            _stream_ptr(stream)))
+
+    def prefill_device_tokens(self, tokens_dev: torch.Tensor, seq_lens: Sequence[int], swift_layer: int,
+                              acrosskv_group: int = 1, stream: Optional[torch.cuda.Stream] = None) -> None:
+        assert tokens_dev.is_cuda and tokens_dev.dtype == torch.int32 and tokens_dev.is_contiguous()
+        lens = (C.c_int32 * len(seq_lens))(*[int(n) for n in seq_lens])
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_prefill_device_tokens(self._h, tokens_dev.data_ptr(), lens, len(seq_lens), swift_layer,
+                                                          acrosskv_group, _stream_ptr(stream)))
+
+    def kv_cache_view(self, layer: int) -> Tuple[torch.Tensor, torch.Tensor, int]:
+        """swiftkv_kv_cache_view -> (K [n_tokens, n_kv, hd], V, owner_layer) as views into the cache tensor."""
+        v = _KVView()
+        _check(self.lib.swiftkv_kv_cache_view(self._h, layer, C.byref(v)))
+        flat = self.kv_cache.view(self.dtype)
+        es = flat.element_size()
+        n = v.n_tokens * v.token_stride
+        shape = (v.n_tokens, self.shape.n_kv_heads, self.shape.head_dim)
+        ko = (v.k - self.kv_cache.data_ptr()) // es
+        vo = (v.v - self.kv_cache.data_ptr()) // es
+        return flat[ko:ko + n].view(shape), flat[vo:vo + n].view(shape), v.owner_layer
+
+    def first_logits(self) -> torch.Tensor:
+        """swiftkv_first_logits -> fp32 [n_seqs, vocab] view into the workspace."""
+        p, n = C.c_void_p(), C.c_int32()
+        _check(self.lib.swiftkv_first_logits(self._h, C.byref(p), C.byref(n)))
+        off = (p.value - self.workspace.data_ptr()) // 4
+        flat = self.workspace[: (self.workspace.numel() // 4) * 4].view(torch.float32)
+        return flat[off: off + n.value * self.shape.vocab].view(n.value, self.shape.vocab)
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> None:
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_status(self._h, _stream_ptr(stream)))
+
+    def profile_enable(self, on: bool) -> None:
+        _check(self.lib.swiftkv_profile_enable(self._h, int(on)))
+
+    def profile_read(self, stream: Optional[torch.cuda.Stream] = None) -> Dict[str, Tuple[float, int]]:
+        ms = (C.c_float * len(KC_NAMES))()
+        cnt = (C.c_int32 * len(KC_NAMES))()
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_profile_read(self._h, _stream_ptr(stream), ms, cnt))
+        return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KC_NAMES)}
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.swiftkv_last_launch_count(self._h))
+
+    def set_kernel_mask(self, mask: int) -> int:
+        return int(self.lib.swiftkv_set_kernel_mask(self._h, mask))
+
+
+def gemm_bf16(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_gemm_bf16: C = A @ B.T with A [M, K], B [N, K] bf16 CUDA tensors."""
+    assert a.is_cuda and b.is_cuda and a.dtype == b.dtype == torch.bfloat16 and a.is_contiguous() and b.is_contiguous()
+    m, k = a.shape
+    n = b.shape[0]
+    c = torch.empty((m, n), dtype=torch.bfloat16, device=a.device)
+    with torch.cuda.device(a.device):
+        _check(load_library().swiftkv_gemm_bf16(a.data_ptr(), b.data_ptr(), c.data_ptr(), m, n, k, _stream_ptr(stream)))
+    return c
+
+
+def attention_prefill(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens: Sequence[int],
+                      use_tensor_cores: bool, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_attention_prefill on packed prompts: q [T, n_q, hd], k/v [T, n_kv, hd] -> [T, n_q*hd]."""
+    assert q.is_cuda and q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
+    t, n_q, hd = q.shape
+    n_kv = k.shape[1]
+    cu = [0]
+    for n in seq_lens:
+        cu.append(cu[-1] + int(n))
+    assert cu[-1] == t
+    cu_dev = torch.tensor(cu, dtype=torch.int32, device=q.device)
+    out = torch.empty((t, n_q * hd), dtype=q.dtype, device=q.device)
+    code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[q.dtype]
+    with torch.cuda.device(q.device):
+        _check(load_library().swiftkv_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
+                                                        cu_dev.data_ptr(), len(seq_lens), t, max(seq_lens), n_q, n_kv, hd,
+                                                        code, int(use_tensor_cores), _stream_ptr(stream)))
+    return out

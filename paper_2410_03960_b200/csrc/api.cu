@@ -1,0 +1,563 @@
+// C ABI and host-side prefill schedule of the SwiftKV prefill library.
+//
+// The schedule follows the paper's inference procedure (Sec. 3.5): layers 1..l on every prompt token, then --
+// immediately after layer l -- the KV caches of all later layers from one fused, gain-folded projection of
+// the layer-l output (Eq. 2; AcrossKV groups, Sec. 3.3, share one cache slot), then only the last token of
+// each prompt through layers l+1..L and the lm_head.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace skv;
+
+// ---------------------------------------------------------------------------------------------------------
+// errors
+// ---------------------------------------------------------------------------------------------------------
+static thread_local std::string g_last_error;
+static int32_t fail(int32_t code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_last_error = buf;
+  return code;
+}
+#define CUDA_TRY(expr)                                                                                   \
+  do {                                                                                                   \
+    cudaError_t e__ = (expr);                                                                            \
+    if (e__ != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------------------------
+// model object
+// ---------------------------------------------------------------------------------------------------------
+struct Carve {   // walks a buffer handing out 256-byte aligned regions; with base == nullptr it only measures
+  uint8_t *base;
+  size_t off = 0;
+  explicit Carve(void *b) : base(reinterpret_cast<uint8_t *>(b)) {}
+  void *take(size_t bytes) {
+    off = (off + 255) & ~(size_t)255;
+    void *p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+struct Buffers {
+  float *x;                 // fp32 residual stream [T, d]
+  void *h, *q, *attn;       // normed hidden [T, d]; queries [T, d_q]; attention output [T, d_q]
+  void *gate, *up;          // unfused MLP scratch [mlp_chunk, F] each
+  void *act;                // SwiGLU output [T, F]
+  void *wfold;              // folded, concatenated SingleInputKV weight [n_groups*2*d_kv, d]
+  float *y;                 // continuing tokens' residual [B, d]
+  void *hy, *qy, *ay, *gy, *uy, *acty;
+  float *tail_scratch;
+  float *logits;            // [B, vocab]
+  int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
+  unsigned int *status;
+  float *cos_tab, *sin_tab;
+};
+
+static const int MLP_CHUNK_ROWS = 8192;
+
+struct swiftkv_model {
+  swiftkv_config cfg;
+  std::vector<swiftkv_layer_weights> layers;
+  const void *embed, *final_norm, *lm_head;
+  int max_tokens, max_seqs;
+  size_t esize;
+  size_t fold_capacity_elems;   // elements reserved for the folded weight
+  int slot_capacity;            // cache slots the KV buffer holds
+  uint8_t *kv;
+  Buffers b;
+  int device;
+  // state of the last prefill
+  bool ready = false;
+  int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;
+  int fold_l = -1, fold_g = -1;
+  int launches = 0;
+  int kernel_mask = 3;
+  // profiling
+  bool profiling = false;
+  std::vector<cudaEvent_t> pool;
+  struct Rec { cudaEvent_t a, b; int cls; };
+  std::vector<Rec> recs;
+  std::vector<int32_t> host_meta;
+};
+
+static size_t dsize(int dtype) { return dtype == SWIFTKV_DTYPE_BF16 ? 2 : 4; }
+static int n_groups(int L, int l, int g) { return (L - l + g - 1) / g; }
+
+static int32_t check_cfg(const swiftkv_config *c, int max_tokens, int max_seqs, int l, int g) {
+  if (!c) return fail(SWIFTKV_ERR_INVALID_ARG, "config is null");
+  if (c->vocab < 1 || c->hidden < 1 || c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->head_dim < 2 || c->ffn < 1)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "non-positive model dimension");
+  if (c->n_q_heads % c->n_kv_heads) return fail(SWIFTKV_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
+  if (c->head_dim % 2 || c->head_dim > 256) return fail(SWIFTKV_ERR_INVALID_ARG, "head_dim must be even and <= 256");
+  if (c->dtype != SWIFTKV_DTYPE_F32 && c->dtype != SWIFTKV_DTYPE_BF16) return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+  if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return fail(SWIFTKV_ERR_INVALID_ARG, "bad rope_theta / rms_eps");
+  if (max_tokens < 1 || max_seqs < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "max_tokens and max_seqs must be positive");
+  if (l < 1 || l > c->n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c->n_layers);
+  if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
+  return SWIFTKV_OK;
+}
+
+static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, Carve &cv, Buffers &b) {
+  const size_t E = dsize(c.dtype);
+  const size_t d = c.hidden, dq = (size_t)c.n_q_heads * c.head_dim, F = c.ffn;
+  const size_t chunk = std::min<size_t>(T, MLP_CHUNK_ROWS);
+  b.x = (float *)cv.take((size_t)T * d * 4);
+  b.h = cv.take((size_t)T * d * E);
+  b.q = cv.take((size_t)T * dq * E);
+  b.attn = cv.take((size_t)T * dq * E);
+  b.gate = cv.take(chunk * F * E);
+  b.up = cv.take(chunk * F * E);
+  b.act = cv.take((size_t)T * F * E);
+  b.wfold = cv.take(fold_elems * E);
+  b.y = (float *)cv.take((size_t)B * d * 4);
+  b.hy = cv.take((size_t)B * std::max(d, dq) * E);
+  b.qy = cv.take((size_t)B * dq * E);
+  b.ay = cv.take((size_t)B * dq * E);
+  b.gy = cv.take((size_t)B * F * E);
+  b.uy = cv.take((size_t)B * F * E);
+  b.acty = cv.take((size_t)B * F * E);
+  b.tail_scratch = (float *)cv.take(tail_attention_scratch_bytes(B, c.n_q_heads, c.head_dim, T));
+  b.logits = (float *)cv.take((size_t)B * c.vocab * 4);
+  b.tokens = (int32_t *)cv.take((size_t)T * 4);
+  b.cu = (int32_t *)cv.take((size_t)(B + 1) * 4);
+  b.pos = (int32_t *)cv.take((size_t)T * 4);
+  b.last_idx = (int32_t *)cv.take((size_t)B * 4);
+  b.last_pos = (int32_t *)cv.take((size_t)B * 4);
+  b.status = (unsigned int *)cv.take(256);
+  b.cos_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
+  b.sin_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
+}
+
+static size_t fold_elems_for(const swiftkv_config &c, int l, int g) {
+  return (size_t)n_groups(c.n_layers, l, g) * 2 * c.n_kv_heads * c.head_dim * c.hidden;
+}
+static size_t slot_elems(const swiftkv_config &c, int T) { return (size_t)2 * T * c.n_kv_heads * c.head_dim; }
+
+// ---------------------------------------------------------------------------------------------------------
+extern "C" int32_t swiftkv_version(void) { return 100; }
+extern "C" const char *swiftkv_last_error(void) { return g_last_error.c_str(); }
+
+extern "C" int32_t swiftkv_workspace_bytes(const swiftkv_config *cfg, int32_t max_tokens, int32_t max_seqs,
+                                           int32_t swift_layer, int32_t acrosskv_group, size_t *workspace_bytes,
+                                           size_t *kv_cache_bytes) {
+  int32_t rc = check_cfg(cfg, max_tokens, max_seqs, swift_layer, acrosskv_group);
+  if (rc) return rc;
+  if (!workspace_bytes || !kv_cache_bytes) return fail(SWIFTKV_ERR_INVALID_ARG, "output pointer is null");
+  Carve cv(nullptr);
+  Buffers b;
+  carve_all(*cfg, max_tokens, max_seqs, fold_elems_for(*cfg, swift_layer, acrosskv_group), cv, b);
+  *workspace_bytes = ((cv.off + 255) & ~(size_t)255) + 512;
+  const int slots = swift_layer + n_groups(cfg->n_layers, swift_layer, acrosskv_group);
+  *kv_cache_bytes = (size_t)slots * slot_elems(*cfg, max_tokens) * dsize(cfg->dtype);
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_weights *w, void *workspace,
+                                      size_t workspace_bytes, void *kv_cache, size_t kv_cache_bytes,
+                                      int32_t max_tokens, int32_t max_seqs, swiftkv_model **out) {
+  if (!out) return fail(SWIFTKV_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  int32_t rc = check_cfg(cfg, max_tokens, max_seqs, 1, 1);
+  if (rc) return rc;
+  if (!w || !w->embed || !w->final_norm || !w->lm_head || !w->layers) return fail(SWIFTKV_ERR_INVALID_ARG, "a weight pointer is null");
+  if (!workspace || !kv_cache) return fail(SWIFTKV_ERR_INVALID_ARG, "workspace / kv_cache is null");
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(kv_cache) & 255))
+    return fail(SWIFTKV_ERR_INVALID_ARG, "workspace and kv_cache must be 256-byte aligned");
+  for (int j = 0; j < cfg->n_layers; ++j) {
+    const swiftkv_layer_weights &lw = w->layers[j];
+    const void *ps[9] = {lw.in_norm, lw.wq, lw.wk, lw.wv, lw.wo, lw.post_norm, lw.w_gate, lw.w_up, lw.w_down};
+    for (const void *p : ps) {
+      if (!p) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d: a weight pointer is null", j);
+      if (reinterpret_cast<uintptr_t>(p) & 15) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d: weights must be 16-byte aligned", j);
+    }
+  }
+  // smallest workspace: no folded weight at all (l = L)
+  Carve measure(nullptr);
+  Buffers tmp;
+  carve_all(*cfg, max_tokens, max_seqs, 0, measure, tmp);
+  const size_t base_need = (measure.off + 255) & ~(size_t)255;
+  if (workspace_bytes < base_need) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "workspace %zu < %zu bytes", workspace_bytes, base_need);
+  const size_t E = dsize(cfg->dtype);
+  const size_t slot_bytes = slot_elems(*cfg, max_tokens) * E;
+  if (kv_cache_bytes < slot_bytes) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "kv cache smaller than one slot");
+
+  swiftkv_model *m = new (std::nothrow) swiftkv_model();
+  if (!m) return fail(SWIFTKV_ERR_CUDA, "out of host memory");
+  m->cfg = *cfg;
+  m->layers.assign(w->layers, w->layers + cfg->n_layers);
+  m->embed = w->embed; m->final_norm = w->final_norm; m->lm_head = w->lm_head;
+  m->max_tokens = max_tokens; m->max_seqs = max_seqs; m->esize = E;
+  // everything beyond the base need is room for the folded weight (kept 256-byte slack for alignment)
+  m->fold_capacity_elems = workspace_bytes - base_need > 256 ? (workspace_bytes - base_need - 256) / E : 0;
+  m->slot_capacity = (int)std::min<size_t>(kv_cache_bytes / slot_bytes, 1u << 20);
+  m->kv = reinterpret_cast<uint8_t *>(kv_cache);
+  Carve cv(workspace);
+  carve_all(*cfg, max_tokens, max_seqs, m->fold_capacity_elems, cv, m->b);
+  if (cudaGetDevice(&m->device) != cudaSuccess) { delete m; return fail(SWIFTKV_ERR_CUDA, "cudaGetDevice failed"); }
+  cudaError_t e = cudaMemsetAsync(m->b.status, 0, 256, 0);
+  if (e == cudaSuccess) {
+    launch_rope_table(m->b.cos_tab, m->b.sin_tab, max_tokens, cfg->head_dim, (double)cfg->rope_theta, 0);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+  if (e != cudaSuccess) { delete m; return fail(SWIFTKV_ERR_CUDA, "model_load: %s", cudaGetErrorString(e)); }
+  *out = m;
+  return SWIFTKV_OK;
+}
+
+extern "C" void swiftkv_model_free(swiftkv_model *m) {
+  if (!m) return;
+  for (cudaEvent_t ev : m->pool) cudaEventDestroy(ev);
+  for (auto &r : m->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  delete m;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// launch bookkeeping: counts launches; with profiling on, brackets each launch with events
+// ---------------------------------------------------------------------------------------------------------
+struct Scope {
+  swiftkv_model *m; cudaStream_t st; int cls; cudaEvent_t a = nullptr, b = nullptr;
+  static cudaEvent_t get(swiftkv_model *m) {
+    if (!m->pool.empty()) { cudaEvent_t e = m->pool.back(); m->pool.pop_back(); return e; }
+    cudaEvent_t e; cudaEventCreate(&e); return e;
+  }
+  Scope(swiftkv_model *m_, cudaStream_t s, int c, int n_launches = 1) : m(m_), st(s), cls(c) {
+    m->launches += n_launches;
+    if (m->profiling) { a = get(m); b = get(m); cudaEventRecord(a, st); }
+  }
+  ~Scope() {
+    if (m->profiling) { cudaEventRecord(b, st); m->recs.push_back({a, b, cls}); }
+  }
+};
+
+// ---------------------------------------------------------------------------------------------------------
+// the schedule
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+static int32_t gemm_any(swiftkv_model *m, const T *A, int M, int K, const T *B0, int n0, const T *B1, int n1,
+                        const T *B2, int n2, const OutDesc &out, cudaStream_t st) {
+  Scope sc(m, st, SWIFTKV_KC_GEMM, 0);
+  if constexpr (sizeof(T) == 2) {
+    if ((m->kernel_mask & 1) && tc_gemm_supported(M, n0 + n1 + n2, K)) {
+      int rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, m->b.status, st);
+      if (rc == SWIFTKV_OK) { m->launches += 1; return rc; }
+      if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "tensor-core GEMM launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+  }
+  launch_gemm_simt<T>(A, B0, M, n0, K, out, 0, st);
+  m->launches += 1;
+  if (n1 > 0) { launch_gemm_simt<T>(A, B1, M, n1, K, out, n0, st); m->launches += 1; }
+  if (n2 > 0) { launch_gemm_simt<T>(A, B2, M, n2, K, out, n0 + n1, st); m->launches += 1; }
+  return SWIFTKV_OK;
+}
+
+template <typename T>
+static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int l, int g, cudaStream_t st) {
+  const swiftkv_config &c = m->cfg;
+  Buffers &b = m->b;
+  const int d = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim, F = c.ffn, L = c.n_layers;
+  const size_t plane = (size_t)m->max_tokens * dkv;          // elements of one K (or V) plane
+  T *kv = reinterpret_cast<T *>(m->kv);
+  T *h = (T *)b.h, *q = (T *)b.q, *attn = (T *)b.attn, *act = (T *)b.act;
+  int32_t rc;
+
+  { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_positions(b.cu, B, b.pos, b.last_idx, T_tok, st); }
+  { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_embed<T>((const T *)m->embed, b.tokens, b.x, T_tok, d, c.vocab, b.status, st); }
+
+  // one-time model transformation for this (l, g): fold each group leader's input-norm gain into its W_K, W_V
+  // and stack them (Sec. 3.5)
+  const int ng = n_groups(L, l, g);
+  if (l < L && (m->fold_l != l || m->fold_g != g)) {
+    for (int i = 0; i < ng; ++i) {
+      const swiftkv_layer_weights &lw = m->layers[l + i * g];
+      T *dst = (T *)b.wfold + (size_t)i * 2 * dkv * d;
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T>((const T *)lw.wk, (const T *)lw.in_norm, dst, dkv, d, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T>((const T *)lw.wv, (const T *)lw.in_norm, dst + (size_t)dkv * d, dkv, d, st); }
+    }
+    m->fold_l = l; m->fold_g = g;
+  }
+
+  // ---- layers 1..l on all prompt tokens (unmodified, Sec. 3.1)
+  for (int j = 0; j < l; ++j) {
+    const swiftkv_layer_weights &lw = m->layers[j];
+    T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
+    OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv};
+    rc = gemm_any<T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st);
+    if (rc) return rc;
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    {
+      Scope s(m, st, SWIFTKV_KC_ATTENTION);
+      bool done = false;
+      if constexpr (sizeof(T) == 2) {
+        if ((m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim)) {
+          rc = launch_attention_tc(q, Kj, Vj, attn, b.cu, B, T_tok, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
+          if (rc == SWIFTKV_OK) done = true;
+          else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
+        }
+      }
+      if (!done) launch_attention_simple<T>(q, Kj, Vj, attn, b.cu, B, b.pos, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
+    }
+    rc = gemm_any<T>(m, attn, T_tok, dq, (const T *)lw.wo, d, (const T *)nullptr, 0, (const T *)nullptr, 0,
+                     out_plain(OUT_RESID_ADD_F32, b.x, d, d), st);
+    if (rc) return rc;
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st); }
+    bool fused = false;
+    if constexpr (sizeof(T) == 2) {
+      if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d)) {
+        Scope s(m, st, SWIFTKV_KC_GEMM);
+        rc = launch_gemm_tc_swiglu(h, T_tok, d, (const bf16 *)lw.w_gate, (const bf16 *)lw.w_up, F, act, b.status, st);
+        if (rc == SWIFTKV_OK) fused = true;
+        else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "SwiGLU GEMM launch failed");
+      }
+    }
+    if (!fused) {
+      for (int r0 = 0; r0 < T_tok; r0 += MLP_CHUNK_ROWS) {
+        const int rows = std::min(MLP_CHUNK_ROWS, T_tok - r0);
+        rc = gemm_any<T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_gate, F, (const T *)nullptr, 0, (const T *)nullptr, 0,
+                         out_plain(OUT_STORE, b.gate, F, F), st);
+        if (rc) return rc;
+        rc = gemm_any<T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_up, F, (const T *)nullptr, 0, (const T *)nullptr, 0,
+                         out_plain(OUT_STORE, b.up, F, F), st);
+        if (rc) return rc;
+        Scope s(m, st, SWIFTKV_KC_ELEMWISE);
+        launch_swiglu<T>((const T *)b.gate, (const T *)b.up, act + (size_t)r0 * F, (long long)rows * F, st);
+      }
+    }
+    rc = gemm_any<T>(m, act, T_tok, F, (const T *)lw.w_down, d, (const T *)nullptr, 0, (const T *)nullptr, 0,
+                     out_plain(OUT_RESID_ADD_F32, b.x, d, d), st);
+    if (rc) return rc;
+  }
+
+  // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
+  if (l < L) {
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
+    T *slot_l = kv + (size_t)l * 2 * plane;
+    OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv};
+    rc = gemm_any<T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, (const T *)nullptr, 0, (const T *)nullptr, 0, o, st);
+    if (rc) return rc;
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+  }
+
+  // ---- the last token of each prompt continues through layers l+1..L (footnote of Sec. 3.2)
+  for (int r0 = 0; r0 < B; r0 += MAX_TAIL_ROWS) {
+    const int rows = std::min(MAX_TAIL_ROWS, B - r0);
+    T *hy = (T *)b.hy, *qy = (T *)b.qy, *ay = (T *)b.ay, *gy = (T *)b.gy, *uy = (T *)b.uy, *acty = (T *)b.acty;
+    float *y = b.y + (size_t)r0 * d;
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
+    for (int j = l; j < L; ++j) {
+      const swiftkv_layer_weights &lw = m->layers[j];
+      const int slot = l + (j - l) / g;
+      const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, rows, dq, d, out_plain(OUT_STORE, qy, dq, dq), st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<T>(qy, 0, 1, b.last_pos + r0, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.cu + r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, rows, d, dq, out_plain(OUT_RESID_ADD_F32, y, d, d), st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, rows, F, d, out_plain(OUT_STORE, gy, F, F), st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_up, rows, F, d, out_plain(OUT_STORE, uy, F, F), st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_swiglu<T>(gy, uy, acty, (long long)rows * F, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, rows, d, F, out_plain(OUT_RESID_ADD_F32, y, d, d), st); }
+    }
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)m->final_norm, hy, rows, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)m->lm_head, rows, c.vocab, d,
+                                                              out_plain(OUT_STORE_F32, b.logits + (size_t)r0 * c.vocab, c.vocab, c.vocab), st); }
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}
+
+static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool tokens_on_device, const int32_t *seq_lens,
+                              int32_t n_seqs, int32_t l, int32_t g, void *stream) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if (!tokens || !seq_lens) return fail(SWIFTKV_ERR_INVALID_ARG, "tokens / seq_lens is null");
+  const swiftkv_config &c = m->cfg;
+  if (l < 1 || l > c.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c.n_layers);
+  if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
+  if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
+  long long total = 0;
+  int max_len = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (seq_lens[i] < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "seq_lens[%d] = %d < 1", i, seq_lens[i]);
+    total += seq_lens[i];
+    max_len = std::max(max_len, seq_lens[i]);
+  }
+  if (total > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "%lld tokens > max_tokens %d", total, m->max_tokens);
+  if (!tokens_on_device)
+    for (long long t = 0; t < total; ++t)
+      if (tokens[t] < 0 || tokens[t] >= c.vocab) return fail(SWIFTKV_ERR_INVALID_ARG, "token %lld = %d outside [0, %d)", t, tokens[t], c.vocab);
+  if (l < c.n_layers && fold_elems_for(c, l, g) > m->fold_capacity_elems)
+    return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "workspace too small for the folded weight of (l=%d, g=%d)", l, g);
+  if (l + n_groups(c.n_layers, l, g) > m->slot_capacity)
+    return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "kv cache holds %d slots, (l=%d, g=%d) needs %d", m->slot_capacity, l, g,
+                l + n_groups(c.n_layers, l, g));
+  int dev = -1;
+  CUDA_TRY(cudaGetDevice(&dev));
+  if (dev != m->device) return fail(SWIFTKV_ERR_INVALID_ARG, "current device %d is not the model's device %d", dev, m->device);
+
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  m->ready = false;
+  m->launches = 0;
+  m->host_meta.resize(n_seqs + 1);
+  m->host_meta[0] = 0;
+  for (int i = 0; i < n_seqs; ++i) m->host_meta[i + 1] = m->host_meta[i] + seq_lens[i];
+  CUDA_TRY(cudaMemcpyAsync(m->b.cu, m->host_meta.data(), (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice, st));
+  std::vector<int32_t> lp(n_seqs);
+  for (int i = 0; i < n_seqs; ++i) lp[i] = seq_lens[i] - 1;
+  CUDA_TRY(cudaMemcpyAsync(m->b.last_pos, lp.data(), (size_t)n_seqs * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(m->b.tokens, tokens, (size_t)total * 4,
+                           tokens_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
+  int32_t rc = c.dtype == SWIFTKV_DTYPE_BF16 ? run_prefill<bf16>(m, (int)total, n_seqs, max_len, l, g, st)
+                                             : run_prefill<float>(m, (int)total, n_seqs, max_len, l, g, st);
+  if (rc) return rc;
+  m->n_tokens = (int)total; m->n_seqs = n_seqs; m->cur_l = l; m->cur_g = g; m->ready = true;
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_prefill(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                                   int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream) {
+  return prefill_common(m, tokens, false, seq_lens, n_seqs, swift_layer, acrosskv_group, cuda_stream);
+}
+extern "C" int32_t swiftkv_prefill_device_tokens(swiftkv_model *m, const int32_t *tokens_dev, const int32_t *seq_lens,
+                                                 int32_t n_seqs, int32_t swift_layer, int32_t acrosskv_group,
+                                                 void *cuda_stream) {
+  return prefill_common(m, tokens_dev, true, seq_lens, n_seqs, swift_layer, acrosskv_group, cuda_stream);
+}
+
+extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out) {
+  if (!m || !out) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (layer < 0 || layer >= m->cfg.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, m->cfg.n_layers);
+  if (!m->ready) return fail(SWIFTKV_ERR_NOT_READY, "no prefill has been run");
+  const int l = m->cur_l, g = m->cur_g;
+  const int dkv = m->cfg.n_kv_heads * m->cfg.head_dim;
+  const size_t plane = (size_t)m->max_tokens * dkv;
+  int slot = layer, owner = layer;
+  if (layer >= l) { slot = l + (layer - l) / g; owner = l + ((layer - l) / g) * g; }
+  const uint8_t *kp = m->kv + (size_t)slot * 2 * plane * m->esize;
+  out->k = kp;
+  out->v = kp + plane * m->esize;
+  out->token_stride = dkv;
+  out->head_stride = m->cfg.head_dim;
+  out->n_tokens = m->n_tokens;
+  out->dtype = m->cfg.dtype;
+  out->owner_layer = owner;
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_first_logits(const swiftkv_model *m, const float **logits, int32_t *n_seqs) {
+  if (!m || !logits) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (!m->ready) return fail(SWIFTKV_ERR_NOT_READY, "no prefill has been run");
+  *logits = m->b.logits;
+  if (n_seqs) *n_seqs = m->n_seqs;
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_status(swiftkv_model *m, void *cuda_stream) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  unsigned int word = 0;
+  CUDA_TRY(cudaMemcpyAsync(&word, m->b.status, 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemsetAsync(m->b.status, 0, 4, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (word & STATUS_TIMEOUT) return fail(SWIFTKV_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel ran out");
+  if (word & STATUS_BAD_TOKEN) return fail(SWIFTKV_ERR_BAD_TOKEN, "a token id outside [0, vocab) was clamped");
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_profile_enable(swiftkv_model *m, int32_t on) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  m->profiling = on != 0;
+  return SWIFTKV_OK;
+}
+extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, float *ms, int32_t *launches) {
+  if (!m || !ms || !launches) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  CUDA_TRY(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
+  for (int i = 0; i < SWIFTKV_KC_COUNT; ++i) { ms[i] = 0.f; launches[i] = 0; }
+  for (auto &r : m->recs) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) { ms[r.cls] += t; launches[r.cls] += 1; }
+    m->pool.push_back(r.a);
+    m->pool.push_back(r.b);
+  }
+  m->recs.clear();
+  return SWIFTKV_OK;
+}
+extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
+extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
+  if (!m) return 0;
+  m->kernel_mask = mask & 3;
+  return m->kernel_mask;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// stand-alone operators
+// ---------------------------------------------------------------------------------------------------------
+// a device word for the stand-alone entry points' bounded waits
+static __device__ unsigned int g_op_status[64];
+static unsigned int *op_status_word() {
+  static unsigned int *ptr = nullptr;
+  if (!ptr) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_op_status) == cudaSuccess) ptr = reinterpret_cast<unsigned int *>(p);
+  }
+  return ptr;
+}
+
+extern "C" int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
+                                     void *cuda_stream) {
+  if (!A || !B || !C || M < 1 || N < 1 || K < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "bad argument");
+  if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15) return fail(SWIFTKV_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  if (!tc_gemm_supported(M, N, K)) return fail(SWIFTKV_ERR_UNSUPPORTED, "needs K %% 64 == 0 and N %% 128 == 0");
+  unsigned int *status = op_status_word();
+  if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+  int rc = launch_gemm_tc((const bf16 *)A, M, K, (const bf16 *)B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N),
+                          status, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, void *out,
+                                             const int32_t *cu_seqlens, int32_t n_seqs, int32_t total_tokens,
+                                             int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                             int32_t head_dim, int32_t dtype, int32_t use_tensor_cores,
+                                             void *cuda_stream) {
+  if (!q || !k || !v || !out || !cu_seqlens) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (n_seqs < 1 || total_tokens < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || head_dim < 2 || head_dim > 256)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "bad shape");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (use_tensor_cores) {
+    if (dtype != SWIFTKV_DTYPE_BF16 || !tc_attention_supported(n_q_heads, n_kv_heads, head_dim))
+      return fail(SWIFTKV_ERR_UNSUPPORTED, "tensor-core attention needs bf16 and head_dim 128");
+    unsigned int *status = op_status_word();
+    if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+    int rc = launch_attention_tc((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs,
+                                 total_tokens, max_seq_len, n_q_heads, n_kv_heads, head_dim, status, st);
+    if (rc) return fail(rc, "attention launch failed");
+    return SWIFTKV_OK;
+  }
+  if (dtype == SWIFTKV_DTYPE_BF16)
+    launch_attention_simple<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr,
+                                  total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+  else if (dtype == SWIFTKV_DTYPE_F32)
+    launch_attention_simple<float>((const float *)q, (const float *)k, (const float *)v, (float *)out, cu_seqlens, n_seqs,
+                                   nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+  else
+    return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}

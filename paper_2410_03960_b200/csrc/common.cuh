@@ -1,0 +1,130 @@
+// Shared declarations of the SwiftKV prefill library (host + device helpers, launch prototypes).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/swiftkv.h"
+
+namespace skv {
+
+// ---- device status word -------------------------------------------------------------------------------
+// Kernels never trap: a bounded wait that runs out, or a bad token id, sets a bit here and carries on.
+enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BAD_TOKEN = 2u };
+
+// ---- element types ---------------------------------------------------------------------------------------
+using bf16 = __nv_bfloat16;
+
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ---- where a GEMM writes its result ----------------------------------------------------------------------
+// Columns [0, n0) go to p0 (row stride ld0).  Columns >= n0 are cut into segments of seg_w columns; segment i
+// goes to seg_base + i*seg_stride (row stride seg_w): this is how one projection lands directly in the
+// K / V planes of the cache (QKV projection of a layer, and the fused SingleInputKV projection of Sec. 3.5).
+enum OutMode : int { OUT_STORE = 0, OUT_RESID_ADD_F32 = 1, OUT_STORE_F32 = 2 };
+struct OutDesc {
+  int mode;
+  void *p0;
+  long long ld0;
+  int n0;
+  void *seg_base;
+  long long seg_stride;   // elements
+  int seg_w;
+};
+inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDesc{mode, p, ld, n, nullptr, 0, 1}; }
+
+#ifdef __CUDACC__
+// write one fp32 accumulator where the descriptor says (device side)
+template <typename T>
+__device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, float acc) {
+  if (o.mode == OUT_RESID_ADD_F32) {
+    float *p = reinterpret_cast<float *>(o.p0) + (size_t)row * o.ld0 + col;
+    *p += acc;
+  } else if (o.mode == OUT_STORE_F32) {
+    reinterpret_cast<float *>(o.p0)[(size_t)row * o.ld0 + col] = acc;
+  } else if (col < o.n0) {
+    reinterpret_cast<T *>(o.p0)[(size_t)row * o.ld0 + col] = from_f<T>(acc);
+  } else {
+    const int c = col - o.n0;
+    const int seg = c / o.seg_w, within = c % o.seg_w;
+    reinterpret_cast<T *>(o.seg_base)[(size_t)seg * o.seg_stride + (size_t)row * o.seg_w + within] = from_f<T>(acc);
+  }
+}
+#endif
+
+// ---- launch prototypes (each queues work on `st`, no synchronisation) -------------------------------------
+// elementwise.cu
+template <typename T>
+void launch_embed(const T *embed, const int32_t *tokens, float *x, int n_tokens, int d, int vocab,
+                  unsigned int *status, cudaStream_t st);
+void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions, int32_t *last_idx, int n_tokens,
+                      cudaStream_t st);
+// y = x * rsqrt(mean(x^2)+eps) * gamma (gamma may be null: unit-rms only).  x fp32 [rows, d] -> out T [rows, d]
+template <typename T>
+void launch_rmsnorm(const float *x, const T *gamma, T *out, int rows, int d, float eps, cudaStream_t st);
+// in-place rotary embedding on `n_batches` tensors [rows, n_heads, hd] spaced batch_stride elements apart
+template <typename T>
+void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const float *cos_tab,
+                 const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st);
+template <typename T>
+void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
+void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
+void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, double theta, cudaStream_t st);
+// dst[r, c] = w[r, c] * gamma[c]   (gain of the input norm folded into a projection weight, Sec. 3.5)
+template <typename T>
+void launch_fold(const T *w, const T *gamma, T *dst, int rows, int cols, cudaStream_t st);
+
+// gemm_simt.cu : C = A[M,K] * B[N,K]^T with fp32 accumulation, any shape; result column c is written as
+// column col0 + c of `out`
+template <typename T>
+void launch_gemm_simt(const T *A, const T *B, int M, int N, int K, OutDesc out, int col0, cudaStream_t st);
+
+// gemm_tc.cu : tcgen05 / TMEM / TMA GEMMs (bf16)
+struct TcGemmPlan;   // host object holding tensor maps
+bool tc_gemm_supported(int M, int N, int K);
+// generic: B rows come from up to three matrices stacked along N: [0,nB0) from B0, [nB0, nB0+nB1) from B1, rest B2
+int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
+                   int nB2, OutDesc out, unsigned int *status, cudaStream_t st);
+// act[M, F] = silu(A Wg^T) * (A Wu^T), gate/up tiles paired inside one CTA tile
+int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
+                          unsigned int *status, cudaStream_t st);
+bool tc_swiglu_supported(int M, int F, int K);
+
+// attention.cu
+template <typename T>
+void launch_attention_simple(const T *q, const T *k, const T *v, T *out, const int32_t *cu_seqlens, int n_seqs,
+                             const int32_t *positions /* may be null */, int n_tokens, int n_q, int n_kv, int hd,
+                             cudaStream_t st);
+bool tc_attention_supported(int n_q, int n_kv, int hd);
+int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, const int32_t *cu_seqlens,
+                        int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd,
+                        unsigned int *status, cudaStream_t st);
+
+// tail.cu : the last-token path (M = n_seqs <= 8 rows)
+// out[b, n] (+)= sum_k act[b, k] * W[n, k]
+template <typename T>
+void launch_skinny_gemm(const T *act, const T *W, int n_rows, int N, int K, OutDesc out, cudaStream_t st);
+// one query token per prompt against that prompt's cache rows [cu[b], cu[b+1]); scratch holds split partials
+size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
+constexpr int MAX_TAIL_ROWS = 8;   // rows one skinny-GEMM launch handles
+template <typename T>
+void launch_tail_attention(const T *q, const T *kc, const T *vc, T *out, const int32_t *cu_seqlens, int n_seqs,
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
+
+}  // namespace skv

@@ -1,0 +1,242 @@
+// Memory-bound kernels of the SwiftKV prefill path: embedding gather, RMSNorm, rotary embedding, SwiGLU,
+// last-token gather, RoPE table, and the one-time gain fold of the SingleInputKV weight (Sec. 3.5).
+// All use 128-bit global accesses where the row length allows and warp-shuffle reductions.
+#include "common.cuh"
+
+namespace skv {
+
+// ---------------------------------------------------------------------------------------------------------
+// embedding gather: x[t, :] = float(E[tok[t], :])      (Sec. 3.1: X are the input embeddings)
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_kernel(const T *__restrict__ embed, const int32_t *__restrict__ tokens, float *__restrict__ x,
+                             int d, int vocab, unsigned int *status) {
+  const int t = blockIdx.x;
+  int id = tokens[t];
+  if (id < 0 || id >= vocab) {
+    if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_TOKEN);
+    id = min(max(id, 0), vocab - 1);
+  }
+  const T *src = embed + (size_t)id * d;
+  float *dst = x + (size_t)t * d;
+  if constexpr (sizeof(T) == 2) {
+    if ((d & 7) == 0) {
+      for (int i = threadIdx.x * 8; i < d; i += blockDim.x * 8) {
+        uint4 raw = *reinterpret_cast<const uint4 *>(src + i);
+        const bf16 *e = reinterpret_cast<const bf16 *>(&raw);
+        float4 a = make_float4(to_f(e[0]), to_f(e[1]), to_f(e[2]), to_f(e[3]));
+        float4 b = make_float4(to_f(e[4]), to_f(e[5]), to_f(e[6]), to_f(e[7]));
+        *reinterpret_cast<float4 *>(dst + i) = a;
+        *reinterpret_cast<float4 *>(dst + i + 4) = b;
+      }
+      return;
+    }
+  }
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = to_f(src[i]);
+}
+
+template <typename T>
+void launch_embed(const T *embed, const int32_t *tokens, float *x, int n_tokens, int d, int vocab,
+                  unsigned int *status, cudaStream_t st) {
+  if (n_tokens <= 0) return;
+  embed_kernel<T><<<n_tokens, 128, 0, st>>>(embed, tokens, x, d, vocab, status);
+}
+template void launch_embed<float>(const float *, const int32_t *, float *, int, int, int, unsigned int *, cudaStream_t);
+template void launch_embed<bf16>(const bf16 *, const int32_t *, float *, int, int, int, unsigned int *, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------------------
+// positions[t] = t - cu_seqlens[b(t)]  (positions restart at 0 for each prompt); last_idx[b] = cu[b+1]-1
+// ---------------------------------------------------------------------------------------------------------
+__global__ void positions_kernel(const int32_t *__restrict__ cu, int n_seqs, int32_t *__restrict__ pos,
+                                 int32_t *__restrict__ last_idx, int n_tokens) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n_seqs) last_idx[t] = cu[t + 1] - 1;
+  if (t >= n_tokens) return;
+  int lo = 0, hi = n_seqs;   // find b with cu[b] <= t < cu[b+1]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
+  }
+  pos[t] = t - cu[lo];
+}
+void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions, int32_t *last_idx, int n_tokens,
+                      cudaStream_t st) {
+  const int n = n_tokens > n_seqs ? n_tokens : n_seqs;
+  positions_kernel<<<(n + 255) / 256, 256, 0, st>>>(cu_seqlens, n_seqs, positions, last_idx, n_tokens);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// RMSNorm: out = x / sqrt(mean(x^2) + eps) * gamma, one block per row, fp32 statistics.
+// The residual stream x is fp32; the output is the model dtype.  gamma == nullptr gives the unit-rms row that
+// feeds the gain-folded SingleInputKV projection (one statistic shared by every later layer).
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ gamma,
+                                                      T *__restrict__ out, int d, float eps) {
+  const size_t row = blockIdx.x;
+  const float *xr = x + row * d;
+  T *orow = out + row * d;
+  __shared__ float red[8];
+  float ss = 0.f;
+  const bool vec = (d & 3) == 0;
+  if (vec) {
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+      const float4 v = *reinterpret_cast<const float4 *>(xr + i);
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  } else {
+    for (int i = threadIdx.x; i < d; i += blockDim.x) ss += xr[i] * xr[i];
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += (w < (blockDim.x >> 5)) ? red[w] : 0.f;
+  const float rstd = rsqrtf(tot / (float)d + eps);
+  if (vec) {
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+      const float4 v = *reinterpret_cast<const float4 *>(xr + i);   // second read hits L1/L2
+      float g0 = 1.f, g1 = 1.f, g2 = 1.f, g3 = 1.f;
+      if (gamma) { g0 = to_f(gamma[i]); g1 = to_f(gamma[i + 1]); g2 = to_f(gamma[i + 2]); g3 = to_f(gamma[i + 3]); }
+      if constexpr (sizeof(T) == 2) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x * rstd * g0, v.y * rstd * g1);
+        __nv_bfloat162 b = __floats2bfloat162_rn(v.z * rstd * g2, v.w * rstd * g3);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t *>(&a);
+        pk.y = *reinterpret_cast<uint32_t *>(&b);
+        *reinterpret_cast<uint2 *>(orow + i) = pk;
+      } else {
+        *reinterpret_cast<float4 *>(orow + i) = make_float4(v.x * rstd * g0, v.y * rstd * g1, v.z * rstd * g2, v.w * rstd * g3);
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < d; i += blockDim.x)
+      orow[i] = from_f<T>(xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f));
+  }
+}
+template <typename T>
+void launch_rmsnorm(const float *x, const T *gamma, T *out, int rows, int d, float eps, cudaStream_t st) {
+  if (rows <= 0) return;
+  rmsnorm_kernel<T><<<rows, 256, 0, st>>>(x, gamma, out, d, eps);
+}
+template void launch_rmsnorm<float>(const float *, const float *, float *, int, int, float, cudaStream_t);
+template void launch_rmsnorm<bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------------------
+// Rotary embedding, rotate-half pairing (i, i + hd/2), in place.  One thread per pair.
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rope_kernel(T *__restrict__ x, long long batch_stride, const int32_t *__restrict__ positions,
+                            const float *__restrict__ cos_tab, const float *__restrict__ sin_tab, int rows,
+                            int n_heads, int hd) {
+  const int half = hd >> 1;
+  const long long per_row = (long long)n_heads * half;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= per_row * rows) return;
+  const int row = (int)(idx / per_row);
+  const int rem = (int)(idx % per_row);
+  const int h = rem / half, i = rem % half;
+  const int p = positions[row];
+  const float c = cos_tab[(size_t)p * half + i], s = sin_tab[(size_t)p * half + i];
+  T *base = x + (size_t)blockIdx.y * batch_stride + ((size_t)row * n_heads + h) * hd;
+  const float a = to_f(base[i]), b = to_f(base[i + half]);
+  base[i] = from_f<T>(a * c - b * s);
+  base[i + half] = from_f<T>(b * c + a * s);
+}
+template <typename T>
+void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const float *cos_tab,
+                 const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st) {
+  const long long n = (long long)rows * n_heads * (hd / 2);
+  if (n <= 0 || n_batches <= 0) return;
+  dim3 grid((unsigned)((n + 255) / 256), (unsigned)n_batches);
+  rope_kernel<T><<<grid, 256, 0, st>>>(x, batch_stride, positions, cos_tab, sin_tab, rows, n_heads, hd);
+}
+template void launch_rope<float>(float *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+
+// cos/sin of p * theta^(-2i/hd), evaluated in double precision and rounded once to fp32.
+__global__ void rope_table_kernel(float *cos_tab, float *sin_tab, int max_pos, int half, double log_theta, int hd) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)max_pos * half) return;
+  const int p = (int)(idx / half), i = (int)(idx % half);
+  const double inv_freq = exp(-2.0 * (double)i / (double)hd * log_theta);
+  double s, c;
+  sincos((double)p * inv_freq, &s, &c);
+  cos_tab[idx] = (float)c;
+  sin_tab[idx] = (float)s;
+}
+void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, double theta, cudaStream_t st) {
+  const long long n = (long long)max_pos * (hd / 2);
+  if (n <= 0) return;
+  rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(cos_tab, sin_tab, max_pos, hd / 2, log(theta), hd);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// SwiGLU: out = silu(gate) * up      (Sec. 3.1 MLP; fp32 arithmetic, model-dtype storage)
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void swiglu_kernel(const T *__restrict__ gate, const T *__restrict__ up, T *__restrict__ out, long long n) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  constexpr int V = 16 / sizeof(T);
+  const long long nv = n / V;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += stride) {
+    uint4 g = reinterpret_cast<const uint4 *>(gate)[i];
+    uint4 u = reinterpret_cast<const uint4 *>(up)[i];
+    uint4 o;
+    const T *ge = reinterpret_cast<const T *>(&g);
+    const T *ue = reinterpret_cast<const T *>(&u);
+    T *oe = reinterpret_cast<T *>(&o);
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+      const float z = to_f(ge[k]);
+      oe[k] = from_f<T>(z / (1.f + __expf(-z)) * to_f(ue[k]));
+    }
+    reinterpret_cast<uint4 *>(out)[i] = o;
+  }
+  for (long long i = nv * V + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float z = to_f(gate[i]);
+    out[i] = from_f<T>(z / (1.f + __expf(-z)) * to_f(up[i]));
+  }
+}
+template <typename T>
+void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st) {
+  if (n <= 0) return;
+  long long blocks = (n / (16 / sizeof(T)) + 255) / 256;
+  if (blocks < 1) blocks = 1;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  swiglu_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(gate, up, out, n);
+}
+template void launch_swiglu<float>(const float *, const float *, float *, long long, cudaStream_t);
+template void launch_swiglu<bf16>(const bf16 *, const bf16 *, bf16 *, long long, cudaStream_t);
+
+// y[b, :] = x[idx[b], :]   (the tokens that continue past layer l: the last token of each prompt)
+__global__ void gather_rows_kernel(const float *__restrict__ x, const int32_t *__restrict__ idx, float *__restrict__ y, int d) {
+  const float *src = x + (size_t)idx[blockIdx.x] * d;
+  float *dst = y + (size_t)blockIdx.x * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+}
+void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st) {
+  if (n_rows <= 0) return;
+  gather_rows_kernel<<<n_rows, 256, 0, st>>>(x, idx, y, d);
+}
+
+// dst[r, c] = w[r, c] * gamma[c], product in fp32, one rounding to the model dtype
+template <typename T>
+__global__ void fold_kernel(const T *__restrict__ w, const T *__restrict__ gamma, T *__restrict__ dst, long long n, int cols) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    dst[i] = from_f<T>(to_f(w[i]) * to_f(gamma[i % cols]));
+}
+template <typename T>
+void launch_fold(const T *w, const T *gamma, T *dst, int rows, int cols, cudaStream_t st) {
+  const long long n = (long long)rows * cols;
+  if (n <= 0) return;
+  long long blocks = (n + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  fold_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(w, gamma, dst, n, cols);
+}
+template void launch_fold<float>(const float *, const float *, float *, int, int, cudaStream_t);
+template void launch_fold<bf16>(const bf16 *, const bf16 *, bf16 *, int, int, cudaStream_t);
+
+}  // namespace skv

@@ -1,0 +1,404 @@
+// bf16 GEMMs of the prefill path on the 5th-generation tensor cores: C = A[M,K] * B[N,K]^T, fp32 accumulation.
+//
+// One persistent CTA per SM, 192 threads in three roles:
+//   warp 0      : TMA producer -- streams 128x64 A tiles and BNx64 B tiles (128-byte swizzle) through a
+//                 shared-memory ring guarded by full/empty mbarriers;
+//   warp 1      : MMA issuer -- one thread issues tcgen05.mma (128 x BN x 16 per instruction) into one of two
+//                 tensor-memory accumulators and commits ring slots / accumulators back through mbarriers;
+//   warps 2..5  : epilogue -- read the finished accumulator from tensor memory (tcgen05.ld, one row per
+//                 thread), apply the fused epilogue and write to global memory while the MMA warp already
+//                 works on the next tile in the other accumulator.
+// Epilogues: store bf16 (optionally scattered into K/V cache planes), accumulate into the fp32 residual
+// stream, or SwiGLU with the gate and up tiles of the same features side by side in one accumulator.
+// Every mbarrier wait is bounded: on timeout the kernel sets a status bit and every role leaves its loop.
+#include <mutex>
+#include <unordered_map>
+
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace skv {
+
+// ---------------------------------------------------------------------------------------------------------
+// host: tensor-map encoding through the driver entry point (no link-time dependency on libcuda)
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
+                      uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return -1;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -2;
+}
+int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1,
+                      uint64_t s2, uint32_t b0, uint32_t b1) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return -1;
+  cuuint64_t dims[3] = {d0, d1, d2};
+  cuuint64_t strides[2] = {s1 * 2, s2 * 2};
+  cuuint32_t box[3] = {b0, b1, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -2;
+}
+
+namespace {
+
+// tensor maps are pure functions of (pointer, shape, box): cache them
+struct TmapKey {
+  const void *p; uint64_t rows, cols, ld; uint32_t br, bc;
+  bool operator==(const TmapKey &o) const { return p == o.p && rows == o.rows && cols == o.cols && ld == o.ld && br == o.br && bc == o.bc; }
+};
+struct TmapKeyHash {
+  size_t operator()(const TmapKey &k) const {
+    size_t h = reinterpret_cast<size_t>(k.p);
+    h = h * 1000003u ^ k.rows; h = h * 1000003u ^ k.cols; h = h * 1000003u ^ k.ld; h = h * 1000003u ^ (k.br * 1024u + k.bc);
+    return h;
+  }
+};
+std::mutex g_tmap_mu;
+std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> g_tmaps;
+
+int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t br, uint32_t bc) {
+  TmapKey k{p, rows, cols, ld, br, bc};
+  std::lock_guard<std::mutex> g(g_tmap_mu);
+  auto it = g_tmaps.find(k);
+  if (it != g_tmaps.end()) { *out = it->second; return 0; }
+  if (g_tmaps.size() > 65536) g_tmaps.clear();
+  CUtensorMap m;
+  int rc = make_tmap_2d_bf16(&m, p, rows, cols, ld, br, bc);
+  if (rc) return rc;
+  g_tmaps.emplace(k, m);
+  *out = m;
+  return 0;
+}
+
+int num_sms() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// device
+// ---------------------------------------------------------------------------------------------------------
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
+constexpr int GEMM_THREADS = 192;
+constexpr int GROUP_M = 16;   // tile rasterisation: bands of 16 row-blocks, column-blocks outer, rows inner
+
+struct GemmTcParams {
+  int M, N, K;
+  int nB0, nB1;          // columns [0,nB0) from B0, [nB0,nB0+nB1) from B1, rest from B2
+  int num_m_blocks, num_n_blocks;
+  OutDesc out;
+  bf16 *act;             // SwiGLU output [M, F]
+  int F;
+  unsigned int *status;
+};
+
+template <int BN, int STAGES>
+struct SmemLayout {
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+  static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
+};
+
+__device__ __forceinline__ void tile_coords(int tile, int num_m_blocks, int num_n_blocks, int &m_blk, int &n_blk) {
+  const int band_tiles = GROUP_M * num_n_blocks;
+  const int band = tile / band_tiles;
+  const int r = tile - band * band_tiles;
+  const int band_h = min(GROUP_M, num_m_blocks - band * GROUP_M);
+  n_blk = r / band_h;
+  m_blk = band * GROUP_M + (r - n_blk * band_h);
+}
+
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
+  if (tc::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!tc::mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > tc::WAIT_LIMIT_CLOCKS) {
+      *abort_flag = 1;
+      atomicOr(status, STATUS_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+
+template <int BN, int STAGES, bool SWIGLU>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmTcParams p) {
+  using L = SmemLayout<BN, STAGES>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET);
+  uint64_t *full_bar = bars;                  // [STAGES]
+  uint64_t *empty_bar = bars + STAGES;        // [STAGES]
+  uint64_t *tfull_bar = bars + 2 * STAGES;    // [2]
+  uint64_t *tempty_bar = bars + 2 * STAGES + 2;   // [2]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 4);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr uint32_t TMEM_COLS = 2 * BN;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { tc::mbar_init(tc::smem_u32(&full_bar[s]), 1); tc::mbar_init(tc::smem_u32(&empty_bar[s]), 1); }
+    for (int a = 0; a < 2; ++a) { tc::mbar_init(tc::smem_u32(&tfull_bar[a]), 1); tc::mbar_init(tc::smem_u32(&tempty_bar[a]), 4); }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmA);
+    tc::tma_prefetch_desc(&tmB0);
+  }
+  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), TMEM_COLS);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_tiles = p.num_m_blocks * p.num_n_blocks;
+  const int num_kb = p.K / BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------ TMA producer
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int m_blk, n_blk;
+        tile_coords(tile, p.num_m_blocks, p.num_n_blocks, m_blk, n_blk);
+        const CUtensorMap *tb = &tmB0;
+        int b_row = n_blk * BN;
+        if constexpr (SWIGLU) {
+          b_row = n_blk * (BN / 2);
+        } else {
+          if (b_row >= p.nB0 + p.nB1) { tb = &tmB2; b_row -= p.nB0 + p.nB1; }
+          else if (b_row >= p.nB0) { tb = &tmB1; b_row -= p.nB0; }
+        }
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!wait_or_abort(tc::smem_u32(&empty_bar[stage]), phase ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t fb = tc::smem_u32(&full_bar[stage]);
+          uint8_t *sa = smem + stage * L::STAGE_BYTES;
+          uint8_t *sb = sa + L::A_BYTES;
+          tc::mbar_expect_tx(fb, L::STAGE_BYTES);
+          tc::tma_load_2d(tc::smem_u32(sa), &tmA, fb, kb * BK, m_blk * BM);
+          if constexpr (SWIGLU) {
+            tc::tma_load_2d(tc::smem_u32(sb), &tmB0, fb, kb * BK, b_row);                     // gate rows
+            tc::tma_load_2d(tc::smem_u32(sb + L::B_BYTES / 2), &tmB1, fb, kb * BK, b_row);   // up rows
+          } else {
+            tc::tma_load_2d(tc::smem_u32(sb), tb, fb, kb * BK, b_row);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------ MMA issuer
+      constexpr uint32_t idesc = tc::umma_idesc_bf16(BM, BN, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1;
+        if (!wait_or_abort(tc::smem_u32(&tempty_bar[acc]), acc_phase ^ 1, abort_flag, p.status)) break;
+        tc::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!wait_or_abort(tc::smem_u32(&full_bar[stage]), phase, abort_flag, p.status)) { ok = false; break; }
+          tc::tc_fence_after_sync();
+          const uint32_t a_addr = tc::smem_u32(smem + stage * L::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + L::A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = tc::umma_desc_sw128(a_addr + k * UMMA_K * 2, 16, 1024);
+            const uint64_t bd = tc::umma_desc_sw128(b_addr + k * UMMA_K * 2, 16, 1024);
+            tc::umma_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc::umma_commit(tc::smem_u32(&empty_bar[stage]));   // frees the ring slot when these MMAs retire
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) tc::umma_commit(tc::smem_u32(&tfull_bar[acc]));   // accumulator complete
+      }
+    }
+  } else {
+    // -------------------------------------------------- epilogue warps (2..5)
+    const int quarter = warp & 3;   // the TMEM lane quarter this warp may read
+    int it = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+      int m_blk, n_blk;
+      tile_coords(tile, p.num_m_blocks, p.num_n_blocks, m_blk, n_blk);
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1;
+      if (!wait_or_abort(tc::smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, p.status)) break;
+      tc::tc_fence_after_sync();
+      const int row = m_blk * BM + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+      if constexpr (SWIGLU) {
+        constexpr int HALF = BN / 2;
+#pragma unroll 1
+        for (int c = 0; c < HALF / 32; ++c) {
+          uint32_t g[32], u[32];
+          tc::tmem_ld_32x32b_x32(t_row + c * 32, g);
+          tc::tmem_ld_32x32b_x32(t_row + HALF + c * 32, u);
+          tc::tmem_ld_wait();
+          if (row < p.M) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+              const float u0 = __uint_as_float(u[2 * i]), u1 = __uint_as_float(u[2 * i + 1]);
+              pk[i] = tc::pack_bf16x2(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+            }
+            uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * p.F + (size_t)n_blk * HALF + c * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld_32x32b_x32(t_row + c * 32, r);
+          tc::tmem_ld_wait();
+          if (row < p.M) {
+            const int col = n_blk * BN + c * 32;
+            if (p.out.mode == OUT_RESID_ADD_F32) {
+              float4 *px = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.out.p0) + (size_t)row * p.out.ld0 + col);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                float4 v = px[i];
+                v.x += __uint_as_float(r[4 * i]); v.y += __uint_as_float(r[4 * i + 1]);
+                v.z += __uint_as_float(r[4 * i + 2]); v.w += __uint_as_float(r[4 * i + 3]);
+                px[i] = v;
+              }
+            } else {
+              bf16 *dstp;
+              if (col < p.out.n0) {
+                dstp = reinterpret_cast<bf16 *>(p.out.p0) + (size_t)row * p.out.ld0 + col;
+              } else {
+                const int cc = col - p.out.n0;
+                const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
+                dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + (size_t)row * p.out.seg_w + within;
+              }
+              uint4 *dst = reinterpret_cast<uint4 *>(dstp);
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                dst[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1])),
+                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3])),
+                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5])),
+                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])));
+            }
+          }
+        }
+      }
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(tc::smem_u32(&tempty_bar[acc]));
+    }
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int BN, int STAGES, bool SWIGLU>
+int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const CUtensorMap &b2,
+               const GemmTcParams &p, cudaStream_t st) {
+  using L = SmemLayout<BN, STAGES>;
+  auto kern = gemm_tc_kernel<BN, STAGES, SWIGLU>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess) return SWIFTKV_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = p.num_m_blocks * p.num_n_blocks;
+  const int grid = tiles < num_sms() ? tiles : num_sms();
+  kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(a, b0, b1, b2, p);
+  return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+}
+
+}  // namespace
+
+bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (N % 128) == 0 && N >= 128; }
+bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
+
+int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
+                   int nB2, OutDesc out, unsigned int *status, cudaStream_t st) {
+  const int N = nB0 + nB1 + nB2;
+  if (!tc_gemm_supported(M, N, K)) return SWIFTKV_ERR_UNSUPPORTED;
+  if (out.mode == OUT_STORE_F32) return SWIFTKV_ERR_UNSUPPORTED;
+  int BN = 256;
+  if ((N % 256) || (nB1 + nB2 > 0 && ((nB0 % 256) || (nB1 % 256)))) BN = 128;
+  if (nB1 + nB2 > 0 && ((nB0 % BN) || (nB1 % BN))) return SWIFTKV_ERR_UNSUPPORTED;
+  if (out.mode == OUT_STORE && ((out.n0 % 32) || (out.n0 < N && (out.seg_w % 32)))) return SWIFTKV_ERR_UNSUPPORTED;
+  CUtensorMap ta, tb0, tb1, tb2;
+  if (get_tmap(&ta, A, M, K, K, BM, BK)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tb0, B0, nB0, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
+  tb1 = tb0; tb2 = tb0;
+  if (nB1 > 0 && get_tmap(&tb1, B1, nB1, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
+  if (nB2 > 0 && get_tmap(&tb2, B2, nB2, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
+  GemmTcParams p{};
+  p.M = M; p.N = N; p.K = K; p.nB0 = nB0; p.nB1 = nB1;
+  p.num_m_blocks = (M + BM - 1) / BM;
+  p.num_n_blocks = N / BN;
+  p.out = out; p.act = nullptr; p.F = 0; p.status = status;
+  if (BN == 256) return launch_cfg<256, 4, false>(ta, tb0, tb1, tb2, p, st);
+  return launch_cfg<128, 6, false>(ta, tb0, tb1, tb2, p, st);
+}
+
+int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
+                          unsigned int *status, cudaStream_t st) {
+  if (!tc_swiglu_supported(M, F, K)) return SWIFTKV_ERR_UNSUPPORTED;
+  CUtensorMap ta, tg, tu;
+  if (get_tmap(&ta, A, M, K, K, BM, BK)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tg, Wg, F, K, K, 128, BK)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tu, Wu, F, K, K, 128, BK)) return SWIFTKV_ERR_CUDA;
+  GemmTcParams p{};
+  p.M = M; p.N = 2 * F; p.K = K; p.nB0 = F; p.nB1 = F;
+  p.num_m_blocks = (M + BM - 1) / BM;
+  p.num_n_blocks = F / 128;
+  p.out = OutDesc{}; p.act = act; p.F = F; p.status = status;
+  return launch_cfg<256, 4, true>(ta, tg, tu, tu, p, st);
+}
+
+}  // namespace skv

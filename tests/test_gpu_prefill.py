@@ -1,0 +1,124 @@
+"""End-to-end parity of the CUDA prefill (through the C ABI) with the CPU oracle: every layer's K / V cache and
+the first-token logits, element by element, on the same seeded inputs.
+
+Bars: fp32 model -- rel-L2 <= 1e-4 on every tensor; bf16 model -- rel-L2 <= 2e-2 per tensor and max-abs logit
+error <= 0.1 (bf16 storage between kernels, fp32 accumulation and fp32 residual stream).
+"""
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as S
+from oracle import swiftkv_oracle as O
+from helpers import check_prefill_against_oracle, oracle_config, oracle_weights, rel_l2, to_np
+
+pytestmark = pytest.mark.gpu
+
+# a shape every tensor-core kernel tiles (K % 64 == 0, N % 256 == 0, head_dim 128) yet small enough for the oracle
+MID = S.ModelShape(1024, 512, 4, 8, 2, 128, 1024, 500000.0, 1e-5, "mid")
+# Llama-3.1-8B widths with a reduced depth (the oracle stays within a minute)
+W8B_4L = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-width-4-layers")
+
+
+def _run(shape, dtype, seed, lens, l, g, max_tokens=None, kernel_mask=None):
+    import paper_2410_03960_b200 as P
+    w = S.make_weights(shape, seed, dtype, "cuda")
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, dtype, max_tokens or sum(lens), len(lens), l, g)
+    if kernel_mask is not None:
+        model.set_kernel_mask(kernel_mask)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    ref = O.swiftkv(oracle_config(shape), oracle_weights(w), tok.numpy(), lens, l, g)
+    return model, ref, w, tok
+
+
+@pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 1), (1, 2), (2, 2), (3, 1), (1, 3)])
+def test_config1_fp32(l, g):
+    """Config 1: tiny Llama-style decoder, fp32 weights, prompts of 128 and 96 tokens (l = 2, g = 1 is the
+    named point; l = 4 is the unmodified model; the rest cover AcrossKV incl. a short last group)."""
+    model, ref, _, _ = _run(S.TINY, torch.float32, 0, [128, 96], l, g)
+    check_prefill_against_oracle(model, ref, S.TINY.n_layers, 1e-4, 1e-4, 1e-3)
+
+
+@pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2)])
+def test_config1_bf16(l, g):
+    model, ref, _, _ = _run(S.TINY, torch.bfloat16, 0, [128, 96], l, g)
+    check_prefill_against_oracle(model, ref, S.TINY.n_layers, 2e-2, 2e-2, 0.1)
+
+
+@pytest.mark.parametrize("lens", [[1], [1, 1, 1], [257, 1, 31, 128, 3]])
+def test_degenerate_and_ragged_batches_fp32(lens):
+    model, ref, _, _ = _run(S.TINY, torch.float32, 7, lens, 2, 1)
+    check_prefill_against_oracle(model, ref, S.TINY.n_layers, 1e-4, 1e-4, 1e-3)
+
+
+def test_more_prompts_than_one_tail_pass():
+    lens = [3, 9, 1, 17, 5, 2, 8, 11, 4, 6, 7]       # 11 prompts: the last-token path runs in two passes of <= 8 rows
+    model, ref, _, _ = _run(S.TINY, torch.float32, 8, lens, 2, 2)
+    check_prefill_against_oracle(model, ref, S.TINY.n_layers, 1e-4, 1e-4, 1e-3)
+
+
+@pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2), (2, 2)])
+@pytest.mark.parametrize("mask", [3, 0])
+def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask):
+    """The same model through the tcgen05 kernels (mask 3) and the SIMT kernels (mask 0); several row tiles and a
+    ragged tail (T = 507), prompts of 1 and 129 tokens included."""
+    lens = [300, 77, 129, 1]
+    model, ref, _, _ = _run(MID, torch.bfloat16, 2, lens, l, g, kernel_mask=mask)
+    check_prefill_against_oracle(model, ref, MID.n_layers, 2e-2, 2e-2, 0.1)
+
+
+def test_reusing_a_model_across_l_g_and_batches():
+    """One model object, several prefills: a smaller later batch must not see stale state, and switching (l, g)
+    re-folds the SingleInputKV weight."""
+    import paper_2410_03960_b200 as P
+    shape, dtype = S.TINY, torch.float32
+    w = S.make_weights(shape, 4, dtype, "cuda")
+    model = P.SwiftKVModel(shape, w, dtype, 300, 4, 1, 1)
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    for lens, l, g in [([200, 100], 2, 1), ([50], 1, 3), ([10, 20, 30, 40], 3, 1), ([64, 64], 4, 1), ([64, 64], 2, 2)]:
+        tok = S.make_prompts(4 + l, lens, shape.vocab)
+        model.prefill(tok, lens, l, g)
+        model.status()
+        ref = O.swiftkv(cfg, ow, tok.numpy(), lens, l, g)
+        check_prefill_against_oracle(model, ref, shape.n_layers, 1e-4, 1e-4, 1e-3)
+        # layers of one AcrossKV group alias one cache slot
+        for j in range(l, shape.n_layers):
+            kj, _, owner = model.kv_cache_view(j)
+            assert owner == l + ((j - l) // g) * g
+            assert kj.data_ptr() == model.kv_cache_view(owner)[0].data_ptr()
+
+
+def test_device_resident_tokens_match_host_tokens():
+    import paper_2410_03960_b200 as P
+    shape, dtype, lens = S.TINY, torch.float32, [40, 25]
+    w = S.make_weights(shape, 5, dtype, "cuda")
+    tok = S.make_prompts(5, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, dtype, 65, 2, 2, 1)
+    model.prefill(tok, lens, 2, 1)
+    model.status()
+    a = model.first_logits().clone()
+    model.prefill_device_tokens(tok.cuda(), lens, 2, 1)
+    model.status()
+    assert torch.equal(a, model.first_logits())
+    bad = tok.clone()
+    bad[3] = shape.vocab + 5
+    with pytest.raises(P.SwiftKVError) as e:
+        model.prefill(bad, lens, 2, 1)
+    assert e.value.code == -1
+    model.prefill_device_tokens(bad.cuda(), lens, 2, 1)
+    with pytest.raises(P.SwiftKVError) as e:
+        model.status()
+    assert e.value.code == -6
+    with pytest.raises(P.SwiftKVError):
+        model.prefill(tok, [40, 26], 2, 1)            # more tokens than max_tokens
+
+
+def test_llama8b_width_reduced_depth():
+    """Llama-3.1-8B widths (hidden 4096, 32/8 heads of 128, FFN 14336, vocab 128256), 4 layers, l = 2:
+    the real GEMM / attention shapes, ragged prompts spanning several 128-row tiles."""
+    lens = [333, 128, 1, 200]
+    model, ref, _, _ = _run(W8B_4L, torch.bfloat16, 1, lens, 2, 1)
+    res = check_prefill_against_oracle(model, ref, W8B_4L.n_layers, 2e-2, 2e-2, 0.1)
+    print("8b-width parity:", res)
