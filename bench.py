@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of SwiftKV prefill on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" = one pass of the whole hot path (embedding, layers 1..l on all prompt tokens, the fused
+SingleInputKV(+AcrossKV) projection, the last-token path through layers l+1..L, first-token logits) over one
+synthetic batch.  Workload at any N: the Llama-3.1-8B shape, bf16, l = 16, AcrossKV group 1, a varlen batch of
+8 prompts with lengths uniform in [2048, 8192] (seed 1), uniform random token ids, random-init weights -- per
+GPU.  With N > 1 every rank runs an independent replica on its own batch (the path has no exchange step), so
+the scaling is weak and `value` is the sum of all ranks' tokens over the slowest rank's device time.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of the same
+workload instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import synthetic_inputs as S  # noqa: E402
+
+SHAPE = S.LLAMA31_8B
+SWIFT_LAYER, ACROSSKV_GROUP = 16, 1
+N_PROMPTS, LEN_LO, LEN_HI, SEED = 8, 2048, 8192, 1
+WORKLOAD = ("llama-3.1-8b shape bf16, swiftkv l=16 g=1, varlen batch of 8 prompts, lengths U[2048,8192] seed 1, "
+            "uniform random token ids")
+ORACLE_SAMPLE_TOKENS_PER_PROMPT = 32
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0
+# DRAM bytes per SwiGLU-GEMM launch of this workload from the committed ncu capture (profiles/), or None
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.lines, self.proc, self.thread = gpu_index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def flops_of(lens, l, g):
+    from paper_2410_03960_b200 import prefill_flops
+    s = SHAPE
+    return prefill_flops(s.hidden, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn, s.vocab, lens, l, g)
+
+
+def time_steps(fn, steps, dist_barrier):
+    """K steps between a barrier + synchronize on both sides; device time from CUDA events on the current stream."""
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist_barrier()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        fn()
+    stop.record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    return start.elapsed_time(stop) / 1e3
+
+
+# ---------------------------------------------------------------------------------------------------------------
+def oracle_setup(lens_full, device):
+    """Inputs of the CPU-oracle leg: the same model, every prompt cut to its first few tokens (a causal prefix of
+    the real prompt), weights upcast once to fp64 outside the timed region."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import numpy as np
+    from oracle import swiftkv_oracle as O
+    lens = [min(n, ORACLE_SAMPLE_TOKENS_PER_PROMPT) for n in lens_full]
+    tok = S.make_prompts(SEED, lens, SHAPE.vocab).numpy()
+    cfg = O.Config(SHAPE.vocab, SHAPE.hidden, SHAPE.n_layers, SHAPE.n_q_heads, SHAPE.n_kv_heads, SHAPE.head_dim,
+                   SHAPE.ffn, SHAPE.rope_theta, SHAPE.rms_eps)
+    f64 = lambda t: t.to("cpu").double().numpy()   # noqa: E731
+    layers = [{k: f64(v) for k, v in S.layer_weights(SHAPE, SEED, j, torch.bfloat16, device).items()}
+              for j in range(SHAPE.n_layers)]
+    g = S.global_weights(SHAPE, SEED, torch.bfloat16, device)
+    emb_rows = {int(t): f64(S.matrix_rows(SEED, 0xF000, torch.tensor([int(t)]), SHAPE.hidden, torch.bfloat16))[0]
+                for t in set(tok.tolist())}
+    lm = f64(g["lm_head"])
+    W = O.Weights(lambda ids: np.stack([emb_rows[int(t)] for t in ids]), f64(g["final_norm"]), lambda: lm,
+                  lambda j: layers[j])
+    del g
+    return O, cfg, W, tok, lens
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, rank):
+    """The reference arm of this tier: the CPU oracle as it stands, timed on the host cores."""
+    if rank != 0:
+        return
+    device = "cuda" if torch.cuda.is_available() else "cpu"
+    lens_full = S.uniform_lengths(SEED, N_PROMPTS, LEN_LO, LEN_HI)
+    O, cfg, W, tok, lens = oracle_setup(lens_full, device)
+    import numpy as np  # noqa: F401
+    for _ in range(args.warmup):
+        O.swiftkv(cfg, W, tok, lens, SWIFT_LAYER, ACROSSKV_GROUP)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.swiftkv(cfg, W, tok, lens, SWIFT_LAYER, ACROSSKV_GROUP)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = sum(lens) / dt
+    cores = oracle_threads()
+    sample = (f"each of the 8 prompts cut to its first {ORACLE_SAMPLE_TOKENS_PER_PROMPT} tokens "
+              f"({sum(lens)} tokens per step), full 32-layer model, fp64 numpy")
+    line = {"impl": "reference", "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+def run_ours(args, rank, world, local_rank):
+    import paper_2410_03960_b200 as P
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the SwiftKV prefill path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    use_dist = world > 1
+    if use_dist:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+        def barrier():
+            dist.barrier()
+    else:
+        def barrier():
+            pass
+
+    seed = SEED + 1000 * rank                      # rank 0 runs exactly the named batch; replicas differ
+    lens = S.uniform_lengths(seed, N_PROMPTS, LEN_LO, LEN_HI)
+    T = sum(lens)
+    tok_host = S.make_prompts(seed, lens, SHAPE.vocab).pin_memory()
+    tok_dev = tok_host.to(dev)
+    w = S.make_weights(SHAPE, SEED, torch.bfloat16, dev)
+    model = P.SwiftKVModel(SHAPE, w, torch.bfloat16, T, N_PROMPTS, SWIFT_LAYER, ACROSSKV_GROUP, device=dev)
+    logits_host = torch.empty((N_PROMPTS, SHAPE.vocab), dtype=torch.float32).pin_memory()
+    L = SHAPE.n_layers
+
+    def step_swift():
+        model.prefill_device_tokens(tok_dev, lens, SWIFT_LAYER, ACROSSKV_GROUP)
+
+    def step_full():
+        model.prefill_device_tokens(tok_dev, lens, L, 1)
+
+    def step_e2e():
+        model.prefill(tok_host, lens, SWIFT_LAYER, ACROSSKV_GROUP)
+        logits_host.copy_(model.first_logits(), non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    # ---- warm-up (also folds the SingleInputKV weight once, outside the timed region)
+    for _ in range(max(args.warmup, 3)):
+        step_swift()
+    model.status()
+
+    # ---- timed: SwiftKV prefill, inputs resident in HBM, with per-class launch timing
+    gpu_index = local_rank
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            gpu_index = int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            pass
+    sampler = ClockSampler(gpu_index)
+    if rank == 0:
+        sampler.start()
+    model.profile_enable(True)
+    model.profile_read()
+    t_swift = time_steps(step_swift, args.steps, barrier)
+    prof = model.profile_read()
+    model.profile_enable(False)
+    launches = model.last_launch_count() * args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    model.status()
+
+    # ---- e2e: host token ids in (pinned), logits out, every step
+    for _ in range(2):
+        step_e2e()
+    t_e2e = time_steps(step_e2e, args.steps, barrier)
+
+    # ---- the unmodified full-depth prefill (l = L) built from the same kernels
+    for _ in range(2):
+        step_full()
+    t_full = time_steps(step_full, args.steps, barrier)
+    model.status()
+
+    tokens_total = float(T * args.steps)
+    times = torch.tensor([t_swift, t_e2e, t_full], dtype=torch.float64, device=dev)
+    toks = torch.tensor([tokens_total], dtype=torch.float64, device=dev)
+    if use_dist:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
+    t_swift, t_e2e, t_full = times.tolist()
+    tokens_all = toks.item()
+
+    if rank == 0:
+        peaks, peaks_kind = measured_peaks()
+        f_sw, f_full = flops_of(lens, SWIFT_LAYER, ACROSSKV_GROUP), flops_of(lens, L, 1)
+        ms_step = t_swift / args.steps * 1e3
+        actual_tflops = f_sw["total"] / (t_swift / args.steps) / 1e12
+        norm_tflops = f_full["total"] / (t_swift / args.steps) / 1e12
+        gemm_ms, gemm_launches = prof["gemm"]
+        gemm_ach = f_sw["gemm"] * args.steps / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else None
+        peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
+        attn_ms = prof["attention"][0]
+        line = {
+            "metric": "prefill_tokens_per_s", "value": tokens_all / t_swift, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_step_per_gpu": T, "seq_lens_rank0": lens,
+                       "l2": "inputs larger than L2 (16 GB of weights, > 3 GB of activations per step)",
+                       "multi_gpu": "replicas only: independent batch per rank, no collective"},
+            "tflops_per_gpu": {"actual": actual_tflops, "normalized_to_full_depth": norm_tflops,
+                               "paper_shortcut_2N": tokens_all / world / t_swift * 2 * SHAPE.n_params() / 1e12,
+                               "frac_of_measured_burst": actual_tflops / peaks["bf16_tflops"],
+                               "frac_of_measured_sustained": actual_tflops / peak,
+                               "frac_of_nominal_2250": actual_tflops / NOMINAL_BF16_TFLOPS, "peaks": peaks_kind},
+            "full_depth": {"tokens_per_s": tokens_all / t_full, "ms_per_step": t_full / args.steps * 1e3,
+                           "tflops": f_full["total"] / (t_full / args.steps) / 1e12,
+                           "swiftkv_speedup": t_full / t_swift, "flop_ratio": f_full["total"] / f_sw["total"]},
+            "e2e": {"value": tokens_all / t_e2e, "unit": "tokens/s", "h2d_bytes_per_step": T * 4 + (N_PROMPTS + 1) * 4 + N_PROMPTS * 4,
+                    "d2h_bytes_per_step": N_PROMPTS * SHAPE.vocab * 4},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (all projection / MLP / SingleInputKV GEMM launches)",
+                         "achieved": gemm_ach, "peak": peak, "unit": "TFLOP/s",
+                         "frac": (gemm_ach / peak) if gemm_ach else None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
+                         "frac_of_burst": (gemm_ach / peaks["bf16_tflops"]) if gemm_ach else None,
+                         "launches_per_step": gemm_launches // max(args.steps, 1), "ms_per_step": gemm_ms / args.steps,
+                         "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH},
+            "time_share_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
+            "attention_tflops": (f_sw["attention"] * args.steps / (attn_ms / 1e3) / 1e12) if attn_ms > 0 else None,
+        }
+        # ---- the CPU oracle, as it stands, on a bounded sample of the same workload (N = 1 only)
+        if world == 1 and not args.no_cpu_baseline:
+            O, cfg, W, tok_s, lens_s = oracle_setup(lens, dev)
+            t0 = time.perf_counter()
+            O.swiftkv(cfg, W, tok_s, lens_s, SWIFT_LAYER, ACROSSKV_GROUP)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {"value": sum(lens_s) / dt, "unit": "tokens/s", "cores": oracle_threads(), "kind": "oracle",
+                                    "sample": f"each prompt cut to its first {ORACLE_SAMPLE_TOKENS_PER_PROMPT} tokens "
+                                              f"({sum(lens_s)} tokens), full 32-layer model, one pass, {dt:.1f} s"}
+        print(json.dumps(line), flush=True)
+    model.close()
+    if use_dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
