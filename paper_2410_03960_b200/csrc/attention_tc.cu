@@ -1,7 +1,332 @@
-// Tensor-core causal varlen GQA prefill attention (placeholder until the tcgen05 kernel lands).
+// Causal varlen grouped-query flash attention for prefill on tcgen05 tensor cores (head_dim 128, bf16).
+//
+// One CTA works on one (prompt, 128-query tile, PAIR of query heads that share a KV head): the two heads see
+// exactly the same keys, values and causal mask, so they ping-pong on the tensor pipe while sharing every K/V
+// tile that TMA brings in.  320 threads:
+//   warp 0      : TMA producer (Q of both heads once; K and V tiles of 128 keys through 2-deep rings)
+//   warp 1      : MMA issuer: S_w = Q_w K^T into tensor memory, then O_w += P_w V with P_w read straight from
+//                 tensor memory (the softmax warps overwrite S_w with bf16 P_w in place)
+//   warps 2..5  : softmax of head 0 -- one query row per thread (a TMEM lane), so row max / sum need no shuffles;
+//   warps 6..9  : softmax of head 1.
+// Online softmax keeps a per-row reference max that only moves when the running max grows by more than 2^8
+// (then O_w is rescaled in tensor memory); the final O_w / l_w is exact for any such reference.
+// Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each (all 512).  Every wait is bounded.
 #include "common.cuh"
+#include "tc_common.cuh"
+
 namespace skv {
-bool tc_attention_supported(int, int, int) { return false; }
-int launch_attention_tc(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int, int, int, int, int, int,
-                        unsigned int *, cudaStream_t) { return SWIFTKV_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int HD = 128;                 // head dim
+constexpr int BQ = 128, BKV = 128;      // query rows / keys per tile
+constexpr int ATT_THREADS = 320;
+constexpr int TILE_BYTES = 128 * HD * 2;          // 32 KB: one [128 x 128] bf16 tile = two 64-column swizzled chunks
+constexpr int CHUNK_BYTES = TILE_BYTES / 2;       // 16 KB
+constexpr int KV_STAGES = 2;
+constexpr int SM_Q = 0, SM_K = 2 * TILE_BYTES, SM_V = SM_K + KV_STAGES * TILE_BYTES;
+constexpr int SM_BAR = SM_V + KV_STAGES * TILE_BYTES;
+constexpr int ATT_SMEM = SM_BAR + 256 + 1024;
+constexpr float RESCALE_THRESHOLD = 8.0f;          // in log2 units
+
+struct AttnParams {
+  const int32_t *cu;
+  bf16 *out;
+  int n_seqs, n_q, n_kv, max_tiles;
+  float scale_log2;     // softmax scale * log2(e)
+  unsigned int *status;
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
+  if (tc::mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!tc::mbar_try_wait(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > tc::WAIT_LIMIT_CLOCKS) {
+      *abort_flag = 1;
+      atomicOr(status, STATUS_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, AttnParams p) {
+  // ---- which work item: heavy (late) query tiles first
+  const int n_pairs = p.n_q >> 1;
+  const int per_tile = p.n_seqs * n_pairs;
+  const int qt = p.max_tiles - 1 - (int)(blockIdx.x / per_tile);
+  const int rem = blockIdx.x % per_tile;
+  const int b = rem / n_pairs, pair = rem % n_pairs;
+  const int tok0 = p.cu[b], n = p.cu[b + 1] - tok0;
+  if (qt * BQ >= n) return;
+  const int h0 = pair * 2;
+  const int kvh = h0 / (p.n_q / p.n_kv);
+  const int n_kv_tiles = qt + 1;
+  const int q_row0 = tok0 + qt * BQ;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM_BAR);
+  uint64_t *q_full = bars;            // [1]
+  uint64_t *k_full = bars + 1;        // [2]
+  uint64_t *k_empty = bars + 3;       // [2]
+  uint64_t *v_full = bars + 5;        // [2]
+  uint64_t *v_empty = bars + 7;       // [2]
+  uint64_t *s_full = bars + 9;        // [2]  S_w ready in tensor memory
+  uint64_t *p_ready = bars + 11;      // [2]  P_w written (and O_w rescaled) by the softmax warps
+  uint64_t *o_full = bars + 13;       // [1]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(q_full), 1);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(tc::smem_u32(&k_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&k_empty[s]), 1);
+      tc::mbar_init(tc::smem_u32(&v_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&v_empty[s]), 1);
+      tc::mbar_init(tc::smem_u32(&s_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&p_ready[s]), 4);   // one arrival per softmax warp
+    }
+    tc::mbar_init(tc::smem_u32(o_full), 1);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmQ);
+    tc::tma_prefetch_desc(&tmK);
+    tc::tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), 512);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  // tensor-memory columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_w aliases the first 64 of S_w
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ TMA producer
+      const uint32_t qb = tc::smem_u32(q_full);
+      tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
+      for (int w = 0; w < 2; ++w)
+        for (int c = 0; c < 2; ++c)
+          tc::tma_load_2d(tc::smem_u32(smem + SM_Q + w * TILE_BYTES + c * CHUNK_BYTES), &tmQ, qb, (h0 + w) * HD + c * 64, q_row0);
+      for (int j = 0; j < n_kv_tiles; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        if (!wait_or_abort(tc::smem_u32(&k_empty[s]), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t kb = tc::smem_u32(&k_full[s]);
+        tc::mbar_expect_tx(kb, TILE_BYTES);
+        for (int c = 0; c < 2; ++c)
+          tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, tok0 + j * BKV);
+        if (!wait_or_abort(tc::smem_u32(&v_empty[s]), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t vb = tc::smem_u32(&v_full[s]);
+        tc::mbar_expect_tx(vb, TILE_BYTES);
+        for (int c = 0; c < 2; ++c)
+          tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, tok0 + j * BKV);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ MMA issuer
+      constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(BQ, BKV, 0, 0);   // Q, K both K-major (head dim contiguous)
+      constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(BQ, HD, 0, 1);    // V is MN-major (head dim contiguous, keys = K)
+      const uint32_t q_addr = tc::smem_u32(smem + SM_Q);
+      auto issue_qk = [&](int w, int s) {   // S_w = Q_w K^T : 8 steps of 16 along the head dim
+        const uint32_t a0 = q_addr + w * TILE_BYTES, b0 = tc::smem_u32(smem + SM_K + s * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * CHUNK_BYTES + (kk & 3) * 32;
+          tc::umma_ss(tmem_base + w * 128, tc::umma_desc_sw128(a0 + off, 16, 1024), tc::umma_desc_sw128(b0 + off, 16, 1024),
+                      idesc_qk, kk != 0);
+        }
+      };
+      auto issue_pv = [&](int w, int s, bool accumulate) {   // O_w (+)= P_w V : 8 steps of 16 keys
+        const uint32_t b0 = tc::smem_u32(smem + SM_V + s * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < BKV / 16; ++kk)
+          tc::umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + kk * 8,
+                      tc::umma_desc_sw128(b0 + kk * 16 * 128, CHUNK_BYTES, 1024), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+      };
+      bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) &&
+                wait_or_abort(tc::smem_u32(&k_full[0]), 0, abort_flag, p.status);
+      if (ok) {
+        tc::tc_fence_after_sync();
+        issue_qk(0, 0);
+        tc::umma_commit(tc::smem_u32(&s_full[0]));
+        issue_qk(1, 0);
+        tc::umma_commit(tc::smem_u32(&s_full[1]));
+        tc::umma_commit(tc::smem_u32(&k_empty[0]));
+      }
+      for (int j = 0; j < n_kv_tiles && ok; ++j) {
+        const int s = j & 1, s1 = (j + 1) & 1;
+        const uint32_t ph = (j >> 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+        const bool more = j + 1 < n_kv_tiles;
+        if (!wait_or_abort(tc::smem_u32(&v_full[s]), ph, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_or_abort(tc::smem_u32(&p_ready[0]), j & 1, abort_flag, p.status)) { ok = false; break; }
+        tc::tc_fence_after_sync();
+        issue_pv(0, s, j > 0);
+        if (more) {
+          if (!wait_or_abort(tc::smem_u32(&k_full[s1]), ph1, abort_flag, p.status)) { ok = false; break; }
+          tc::tc_fence_after_sync();
+          issue_qk(0, s1);
+          tc::umma_commit(tc::smem_u32(&s_full[0]));
+        }
+        if (!wait_or_abort(tc::smem_u32(&p_ready[1]), j & 1, abort_flag, p.status)) { ok = false; break; }
+        tc::tc_fence_after_sync();
+        issue_pv(1, s, j > 0);
+        tc::umma_commit(tc::smem_u32(&v_empty[s]));
+        if (more) {
+          issue_qk(1, s1);
+          tc::umma_commit(tc::smem_u32(&s_full[1]));
+          tc::umma_commit(tc::smem_u32(&k_empty[s1]));
+        }
+      }
+      if (ok) tc::umma_commit(tc::smem_u32(o_full));
+    }
+  } else {
+    // -------------------------------------------------------------- softmax warps: head w, one row per thread
+    const int w = (warp - 2) >> 2;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;                // query row inside the tile = TMEM lane
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t t_s = tmem_base + lane_base + w * 128;
+    const uint32_t t_o = tmem_base + lane_base + 256 + w * 128;
+    const float c = p.scale_log2;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv_tiles; ++j) {
+      if (!wait_or_abort(tc::smem_u32(&s_full[w]), j & 1, abort_flag, p.status)) { ok = false; break; }
+      tc::tc_fence_after_sync();
+      const bool diag = (j == qt);
+      // pass 1: row max of the raw scores
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32b_x32(t_s + ch * 32, r);
+        tc::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float v = __uint_as_float(r[i]);
+          if (diag && (ch * 32 + i > row)) v = -INFINITY;
+          mx = fmaxf(mx, v);
+        }
+      }
+      // move the reference max only when the running max outgrew it by more than the threshold
+      const bool need = (j == 0) || ((mx - m_ref) * c > RESCALE_THRESHOLD);
+      const float m_new = need ? mx : m_ref;
+      if (j > 0 && __any_sync(0xffffffffu, need)) {
+        // S_w of this tile is complete, so every earlier P_w V has retired: O_w is stable and may be rescaled
+        const float f = need ? fast_exp2((m_ref - m_new) * c) : 1.f;
+        l *= f;
+#pragma unroll 1
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t r[16];
+          tc::tmem_ld_32x32b_x16(t_o + ch * 16, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+          tc::tmem_st_32x32b_x16(t_o + ch * 16, r);
+        }
+      }
+      m_ref = m_new;
+      // pass 2: p = 2^(s*c - m_ref*c), row sum, bf16 P written over S (64 packed columns)
+      const float neg_mc = -m_ref * c;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32b_x32(t_s + ch * 32, r);
+        tc::tmem_ld_wait();
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), c, neg_mc));
+          float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), c, neg_mc));
+          if (diag) {
+            if (ch * 32 + 2 * i > row) p0 = 0.f;
+            if (ch * 32 + 2 * i + 1 > row) p1 = 0.f;
+          }
+          l += p0 + p1;
+          pk[i] = tc::pack_bf16x2(p0, p1);
+        }
+        tc::tmem_st_32x32b_x16(t_s + ch * 16, pk);
+      }
+      tc::tmem_st_wait();
+      tc::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(tc::smem_u32(&p_ready[w]));
+    }
+    // ---- epilogue: O_w / l -> bf16 -> out[token, head, :]
+    if (ok && wait_or_abort(tc::smem_u32(o_full), 0, abort_flag, p.status)) {
+      tc::tc_fence_after_sync();
+      const float inv = 1.f / l;
+      const bool valid = qt * BQ + row < n;
+      bf16 *dst = p.out + ((size_t)(q_row0 + row) * p.n_q + (h0 + w)) * HD;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32b_x32(t_o + ch * 32, r);
+        tc::tmem_ld_wait();
+        if (valid) {
+          uint4 *d4 = reinterpret_cast<uint4 *>(dst + ch * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            d4[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv),
+                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv),
+                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv),
+                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv));
+        }
+      }
+    }
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool tc_attention_supported(int n_q, int n_kv, int hd) {
+  return hd == HD && n_kv >= 1 && n_q % n_kv == 0 && ((n_q / n_kv) % 2) == 0;
+}
+
+int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, const int32_t *cu_seqlens, int n_seqs,
+                        int n_tokens, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st) {
+  if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
+  if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1) return SWIFTKV_ERR_INVALID_ARG;
+  CUtensorMap tq, tk, tv;
+  // row extent = the tokens of this call: rows past it read as zero (never stale cache contents)
+  if (get_tmap(&tq, q, n_tokens, (uint64_t)n_q * hd, (uint64_t)n_q * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tk, k, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tv, v, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
+      return SWIFTKV_ERR_CUDA;
+    attr_set = true;
+  }
+  AttnParams p{};
+  p.cu = cu_seqlens; p.out = out; p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
+  p.max_tiles = (max_seq_len + BQ - 1) / BQ;
+  p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
+  p.status = status;
+  const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
+  if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
+  attention_tc_kernel<<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+}
+
 }  // namespace skv

@@ -66,7 +66,6 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t 
 }
 
 namespace {
-
 // tensor maps are pure functions of (pointer, shape, box): cache them
 struct TmapKey {
   const void *p; uint64_t rows, cols, ld; uint32_t br, bc;
@@ -81,6 +80,8 @@ struct TmapKeyHash {
 };
 std::mutex g_tmap_mu;
 std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> g_tmaps;
+
+}  // namespace
 
 int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t br, uint32_t bc) {
   TmapKey k{p, rows, cols, ld, br, bc};
@@ -107,6 +108,7 @@ int num_sms() {
   return n;
 }
 
+namespace {
 // ---------------------------------------------------------------------------------------------------------
 // device
 // ---------------------------------------------------------------------------------------------------------

@@ -175,4 +175,8 @@ int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_
 int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1,
                       uint64_t s2, uint32_t b0, uint32_t b1);
 
+// cached make_tmap_2d_bf16 (tensor maps are pure functions of pointer, shape and box)
+int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, uint32_t box_cols);
+int num_sms();
+
 }  // namespace skv

@@ -42,3 +42,26 @@ def test_attention_simt(dtype, bar, lens, n_q, n_kv, hd):
         ref = O.causal_attention(to_np(q[off:off + n]), to_np(k[off:off + n]), to_np(v[off:off + n]))
         assert rel_l2(to_np(out[off:off + n]), ref) < bar
         off += n
+
+
+@pytest.mark.parametrize("lens,n_q,n_kv", [([5, 1, 70], 8, 2), ([300, 129, 128, 1], 8, 2), ([1000], 4, 1),
+                                           ([128], 2, 1), ([127, 257], 16, 2), ([2500, 700], 8, 4)])
+def test_attention_tcgen05(lens, n_q, n_kv):
+    """Tensor-core flash attention (head_dim 128) against the oracle's explicit softmax(QK^T)V, prompt by prompt:
+    single-tile, multi-tile, ragged and one-token prompts."""
+    import paper_2410_03960_b200 as P
+    hd, T = 128, sum(lens)
+    q = S.matrix(5, 1, T, n_q * hd, torch.bfloat16, "cuda", std=1.0).view(T, n_q, hd)
+    k = S.matrix(5, 2, T, n_kv * hd, torch.bfloat16, "cuda", std=1.0).view(T, n_kv, hd)
+    v = S.matrix(5, 3, T, n_kv * hd, torch.bfloat16, "cuda", std=1.0).view(T, n_kv, hd)
+    out = P.attention_prefill(q, k, v, lens, use_tensor_cores=True)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
+    off = 0
+    for n in lens:
+        ref = O.causal_attention(to_np(q[off:off + n]), to_np(k[off:off + n]), to_np(v[off:off + n]))
+        got = to_np(out[off:off + n])
+        # P is rounded to bf16 before the PV product and the output is stored in bf16
+        assert rel_l2(got, ref) < 1e-2, (n, rel_l2(got, ref))
+        assert np.max(np.abs(got - ref)) < 0.05
+        off += n
