@@ -56,7 +56,7 @@ struct Buffers {
   void *act;                // SwiGLU output [T, F]
   void *wfold;              // folded, concatenated SingleInputKV weight [n_groups*2*d_kv, d]
   float *y;                 // continuing tokens' residual [B, d]
-  void *hy, *qy, *ay, *gy, *uy, *acty;
+  float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
   float *tail_scratch;
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
@@ -121,12 +121,11 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.act = cv.take((size_t)T * F * E);
   b.wfold = cv.take(fold_elems * E);
   b.y = (float *)cv.take((size_t)B * d * 4);
-  b.hy = cv.take((size_t)B * std::max(d, dq) * E);
-  b.qy = cv.take((size_t)B * dq * E);
-  b.ay = cv.take((size_t)B * dq * E);
-  b.gy = cv.take((size_t)B * F * E);
-  b.uy = cv.take((size_t)B * F * E);
-  b.acty = cv.take((size_t)B * F * E);
+  const size_t R = std::min<size_t>(B, MAX_TAIL_ROWS);
+  b.hy = (float *)cv.take(R * std::max(d, dq) * 4);
+  b.qy = (float *)cv.take(R * dq * 4);
+  b.ay = (float *)cv.take(R * dq * 4);
+  b.acty = (float *)cv.take(R * F * 4);
   b.tail_scratch = (float *)cv.take(tail_attention_scratch_bytes(B, c.n_q_heads, c.head_dim, T));
   b.logits = (float *)cv.take((size_t)B * c.vocab * 4);
   b.tokens = (int32_t *)cv.take((size_t)T * 4);
@@ -244,13 +243,21 @@ struct Scope {
 // ---------------------------------------------------------------------------------------------------------
 // the schedule
 // ---------------------------------------------------------------------------------------------------------
+// rope_fused (optional): in: request the rotary embedding in the epilogue; out: whether it was applied
 template <typename T>
 static int32_t gemm_any(swiftkv_model *m, const T *A, int M, int K, const T *B0, int n0, const T *B1, int n1,
-                        const T *B2, int n2, const OutDesc &out, cudaStream_t st) {
+                        const T *B2, int n2, const OutDesc &out, cudaStream_t st, const RopeSpec *rope = nullptr,
+                        bool *rope_fused = nullptr) {
   Scope sc(m, st, SWIFTKV_KC_GEMM, 0);
+  if (rope_fused) *rope_fused = false;
   if constexpr (sizeof(T) == 2) {
     if ((m->kernel_mask & 1) && tc_gemm_supported(M, n0 + n1 + n2, K)) {
-      int rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, m->b.status, st);
+      int rc = SWIFTKV_ERR_UNSUPPORTED;
+      if (rope && rope_fused) {
+        rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, rope, m->b.status, st);
+        if (rc == SWIFTKV_OK) *rope_fused = true;
+      }
+      if (rc == SWIFTKV_ERR_UNSUPPORTED) rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, nullptr, m->b.status, st);
       if (rc == SWIFTKV_OK) { m->launches += 1; return rc; }
       if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "tensor-core GEMM launch failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
@@ -271,6 +278,7 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
   T *kv = reinterpret_cast<T *>(m->kv);
   T *h = (T *)b.h, *q = (T *)b.q, *attn = (T *)b.attn, *act = (T *)b.act;
   int32_t rc;
+  const RopeSpec rope{b.pos, b.cos_tab, b.sin_tab, c.head_dim};
 
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_positions(b.cu, B, b.pos, b.last_idx, T_tok, st); }
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_embed<T>((const T *)m->embed, b.tokens, b.x, T_tok, d, c.vocab, b.status, st); }
@@ -294,10 +302,13 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
     T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
     OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv};
-    rc = gemm_any<T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st);
+    bool roped = false;
+    rc = gemm_any<T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st, &rope, &roped);
     if (rc) return rc;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    if (!roped) {
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    }
     {
       Scope s(m, st, SWIFTKV_KC_ATTENTION);
       bool done = false;
@@ -346,35 +357,34 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
     T *slot_l = kv + (size_t)l * 2 * plane;
     OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv};
-    rc = gemm_any<T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, (const T *)nullptr, 0, (const T *)nullptr, 0, o, st);
+    bool roped = false;
+    rc = gemm_any<T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, (const T *)nullptr, 0, (const T *)nullptr, 0, o, st, &rope, &roped);
     if (rc) return rc;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
   }
 
   // ---- the last token of each prompt continues through layers l+1..L (footnote of Sec. 3.2)
   for (int r0 = 0; r0 < B; r0 += MAX_TAIL_ROWS) {
     const int rows = std::min(MAX_TAIL_ROWS, B - r0);
-    T *hy = (T *)b.hy, *qy = (T *)b.qy, *ay = (T *)b.ay, *gy = (T *)b.gy, *uy = (T *)b.uy, *acty = (T *)b.acty;
+    float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
     float *y = b.y + (size_t)r0 * d;
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
     for (int j = l; j < L; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
       const int slot = l + (j - l) / g;
       const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, rows, dq, d, out_plain(OUT_STORE, qy, dq, dq), st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<T>(qy, 0, 1, b.last_pos + r0, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.cu + r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, rows, d, dq, out_plain(OUT_RESID_ADD_F32, y, d, d), st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, rows, F, d, out_plain(OUT_STORE, gy, F, F), st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_up, rows, F, d, out_plain(OUT_STORE, uy, F, F), st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_swiglu<T>(gy, uy, acty, (long long)rows * F, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, rows, d, F, out_plain(OUT_RESID_ADD_F32, y, d, d), st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, nullptr, rows, d, F, y, d, OUT_RESID_ADD_F32, st); }
     }
-    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rmsnorm<T>(y, (const T *)m->final_norm, hy, rows, d, c.rms_eps, st); }
-    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)m->lm_head, rows, c.vocab, d,
-                                                              out_plain(OUT_STORE_F32, b.logits + (size_t)r0 * c.vocab, c.vocab, c.vocab), st); }
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)m->final_norm, hy, rows, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)m->lm_head, nullptr, rows, c.vocab, d,
+                                                              b.logits + (size_t)r0 * c.vocab, c.vocab, OUT_STORE_F32, st); }
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -525,7 +535,7 @@ extern "C" int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int3
   unsigned int *status = op_status_word();
   if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
   int rc = launch_gemm_tc((const bf16 *)A, M, K, (const bf16 *)B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N),
-                          status, reinterpret_cast<cudaStream_t>(cuda_stream));
+                          nullptr, status, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
   return SWIFTKV_OK;
 }

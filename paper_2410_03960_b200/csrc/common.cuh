@@ -99,8 +99,15 @@ void launch_gemm_simt(const T *A, const T *B, int M, int N, int K, OutDesc out, 
 struct TcGemmPlan;   // host object holding tensor maps
 bool tc_gemm_supported(int M, int N, int K);
 // generic: B rows come from up to three matrices stacked along N: [0,nB0) from B0, [nB0, nB0+nB1) from B1, rest B2
+// rope != nullptr: the rotary embedding (rotate-half pairs (i, i + hd/2)) is applied in the epilogue, in fp32,
+// to the columns below out.n0 and to the even-numbered segments above it (K planes; odd ones are V planes)
+struct RopeSpec {
+  const int32_t *positions;
+  const float *cos_tab, *sin_tab;   // [position][hd/2]
+  int hd;
+};
 int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
-                   int nB2, OutDesc out, unsigned int *status, cudaStream_t st);
+                   int nB2, OutDesc out, const RopeSpec *rope, unsigned int *status, cudaStream_t st);
 // act[M, F] = silu(A Wg^T) * (A Wu^T), gate/up tiles paired inside one CTA tile
 int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
                           unsigned int *status, cudaStream_t st);
@@ -116,15 +123,19 @@ int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, 
                         int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd,
                         unsigned int *status, cudaStream_t st);
 
-// tail.cu : the last-token path (M = n_seqs <= 8 rows)
-// out[b, n] (+)= sum_k act[b, k] * W[n, k]
+// tail.cu : the last-token path (at most MAX_TAIL_ROWS activation rows per launch, fp32 activations)
+constexpr int MAX_TAIL_ROWS = 8;
 template <typename T>
-void launch_skinny_gemm(const T *act, const T *W, int n_rows, int N, int K, OutDesc out, cudaStream_t st);
+void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, int d, float eps, cudaStream_t st);
+// out[r, n] = sum_k act[r, k] * W[n, k]  (mode OUT_STORE_F32 or OUT_RESID_ADD_F32);
+// with W2: out[r, n] = silu(act W^T) * (act W2^T)
+template <typename T>
+void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
+                        int mode, cudaStream_t st);
 // one query token per prompt against that prompt's cache rows [cu[b], cu[b+1]); scratch holds split partials
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
-constexpr int MAX_TAIL_ROWS = 8;   // rows one skinny-GEMM launch handles
 template <typename T>
-void launch_tail_attention(const T *q, const T *kc, const T *vc, T *out, const int32_t *cu_seqlens, int n_seqs,
+void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens, int n_seqs,
                            int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
 
 }  // namespace skv

@@ -123,8 +123,11 @@ struct GemmTcParams {
   OutDesc out;
   bf16 *act;             // SwiGLU output [M, F]
   int F;
+  const int32_t *rope_pos;   // EPI_ROPE: position of every row; cos/sin tables [pos][64]
+  const float *cos_tab, *sin_tab;
   unsigned int *status;
 };
+enum { EPI_PLAIN = 0, EPI_SWIGLU = 1, EPI_ROPE = 2 };
 
 template <int BN, int STAGES>
 struct SmemLayout {
@@ -158,11 +161,12 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
   return true;
 }
 
-template <int BN, int STAGES, bool SWIGLU>
+template <int BN, int STAGES, int EPI>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmTcParams p) {
   using L = SmemLayout<BN, STAGES>;
+  constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::BAR_OFFSET);
@@ -292,6 +296,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
           }
         }
+      } else if constexpr (EPI == EPI_ROPE) {
+        // head-aligned tiles (head_dim 128): rotate pairs (i, i + 64) of the q / K heads in fp32 before the one
+        // rounding to bf16; V heads are stored as they are
+        const int pos = row < p.M ? p.rope_pos[row] : 0;
+        const float4 *ct = reinterpret_cast<const float4 *>(p.cos_tab + (size_t)pos * 64);
+        const float4 *sn = reinterpret_cast<const float4 *>(p.sin_tab + (size_t)pos * 64);
+#pragma unroll 1
+        for (int hh = 0; hh < BN / 128; ++hh) {
+          const int col_h = n_blk * BN + hh * 128;
+          bf16 *dstp;
+          bool rope;
+          if (col_h < p.out.n0) {
+            dstp = reinterpret_cast<bf16 *>(p.out.p0) + (size_t)row * p.out.ld0 + col_h;
+            rope = true;
+          } else {
+            const int cc = col_h - p.out.n0;
+            const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
+            dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + (size_t)row * p.out.seg_w + within;
+            rope = (seg & 1) == 0;      // segments alternate K (rotated) and V (not)
+          }
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            uint32_t a[32], bq[32];
+            tc::tmem_ld_32x32b_x32(t_row + hh * 128 + c * 32, a);
+            tc::tmem_ld_32x32b_x32(t_row + hh * 128 + 64 + c * 32, bq);
+            tc::tmem_ld_wait();
+            if (row < p.M) {
+              if (rope) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                  const float4 cv = ct[c * 8 + i], sv = sn[c * 8 + i];
+                  const float cc4[4] = {cv.x, cv.y, cv.z, cv.w}, ss4[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float x = __uint_as_float(a[4 * i + e]), y = __uint_as_float(bq[4 * i + e]);
+                    a[4 * i + e] = __float_as_uint(x * cc4[e] - y * ss4[e]);
+                    bq[4 * i + e] = __float_as_uint(y * cc4[e] + x * ss4[e]);
+                  }
+                }
+              }
+              uint4 *d0 = reinterpret_cast<uint4 *>(dstp + c * 32);
+              uint4 *d1 = reinterpret_cast<uint4 *>(dstp + 64 + c * 32);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                d0[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(a[8 * i]), __uint_as_float(a[8 * i + 1])),
+                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3])),
+                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5])),
+                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7])));
+                d1[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(bq[8 * i]), __uint_as_float(bq[8 * i + 1])),
+                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 2]), __uint_as_float(bq[8 * i + 3])),
+                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 4]), __uint_as_float(bq[8 * i + 5])),
+                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 6]), __uint_as_float(bq[8 * i + 7])));
+              }
+            }
+          }
+        }
       } else {
 #pragma unroll 1
         for (int c = 0; c < BN / 32; ++c) {
@@ -343,11 +403,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
-template <int BN, int STAGES, bool SWIGLU>
+template <int BN, int STAGES, int EPI>
 int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const CUtensorMap &b2,
                const GemmTcParams &p, cudaStream_t st) {
   using L = SmemLayout<BN, STAGES>;
-  auto kern = gemm_tc_kernel<BN, STAGES, SWIGLU>;
+  auto kern = gemm_tc_kernel<BN, STAGES, EPI>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess) return SWIFTKV_ERR_CUDA;
@@ -365,7 +425,7 @@ bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 6
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
 
 int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
-                   int nB2, OutDesc out, unsigned int *status, cudaStream_t st) {
+                   int nB2, OutDesc out, const RopeSpec *rope, unsigned int *status, cudaStream_t st) {
   const int N = nB0 + nB1 + nB2;
   if (!tc_gemm_supported(M, N, K)) return SWIFTKV_ERR_UNSUPPORTED;
   if (out.mode == OUT_STORE_F32) return SWIFTKV_ERR_UNSUPPORTED;
@@ -384,8 +444,16 @@ int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const b
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = N / BN;
   p.out = out; p.act = nullptr; p.F = 0; p.status = status;
-  if (BN == 256) return launch_cfg<256, 4, false>(ta, tb0, tb1, tb2, p, st);
-  return launch_cfg<128, 6, false>(ta, tb0, tb1, tb2, p, st);
+  if (rope) {
+    // fused rotary embedding needs head-aligned tiles of 128-wide heads and a bf16 store
+    if (rope->hd != 128 || out.mode != OUT_STORE || (out.n0 % 128) || (out.n0 < N && (out.seg_w % 128)))
+      return SWIFTKV_ERR_UNSUPPORTED;
+    p.rope_pos = rope->positions; p.cos_tab = rope->cos_tab; p.sin_tab = rope->sin_tab;
+    if (BN == 256) return launch_cfg<256, 4, EPI_ROPE>(ta, tb0, tb1, tb2, p, st);
+    return launch_cfg<128, 6, EPI_ROPE>(ta, tb0, tb1, tb2, p, st);
+  }
+  if (BN == 256) return launch_cfg<256, 4, EPI_PLAIN>(ta, tb0, tb1, tb2, p, st);
+  return launch_cfg<128, 6, EPI_PLAIN>(ta, tb0, tb1, tb2, p, st);
 }
 
 int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
@@ -400,7 +468,7 @@ int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf1
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = F / 128;
   p.out = OutDesc{}; p.act = act; p.F = F; p.status = status;
-  return launch_cfg<256, 4, true>(ta, tg, tu, tu, p, st);
+  return launch_cfg<256, 4, EPI_SWIGLU>(ta, tg, tu, tu, p, st);
 }
 
 }  // namespace skv

@@ -1,78 +1,213 @@
 // The last-token path of SwiftKV prefill: only the last token of each prompt runs layers l+1..L (footnote of
-// Sec. 3.2; Sec. 3.5), so every projection here has at most a handful of rows and is bound by streaming the
-// weights from HBM exactly once, and attention is one query per (prompt, head) over the cache that the
-// SingleInputKV projection filled.
+// Sec. 3.2; Sec. 3.5), so every projection here has at most 8 activation rows and is bound by streaming the
+// weights from HBM exactly once; attention is one query per (prompt, head) over the cache that the
+// SingleInputKV projection filled.  Activations of this path stay in fp32 (they are tiny), weights and the
+// cache stay in the model dtype.
+#include <mma.h>
+
 #include "common.cuh"
 
 namespace skv {
 
 // ---------------------------------------------------------------------------------------------------------
-// skinny GEMM: out[b, n] = sum_k act[b, k] * W[n, k] for b < n_rows <= 8.  One warp per output feature:
-// the lanes stream W's row with 128-bit loads (each byte of W is read once), the few activation rows come
-// from L1/L2, fp32 accumulation, warp-shuffle reduction.
+// RMSNorm of the few continuing rows: fp32 in, fp32 out, gain in the model dtype
 // ---------------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) skinny_gemm_kernel(const T *__restrict__ act, const T *__restrict__ W,
-                                                          int n_rows, int N, int K, OutDesc out) {
-  constexpr int V = 16 / sizeof(T);
+__global__ void __launch_bounds__(256) tail_rmsnorm_kernel(const float *__restrict__ y, const T *__restrict__ gamma,
+                                                           float *__restrict__ out, int d, float eps) {
+  const float *yr = y + (size_t)blockIdx.x * d;
+  float *orow = out + (size_t)blockIdx.x * d;
+  __shared__ float red[8];
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += yr[i] * yr[i];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float rstd = rsqrtf(tot / (float)d + eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x) orow[i] = yr[i] * rstd * to_f(gamma[i]);
+}
+template <typename T>
+void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, int d, float eps, cudaStream_t st) {
+  if (rows > 0) tail_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(y, gamma, out, d, eps);
+}
+template void launch_tail_rmsnorm<float>(const float *, const float *, float *, int, int, float, cudaStream_t);
+template void launch_tail_rmsnorm<bf16>(const float *, const bf16 *, float *, int, int, float, cudaStream_t);
+
+// ---------------------------------------------------------------------------------------------------------
+// Skinny GEMM, generic: out[r, n] = sum_k act[r, k] * W[n, k] for r < n_rows <= 8; one warp per output feature.
+// Used by the fp32 model and for shapes the tensor-core variant does not tile.
+// mode: OUT_STORE_F32 / OUT_RESID_ADD_F32; W2 != nullptr -> out = silu(act W^T) * (act W2^T)  (SwiGLU)
+// ---------------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) skinny_generic_kernel(const float *__restrict__ act, const T *__restrict__ W,
+                                                             const T *__restrict__ W2, int n_rows, int N, int K,
+                                                             float *__restrict__ out, int ldo, int mode) {
   const int lane = threadIdx.x & 31;
   const int warps_total = gridDim.x * (blockDim.x >> 5);
-  const bool vec = (K % V) == 0;
   for (int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); n < N; n += warps_total) {
-    float acc[MAX_TAIL_ROWS];
+    float acc[MAX_TAIL_ROWS], acc2[MAX_TAIL_ROWS];
 #pragma unroll
-    for (int r = 0; r < MAX_TAIL_ROWS; ++r) acc[r] = 0.f;
+    for (int r = 0; r < MAX_TAIL_ROWS; ++r) acc[r] = acc2[r] = 0.f;
     const T *wr = W + (size_t)n * K;
-    if (vec) {
-      for (int k = lane * V; k < K; k += 32 * V) {
-        const uint4 wraw = __ldcs(reinterpret_cast<const uint4 *>(wr + k));   // streamed once: evict first
-        const T *we = reinterpret_cast<const T *>(&wraw);
-        float wf[V];
+    const T *wr2 = W2 ? W2 + (size_t)n * K : nullptr;
+    for (int k = lane; k < K; k += 32) {
+      const float w = to_f(wr[k]);
+      const float w2 = wr2 ? to_f(wr2[k]) : 0.f;
 #pragma unroll
-        for (int i = 0; i < V; ++i) wf[i] = to_f(we[i]);
-#pragma unroll
-        for (int r = 0; r < MAX_TAIL_ROWS; ++r) {
-          if (r < n_rows) {
-            const uint4 araw = *reinterpret_cast<const uint4 *>(act + (size_t)r * K + k);
-            const T *ae = reinterpret_cast<const T *>(&araw);
-#pragma unroll
-            for (int i = 0; i < V; ++i) acc[r] = fmaf(wf[i], to_f(ae[i]), acc[r]);
-          }
+      for (int r = 0; r < MAX_TAIL_ROWS; ++r)
+        if (r < n_rows) {
+          const float a = act[(size_t)r * K + k];
+          acc[r] = fmaf(w, a, acc[r]);
+          acc2[r] = fmaf(w2, a, acc2[r]);
         }
-      }
-    } else {
-      for (int k = lane; k < K; k += 32) {
-        const float w = to_f(wr[k]);
-#pragma unroll
-        for (int r = 0; r < MAX_TAIL_ROWS; ++r)
-          if (r < n_rows) acc[r] = fmaf(w, to_f(act[(size_t)r * K + k]), acc[r]);
-      }
     }
 #pragma unroll
     for (int r = 0; r < MAX_TAIL_ROWS; ++r) {
       if (r < n_rows) {
-        const float s = warp_sum(acc[r]);
-        if (lane == 0) store_out<T>(out, r, n, s);
+        float s = warp_sum(acc[r]);
+        const float s2 = warp_sum(acc2[r]);
+        if (lane == 0) {
+          if (W2) s = s / (1.f + __expf(-s)) * s2;
+          float *o = out + (size_t)r * ldo + n;
+          *o = (mode == OUT_RESID_ADD_F32) ? *o + s : s;
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Skinny GEMM on tensor cores with the operands swapped: the 16 x 16 "A" tile of mma.m16n8k16 holds 16 output
+// features (rows of W) and the 8-wide "B" tile holds the (at most 8) continuing tokens, so no tensor-core
+// work is wasted on padding rows.  Each lane fetches 16 contiguous bytes of two W rows per 32-wide K step
+// straight from global memory; the K index is permuted identically for W and the activations (a dot product
+// does not care), which makes those 16 bytes exactly the lane's fragment of two MMAs.  fp32 activations are
+// split into bf16 hi + lo parts (two MMAs), so the activations keep ~16 mantissa bits.
+// A block = 8 warps works on one 16-feature tile with K split across the warps, then reduces in shared memory.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t &hi, uint32_t &lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  const float2 hf = __bfloat1622float2(h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - hf.x, x1 - hf.y);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+
+constexpr int SK_WARPS = 8;
+
+template <bool SWIGLU>
+__global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *__restrict__ act, const bf16 *__restrict__ W,
+                                                                   const bf16 *__restrict__ W2, int n_rows, int N, int K,
+                                                                   float *__restrict__ out, int ldo, int mode) {
+  __shared__ float red[SK_WARPS][SWIGLU ? 2 : 1][32][4];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int n0 = blockIdx.x * 16;
+  const bf16 *w_lo = W + (size_t)(n0 + g) * K + 8 * t;          // row g of the tile
+  const bf16 *w_hi = W + (size_t)(n0 + g + 8) * K + 8 * t;      // row g + 8
+  const bf16 *u_lo = SWIGLU ? W2 + (size_t)(n0 + g) * K + 8 * t : nullptr;
+  const bf16 *u_hi = SWIGLU ? W2 + (size_t)(n0 + g + 8) * K + 8 * t : nullptr;
+  const float *a_row = act + (size_t)g * K + 8 * t;              // token g
+  const bool tok_ok = g < n_rows;
+  float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+  const int steps = K / 32;
+#pragma unroll 2
+  for (int s = warp; s < steps; s += SK_WARPS) {
+    const int kb = s * 32;
+    const uint4 wl = __ldcs(reinterpret_cast<const uint4 *>(w_lo + kb));   // weights are streamed once
+    const uint4 wh = __ldcs(reinterpret_cast<const uint4 *>(w_hi + kb));
+    uint4 ul, uh;
+    if (SWIGLU) {
+      ul = __ldcs(reinterpret_cast<const uint4 *>(u_lo + kb));
+      uh = __ldcs(reinterpret_cast<const uint4 *>(u_hi + kb));
+    }
+    float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0;
+    if (tok_ok) {
+      x0 = *reinterpret_cast<const float4 *>(a_row + kb);
+      x1 = *reinterpret_cast<const float4 *>(a_row + kb + 4);
+    }
+    uint32_t bh[4], bl[4];
+    split_hi_lo(x0.x, x0.y, bh[0], bl[0]);
+    split_hi_lo(x0.z, x0.w, bh[1], bl[1]);
+    split_hi_lo(x1.x, x1.y, bh[2], bl[2]);
+    split_hi_lo(x1.z, x1.w, bh[3], bl[3]);
+    // first MMA: K slots (2t,2t+1) <- elements 0,1 and (2t+8,2t+9) <- elements 2,3; second MMA: elements 4..7
+    const uint32_t a1[4] = {wl.x, wh.x, wl.y, wh.y}, a2[4] = {wl.z, wh.z, wl.w, wh.w};
+    mma_bf16_16816(c, a1, bh[0], bh[1]);
+    mma_bf16_16816(c, a1, bl[0], bl[1]);
+    mma_bf16_16816(c, a2, bh[2], bh[3]);
+    mma_bf16_16816(c, a2, bl[2], bl[3]);
+    if (SWIGLU) {
+      const uint32_t d1[4] = {ul.x, uh.x, ul.y, uh.y}, d2[4] = {ul.z, uh.z, ul.w, uh.w};
+      mma_bf16_16816(c2, d1, bh[0], bh[1]);
+      mma_bf16_16816(c2, d1, bl[0], bl[1]);
+      mma_bf16_16816(c2, d2, bh[2], bh[3]);
+      mma_bf16_16816(c2, d2, bl[2], bl[3]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    red[warp][0][lane][i] = c[i];
+    if (SWIGLU) red[warp][SWIGLU ? 1 : 0][lane][i] = c2[i];
+  }
+  __syncthreads();
+  if (warp == 0) {
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int w = 0; w < SK_WARPS; ++w)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        s[i] += red[w][0][lane][i];
+        if (SWIGLU) s2[i] += red[w][SWIGLU ? 1 : 0][lane][i];
+      }
+    // fragment element i: feature n0 + g + 8*(i/2), token 2t + (i%2)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int n = n0 + g + 8 * (i >> 1), r = 2 * t + (i & 1);
+      if (r < n_rows && n < N) {
+        float v = s[i];
+        if (SWIGLU) v = v / (1.f + __expf(-v)) * s2[i];
+        float *o = out + (size_t)r * ldo + n;
+        *o = (mode == OUT_RESID_ADD_F32) ? *o + v : v;
       }
     }
   }
 }
 
 template <typename T>
-void launch_skinny_gemm(const T *act, const T *W, int n_rows, int N, int K, OutDesc out, cudaStream_t st) {
+void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
+                        int mode, cudaStream_t st) {
   if (n_rows <= 0 || N <= 0) return;
+  if constexpr (sizeof(T) == 2) {
+    if ((K % 32) == 0 && (N % 16) == 0) {
+      if (W2) skinny_mma_kernel<true><<<N / 16, SK_WARPS * 32, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
+      else skinny_mma_kernel<false><<<N / 16, SK_WARPS * 32, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
+      return;
+    }
+  }
   int blocks = (N + 7) / 8;
   if (blocks > 148 * 8) blocks = 148 * 8;
-  skinny_gemm_kernel<T><<<blocks, 256, 0, st>>>(act, W, n_rows, N, K, out);
+  skinny_generic_kernel<T><<<blocks, 256, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
 }
-template void launch_skinny_gemm<float>(const float *, const float *, int, int, int, OutDesc, cudaStream_t);
-template void launch_skinny_gemm<bf16>(const bf16 *, const bf16 *, int, int, int, OutDesc, cudaStream_t);
+template void launch_skinny_gemm<float>(const float *, const float *, const float *, int, int, int, float *, int, int, cudaStream_t);
+template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, int, int, cudaStream_t);
 
 // ---------------------------------------------------------------------------------------------------------
 // single-query attention over the cache, split along the keys.
-//   pass 1: block (split, head, prompt) scans its key range with 4 warps (online softmax as in the
-//           prefill kernel), merges the warps in shared memory and writes (max, sum, acc[hd]) to scratch;
-//   pass 2: block (head, prompt) merges the splits and writes the normalised output row.
+//   pass 1: block (split, head, prompt) scans its key range with 4 warps -- 32 keys at a time, one key per
+//           lane for the scores (128-bit loads of the K row), online softmax, then the probabilities are
+//           broadcast while the lanes accumulate their slice of the output -- merges the warps in shared
+//           memory and writes (max, sum, acc[hd]) to scratch;
+//   pass 2: block (head, prompt) merges the splits and writes the normalised fp32 output row.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int TAIL_WARPS = 4;
 
@@ -82,9 +217,26 @@ __host__ __device__ inline int tail_chunk(int max_seq_len) {
   return c < 256 ? 256 : c;
 }
 
+template <typename T>
+__device__ __forceinline__ float dot_row(const float *__restrict__ qs, const T *__restrict__ kr, int hd) {
+  constexpr int V = 16 / sizeof(T);
+  float dot = 0.f;
+  if ((hd % V) == 0) {
+    for (int i = 0; i < hd; i += V) {
+      const uint4 raw = *reinterpret_cast<const uint4 *>(kr + i);
+      const T *e = reinterpret_cast<const T *>(&raw);
+#pragma unroll
+      for (int k = 0; k < V; ++k) dot = fmaf(qs[i + k], to_f(e[k]), dot);
+    }
+  } else {
+    for (int i = 0; i < hd; ++i) dot = fmaf(qs[i], to_f(kr[i]), dot);
+  }
+  return dot;
+}
+
 template <typename T, int MAX_E>
 __global__ void __launch_bounds__(TAIL_WARPS * 32) tail_attention_partial_kernel(
-    const T *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
+    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
     int n_q, int n_kv, int hd, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
   extern __shared__ float sm[];   // q[hd] | per-warp (m, l) [2*TAIL_WARPS] | per-warp acc [TAIL_WARPS*hd]
   float *qs = sm;
@@ -95,8 +247,8 @@ __global__ void __launch_bounds__(TAIL_WARPS * 32) tail_attention_partial_kernel
   const int first = cu[b], n = cu[b + 1] - cu[b];
   const int kvh = h / (n_q / n_kv);
   const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
-  const T *qr = q + ((size_t)b * n_q + h) * hd;
-  for (int i = threadIdx.x; i < hd; i += blockDim.x) qs[i] = to_f(qr[i]) * scale;
+  const float *qr = q + ((size_t)b * n_q + h) * hd;
+  for (int i = threadIdx.x; i < hd; i += blockDim.x) qs[i] = qr[i] * scale;
   __syncthreads();
 
   float m = -INFINITY, l = 0.f;
@@ -106,12 +258,7 @@ __global__ void __launch_bounds__(TAIL_WARPS * 32) tail_attention_partial_kernel
   for (int c0 = k_begin + warp * 32; c0 < k_end; c0 += TAIL_WARPS * 32) {
     const int key = c0 + lane;
     float s = -INFINITY;
-    if (key < k_end) {
-      const T *kr = kc + ((size_t)(first + key) * n_kv + kvh) * hd;
-      float dot = 0.f;
-      for (int i = 0; i < hd; ++i) dot = fmaf(qs[i], to_f(kr[i]), dot);
-      s = dot;
-    }
+    if (key < k_end) s = dot_row<T>(qs, kc + ((size_t)(first + key) * n_kv + kvh) * hd, hd);
     const float m_new = fmaxf(m, warp_max(s));
     const float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
     const float corr = __expf(m - m_new);
@@ -153,8 +300,7 @@ __global__ void __launch_bounds__(TAIL_WARPS * 32) tail_attention_partial_kernel
   }
 }
 
-template <typename T>
-__global__ void tail_attention_merge_kernel(const float *__restrict__ scratch, T *__restrict__ out, int n_q, int hd,
+__global__ void tail_attention_merge_kernel(const float *__restrict__ scratch, float *__restrict__ out, int n_q, int hd,
                                             int n_splits) {
   const int h = blockIdx.x, b = blockIdx.y;
   const float *src = scratch + ((size_t)b * n_q + h) * n_splits * (hd + 2);
@@ -171,18 +317,19 @@ __global__ void tail_attention_merge_kernel(const float *__restrict__ scratch, T
       const float ms = src[(size_t)s * (hd + 2)];
       if (ms != -INFINITY) a += src[(size_t)s * (hd + 2) + 2 + dd] * __expf(ms - M);
     }
-    out[((size_t)b * n_q + h) * hd + dd] = from_f<T>(a / L);
+    out[((size_t)b * n_q + h) * hd + dd] = a / L;
   }
 }
 
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens) {
   const int chunk = tail_chunk(max_tokens);
   const int n_splits = (max_tokens + chunk - 1) / chunk;
-  return (size_t)max_seqs * n_q * n_splits * (hd + 2) * sizeof(float);
+  const int rows = max_seqs < MAX_TAIL_ROWS ? max_seqs : MAX_TAIL_ROWS;
+  return (size_t)rows * n_q * n_splits * (hd + 2) * sizeof(float);
 }
 
 template <typename T>
-void launch_tail_attention(const T *q, const T *kc, const T *vc, T *out, const int32_t *cu_seqlens, int n_seqs,
+void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens, int n_seqs,
                            int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st) {
   if (n_seqs <= 0) return;
   const int chunk = tail_chunk(max_seq_len);
@@ -194,11 +341,11 @@ void launch_tail_attention(const T *q, const T *kc, const T *vc, T *out, const i
   else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   else tail_attention_partial_kernel<T, 8><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  tail_attention_merge_kernel<T><<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
+  tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
 template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *, int,
                                            int, int, int, int, float *, cudaStream_t);
-template void launch_tail_attention<bf16>(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int, int,
+template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, float *, const int32_t *, int, int,
                                           int, int, int, float *, cudaStream_t);
 
 }  // namespace skv
