@@ -40,8 +40,18 @@ ORACLE_SAMPLE_TOKENS_PER_PROMPT = 32
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
-# DRAM bytes per SwiGLU-GEMM launch of this workload from the committed ncu capture (profiles/), or None
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM traffic of one fused gate/up GEMM launch.  The committed ncu capture (profiles/gemm_tc_kernel_8b_widths.md)
+# measured 1.2315 GB at T = 8192 tokens: the two weight matrices (235 MB) are re-streamed once per band of 2048
+# rows (4 bands), A (67 MB) and the SwiGLU output (235 MB, 225 MB seen at capture end) move once.  The full
+# workload cannot be captured under the profiling size rule, so the capture is scaled with that model:
+SWIGLU_WEIGHT_BYTES = 2 * 14336 * 4096 * 2
+SWIGLU_CAPTURE_TOKENS, SWIGLU_CAPTURE_BYTES, SWIGLU_BAND_ROWS = 8192, 1.2315e9, 2048
+
+
+def swiglu_traffic_bytes(tokens: int) -> float:
+    per_token = (SWIGLU_CAPTURE_BYTES - (SWIGLU_CAPTURE_TOKENS // SWIGLU_BAND_ROWS) * SWIGLU_WEIGHT_BYTES) / SWIGLU_CAPTURE_TOKENS
+    bands = -(-tokens // SWIGLU_BAND_ROWS)
+    return bands * SWIGLU_WEIGHT_BYTES + per_token * tokens
 
 
 def measured_peaks():
@@ -108,6 +118,23 @@ def flops_of(lens, l, g):
     from paper_2410_03960_b200 import prefill_flops
     s = SHAPE
     return prefill_flops(s.hidden, s.n_layers, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn, s.vocab, lens, l, g)
+
+
+def rank_batch(rank: int):
+    """Replicas only: rank 0 runs exactly the named batch, every other rank an independent batch of the same recipe."""
+    seed = SEED + 1000 * rank
+    return seed, S.uniform_lengths(seed, N_PROMPTS, LEN_LO, LEN_HI)
+
+
+def reduce_over_ranks(times, tokens: float, device, use_dist: bool):
+    """Whole-job figures: the slowest rank's device time for each timed region, the sum of all ranks' tokens."""
+    t = torch.tensor(list(times), dtype=torch.float64, device=device)
+    n = torch.tensor([tokens], dtype=torch.float64, device=device)
+    if use_dist:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return t.tolist(), n.item()
 
 
 def time_steps(fn, steps, dist_barrier):
@@ -202,8 +229,7 @@ def run_ours(args, rank, world, local_rank):
         def barrier():
             pass
 
-    seed = SEED + 1000 * rank                      # rank 0 runs exactly the named batch; replicas differ
-    lens = S.uniform_lengths(seed, N_PROMPTS, LEN_LO, LEN_HI)
+    seed, lens = rank_batch(rank)
     T = sum(lens)
     tok_host = S.make_prompts(seed, lens, SHAPE.vocab).pin_memory()
     tok_dev = tok_host.to(dev)
@@ -259,14 +285,7 @@ def run_ours(args, rank, world, local_rank):
     t_full = time_steps(step_full, args.steps, barrier)
     model.status()
 
-    tokens_total = float(T * args.steps)
-    times = torch.tensor([t_swift, t_e2e, t_full], dtype=torch.float64, device=dev)
-    toks = torch.tensor([tokens_total], dtype=torch.float64, device=dev)
-    if use_dist:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    t_swift, t_e2e, t_full = times.tolist()
-    tokens_all = toks.item()
+    (t_swift, t_e2e, t_full), tokens_all = reduce_over_ranks([t_swift, t_e2e, t_full], float(T * args.steps), dev, use_dist)
 
     if rank == 0:
         peaks, peaks_kind = measured_peaks()
@@ -274,8 +293,11 @@ def run_ours(args, rank, world, local_rank):
         ms_step = t_swift / args.steps * 1e3
         actual_tflops = f_sw["total"] / (t_swift / args.steps) / 1e12
         norm_tflops = f_full["total"] / (t_swift / args.steps) / 1e12
-        gemm_ms, gemm_launches = prof["gemm"]
+        gemm_ms = prof["gemm"][0] + prof["gemm_swiglu"][0]
         gemm_ach = f_sw["gemm"] * args.steps / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else None
+        sw_ms, sw_launches = prof["gemm_swiglu"]
+        sw_flops_per_launch = 2.0 * T * (2 * SHAPE.ffn) * SHAPE.hidden
+        sw_ach = sw_flops_per_launch / (sw_ms / sw_launches / 1e3) / 1e12 if sw_launches else None
         peak = peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"]
         attn_ms = prof["attention"][0]
         line = {
@@ -297,12 +319,16 @@ def run_ours(args, rank, world, local_rank):
                     "d2h_bytes_per_step": N_PROMPTS * SHAPE.vocab * 4},
             "gpu_launches": launches,
             "clocks": clocks,
-            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (all projection / MLP / SingleInputKV GEMM launches)",
-                         "achieved": gemm_ach, "peak": peak, "unit": "TFLOP/s",
-                         "frac": (gemm_ach / peak) if gemm_ach else None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
-                         "frac_of_burst": (gemm_ach / peaks["bf16_tflops"]) if gemm_ach else None,
-                         "launches_per_step": gemm_launches // max(args.steps, 1), "ms_per_step": gemm_ms / args.steps,
-                         "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH},
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel<256,4,SWIGLU>: fused gate/up projection + SwiGLU, "
+                                                       "M=T, N=2*14336, K=4096 (dominant kernel)",
+                         "achieved": sw_ach, "peak": peak, "unit": "TFLOP/s",
+                         "frac": (sw_ach / peak) if sw_ach else None, "peak_kind": f"{peaks_kind} sustained cuBLAS bf16",
+                         "frac_of_burst": (sw_ach / peaks["bf16_tflops"]) if sw_ach else None,
+                         "flops_per_launch": sw_flops_per_launch,
+                         "launches_per_step": sw_launches // max(args.steps, 1), "ms_per_launch": sw_ms / max(sw_launches, 1),
+                         "traffic": swiglu_traffic_bytes(T),
+                         "traffic_note": "scaled from the ncu capture at 8192 tokens (see profiles/)",
+                         "all_gemms_tflops": gemm_ach, "all_gemms_ms_per_step": gemm_ms / args.steps},
             "time_share_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
             "attention_tflops": (f_sw["attention"] * args.steps / (attn_ms / 1e3) / 1e12) if attn_ms > 0 else None,
         }

@@ -93,8 +93,8 @@ int32_t swiftkv_workspace_bytes(const swiftkv_config *cfg, int32_t max_tokens, i
                                 size_t *workspace_bytes, size_t *kv_cache_bytes);
 
 /*
- * Create a model over caller-owned device buffers.  Records the (borrowed) weight pointers, builds the TMA
- * descriptors of the weight matrices and fills the RoPE table (cos/sin of p * theta^(-2i/hd), evaluated in
+ * Create a model over caller-owned device buffers.  Records the (borrowed) weight pointers and fills the RoPE
+ * table (cos/sin of p * theta^(-2i/hd), evaluated in
  * double precision, rotate-half pairing (i, i + hd/2)) on the current device's default stream, then
  * synchronises that stream.  The device current at this call is the model's device.
  * Errors: INVALID_ARG (as above, or a null / misaligned pointer), WORKSPACE_SMALL, CUDA.
@@ -164,11 +164,12 @@ int32_t swiftkv_status(swiftkv_model *m, void *cuda_stream);
  * prefill's stream; swiftkv_profile_read synchronises the stream and returns the device time (ms) and launch
  * count accumulated per class since the last read, then resets them.  Classes are SWIFTKV_KC_*.
  */
-#define SWIFTKV_KC_GEMM      0   /* projection / MLP / SingleInputKV GEMMs (M = all prompt tokens)       */
+#define SWIFTKV_KC_GEMM      0   /* QKV / O / down / SingleInputKV GEMMs (M = all prompt tokens)          */
 #define SWIFTKV_KC_ATTENTION 1   /* causal varlen GQA prefill attention                                   */
 #define SWIFTKV_KC_ELEMWISE  2   /* embedding gather, RMSNorm, RoPE, SwiGLU, gathers, weight fold         */
 #define SWIFTKV_KC_TAIL      3   /* last-token path of layers > l and the lm_head                         */
-#define SWIFTKV_KC_COUNT     4
+#define SWIFTKV_KC_SWIGLU    4   /* the fused gate/up GEMM + SwiGLU, the single largest kernel            */
+#define SWIFTKV_KC_COUNT     5
 int32_t swiftkv_profile_enable(swiftkv_model *m, int32_t on);
 int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, float *ms_per_class /*[KC_COUNT]*/,
                              int32_t *launches_per_class /*[KC_COUNT]*/);

@@ -11,7 +11,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB: Optional[C.CDLL] = None
 
 DTYPE_F32, DTYPE_BF16 = 0, 1
-KC_NAMES = ("gemm", "attention", "elementwise", "tail")
+KC_NAMES = ("gemm", "attention", "elementwise", "tail", "gemm_swiglu")
 
 # every symbol include/swiftkv.h declares
 EXPORTS = (

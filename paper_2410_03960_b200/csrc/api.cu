@@ -328,7 +328,7 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
     bool fused = false;
     if constexpr (sizeof(T) == 2) {
       if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d)) {
-        Scope s(m, st, SWIFTKV_KC_GEMM);
+        Scope s(m, st, SWIFTKV_KC_SWIGLU);
         rc = launch_gemm_tc_swiglu(h, T_tok, d, (const bf16 *)lw.w_gate, (const bf16 *)lw.w_up, F, act, b.status, st);
         if (rc == SWIFTKV_OK) fused = true;
         else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "SwiGLU GEMM launch failed");
