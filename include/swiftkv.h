@@ -202,6 +202,19 @@ int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, v
                                   int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                   int32_t dtype, int32_t use_tensor_cores, void *cuda_stream);
 
+/* Single-query attention of the last-token path (footnote of Sec. 3.2: the last prompt token still runs every
+ * layer; Sec. 3.5: it attends to the caches the SingleInputKV projection filled).  One query per prompt:
+ * q DEVICE fp32 [n_seqs, n_q, hd] (already rotated); k_cache, v_cache DEVICE [total_tokens, n_kv, hd] in `dtype`,
+ * prompt b occupying rows [cu_seqlens[b], cu_seqlens[b+1]); out DEVICE fp32 [n_seqs, n_q*hd]; softmax scale
+ * 1/sqrt(hd).  n_seqs <= 8.  The keys are split across CTAs; `scratch` (DEVICE, caller-owned, at least
+ * swiftkv_tail_attention_scratch_bytes(...) bytes, 16-byte aligned) holds the per-split partial results.
+ * Errors: INVALID_ARG, WORKSPACE_SMALL (scratch too small), CUDA. */
+size_t  swiftkv_tail_attention_scratch_bytes(int32_t n_seqs, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len);
+int32_t swiftkv_tail_attention(const float *q, const void *k_cache, const void *v_cache, float *out,
+                               const int32_t *cu_seqlens, int32_t n_seqs, int32_t max_seq_len, int32_t n_q_heads,
+                               int32_t n_kv_heads, int32_t head_dim, int32_t dtype, void *scratch, size_t scratch_bytes,
+                               void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

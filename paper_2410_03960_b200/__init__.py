@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     gemm_bf16,
     library_path,
     load_library,
+    tail_attention,
     workspace_bytes,
 )
 from .flops import prefill_flops  # noqa: F401

@@ -18,7 +18,8 @@ EXPORTS = (
     "swiftkv_version", "swiftkv_last_error", "swiftkv_workspace_bytes", "swiftkv_model_load", "swiftkv_prefill",
     "swiftkv_prefill_device_tokens", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
-    "swiftkv_model_free", "swiftkv_gemm_bf16", "swiftkv_attention_prefill",
+    "swiftkv_model_free", "swiftkv_gemm_bf16", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
+    "swiftkv_tail_attention",
 )
 
 
@@ -79,6 +80,9 @@ def load_library() -> C.CDLL:
     lib.swiftkv_model_free.restype = None
     lib.swiftkv_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 8 + [C.c_void_p]
+    lib.swiftkv_tail_attention_scratch_bytes.argtypes = [C.c_int32] * 4
+    lib.swiftkv_tail_attention_scratch_bytes.restype = C.c_size_t
+    lib.swiftkv_tail_attention.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
     _LIB = lib
     return lib
 
@@ -235,4 +239,30 @@ def attention_prefill(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_len
         _check(load_library().swiftkv_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                                         cu_dev.data_ptr(), len(seq_lens), t, max(seq_lens), n_q, n_kv, hd,
                                                         code, int(use_tensor_cores), _stream_ptr(stream)))
+    return out
+
+
+def _cu_seqlens(seq_lens: Sequence[int], device) -> torch.Tensor:
+    cu = [0]
+    for n in seq_lens:
+        cu.append(cu[-1] + int(n))
+    return torch.tensor(cu, dtype=torch.int32, device=device)
+
+
+def tail_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, seq_lens: Sequence[int],
+                   stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_tail_attention: q fp32 [n_seqs, n_q, hd]; caches [T, n_kv, hd] (bf16 or fp32) -> fp32 [n_seqs, n_q*hd]."""
+    assert q.is_cuda and q.dtype == torch.float32 and q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous()
+    b, n_q, hd = q.shape
+    n_kv = k_cache.shape[1]
+    lib = load_library()
+    cu = _cu_seqlens(seq_lens, q.device)
+    nbytes = lib.swiftkv_tail_attention_scratch_bytes(b, n_q, hd, max(seq_lens))
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    out = torch.empty((b, n_q * hd), dtype=torch.float32, device=q.device)
+    code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[k_cache.dtype]
+    with torch.cuda.device(q.device):
+        _check(lib.swiftkv_tail_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr(), cu.data_ptr(),
+                                          b, max(seq_lens), n_q, n_kv, hd, code, scratch.data_ptr(), nbytes,
+                                          _stream_ptr(stream)))
     return out

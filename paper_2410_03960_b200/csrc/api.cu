@@ -571,3 +571,34 @@ extern "C" int32_t swiftkv_attention_prefill(const void *q, const void *k, const
   if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
   return SWIFTKV_OK;
 }
+
+extern "C" size_t swiftkv_tail_attention_scratch_bytes(int32_t n_seqs, int32_t n_q_heads, int32_t head_dim,
+                                                       int32_t max_seq_len) {
+  if (n_seqs < 1 || n_q_heads < 1 || head_dim < 1 || max_seq_len < 1) return 0;
+  return tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len);
+}
+
+extern "C" int32_t swiftkv_tail_attention(const float *q, const void *k_cache, const void *v_cache, float *out,
+                                          const int32_t *cu_seqlens, int32_t n_seqs, int32_t max_seq_len,
+                                          int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,
+                                          void *scratch, size_t scratch_bytes, void *cuda_stream) {
+  if (!q || !k_cache || !v_cache || !out || !cu_seqlens || !scratch) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (n_seqs < 1 || n_seqs > MAX_TAIL_ROWS || max_seq_len < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
+      head_dim < 2 || head_dim > 256)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "bad shape (n_seqs must be in [1, %d])", MAX_TAIL_ROWS);
+  if (scratch_bytes < tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len))
+    return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "scratch %zu < %zu bytes", scratch_bytes,
+                tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len));
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (dtype == SWIFTKV_DTYPE_BF16)
+    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, n_seqs, max_seq_len, n_q_heads,
+                                n_kv_heads, head_dim, (float *)scratch, st);
+  else if (dtype == SWIFTKV_DTYPE_F32)
+    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, n_seqs, max_seq_len,
+                                 n_q_heads, n_kv_heads, head_dim, (float *)scratch, st);
+  else
+    return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}

@@ -65,3 +65,23 @@ def test_attention_tcgen05(lens, n_q, n_kv):
         assert rel_l2(got, ref) < 1e-2, (n, rel_l2(got, ref))
         assert np.max(np.abs(got - ref)) < 0.05
         off += n
+
+
+@pytest.mark.parametrize("dtype,bar", [(torch.float32, 1e-5), (torch.bfloat16, 1e-5)])
+@pytest.mark.parametrize("lens,n_q,n_kv,hd", [([5, 1, 70], 8, 2, 32), ([1000, 3000, 257], 8, 2, 128), ([20000], 4, 1, 128),
+                                              ([300] * 8, 32, 8, 128)])
+def test_tail_attention(dtype, bar, lens, n_q, n_kv, hd):
+    """One query per prompt over its cache rows, keys split across CTAs, against the oracle's definition.  The
+    cache values are exactly representable (bf16 inputs are upcast), so only fp32 arithmetic separates the two."""
+    import paper_2410_03960_b200 as P
+    T, B = sum(lens), len(lens)
+    q = S.matrix(6, 1, B, n_q * hd, torch.float32, "cuda", std=1.0).view(B, n_q, hd)
+    k = S.matrix(6, 2, T, n_kv * hd, dtype, "cuda", std=1.0).view(T, n_kv, hd)
+    v = S.matrix(6, 3, T, n_kv * hd, dtype, "cuda", std=1.0).view(T, n_kv, hd)
+    out = P.tail_attention(q, k, v, lens)
+    torch.cuda.synchronize()
+    off = 0
+    for b, n in enumerate(lens):
+        ref = O.single_query_attention(to_np(q[b]), to_np(k[off:off + n]), to_np(v[off:off + n]))
+        assert rel_l2(to_np(out[b]), ref) < bar
+        off += n
