@@ -215,6 +215,28 @@ int32_t swiftkv_tail_attention(const float *q, const void *k_cache, const void *
                                int32_t n_kv_heads, int32_t head_dim, int32_t dtype, void *scratch, size_t scratch_bytes,
                                void *cuda_stream);
 
+/* (No counterpart in the paper: an integration aid.)
+ * swiftkv_tail_attention for callers that must not allocate device memory and have no spare buffer to lend --
+ * for example a plug-in running inside a serving process whose memory pool is fully committed to weights and KV
+ * cache, or code running where cudaMalloc is forbidden (between a stream-capture begin/end, in a latency-critical
+ * loop, under a memory-accounting harness).  Same arguments and result as swiftkv_tail_attention minus the
+ * scratch pair: the per-split partial results live in a fixed array inside the library's device image instead.
+ *   - Limit: that array is SWIFTKV_NOALLOC_SCRATCH_BYTES (9 MiB); it exists once per GPU that loads the library
+ *     and stays until the process exits.  A call whose partials need more (see
+ *     swiftkv_tail_attention_scratch_bytes) is rejected with SWIFTKV_ERR_WORKSPACE_SMALL and does nothing.
+ *   - The first call on each device looks up the array's device address (no allocation); make that first call
+ *     outside any stream capture.
+ *   - The array is shared by every call in the process and keeps whatever the previous call left; each call
+ *     overwrites every entry it later reads, so nothing needs clearing, but two calls that overlap on the GPU
+ *     (different streams, or different host threads) race on it: serialise them.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA. */
+#define SWIFTKV_NOALLOC_SCRATCH_BYTES (9u * 1024u * 1024u)
+int32_t swiftkv_tail_attention_noalloc(const float *q, const void *k_cache, const void *v_cache, float *out,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int32_t max_seq_len,
+                                       int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t dtype,
+                                       void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -12,6 +12,7 @@ from .binding import (  # noqa: F401
     library_path,
     load_library,
     tail_attention,
+    tail_attention_noalloc,
     workspace_bytes,
 )
 from .flops import prefill_flops  # noqa: F401

@@ -19,7 +19,7 @@ EXPORTS = (
     "swiftkv_prefill_device_tokens", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
     "swiftkv_model_free", "swiftkv_gemm_bf16", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
-    "swiftkv_tail_attention",
+    "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc",
 )
 
 
@@ -83,6 +83,7 @@ def load_library() -> C.CDLL:
     lib.swiftkv_tail_attention_scratch_bytes.argtypes = [C.c_int32] * 4
     lib.swiftkv_tail_attention_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_tail_attention.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.swiftkv_tail_attention_noalloc.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p]
     _LIB = lib
     return lib
 
@@ -266,3 +267,18 @@ def tail_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor
                                           b, max(seq_lens), n_q, n_kv, hd, code, scratch.data_ptr(), nbytes,
                                           _stream_ptr(stream)))
     return out
+
+
+def tail_attention_noalloc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, out: torch.Tensor,
+                           cu_seqlens: torch.Tensor, max_seq_len: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """swiftkv_tail_attention_noalloc: like tail_attention, but the library keeps the split-KV partials in its own
+    fixed device array, so neither this wrapper nor the library allocates anything: the caller passes the output
+    tensor and the prompt offsets (device int32 [n_seqs+1]).  For callers whose memory is fully committed or who may
+    not call the allocator where they run; problems needing more than 9 MiB of partials raise SwiftKVError(-2)."""
+    b, n_q, hd = q.shape
+    n_kv = k_cache.shape[1]
+    code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[k_cache.dtype]
+    with torch.cuda.device(q.device):
+        _check(load_library().swiftkv_tail_attention_noalloc(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                                             out.data_ptr(), cu_seqlens.data_ptr(), b, max_seq_len, n_q, n_kv,
+                                                             hd, code, _stream_ptr(stream)))

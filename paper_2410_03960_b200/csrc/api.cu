@@ -28,6 +28,10 @@ static int32_t fail(int32_t code, const char *fmt, ...) {
   g_last_error = buf;
   return code;
 }
+namespace skv {
+// records the calling thread's last-error text for entry points defined in other translation units
+int32_t report_error(int32_t code, const char *msg) { return fail(code, "%s", msg); }
+}  // namespace skv
 #define CUDA_TRY(expr)                                                                                   \
   do {                                                                                                   \
     cudaError_t e__ = (expr);                                                                            \

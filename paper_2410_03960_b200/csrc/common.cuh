@@ -68,6 +68,9 @@ __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, fl
 }
 #endif
 
+// sets the calling thread's swiftkv_last_error() text and returns `code` (defined with the C ABI)
+int32_t report_error(int32_t code, const char *msg);
+
 // ---- launch prototypes (each queues work on `st`, no synchronisation) -------------------------------------
 // elementwise.cu
 template <typename T>
