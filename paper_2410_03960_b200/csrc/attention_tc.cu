@@ -207,20 +207,27 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!wait_or_abort(tc::smem_u32(&s_full[w]), j & 1, abort_flag, p.status)) { ok = false; break; }
       tc::tc_fence_after_sync();
       const bool diag = (j == qt);
-      // pass 1: row max of the raw scores
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32b_x32(t_s + ch * 32, r);
-        tc::tmem_ld_wait();
+      // the whole score row (128 fp32) in registers: one pass over tensor memory
+      uint32_t s[128];
+      tc::tmem_ld_32x32b_x32p(t_s, s);
+      tc::tmem_ld_32x32b_x32p(t_s + 32, s + 32);
+      tc::tmem_ld_32x32b_x32p(t_s + 64, s + 64);
+      tc::tmem_ld_32x32b_x32p(t_s + 96, s + 96);
+      tc::tmem_ld_wait();
+      if (diag) {   // causal mask, only on the diagonal tile: key index > query index
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float v = __uint_as_float(r[i]);
-          if (diag && (ch * 32 + i > row)) v = -INFINITY;
-          mx = fmaxf(mx, v);
-        }
+        for (int i = 0; i < 128; ++i)
+          if (i > row) s[i] = 0xff800000u;   // -inf
       }
+      float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 8) {
+        m0 = tc::max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        m1 = tc::max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        m2 = tc::max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        m3 = tc::max3(m3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+      }
+      const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
       // move the reference max only when the running max outgrew it by more than the threshold
       const bool need = (j == 0) || ((mx - m_ref) * c > RESCALE_THRESHOLD);
       const float m_new = need ? mx : m_ref;
@@ -239,27 +246,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
       }
       m_ref = m_new;
-      // pass 2: p = 2^(s*c - m_ref*c), row sum, bf16 P written over S (64 packed columns)
+      // p = 2^(s*c - m_ref*c) (masked entries: 2^-inf = 0), row sum, bf16 P written over S (64 packed columns)
       const float neg_mc = -m_ref * c;
-#pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32b_x32(t_s + ch * 32, r);
-        tc::tmem_ld_wait();
-        uint32_t pk[16];
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * i]), c, neg_mc));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * i + 1]), c, neg_mc));
-          if (diag) {
-            if (ch * 32 + 2 * i > row) p0 = 0.f;
-            if (ch * 32 + 2 * i + 1 > row) p1 = 0.f;
-          }
-          l += p0 + p1;
-          pk[i] = tc::pack_bf16x2(p0, p1);
-        }
-        tc::tmem_st_32x32b_x16(t_s + ch * 16, pk);
+      for (int i = 0; i < 64; i += 2) {
+        const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, neg_mc));
+        const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, neg_mc));
+        const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 2]), c, neg_mc));
+        const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 3]), c, neg_mc));
+        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+        s[i] = tc::pack_bf16x2(p0, p1);
+        s[i + 1] = tc::pack_bf16x2(p2, p3);
       }
+      l += (l0 + l1) + (l2 + l3);
+      tc::tmem_st_32x32b_x32(t_s, s);
+      tc::tmem_st_32x32b_x32(t_s + 32, s + 32);
       tc::tmem_st_wait();
       tc::tc_fence_before_sync();
       __syncwarp();
