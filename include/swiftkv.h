@@ -47,6 +47,7 @@ extern "C" {
 
 #define SWIFTKV_DTYPE_F32  0
 #define SWIFTKV_DTYPE_BF16 1
+#define SWIFTKV_DTYPE_F16  2   /* IEEE half: only as the activation type of the stand-alone operators */
 
 typedef struct swiftkv_model swiftkv_model;   /* opaque, library-owned host object */
 
@@ -181,6 +182,18 @@ int32_t swiftkv_last_launch_count(const swiftkv_model *m);
  * Default: all that the model's shape and dtype support.  Returns the mask in effect. */
 int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
+/* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention
+ * output, SwiGLU output, softmax probabilities) -- never of weights or the KV cache, which stay bf16.
+ *   SWIFTKV_ACT_F16  (default): IEEE half, 8x finer rounding than bf16; conversions saturate at +-65504.  Because
+ *                      both operands of a tensor-core MMA must share one 16-bit type, each layer's matrices are
+ *                      copied to half right before use (workspace scratch for one layer; exact for |w| >= 2^-17)
+ *                      and the current layer's K / V get a half copy beside the bf16 cache.
+ *   SWIFTKV_ACT_BF16          : bfloat16 end to end, for checkpoints whose activations exceed the half range.
+ * Ignored by fp32 models.  Takes effect at the next prefill. */
+#define SWIFTKV_ACT_BF16 0
+#define SWIFTKV_ACT_F16  1
+int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format);
+
 /* Destroys the host object (never the caller's buffers).  Null is allowed. */
 void swiftkv_model_free(swiftkv_model *m);
 
@@ -189,18 +202,20 @@ void swiftkv_model_free(swiftkv_model *m);
  * All pointers are DEVICE memory; all run on `cuda_stream` without synchronising.
  */
 
-/* C[M,N] = A[M,K] * B[N,K]^T, bf16 in, fp32 accumulate on the tensor cores (tcgen05), bf16 out, row-major,
- * ldc = N.  Needs K % 64 == 0, N % 128 == 0, 16-byte aligned pointers.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
-int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
-                          void *cuda_stream);
+/* C[M,N] = A[M,K] * B[N,K]^T on the tensor cores (tcgen05), fp32 accumulation, row-major, ldc = N.  A, B and C
+ * are all of `dtype` (SWIFTKV_DTYPE_BF16 or SWIFTKV_DTYPE_F16; the two operands of one MMA must share a type).
+ * Needs K % 64 == 0, N % 128 == 0, 16-byte aligned pointers.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K, int32_t dtype,
+                        void *cuda_stream);
 
-/* Causal varlen grouped-query attention (Sec. 3.1) on packed prompts.  q [T, n_q, hd], k, v [T, n_kv, hd],
- * out [T, n_q*hd] in `dtype`; cu_seqlens DEVICE int32 [n_seqs+1]; softmax scale 1/sqrt(hd).
- * max_seq_len bounds the longest prompt (grid sizing). */
+/* Causal varlen grouped-query attention (Sec. 3.1) on packed prompts.  q [T, n_q, hd] and out [T, n_q*hd] in
+ * q_dtype, k, v [T, n_kv, hd] in kv_dtype; cu_seqlens DEVICE int32 [n_seqs+1]; softmax scale 1/sqrt(hd).
+ * max_seq_len bounds the longest prompt (grid sizing).  Type pairs: (F32, F32), (BF16, BF16), (F16, BF16) on the
+ * SIMT kernel; (BF16, BF16) or (F16, F16), head_dim 128 and an even n_q / n_kv on the tensor-core kernel. */
 int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, void *out,
                                   const int32_t *cu_seqlens, int32_t n_seqs, int32_t total_tokens,
                                   int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
-                                  int32_t dtype, int32_t use_tensor_cores, void *cuda_stream);
+                                  int32_t q_dtype, int32_t kv_dtype, int32_t use_tensor_cores, void *cuda_stream);
 
 /* Single-query attention of the last-token path (footnote of Sec. 3.2: the last prompt token still runs every
  * layer; Sec. 3.5: it attends to the caches the SingleInputKV projection filled).  One query per prompt:

@@ -4,11 +4,13 @@ Every step of the prefill runs in the library's kernels; this package only marsh
 PyTorch is used for device memory and streams.
 """
 from .binding import (  # noqa: F401
+    ACT_BF16,
+    ACT_F16,
     KC_NAMES,
     SwiftKVError,
     SwiftKVModel,
     attention_prefill,
-    gemm_bf16,
+    gemm_tc,
     library_path,
     load_library,
     tail_attention,

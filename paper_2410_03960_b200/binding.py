@@ -10,7 +10,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB: Optional[C.CDLL] = None
 
-DTYPE_F32, DTYPE_BF16 = 0, 1
+DTYPE_F32, DTYPE_BF16, DTYPE_F16 = 0, 1, 2
+ACT_BF16, ACT_F16 = 0, 1
+_DTYPE_CODE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 KC_NAMES = ("gemm", "attention", "elementwise", "tail", "gemm_swiglu")
 
 # every symbol include/swiftkv.h declares
@@ -18,7 +20,7 @@ EXPORTS = (
     "swiftkv_version", "swiftkv_last_error", "swiftkv_workspace_bytes", "swiftkv_model_load", "swiftkv_prefill",
     "swiftkv_prefill_device_tokens", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
-    "swiftkv_model_free", "swiftkv_gemm_bf16", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
+    "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc",
 )
 
@@ -78,8 +80,9 @@ def load_library() -> C.CDLL:
     lib.swiftkv_set_kernel_mask.argtypes = [C.c_void_p, C.c_int32]
     lib.swiftkv_model_free.argtypes = [C.c_void_p]
     lib.swiftkv_model_free.restype = None
-    lib.swiftkv_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
-    lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 8 + [C.c_void_p]
+    lib.swiftkv_set_activation_format.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+    lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
     lib.swiftkv_tail_attention_scratch_bytes.argtypes = [C.c_int32] * 4
     lib.swiftkv_tail_attention_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_tail_attention.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
@@ -211,15 +214,21 @@ class SwiftKVModel:
     def set_kernel_mask(self, mask: int) -> int:
         return int(self.lib.swiftkv_set_kernel_mask(self._h, mask))
 
+    def set_activation_format(self, fmt: int) -> None:
+        """swiftkv_set_activation_format: ACT_F16 (default) or ACT_BF16."""
+        _check(self.lib.swiftkv_set_activation_format(self._h, fmt))
 
-def gemm_bf16(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-    """swiftkv_gemm_bf16: C = A @ B.T with A [M, K], B [N, K] bf16 CUDA tensors."""
-    assert a.is_cuda and b.is_cuda and a.dtype == b.dtype == torch.bfloat16 and a.is_contiguous() and b.is_contiguous()
+
+def gemm_tc(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_gemm_tc: C = A @ B.T with A [M, K], B [N, K] CUDA tensors, both bf16 or both fp16; C has their dtype."""
+    assert a.is_cuda and b.is_cuda and b.dtype == a.dtype and a.dtype in (torch.bfloat16, torch.float16)
+    assert a.is_contiguous() and b.is_contiguous()
     m, k = a.shape
     n = b.shape[0]
-    c = torch.empty((m, n), dtype=torch.bfloat16, device=a.device)
+    c = torch.empty((m, n), dtype=a.dtype, device=a.device)
     with torch.cuda.device(a.device):
-        _check(load_library().swiftkv_gemm_bf16(a.data_ptr(), b.data_ptr(), c.data_ptr(), m, n, k, _stream_ptr(stream)))
+        _check(load_library().swiftkv_gemm_tc(a.data_ptr(), b.data_ptr(), c.data_ptr(), m, n, k, _DTYPE_CODE[a.dtype],
+                                              _stream_ptr(stream)))
     return c
 
 
@@ -235,11 +244,11 @@ def attention_prefill(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_len
     assert cu[-1] == t
     cu_dev = torch.tensor(cu, dtype=torch.int32, device=q.device)
     out = torch.empty((t, n_q * hd), dtype=q.dtype, device=q.device)
-    code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[q.dtype]
     with torch.cuda.device(q.device):
         _check(load_library().swiftkv_attention_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                                         cu_dev.data_ptr(), len(seq_lens), t, max(seq_lens), n_q, n_kv, hd,
-                                                        code, int(use_tensor_cores), _stream_ptr(stream)))
+                                                        _DTYPE_CODE[q.dtype], _DTYPE_CODE[k.dtype], int(use_tensor_cores),
+                                                        _stream_ptr(stream)))
     return out
 
 

@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "common.cuh"
@@ -59,6 +60,8 @@ struct Buffers {
   void *gate, *up;          // unfused MLP scratch [mlp_chunk, F] each
   void *act;                // SwiGLU output [T, F]
   void *wfold;              // folded, concatenated SingleInputKV weight [n_groups*2*d_kv, d]
+  void *w16;                // bf16 models: IEEE-half compute copy of ONE layer's seven matrices (refilled per layer)
+  void *kv16;               // bf16 models: half copies of the current layer's K and V, [2][T, d_kv]
   float *y;                 // continuing tokens' residual [B, d]
   float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
   float *tail_scratch;
@@ -84,9 +87,10 @@ struct swiftkv_model {
   // state of the last prefill
   bool ready = false;
   int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;
-  int fold_l = -1, fold_g = -1;
+  int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
   int kernel_mask = 3;
+  int act_format = SWIFTKV_ACT_F16;
   // profiling
   bool profiling = false;
   std::vector<cudaEvent_t> pool;
@@ -124,6 +128,10 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.up = cv.take(chunk * F * E);
   b.act = cv.take((size_t)T * F * E);
   b.wfold = cv.take(fold_elems * E);
+  const size_t dkv_ = (size_t)c.n_kv_heads * c.head_dim;
+  const bool bf = c.dtype == SWIFTKV_DTYPE_BF16;
+  b.w16 = cv.take(bf ? (2 * d * dq + 2 * d * dkv_ + 3 * d * F) * 2 : 0);
+  b.kv16 = cv.take(bf ? (size_t)2 * T * dkv_ * 2 : 0);
   b.y = (float *)cv.take((size_t)B * d * 4);
   const size_t R = std::min<size_t>(B, MAX_TAIL_ROWS);
   b.hy = (float *)cv.take(R * std::max(d, dq) * 4);
@@ -247,42 +255,64 @@ struct Scope {
 // ---------------------------------------------------------------------------------------------------------
 // the schedule
 // ---------------------------------------------------------------------------------------------------------
+// TA: storage type of the activations that feed GEMMs and attention (h, q, attention output, SwiGLU output):
+//     float for an fp32 model; for a bf16 model either bf16 or IEEE half (8x finer rounding, saturating).
+// TW: storage type of weights and of the KV cache (the model dtype).
 // rope_fused (optional): in: request the rotary embedding in the epilogue; out: whether it was applied
-template <typename T>
-static int32_t gemm_any(swiftkv_model *m, const T *A, int M, int K, const T *B0, int n0, const T *B1, int n1,
-                        const T *B2, int n2, const OutDesc &out, cudaStream_t st, const RopeSpec *rope = nullptr,
-                        bool *rope_fused = nullptr) {
+// Bh0..2 (optional): IEEE-half copies of B0..2, used by the tensor-core path when TA is half (both MMA operands must
+// have the same 16-bit type); dup: half copy of the segment columns (see launch_gemm_tc)
+template <typename TA, typename TW>
+static int32_t gemm_any(swiftkv_model *m, const TA *A, int M, int K, const TW *B0, int n0, const TW *B1, int n1,
+                        const TW *B2, int n2, const OutDesc &out, cudaStream_t st, const __half *Bh0 = nullptr,
+                        const __half *Bh1 = nullptr, const __half *Bh2 = nullptr, const RopeSpec *rope = nullptr,
+                        bool *rope_fused = nullptr, void *dup = nullptr, long long dup_stride = 0) {
   Scope sc(m, st, SWIFTKV_KC_GEMM, 0);
   if (rope_fused) *rope_fused = false;
-  if constexpr (sizeof(T) == 2) {
-    if ((m->kernel_mask & 1) && tc_gemm_supported(M, n0 + n1 + n2, K)) {
+  if constexpr (sizeof(TW) == 2) {
+    constexpr bool f16 = std::is_same<TA, __half>::value;
+    const bool have_b = !f16 || (Bh0 && (n1 == 0 || Bh1) && (n2 == 0 || Bh2));
+    if ((m->kernel_mask & 1) && have_b && tc_gemm_supported(M, n0 + n1 + n2, K)) {
+      const void *b0 = f16 ? (const void *)Bh0 : (const void *)B0;
+      const void *b1 = f16 ? (const void *)Bh1 : (const void *)B1;
+      const void *b2 = f16 ? (const void *)Bh2 : (const void *)B2;
       int rc = SWIFTKV_ERR_UNSUPPORTED;
       if (rope && rope_fused) {
-        rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, rope, m->b.status, st);
+        rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, dup, dup_stride, rope, m->b.status, st);
         if (rc == SWIFTKV_OK) *rope_fused = true;
       }
-      if (rc == SWIFTKV_ERR_UNSUPPORTED) rc = launch_gemm_tc(A, M, K, B0, n0, B1, n1, B2, n2, out, nullptr, m->b.status, st);
+      if (rc == SWIFTKV_ERR_UNSUPPORTED) rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, nullptr, 0, nullptr, m->b.status, st);
       if (rc == SWIFTKV_OK) { m->launches += 1; return rc; }
       if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "tensor-core GEMM launch failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
   }
-  launch_gemm_simt<T>(A, B0, M, n0, K, out, 0, st);
+  launch_gemm_simt<TA, TW>(A, B0, M, n0, K, out, 0, st);
   m->launches += 1;
-  if (n1 > 0) { launch_gemm_simt<T>(A, B1, M, n1, K, out, n0, st); m->launches += 1; }
-  if (n2 > 0) { launch_gemm_simt<T>(A, B2, M, n2, K, out, n0 + n1, st); m->launches += 1; }
+  if (n1 > 0) { launch_gemm_simt<TA, TW>(A, B1, M, n1, K, out, n0, st); m->launches += 1; }
+  if (n2 > 0) { launch_gemm_simt<TA, TW>(A, B2, M, n2, K, out, n0 + n1, st); m->launches += 1; }
   return SWIFTKV_OK;
 }
 
-template <typename T>
+template <typename TA, typename T>
 static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int l, int g, cudaStream_t st) {
   const swiftkv_config &c = m->cfg;
   Buffers &b = m->b;
   const int d = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim, F = c.ffn, L = c.n_layers;
   const size_t plane = (size_t)m->max_tokens * dkv;          // elements of one K (or V) plane
+  constexpr bool act_f16 = std::is_same<TA, __half>::value;
   T *kv = reinterpret_cast<T *>(m->kv);
-  T *h = (T *)b.h, *q = (T *)b.q, *attn = (T *)b.attn, *act = (T *)b.act;
+  TA *h = (TA *)b.h, *q = (TA *)b.q, *attn = (TA *)b.attn, *act = (TA *)b.act;
+  const T *no_w = nullptr;
   int32_t rc;
   const RopeSpec rope{b.pos, b.cos_tab, b.sin_tab, c.head_dim};
+  // With half activations the tensor-core kernels need both MMA operands in half: each layer's matrices are copied
+  // to half right before use (one 0.4 GB pass per layer on the 8B shape, exact for |w| >= 2^-17), K / V get a half
+  // copy beside the bf16 cache, and the folded SingleInputKV weight is produced in half directly.
+  const bool use_w16 = act_f16 && (m->kernel_mask & 1) && tc_gemm_supported(T_tok, dq, d) && tc_gemm_supported(T_tok, d, dq) &&
+                       tc_gemm_supported(T_tok, d, F) && (dkv % 256 == 0) && (dq % 256 == 0) && c.head_dim == 128;
+  const bool attn_tc = sizeof(T) == 2 && (m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim);
+  __half *wq16 = (__half *)b.w16, *wk16 = wq16 + (size_t)dq * d, *wv16 = wk16 + (size_t)dkv * d, *wo16 = wv16 + (size_t)dkv * d;
+  __half *wg16 = wo16 + (size_t)d * dq, *wu16 = wg16 + (size_t)F * d, *wd16 = wu16 + (size_t)F * d;
+  __half *k16 = (__half *)b.kv16, *v16 = k16 + plane;
 
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_positions(b.cu, B, b.pos, b.last_idx, T_tok, st); }
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_embed<T>((const T *)m->embed, b.tokens, b.x, T_tok, d, c.vocab, b.status, st); }
@@ -290,50 +320,78 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
   // one-time model transformation for this (l, g): fold each group leader's input-norm gain into its W_K, W_V
   // and stack them (Sec. 3.5)
   const int ng = n_groups(L, l, g);
-  if (l < L && (m->fold_l != l || m->fold_g != g)) {
+  const int fold_fmt = use_w16 ? 1 : 0;
+  if (l < L && (m->fold_l != l || m->fold_g != g || m->fold_fmt != fold_fmt)) {
     for (int i = 0; i < ng; ++i) {
       const swiftkv_layer_weights &lw = m->layers[l + i * g];
-      T *dst = (T *)b.wfold + (size_t)i * 2 * dkv * d;
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T>((const T *)lw.wk, (const T *)lw.in_norm, dst, dkv, d, st); }
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T>((const T *)lw.wv, (const T *)lw.in_norm, dst + (size_t)dkv * d, dkv, d, st); }
+      const size_t off = (size_t)i * 2 * dkv * d;
+      if constexpr (sizeof(T) == 2) {
+        if (use_w16) {
+          __half *dst = (__half *)b.wfold + off;
+          { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<bf16, __half>((const bf16 *)lw.wk, (const bf16 *)lw.in_norm, dst, dkv, d, st); }
+          { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<bf16, __half>((const bf16 *)lw.wv, (const bf16 *)lw.in_norm, dst + (size_t)dkv * d, dkv, d, st); }
+          continue;
+        }
+      }
+      T *dst = (T *)b.wfold + off;
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T, T>((const T *)lw.wk, (const T *)lw.in_norm, dst, dkv, d, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_fold<T, T>((const T *)lw.wv, (const T *)lw.in_norm, dst + (size_t)dkv * d, dkv, d, st); }
     }
-    m->fold_l = l; m->fold_g = g;
+    m->fold_l = l; m->fold_g = g; m->fold_fmt = fold_fmt;
   }
 
   // ---- layers 1..l on all prompt tokens (unmodified, Sec. 3.1)
   for (int j = 0; j < l; ++j) {
     const swiftkv_layer_weights &lw = m->layers[j];
     T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
+    if constexpr (sizeof(T) == 2) {
+      if (use_w16) {
+        Scope s(m, st, SWIFTKV_KC_ELEMWISE, 7);
+        launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, st);
+        launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, st);
+        launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, st);
+        launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, st);
+        launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, st);
+        launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, st);
+        launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, st);
+      }
+    }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
     OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv};
     bool roped = false;
-    rc = gemm_any<T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st, &rope, &roped);
+    const bool want_dup = use_w16 && attn_tc;    // the attention kernel then reads half copies of this layer's K / V
+    rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st,
+                         use_w16 ? wq16 : nullptr, use_w16 ? wk16 : nullptr, use_w16 ? wv16 : nullptr, &rope, &roped,
+                         want_dup ? k16 : nullptr, (long long)plane);
     if (rc) return rc;
     if (!roped) {
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
       { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
     }
     {
       Scope s(m, st, SWIFTKV_KC_ATTENTION);
       bool done = false;
       if constexpr (sizeof(T) == 2) {
-        if ((m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim)) {
-          rc = launch_attention_tc(q, Kj, Vj, attn, b.cu, B, T_tok, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
+        // (half activations: only when the QKV epilogue really wrote the half copies of K and V)
+        if (attn_tc && (!act_f16 || (want_dup && roped))) {
+          const void *kk = act_f16 ? (const void *)k16 : (const void *)Kj, *vv = act_f16 ? (const void *)v16 : (const void *)Vj;
+          rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, B, T_tok, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
           if (rc == SWIFTKV_OK) done = true;
           else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
         }
       }
-      if (!done) launch_attention_simple<T>(q, Kj, Vj, attn, b.cu, B, b.pos, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
+      if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, b.pos, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
     }
-    rc = gemm_any<T>(m, attn, T_tok, dq, (const T *)lw.wo, d, (const T *)nullptr, 0, (const T *)nullptr, 0,
-                     out_plain(OUT_RESID_ADD_F32, b.x, d, d), st);
+    rc = gemm_any<TA, T>(m, attn, T_tok, dq, (const T *)lw.wo, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
+                         use_w16 ? wo16 : nullptr);
     if (rc) return rc;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st); }
     bool fused = false;
     if constexpr (sizeof(T) == 2) {
-      if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d)) {
+      if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d) && (!act_f16 || use_w16)) {
         Scope s(m, st, SWIFTKV_KC_SWIGLU);
-        rc = launch_gemm_tc_swiglu(h, T_tok, d, (const bf16 *)lw.w_gate, (const bf16 *)lw.w_up, F, act, b.status, st);
+        const void *wg = act_f16 ? (const void *)wg16 : lw.w_gate, *wu = act_f16 ? (const void *)wu16 : lw.w_up;
+        rc = launch_gemm_tc_swiglu(h, act_f16, T_tok, d, wg, wu, F, act, b.status, st);
         if (rc == SWIFTKV_OK) fused = true;
         else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "SwiGLU GEMM launch failed");
       }
@@ -341,29 +399,31 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
     if (!fused) {
       for (int r0 = 0; r0 < T_tok; r0 += MLP_CHUNK_ROWS) {
         const int rows = std::min(MLP_CHUNK_ROWS, T_tok - r0);
-        rc = gemm_any<T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_gate, F, (const T *)nullptr, 0, (const T *)nullptr, 0,
-                         out_plain(OUT_STORE, b.gate, F, F), st);
+        rc = gemm_any<TA, T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_gate, F, no_w, 0, no_w, 0, out_plain(OUT_STORE, b.gate, F, F), st,
+                             use_w16 ? wg16 : nullptr);
         if (rc) return rc;
-        rc = gemm_any<T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_up, F, (const T *)nullptr, 0, (const T *)nullptr, 0,
-                         out_plain(OUT_STORE, b.up, F, F), st);
+        rc = gemm_any<TA, T>(m, h + (size_t)r0 * d, rows, d, (const T *)lw.w_up, F, no_w, 0, no_w, 0, out_plain(OUT_STORE, b.up, F, F), st,
+                             use_w16 ? wu16 : nullptr);
         if (rc) return rc;
         Scope s(m, st, SWIFTKV_KC_ELEMWISE);
-        launch_swiglu<T>((const T *)b.gate, (const T *)b.up, act + (size_t)r0 * F, (long long)rows * F, st);
+        launch_swiglu<TA>((const TA *)b.gate, (const TA *)b.up, act + (size_t)r0 * F, (long long)rows * F, st);
       }
     }
-    rc = gemm_any<T>(m, act, T_tok, F, (const T *)lw.w_down, d, (const T *)nullptr, 0, (const T *)nullptr, 0,
-                     out_plain(OUT_RESID_ADD_F32, b.x, d, d), st);
+    rc = gemm_any<TA, T>(m, act, T_tok, F, (const T *)lw.w_down, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
+                         use_w16 ? wd16 : nullptr);
     if (rc) return rc;
   }
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
   if (l < L) {
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
     T *slot_l = kv + (size_t)l * 2 * plane;
     OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv};
     bool roped = false;
-    rc = gemm_any<T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, (const T *)nullptr, 0, (const T *)nullptr, 0, o, st, &rope, &roped);
+    rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, no_w, 0, no_w, 0, o, st,
+                         use_w16 ? (const __half *)b.wfold : nullptr, nullptr, nullptr, &rope, &roped);
     if (rc) return rc;
+    if (use_w16 && !roped) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-folded SingleInputKV weight needs the tensor-core GEMM");
     if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
   }
 
@@ -435,8 +495,10 @@ static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool toke
   CUDA_TRY(cudaMemcpyAsync(m->b.last_pos, lp.data(), (size_t)n_seqs * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(m->b.tokens, tokens, (size_t)total * 4,
                            tokens_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
-  int32_t rc = c.dtype == SWIFTKV_DTYPE_BF16 ? run_prefill<bf16>(m, (int)total, n_seqs, max_len, l, g, st)
-                                             : run_prefill<float>(m, (int)total, n_seqs, max_len, l, g, st);
+  int32_t rc;
+  if (c.dtype == SWIFTKV_DTYPE_F32) rc = run_prefill<float, float>(m, (int)total, n_seqs, max_len, l, g, st);
+  else if (m->act_format == SWIFTKV_ACT_F16) rc = run_prefill<__half, bf16>(m, (int)total, n_seqs, max_len, l, g, st);
+  else rc = run_prefill<bf16, bf16>(m, (int)total, n_seqs, max_len, l, g, st);
   if (rc) return rc;
   m->n_tokens = (int)total; m->n_seqs = n_seqs; m->cur_l = l; m->cur_g = g; m->ready = true;
   return SWIFTKV_OK;
@@ -517,6 +579,13 @@ extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   return m->kernel_mask;
 }
 
+extern "C" int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if (format != SWIFTKV_ACT_BF16 && format != SWIFTKV_ACT_F16) return fail(SWIFTKV_ERR_INVALID_ARG, "unknown activation format");
+  m->act_format = format;
+  return SWIFTKV_OK;
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // stand-alone operators
 // ---------------------------------------------------------------------------------------------------------
@@ -531,15 +600,18 @@ static unsigned int *op_status_word() {
   return ptr;
 }
 
-extern "C" int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
-                                     void *cuda_stream) {
+extern "C" int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
+                                   int32_t dtype, void *cuda_stream) {
+  const int32_t act_dtype = dtype;
   if (!A || !B || !C || M < 1 || N < 1 || K < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "bad argument");
+  if (act_dtype != SWIFTKV_DTYPE_BF16 && act_dtype != SWIFTKV_DTYPE_F16) return fail(SWIFTKV_ERR_INVALID_ARG, "act_dtype must be bf16 or f16");
   if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15) return fail(SWIFTKV_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
   if (!tc_gemm_supported(M, N, K)) return fail(SWIFTKV_ERR_UNSUPPORTED, "needs K %% 64 == 0 and N %% 128 == 0");
   unsigned int *status = op_status_word();
   if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
-  int rc = launch_gemm_tc((const bf16 *)A, M, K, (const bf16 *)B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N),
-                          nullptr, status, reinterpret_cast<cudaStream_t>(cuda_stream));
+  const bool f16 = act_dtype == SWIFTKV_DTYPE_F16;
+  int rc = launch_gemm_tc(A, f16, M, K, B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N), nullptr, 0, nullptr,
+                          status, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
   return SWIFTKV_OK;
 }
@@ -547,30 +619,34 @@ extern "C" int32_t swiftkv_gemm_bf16(const void *A, const void *B, void *C, int3
 extern "C" int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, void *out,
                                              const int32_t *cu_seqlens, int32_t n_seqs, int32_t total_tokens,
                                              int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads,
-                                             int32_t head_dim, int32_t dtype, int32_t use_tensor_cores,
-                                             void *cuda_stream) {
+                                             int32_t head_dim, int32_t q_dtype, int32_t kv_dtype,
+                                             int32_t use_tensor_cores, void *cuda_stream) {
   if (!q || !k || !v || !out || !cu_seqlens) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
   if (n_seqs < 1 || total_tokens < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || head_dim < 2 || head_dim > 256)
     return fail(SWIFTKV_ERR_INVALID_ARG, "bad shape");
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const bool q16 = q_dtype == SWIFTKV_DTYPE_BF16 || q_dtype == SWIFTKV_DTYPE_F16;
   if (use_tensor_cores) {
-    if (dtype != SWIFTKV_DTYPE_BF16 || !tc_attention_supported(n_q_heads, n_kv_heads, head_dim))
-      return fail(SWIFTKV_ERR_UNSUPPORTED, "tensor-core attention needs bf16 and head_dim 128");
+    if (kv_dtype != q_dtype || !q16 || !tc_attention_supported(n_q_heads, n_kv_heads, head_dim))
+      return fail(SWIFTKV_ERR_UNSUPPORTED, "tensor-core attention needs q, K, V of one 16-bit type, head_dim 128, an even group size");
     unsigned int *status = op_status_word();
     if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
-    int rc = launch_attention_tc((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs,
+    int rc = launch_attention_tc(q, q_dtype == SWIFTKV_DTYPE_F16, k, v, out, cu_seqlens, n_seqs,
                                  total_tokens, max_seq_len, n_q_heads, n_kv_heads, head_dim, status, st);
     if (rc) return fail(rc, "attention launch failed");
     return SWIFTKV_OK;
   }
-  if (dtype == SWIFTKV_DTYPE_BF16)
-    launch_attention_simple<bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr,
-                                  total_tokens, n_q_heads, n_kv_heads, head_dim, st);
-  else if (dtype == SWIFTKV_DTYPE_F32)
-    launch_attention_simple<float>((const float *)q, (const float *)k, (const float *)v, (float *)out, cu_seqlens, n_seqs,
-                                   nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+  if (q_dtype == SWIFTKV_DTYPE_BF16 && kv_dtype == SWIFTKV_DTYPE_BF16)
+    launch_attention_simple<bf16, bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr,
+                                        total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+  else if (q_dtype == SWIFTKV_DTYPE_F16 && kv_dtype == SWIFTKV_DTYPE_BF16)
+    launch_attention_simple<__half, bf16>((const __half *)q, (const bf16 *)k, (const bf16 *)v, (__half *)out, cu_seqlens, n_seqs,
+                                          nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+  else if (q_dtype == SWIFTKV_DTYPE_F32 && kv_dtype == SWIFTKV_DTYPE_F32)
+    launch_attention_simple<float, float>((const float *)q, (const float *)k, (const float *)v, (float *)out, cu_seqlens, n_seqs,
+                                          nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else
-    return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+    return fail(SWIFTKV_ERR_INVALID_ARG, "unsupported dtype combination");
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
   return SWIFTKV_OK;

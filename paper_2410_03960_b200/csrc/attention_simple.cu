@@ -8,9 +8,9 @@
 
 namespace skv {
 
-template <typename T, int MAX_E>   // MAX_E = ceil(hd / 32) output elements per lane
-__global__ void __launch_bounds__(128) attention_simple_kernel(const T *__restrict__ q, const T *__restrict__ k,
-                                                               const T *__restrict__ v, T *__restrict__ out,
+template <typename TQ, typename T, int MAX_E>   // MAX_E = ceil(hd / 32) output elements per lane
+__global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restrict__ q, const T *__restrict__ k,
+                                                               const T *__restrict__ v, TQ *__restrict__ out,
                                                                const int32_t *__restrict__ cu, int n_seqs,
                                                                const int32_t *__restrict__ positions, int n_tokens,
                                                                int n_q, int n_kv, int hd, float scale) {
@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const T *__restri
   }
   const int first = t - p;   // packed index of this prompt's first token
   float *qs = q_sm + warp * hd;
-  const T *qr = q + ((size_t)t * n_q + h) * hd;
+  const TQ *qr = q + ((size_t)t * n_q + h) * hd;
   for (int i = lane; i < hd; i += 32) qs[i] = to_f(qr[i]) * scale;
   __syncwarp();
 
@@ -69,31 +69,33 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const T *__restri
       }
     }
   }
-  T *orow = out + ((size_t)t * n_q + h) * hd;
+  TQ *orow = out + ((size_t)t * n_q + h) * hd;
   const float inv = 1.f / l;
 #pragma unroll
   for (int e = 0; e < MAX_E; ++e) {
     const int dd = lane + 32 * e;
-    if (dd < hd) orow[dd] = from_f<T>(acc[e] * inv);
+    if (dd < hd) orow[dd] = from_f<TQ>(acc[e] * inv);
   }
 }
 
-template <typename T>
-void launch_attention_simple(const T *q, const T *k, const T *v, T *out, const int32_t *cu_seqlens, int n_seqs,
+template <typename TQ, typename T>
+void launch_attention_simple(const TQ *q, const T *k, const T *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
                              const int32_t *positions, int n_tokens, int n_q, int n_kv, int hd, cudaStream_t st) {
   if (n_tokens <= 0) return;
   const long long items = (long long)n_tokens * n_q;
   const unsigned blocks = (unsigned)((items + 3) / 4);
   const float scale = 1.0f / sqrtf((float)hd);
   const size_t smem = 4 * hd * sizeof(float);
-  if (hd <= 32) attention_simple_kernel<T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 64) attention_simple_kernel<T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 128) attention_simple_kernel<T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else attention_simple_kernel<T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
+  if (hd <= 32) attention_simple_kernel<TQ, T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 64) attention_simple_kernel<TQ, T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 128) attention_simple_kernel<TQ, T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
+  else attention_simple_kernel<TQ, T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
 }
-template void launch_attention_simple<float>(const float *, const float *, const float *, float *, const int32_t *, int,
-                                             const int32_t *, int, int, int, int, cudaStream_t);
-template void launch_attention_simple<bf16>(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int,
-                                            const int32_t *, int, int, int, int, cudaStream_t);
+template void launch_attention_simple<float, float>(const float *, const float *, const float *, float *, const int32_t *, int,
+                                                    const int32_t *, int, int, int, int, cudaStream_t);
+template void launch_attention_simple<bf16, bf16>(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int,
+                                                  const int32_t *, int, int, int, int, cudaStream_t);
+template void launch_attention_simple<__half, bf16>(const __half *, const bf16 *, const bf16 *, __half *, const int32_t *, int,
+                                                    const int32_t *, int, int, int, int, cudaStream_t);
 
 }  // namespace skv

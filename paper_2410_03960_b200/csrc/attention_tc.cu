@@ -56,6 +56,8 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// ACT_F16: q, K, V, P and the output are all IEEE halves (else all bfloat16)
+template <bool ACT_F16>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, AttnParams p) {
@@ -137,8 +139,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   } else if (warp == 1) {
     if (lane == 0) {
       // ------------------------------------------------------------ MMA issuer
-      constexpr uint32_t idesc_qk = tc::umma_idesc_bf16(BQ, BKV, 0, 0);   // Q, K both K-major (head dim contiguous)
-      constexpr uint32_t idesc_pv = tc::umma_idesc_bf16(BQ, HD, 0, 1);    // V is MN-major (head dim contiguous, keys = K)
+      constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);   // Q, K both K-major (head dim contiguous)
+      constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);    // V is MN-major (head dim contiguous, keys = K)
       const uint32_t q_addr = tc::smem_u32(smem + SM_Q);
       auto issue_qk = [&](int w, int s) {   // S_w = Q_w K^T : 8 steps of 16 along the head dim
         const uint32_t a0 = q_addr + w * TILE_BYTES, b0 = tc::smem_u32(smem + SM_K + s * TILE_BYTES);
@@ -256,8 +258,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 2]), c, neg_mc));
         const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 3]), c, neg_mc));
         l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-        s[i] = tc::pack_bf16x2(p0, p1);
-        s[i + 1] = tc::pack_bf16x2(p2, p3);
+        s[i] = ACT_F16 ? tc::pack_f16x2(p0, p1) : tc::pack_bf16x2(p0, p1);
+        s[i + 1] = ACT_F16 ? tc::pack_f16x2(p2, p3) : tc::pack_bf16x2(p2, p3);
       }
       l += (l0 + l1) + (l2 + l3);
       tc::tmem_st_32x32b_x32(t_s, s);
@@ -282,10 +284,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           uint4 *d4 = reinterpret_cast<uint4 *>(dst + ch * 32);
 #pragma unroll
           for (int i = 0; i < 4; ++i)
-            d4[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv),
-                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv),
-                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv),
-                               tc::pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv));
+            d4[i] = make_uint4(tc::pack_act(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv, ACT_F16));
         }
       }
     }
@@ -305,8 +307,9 @@ bool tc_attention_supported(int n_q, int n_kv, int hd) {
   return hd == HD && n_kv >= 1 && n_q % n_kv == 0 && ((n_q / n_kv) % 2) == 0;
 }
 
-int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, const int32_t *cu_seqlens, int n_seqs,
-                        int n_tokens, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st) {
+int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
+                        int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
+                        cudaStream_t st) {
   if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
   if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1) return SWIFTKV_ERR_INVALID_ARG;
   CUtensorMap tq, tk, tv;
@@ -316,18 +319,20 @@ int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, 
   if (get_tmap(&tv, v, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
       return SWIFTKV_ERR_CUDA;
     attr_set = true;
   }
   AttnParams p{};
-  p.cu = cu_seqlens; p.out = out; p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
+  p.cu = cu_seqlens; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
   p.max_tiles = (max_seq_len + BQ - 1) / BQ;
   p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
   p.status = status;
   const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
   if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
-  attention_tc_kernel<<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  if (act_f16) attention_tc_kernel<true><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  else attention_tc_kernel<false><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
   return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
 }
 

@@ -1,6 +1,7 @@
 // Shared declarations of the SwiftKV prefill library (host + device helpers, launch prototypes).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -21,6 +22,11 @@ template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloa
 template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+// IEEE half: the precise storage format for activations of a bf16 model; conversion saturates at +-65504
+template <> __device__ __forceinline__ float to_f<__half>(__half v) { return __half2float(v); }
+template <> __device__ __forceinline__ __half from_f<__half>(float v) {
+  return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -51,7 +57,8 @@ inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDes
 
 #ifdef __CUDACC__
 // write one fp32 accumulator where the descriptor says (device side)
-template <typename T>
+// TP: element type of the p0 region; TS: element type of the segments (K / V cache planes)
+template <typename TP, typename TS>
 __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, float acc) {
   if (o.mode == OUT_RESID_ADD_F32) {
     float *p = reinterpret_cast<float *>(o.p0) + (size_t)row * o.ld0 + col;
@@ -59,11 +66,11 @@ __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, fl
   } else if (o.mode == OUT_STORE_F32) {
     reinterpret_cast<float *>(o.p0)[(size_t)row * o.ld0 + col] = acc;
   } else if (col < o.n0) {
-    reinterpret_cast<T *>(o.p0)[(size_t)row * o.ld0 + col] = from_f<T>(acc);
+    reinterpret_cast<TP *>(o.p0)[(size_t)row * o.ld0 + col] = from_f<TP>(acc);
   } else {
     const int c = col - o.n0;
     const int seg = c / o.seg_w, within = c % o.seg_w;
-    reinterpret_cast<T *>(o.seg_base)[(size_t)seg * o.seg_stride + (size_t)row * o.seg_w + within] = from_f<T>(acc);
+    reinterpret_cast<TS *>(o.seg_base)[(size_t)seg * o.seg_stride + (size_t)row * o.seg_w + within] = from_f<TS>(acc);
   }
 }
 #endif
@@ -78,9 +85,9 @@ void launch_embed(const T *embed, const int32_t *tokens, float *x, int n_tokens,
                   unsigned int *status, cudaStream_t st);
 void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions, int32_t *last_idx, int n_tokens,
                       cudaStream_t st);
-// y = x * rsqrt(mean(x^2)+eps) * gamma (gamma may be null: unit-rms only).  x fp32 [rows, d] -> out T [rows, d]
-template <typename T>
-void launch_rmsnorm(const float *x, const T *gamma, T *out, int rows, int d, float eps, cudaStream_t st);
+// y = x * rsqrt(mean(x^2)+eps) * gamma (gamma may be null: unit-rms only).  x fp32 [rows, d] -> out TO [rows, d]
+template <typename TG, typename TO>
+void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st);
 // in-place rotary embedding on `n_batches` tensors [rows, n_heads, hd] spaced batch_stride elements apart
 template <typename T>
 void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const float *cos_tab,
@@ -90,13 +97,15 @@ void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
 void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, double theta, cudaStream_t st);
 // dst[r, c] = w[r, c] * gamma[c]   (gain of the input norm folded into a projection weight, Sec. 3.5)
-template <typename T>
-void launch_fold(const T *w, const T *gamma, T *dst, int rows, int cols, cudaStream_t st);
+template <typename T, typename TO>
+void launch_fold(const T *w, const T *gamma, TO *dst, int rows, int cols, cudaStream_t st);
+// IEEE-half copy of a bf16 matrix (the compute copy of a layer's weights when activations are kept in half)
+void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st);
 
 // gemm_simt.cu : C = A[M,K] * B[N,K]^T with fp32 accumulation, any shape; result column c is written as
-// column col0 + c of `out`
-template <typename T>
-void launch_gemm_simt(const T *A, const T *B, int M, int N, int K, OutDesc out, int col0, cudaStream_t st);
+// column col0 + c of `out` (p0 region in the activation type TA, segments in the weight / cache type TW)
+template <typename TA, typename TW>
+void launch_gemm_simt(const TA *A, const TW *B, int M, int N, int K, OutDesc out, int col0, cudaStream_t st);
 
 // gemm_tc.cu : tcgen05 / TMEM / TMA GEMMs (bf16)
 struct TcGemmPlan;   // host object holding tensor maps
@@ -109,20 +118,25 @@ struct RopeSpec {
   const float *cos_tab, *sin_tab;   // [position][hd/2]
   int hd;
 };
-int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
-                   int nB2, OutDesc out, const RopeSpec *rope, unsigned int *status, cudaStream_t st);
-// act[M, F] = silu(A Wg^T) * (A Wu^T), gate/up tiles paired inside one CTA tile
-int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
+// f16: A, every B and the columns below out.n0 hold IEEE halves instead of bfloat16 (same type on both operands);
+// columns routed to segments (the K / V cache planes) are always stored as bfloat16, and -- if dup_base is given --
+// stored a second time as halves at dup_base + segment * dup_stride (the attention kernel's operand copy)
+int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB0, const void *B1, int nB1, const void *B2,
+                   int nB2, OutDesc out, void *dup_base, long long dup_stride, const RopeSpec *rope, unsigned int *status,
+                   cudaStream_t st);
+// act[M, F] = silu(A Wg^T) * (A Wu^T), gate/up tiles paired inside one CTA tile; f16: all three in IEEE half
+int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg, const void *Wu, int F, void *act,
                           unsigned int *status, cudaStream_t st);
 bool tc_swiglu_supported(int M, int F, int K);
 
 // attention.cu
-template <typename T>
-void launch_attention_simple(const T *q, const T *k, const T *v, T *out, const int32_t *cu_seqlens, int n_seqs,
+template <typename TQ, typename TKV>
+void launch_attention_simple(const TQ *q, const TKV *k, const TKV *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
                              const int32_t *positions /* may be null */, int n_tokens, int n_q, int n_kv, int hd,
                              cudaStream_t st);
 bool tc_attention_supported(int n_q, int n_kv, int hd);
-int launch_attention_tc(const bf16 *q, const bf16 *k, const bf16 *v, bf16 *out, const int32_t *cu_seqlens,
+// f16: q, k, v and out all hold IEEE halves (else all bfloat16)
+int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
                         int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd,
                         unsigned int *status, cudaStream_t st);
 

@@ -70,8 +70,8 @@ void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions,
 // The residual stream x is fp32; the output is the model dtype.  gamma == nullptr gives the unit-rms row that
 // feeds the gain-folded SingleInputKV projection (one statistic shared by every later layer).
 // ---------------------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const T *__restrict__ gamma,
+template <typename TG, typename T>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
                                                       T *__restrict__ out, int d, float eps) {
   const size_t row = blockIdx.x;
   const float *xr = x + row * d;
@@ -100,12 +100,8 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
       float g0 = 1.f, g1 = 1.f, g2 = 1.f, g3 = 1.f;
       if (gamma) { g0 = to_f(gamma[i]); g1 = to_f(gamma[i + 1]); g2 = to_f(gamma[i + 2]); g3 = to_f(gamma[i + 3]); }
       if constexpr (sizeof(T) == 2) {
-        __nv_bfloat162 a = __floats2bfloat162_rn(v.x * rstd * g0, v.y * rstd * g1);
-        __nv_bfloat162 b = __floats2bfloat162_rn(v.z * rstd * g2, v.w * rstd * g3);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t *>(&a);
-        pk.y = *reinterpret_cast<uint32_t *>(&b);
-        *reinterpret_cast<uint2 *>(orow + i) = pk;
+        T o4[4] = {from_f<T>(v.x * rstd * g0), from_f<T>(v.y * rstd * g1), from_f<T>(v.z * rstd * g2), from_f<T>(v.w * rstd * g3)};
+        *reinterpret_cast<uint2 *>(orow + i) = *reinterpret_cast<uint2 *>(o4);
       } else {
         *reinterpret_cast<float4 *>(orow + i) = make_float4(v.x * rstd * g0, v.y * rstd * g1, v.z * rstd * g2, v.w * rstd * g3);
       }
@@ -115,13 +111,14 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
       orow[i] = from_f<T>(xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f));
   }
 }
-template <typename T>
-void launch_rmsnorm(const float *x, const T *gamma, T *out, int rows, int d, float eps, cudaStream_t st) {
+template <typename TG, typename TO>
+void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st) {
   if (rows <= 0) return;
-  rmsnorm_kernel<T><<<rows, 256, 0, st>>>(x, gamma, out, d, eps);
+  rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps);
 }
-template void launch_rmsnorm<float>(const float *, const float *, float *, int, int, float, cudaStream_t);
-template void launch_rmsnorm<bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t);
+template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t);
+template void launch_rmsnorm<bf16, bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t);
+template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *, int, int, float, cudaStream_t);
 
 // ---------------------------------------------------------------------------------------------------------
 // Rotary embedding, rotate-half pairing (i, i + hd/2), in place.  One thread per pair.
@@ -154,6 +151,7 @@ void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *pos
 }
 template void launch_rope<float>(float *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
 template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<__half>(__half *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
 
 // cos/sin of p * theta^(-2i/hd), evaluated in double precision and rounded once to fp32.
 __global__ void rope_table_kernel(float *cos_tab, float *sin_tab, int max_pos, int half, double log_theta, int hd) {
@@ -209,6 +207,7 @@ void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t
 }
 template void launch_swiglu<float>(const float *, const float *, float *, long long, cudaStream_t);
 template void launch_swiglu<bf16>(const bf16 *, const bf16 *, bf16 *, long long, cudaStream_t);
+template void launch_swiglu<__half>(const __half *, const __half *, __half *, long long, cudaStream_t);
 
 // y[b, :] = x[idx[b], :]   (the tokens that continue past layer l: the last token of each prompt)
 __global__ void gather_rows_kernel(const float *__restrict__ x, const int32_t *__restrict__ idx, float *__restrict__ y, int d) {
@@ -221,22 +220,47 @@ void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows
   gather_rows_kernel<<<n_rows, 256, 0, st>>>(x, idx, y, d);
 }
 
-// dst[r, c] = w[r, c] * gamma[c], product in fp32, one rounding to the model dtype
-template <typename T>
-__global__ void fold_kernel(const T *__restrict__ w, const T *__restrict__ gamma, T *__restrict__ dst, long long n, int cols) {
+// dst[r, c] = w[r, c] * gamma[c], product in fp32, one rounding to the output type
+template <typename T, typename TO>
+__global__ void fold_kernel(const T *__restrict__ w, const T *__restrict__ gamma, TO *__restrict__ dst, long long n, int cols) {
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
-    dst[i] = from_f<T>(to_f(w[i]) * to_f(gamma[i % cols]));
+    dst[i] = from_f<TO>(to_f(w[i]) * to_f(gamma[i % cols]));
 }
-template <typename T>
-void launch_fold(const T *w, const T *gamma, T *dst, int rows, int cols, cudaStream_t st) {
+template <typename T, typename TO>
+void launch_fold(const T *w, const T *gamma, TO *dst, int rows, int cols, cudaStream_t st) {
   const long long n = (long long)rows * cols;
   if (n <= 0) return;
   long long blocks = (n + 255) / 256;
   if (blocks > 148 * 8) blocks = 148 * 8;
-  fold_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(w, gamma, dst, n, cols);
+  fold_kernel<T, TO><<<(unsigned)blocks, 256, 0, st>>>(w, gamma, dst, n, cols);
 }
-template void launch_fold<float>(const float *, const float *, float *, int, int, cudaStream_t);
-template void launch_fold<bf16>(const bf16 *, const bf16 *, bf16 *, int, int, cudaStream_t);
+template void launch_fold<float, float>(const float *, const float *, float *, int, int, cudaStream_t);
+template void launch_fold<bf16, bf16>(const bf16 *, const bf16 *, bf16 *, int, int, cudaStream_t);
+template void launch_fold<bf16, __half>(const bf16 *, const bf16 *, __half *, int, int, cudaStream_t);
+
+// bfloat16 -> IEEE half copy of a weight matrix (exact for |w| >= 2^-17, absolute error <= 2^-25 below), 128-bit accesses
+__global__ void bf16_to_f16_kernel(const bf16 *__restrict__ src, __half *__restrict__ dst, long long n) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long nv = n / 8;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += stride) {
+    const uint4 raw = __ldcs(reinterpret_cast<const uint4 *>(src) + i);
+    const __nv_bfloat162 *in2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    uint4 o;
+    __half2 *o2 = reinterpret_cast<__half2 *>(&o);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o2[k] = __float22half2_rn(__bfloat1622float2(in2[k]));
+    reinterpret_cast<uint4 *>(dst)[i] = o;
+  }
+  for (long long i = nv * 8 + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    dst[i] = __float2half_rn(__bfloat162float(src[i]));
+}
+void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st) {
+  if (n <= 0) return;
+  long long blocks = (n / 8 + 255) / 256;
+  if (blocks < 1) blocks = 1;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  bf16_to_f16_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, dst, n);
+}
 
 }  // namespace skv

@@ -7,8 +7,8 @@ namespace skv {
 
 constexpr int SBM = 64, SBN = 64, SBK = 16;
 
-template <typename T>
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const T *__restrict__ A, const T *__restrict__ B, int M, int N,
+template <typename TA, typename TW>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const TA *__restrict__ A, const TW *__restrict__ B, int M, int N,
                                                         int K, OutDesc out, int col0) {
   __shared__ float As[SBK][SBM + 1];
   __shared__ float Bs[SBK][SBN + 1];
@@ -48,18 +48,19 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T *__restrict__ A,
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int col = n0 + tx * 4 + j;
-      if (col < N) store_out<T>(out, row, col0 + col, acc[i][j]);
+      if (col < N) store_out<TA, TW>(out, row, col0 + col, acc[i][j]);
     }
   }
 }
 
-template <typename T>
-void launch_gemm_simt(const T *A, const T *B, int M, int N, int K, OutDesc out, int col0, cudaStream_t st) {
+template <typename TA, typename TW>
+void launch_gemm_simt(const TA *A, const TW *B, int M, int N, int K, OutDesc out, int col0, cudaStream_t st) {
   if (M <= 0 || N <= 0) return;
   dim3 grid((N + SBN - 1) / SBN, (M + SBM - 1) / SBM);
-  gemm_simt_kernel<T><<<grid, 256, 0, st>>>(A, B, M, N, K, out, col0);
+  gemm_simt_kernel<TA, TW><<<grid, 256, 0, st>>>(A, B, M, N, K, out, col0);
 }
-template void launch_gemm_simt<float>(const float *, const float *, int, int, int, OutDesc, int, cudaStream_t);
-template void launch_gemm_simt<bf16>(const bf16 *, const bf16 *, int, int, int, OutDesc, int, cudaStream_t);
+template void launch_gemm_simt<float, float>(const float *, const float *, int, int, int, OutDesc, int, cudaStream_t);
+template void launch_gemm_simt<bf16, bf16>(const bf16 *, const bf16 *, int, int, int, OutDesc, int, cudaStream_t);
+template void launch_gemm_simt<__half, bf16>(const __half *, const bf16 *, int, int, int, OutDesc, int, cudaStream_t);
 
 }  // namespace skv

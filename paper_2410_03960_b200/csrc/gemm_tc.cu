@@ -123,6 +123,9 @@ struct GemmTcParams {
   OutDesc out;
   bf16 *act;             // SwiGLU output [M, F]
   int F;
+  int f16;               // A, B and the columns below out.n0 (and the SwiGLU output) hold IEEE halves (else bfloat16)
+  __half *dup_base;      // optional second copy (halves) of the columns routed to segments
+  long long dup_stride;
   const int32_t *rope_pos;   // EPI_ROPE: position of every row; cos/sin tables [pos][64]
   const float *cos_tab, *sin_tab;
   unsigned int *status;
@@ -234,7 +237,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     if (lane == 0) {
       // ------------------------------------------------ MMA issuer
-      constexpr uint32_t idesc = tc::umma_idesc_bf16(BM, BN, 0, 0);
+      const uint32_t idesc = tc::umma_idesc(BM, BN, 0, 0, p.f16, p.f16);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -289,7 +292,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int i = 0; i < 16; ++i) {
               const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
               const float u0 = __uint_as_float(u[2 * i]), u1 = __uint_as_float(u[2 * i + 1]);
-              pk[i] = tc::pack_bf16x2(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1);
+              pk[i] = tc::pack_act(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1, p.f16 != 0);
             }
             uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * p.F + (size_t)n_blk * HALF + c * 32);
 #pragma unroll
@@ -306,14 +309,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int hh = 0; hh < BN / 128; ++hh) {
           const int col_h = n_blk * BN + hh * 128;
           bf16 *dstp;
-          bool rope;
+          __half *dupp = nullptr;
+          bool rope, f16 = false;
           if (col_h < p.out.n0) {
             dstp = reinterpret_cast<bf16 *>(p.out.p0) + (size_t)row * p.out.ld0 + col_h;
             rope = true;
+            f16 = p.f16 != 0;
           } else {
             const int cc = col_h - p.out.n0;
             const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
             dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + (size_t)row * p.out.seg_w + within;
+            if (p.dup_base) dupp = p.dup_base + (size_t)seg * p.dup_stride + (size_t)row * p.out.seg_w + within;
             rope = (seg & 1) == 0;      // segments alternate K (rotated) and V (not)
           }
 #pragma unroll 1
@@ -340,14 +346,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               uint4 *d1 = reinterpret_cast<uint4 *>(dstp + 64 + c * 32);
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
-                d0[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(a[8 * i]), __uint_as_float(a[8 * i + 1])),
-                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3])),
-                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5])),
-                                   tc::pack_bf16x2(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7])));
-                d1[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(bq[8 * i]), __uint_as_float(bq[8 * i + 1])),
-                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 2]), __uint_as_float(bq[8 * i + 3])),
-                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 4]), __uint_as_float(bq[8 * i + 5])),
-                                   tc::pack_bf16x2(__uint_as_float(bq[8 * i + 6]), __uint_as_float(bq[8 * i + 7])));
+                d0[i] = make_uint4(tc::pack_act(__uint_as_float(a[8 * i]), __uint_as_float(a[8 * i + 1]), f16),
+                                   tc::pack_act(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3]), f16),
+                                   tc::pack_act(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5]), f16),
+                                   tc::pack_act(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7]), f16));
+                d1[i] = make_uint4(tc::pack_act(__uint_as_float(bq[8 * i]), __uint_as_float(bq[8 * i + 1]), f16),
+                                   tc::pack_act(__uint_as_float(bq[8 * i + 2]), __uint_as_float(bq[8 * i + 3]), f16),
+                                   tc::pack_act(__uint_as_float(bq[8 * i + 4]), __uint_as_float(bq[8 * i + 5]), f16),
+                                   tc::pack_act(__uint_as_float(bq[8 * i + 6]), __uint_as_float(bq[8 * i + 7]), f16));
+              }
+              if (dupp) {   // the same values once more as halves, straight from the fp32 accumulators
+                uint4 *e0 = reinterpret_cast<uint4 *>(dupp + c * 32);
+                uint4 *e1 = reinterpret_cast<uint4 *>(dupp + 64 + c * 32);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  e0[i] = make_uint4(tc::pack_f16x2(__uint_as_float(a[8 * i]), __uint_as_float(a[8 * i + 1])),
+                                     tc::pack_f16x2(__uint_as_float(a[8 * i + 2]), __uint_as_float(a[8 * i + 3])),
+                                     tc::pack_f16x2(__uint_as_float(a[8 * i + 4]), __uint_as_float(a[8 * i + 5])),
+                                     tc::pack_f16x2(__uint_as_float(a[8 * i + 6]), __uint_as_float(a[8 * i + 7])));
+                  e1[i] = make_uint4(tc::pack_f16x2(__uint_as_float(bq[8 * i]), __uint_as_float(bq[8 * i + 1])),
+                                     tc::pack_f16x2(__uint_as_float(bq[8 * i + 2]), __uint_as_float(bq[8 * i + 3])),
+                                     tc::pack_f16x2(__uint_as_float(bq[8 * i + 4]), __uint_as_float(bq[8 * i + 5])),
+                                     tc::pack_f16x2(__uint_as_float(bq[8 * i + 6]), __uint_as_float(bq[8 * i + 7])));
+                }
               }
             }
           }
@@ -371,8 +392,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             } else {
               bf16 *dstp;
+              bool f16 = false;
               if (col < p.out.n0) {
                 dstp = reinterpret_cast<bf16 *>(p.out.p0) + (size_t)row * p.out.ld0 + col;
+                f16 = p.f16 != 0;
               } else {
                 const int cc = col - p.out.n0;
                 const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
@@ -381,10 +404,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               uint4 *dst = reinterpret_cast<uint4 *>(dstp);
 #pragma unroll
               for (int i = 0; i < 4; ++i)
-                dst[i] = make_uint4(tc::pack_bf16x2(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1])),
-                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3])),
-                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5])),
-                                    tc::pack_bf16x2(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7])));
+                dst[i] = make_uint4(tc::pack_act(__uint_as_float(r[8 * i]), __uint_as_float(r[8 * i + 1]), f16),
+                                    tc::pack_act(__uint_as_float(r[8 * i + 2]), __uint_as_float(r[8 * i + 3]), f16),
+                                    tc::pack_act(__uint_as_float(r[8 * i + 4]), __uint_as_float(r[8 * i + 5]), f16),
+                                    tc::pack_act(__uint_as_float(r[8 * i + 6]), __uint_as_float(r[8 * i + 7]), f16));
             }
           }
         }
@@ -424,8 +447,9 @@ int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b
 bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (N % 128) == 0 && N >= 128; }
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
 
-int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const bf16 *B1, int nB1, const bf16 *B2,
-                   int nB2, OutDesc out, const RopeSpec *rope, unsigned int *status, cudaStream_t st) {
+int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB0, const void *B1, int nB1, const void *B2,
+                   int nB2, OutDesc out, void *dup_base, long long dup_stride, const RopeSpec *rope, unsigned int *status,
+                   cudaStream_t st) {
   const int N = nB0 + nB1 + nB2;
   if (!tc_gemm_supported(M, N, K)) return SWIFTKV_ERR_UNSUPPORTED;
   if (out.mode == OUT_STORE_F32) return SWIFTKV_ERR_UNSUPPORTED;
@@ -444,6 +468,8 @@ int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const b
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = N / BN;
   p.out = out; p.act = nullptr; p.F = 0; p.status = status;
+  p.f16 = f16; p.dup_base = reinterpret_cast<__half *>(dup_base); p.dup_stride = dup_stride;
+  if (dup_base && !rope) return SWIFTKV_ERR_UNSUPPORTED;
   if (rope) {
     // fused rotary embedding needs head-aligned tiles of 128-wide heads and a bf16 store
     if (rope->hd != 128 || out.mode != OUT_STORE || (out.n0 % 128) || (out.n0 < N && (out.seg_w % 128)))
@@ -456,7 +482,7 @@ int launch_gemm_tc(const bf16 *A, int M, int K, const bf16 *B0, int nB0, const b
   return launch_cfg<128, 6, EPI_PLAIN>(ta, tb0, tb1, tb2, p, st);
 }
 
-int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf16 *Wu, int F, bf16 *act,
+int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg, const void *Wu, int F, void *act,
                           unsigned int *status, cudaStream_t st) {
   if (!tc_swiglu_supported(M, F, K)) return SWIFTKV_ERR_UNSUPPORTED;
   CUtensorMap ta, tg, tu;
@@ -467,7 +493,8 @@ int launch_gemm_tc_swiglu(const bf16 *A, int M, int K, const bf16 *Wg, const bf1
   p.M = M; p.N = 2 * F; p.K = K; p.nB0 = F; p.nB1 = F;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = F / 128;
-  p.out = OutDesc{}; p.act = act; p.F = F; p.status = status;
+  p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status;
+  p.f16 = f16; p.dup_base = nullptr; p.dup_stride = 0;
   return launch_cfg<256, 4, EPI_SWIGLU>(ta, tg, tu, tu, p, st);
 }
 

@@ -203,14 +203,12 @@ template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *
 
 // ---------------------------------------------------------------------------------------------------------
 // single-query attention over the cache, split along the keys.
-//   pass 1: block (split, head, prompt) scans its key range with 4 warps -- 32 keys at a time, one key per
-//           lane for the scores (128-bit loads of the K row), online softmax, then the probabilities are
-//           broadcast while the lanes accumulate their slice of the output -- merges the warps in shared
-//           memory and writes (max, sum, acc[hd]) to scratch;
+//   pass 1: block (split, KV head, prompt), one warp per query head of the group, scans its key range 32 keys
+//           at a time -- one key per lane for the scores (128-bit loads of the K row), online softmax, then the
+//           probabilities are broadcast while the lanes accumulate their slice of the output -- and writes
+//           (max, sum, acc[hd]) to scratch;
 //   pass 2: block (head, prompt) merges the splits and writes the normalised fp32 output row.
 // ---------------------------------------------------------------------------------------------------------
-constexpr int TAIL_WARPS = 4;
-
 __host__ __device__ inline int tail_chunk(int max_seq_len) {
   int c = (max_seq_len + 63) / 64;          // at most 64 splits
   c = (c + 31) / 32 * 32;
@@ -234,69 +232,57 @@ __device__ __forceinline__ float dot_row(const float *__restrict__ qs, const T *
   return dot;
 }
 
+// Block (split, KV head, prompt); warp w = query head kvh*rep + w of that KV head's group, so the K / V rows of
+// the block's key range come from HBM once and are shared by the group's heads through L1.
 template <typename T, int MAX_E>
-__global__ void __launch_bounds__(TAIL_WARPS * 32) tail_attention_partial_kernel(
+__global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
     int n_q, int n_kv, int hd, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
-  extern __shared__ float sm[];   // q[hd] | per-warp (m, l) [2*TAIL_WARPS] | per-warp acc [TAIL_WARPS*hd]
-  float *qs = sm;
-  float *ml = sm + hd;
-  float *accs = ml + 2 * TAIL_WARPS;
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rep = n_q / n_kv;
   const int first = cu[b], n = cu[b + 1] - cu[b];
-  const int kvh = h / (n_q / n_kv);
   const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
-  const float *qr = q + ((size_t)b * n_q + h) * hd;
-  for (int i = threadIdx.x; i < hd; i += blockDim.x) qs[i] = qr[i] * scale;
-  __syncthreads();
-
-  float m = -INFINITY, l = 0.f;
-  float acc[MAX_E];
+  for (int hw = warp; hw < rep; hw += (blockDim.x >> 5)) {   // (more heads per group than warps: loop)
+    const int h = kvh * rep + hw;
+    float *qs = sm + hw * hd;
+    const float *qr = q + ((size_t)b * n_q + h) * hd;
+    for (int i = lane; i < hd; i += 32) qs[i] = qr[i] * scale;
+    __syncwarp();
+    float m = -INFINITY, l = 0.f;
+    float acc[MAX_E];
 #pragma unroll
-  for (int e = 0; e < MAX_E; ++e) acc[e] = 0.f;
-  for (int c0 = k_begin + warp * 32; c0 < k_end; c0 += TAIL_WARPS * 32) {
-    const int key = c0 + lane;
-    float s = -INFINITY;
-    if (key < k_end) s = dot_row<T>(qs, kc + ((size_t)(first + key) * n_kv + kvh) * hd, hd);
-    const float m_new = fmaxf(m, warp_max(s));
-    const float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
-    const float corr = __expf(m - m_new);
-    l = l * corr + warp_sum(pe);
+    for (int e = 0; e < MAX_E; ++e) acc[e] = 0.f;
+    for (int c0 = k_begin; c0 < k_end; c0 += 32) {
+      const int key = c0 + lane;
+      float s = -INFINITY;
+      if (key < k_end) s = dot_row<T>(qs, kc + ((size_t)(first + key) * n_kv + kvh) * hd, hd);
+      const float m_new = fmaxf(m, warp_max(s));
+      const float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
+      const float corr = __expf(m - m_new);
+      l = l * corr + warp_sum(pe);
 #pragma unroll
-    for (int e = 0; e < MAX_E; ++e) acc[e] *= corr;
-    m = m_new;
-    const int n_here = min(32, k_end - c0);
-    for (int i = 0; i < n_here; ++i) {
-      const float pi = __shfl_sync(0xffffffffu, pe, i);
-      const T *vr = vc + ((size_t)(first + c0 + i) * n_kv + kvh) * hd;
+      for (int e = 0; e < MAX_E; ++e) acc[e] *= corr;
+      m = m_new;
+      const int n_here = min(32, k_end - c0);
+      for (int i = 0; i < n_here; ++i) {
+        const float pi = __shfl_sync(0xffffffffu, pe, i);
+        const T *vr = vc + ((size_t)(first + c0 + i) * n_kv + kvh) * hd;
 #pragma unroll
-      for (int e = 0; e < MAX_E; ++e) {
-        const int dd = lane + 32 * e;
-        if (dd < hd) acc[e] = fmaf(pi, to_f(vr[dd]), acc[e]);
+        for (int e = 0; e < MAX_E; ++e) {
+          const int dd = lane + 32 * e;
+          if (dd < hd) acc[e] = fmaf(pi, to_f(vr[dd]), acc[e]);
+        }
       }
     }
-  }
-  if (lane == 0) { ml[2 * warp] = m; ml[2 * warp + 1] = l; }
+    float *dst = scratch + (((size_t)b * n_q + h) * n_splits + split) * (hd + 2);
+    if (lane == 0) { dst[0] = m; dst[1] = l; }
 #pragma unroll
-  for (int e = 0; e < MAX_E; ++e) {
-    const int dd = lane + 32 * e;
-    if (dd < hd) accs[warp * hd + dd] = acc[e];
-  }
-  __syncthreads();
-  float M = -INFINITY;
-#pragma unroll
-  for (int w = 0; w < TAIL_WARPS; ++w) M = fmaxf(M, ml[2 * w]);
-  float *dst = scratch + (((size_t)b * n_q + h) * n_splits + split) * (hd + 2);
-  float Lsum = 0.f;
-#pragma unroll
-  for (int w = 0; w < TAIL_WARPS; ++w) Lsum += (ml[2 * w] == -INFINITY) ? 0.f : ml[2 * w + 1] * __expf(ml[2 * w] - M);
-  if (threadIdx.x == 0) { dst[0] = M; dst[1] = Lsum; }
-  for (int dd = threadIdx.x; dd < hd; dd += blockDim.x) {
-    float a = 0.f;
-#pragma unroll
-    for (int w = 0; w < TAIL_WARPS; ++w) a += (ml[2 * w] == -INFINITY) ? 0.f : accs[w * hd + dd] * __expf(ml[2 * w] - M);
-    dst[2 + dd] = a;
+    for (int e = 0; e < MAX_E; ++e) {
+      const int dd = lane + 32 * e;
+      if (dd < hd) dst[2 + dd] = acc[e];
+    }
   }
 }
 
@@ -335,12 +321,14 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out,
   const int chunk = tail_chunk(max_seq_len);
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
   const float scale = 1.0f / sqrtf((float)hd);
-  const size_t smem = (size_t)(hd + 2 * TAIL_WARPS + TAIL_WARPS * hd) * sizeof(float);
-  dim3 grid(n_splits, n_q, n_seqs);
-  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else tail_attention_partial_kernel<T, 8><<<grid, TAIL_WARPS * 32, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  const int rep = n_q / n_kv;
+  const int threads = 32 * (rep < 8 ? rep : 8);
+  const size_t smem = (size_t)rep * hd * sizeof(float);
+  dim3 grid(n_splits, n_kv, n_seqs);
+  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
 template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *, int,

@@ -94,12 +94,13 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
   d |= (uint64_t)2 << 61;    // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor for kind::f16 with bf16 A/B and fp32 accumulation.
-// a_mn / b_mn: 1 if that operand is MN-major (0 = K-major).
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, int a_mn, int b_mn) {
-  return (1u << 4)                 // D format: F32
-         | (1u << 7)               // A format: BF16
-         | (1u << 10)              // B format: BF16
+// Instruction descriptor for kind::f16 with 16-bit A/B and fp32 accumulation.
+// a_mn / b_mn: 1 if that operand is MN-major (0 = K-major); a_f16 / b_f16: 1 = IEEE half, 0 = bfloat16
+// (the two operands may differ: fp16 activations against bf16 weights / cache).
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int a_mn, int b_mn, int a_f16, int b_f16) {
+  return (1u << 4)                                   // D format: F32
+         | ((a_f16 ? 0u : 1u) << 7)                  // A format: 0 = F16, 1 = BF16
+         | ((b_f16 ? 0u : 1u) << 10)                 // B format
          | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
          | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
@@ -191,6 +192,16 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
+}
+// two floats -> packed IEEE halves, round to nearest, saturating at +-65504 (never inf)
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// activation storage format chosen at run time (uniform across the grid)
+__device__ __forceinline__ uint32_t pack_act(float lo, float hi, bool f16) {
+  return f16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
 }
 
 }  // namespace tc

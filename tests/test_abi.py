@@ -67,7 +67,7 @@ def test_null_arguments_return_status_codes(lib):
     assert lib.swiftkv_kv_cache_view(None, 0, None) == -1
     assert lib.swiftkv_first_logits(None, None, None) == -1
     assert lib.swiftkv_status(None, None) == -1
-    assert lib.swiftkv_gemm_bf16(None, None, None, 1, 1, 1, None) == -1
+    assert lib.swiftkv_gemm_tc(None, None, None, 1, 1, 1, 1, None) == -1
     lib.swiftkv_model_free(None)
 
 

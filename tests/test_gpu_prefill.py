@@ -20,13 +20,15 @@ MID = S.ModelShape(1024, 512, 4, 8, 2, 128, 1024, 500000.0, 1e-5, "mid")
 W8B_4L = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-width-4-layers")
 
 
-def _run(shape, dtype, seed, lens, l, g, max_tokens=None, kernel_mask=None):
+def _run(shape, dtype, seed, lens, l, g, max_tokens=None, kernel_mask=None, act_format=None):
     import paper_2410_03960_b200 as P
     w = S.make_weights(shape, seed, dtype, "cuda")
     tok = S.make_prompts(seed, lens, shape.vocab)
     model = P.SwiftKVModel(shape, w, dtype, max_tokens or sum(lens), len(lens), l, g)
     if kernel_mask is not None:
         model.set_kernel_mask(kernel_mask)
+    if act_format is not None:
+        model.set_activation_format(act_format)
     model.prefill(tok, lens, l, g)
     model.status()
     ref = O.swiftkv(oracle_config(shape), oracle_weights(w), tok.numpy(), lens, l, g)
@@ -41,9 +43,10 @@ def test_config1_fp32(l, g):
     check_prefill_against_oracle(model, ref, S.TINY.n_layers, 1e-4, 1e-4, 1e-3)
 
 
+@pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2)])
-def test_config1_bf16(l, g):
-    model, ref, _, _ = _run(S.TINY, torch.bfloat16, 0, [128, 96], l, g)
+def test_config1_bf16(l, g, act):
+    model, ref, _, _ = _run(S.TINY, torch.bfloat16, 0, [128, 96], l, g, act_format=act)
     check_prefill_against_oracle(model, ref, S.TINY.n_layers, 2e-2, 2e-2, 0.1)
 
 
@@ -60,12 +63,13 @@ def test_more_prompts_than_one_tail_pass():
 
 
 @pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2), (2, 2)])
-@pytest.mark.parametrize("mask", [3, 0])
-def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask):
-    """The same model through the tcgen05 kernels (mask 3) and the SIMT kernels (mask 0); several row tiles and a
-    ragged tail (T = 507), prompts of 1 and 129 tokens included."""
+@pytest.mark.parametrize("mask,act", [(3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
+def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask, act):
+    """The same model through the tcgen05 kernels (mask 3), the SIMT kernels (mask 0) and the two mixtures, with
+    half (act 1) and bfloat16 (act 0) activations; several row tiles and a ragged tail (T = 507), prompts of 1 and
+    129 tokens included."""
     lens = [300, 77, 129, 1]
-    model, ref, _, _ = _run(MID, torch.bfloat16, 2, lens, l, g, kernel_mask=mask)
+    model, ref, _, _ = _run(MID, torch.bfloat16, 2, lens, l, g, kernel_mask=mask, act_format=act)
     check_prefill_against_oracle(model, ref, MID.n_layers, 2e-2, 2e-2, 0.1)
 
 
@@ -122,3 +126,63 @@ def test_llama8b_width_reduced_depth():
     model, ref, _, _ = _run(W8B_4L, torch.bfloat16, 1, lens, 2, 1)
     res = check_prefill_against_oracle(model, ref, W8B_4L.n_layers, 2e-2, 2e-2, 0.1)
     print("8b-width parity:", res)
+
+
+W70B_2L = S.ModelShape(128256, 8192, 2, 64, 8, 128, 28672, 500000.0, 1e-5, "70b-width-2-layers")
+
+
+def test_llama70b_width_reduced_depth():
+    """Llama-3.1-70B widths (hidden 8192, 64/8 heads of 128 -- 8 query heads per KV head --, FFN 28672), 2 layers,
+    l = 1: the config-4 GEMM / attention / last-token shapes at a size the oracle finishes in seconds."""
+    lens = [200, 1, 140]
+    model, ref, _, _ = _run(W70B_2L, torch.bfloat16, 3, lens, 1, 1)
+    res = check_prefill_against_oracle(model, ref, W70B_2L.n_layers, 2e-2, 2e-2, 0.1)
+    print("70b-width parity:", res)
+
+
+def _truncated(lens, factor):
+    return [max(1, n // factor) for n in lens]
+
+
+@pytest.mark.parametrize("cfg_name,seed,full_lens,l,g,factor", [
+    ("config2", 1, S.uniform_lengths(1, 8, 2048, 8192), 16, 1, 32),      # 8 prompts U[2048, 8192], l = 16
+    ("config3", 2, [16384] * 4, 24, 2, 64),                               # 4 x 16384, l = 24, AcrossKV 2
+])
+def test_llama8b_full_depth_truncated_prompts(cfg_name, seed, full_lens, l, g, factor):
+    """The full 32-layer Llama-3.1-8B shape with the named seeds, l and g, prompts cut to their first n/factor
+    tokens (ragged lengths survive): every layer's cache and the first-token logits against the oracle."""
+    lens = _truncated(full_lens, factor)
+    model, ref, _, _ = _run(S.LLAMA31_8B, torch.bfloat16, seed, lens, l, g)
+    res = check_prefill_against_oracle(model, ref, 32, 2e-2, 2e-2, 0.1)
+    print(cfg_name, "truncated parity:", lens, res)
+
+
+def test_config2_full_size_prefix_parity_and_determinism():
+    """The benchmark's configuration at full size (41123 tokens, l = 16): by causality the cache rows of the first P
+    tokens of every prompt equal those of the truncated prompts, which the oracle can afford; the logits of the
+    full-length run are checked for run-to-run bitwise determinism and finiteness."""
+    import paper_2410_03960_b200 as P
+    shape, seed, l, g, prefix = S.LLAMA31_8B, 1, 16, 1, 24
+    lens = S.uniform_lengths(seed, 8, 2048, 8192)
+    assert sum(lens) == 41123
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    logits1 = model.first_logits().clone()
+    assert torch.isfinite(logits1).all()
+    # the oracle on the first `prefix` tokens of every prompt
+    short = [prefix] * len(lens)
+    tok_short = S.make_prompts(seed, short, shape.vocab)
+    ref = O.swiftkv(oracle_config(shape), oracle_weights(w), tok_short.numpy(), short, l, g)
+    offs = np.concatenate([[0], np.cumsum(lens)])[:-1]
+    rows = np.concatenate([np.arange(o, o + prefix) for o in offs])
+    idx = torch.as_tensor(rows, device="cuda")
+    for j in range(shape.n_layers):
+        K, V, _ = model.kv_cache_view(j)
+        assert rel_l2(to_np(K[idx]), ref["K"][j]) <= 2e-2, j
+        assert rel_l2(to_np(V[idx]), ref["V"][j]) <= 2e-2, j
+    model.prefill(tok, lens, l, g)
+    model.status()
+    assert torch.equal(logits1, model.first_logits())
