@@ -89,7 +89,7 @@ struct swiftkv_model {
   int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;
   int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
-  int kernel_mask = 3;
+  int kernel_mask = 7;
   int act_format = SWIFTKV_ACT_F16;
   // profiling
   bool profiling = false;
@@ -484,6 +484,7 @@ static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool toke
   if (dev != m->device) return fail(SWIFTKV_ERR_INVALID_ARG, "current device %d is not the model's device %d", dev, m->device);
 
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  tc_gemm_use_cta_pairs((m->kernel_mask & 4) != 0, (m->kernel_mask & 8) != 0);
   m->ready = false;
   m->launches = 0;
   m->host_meta.resize(n_seqs + 1);
@@ -575,7 +576,7 @@ extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, flo
 extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
 extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   if (!m) return 0;
-  m->kernel_mask = mask & 3;
+  m->kernel_mask = mask & 15;
   return m->kernel_mask;
 }
 

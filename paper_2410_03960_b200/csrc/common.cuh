@@ -110,6 +110,8 @@ void launch_gemm_simt(const TA *A, const TW *B, int M, int N, int K, OutDesc out
 // gemm_tc.cu : tcgen05 / TMEM / TMA GEMMs (bf16)
 struct TcGemmPlan;   // host object holding tensor maps
 bool tc_gemm_supported(int M, int N, int K);
+// CTA-pair (cta_group::2) kernels on / off (default on)
+void tc_gemm_use_cta_pairs(bool on, bool swiglu_too);
 // generic: B rows come from up to three matrices stacked along N: [0,nB0) from B0, [nB0, nB0+nB1) from B1, rest B2
 // rope != nullptr: the rotary embedding (rotate-half pairs (i, i + hd/2)) is applied in the epilogue, in fp32,
 // to the columns below out.n0 and to the even-numbered segments above it (K planes; odd ones are V planes)
