@@ -19,7 +19,16 @@ __global__ void __launch_bounds__(256) tail_rmsnorm_kernel(const float *__restri
   float *orow = out + (size_t)blockIdx.x * d;
   __shared__ float red[8];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) ss += yr[i] * yr[i];
+  const bool vec = (d & 3) == 0;
+  if (vec) {
+#pragma unroll 4
+    for (int i = threadIdx.x * 4; i < d; i += 1024) {
+      const float4 v = *reinterpret_cast<const float4 *>(yr + i);
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  } else {
+    for (int i = threadIdx.x; i < d; i += blockDim.x) ss += yr[i] * yr[i];
+  }
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
@@ -27,7 +36,16 @@ __global__ void __launch_bounds__(256) tail_rmsnorm_kernel(const float *__restri
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float rstd = rsqrtf(tot / (float)d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) orow[i] = yr[i] * rstd * to_f(gamma[i]);
+  if (vec) {
+#pragma unroll 4
+    for (int i = threadIdx.x * 4; i < d; i += 1024) {
+      const float4 v = *reinterpret_cast<const float4 *>(yr + i);
+      *reinterpret_cast<float4 *>(orow + i) = make_float4(v.x * rstd * to_f(gamma[i]), v.y * rstd * to_f(gamma[i + 1]),
+                                                          v.z * rstd * to_f(gamma[i + 2]), v.w * rstd * to_f(gamma[i + 3]));
+    }
+  } else {
+    for (int i = threadIdx.x; i < d; i += blockDim.x) orow[i] = yr[i] * rstd * to_f(gamma[i]);
+  }
 }
 template <typename T>
 void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, int d, float eps, cudaStream_t st) {
@@ -89,7 +107,7 @@ __global__ void __launch_bounds__(256) skinny_generic_kernel(const float *__rest
 // A block = 8 warps works on one 16-feature tile with K split across the warps, then reduces in shared memory.
 // ---------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -120,38 +138,51 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
   const bool tok_ok = g < n_rows;
   float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
   const int steps = K / 32;
-#pragma unroll 2
-  for (int s = warp; s < steps; s += SK_WARPS) {
-    const int kb = s * 32;
-    const uint4 wl = __ldcs(reinterpret_cast<const uint4 *>(w_lo + kb));   // weights are streamed once
-    const uint4 wh = __ldcs(reinterpret_cast<const uint4 *>(w_hi + kb));
-    uint4 ul, uh;
-    if (SWIGLU) {
-      ul = __ldcs(reinterpret_cast<const uint4 *>(u_lo + kb));
-      uh = __ldcs(reinterpret_cast<const uint4 *>(u_hi + kb));
+  // software pipeline: the loads of U K-steps are issued together before any of their MMAs, so that each lane keeps
+  // 2U (4U with SwiGLU) 16-byte weight loads in flight
+  constexpr int U = SWIGLU ? 2 : 4;
+  for (int s0 = warp; s0 < steps; s0 += U * SK_WARPS) {
+    uint4 wl[U], wh[U], ul[U], uh[U];
+    float4 xa[U], xb[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int s = s0 + u * SK_WARPS;
+      const bool on = s < steps;
+      const int kb = on ? s * 32 : 0;
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      wl[u] = on ? __ldcs(reinterpret_cast<const uint4 *>(w_lo + kb)) : z;   // weights are streamed once
+      wh[u] = on ? __ldcs(reinterpret_cast<const uint4 *>(w_hi + kb)) : z;
+      if (SWIGLU) {
+        ul[u] = on ? __ldcs(reinterpret_cast<const uint4 *>(u_lo + kb)) : z;
+        uh[u] = on ? __ldcs(reinterpret_cast<const uint4 *>(u_hi + kb)) : z;
+      }
+      xa[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      xb[u] = xa[u];
+      if (tok_ok && on) {
+        xa[u] = *reinterpret_cast<const float4 *>(a_row + kb);
+        xb[u] = *reinterpret_cast<const float4 *>(a_row + kb + 4);
+      }
     }
-    float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0;
-    if (tok_ok) {
-      x0 = *reinterpret_cast<const float4 *>(a_row + kb);
-      x1 = *reinterpret_cast<const float4 *>(a_row + kb + 4);
-    }
-    uint32_t bh[4], bl[4];
-    split_hi_lo(x0.x, x0.y, bh[0], bl[0]);
-    split_hi_lo(x0.z, x0.w, bh[1], bl[1]);
-    split_hi_lo(x1.x, x1.y, bh[2], bl[2]);
-    split_hi_lo(x1.z, x1.w, bh[3], bl[3]);
-    // first MMA: K slots (2t,2t+1) <- elements 0,1 and (2t+8,2t+9) <- elements 2,3; second MMA: elements 4..7
-    const uint32_t a1[4] = {wl.x, wh.x, wl.y, wh.y}, a2[4] = {wl.z, wh.z, wl.w, wh.w};
-    mma_bf16_16816(c, a1, bh[0], bh[1]);
-    mma_bf16_16816(c, a1, bl[0], bl[1]);
-    mma_bf16_16816(c, a2, bh[2], bh[3]);
-    mma_bf16_16816(c, a2, bl[2], bl[3]);
-    if (SWIGLU) {
-      const uint32_t d1[4] = {ul.x, uh.x, ul.y, uh.y}, d2[4] = {ul.z, uh.z, ul.w, uh.w};
-      mma_bf16_16816(c2, d1, bh[0], bh[1]);
-      mma_bf16_16816(c2, d1, bl[0], bl[1]);
-      mma_bf16_16816(c2, d2, bh[2], bh[3]);
-      mma_bf16_16816(c2, d2, bl[2], bl[3]);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      uint32_t bh[4], bl[4];
+      split_hi_lo(xa[u].x, xa[u].y, bh[0], bl[0]);
+      split_hi_lo(xa[u].z, xa[u].w, bh[1], bl[1]);
+      split_hi_lo(xb[u].x, xb[u].y, bh[2], bl[2]);
+      split_hi_lo(xb[u].z, xb[u].w, bh[3], bl[3]);
+      // first MMA: K slots (2t,2t+1) <- elements 0,1 and (2t+8,2t+9) <- elements 2,3; second MMA: elements 4..7
+      const uint32_t a1[4] = {wl[u].x, wh[u].x, wl[u].y, wh[u].y}, a2[4] = {wl[u].z, wh[u].z, wl[u].w, wh[u].w};
+      mma_bf16_16816(c, a1, bh[0], bh[1]);
+      mma_bf16_16816(c, a1, bl[0], bl[1]);
+      mma_bf16_16816(c, a2, bh[2], bh[3]);
+      mma_bf16_16816(c, a2, bl[2], bl[3]);
+      if (SWIGLU) {
+        const uint32_t d1[4] = {ul[u].x, uh[u].x, ul[u].y, uh[u].y}, d2[4] = {ul[u].z, uh[u].z, ul[u].w, uh[u].w};
+        mma_bf16_16816(c2, d1, bh[0], bh[1]);
+        mma_bf16_16816(c2, d1, bl[0], bl[1]);
+        mma_bf16_16816(c2, d2, bh[2], bh[3]);
+        mma_bf16_16816(c2, d2, bl[2], bl[3]);
+      }
     }
   }
 #pragma unroll
@@ -232,8 +263,114 @@ __device__ __forceinline__ float dot_row(const float *__restrict__ qs, const T *
   return dot;
 }
 
-// Block (split, KV head, prompt); warp w = query head kvh*rep + w of that KV head's group, so the K / V rows of
-// the block's key range come from HBM once and are shared by the group's heads through L1.
+// Block (split, KV head, prompt), 4 warps.  Every warp walks 32-key chunks of the block's key range for ALL query heads
+// of the KV head's group at once, so each K and V row is fetched once per group:
+//   scores : lane = key; the 256-byte K row is read with 128-bit loads and dotted with the REP query vectors (smem)
+//   softmax: online, per head, warp-wide max / sum
+//   output : for each of the 32 keys the V row is read once (coalesced, lane = 4 consecutive dims) and accumulated
+//            into REP x 4 registers with the probabilities broadcast by shuffle
+// then the warps are merged in shared memory and (max, sum, acc[hd]) per head goes to scratch.
+constexpr int TA_WARPS = 4;
+template <typename T, int REP, int HD>
+__global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
+    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
+    int n_q, int n_kv, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
+  static_assert(HD == 128, "one lane owns 4 consecutive output dims");
+  __shared__ float qs[REP][HD];
+  __shared__ float w_m[TA_WARPS][REP], w_l[TA_WARPS][REP];
+  __shared__ float w_acc[TA_WARPS][REP][HD];
+  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int first = cu[b], n = cu[b + 1] - cu[b];
+  const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
+  for (int i = threadIdx.x; i < REP * HD; i += blockDim.x)
+    qs[i / HD][i % HD] = q[((size_t)b * n_q + kvh * REP + i / HD) * HD + i % HD] * scale;
+  __syncthreads();
+
+  float m[REP], l[REP], acc[REP][4];
+#pragma unroll
+  for (int r = 0; r < REP; ++r) { m[r] = -INFINITY; l[r] = 0.f; acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f; }
+
+  for (int c0 = k_begin + warp * 32; c0 < k_end; c0 += TA_WARPS * 32) {
+    const int key = c0 + lane;
+    const bool valid = key < k_end;
+    float sc[REP];
+#pragma unroll
+    for (int r = 0; r < REP; ++r) sc[r] = 0.f;
+    if (valid) {
+      const T *kr = kc + ((size_t)(first + key) * n_kv + kvh) * HD;
+      constexpr int V = 16 / sizeof(T);
+#pragma unroll 4
+      for (int i = 0; i < HD; i += V) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(kr + i);
+        const T *e = reinterpret_cast<const T *>(&raw);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+          const float kv_ = to_f(e[k]);
+#pragma unroll
+          for (int r = 0; r < REP; ++r) sc[r] = fmaf(qs[r][i + k], kv_, sc[r]);
+        }
+      }
+    }
+    float pe[REP];
+#pragma unroll
+    for (int r = 0; r < REP; ++r) {
+      const float s = valid ? sc[r] : -INFINITY;
+      const float m_new = fmaxf(m[r], warp_max(s));
+      pe[r] = valid ? __expf(s - m_new) : 0.f;
+      const float corr = __expf(m[r] - m_new);
+      l[r] = l[r] * corr + warp_sum(pe[r]);
+      acc[r][0] *= corr; acc[r][1] *= corr; acc[r][2] *= corr; acc[r][3] *= corr;
+      m[r] = m_new;
+    }
+    const int n_here = min(32, k_end - c0);
+    const T *vbase = vc + ((size_t)(first + c0) * n_kv + kvh) * HD + lane * 4;
+#pragma unroll 4
+    for (int i = 0; i < n_here; ++i) {
+      const T *vr = vbase + (size_t)i * n_kv * HD;
+      float v0, v1, v2, v3;
+      if constexpr (sizeof(T) == 2) {
+        const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
+        const T *e = reinterpret_cast<const T *>(&raw);
+        v0 = to_f(e[0]); v1 = to_f(e[1]); v2 = to_f(e[2]); v3 = to_f(e[3]);
+      } else {
+        const float4 raw = *reinterpret_cast<const float4 *>(vr);
+        v0 = raw.x; v1 = raw.y; v2 = raw.z; v3 = raw.w;
+      }
+#pragma unroll
+      for (int r = 0; r < REP; ++r) {
+        const float pi = __shfl_sync(0xffffffffu, pe[r], i);
+        acc[r][0] = fmaf(pi, v0, acc[r][0]); acc[r][1] = fmaf(pi, v1, acc[r][1]);
+        acc[r][2] = fmaf(pi, v2, acc[r][2]); acc[r][3] = fmaf(pi, v3, acc[r][3]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < REP; ++r) {
+    if (lane == 0) { w_m[warp][r] = m[r]; w_l[warp][r] = l[r]; }
+    *reinterpret_cast<float4 *>(&w_acc[warp][r][lane * 4]) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < REP * HD; idx += blockDim.x) {
+    const int r = idx / HD, dd = idx % HD;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < TA_WARPS; ++w) M = fmaxf(M, w_m[w][r]);
+    float a = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < TA_WARPS; ++w) {
+      const float f = (w_m[w][r] == -INFINITY) ? 0.f : __expf(w_m[w][r] - M);
+      a += w_acc[w][r][dd] * f;
+      L += w_l[w][r] * f;
+    }
+    float *dst = scratch + (((size_t)b * n_q + kvh * REP + r) * n_splits + split) * (HD + 2);
+    if (dd == 0) { dst[0] = M; dst[1] = L; }
+    dst[2 + dd] = a;
+  }
+}
+
+// Shape-generic form: block (split, KV head, prompt); warp w = query head kvh*rep + w of that KV head's group, so the
+// K / V rows of the block's key range come from HBM once and are shared by the group's heads through L1.
 template <typename T, int MAX_E>
 __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
@@ -322,6 +459,15 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out,
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
   const float scale = 1.0f / sqrtf((float)hd);
   const int rep = n_q / n_kv;
+  if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
+    dim3 grid(n_splits, n_kv, n_seqs);
+    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
+    tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
+    return;
+  }
   const int threads = 32 * (rep < 8 ? rep : 8);
   const size_t smem = (size_t)rep * hd * sizeof(float);
   dim3 grid(n_splits, n_kv, n_seqs);
