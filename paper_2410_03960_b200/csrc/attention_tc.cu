@@ -11,6 +11,8 @@
 // Online softmax keeps a per-row reference max that only moves when the running max grows by more than 2^8
 // (then O_w is rescaled in tensor memory); the final O_w / l_w is exact for any such reference.
 // Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each (all 512).  Every wait is bounded.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -57,7 +59,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 // ACT_F16: q, K, V, P and the output are all IEEE halves (else all bfloat16)
-template <bool ACT_F16>
+template <bool ACT_F16, bool SPLIT_P>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, AttnParams p) {
@@ -83,9 +85,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint64_t *v_full = bars + 5;        // [2]
   uint64_t *v_empty = bars + 7;       // [2]
   uint64_t *s_full = bars + 9;        // [2]  S_w ready in tensor memory
-  uint64_t *p_ready = bars + 11;      // [2]  P_w written (and O_w rescaled) by the softmax warps
-  uint64_t *o_full = bars + 13;       // [1]
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 14);
+  uint64_t *p_ready = bars + 11;      // [2]  first 64 keys of P_w written (and O_w rescaled) by the softmax warps
+  uint64_t *p_ready2 = bars + 13;     // [2]  last 64 keys of P_w written
+  uint64_t *o_full = bars + 15;       // [1]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,6 +101,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::mbar_init(tc::smem_u32(&v_empty[s]), 1);
       tc::mbar_init(tc::smem_u32(&s_full[s]), 1);
       tc::mbar_init(tc::smem_u32(&p_ready[s]), 4);   // one arrival per softmax warp
+      tc::mbar_init(tc::smem_u32(&p_ready2[s]), 4);
     }
     tc::mbar_init(tc::smem_u32(o_full), 1);
     *abort_flag = 0;
@@ -151,12 +155,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                       idesc_qk, kk != 0);
         }
       };
-      auto issue_pv = [&](int w, int s, bool accumulate) {   // O_w (+)= P_w V : 8 steps of 16 keys
+      // O_w (+)= P_w V : 8 steps of 16 keys, issued in two halves so that the first 64 keys can run on the tensor
+      // pipe while the softmax warps still exponentiate the last 64
+      auto issue_pv = [&](int w, int s, bool accumulate, int half) {
         const uint32_t b0 = tc::smem_u32(smem + SM_V + s * TILE_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < BKV / 16; ++kk)
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const int kk = half * 4 + k4;
           tc::umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + kk * 8,
                       tc::umma_desc_sw128(b0 + kk * 16 * 128, CHUNK_BYTES, 1024), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+        }
       };
       bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) &&
                 wait_or_abort(tc::smem_u32(&k_full[0]), 0, abort_flag, p.status);
@@ -175,7 +183,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (!wait_or_abort(tc::smem_u32(&v_full[s]), ph, abort_flag, p.status)) { ok = false; break; }
         if (!wait_or_abort(tc::smem_u32(&p_ready[0]), j & 1, abort_flag, p.status)) { ok = false; break; }
         tc::tc_fence_after_sync();
-        issue_pv(0, s, j > 0);
+        issue_pv(0, s, j > 0, 0);
+        if (SPLIT_P) {
+          if (!wait_or_abort(tc::smem_u32(&p_ready2[0]), j & 1, abort_flag, p.status)) { ok = false; break; }
+          tc::tc_fence_after_sync();
+        }
+        issue_pv(0, s, j > 0, 1);
         if (more) {
           if (!wait_or_abort(tc::smem_u32(&k_full[s1]), ph1, abort_flag, p.status)) { ok = false; break; }
           tc::tc_fence_after_sync();
@@ -184,7 +197,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         if (!wait_or_abort(tc::smem_u32(&p_ready[1]), j & 1, abort_flag, p.status)) { ok = false; break; }
         tc::tc_fence_after_sync();
-        issue_pv(1, s, j > 0);
+        issue_pv(1, s, j > 0, 0);
+        if (SPLIT_P) {
+          if (!wait_or_abort(tc::smem_u32(&p_ready2[1]), j & 1, abort_flag, p.status)) { ok = false; break; }
+          tc::tc_fence_after_sync();
+        }
+        issue_pv(1, s, j > 0, 1);
         tc::umma_commit(tc::smem_u32(&v_empty[s]));
         if (more) {
           issue_qk(1, s1);
@@ -209,21 +227,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (!wait_or_abort(tc::smem_u32(&s_full[w]), j & 1, abort_flag, p.status)) { ok = false; break; }
       tc::tc_fence_after_sync();
       const bool diag = (j == qt);
-      // the whole score row (128 fp32) in registers: one pass over tensor memory
+      // the whole score row (128 fp32) in registers: one pass over tensor memory, the second half of the loads in
+      // flight while the first half is reduced
       uint32_t s[128];
       tc::tmem_ld_32x32b_x32p(t_s, s);
       tc::tmem_ld_32x32b_x32p(t_s + 32, s + 32);
+      tc::tmem_ld_wait();
       tc::tmem_ld_32x32b_x32p(t_s + 64, s + 64);
       tc::tmem_ld_32x32b_x32p(t_s + 96, s + 96);
-      tc::tmem_ld_wait();
       if (diag) {   // causal mask, only on the diagonal tile: key index > query index
 #pragma unroll
-        for (int i = 0; i < 128; ++i)
+        for (int i = 0; i < 64; ++i)
           if (i > row) s[i] = 0xff800000u;   // -inf
       }
       float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-      for (int i = 0; i < 128; i += 8) {
+      for (int i = 0; i < 64; i += 8) {
+        m0 = tc::max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        m1 = tc::max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        m2 = tc::max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        m3 = tc::max3(m3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+      }
+      tc::tmem_ld_wait();
+      if (diag) {
+#pragma unroll
+        for (int i = 64; i < 128; ++i)
+          if (i > row) s[i] = 0xff800000u;
+      }
+#pragma unroll
+      for (int i = 64; i < 128; i += 8) {
         m0 = tc::max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
         m1 = tc::max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
         m2 = tc::max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
@@ -248,26 +280,31 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
       }
       m_ref = m_new;
-      // p = 2^(s*c - m_ref*c) (masked entries: 2^-inf = 0), row sum, bf16 P written over S (64 packed columns)
+      // p = 2^(s*c - m_ref*c) (masked entries: 2^-inf = 0), row sum, 16-bit P written over S (64 packed columns) in
+      // two halves of 64 keys, each announced to the MMA warp as soon as it is in tensor memory
       const float neg_mc = -m_ref * c;
       float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-      for (int i = 0; i < 64; i += 2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, neg_mc));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, neg_mc));
-        const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 2]), c, neg_mc));
-        const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 3]), c, neg_mc));
-        l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-        s[i] = ACT_F16 ? tc::pack_f16x2(p0, p1) : tc::pack_bf16x2(p0, p1);
-        s[i + 1] = ACT_F16 ? tc::pack_f16x2(p2, p3) : tc::pack_bf16x2(p2, p3);
+      for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+        for (int i = hf * 32; i < hf * 32 + 32; i += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, neg_mc));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, neg_mc));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 2]), c, neg_mc));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 3]), c, neg_mc));
+          l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+          s[i] = ACT_F16 ? tc::pack_f16x2(p0, p1) : tc::pack_bf16x2(p0, p1);
+          s[i + 1] = ACT_F16 ? tc::pack_f16x2(p2, p3) : tc::pack_bf16x2(p2, p3);
+        }
+        tc::tmem_st_32x32b_x32(t_s + hf * 32, s + hf * 32);
+        if (SPLIT_P || hf == 1) {
+          tc::tmem_st_wait();
+          tc::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(tc::smem_u32((SPLIT_P && hf == 1) ? &p_ready2[w] : &p_ready[w]));
+        }
       }
       l += (l0 + l1) + (l2 + l3);
-      tc::tmem_st_32x32b_x32(t_s, s);
-      tc::tmem_st_32x32b_x32(t_s + 32, s + 32);
-      tc::tmem_st_wait();
-      tc::tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) tc::mbar_arrive(tc::smem_u32(&p_ready[w]));
     }
     // ---- epilogue: O_w / l -> bf16 -> out[token, head, :]
     if (ok && wait_or_abort(tc::smem_u32(o_full), 0, abort_flag, p.status)) {
@@ -319,8 +356,10 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
   if (get_tmap(&tv, v, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attention_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
       return SWIFTKV_ERR_CUDA;
     attr_set = true;
   }
@@ -331,8 +370,15 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
   p.status = status;
   const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
   if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
-  if (act_f16) attention_tc_kernel<true><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
-  else attention_tc_kernel<false><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  static int split = -1;
+  if (split < 0) { const char *e = getenv("SWIFTKV_ATT_SPLIT_P"); split = e ? atoi(e) : 1; }
+  if (act_f16) {
+    if (split) attention_tc_kernel<true, true><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+    else attention_tc_kernel<true, false><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  } else {
+    if (split) attention_tc_kernel<false, true><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+    else attention_tc_kernel<false, false><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
+  }
   return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
 }
 

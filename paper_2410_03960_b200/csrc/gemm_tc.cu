@@ -11,6 +11,7 @@
 // Epilogues: store bf16 (optionally scattered into K/V cache planes), accumulate into the fp32 residual
 // stream, or SwiGLU with the gate and up tiles of the same features side by side in one accumulator.
 // Every mbarrier wait is bounded: on timeout the kernel sets a status bit and every role leaves its loop.
+#include <cstdlib>
 #include <mutex>
 #include <unordered_map>
 
@@ -114,12 +115,13 @@ namespace {
 // ---------------------------------------------------------------------------------------------------------
 constexpr int BM = 128, BK = 64, UMMA_K = 16;
 constexpr int GEMM_THREADS = 192;
-constexpr int GROUP_M = 16;   // tile rasterisation: bands of 16 row-blocks, column-blocks outer, rows inner
+// tile rasterisation: bands of group_m row-blocks, column-blocks outer, rows inner (GemmTcParams::group_m)
 
 struct GemmTcParams {
   int M, N, K;
   int nB0, nB1;          // columns [0,nB0) from B0, [nB0,nB0+nB1) from B1, rest from B2
   int num_m_blocks, num_n_blocks;
+  int group_m;           // raster band height in 128-row blocks
   OutDesc out;
   bf16 *act;             // SwiGLU output [M, F]
   int F;
@@ -141,13 +143,13 @@ struct SmemLayout {
   static constexpr int TOTAL = BAR_OFFSET + 256 + 1024;   // barriers + slack for 1024-byte alignment
 };
 
-__device__ __forceinline__ void tile_coords(int tile, int num_m_blocks, int num_n_blocks, int &m_blk, int &n_blk) {
-  const int band_tiles = GROUP_M * num_n_blocks;
+__device__ __forceinline__ void tile_coords(int tile, int num_m_blocks, int num_n_blocks, int group_m, int &m_blk, int &n_blk) {
+  const int band_tiles = group_m * num_n_blocks;
   const int band = tile / band_tiles;
   const int r = tile - band * band_tiles;
-  const int band_h = min(GROUP_M, num_m_blocks - band * GROUP_M);
+  const int band_h = min(group_m, num_m_blocks - band * group_m);
   n_blk = r / band_h;
-  m_blk = band * GROUP_M + (r - n_blk * band_h);
+  m_blk = band * group_m + (r - n_blk * band_h);
 }
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
@@ -349,7 +351,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
-        tile_coords(tile, p.num_m_blocks, p.num_n_blocks, m_blk, n_blk);
+        tile_coords(tile, p.num_m_blocks, p.num_n_blocks, p.group_m, m_blk, n_blk);
         const CUtensorMap *tb = &tmB0;
         int b_row = n_blk * BN;
         if constexpr (SWIGLU) {
@@ -412,7 +414,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int it = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
       int m_blk, n_blk;
-      tile_coords(tile, p.num_m_blocks, p.num_n_blocks, m_blk, n_blk);
+      tile_coords(tile, p.num_m_blocks, p.num_n_blocks, p.group_m, m_blk, n_blk);
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1;
       if (!wait_or_abort(tc::smem_u32(&tfull_bar[acc]), acc_phase, abort_flag, p.status)) break;
@@ -443,7 +445,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // barriers of both CTAs; the accumulator-empty barrier lives in the leader and takes 8 warp arrivals.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int PAIR_BN = 256;
-constexpr int GROUP_M2 = 8;   // raster bands of 8 pair-rows (2048 rows)
 
 template <int STAGES>
 struct PairSmem {
@@ -496,12 +497,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int num_tiles = num_m2 * num_n;
   const int num_kb = p.K / BK;
   auto coords = [&](int tile, int &m2, int &n_blk) {
-    const int band_tiles = GROUP_M2 * num_n;
+    const int gm2 = max(1, p.group_m >> 1);
+    const int band_tiles = gm2 * num_n;
     const int band = tile / band_tiles;
     const int r = tile - band * band_tiles;
-    const int band_h = min(GROUP_M2, num_m2 - band * GROUP_M2);
+    const int band_h = min(gm2, num_m2 - band * gm2);
     n_blk = r / band_h;
-    m2 = band * GROUP_M2 + (r - n_blk * band_h);
+    m2 = band * gm2 + (r - n_blk * band_h);
   };
 
   if (warp == 0) {
@@ -637,6 +639,15 @@ int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b
 bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (N % 128) == 0 && N >= 128; }
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
 
+static int group_m_setting() {
+  static int v = 0;
+  if (!v) {
+    const char *e = getenv("SWIFTKV_GROUP_M");
+    v = e ? atoi(e) : 16;
+    if (v < 1) v = 16;
+  }
+  return v;
+}
 static bool g_use_pairs = true, g_swiglu_pairs = false;
 void tc_gemm_use_cta_pairs(bool on, bool swiglu_too) { g_use_pairs = on; g_swiglu_pairs = swiglu_too; }
 
@@ -660,7 +671,7 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
   p.M = M; p.N = N; p.K = K; p.nB0 = nB0; p.nB1 = nB1;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = N / BN;
-  p.out = out; p.act = nullptr; p.F = 0; p.status = status;
+  p.out = out; p.act = nullptr; p.F = 0; p.status = status; p.group_m = group_m_setting();
   p.f16 = f16; p.dup_base = reinterpret_cast<__half *>(dup_base); p.dup_stride = dup_stride;
   if (dup_base && !rope) return SWIFTKV_ERR_UNSUPPORTED;
   const bool pairs = g_use_pairs && BN == 256 && M > 128;
@@ -697,7 +708,7 @@ int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg,
   p.M = M; p.N = 2 * F; p.K = K; p.nB0 = F; p.nB1 = F;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = F / 128;
-  p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status;
+  p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status; p.group_m = group_m_setting();
   p.f16 = f16; p.dup_base = nullptr; p.dup_stride = 0;
   // measured on the 8B shape under the power cap: the single-CTA form is 3 % faster for this launch (it already keeps
   // the tensor pipe 85 % busy), while the pair form wins 7-10 % on the N = 4096 / 6144 projections

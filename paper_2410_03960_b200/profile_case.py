@@ -31,6 +31,10 @@ def main() -> None:
     tokens = sum(lens)
     tok = S.make_prompts(1, lens, shape.vocab).cuda()
     model = P.SwiftKVModel(shape, w, torch.bfloat16, tokens, n_prompts, l, 1)
+    if os.environ.get("SWIFTKV_KERNEL_MASK"):
+        model.set_kernel_mask(int(os.environ["SWIFTKV_KERNEL_MASK"]))
+    if os.environ.get("SWIFTKV_ACT_FORMAT"):
+        model.set_activation_format(int(os.environ["SWIFTKV_ACT_FORMAT"]))
     for _ in range(steps):
         model.prefill_device_tokens(tok, lens, l, 1)
     model.status()
