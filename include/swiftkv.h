@@ -129,12 +129,42 @@ int32_t swiftkv_prefill_device_tokens(swiftkv_model *m, const int32_t *tokens_de
                                       int32_t n_seqs, int32_t swift_layer, int32_t acrosskv_group,
                                       void *cuda_stream);
 
+/*
+ * One sequence's part of a mixed minibatch (Sec. 3.5: "chunks of prefill tokens and decode tokens in each minibatch").
+ */
+typedef struct {
+  int32_t n_new;       /* new tokens of this sequence in this step (>= 1): a prefill chunk, or 1 for a decode token   */
+  int32_t n_past;      /* tokens of this sequence already in the cache (0 for the first chunk of a prompt)            */
+  int32_t cache_row;   /* first row of the sequence's region in every cache plane: token p of the sequence lives in
+                          row cache_row + p.  Regions of different sequences must not overlap and must end inside
+                          max_tokens; the caller keeps a sequence's region fixed for the sequence's lifetime        */
+  int32_t emit;        /* != 0: the last new token continues through layers l+1..L and gets logits (every decode
+                          token; the last chunk of a prompt)                                                         */
+} swiftkv_seq_step;
+
+/*
+ * One forward pass over a mixed minibatch with SwiftKV (Sec. 3.5): layers 1..l run on all new tokens, which attend to
+ * their sequence's cached tokens and, causally, to themselves; right after layer l the SingleInputKV projection
+ * (Eq. 2, with AcrossKV grouping) writes the new tokens' K / V of every later layer into the cache; then only the
+ * emitting tokens run layers l+1..L against those caches and produce logits.  A whole-prompt swiftkv_prefill is the
+ * special case n_past = 0, packed regions, every sequence emitting.
+ *   tokens : HOST int32, the new tokens of all sequences packed in order (sum of n_new)
+ *   seqs   : HOST array of n_seqs entries
+ * swift_layer and acrosskv_group must stay the same for all steps that share cached state.  Sum of n_new and sum of
+ * (n_past + n_new) must not exceed max_tokens.  swiftkv_first_logits afterwards returns one row per emitting
+ * sequence, in order; swiftkv_kv_cache_view returns whole planes (index them with cache_row + position).
+ * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA.
+ */
+int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const swiftkv_seq_step *seqs, int32_t n_seqs,
+                     int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream);
+
 typedef struct {
   const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype, AFTER RoPE            */
   const void *v;            /* device, same shape                                                           */
   int64_t token_stride;     /* elements between consecutive tokens (= n_kv_heads * head_dim)               */
   int64_t head_stride;      /* elements between consecutive KV heads (= head_dim)                          */
-  int32_t n_tokens;         /* packed prompt tokens of the last prefill, prompt-major order                */
+  int32_t n_tokens;         /* rows in use: the packed prompt tokens of the last prefill (prompt-major), or the
+                               highest cache row written so far by swiftkv_step                            */
   int32_t dtype;            /* SWIFTKV_DTYPE_*                                                              */
   int32_t owner_layer;      /* 0-based layer whose projection produced this cache (the AcrossKV group's
                                first layer for layers >= l; the layer itself otherwise)                    */

@@ -18,7 +18,7 @@ KC_NAMES = ("gemm", "attention", "elementwise", "tail", "gemm_swiglu")
 # every symbol include/swiftkv.h declares
 EXPORTS = (
     "swiftkv_version", "swiftkv_last_error", "swiftkv_workspace_bytes", "swiftkv_model_load", "swiftkv_prefill",
-    "swiftkv_prefill_device_tokens", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
+    "swiftkv_prefill_device_tokens", "swiftkv_step", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
     "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc",
@@ -43,6 +43,10 @@ class _LayerWeights(C.Structure):
 class _Weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("final_norm", C.c_void_p), ("lm_head", C.c_void_p),
                 ("layers", C.POINTER(_LayerWeights))]
+
+
+class _SeqStep(C.Structure):
+    _fields_ = [("n_new", C.c_int32), ("n_past", C.c_int32), ("cache_row", C.c_int32), ("emit", C.c_int32)]
 
 
 class _KVView(C.Structure):
@@ -71,6 +75,7 @@ def load_library() -> C.CDLL:
                                        C.c_size_t, C.c_int32, C.c_int32, C.POINTER(C.c_void_p)]
     lib.swiftkv_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_prefill_device_tokens.argtypes = lib.swiftkv_prefill.argtypes
+    lib.swiftkv_step.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_SeqStep), C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_kv_cache_view.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_KVView)]
     lib.swiftkv_first_logits.argtypes = [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)]
     lib.swiftkv_status.argtypes = [C.c_void_p, C.c_void_p]
@@ -173,6 +178,17 @@ class SwiftKVModel:
         with torch.cuda.device(self.device):
             _check(self.lib.swiftkv_prefill_device_tokens(self._h, tokens_dev.data_ptr(), lens, len(seq_lens), swift_layer,
                                                           acrosskv_group, _stream_ptr(stream)))
+
+    def step(self, tokens, seqs: Sequence[Tuple[int, int, int, int]], swift_layer: int, acrosskv_group: int = 1,
+             stream: Optional[torch.cuda.Stream] = None) -> None:
+        """swiftkv_step: one forward pass over a mixed minibatch.  `tokens`: HOST int32, the new tokens of all sequences
+        packed in order; `seqs`: one (n_new, n_past, cache_row, emit) tuple per sequence."""
+        tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous()
+        assert not tokens.is_cuda and tokens.numel() == sum(s[0] for s in seqs)
+        arr = (_SeqStep * len(seqs))(*[_SeqStep(int(a), int(p), int(r), int(e)) for a, p, r, e in seqs])
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_step(self._h, tokens.data_ptr(), arr, len(seqs), swift_layer, acrosskv_group,
+                                         _stream_ptr(stream)))
 
     def kv_cache_view(self, layer: int) -> Tuple[torch.Tensor, torch.Tensor, int]:
         """swiftkv_kv_cache_view -> (K [n_tokens, n_kv, hd], V, owner_layer) as views into the cache tensor."""

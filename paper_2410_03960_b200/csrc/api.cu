@@ -67,6 +67,10 @@ struct Buffers {
   float *tail_scratch;
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
+  int32_t *slot;            // [T] cache row of every new token
+  int32_t *kv_row0, *kv_len;   // [B] first cache row / number of cached + new tokens of every sequence
+  int32_t *kcu;             // [B+1] offsets of the sequences in the gathered half K / V copy (chunked steps)
+  int32_t *emit_row0, *emit_len;   // [B] cache range of the sequences whose last new token continues
   unsigned int *status;
   float *cos_tab, *sin_tab;
 };
@@ -86,7 +90,7 @@ struct swiftkv_model {
   int device;
   // state of the last prefill
   bool ready = false;
-  int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;
+  int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;   // rows in use per cache plane, sequences with logits
   int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
   int kernel_mask = 7;
@@ -145,6 +149,12 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.pos = (int32_t *)cv.take((size_t)T * 4);
   b.last_idx = (int32_t *)cv.take((size_t)B * 4);
   b.last_pos = (int32_t *)cv.take((size_t)B * 4);
+  b.slot = (int32_t *)cv.take((size_t)T * 4);
+  b.kv_row0 = (int32_t *)cv.take((size_t)B * 4);
+  b.kv_len = (int32_t *)cv.take((size_t)B * 4);
+  b.kcu = (int32_t *)cv.take((size_t)(B + 1) * 4);
+  b.emit_row0 = (int32_t *)cv.take((size_t)B * 4);
+  b.emit_len = (int32_t *)cv.take((size_t)B * 4);
   b.status = (unsigned int *)cv.take(256);
   b.cos_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
   b.sin_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
@@ -216,7 +226,10 @@ extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_w
   Carve cv(workspace);
   carve_all(*cfg, max_tokens, max_seqs, m->fold_capacity_elems, cv, m->b);
   if (cudaGetDevice(&m->device) != cudaSuccess) { delete m; return fail(SWIFTKV_ERR_CUDA, "cudaGetDevice failed"); }
-  cudaError_t e = cudaMemsetAsync(m->b.status, 0, 256, 0);
+  // the cache starts as zeros: attention tiles may touch rows past a sequence's end (masked to probability 0), which
+  // must never hold NaN / Inf bit patterns
+  cudaError_t e = cudaMemsetAsync(kv_cache, 0, (size_t)m->slot_capacity * slot_bytes, 0);
+  if (e == cudaSuccess) e = cudaMemsetAsync(m->b.status, 0, 256, 0);
   if (e == cudaSuccess) {
     launch_rope_table(m->b.cos_tab, m->b.sin_tab, max_tokens, cfg->head_dim, (double)cfg->rope_theta, 0);
     e = cudaGetLastError();
@@ -292,8 +305,20 @@ static int32_t gemm_any(swiftkv_model *m, const TA *A, int M, int K, const TW *B
   return SWIFTKV_OK;
 }
 
+// One forward pass over a minibatch (Sec. 3.5).  `plain`: every sequence starts at position 0 and its cache rows are
+// its rows in the packed batch (a whole-prompt prefill); otherwise sequences carry cached prefixes (chunked prefill,
+// decode tokens) and new tokens are scattered to slot[t].
+struct Batch {
+  int T_tok, B, n_emit;
+  int max_new;        // longest run of new tokens
+  int max_kv;         // longest cached + new length
+  int total_kv;       // sum of cached + new lengths
+  bool plain;
+};
+
 template <typename TA, typename T>
-static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int l, int g, cudaStream_t st) {
+static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cudaStream_t st) {
+  const int T_tok = bt.T_tok, B = bt.B, max_len = bt.max_kv;
   const swiftkv_config &c = m->cfg;
   Buffers &b = m->b;
   const int d = c.hidden, dq = c.n_q_heads * c.head_dim, dkv = c.n_kv_heads * c.head_dim, F = c.ffn, L = c.n_layers;
@@ -314,7 +339,9 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
   __half *wg16 = wo16 + (size_t)d * dq, *wu16 = wg16 + (size_t)F * d, *wd16 = wu16 + (size_t)F * d;
   __half *k16 = (__half *)b.kv16, *v16 = k16 + plane;
 
-  { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_positions(b.cu, B, b.pos, b.last_idx, T_tok, st); }
+  const int32_t *slot_map = bt.plain ? nullptr : b.slot;        // cache row of each new token (identity when plain)
+  const int32_t *k_row0 = bt.plain ? nullptr : b.kv_row0;
+  const int32_t *kv_len = bt.plain ? nullptr : b.kv_len;
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_embed<T>((const T *)m->embed, b.tokens, b.x, T_tok, d, c.vocab, b.status, st); }
 
   // one-time model transformation for this (l, g): fold each group leader's input-norm gain into its W_K, W_V
@@ -357,30 +384,44 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
       }
     }
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
-    OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv};
+    OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv, slot_map};
     bool roped = false;
-    const bool want_dup = use_w16 && attn_tc;    // the attention kernel then reads half copies of this layer's K / V
+    // the attention kernel reads half copies of this layer's K / V: written by the QKV epilogue for a plain prefill,
+    // gathered from the cache (cached prefix + new tokens) otherwise
+    const bool want_dup = use_w16 && attn_tc && bt.plain;
     rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st,
                          use_w16 ? wq16 : nullptr, use_w16 ? wk16 : nullptr, use_w16 ? wv16 : nullptr, &rope, &roped,
                          want_dup ? k16 : nullptr, (long long)plane);
     if (rc) return rc;
     if (!roped) {
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
     }
     {
       Scope s(m, st, SWIFTKV_KC_ATTENTION);
       bool done = false;
       if constexpr (sizeof(T) == 2) {
-        // (half activations: only when the QKV epilogue really wrote the half copies of K and V)
-        if (attn_tc && (!act_f16 || (want_dup && roped))) {
-          const void *kk = act_f16 ? (const void *)k16 : (const void *)Kj, *vv = act_f16 ? (const void *)v16 : (const void *)Vj;
-          rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, B, T_tok, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
+        // (half activations: the kernel needs half copies of K and V -- from the QKV epilogue, or gathered here)
+        if (attn_tc && (!act_f16 || (use_w16 && roped))) {
+          const void *kk = Kj, *vv = Vj;
+          const int32_t *kr0 = k_row0;
+          int kv_rows = bt.plain ? T_tok : m->max_tokens;
+          if (act_f16) {
+            kk = k16; vv = v16;
+            if (!bt.plain) {
+              Scope s2(m, st, SWIFTKV_KC_ELEMWISE);
+              launch_gather_kv_half((const bf16 *)Kj, (const bf16 *)Vj, k16, v16, b.kv_row0, b.kv_len, b.kcu, B, bt.max_kv, dkv, st);
+              kr0 = b.kcu;
+              kv_rows = bt.total_kv;
+            }
+          }
+          rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, kr0, kv_len, B, T_tok, kv_rows, bt.max_new, c.n_q_heads,
+                                   c.n_kv_heads, c.head_dim, b.status, st);
           if (rc == SWIFTKV_OK) done = true;
           else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
         }
       }
-      if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, b.pos, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
+      if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, k_row0, kv_len, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
     }
     rc = gemm_any<TA, T>(m, attn, T_tok, dq, (const T *)lw.wo, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
                          use_w16 ? wo16 : nullptr);
@@ -418,18 +459,19 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
   if (l < L) {
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
     T *slot_l = kv + (size_t)l * 2 * plane;
-    OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv};
+    OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv, slot_map};
     bool roped = false;
     rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, no_w, 0, no_w, 0, o, st,
                          use_w16 ? (const __half *)b.wfold : nullptr, nullptr, nullptr, &rope, &roped);
     if (rc) return rc;
     if (use_w16 && !roped) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-folded SingleInputKV weight needs the tensor-core GEMM");
-    if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
   }
 
-  // ---- the last token of each prompt continues through layers l+1..L (footnote of Sec. 3.2)
-  for (int r0 = 0; r0 < B; r0 += MAX_TAIL_ROWS) {
-    const int rows = std::min(MAX_TAIL_ROWS, B - r0);
+  // ---- the tokens that must produce output -- the last token of a prompt (footnote of Sec. 3.2), decode tokens
+  //      (Sec. 3.5) -- continue through layers l+1..L
+  for (int r0 = 0; r0 < bt.n_emit; r0 += MAX_TAIL_ROWS) {
+    const int rows = std::min(MAX_TAIL_ROWS, bt.n_emit - r0);
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
     float *y = b.y + (size_t)r0 * d;
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
@@ -439,8 +481,8 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
       const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.cu + r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.emit_row0 + r0, b.emit_len + r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
@@ -455,22 +497,37 @@ static int32_t run_prefill(swiftkv_model *m, int T_tok, int B, int max_len, int 
   return SWIFTKV_OK;
 }
 
-static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool tokens_on_device, const int32_t *seq_lens,
-                              int32_t n_seqs, int32_t l, int32_t g, void *stream) {
-  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
-  if (!tokens || !seq_lens) return fail(SWIFTKV_ERR_INVALID_ARG, "tokens / seq_lens is null");
+static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool tokens_on_device, const swiftkv_seq_step *seqs,
+                              int32_t n_seqs, bool plain, int32_t l, int32_t g, void *stream) {
   const swiftkv_config &c = m->cfg;
   if (l < 1 || l > c.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c.n_layers);
   if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
   if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
-  long long total = 0;
-  int max_len = 0;
+  Batch bt{};
+  bt.B = n_seqs; bt.plain = plain;
+  long long total = 0, total_kv = 0;
+  int rows_used = 0;
   for (int i = 0; i < n_seqs; ++i) {
-    if (seq_lens[i] < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "seq_lens[%d] = %d < 1", i, seq_lens[i]);
-    total += seq_lens[i];
-    max_len = std::max(max_len, seq_lens[i]);
+    const swiftkv_seq_step &s = seqs[i];
+    if (s.n_new < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: n_new = %d < 1", i, s.n_new);
+    if (s.n_past < 0 || s.cache_row < 0) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: negative n_past / cache_row", i);
+    const long long end = (long long)s.cache_row + s.n_past + s.n_new;
+    if (end > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: cache rows up to %lld exceed max_tokens %d", i, end, m->max_tokens);
+    for (int k = 0; k < i; ++k) {   // regions of different sequences must not overlap
+      const long long a0 = seqs[k].cache_row, a1 = a0 + seqs[k].n_past + seqs[k].n_new;
+      if (s.cache_row < a1 && a0 < end) return fail(SWIFTKV_ERR_INVALID_ARG, "cache rows of sequences %d and %d overlap", k, i);
+    }
+    total += s.n_new;
+    total_kv += s.n_past + s.n_new;
+    bt.max_new = std::max(bt.max_new, s.n_new);
+    bt.max_kv = std::max(bt.max_kv, s.n_past + s.n_new);
+    rows_used = std::max(rows_used, (int)end);
+    if (s.emit) bt.n_emit += 1;
   }
-  if (total > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "%lld tokens > max_tokens %d", total, m->max_tokens);
+  if (total > m->max_tokens || total_kv > m->max_tokens)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "%lld new / %lld cached+new tokens > max_tokens %d", total, total_kv, m->max_tokens);
+  if (bt.n_emit < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "no sequence is marked to emit logits");
+  bt.T_tok = (int)total; bt.total_kv = (int)total_kv;
   if (!tokens_on_device)
     for (long long t = 0; t < total; ++t)
       if (tokens[t] < 0 || tokens[t] >= c.vocab) return fail(SWIFTKV_ERR_INVALID_ARG, "token %lld = %d outside [0, %d)", t, tokens[t], c.vocab);
@@ -487,22 +544,59 @@ static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool toke
   tc_gemm_use_cta_pairs((m->kernel_mask & 4) != 0, (m->kernel_mask & 8) != 0);
   m->ready = false;
   m->launches = 0;
-  m->host_meta.resize(n_seqs + 1);
-  m->host_meta[0] = 0;
-  for (int i = 0; i < n_seqs; ++i) m->host_meta[i + 1] = m->host_meta[i] + seq_lens[i];
-  CUDA_TRY(cudaMemcpyAsync(m->b.cu, m->host_meta.data(), (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice, st));
-  std::vector<int32_t> lp(n_seqs);
-  for (int i = 0; i < n_seqs; ++i) lp[i] = seq_lens[i] - 1;
-  CUDA_TRY(cudaMemcpyAsync(m->b.last_pos, lp.data(), (size_t)n_seqs * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(cudaMemcpyAsync(m->b.tokens, tokens, (size_t)total * 4,
+  // host-side metadata -> one staging vector -> device arrays
+  const int B = n_seqs, T = bt.T_tok;
+  std::vector<int32_t> &hm = m->host_meta;
+  hm.assign((size_t)(B + 1) + 2 * (size_t)T + 2 * B + (B + 1) + 4 * (size_t)B, 0);
+  int32_t *cu = hm.data(), *pos = cu + B + 1, *slot = pos + T, *row0 = slot + T, *klen = row0 + B, *kcu = klen + B;
+  int32_t *last_idx = kcu + B + 1, *last_pos = last_idx + B, *e_row0 = last_pos + B, *e_len = e_row0 + B;
+  int ne = 0;
+  for (int i = 0; i < B; ++i) {
+    const swiftkv_seq_step &s = seqs[i];
+    cu[i + 1] = cu[i] + s.n_new;
+    row0[i] = s.cache_row;
+    klen[i] = s.n_past + s.n_new;
+    kcu[i + 1] = kcu[i] + klen[i];
+    for (int k = 0; k < s.n_new; ++k) { pos[cu[i] + k] = s.n_past + k; slot[cu[i] + k] = s.cache_row + s.n_past + k; }
+    if (s.emit) { last_idx[ne] = cu[i + 1] - 1; last_pos[ne] = klen[i] - 1; e_row0[ne] = s.cache_row; e_len[ne] = klen[i]; ++ne; }
+  }
+  Buffers &b = m->b;
+  CUDA_TRY(cudaMemcpyAsync(b.cu, cu, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.pos, pos, (size_t)T * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.slot, slot, (size_t)T * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.kv_row0, row0, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.kv_len, klen, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.kcu, kcu, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.last_idx, last_idx, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.last_pos, last_pos, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.emit_row0, e_row0, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.emit_len, e_len, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(cudaMemcpyAsync(b.tokens, tokens, (size_t)total * 4,
                            tokens_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
   int32_t rc;
-  if (c.dtype == SWIFTKV_DTYPE_F32) rc = run_prefill<float, float>(m, (int)total, n_seqs, max_len, l, g, st);
-  else if (m->act_format == SWIFTKV_ACT_F16) rc = run_prefill<__half, bf16>(m, (int)total, n_seqs, max_len, l, g, st);
-  else rc = run_prefill<bf16, bf16>(m, (int)total, n_seqs, max_len, l, g, st);
+  if (c.dtype == SWIFTKV_DTYPE_F32) rc = run_prefill<float, float>(m, bt, l, g, st);
+  else if (m->act_format == SWIFTKV_ACT_F16) rc = run_prefill<__half, bf16>(m, bt, l, g, st);
+  else rc = run_prefill<bf16, bf16>(m, bt, l, g, st);
   if (rc) return rc;
-  m->n_tokens = (int)total; m->n_seqs = n_seqs; m->cur_l = l; m->cur_g = g; m->ready = true;
+  m->n_tokens = plain ? T : std::max(rows_used, m->n_tokens);
+  m->n_seqs = ne; m->cur_l = l; m->cur_g = g; m->ready = true;
   return SWIFTKV_OK;
+}
+
+static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool tokens_on_device, const int32_t *seq_lens,
+                              int32_t n_seqs, int32_t l, int32_t g, void *stream) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if (!tokens || !seq_lens) return fail(SWIFTKV_ERR_INVALID_ARG, "tokens / seq_lens is null");
+  if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
+  std::vector<swiftkv_seq_step> seqs(n_seqs);
+  long long row = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (seq_lens[i] < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "seq_lens[%d] = %d < 1", i, seq_lens[i]);
+    if (row + seq_lens[i] > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "more than max_tokens %d tokens", m->max_tokens);
+    seqs[i] = swiftkv_seq_step{seq_lens[i], 0, (int32_t)row, 1};   // whole prompt, packed rows, last token emits
+    row += seq_lens[i];
+  }
+  return forward_common(m, tokens, tokens_on_device, seqs.data(), n_seqs, true, l, g, stream);
 }
 
 extern "C" int32_t swiftkv_prefill(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
@@ -513,6 +607,13 @@ extern "C" int32_t swiftkv_prefill_device_tokens(swiftkv_model *m, const int32_t
                                                  int32_t n_seqs, int32_t swift_layer, int32_t acrosskv_group,
                                                  void *cuda_stream) {
   return prefill_common(m, tokens_dev, true, seq_lens, n_seqs, swift_layer, acrosskv_group, cuda_stream);
+}
+
+extern "C" int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const swiftkv_seq_step *seqs, int32_t n_seqs,
+                                int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if (!tokens || !seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "tokens / seqs is null");
+  return forward_common(m, tokens, false, seqs, n_seqs, false, swift_layer, acrosskv_group, cuda_stream);
 }
 
 extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out) {
@@ -632,20 +733,20 @@ extern "C" int32_t swiftkv_attention_prefill(const void *q, const void *k, const
       return fail(SWIFTKV_ERR_UNSUPPORTED, "tensor-core attention needs q, K, V of one 16-bit type, head_dim 128, an even group size");
     unsigned int *status = op_status_word();
     if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
-    int rc = launch_attention_tc(q, q_dtype == SWIFTKV_DTYPE_F16, k, v, out, cu_seqlens, n_seqs,
-                                 total_tokens, max_seq_len, n_q_heads, n_kv_heads, head_dim, status, st);
+    int rc = launch_attention_tc(q, q_dtype == SWIFTKV_DTYPE_F16, k, v, out, cu_seqlens, nullptr, nullptr, n_seqs,
+                                 total_tokens, total_tokens, max_seq_len, n_q_heads, n_kv_heads, head_dim, status, st);
     if (rc) return fail(rc, "attention launch failed");
     return SWIFTKV_OK;
   }
   if (q_dtype == SWIFTKV_DTYPE_BF16 && kv_dtype == SWIFTKV_DTYPE_BF16)
-    launch_attention_simple<bf16, bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr,
+    launch_attention_simple<bf16, bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr, nullptr,
                                         total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else if (q_dtype == SWIFTKV_DTYPE_F16 && kv_dtype == SWIFTKV_DTYPE_BF16)
     launch_attention_simple<__half, bf16>((const __half *)q, (const bf16 *)k, (const bf16 *)v, (__half *)out, cu_seqlens, n_seqs,
-                                          nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+                                          nullptr, nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else if (q_dtype == SWIFTKV_DTYPE_F32 && kv_dtype == SWIFTKV_DTYPE_F32)
     launch_attention_simple<float, float>((const float *)q, (const float *)k, (const float *)v, (float *)out, cu_seqlens, n_seqs,
-                                          nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+                                          nullptr, nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else
     return fail(SWIFTKV_ERR_INVALID_ARG, "unsupported dtype combination");
   cudaError_t e = cudaGetLastError();
@@ -672,10 +773,10 @@ extern "C" int32_t swiftkv_tail_attention(const float *q, const void *k_cache, c
                 tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (dtype == SWIFTKV_DTYPE_BF16)
-    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, n_seqs, max_seq_len, n_q_heads,
+    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, nullptr, n_seqs, max_seq_len, n_q_heads,
                                 n_kv_heads, head_dim, (float *)scratch, st);
   else if (dtype == SWIFTKV_DTYPE_F32)
-    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, n_seqs, max_seq_len,
+    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, nullptr, n_seqs, max_seq_len,
                                  n_q_heads, n_kv_heads, head_dim, (float *)scratch, st);
   else
     return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");

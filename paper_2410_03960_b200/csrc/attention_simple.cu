@@ -12,7 +12,8 @@ template <typename TQ, typename T, int MAX_E>   // MAX_E = ceil(hd / 32) output 
 __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restrict__ q, const T *__restrict__ k,
                                                                const T *__restrict__ v, TQ *__restrict__ out,
                                                                const int32_t *__restrict__ cu, int n_seqs,
-                                                               const int32_t *__restrict__ positions, int n_tokens,
+                                                               const int32_t *__restrict__ k_row0,
+                                                               const int32_t *__restrict__ kv_len, int n_tokens,
                                                                int n_q, int n_kv, int hd, float scale) {
   extern __shared__ float q_sm[];   // [4 warps][hd]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -20,18 +21,15 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
   if (item >= (long long)n_tokens * n_q) return;
   const int t = (int)(item / n_q), h = (int)(item % n_q);
   const int kvh = h / (n_q / n_kv);
-  int p;
-  if (positions) {
-    p = positions[t];
-  } else {   // position inside its prompt from the prompt offsets
-    int lo = 0, hi = n_seqs;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (cu[mid] <= t) lo = mid; else hi = mid;
-    }
-    p = t - cu[lo];
+  int lo = 0, hi = n_seqs;   // the sequence of query t from the offsets of the new tokens
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
   }
-  const int first = t - p;   // packed index of this prompt's first token
+  const int n_new = cu[lo + 1] - cu[lo];
+  const int past = kv_len ? kv_len[lo] - n_new : 0;
+  const int p = past + (t - cu[lo]);                    // position of this query: it sees keys 0..p
+  const int first = k_row0 ? k_row0[lo] : cu[lo];       // K / V row of the sequence's first token
   float *qs = q_sm + warp * hd;
   const TQ *qr = q + ((size_t)t * n_q + h) * hd;
   for (int i = lane; i < hd; i += 32) qs[i] = to_f(qr[i]) * scale;
@@ -80,22 +78,23 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
 
 template <typename TQ, typename T>
 void launch_attention_simple(const TQ *q, const T *k, const T *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
-                             const int32_t *positions, int n_tokens, int n_q, int n_kv, int hd, cudaStream_t st) {
+                             const int32_t *k_row0, const int32_t *kv_len, int n_tokens, int n_q, int n_kv, int hd,
+                             cudaStream_t st) {
   if (n_tokens <= 0) return;
   const long long items = (long long)n_tokens * n_q;
   const unsigned blocks = (unsigned)((items + 3) / 4);
   const float scale = 1.0f / sqrtf((float)hd);
   const size_t smem = 4 * hd * sizeof(float);
-  if (hd <= 32) attention_simple_kernel<TQ, T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 64) attention_simple_kernel<TQ, T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 128) attention_simple_kernel<TQ, T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
-  else attention_simple_kernel<TQ, T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, positions, n_tokens, n_q, n_kv, hd, scale);
+  if (hd <= 32) attention_simple_kernel<TQ, T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 64) attention_simple_kernel<TQ, T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 128) attention_simple_kernel<TQ, T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
+  else attention_simple_kernel<TQ, T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
 }
 template void launch_attention_simple<float, float>(const float *, const float *, const float *, float *, const int32_t *, int,
-                                                    const int32_t *, int, int, int, int, cudaStream_t);
+                                                    const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
 template void launch_attention_simple<bf16, bf16>(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int,
-                                                  const int32_t *, int, int, int, int, cudaStream_t);
+                                                  const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
 template void launch_attention_simple<__half, bf16>(const __half *, const bf16 *, const bf16 *, __half *, const int32_t *, int,
-                                                    const int32_t *, int, int, int, int, cudaStream_t);
+                                                    const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
 
 }  // namespace skv

@@ -31,7 +31,9 @@ constexpr int ATT_SMEM = SM_BAR + 256 + 1024;
 constexpr float RESCALE_THRESHOLD = 8.0f;          // in log2 units
 
 struct AttnParams {
-  const int32_t *cu;
+  const int32_t *cu;        // [n_seqs+1] offsets of each sequence's NEW tokens (the queries) in q / out
+  const int32_t *k_row0;    // [n_seqs] first K / V row of each sequence (null: same as cu, i.e. a plain prefill)
+  const int32_t *kv_len;    // [n_seqs] keys of each sequence = tokens already cached + new tokens (null: new tokens only)
   bf16 *out;
   int n_seqs, n_q, n_kv, max_tiles;
   float scale_log2;     // softmax scale * log2(e)
@@ -71,9 +73,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const int b = rem / n_pairs, pair = rem % n_pairs;
   const int tok0 = p.cu[b], n = p.cu[b + 1] - tok0;
   if (qt * BQ >= n) return;
+  const int k0 = p.k_row0 ? p.k_row0[b] : tok0;
+  const int past = p.kv_len ? p.kv_len[b] - n : 0;       // query i of this sequence sits at position past + i
   const int h0 = pair * 2;
   const int kvh = h0 / (p.n_q / p.n_kv);
-  const int n_kv_tiles = qt + 1;
+  const int n_kv_tiles = (past + min(n, (qt + 1) * BQ) - 1) / BKV + 1;   // keys 0 .. position of the tile's last query
   const int q_row0 = tok0 + qt * BQ;
 
   extern __shared__ uint8_t smem_raw[];
@@ -132,12 +136,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t kb = tc::smem_u32(&k_full[s]);
         tc::mbar_expect_tx(kb, TILE_BYTES);
         for (int c = 0; c < 2; ++c)
-          tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, tok0 + j * BKV);
+          tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, k0 + j * BKV);
         if (!wait_or_abort(tc::smem_u32(&v_empty[s]), ph ^ 1, abort_flag, p.status)) break;
         const uint32_t vb = tc::smem_u32(&v_full[s]);
         tc::mbar_expect_tx(vb, TILE_BYTES);
         for (int c = 0; c < 2; ++c)
-          tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, tok0 + j * BKV);
+          tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, k0 + j * BKV);
       }
     }
   } else if (warp == 1) {
@@ -226,7 +230,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int j = 0; j < n_kv_tiles; ++j) {
       if (!wait_or_abort(tc::smem_u32(&s_full[w]), j & 1, abort_flag, p.status)) { ok = false; break; }
       tc::tc_fence_after_sync();
-      const bool diag = (j == qt);
+      // causal mask: key column i of this tile is visible to query row r iff i <= r + shift; only the tiles that
+      // straddle the diagonal (at most two when the cached prefix is not a multiple of the tile) need it
+      const int shift = past + qt * BQ - j * BKV;
+      const bool diag = shift < BKV - 1;
+      const int lim = row + shift;
       // the whole score row (128 fp32) in registers: one pass over tensor memory, the second half of the loads in
       // flight while the first half is reduced
       uint32_t s[128];
@@ -235,10 +243,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc::tmem_ld_wait();
       tc::tmem_ld_32x32b_x32p(t_s + 64, s + 64);
       tc::tmem_ld_32x32b_x32p(t_s + 96, s + 96);
-      if (diag) {   // causal mask, only on the diagonal tile: key index > query index
+      if (diag) {
 #pragma unroll
         for (int i = 0; i < 64; ++i)
-          if (i > row) s[i] = 0xff800000u;   // -inf
+          if (i > lim) s[i] = 0xff800000u;   // -inf
       }
       float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
@@ -252,7 +260,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (diag) {
 #pragma unroll
         for (int i = 64; i < 128; ++i)
-          if (i > row) s[i] = 0xff800000u;
+          if (i > lim) s[i] = 0xff800000u;
       }
 #pragma unroll
       for (int i = 64; i < 128; i += 8) {
@@ -345,15 +353,15 @@ bool tc_attention_supported(int n_q, int n_kv, int hd) {
 }
 
 int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
-                        int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
-                        cudaStream_t st) {
+                        const int32_t *k_row0, const int32_t *kv_len, int n_seqs, int n_tokens, int kv_rows,
+                        int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st) {
   if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
-  if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1) return SWIFTKV_ERR_INVALID_ARG;
+  if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1 || kv_rows < 1) return SWIFTKV_ERR_INVALID_ARG;
   CUtensorMap tq, tk, tv;
-  // row extent = the tokens of this call: rows past it read as zero (never stale cache contents)
+  // row extents = the rows that hold data of this call: rows past them read as zero (never stale memory)
   if (get_tmap(&tq, q, n_tokens, (uint64_t)n_q * hd, (uint64_t)n_q * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
-  if (get_tmap(&tk, k, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
-  if (get_tmap(&tv, v, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tk, k, kv_rows, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tv, v, kv_rows, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attention_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
@@ -364,7 +372,7 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
     attr_set = true;
   }
   AttnParams p{};
-  p.cu = cu_seqlens; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
+  p.cu = cu_seqlens; p.k_row0 = k_row0; p.kv_len = kv_len; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
   p.max_tiles = (max_seq_len + BQ - 1) / BQ;
   p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
   p.status = status;

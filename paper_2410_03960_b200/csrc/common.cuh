@@ -52,8 +52,9 @@ struct OutDesc {
   void *seg_base;
   long long seg_stride;   // elements
   int seg_w;
+  const int32_t *slot_map;   // optional: GEMM row r lands in row slot_map[r] of a segment (cache row of token r)
 };
-inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDesc{mode, p, ld, n, nullptr, 0, 1}; }
+inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDesc{mode, p, ld, n, nullptr, 0, 1, nullptr}; }
 
 #ifdef __CUDACC__
 // write one fp32 accumulator where the descriptor says (device side)
@@ -70,7 +71,8 @@ __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, fl
   } else {
     const int c = col - o.n0;
     const int seg = c / o.seg_w, within = c % o.seg_w;
-    reinterpret_cast<TS *>(o.seg_base)[(size_t)seg * o.seg_stride + (size_t)row * o.seg_w + within] = from_f<TS>(acc);
+    const size_t srow = o.slot_map ? (size_t)o.slot_map[row] : (size_t)row;
+    reinterpret_cast<TS *>(o.seg_base)[(size_t)seg * o.seg_stride + srow * o.seg_w + within] = from_f<TS>(acc);
   }
 }
 #endif
@@ -88,10 +90,15 @@ void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions,
 // y = x * rsqrt(mean(x^2)+eps) * gamma (gamma may be null: unit-rms only).  x fp32 [rows, d] -> out TO [rows, d]
 template <typename TG, typename TO>
 void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st);
-// in-place rotary embedding on `n_batches` tensors [rows, n_heads, hd] spaced batch_stride elements apart
+// in-place rotary embedding on `n_batches` tensors [*, n_heads, hd] spaced batch_stride elements apart; logical row r
+// (position positions[r]) lives in tensor row slot_map[r] (null: row r)
 template <typename T>
-void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const float *cos_tab,
-                 const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st);
+void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const int32_t *slot_map,
+                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st);
+// packs each sequence's cache rows [row0[b], row0[b] + len[b]) of one layer's K and V planes (bf16) into contiguous half
+// copies starting at row kcu[b]: the tensor-core attention kernel's operands in a chunked step with half activations
+void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
+                           const int32_t *kcu, int n_seqs, int max_len, int dkv, cudaStream_t st);
 template <typename T>
 void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
@@ -132,15 +139,19 @@ int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg,
 bool tc_swiglu_supported(int M, int F, int K);
 
 // attention.cu
+// k_row0 / kv_len as for launch_attention_tc
 template <typename TQ, typename TKV>
 void launch_attention_simple(const TQ *q, const TKV *k, const TKV *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
-                             const int32_t *positions /* may be null */, int n_tokens, int n_q, int n_kv, int hd,
+                             const int32_t *k_row0, const int32_t *kv_len, int n_tokens, int n_q, int n_kv, int hd,
                              cudaStream_t st);
 bool tc_attention_supported(int n_q, int n_kv, int hd);
-// f16: q, k, v and out all hold IEEE halves (else all bfloat16)
+// f16: q, k, v and out all hold IEEE halves (else all bfloat16).  cu_seqlens: offsets of each sequence's new tokens
+// (queries) in q / out; k_row0 / kv_len (both nullable): first K / V row and number of keys (cached + new) of each
+// sequence -- null means a plain prefill whose K / V rows are packed like q; kv_rows: rows of k / v that hold data;
+// max_seq_len bounds the new tokens of one sequence
 int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
-                        int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv, int hd,
-                        unsigned int *status, cudaStream_t st);
+                        const int32_t *k_row0, const int32_t *kv_len, int n_seqs, int n_tokens, int kv_rows,
+                        int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st);
 
 // tail.cu : the last-token path (at most MAX_TAIL_ROWS activation rows per launch, fp32 activations)
 constexpr int MAX_TAIL_ROWS = 8;
@@ -151,10 +162,11 @@ void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, i
 template <typename T>
 void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
                         int mode, cudaStream_t st);
-// one query token per prompt against that prompt's cache rows [cu[b], cu[b+1]); scratch holds split partials
+// one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
+// row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
 template <typename T>
-void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
+void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *row0, const int32_t *len,
+                           int n_seqs, int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
 
 }  // namespace skv

@@ -125,8 +125,8 @@ template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *
 // ---------------------------------------------------------------------------------------------------------
 template <typename T>
 __global__ void rope_kernel(T *__restrict__ x, long long batch_stride, const int32_t *__restrict__ positions,
-                            const float *__restrict__ cos_tab, const float *__restrict__ sin_tab, int rows,
-                            int n_heads, int hd) {
+                            const int32_t *__restrict__ slot_map, const float *__restrict__ cos_tab,
+                            const float *__restrict__ sin_tab, int rows, int n_heads, int hd) {
   const int half = hd >> 1;
   const long long per_row = (long long)n_heads * half;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -136,22 +136,23 @@ __global__ void rope_kernel(T *__restrict__ x, long long batch_stride, const int
   const int h = rem / half, i = rem % half;
   const int p = positions[row];
   const float c = cos_tab[(size_t)p * half + i], s = sin_tab[(size_t)p * half + i];
-  T *base = x + (size_t)blockIdx.y * batch_stride + ((size_t)row * n_heads + h) * hd;
+  const size_t trow = slot_map ? (size_t)slot_map[row] : (size_t)row;
+  T *base = x + (size_t)blockIdx.y * batch_stride + (trow * n_heads + h) * hd;
   const float a = to_f(base[i]), b = to_f(base[i + half]);
   base[i] = from_f<T>(a * c - b * s);
   base[i + half] = from_f<T>(b * c + a * s);
 }
 template <typename T>
-void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const float *cos_tab,
-                 const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st) {
+void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const int32_t *slot_map,
+                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st) {
   const long long n = (long long)rows * n_heads * (hd / 2);
   if (n <= 0 || n_batches <= 0) return;
   dim3 grid((unsigned)((n + 255) / 256), (unsigned)n_batches);
-  rope_kernel<T><<<grid, 256, 0, st>>>(x, batch_stride, positions, cos_tab, sin_tab, rows, n_heads, hd);
+  rope_kernel<T><<<grid, 256, 0, st>>>(x, batch_stride, positions, slot_map, cos_tab, sin_tab, rows, n_heads, hd);
 }
-template void launch_rope<float>(float *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
-template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
-template void launch_rope<__half>(__half *, long long, int, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<float>(float *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<__half>(__half *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
 
 // cos/sin of p * theta^(-2i/hd), evaluated in double precision and rounded once to fp32.
 __global__ void rope_table_kernel(float *cos_tab, float *sin_tab, int max_pos, int half, double log_theta, int hd) {
@@ -238,6 +239,29 @@ void launch_fold(const T *w, const T *gamma, TO *dst, int rows, int cols, cudaSt
 template void launch_fold<float, float>(const float *, const float *, float *, int, int, cudaStream_t);
 template void launch_fold<bf16, bf16>(const bf16 *, const bf16 *, bf16 *, int, int, cudaStream_t);
 template void launch_fold<bf16, __half>(const bf16 *, const bf16 *, __half *, int, int, cudaStream_t);
+
+__global__ void gather_kv_half_kernel(const bf16 *__restrict__ k, const bf16 *__restrict__ v, __half *__restrict__ k16,
+                                      __half *__restrict__ v16, const int32_t *__restrict__ row0,
+                                      const int32_t *__restrict__ len, const int32_t *__restrict__ kcu, int dkv) {
+  const int b = blockIdx.y, r = blockIdx.x;
+  if (r >= len[b]) return;
+  const size_t src = ((size_t)row0[b] + r) * dkv, dst = ((size_t)kcu[b] + r) * dkv;
+  for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
+    const uint4 kr = *reinterpret_cast<const uint4 *>(k + src + i), vr = *reinterpret_cast<const uint4 *>(v + src + i);
+    const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr), *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vr);
+    uint4 ko, vo;
+    __half2 *ko2 = reinterpret_cast<__half2 *>(&ko), *vo2 = reinterpret_cast<__half2 *>(&vo);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { ko2[q] = __float22half2_rn(__bfloat1622float2(k2[q])); vo2[q] = __float22half2_rn(__bfloat1622float2(v2[q])); }
+    *reinterpret_cast<uint4 *>(k16 + dst + i) = ko;
+    *reinterpret_cast<uint4 *>(v16 + dst + i) = vo;
+  }
+}
+void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
+                           const int32_t *kcu, int n_seqs, int max_len, int dkv, cudaStream_t st) {
+  if (n_seqs <= 0 || max_len <= 0) return;
+  gather_kv_half_kernel<<<dim3(max_len, n_seqs), 128, 0, st>>>(k, v, k16, v16, row0, len, kcu, dkv);
+}
 
 // bfloat16 -> IEEE half copy of a weight matrix (exact for |w| >= 2^-17, absolute error <= 2^-25 below), 128-bit accesses
 __global__ void bf16_to_f16_kernel(const bf16 *__restrict__ src, __half *__restrict__ dst, long long n) {

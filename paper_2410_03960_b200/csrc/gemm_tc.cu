@@ -211,7 +211,8 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
       } else {
         const int cc = col_h - p.out.n0;
         const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
-        dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + (size_t)row * p.out.seg_w + within;
+        const size_t srow = (p.out.slot_map && row < p.M) ? (size_t)p.out.slot_map[row] : (size_t)row;
+        dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + srow * p.out.seg_w + within;
         if (p.dup_base) dupp = p.dup_base + (size_t)seg * p.dup_stride + (size_t)row * p.out.seg_w + within;
         rope = (seg & 1) == 0;      // segments alternate K (rotated) and V (not)
       }
@@ -292,7 +293,8 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
           } else {
             const int cc = col - p.out.n0;
             const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
-            dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + (size_t)row * p.out.seg_w + within;
+            const size_t srow = p.out.slot_map ? (size_t)p.out.slot_map[row] : (size_t)row;
+            dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + srow * p.out.seg_w + within;
           }
           uint4 *dst = reinterpret_cast<uint4 *>(dstp);
 #pragma unroll

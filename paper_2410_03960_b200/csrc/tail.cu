@@ -274,14 +274,14 @@ constexpr int TA_WARPS = 4;
 template <typename T, int REP, int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    int n_q, int n_kv, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
+    const int32_t *__restrict__ len, int n_q, int n_kv, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
   __shared__ float qs[REP][HD];
   __shared__ float w_m[TA_WARPS][REP], w_l[TA_WARPS][REP];
   __shared__ float w_acc[TA_WARPS][REP][HD];
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int first = cu[b], n = cu[b + 1] - cu[b];
+  const int first = cu[b], n = len ? len[b] : cu[b + 1] - cu[b];
   const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
   for (int i = threadIdx.x; i < REP * HD; i += blockDim.x)
     qs[i / HD][i % HD] = q[((size_t)b * n_q + kvh * REP + i / HD) * HD + i % HD] * scale;
@@ -374,12 +374,13 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
 template <typename T, int MAX_E>
 __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    int n_q, int n_kv, int hd, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
+    const int32_t *__restrict__ len, int n_q, int n_kv, int hd, int chunk, int n_splits, float scale,
+    float *__restrict__ scratch) {
   extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rep = n_q / n_kv;
-  const int first = cu[b], n = cu[b + 1] - cu[b];
+  const int first = cu[b], n = len ? len[b] : cu[b + 1] - cu[b];
   const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
   for (int hw = warp; hw < rep; hw += (blockDim.x >> 5)) {   // (more heads per group than warps: loop)
     const int h = kvh * rep + hw;
@@ -452,8 +453,9 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 }
 
 template <typename T>
-void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st) {
+void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens,
+                           const int32_t *len, int n_seqs, int max_seq_len, int n_q, int n_kv, int hd, float *scratch,
+                           cudaStream_t st) {
   if (n_seqs <= 0) return;
   const int chunk = tail_chunk(max_seq_len);
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
@@ -461,25 +463,25 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out,
   const int rep = n_q / n_kv;
   if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
     dim3 grid(n_splits, n_kv, n_seqs);
-    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, chunk, n_splits, scale, scratch);
+    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
     tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
     return;
   }
   const int threads = 32 * (rep < 8 ? rep : 8);
   const size_t smem = (size_t)rep * hd * sizeof(float);
   dim3 grid(n_splits, n_kv, n_seqs);
-  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
-template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *, int,
-                                           int, int, int, int, float *, cudaStream_t);
-template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, float *, const int32_t *, int, int,
-                                          int, int, int, float *, cudaStream_t);
+template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *,
+                                           const int32_t *, int, int, int, int, int, float *, cudaStream_t);
+template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, float *, const int32_t *,
+                                          const int32_t *, int, int, int, int, int, float *, cudaStream_t);
 
 }  // namespace skv

@@ -1,0 +1,124 @@
+"""Chunked prefill and decode steps (the paper's Sec. 3.5 deployment: minibatches that mix chunks of prefill tokens and
+decode tokens; after layer l the later layers' caches are filled and only the tokens that must produce output go
+on).  Feeding a sequence in chunks, or one token at a time, is an exact reformulation: the caches and logits must
+equal the oracle's one-shot SwiftKV prefill of the same token sequence."""
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as S
+from oracle import swiftkv_oracle as O
+from helpers import oracle_config, oracle_weights, rel_l2, to_np
+
+pytestmark = pytest.mark.gpu
+
+MID = S.ModelShape(1024, 512, 4, 8, 2, 128, 1024, 500000.0, 1e-5, "mid")
+
+
+def _check_seq(model, shape, ref, row0, n, kv_bar):
+    for j in range(shape.n_layers):
+        K, V, _ = model.kv_cache_view(j)
+        assert rel_l2(to_np(K[row0:row0 + n]), ref["K"][j][:n]) <= kv_bar, j
+        assert rel_l2(to_np(V[row0:row0 + n]), ref["V"][j][:n]) <= kv_bar, j
+
+
+@pytest.mark.parametrize("shape,dtype,act,kv_bar,lg_bar", [
+    (S.TINY, torch.float32, None, 1e-4, 1e-3),
+    (S.TINY, torch.bfloat16, 1, 2e-2, 0.1),
+    (MID, torch.bfloat16, 1, 2e-2, 0.1),        # tensor-core kernels, half activations (gathered half K / V copies)
+    (MID, torch.bfloat16, 0, 2e-2, 0.1),        # tensor-core kernels reading the bf16 cache in place
+])
+@pytest.mark.parametrize("l,g", [(2, 1), (1, 2), (4, 1)])
+def test_chunked_prefill_then_decode(shape, dtype, act, kv_bar, lg_bar, l, g):
+    import paper_2410_03960_b200 as P
+    seed = 11
+    lens = [300, 77, 129]                      # prompt lengths
+    n_decode = 3
+    cap = 512                                  # cache rows reserved per sequence
+    w = S.make_weights(shape, seed, dtype, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    toks = [S.token_ids(seed, b, n + n_decode, shape.vocab) for b, n in enumerate(lens)]   # prompt + "generated" tokens
+    model = P.SwiftKVModel(shape, w, dtype, cap * len(lens), len(lens), min(l, 1), 1)
+    if act is not None:
+        model.set_activation_format(act)
+
+    # ---- chunked prefill: 100-token chunks, all sequences that still have prompt left share a minibatch
+    chunk = 100
+    done = [0] * len(lens)
+    last_logits = {}
+    while any(d < n for d, n in zip(done, lens)):
+        seqs, packed, emitting = [], [], []
+        for b, n in enumerate(lens):
+            if done[b] >= n:
+                continue
+            k = min(chunk, n - done[b])
+            emit = int(done[b] + k == n)
+            seqs.append((k, done[b], b * cap, emit))
+            packed.append(toks[b][done[b]:done[b] + k])
+            if emit:
+                emitting.append(b)
+            done[b] += k
+        if not emitting:                       # the library wants at least one emitting sequence per step
+            seqs[0] = (seqs[0][0], seqs[0][1], seqs[0][2], 1)
+            emitting = [-1]
+        model.step(torch.cat(packed), seqs, l, g)
+        model.status()
+        lg = model.first_logits().clone()
+        for i, b in enumerate(emitting):
+            if b >= 0:
+                last_logits[b] = lg[i]
+    for b, n in enumerate(lens):
+        ref = O.swiftkv(cfg, ow, toks[b][:n].numpy(), [n], l, g)
+        _check_seq(model, shape, ref, b * cap, n, kv_bar)
+        assert np.max(np.abs(to_np(last_logits[b]) - ref["logits"][0])) <= lg_bar, b
+
+    # ---- decode: every sequence appends one token per step (a minibatch of decode tokens)
+    for t in range(n_decode):
+        seqs = [(1, n + t, b * cap, 1) for b, n in enumerate(lens)]
+        model.step(torch.stack([toks[b][n + t] for b, n in enumerate(lens)]), seqs, l, g)
+        model.status()
+        lg = to_np(model.first_logits())
+        for b, n in enumerate(lens):
+            ref = O.swiftkv(cfg, ow, toks[b][:n + t + 1].numpy(), [n + t + 1], l, g)
+            assert np.max(np.abs(lg[b] - ref["logits"][0])) <= lg_bar, (t, b)
+            if t == n_decode - 1:
+                _check_seq(model, shape, ref, b * cap, n + t + 1, kv_bar)
+
+
+def test_mixed_minibatch_of_prefill_chunk_and_decode_token():
+    """One step carries a decode token of sequence 0 and a prefill chunk of sequence 1; only sequence 0 emits."""
+    import paper_2410_03960_b200 as P
+    shape, dtype, l, g, cap = MID, torch.bfloat16, 2, 1, 512
+    w = S.make_weights(shape, 5, dtype, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    t0, t1 = S.token_ids(5, 0, 141, shape.vocab), S.token_ids(5, 1, 260, shape.vocab)
+    model = P.SwiftKVModel(shape, w, dtype, 2 * cap, 2, l, g)
+    model.step(t0[:140], [(140, 0, 0, 1)], l, g)                                     # prompt of sequence 0
+    model.step(torch.cat([t0[140:141], t1[:130]]), [(1, 140, 0, 1), (130, 0, cap, 0)], l, g)   # decode + first chunk
+    model.status()
+    lg = to_np(model.first_logits())
+    assert lg.shape[0] == 1
+    ref0 = O.swiftkv(cfg, ow, t0.numpy(), [141], l, g)
+    assert np.max(np.abs(lg[0] - ref0["logits"][0])) <= 0.1
+    model.step(t1[130:], [(130, 130, cap, 1)], l, g)                                 # second chunk of sequence 1
+    model.status()
+    ref1 = O.swiftkv(cfg, ow, t1.numpy(), [260], l, g)
+    assert np.max(np.abs(to_np(model.first_logits())[0] - ref1["logits"][0])) <= 0.1
+    _check_seq(model, shape, ref0, 0, 141, 2e-2)
+    _check_seq(model, shape, ref1, cap, 260, 2e-2)
+
+
+def test_step_argument_checks():
+    import paper_2410_03960_b200 as P
+    shape = S.TINY
+    w = S.make_weights(shape, 0, torch.float32, "cuda")
+    model = P.SwiftKVModel(shape, w, torch.float32, 256, 2, 2, 1)
+    tok = S.token_ids(0, 0, 40, shape.vocab)
+    for bad in ([(40, 0, 250, 1)],                      # runs past max_tokens
+                [(20, 0, 0, 1), (20, 0, 10, 1)],        # overlapping regions
+                [(40, 0, 0, 0)],                        # nobody emits
+                [(0, 0, 0, 1)]):                        # empty chunk
+        n = sum(s[0] for s in bad)
+        with pytest.raises(P.SwiftKVError) as e:
+            model.step(tok[:max(n, 1)] if n else tok[:0], bad, 2, 1)
+        assert e.value.code == -1
