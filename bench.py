@@ -303,8 +303,10 @@ def run_ours(args, rank, world, local_rank):
         line = {
             "metric": "prefill_tokens_per_s", "value": tokens_all / t_swift, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "tokens_per_step_per_gpu": T, "seq_lens_rank0": lens,
+                       "arithmetic": "bf16 weights and KV cache; tensor-core operands are IEEE-half copies (same tensor rate as "
+                                     "bf16, 8x finer rounding), fp32 accumulation, fp32 residual stream",
                        "l2": "inputs larger than L2 (16 GB of weights, > 3 GB of activations per step)",
                        "multi_gpu": "replicas only: independent batch per rank, no collective"},
             "tflops_per_gpu": {"actual": actual_tflops, "normalized_to_full_depth": norm_tflops,
