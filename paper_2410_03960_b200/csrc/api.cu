@@ -101,6 +101,9 @@ struct swiftkv_model {
   struct Rec { cudaEvent_t a, b; int cls; };
   std::vector<Rec> recs;
   std::vector<int32_t> host_meta;
+  // side stream on which the next layer's weights are copied to half while the current layer computes
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
 };
 
 static size_t dsize(int dtype) { return dtype == SWIFTKV_DTYPE_BF16 ? 2 : 4; }
@@ -134,7 +137,7 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.wfold = cv.take(fold_elems * E);
   const size_t dkv_ = (size_t)c.n_kv_heads * c.head_dim;
   const bool bf = c.dtype == SWIFTKV_DTYPE_BF16;
-  b.w16 = cv.take(bf ? (2 * d * dq + 2 * d * dkv_ + 3 * d * F) * 2 : 0);
+  b.w16 = cv.take(bf ? 2 * (2 * d * dq + 2 * d * dkv_ + 3 * d * F) * 2 : 0);   // two layers: double buffer
   b.kv16 = cv.take(bf ? (size_t)2 * T * dkv_ * 2 : 0);
   b.y = (float *)cv.take((size_t)B * d * 4);
   const size_t R = std::min<size_t>(B, MAX_TAIL_ROWS);
@@ -183,6 +186,8 @@ extern "C" int32_t swiftkv_workspace_bytes(const swiftkv_config *cfg, int32_t ma
   *kv_cache_bytes = (size_t)slots * slot_elems(*cfg, max_tokens) * dsize(cfg->dtype);
   return SWIFTKV_OK;
 }
+
+extern "C" void swiftkv_model_free(swiftkv_model *m);
 
 extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_weights *w, void *workspace,
                                       size_t workspace_bytes, void *kv_cache, size_t kv_cache_bytes,
@@ -235,7 +240,13 @@ extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_w
     e = cudaGetLastError();
   }
   if (e == cudaSuccess) e = cudaStreamSynchronize(0);
-  if (e != cudaSuccess) { delete m; return fail(SWIFTKV_ERR_CUDA, "model_load: %s", cudaGetErrorString(e)); }
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_start, cudaEventDisableTiming);
+  for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+    e = cudaEventCreateWithFlags(&m->ev_ready[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->ev_free[i], cudaEventDisableTiming);
+  }
+  if (e != cudaSuccess) { swiftkv_model_free(m); return fail(SWIFTKV_ERR_CUDA, "model_load: %s", cudaGetErrorString(e)); }
   *out = m;
   return SWIFTKV_OK;
 }
@@ -244,6 +255,12 @@ extern "C" void swiftkv_model_free(swiftkv_model *m) {
   if (!m) return;
   for (cudaEvent_t ev : m->pool) cudaEventDestroy(ev);
   for (auto &r : m->recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  if (m->side) { cudaStreamSynchronize(m->side); cudaStreamDestroy(m->side); }
+  if (m->ev_start) cudaEventDestroy(m->ev_start);
+  for (int i = 0; i < 2; ++i) {
+    if (m->ev_ready[i]) cudaEventDestroy(m->ev_ready[i]);
+    if (m->ev_free[i]) cudaEventDestroy(m->ev_free[i]);
+  }
   delete m;
 }
 
@@ -256,12 +273,16 @@ struct Scope {
     if (!m->pool.empty()) { cudaEvent_t e = m->pool.back(); m->pool.pop_back(); return e; }
     cudaEvent_t e; cudaEventCreate(&e); return e;
   }
-  Scope(swiftkv_model *m_, cudaStream_t s, int c, int n_launches = 1) : m(m_), st(s), cls(c) {
+  bool timed;
+  // timed = false: count the launches only (work on the side stream overlaps the main stream's kernels, so its
+  // wall time is not part of any class)
+  Scope(swiftkv_model *m_, cudaStream_t s, int c, int n_launches = 1, bool timed_ = true) : m(m_), st(s), cls(c) {
     m->launches += n_launches;
-    if (m->profiling) { a = get(m); b = get(m); cudaEventRecord(a, st); }
+    timed = timed_ && m->profiling;
+    if (timed) { a = get(m); b = get(m); cudaEventRecord(a, st); }
   }
   ~Scope() {
-    if (m->profiling) { cudaEventRecord(b, st); m->recs.push_back({a, b, cls}); }
+    if (timed) { cudaEventRecord(b, st); m->recs.push_back({a, b, cls}); }
   }
 };
 
@@ -335,8 +356,37 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const bool use_w16 = act_f16 && (m->kernel_mask & 1) && tc_gemm_supported(T_tok, dq, d) && tc_gemm_supported(T_tok, d, dq) &&
                        tc_gemm_supported(T_tok, d, F) && (dkv % 256 == 0) && (dq % 256 == 0) && c.head_dim == 128;
   const bool attn_tc = sizeof(T) == 2 && (m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim);
-  __half *wq16 = (__half *)b.w16, *wk16 = wq16 + (size_t)dq * d, *wv16 = wk16 + (size_t)dkv * d, *wo16 = wv16 + (size_t)dkv * d;
-  __half *wg16 = wo16 + (size_t)d * dq, *wu16 = wg16 + (size_t)F * d, *wd16 = wu16 + (size_t)F * d;
+  const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
+  __half *wq16 = nullptr, *wk16 = nullptr, *wv16 = nullptr, *wo16 = nullptr, *wg16 = nullptr, *wu16 = nullptr, *wd16 = nullptr;
+  auto w16_select = [&](int buf) {
+    wq16 = (__half *)b.w16 + (size_t)buf * w16_layer; wk16 = wq16 + (size_t)dq * d; wv16 = wk16 + (size_t)dkv * d;
+    wo16 = wv16 + (size_t)dkv * d; wg16 = wo16 + (size_t)d * dq; wu16 = wg16 + (size_t)F * d; wd16 = wu16 + (size_t)F * d;
+  };
+  // layer j's copy is made on the side stream into buffer j % 2 while layer j - 1 computes on `st`
+  auto convert_layer = [&](int j) {
+    const swiftkv_layer_weights &lw = m->layers[j];
+    const int buf = j & 1;
+    if (j >= 2) cudaStreamWaitEvent(m->side, m->ev_free[buf], 0);   // layer j - 2 has finished with this buffer
+    w16_select(buf);
+    {
+      Scope s(m, m->side, SWIFTKV_KC_ELEMWISE, 7, false);
+      launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, m->side);
+    }
+    cudaEventRecord(m->ev_ready[buf], m->side);
+  };
+  if constexpr (sizeof(T) == 2) {
+    if (use_w16 && l > 0) {
+      cudaEventRecord(m->ev_start, st);                 // the side stream starts after everything queued before
+      cudaStreamWaitEvent(m->side, m->ev_start, 0);
+      convert_layer(0);
+    }
+  }
   __half *k16 = (__half *)b.kv16, *v16 = k16 + plane;
 
   const int32_t *slot_map = bt.plain ? nullptr : b.slot;        // cache row of each new token (identity when plain)
@@ -373,14 +423,9 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
     if constexpr (sizeof(T) == 2) {
       if (use_w16) {
-        Scope s(m, st, SWIFTKV_KC_ELEMWISE, 7);
-        launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, st);
-        launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, st);
-        launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, st);
-        launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, st);
-        launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, st);
-        launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, st);
-        launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, st);
+        if (j + 1 < l) convert_layer(j + 1);            // queued now, runs beside this layer's kernels
+        w16_select(j & 1);
+        cudaStreamWaitEvent(st, m->ev_ready[j & 1], 0);
       }
     }
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
@@ -453,6 +498,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     rc = gemm_any<TA, T>(m, act, T_tok, F, (const T *)lw.w_down, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
                          use_w16 ? wd16 : nullptr);
     if (rc) return rc;
+    if (use_w16) cudaEventRecord(m->ev_free[j & 1], st);   // this layer's half copies may be overwritten
   }
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
