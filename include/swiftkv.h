@@ -140,7 +140,14 @@ typedef struct {
                           max_tokens; the caller keeps a sequence's region fixed for the sequence's lifetime        */
   int32_t emit;        /* != 0: the last new token continues through layers l+1..L and gets logits (every decode
                           token; the last chunk of a prompt)                                                         */
+  const int32_t *block_table;   /* paged cache (optional, HOST array): page numbers of this sequence; token p lives in
+                          row block_table[p / 128] * 128 + p % 128 of every cache plane and cache_row is ignored.
+                          Pages are SWIFTKV_PAGE_ROWS = 128 rows; a page belongs to one sequence; either every sequence
+                          of a step has a table or none has.  With AcrossKV the layers of a group share the pages
+                          (one slot per group), which is how an allocator turns the grouping into memory savings.  */
+  int32_t n_blocks;    /* entries of block_table; must cover n_past + n_new tokens                                  */
 } swiftkv_seq_step;
+#define SWIFTKV_PAGE_ROWS 128
 
 /*
  * One forward pass over a mixed minibatch with SwiftKV (Sec. 3.5): layers 1..l run on all new tokens, which attend to

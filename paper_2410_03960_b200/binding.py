@@ -46,7 +46,8 @@ class _Weights(C.Structure):
 
 
 class _SeqStep(C.Structure):
-    _fields_ = [("n_new", C.c_int32), ("n_past", C.c_int32), ("cache_row", C.c_int32), ("emit", C.c_int32)]
+    _fields_ = [("n_new", C.c_int32), ("n_past", C.c_int32), ("cache_row", C.c_int32), ("emit", C.c_int32),
+                ("block_table", C.POINTER(C.c_int32)), ("n_blocks", C.c_int32)]
 
 
 class _KVView(C.Structure):
@@ -182,10 +183,20 @@ class SwiftKVModel:
     def step(self, tokens, seqs: Sequence[Tuple[int, int, int, int]], swift_layer: int, acrosskv_group: int = 1,
              stream: Optional[torch.cuda.Stream] = None) -> None:
         """swiftkv_step: one forward pass over a mixed minibatch.  `tokens`: HOST int32, the new tokens of all sequences
-        packed in order; `seqs`: one (n_new, n_past, cache_row, emit) tuple per sequence."""
+        packed in order; `seqs`: one (n_new, n_past, cache_row, emit) tuple per sequence, or -- paged cache --
+        (n_new, n_past, block_table, emit) with block_table a list of 128-row page numbers."""
         tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous()
         assert not tokens.is_cuda and tokens.numel() == sum(s[0] for s in seqs)
-        arr = (_SeqStep * len(seqs))(*[_SeqStep(int(a), int(p), int(r), int(e)) for a, p, r, e in seqs])
+        keep = []                      # ctypes arrays of the block tables must outlive the call
+        items = []
+        for a, p, r, e in seqs:
+            if isinstance(r, (list, tuple)):
+                tab = (C.c_int32 * len(r))(*[int(x) for x in r])
+                keep.append(tab)
+                items.append(_SeqStep(int(a), int(p), 0, int(e), tab, len(r)))
+            else:
+                items.append(_SeqStep(int(a), int(p), int(r), int(e), None, 0))
+        arr = (_SeqStep * len(seqs))(*items)
         with torch.cuda.device(self.device):
             _check(self.lib.swiftkv_step(self._h, tokens.data_ptr(), arr, len(seqs), swift_layer, acrosskv_group,
                                          _stream_ptr(stream)))

@@ -71,6 +71,7 @@ struct Buffers {
   int32_t *kv_row0, *kv_len;   // [B] first cache row / number of cached + new tokens of every sequence
   int32_t *kcu;             // [B+1] offsets of the sequences in the gathered half K / V copy (chunked steps)
   int32_t *emit_row0, *emit_len;   // [B] cache range of the sequences whose last new token continues
+  int32_t *blk, *blk_emit;  // [B][pages] block tables of a paged step, and the rows of the emitting sequences
   unsigned int *status;
   float *cos_tab, *sin_tab;
 };
@@ -158,6 +159,9 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.kcu = (int32_t *)cv.take((size_t)(B + 1) * 4);
   b.emit_row0 = (int32_t *)cv.take((size_t)B * 4);
   b.emit_len = (int32_t *)cv.take((size_t)B * 4);
+  const size_t pages = ((size_t)T + PAGE_ROWS - 1) / PAGE_ROWS;
+  b.blk = (int32_t *)cv.take((size_t)B * pages * 4);
+  b.blk_emit = (int32_t *)cv.take((size_t)B * pages * 4);
   b.status = (unsigned int *)cv.take(256);
   b.cos_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
   b.sin_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
@@ -335,6 +339,8 @@ struct Batch {
   int max_kv;         // longest cached + new length
   int total_kv;       // sum of cached + new lengths
   bool plain;
+  bool paged;         // sequences own lists of 128-row pages instead of one contiguous region
+  int blk_stride;     // pages per sequence in the device block tables
 };
 
 template <typename TA, typename T>
@@ -392,6 +398,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const int32_t *slot_map = bt.plain ? nullptr : b.slot;        // cache row of each new token (identity when plain)
   const int32_t *k_row0 = bt.plain ? nullptr : b.kv_row0;
   const int32_t *kv_len = bt.plain ? nullptr : b.kv_len;
+  const int32_t *blk = bt.paged ? b.blk : nullptr, *blk_emit = bt.paged ? b.blk_emit : nullptr;
   { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_embed<T>((const T *)m->embed, b.tokens, b.x, T_tok, d, c.vocab, b.status, st); }
 
   // one-time model transformation for this (l, g): fold each group leader's input-norm gain into its W_K, W_V
@@ -455,18 +462,20 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
             kk = k16; vv = v16;
             if (!bt.plain) {
               Scope s2(m, st, SWIFTKV_KC_ELEMWISE);
-              launch_gather_kv_half((const bf16 *)Kj, (const bf16 *)Vj, k16, v16, b.kv_row0, b.kv_len, b.kcu, B, bt.max_kv, dkv, st);
+              launch_gather_kv_half((const bf16 *)Kj, (const bf16 *)Vj, k16, v16, b.kv_row0, b.kv_len, b.kcu, blk, bt.blk_stride, B, bt.max_kv, dkv, st);
               kr0 = b.kcu;
               kv_rows = bt.total_kv;
             }
           }
-          rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, kr0, kv_len, B, T_tok, kv_rows, bt.max_new, c.n_q_heads,
+          // (the gathered half copies are contiguous: only a direct read of the cache follows the block tables)
+          const int32_t *ablk = (act_f16 && !bt.plain) ? nullptr : blk;
+          rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, kr0, kv_len, ablk, bt.blk_stride, B, T_tok, kv_rows, bt.max_new, c.n_q_heads,
                                    c.n_kv_heads, c.head_dim, b.status, st);
           if (rc == SWIFTKV_OK) done = true;
           else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
         }
       }
-      if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, k_row0, kv_len, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
+      if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, k_row0, kv_len, blk, bt.blk_stride, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
     }
     rc = gemm_any<TA, T>(m, attn, T_tok, dq, (const T *)lw.wo, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
                          use_w16 ? wo16 : nullptr);
@@ -528,7 +537,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.emit_row0 + r0, b.emit_len + r0, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.emit_row0 + r0, b.emit_len + r0, blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
@@ -551,17 +560,35 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
   if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
   Batch bt{};
   bt.B = n_seqs; bt.plain = plain;
+  bt.paged = seqs[0].block_table != nullptr;
+  bt.blk_stride = (m->max_tokens + PAGE_ROWS - 1) / PAGE_ROWS;
+  const int n_pages = m->max_tokens / PAGE_ROWS;          // whole pages inside a cache plane
+  std::vector<char> page_used(bt.paged ? n_pages : 0, 0);
   long long total = 0, total_kv = 0;
   int rows_used = 0;
   for (int i = 0; i < n_seqs; ++i) {
     const swiftkv_seq_step &s = seqs[i];
     if (s.n_new < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: n_new = %d < 1", i, s.n_new);
     if (s.n_past < 0 || s.cache_row < 0) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: negative n_past / cache_row", i);
-    const long long end = (long long)s.cache_row + s.n_past + s.n_new;
-    if (end > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: cache rows up to %lld exceed max_tokens %d", i, end, m->max_tokens);
-    for (int k = 0; k < i; ++k) {   // regions of different sequences must not overlap
-      const long long a0 = seqs[k].cache_row, a1 = a0 + seqs[k].n_past + seqs[k].n_new;
-      if (s.cache_row < a1 && a0 < end) return fail(SWIFTKV_ERR_INVALID_ARG, "cache rows of sequences %d and %d overlap", k, i);
+    if ((s.block_table != nullptr) != bt.paged) return fail(SWIFTKV_ERR_INVALID_ARG, "either every sequence has a block table or none");
+    long long end = (long long)s.cache_row + s.n_past + s.n_new;
+    if (bt.paged) {
+      const int need = (s.n_past + s.n_new + PAGE_ROWS - 1) / PAGE_ROWS;
+      if (s.n_blocks < need) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: %d pages listed, %d needed", i, s.n_blocks, need);
+      end = 0;
+      for (int k = 0; k < need; ++k) {
+        const int pg = s.block_table[k];
+        if (pg < 0 || pg >= n_pages) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: page %d outside [0, %d)", i, pg, n_pages);
+        if (page_used[pg]) return fail(SWIFTKV_ERR_INVALID_ARG, "page %d is listed twice", pg);
+        page_used[pg] = 1;
+        end = std::max(end, (long long)(pg + 1) * PAGE_ROWS);
+      }
+    } else {
+      if (end > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: cache rows up to %lld exceed max_tokens %d", i, end, m->max_tokens);
+      for (int k = 0; k < i; ++k) {   // regions of different sequences must not overlap
+        const long long a0 = seqs[k].cache_row, a1 = a0 + seqs[k].n_past + seqs[k].n_new;
+        if (s.cache_row < a1 && a0 < end) return fail(SWIFTKV_ERR_INVALID_ARG, "cache rows of sequences %d and %d overlap", k, i);
+      }
     }
     total += s.n_new;
     total_kv += s.n_past + s.n_new;
@@ -603,10 +630,25 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
     row0[i] = s.cache_row;
     klen[i] = s.n_past + s.n_new;
     kcu[i + 1] = kcu[i] + klen[i];
-    for (int k = 0; k < s.n_new; ++k) { pos[cu[i] + k] = s.n_past + k; slot[cu[i] + k] = s.cache_row + s.n_past + k; }
+    for (int k = 0; k < s.n_new; ++k) {
+      const int pp = s.n_past + k;
+      pos[cu[i] + k] = pp;
+      slot[cu[i] + k] = bt.paged ? s.block_table[pp / PAGE_ROWS] * PAGE_ROWS + pp % PAGE_ROWS : s.cache_row + pp;
+    }
     if (s.emit) { last_idx[ne] = cu[i + 1] - 1; last_pos[ne] = klen[i] - 1; e_row0[ne] = s.cache_row; e_len[ne] = klen[i]; ++ne; }
   }
   Buffers &b = m->b;
+  if (bt.paged) {   // block tables of all sequences, and once more for the emitting ones in their order
+    std::vector<int32_t> tb((size_t)B * bt.blk_stride, 0), te((size_t)B * bt.blk_stride, 0);
+    int e = 0;
+    for (int i = 0; i < B; ++i) {
+      const int need = (klen[i] + PAGE_ROWS - 1) / PAGE_ROWS;
+      for (int k = 0; k < need; ++k) tb[(size_t)i * bt.blk_stride + k] = seqs[i].block_table[k];
+      if (seqs[i].emit) { std::copy_n(&tb[(size_t)i * bt.blk_stride], need, &te[(size_t)e * bt.blk_stride]); ++e; }
+    }
+    CUDA_TRY(cudaMemcpyAsync(b.blk, tb.data(), tb.size() * 4, cudaMemcpyHostToDevice, st));
+    CUDA_TRY(cudaMemcpyAsync(b.blk_emit, te.data(), te.size() * 4, cudaMemcpyHostToDevice, st));
+  }
   CUDA_TRY(cudaMemcpyAsync(b.cu, cu, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.pos, pos, (size_t)T * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.slot, slot, (size_t)T * 4, cudaMemcpyHostToDevice, st));
@@ -639,7 +681,7 @@ static int32_t prefill_common(swiftkv_model *m, const int32_t *tokens, bool toke
   for (int i = 0; i < n_seqs; ++i) {
     if (seq_lens[i] < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "seq_lens[%d] = %d < 1", i, seq_lens[i]);
     if (row + seq_lens[i] > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "more than max_tokens %d tokens", m->max_tokens);
-    seqs[i] = swiftkv_seq_step{seq_lens[i], 0, (int32_t)row, 1};   // whole prompt, packed rows, last token emits
+    seqs[i] = swiftkv_seq_step{seq_lens[i], 0, (int32_t)row, 1, nullptr, 0};   // whole prompt, packed rows, last token emits
     row += seq_lens[i];
   }
   return forward_common(m, tokens, tokens_on_device, seqs.data(), n_seqs, true, l, g, stream);
@@ -779,20 +821,20 @@ extern "C" int32_t swiftkv_attention_prefill(const void *q, const void *k, const
       return fail(SWIFTKV_ERR_UNSUPPORTED, "tensor-core attention needs q, K, V of one 16-bit type, head_dim 128, an even group size");
     unsigned int *status = op_status_word();
     if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
-    int rc = launch_attention_tc(q, q_dtype == SWIFTKV_DTYPE_F16, k, v, out, cu_seqlens, nullptr, nullptr, n_seqs,
+    int rc = launch_attention_tc(q, q_dtype == SWIFTKV_DTYPE_F16, k, v, out, cu_seqlens, nullptr, nullptr, nullptr, 0, n_seqs,
                                  total_tokens, total_tokens, max_seq_len, n_q_heads, n_kv_heads, head_dim, status, st);
     if (rc) return fail(rc, "attention launch failed");
     return SWIFTKV_OK;
   }
   if (q_dtype == SWIFTKV_DTYPE_BF16 && kv_dtype == SWIFTKV_DTYPE_BF16)
-    launch_attention_simple<bf16, bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr, nullptr,
+    launch_attention_simple<bf16, bf16>((const bf16 *)q, (const bf16 *)k, (const bf16 *)v, (bf16 *)out, cu_seqlens, n_seqs, nullptr, nullptr, nullptr, 0,
                                         total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else if (q_dtype == SWIFTKV_DTYPE_F16 && kv_dtype == SWIFTKV_DTYPE_BF16)
     launch_attention_simple<__half, bf16>((const __half *)q, (const bf16 *)k, (const bf16 *)v, (__half *)out, cu_seqlens, n_seqs,
-                                          nullptr, nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+                                          nullptr, nullptr, nullptr, 0, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else if (q_dtype == SWIFTKV_DTYPE_F32 && kv_dtype == SWIFTKV_DTYPE_F32)
     launch_attention_simple<float, float>((const float *)q, (const float *)k, (const float *)v, (float *)out, cu_seqlens, n_seqs,
-                                          nullptr, nullptr, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
+                                          nullptr, nullptr, nullptr, 0, total_tokens, n_q_heads, n_kv_heads, head_dim, st);
   else
     return fail(SWIFTKV_ERR_INVALID_ARG, "unsupported dtype combination");
   cudaError_t e = cudaGetLastError();
@@ -819,10 +861,10 @@ extern "C" int32_t swiftkv_tail_attention(const float *q, const void *k_cache, c
                 tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (dtype == SWIFTKV_DTYPE_BF16)
-    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, nullptr, n_seqs, max_seq_len, n_q_heads,
+    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len, n_q_heads,
                                 n_kv_heads, head_dim, (float *)scratch, st);
   else if (dtype == SWIFTKV_DTYPE_F32)
-    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, nullptr, n_seqs, max_seq_len,
+    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len,
                                  n_q_heads, n_kv_heads, head_dim, (float *)scratch, st);
   else
     return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");

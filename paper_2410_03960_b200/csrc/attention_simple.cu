@@ -13,7 +13,8 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
                                                                const T *__restrict__ v, TQ *__restrict__ out,
                                                                const int32_t *__restrict__ cu, int n_seqs,
                                                                const int32_t *__restrict__ k_row0,
-                                                               const int32_t *__restrict__ kv_len, int n_tokens,
+                                                               const int32_t *__restrict__ kv_len,
+                                                               const int32_t *__restrict__ blk, int blk_stride, int n_tokens,
                                                                int n_q, int n_kv, int hd, float scale) {
   extern __shared__ float q_sm[];   // [4 warps][hd]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
     const int key = c0 + lane;
     float s = -INFINITY;
     if (key <= p) {
-      const T *kr = k + ((size_t)(first + key) * n_kv + kvh) * hd;
+      const T *kr = k + (kv_row_of(blk, blk_stride, lo, first, key) * n_kv + kvh) * hd;
       float dot = 0.f;
       for (int i = 0; i < hd; ++i) dot = fmaf(qs[i], to_f(kr[i]), dot);
       s = dot;
@@ -59,7 +60,7 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
     const int n_here = min(32, p - c0 + 1);
     for (int i = 0; i < n_here; ++i) {
       const float pi = __shfl_sync(0xffffffffu, pe, i);
-      const T *vr = v + ((size_t)(first + c0 + i) * n_kv + kvh) * hd;
+      const T *vr = v + (kv_row_of(blk, blk_stride, lo, first, c0 + i) * n_kv + kvh) * hd;
 #pragma unroll
       for (int e = 0; e < MAX_E; ++e) {
         const int dd = lane + 32 * e;
@@ -78,23 +79,23 @@ __global__ void __launch_bounds__(128) attention_simple_kernel(const TQ *__restr
 
 template <typename TQ, typename T>
 void launch_attention_simple(const TQ *q, const T *k, const T *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
-                             const int32_t *k_row0, const int32_t *kv_len, int n_tokens, int n_q, int n_kv, int hd,
-                             cudaStream_t st) {
+                             const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride,
+                             int n_tokens, int n_q, int n_kv, int hd, cudaStream_t st) {
   if (n_tokens <= 0) return;
   const long long items = (long long)n_tokens * n_q;
   const unsigned blocks = (unsigned)((items + 3) / 4);
   const float scale = 1.0f / sqrtf((float)hd);
   const size_t smem = 4 * hd * sizeof(float);
-  if (hd <= 32) attention_simple_kernel<TQ, T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 64) attention_simple_kernel<TQ, T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
-  else if (hd <= 128) attention_simple_kernel<TQ, T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
-  else attention_simple_kernel<TQ, T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, n_tokens, n_q, n_kv, hd, scale);
+  if (hd <= 32) attention_simple_kernel<TQ, T, 1><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, blk, blk_stride, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 64) attention_simple_kernel<TQ, T, 2><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, blk, blk_stride, n_tokens, n_q, n_kv, hd, scale);
+  else if (hd <= 128) attention_simple_kernel<TQ, T, 4><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, blk, blk_stride, n_tokens, n_q, n_kv, hd, scale);
+  else attention_simple_kernel<TQ, T, 8><<<blocks, 128, smem, st>>>(q, k, v, out, cu_seqlens, n_seqs, k_row0, kv_len, blk, blk_stride, n_tokens, n_q, n_kv, hd, scale);
 }
 template void launch_attention_simple<float, float>(const float *, const float *, const float *, float *, const int32_t *, int,
-                                                    const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
+                                                    const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, cudaStream_t);
 template void launch_attention_simple<bf16, bf16>(const bf16 *, const bf16 *, const bf16 *, bf16 *, const int32_t *, int,
-                                                  const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
+                                                  const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, cudaStream_t);
 template void launch_attention_simple<__half, bf16>(const __half *, const bf16 *, const bf16 *, __half *, const int32_t *, int,
-                                                    const int32_t *, const int32_t *, int, int, int, int, cudaStream_t);
+                                                    const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, cudaStream_t);
 
 }  // namespace skv

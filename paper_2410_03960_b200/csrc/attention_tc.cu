@@ -34,6 +34,8 @@ struct AttnParams {
   const int32_t *cu;        // [n_seqs+1] offsets of each sequence's NEW tokens (the queries) in q / out
   const int32_t *k_row0;    // [n_seqs] first K / V row of each sequence (null: same as cu, i.e. a plain prefill)
   const int32_t *kv_len;    // [n_seqs] keys of each sequence = tokens already cached + new tokens (null: new tokens only)
+  const int32_t *blk;       // optional block tables of a paged cache: key tile j of sequence b starts at row
+  int blk_stride;           //   blk[b * blk_stride + j] * 128 (a key tile is exactly one page)
   bf16 *out;
   int n_seqs, n_q, n_kv, max_tiles;
   float scale_log2;     // softmax scale * log2(e)
@@ -132,16 +134,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       for (int j = 0; j < n_kv_tiles; ++j) {
         const int s = j & 1;
         const uint32_t ph = (j >> 1) & 1;
+        const int krow = p.blk ? p.blk[(size_t)b * p.blk_stride + j] * BKV : k0 + j * BKV;
         if (!wait_or_abort(tc::smem_u32(&k_empty[s]), ph ^ 1, abort_flag, p.status)) break;
         const uint32_t kb = tc::smem_u32(&k_full[s]);
         tc::mbar_expect_tx(kb, TILE_BYTES);
         for (int c = 0; c < 2; ++c)
-          tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, k0 + j * BKV);
+          tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, krow);
         if (!wait_or_abort(tc::smem_u32(&v_empty[s]), ph ^ 1, abort_flag, p.status)) break;
         const uint32_t vb = tc::smem_u32(&v_full[s]);
         tc::mbar_expect_tx(vb, TILE_BYTES);
         for (int c = 0; c < 2; ++c)
-          tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, k0 + j * BKV);
+          tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, krow);
       }
     }
   } else if (warp == 1) {
@@ -353,8 +356,9 @@ bool tc_attention_supported(int n_q, int n_kv, int hd) {
 }
 
 int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
-                        const int32_t *k_row0, const int32_t *kv_len, int n_seqs, int n_tokens, int kv_rows,
-                        int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st) {
+                        const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
+                        int n_tokens, int kv_rows, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
+                        cudaStream_t st) {
   if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
   if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1 || kv_rows < 1) return SWIFTKV_ERR_INVALID_ARG;
   CUtensorMap tq, tk, tv;
@@ -372,7 +376,7 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
     attr_set = true;
   }
   AttnParams p{};
-  p.cu = cu_seqlens; p.k_row0 = k_row0; p.kv_len = kv_len; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
+  p.cu = cu_seqlens; p.k_row0 = k_row0; p.kv_len = kv_len; p.blk = blk; p.blk_stride = blk_stride; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
   p.max_tiles = (max_seq_len + BQ - 1) / BQ;
   p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
   p.status = status;

@@ -56,7 +56,14 @@ struct OutDesc {
 };
 inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDesc{mode, p, ld, n, nullptr, 0, 1, nullptr}; }
 
+// ---- paged cache rows ------------------------------------------------------------------------------------
+// A sequence's token p lives in cache row first + p (contiguous region), or -- with a block table -- in row
+// blk[b * stride + p / PAGE_ROWS] * PAGE_ROWS + p % PAGE_ROWS.
+constexpr int PAGE_ROWS = 128;
 #ifdef __CUDACC__
+__device__ __forceinline__ size_t kv_row_of(const int32_t *blk, int stride, int b, int first, int p) {
+  return blk ? (size_t)blk[(size_t)b * stride + (p >> 7)] * PAGE_ROWS + (p & (PAGE_ROWS - 1)) : (size_t)first + p;
+}
 // write one fp32 accumulator where the descriptor says (device side)
 // TP: element type of the p0 region; TS: element type of the segments (K / V cache planes)
 template <typename TP, typename TS>
@@ -98,7 +105,8 @@ void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *pos
 // packs each sequence's cache rows [row0[b], row0[b] + len[b]) of one layer's K and V planes (bf16) into contiguous half
 // copies starting at row kcu[b]: the tensor-core attention kernel's operands in a chunked step with half activations
 void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
-                           const int32_t *kcu, int n_seqs, int max_len, int dkv, cudaStream_t st);
+                           const int32_t *kcu, const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv,
+                           cudaStream_t st);
 template <typename T>
 void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
@@ -142,16 +150,18 @@ bool tc_swiglu_supported(int M, int F, int K);
 // k_row0 / kv_len as for launch_attention_tc
 template <typename TQ, typename TKV>
 void launch_attention_simple(const TQ *q, const TKV *k, const TKV *v, TQ *out, const int32_t *cu_seqlens, int n_seqs,
-                             const int32_t *k_row0, const int32_t *kv_len, int n_tokens, int n_q, int n_kv, int hd,
-                             cudaStream_t st);
+                             const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride,
+                             int n_tokens, int n_q, int n_kv, int hd, cudaStream_t st);
 bool tc_attention_supported(int n_q, int n_kv, int hd);
 // f16: q, k, v and out all hold IEEE halves (else all bfloat16).  cu_seqlens: offsets of each sequence's new tokens
 // (queries) in q / out; k_row0 / kv_len (both nullable): first K / V row and number of keys (cached + new) of each
 // sequence -- null means a plain prefill whose K / V rows are packed like q; kv_rows: rows of k / v that hold data;
 // max_seq_len bounds the new tokens of one sequence
+// blk / blk_stride (nullable): block tables of a paged cache, see kv_row_of (then k_row0 is ignored)
 int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
-                        const int32_t *k_row0, const int32_t *kv_len, int n_seqs, int n_tokens, int kv_rows,
-                        int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status, cudaStream_t st);
+                        const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
+                        int n_tokens, int kv_rows, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
+                        cudaStream_t st);
 
 // tail.cu : the last-token path (at most MAX_TAIL_ROWS activation rows per launch, fp32 activations)
 constexpr int MAX_TAIL_ROWS = 8;
@@ -167,6 +177,7 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *row0, const int32_t *len,
-                           int n_seqs, int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
+                           const int32_t *blk, int blk_stride, int n_seqs, int max_seq_len, int n_q, int n_kv, int hd,
+                           float *scratch, cudaStream_t st);
 
 }  // namespace skv

@@ -242,10 +242,11 @@ template void launch_fold<bf16, __half>(const bf16 *, const bf16 *, __half *, in
 
 __global__ void gather_kv_half_kernel(const bf16 *__restrict__ k, const bf16 *__restrict__ v, __half *__restrict__ k16,
                                       __half *__restrict__ v16, const int32_t *__restrict__ row0,
-                                      const int32_t *__restrict__ len, const int32_t *__restrict__ kcu, int dkv) {
+                                      const int32_t *__restrict__ len, const int32_t *__restrict__ kcu,
+                                      const int32_t *__restrict__ blk, int blk_stride, int dkv) {
   const int b = blockIdx.y, r = blockIdx.x;
   if (r >= len[b]) return;
-  const size_t src = ((size_t)row0[b] + r) * dkv, dst = ((size_t)kcu[b] + r) * dkv;
+  const size_t src = kv_row_of(blk, blk_stride, b, row0[b], r) * dkv, dst = ((size_t)kcu[b] + r) * dkv;
   for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
     const uint4 kr = *reinterpret_cast<const uint4 *>(k + src + i), vr = *reinterpret_cast<const uint4 *>(v + src + i);
     const __nv_bfloat162 *k2 = reinterpret_cast<const __nv_bfloat162 *>(&kr), *v2 = reinterpret_cast<const __nv_bfloat162 *>(&vr);
@@ -258,9 +259,10 @@ __global__ void gather_kv_half_kernel(const bf16 *__restrict__ k, const bf16 *__
   }
 }
 void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
-                           const int32_t *kcu, int n_seqs, int max_len, int dkv, cudaStream_t st) {
+                           const int32_t *kcu, const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv,
+                           cudaStream_t st) {
   if (n_seqs <= 0 || max_len <= 0) return;
-  gather_kv_half_kernel<<<dim3(max_len, n_seqs), 128, 0, st>>>(k, v, k16, v16, row0, len, kcu, dkv);
+  gather_kv_half_kernel<<<dim3(max_len, n_seqs), 128, 0, st>>>(k, v, k16, v16, row0, len, kcu, blk, blk_stride, dkv);
 }
 
 // bfloat16 -> IEEE half copy of a weight matrix (exact for |w| >= 2^-17, absolute error <= 2^-25 below), 128-bit accesses

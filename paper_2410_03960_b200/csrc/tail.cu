@@ -274,7 +274,8 @@ constexpr int TA_WARPS = 4;
 template <typename T, int REP, int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    const int32_t *__restrict__ len, int n_q, int n_kv, int chunk, int n_splits, float scale, float *__restrict__ scratch) {
+    const int32_t *__restrict__ len, const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk,
+    int n_splits, float scale, float *__restrict__ scratch) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
   __shared__ float qs[REP][HD];
   __shared__ float w_m[TA_WARPS][REP], w_l[TA_WARPS][REP];
@@ -298,7 +299,7 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
 #pragma unroll
     for (int r = 0; r < REP; ++r) sc[r] = 0.f;
     if (valid) {
-      const T *kr = kc + ((size_t)(first + key) * n_kv + kvh) * HD;
+      const T *kr = kc + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * HD;
       constexpr int V = 16 / sizeof(T);
 #pragma unroll 4
       for (int i = 0; i < HD; i += V) {
@@ -324,7 +325,8 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
       m[r] = m_new;
     }
     const int n_here = min(32, k_end - c0);
-    const T *vbase = vc + ((size_t)(first + c0) * n_kv + kvh) * HD + lane * 4;
+    // (a 32-key chunk never straddles a 128-row page: c0 is a multiple of 32)
+    const T *vbase = vc + (kv_row_of(blk, blk_stride, b, first, c0) * n_kv + kvh) * HD + lane * 4;
 #pragma unroll 4
     for (int i = 0; i < n_here; ++i) {
       const T *vr = vbase + (size_t)i * n_kv * HD;
@@ -374,8 +376,8 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
 template <typename T, int MAX_E>
 __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    const int32_t *__restrict__ len, int n_q, int n_kv, int hd, int chunk, int n_splits, float scale,
-    float *__restrict__ scratch) {
+    const int32_t *__restrict__ len, const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int hd, int chunk,
+    int n_splits, float scale, float *__restrict__ scratch) {
   extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -395,7 +397,7 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     for (int c0 = k_begin; c0 < k_end; c0 += 32) {
       const int key = c0 + lane;
       float s = -INFINITY;
-      if (key < k_end) s = dot_row<T>(qs, kc + ((size_t)(first + key) * n_kv + kvh) * hd, hd);
+      if (key < k_end) s = dot_row<T>(qs, kc + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * hd, hd);
       const float m_new = fmaxf(m, warp_max(s));
       const float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
       const float corr = __expf(m - m_new);
@@ -406,7 +408,7 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
       const int n_here = min(32, k_end - c0);
       for (int i = 0; i < n_here; ++i) {
         const float pi = __shfl_sync(0xffffffffu, pe, i);
-        const T *vr = vc + ((size_t)(first + c0 + i) * n_kv + kvh) * hd;
+        const T *vr = vc + (kv_row_of(blk, blk_stride, b, first, c0 + i) * n_kv + kvh) * hd;
 #pragma unroll
         for (int e = 0; e < MAX_E; ++e) {
           const int dd = lane + 32 * e;
@@ -454,8 +456,8 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens,
-                           const int32_t *len, int n_seqs, int max_seq_len, int n_q, int n_kv, int hd, float *scratch,
-                           cudaStream_t st) {
+                           const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs, int max_seq_len, int n_q,
+                           int n_kv, int hd, float *scratch, cudaStream_t st) {
   if (n_seqs <= 0) return;
   const int chunk = tail_chunk(max_seq_len);
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
@@ -463,25 +465,25 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out,
   const int rep = n_q / n_kv;
   if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
     dim3 grid(n_splits, n_kv, n_seqs);
-    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, chunk, n_splits, scale, scratch);
+    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
     tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
     return;
   }
   const int threads = 32 * (rep < 8 ? rep : 8);
   const size_t smem = (size_t)rep * hd * sizeof(float);
   dim3 grid(n_splits, n_kv, n_seqs);
-  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
 template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *,
-                                           const int32_t *, int, int, int, int, int, float *, cudaStream_t);
+                                           const int32_t *, const int32_t *, int, int, int, int, int, int, float *, cudaStream_t);
 template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, float *, const int32_t *,
-                                          const int32_t *, int, int, int, int, int, float *, cudaStream_t);
+                                          const int32_t *, const int32_t *, int, int, int, int, int, int, float *, cudaStream_t);
 
 }  // namespace skv

@@ -122,3 +122,72 @@ def test_step_argument_checks():
         with pytest.raises(P.SwiftKVError) as e:
             model.step(tok[:max(n, 1)] if n else tok[:0], bad, 2, 1)
         assert e.value.code == -1
+
+
+def _paged_rows(pages, n):
+    """Cache rows of tokens 0..n-1 of a sequence that owns `pages` (128-row pages)."""
+    p = np.arange(n)
+    return np.asarray(pages)[p // 128] * 128 + p % 128
+
+
+@pytest.mark.parametrize("shape,dtype,act,kv_bar,lg_bar", [
+    (S.TINY, torch.float32, None, 1e-4, 1e-3),  # SIMT kernels follow the block tables
+    (MID, torch.bfloat16, 1, 2e-2, 0.1),        # half copies gathered through the block tables
+    (MID, torch.bfloat16, 0, 2e-2, 0.1),        # tcgen05 attention fetches K / V tiles page by page
+])
+@pytest.mark.parametrize("l,g", [(2, 1), (1, 2)])
+def test_paged_cache_chunks_and_decode(shape, dtype, act, kv_bar, lg_bar, l, g):
+    """Sequences own scattered, interleaved 128-row pages instead of contiguous regions; results are unchanged."""
+    import paper_2410_03960_b200 as P
+    seed, lens, n_decode = 23, [300, 77, 129], 2
+    n_pages = 12
+    perm = [7, 2, 10, 0, 5, 11, 3, 8, 1, 9, 4, 6]                 # page numbers handed out round-robin
+    pages = [perm[0:9:3], perm[1:4:3], perm[2:9:3][:2]]           # 3, 1, 2 pages: [7,0,3], [2], [10,11]
+    w = S.make_weights(shape, seed, dtype, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    toks = [S.token_ids(seed, b, n + n_decode, shape.vocab) for b, n in enumerate(lens)]
+    model = P.SwiftKVModel(shape, w, dtype, n_pages * 128, len(lens), min(l, 1), 1)
+    if act is not None:
+        model.set_activation_format(act)
+    # two prefill steps (first 60 tokens, then the rest), then decode steps
+    cut = 60
+    model.step(torch.cat([t[:cut] for t in toks]), [(cut, 0, pages[b], int(b == 0)) for b in range(3)], l, g)
+    model.step(torch.cat([toks[b][cut:n] for b, n in enumerate(lens)]),
+               [(n - cut, cut, pages[b], 1) for b, n in enumerate(lens)], l, g)
+    model.status()
+    lg = to_np(model.first_logits())
+
+    def check(n_extra, lg):
+        for b, n in enumerate(lens):
+            m = n + n_extra
+            ref = O.swiftkv(cfg, ow, toks[b][:m].numpy(), [m], l, g)
+            assert np.max(np.abs(lg[b] - ref["logits"][0])) <= lg_bar, (n_extra, b)
+            rows = torch.as_tensor(_paged_rows(pages[b], m), device="cuda")
+            for j in range(shape.n_layers):
+                K, V, _ = model.kv_cache_view(j)
+                assert rel_l2(to_np(K[rows]), ref["K"][j][:m]) <= kv_bar, (b, j)
+                assert rel_l2(to_np(V[rows]), ref["V"][j][:m]) <= kv_bar, (b, j)
+
+    check(0, lg)
+    for t in range(n_decode):
+        if t == 1:
+            pages[2] = pages[2] + [4]          # a fresh page may join a table at any step (unused until needed)
+        model.step(torch.stack([toks[b][n + t] for b, n in enumerate(lens)]),
+                   [(1, n + t, pages[b], 1) for b, n in enumerate(lens)], l, g)
+        model.status()
+        check(t + 1, to_np(model.first_logits()))
+
+
+def test_paged_argument_checks():
+    import paper_2410_03960_b200 as P
+    shape = S.TINY
+    w = S.make_weights(shape, 0, torch.float32, "cuda")
+    model = P.SwiftKVModel(shape, w, torch.float32, 512, 2, 2, 1)      # 4 pages
+    tok = S.token_ids(0, 0, 300, shape.vocab)
+    for bad, n in (([(200, 0, [0], 1)], 200),                       # 2 pages needed, 1 listed
+                   ([(100, 0, [4], 1)], 100),                       # page outside the cache
+                   ([(100, 0, [1], 1), (100, 0, [1], 1)], 200),     # page listed twice
+                   ([(100, 0, [1], 1), (100, 0, 0, 1)], 200)):      # paged and contiguous sequences mixed
+        with pytest.raises(P.SwiftKVError) as e:
+            model.step(tok[:n], bad, 2, 1)
+        assert e.value.code == -1
