@@ -12,6 +12,17 @@ the KV-cache reduction percentages of Sec. 4, and library routines (torch fp64) 
 The paper prints no worked numerical example of a forward pass, so K/V/logit VALUES are pinned by these
 structural facts and library cross-checks only.
 
+FP8 KV cache (appendix "KV quantization": per-token FP8 quantization of the cache, combined with AcrossKV):
+`e4m3_decode` / `e4m3_encode` are the 8-bit format written out from its definition (1 sign, 4 exponent bits with
+bias 7, 3 mantissa bits, no infinities, one NaN pattern, largest finite value 448), `quantize_per_token` gives
+every token's K row and V row of a layer one fp32 scale (row maximum mapped to 448).  The code is an integer
+decided by floating point, so that decision is taken in fp32 exactly as the kernel takes it: fp32 inputs,
+correctly rounded fp32 divisions, round-to-nearest-even, saturation.  With `kv_fp8=True` the cache IS the
+quantized representation: every attention read (prefill of layers <= l included) sees code * scale.
+Pins: the format's defining values and torch's float8_e4m3fn (decode table, encode of random values and of
+every midpoint), a pure-Python nearest-value search, the half-step error bound, scale equivariance, and the
+paper's combined cache reductions (62.5 % and 68.75 %).
+
 Conventions.  Row vectors: a projection is  h @ W.T  with W stored [out_features, in_features] (the paper
 writes W x, Eq. 2).  `l` (swift_layer) is a COUNT: layers 1..l (0-based 0..l-1) run on every prompt token;
 s = output of layer l = the paper's x_{l+1}.  `g` = AcrossKV group size; groups are consecutive, aligned at
@@ -148,8 +159,59 @@ def mlp(m: np.ndarray, w: Dict[str, np.ndarray]) -> np.ndarray:
     return (silu(m @ w["w_gate"].T) * (m @ w["w_up"].T)) @ w["w_down"].T
 
 
-def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.ndarray):
-    """One unmodified decoder layer on all rows of one prompt.  Returns (X_out, K, V) with K after RoPE."""
+# ---------------------------------------------------------------------------------------------------
+# FP8 (e4m3, "fn" flavour: finite only) per-token quantization of cache rows (appendix, KV quantization)
+# ---------------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+AMAX_FLOOR = 2.0 ** -64          # rows that are all (nearly) zero: keeps the scale a normal fp32 number
+
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """Value of each 8-bit code: sign s, exponent field e (4 bits, bias 7), mantissa field m (3 bits).
+    e = 0: subnormal m/8 * 2^-6;  otherwise (1 + m/8) * 2^(e-7);  e = 15, m = 7 is NaN (there are no infinities)."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    s, e, m = c >> 7, (c >> 3) & 15, c & 7
+    val = np.where(e == 0, (m / 8.0) * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(F64)))
+    val = np.where((e == 15) & (m == 7), np.nan, val)
+    return np.where(s == 1, -val, val)
+
+
+def e4m3_encode(y: np.ndarray) -> np.ndarray:
+    """Nearest e4m3 code of each fp32 value, ties to the even mantissa, magnitudes beyond 448 saturate to 448.
+    Works on the exact value of the fp32 input (scaling by powers of two in fp64 is exact)."""
+    y = np.asarray(y, dtype=np.float32).astype(F64)
+    a = np.abs(y)
+    sign = (np.signbit(y)).astype(np.int64) << 7
+    # subnormal range [0, 2^-6): multiples of 2^-9; the count of steps IS the code (8 steps = first normal code)
+    sub = np.rint(a * 2.0 ** 9).astype(np.int64)
+    # normal range: a = (1 + f) * 2^e with f in [0, 1); mantissa steps of 1/8; a carry walks into the exponent field
+    mant, ex = np.frexp(np.where(a > 0, a, 1.0))          # a = mant * 2^ex, mant in [0.5, 1)
+    e = ex - 1
+    q = np.rint((mant * 2.0 - 1.0) * 8.0).astype(np.int64)
+    norm = ((e + 7) << 3) + q
+    code = np.where(a < 2.0 ** -6, sub, norm)
+    code = np.where(a > E4M3_MAX, 0x7E, np.minimum(code, 0x7E))
+    code = np.where(np.isnan(y), 0x7F, code)
+    return (code | sign).astype(np.uint8)
+
+
+def quantize_per_token(x: np.ndarray):
+    """x [n_rows, ...]: one scale per row (token).  scale = max(amax, 2^-64) / 448, code = e4m3(x / scale), every
+    operation on fp32 values with one correctly rounded fp32 result (what `/` on numpy float32 arrays does).
+    Returns (codes uint8 like x, scale float32 [n_rows], dequantized float64 like x = value(code) * scale)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    flat = x32.reshape(x32.shape[0], -1)
+    amax = np.maximum(np.max(np.abs(flat), axis=1), np.float32(AMAX_FLOOR)).astype(np.float32)
+    scale = (amax / np.float32(E4M3_MAX)).astype(np.float32)
+    y = (flat / scale[:, None]).astype(np.float32)
+    codes = e4m3_encode(y)
+    deq = e4m3_decode(codes) * scale.astype(F64)[:, None]
+    return codes.reshape(x32.shape), scale, deq.reshape(x32.shape)
+
+
+def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.ndarray, kv_fp8: bool = False):
+    """One unmodified decoder layer on all rows of one prompt.  Returns (X_out, K, V) with K after RoPE.
+    kv_fp8: K (after RoPE) and V go through the cache's per-token FP8 representation before anyone attends to them."""
     n = X.shape[0]
     h = rmsnorm(X, w["in_norm"], cfg.rms_eps)
     q = (h @ w["wq"].T).reshape(n, cfg.n_q_heads, cfg.head_dim)
@@ -157,6 +219,8 @@ def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.
     v = (h @ w["wv"].T).reshape(n, cfg.n_kv_heads, cfg.head_dim)
     q = rope(q, pos, cfg.rope_theta)
     k = rope(k, pos, cfg.rope_theta)
+    if kv_fp8:
+        k, v = quantize_per_token(k)[2], quantize_per_token(v)[2]
     a = causal_attention(q, k, v)
     X = X + a @ w["wo"].T
     m = rmsnorm(X, w["post_norm"], cfg.rms_eps)
@@ -197,11 +261,14 @@ def group_leader(l: int, g: int, j: int) -> int:
     return l + 1 + g * ((j - l - 1) // g)
 
 
-def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int], l: int, g: int = 1):
+def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int], l: int, g: int = 1,
+            kv_fp8: bool = False):
     """SwiftKV prefill.  Layers 1..l as in the unmodified model; s = x_{l+1}; for every later layer j the
     cache is  K_j = rope(rmsnorm(s, gamma_in[r]) @ W_K[r].T),  V_j = rmsnorm(s, gamma_in[r]) @ W_V[r].T
     with r the leader of j's AcrossKV group (Eq. 2, Sec. 3.3); only the last token of each prompt runs
-    layers l+1..L (footnote in Sec. 3.2; Sec. 3.5), attending to those caches."""
+    layers l+1..L (footnote in Sec. 3.2; Sec. 3.5), attending to those caches.
+    kv_fp8: every cache row is stored as per-token FP8 codes + scale; "K", "V" are then the dequantized values and
+    "K_codes", "K_scale", "V_codes", "V_scale" the stored representation."""
     L = cfg.n_layers
     assert 1 <= l <= L and g >= 1
     tokens = np.asarray(tokens, dtype=np.int64)
@@ -220,7 +287,7 @@ def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]
         Xn = np.empty_like(X)
         for b in range(B):
             a, e = off[b], off[b + 1]
-            Xn[a:e], Kj[a:e], Vj[a:e] = decoder_layer(cfg, w, X[a:e], pos[a:e])
+            Xn[a:e], Kj[a:e], Vj[a:e] = decoder_layer(cfg, w, X[a:e], pos[a:e], kv_fp8)
         X, K[j], V[j] = Xn, Kj, Vj
     s = X                                                      # x_{l+1}
 
@@ -232,6 +299,8 @@ def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]
             k = (h @ w["wk"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
             K[j1 - 1] = rope(k, pos, cfg.rope_theta)
             V[j1 - 1] = (h @ w["wv"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+            if kv_fp8:
+                K[j1 - 1], V[j1 - 1] = quantize_per_token(K[j1 - 1])[2], quantize_per_token(V[j1 - 1])[2]
         else:
             K[j1 - 1] = K[r1 - 1]                              # alias: one cache per group
             V[j1 - 1] = V[r1 - 1]
@@ -244,7 +313,15 @@ def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]
             a, e = off[b], off[b + 1]
             Y[b] = tail_layer(cfg, w, Y[b], e - a - 1, K[j][a:e], V[j][a:e])
     logits = rmsnorm(Y, W.final_norm, cfg.rms_eps) @ W.lm_head().T
-    return {"K": K, "V": V, "logits": logits}
+    out = {"K": K, "V": V, "logits": logits}
+    if kv_fp8:
+        # the stored representation: quantizing a dequantized row again returns its codes (every value is
+        # code * scale with the row maximum at code 448, so the scale comes back up to one fp32 rounding)
+        for name, planes in (("K", K), ("V", V)):
+            qs = [quantize_per_token(pl) for pl in planes]
+            out[name + "_codes"] = [q[0] for q in qs]
+            out[name + "_scale"] = [q[1] for q in qs]
+    return out
 
 
 def swiftkv_eq2_ungrouped(cfg: Config, W: Weights, s: np.ndarray, pos: np.ndarray, l: int):
@@ -323,7 +400,8 @@ def table1_gflops_per_token(cfg: Config, l: int, g: int, context: float) -> Dict
     return {k: v / 1e9 for k, v in dict(vocab=vocab, kv=kv, qo=qo, mlp=mlp_f, attn=attn, total=tot).items()}
 
 
-def kv_cache_reduction(n_layers: int, l: int, g: int) -> float:
-    """Fraction of KV-cache memory saved: layers > l keep one cache per AcrossKV group."""
+def kv_cache_reduction(n_layers: int, l: int, g: int, bytes_ratio: float = 1.0) -> float:
+    """Fraction of KV-cache memory saved: layers > l keep one cache per AcrossKV group; bytes_ratio = bytes of a
+    stored element over bytes of a 16-bit one (0.5 for the FP8 cache; the paper's figures ignore the scales)."""
     n_groups = -(-(n_layers - l) // g)
-    return 1.0 - (l + n_groups) / n_layers
+    return 1.0 - bytes_ratio * (l + n_groups) / n_layers

@@ -349,3 +349,133 @@ def test_normalized_throughput_arithmetic():
     for name, tps, n_gpus, tflops in _rows("normalized_throughput.txt"):
         got = float(tps) * 2 * shapes[name].n_params() / int(n_gpus) / 1e12
         assert abs(got - float(tflops)) / float(tflops) < 0.01
+
+
+# ---------------------------------------------------------------------------------------------------
+# FP8 (e4m3) per-token cache quantization (appendix, KV quantization)
+# ---------------------------------------------------------------------------------------------------
+def test_e4m3_format_defining_values():
+    """Values fixed by the format's definition: bias 7, 3 mantissa bits, no infinities, largest finite 448."""
+    dec = O.e4m3_decode(np.arange(256))
+    assert dec[0x00] == 0.0 and dec[0x80] == 0.0 and np.signbit(dec[0x80])
+    assert dec[0x38] == 1.0 and dec[0x40] == 2.0 and dec[0x3C] == 1.5 and dec[0xB8] == -1.0
+    assert dec[0x01] == 2.0 ** -9 and dec[0x07] == 7 * 2.0 ** -9 and dec[0x08] == 2.0 ** -6
+    assert dec[0x7E] == 448.0 and dec[0xFE] == -448.0 and dec[0x77] == 240.0 and dec[0x78] == 256.0
+    assert np.isnan(dec[0x7F]) and np.isnan(dec[0xFF]) and np.isfinite(np.delete(dec, [0x7F, 0xFF])).all()
+    pos = dec[:0x7F]
+    assert (np.diff(pos) > 0).all()                                # codes order like their values
+    # library cross-check: torch's float8_e4m3fn reads the same 256 bit patterns
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(np.isnan(dec), np.isnan(lib))
+    assert np.array_equal(dec[~np.isnan(dec)], lib[~np.isnan(lib)])
+
+
+def _nearest_code_by_search(y: float) -> int:
+    """Brute force in plain Python: the finite code whose value is nearest to y; of two equally near values the one
+    with the even code (even mantissa field); beyond the largest value, the largest value."""
+    vals = [float(v) for v in O.e4m3_decode(np.arange(0x7F))]     # non-negative finite values, ascending
+    a = abs(y)
+    best, best_d = 0, None
+    for c, v in enumerate(vals):
+        d = abs(a - v)
+        if best_d is None or d < best_d or (d == best_d and c % 2 == 0):
+            best, best_d = c, d
+    return best | (0x80 if math.copysign(1.0, y) < 0 else 0)
+
+
+def test_e4m3_encode_against_search_and_library():
+    vals = O.e4m3_decode(np.arange(0x7F))
+    mid = (vals[:-1] + vals[1:]) / 2                               # every tie point (all exact in fp32)
+    rng = np.random.default_rng(5)
+    probe = np.concatenate([vals, mid, np.nextafter(mid.astype(np.float32), np.float32(0)),
+                            np.nextafter(mid.astype(np.float32), np.float32(1e9)),
+                            rng.uniform(0, 448, 300), rng.uniform(0, 2.0 ** -5, 100), [448.5, 463.9, 464.0, 1e6]])
+    probe = np.concatenate([probe, -probe]).astype(np.float32)
+    got = O.e4m3_encode(probe)
+    want = np.array([_nearest_code_by_search(float(v)) for v in probe], dtype=np.uint8)
+    assert np.array_equal(got, want)
+    # every finite code is a fixed point
+    codes = np.delete(np.arange(256), [0x7F, 0xFF]).astype(np.uint8)
+    assert np.array_equal(O.e4m3_encode(O.e4m3_decode(codes)), codes)
+    # library: torch's conversion rounds to nearest even as well (inside the finite range)
+    big = np.concatenate([probe[np.abs(probe) <= 448], rng.standard_normal(200000).astype(np.float32) * 120]).astype(np.float32)
+    big = big[np.abs(big) <= 448]
+    lib = torch.from_numpy(big).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(O.e4m3_encode(big), lib)
+
+
+def test_quantize_per_token_properties():
+    rng = np.random.default_rng(9)
+    x = (rng.standard_normal((37, 2, 32)) * np.exp(rng.uniform(-6, 6, (37, 1, 1)))).astype(np.float32)
+    x[5] = 0.0                                                     # an all-zero row
+    codes, scale, deq = O.quantize_per_token(x)
+    assert codes.dtype == np.uint8 and codes.shape == x.shape and scale.dtype == np.float32 and scale.shape == (37,)
+    flat, dflat, cflat = x.reshape(37, -1).astype(np.float64), deq.reshape(37, -1), codes.reshape(37, -1)
+    amax = np.abs(flat).max(axis=1)
+    # the scale maps the row maximum to 448 (one fp32 rounding), the maximum itself is stored as +-448
+    nz = amax > 0
+    assert np.allclose(scale[nz].astype(np.float64) * 448, amax[nz], rtol=2.0 ** -23, atol=0)
+    assert ((cflat[nz] & 0x7F).max(axis=1) == 0x7E).all()
+    assert (cflat[5] & 0x7F).max() == 0 and (dflat[5] == 0).all() and scale[5] == np.float32(2.0 ** -64 / 448)
+    # error bound of round-to-nearest: half a step of the code's binade (3 mantissa bits), in units of the scale;
+    # relative error at most 2^-4 for values in the normal range
+    y = flat / scale.astype(np.float64)[:, None]
+    step = np.where(np.abs(y) < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y), 2.0 ** -6))) - 3))
+    err = np.abs(dflat - flat) / scale.astype(np.float64)[:, None]
+    assert (err <= step / 2 * (1 + 1e-6) + 1e-12).all()
+    normal = np.abs(y) >= 2.0 ** -6
+    assert (np.abs(dflat - flat)[normal] <= np.abs(flat)[normal] * 2.0 ** -4 * (1 + 1e-6)).all()
+    assert (np.sign(dflat) * np.sign(flat) >= 0).all()
+    # rows are independent, and a power-of-two factor moves into the scale only
+    c1, s1, _ = O.quantize_per_token(x[3:4])
+    assert np.array_equal(c1[0], codes[3]) and s1[0] == scale[3]
+    c2, s2, d2 = O.quantize_per_token(x * np.float32(8.0))
+    assert np.array_equal(c2[nz], codes[nz]) and np.array_equal(s2[nz], scale[nz] * np.float32(8)) and np.array_equal(d2[nz], deq[nz] * 8)
+    # sign symmetry
+    c3, s3, _ = O.quantize_per_token(-x)
+    assert np.array_equal(c3[nz] ^ 0x80, codes[nz]) and np.array_equal(s3, scale)
+
+
+def test_kv_cache_reduction_with_fp8():
+    for g, fp8, pct in _rows("kv_cache_reduction_fp8.txt"):
+        got = 100 * O.kv_cache_reduction(32, 16, int(g), 0.5 if int(fp8) else 1.0)
+        assert abs(got - float(pct)) < 1e-9
+
+
+def test_swiftkv_with_fp8_cache_structure():
+    """The quantized model: the stored rows are exactly the quantization of what the layer would have cached,
+    everything downstream sees only them, and the structural facts of SwiftKV survive."""
+    shape = S.TINY
+    cfg, W = _cfg(shape), _weights(shape, seed=3)
+    lens = [21, 9]
+    tok = np.concatenate([S.token_ids(3, b, n, shape.vocab).numpy() for b, n in enumerate(lens)])
+    ref = O.swiftkv(cfg, W, tok, lens, 2, 1)
+    q = O.swiftkv(cfg, W, tok, lens, 2, 1, kv_fp8=True)
+    # layer 1 sees the same input either way: its cache is the quantization of the unquantized run's cache
+    for name in ("K", "V"):
+        codes, scale, deq = O.quantize_per_token(ref[name][0])
+        assert np.array_equal(q[name + "_codes"][0], codes) and np.array_equal(q[name + "_scale"][0], scale)
+        assert np.array_equal(q[name][0], deq)
+    # stored representation <-> values, every layer
+    for j in range(shape.n_layers):
+        for name in ("K", "V"):
+            back = O.e4m3_decode(q[name + "_codes"][j]) * q[name + "_scale"][j].astype(np.float64)[:, None, None]
+            assert np.allclose(back, q[name][j], rtol=2.0 ** -22, atol=0)
+            assert 0.005 < rel_l2(q[name][j], ref[name][j]) < 0.06     # 3 mantissa bits: a few percent, not zero
+    assert 0 < rel_l2(q["logits"], ref["logits"]) < 0.2
+    # layer 2's attention read the quantized layer-2 cache: with the quantizer bypassed there, layer 3's input changes
+    # (checked through the SingleInputKV rows, which are a function of the layer-2 output)
+    assert not np.array_equal(q["K_codes"][2], O.quantize_per_token(ref["K"][2])[0])
+    # AcrossKV aliasing and l = L (baseline) still hold
+    q2 = O.swiftkv(cfg, W, tok, lens, 2, 2, kv_fp8=True)
+    assert q2["K"][3] is q2["K"][2] and np.array_equal(q2["K_codes"][2], q["K_codes"][2])
+    full = O.swiftkv(cfg, W, tok, lens, shape.n_layers, 1, kv_fp8=True)
+    assert np.array_equal(full["K_codes"][0], q["K_codes"][0]) and np.array_equal(full["K_codes"][1], q["K_codes"][1])
+    # a prompt alone equals the prompt inside the batch (per-token scales do not couple prompts)
+    alone = O.swiftkv(cfg, W, tok[:21], [21], 2, 1, kv_fp8=True)
+    assert np.array_equal(alone["K_codes"][3], q["K_codes"][3][:21]) and np.allclose(alone["logits"][0], q["logits"][0], rtol=1e-12)
+    # constant prompt: all V rows equal, attention output = that row whatever the scores, so the logits do not
+    # depend on the prompt length (the quantized rows are still identical to each other)
+    c5 = O.swiftkv(cfg, W, np.full(5, 17), [5], 2, 1, kv_fp8=True)
+    c1 = O.swiftkv(cfg, W, np.full(1, 17), [1], 2, 1, kv_fp8=True)
+    assert np.allclose(c5["logits"], c1["logits"], rtol=1e-9, atol=1e-12)
