@@ -48,14 +48,29 @@ extern "C" {
 #define SWIFTKV_DTYPE_F32  0
 #define SWIFTKV_DTYPE_BF16 1
 #define SWIFTKV_DTYPE_F16  2   /* IEEE half: only as the activation type of the stand-alone operators */
+#define SWIFTKV_DTYPE_FP8_E4M3 3   /* element type of the FP8 cache's code planes (see SWIFTKV_KV_FP8)      */
 
 typedef struct swiftkv_model swiftkv_model;   /* opaque, library-owned host object */
 
 typedef struct {
   int32_t vocab, hidden, n_layers, n_q_heads, n_kv_heads, head_dim, ffn;
   float   rope_theta, rms_eps;
-  int32_t dtype;                               /* SWIFTKV_DTYPE_*: storage type of weights, activations, KV cache */
+  int32_t dtype;                               /* SWIFTKV_DTYPE_F32 / BF16: storage type of weights, activations, KV cache */
+  int32_t kv_format;                           /* SWIFTKV_KV_*: how cache rows are stored                          */
 } swiftkv_config;
+
+/*
+ * Cache formats.  SWIFTKV_KV_MODEL_DTYPE: rows in the model dtype.  SWIFTKV_KV_FP8: the per-token FP8 cache that the
+ * paper combines with AcrossKV (appendix "KV quantization"; 62.5 % / 68.75 % cache reduction with 2- / 4-way sharing):
+ * every token's K row and V row ([n_kv_heads * head_dim] values) of a layer is stored as e4m3 codes (1 sign, 4
+ * exponent bits with bias 7, 3 mantissa bits, finite only, largest value 448) plus one fp32 scale,
+ *     scale = max(max|x|, 2^-64) / 448,   code = e4m3(x / scale)   (fp32, round to nearest even, saturating),
+ * and every attention read -- the prefill attention of layers <= l included -- sees value(code) * scale, so chunked
+ * and one-shot prefill stay identical.  A cache slot is then  K codes | V codes | K scales | V scales  (each part
+ * padded to 256 bytes); swiftkv_workspace_bytes and swiftkv_kv_cache_view account for it.
+ */
+#define SWIFTKV_KV_MODEL_DTYPE 0
+#define SWIFTKV_KV_FP8         1
 
 typedef struct {                               /* one decoder layer; all device pointers                */
   const void *in_norm;                         /* [hidden]                 gain of the input RMSNorm    */
@@ -166,13 +181,16 @@ int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const swiftkv_seq_
                      int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream);
 
 typedef struct {
-  const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype, AFTER RoPE            */
+  const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype (FP8 cache: uint8 e4m3
+                               codes), AFTER RoPE                                                           */
   const void *v;            /* device, same shape                                                           */
+  const float *k_scale;     /* FP8 cache: device fp32 [n_tokens], scale of every K row; else null          */
+  const float *v_scale;     /* FP8 cache: device fp32 [n_tokens], scale of every V row; else null          */
   int64_t token_stride;     /* elements between consecutive tokens (= n_kv_heads * head_dim)               */
   int64_t head_stride;      /* elements between consecutive KV heads (= head_dim)                          */
   int32_t n_tokens;         /* rows in use: the packed prompt tokens of the last prefill (prompt-major), or the
                                highest cache row written so far by swiftkv_step                            */
-  int32_t dtype;            /* SWIFTKV_DTYPE_*                                                              */
+  int32_t dtype;            /* SWIFTKV_DTYPE_* (SWIFTKV_DTYPE_FP8_E4M3 for the FP8 cache)                   */
   int32_t owner_layer;      /* 0-based layer whose projection produced this cache (the AcrossKV group's
                                first layer for layers >= l; the layer itself otherwise)                    */
 } swiftkv_kv_view;
@@ -267,6 +285,21 @@ int32_t swiftkv_tail_attention(const float *q, const void *k_cache, const void *
                                const int32_t *cu_seqlens, int32_t n_seqs, int32_t max_seq_len, int32_t n_q_heads,
                                int32_t n_kv_heads, int32_t head_dim, int32_t dtype, void *scratch, size_t scratch_bytes,
                                void *cuda_stream);
+
+/* The row pass that fills the FP8 cache (SWIFTKV_KV_FP8; appendix "KV quantization", per-token FP8), stand-alone:
+ * x DEVICE fp32 [rows, width]; codes DEVICE uint8 [rows, width]; scales DEVICE fp32 [rows];
+ * deq (nullable) DEVICE fp32 [rows, width] receives value(code) * scale.  Per row: scale = max(max|x|, 2^-64) / 448,
+ * code = e4m3(x / scale), each step one correctly rounded fp32 operation, round to nearest even, saturating --
+ * so codes and scales are bit-exact functions of x.  Errors: INVALID_ARG, CUDA. */
+int32_t swiftkv_quantize_rows_fp8(const float *x, int32_t rows, int32_t width, uint8_t *codes, float *scales,
+                                  float *deq, void *cuda_stream);
+
+/* swiftkv_tail_attention over an FP8 cache: k_codes, v_codes DEVICE uint8 [total_tokens, n_kv, hd], k_scale, v_scale
+ * DEVICE fp32 [total_tokens] (one scale per token row and plane); everything else as swiftkv_tail_attention. */
+int32_t swiftkv_tail_attention_fp8(const float *q, const uint8_t *k_codes, const uint8_t *v_codes, const float *k_scale,
+                                   const float *v_scale, float *out, const int32_t *cu_seqlens, int32_t n_seqs,
+                                   int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                   void *scratch, size_t scratch_bytes, void *cuda_stream);
 
 /* (No counterpart in the paper: an integration aid.)
  * swiftkv_tail_attention for callers that must not allocate device memory and have no spare buffer to lend --

@@ -7,13 +7,17 @@ from .binding import (  # noqa: F401
     ACT_BF16,
     ACT_F16,
     KC_NAMES,
+    KV_FP8,
+    KV_MODEL_DTYPE,
     SwiftKVError,
     SwiftKVModel,
     attention_prefill,
     gemm_tc,
     library_path,
     load_library,
+    quantize_rows_fp8,
     tail_attention,
+    tail_attention_fp8,
     tail_attention_noalloc,
     workspace_bytes,
 )

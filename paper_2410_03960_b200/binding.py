@@ -10,8 +10,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB: Optional[C.CDLL] = None
 
-DTYPE_F32, DTYPE_BF16, DTYPE_F16 = 0, 1, 2
+DTYPE_F32, DTYPE_BF16, DTYPE_F16, DTYPE_FP8_E4M3 = 0, 1, 2, 3
 ACT_BF16, ACT_F16 = 0, 1
+KV_MODEL_DTYPE, KV_FP8 = 0, 1
 _DTYPE_CODE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 KC_NAMES = ("gemm", "attention", "elementwise", "tail", "gemm_swiglu")
 
@@ -21,7 +22,7 @@ EXPORTS = (
     "swiftkv_prefill_device_tokens", "swiftkv_step", "swiftkv_kv_cache_view", "swiftkv_first_logits", "swiftkv_status",
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
     "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
-    "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc",
+    "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
 )
 
 
@@ -33,7 +34,7 @@ class SwiftKVError(RuntimeError):
 
 class _Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("vocab", "hidden", "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "ffn")] + \
-               [("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32)]
+               [("rope_theta", C.c_float), ("rms_eps", C.c_float), ("dtype", C.c_int32), ("kv_format", C.c_int32)]
 
 
 class _LayerWeights(C.Structure):
@@ -51,7 +52,8 @@ class _SeqStep(C.Structure):
 
 
 class _KVView(C.Structure):
-    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("token_stride", C.c_int64), ("head_stride", C.c_int64),
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
+                ("token_stride", C.c_int64), ("head_stride", C.c_int64),
                 ("n_tokens", C.c_int32), ("dtype", C.c_int32), ("owner_layer", C.c_int32)]
 
 
@@ -93,6 +95,8 @@ def load_library() -> C.CDLL:
     lib.swiftkv_tail_attention_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_tail_attention.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.swiftkv_tail_attention_noalloc.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p]
+    lib.swiftkv_quantize_rows_fp8.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.swiftkv_tail_attention_fp8.argtypes = [C.c_void_p] * 7 + [C.c_int32] * 5 + [C.c_void_p, C.c_size_t, C.c_void_p]
     _LIB = lib
     return lib
 
@@ -106,16 +110,16 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     return (stream or torch.cuda.current_stream()).cuda_stream
 
 
-def _make_config(shape, dtype: torch.dtype) -> _Config:
+def _make_config(shape, dtype: torch.dtype, kv_format: int = KV_MODEL_DTYPE) -> _Config:
     code = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[dtype]
     return _Config(shape.vocab, shape.hidden, shape.n_layers, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
-                   shape.ffn, float(shape.rope_theta), float(shape.rms_eps), code)
+                   shape.ffn, float(shape.rope_theta), float(shape.rms_eps), code, kv_format)
 
 
 def workspace_bytes(shape, dtype: torch.dtype, max_tokens: int, max_seqs: int, swift_layer: int,
-                    acrosskv_group: int) -> Tuple[int, int]:
+                    acrosskv_group: int, kv_format: int = KV_MODEL_DTYPE) -> Tuple[int, int]:
     """swiftkv_workspace_bytes -> (workspace_bytes, kv_cache_bytes)."""
-    cfg = _make_config(shape, dtype)
+    cfg = _make_config(shape, dtype, kv_format)
     ws, kv = C.c_size_t(0), C.c_size_t(0)
     _check(load_library().swiftkv_workspace_bytes(C.byref(cfg), max_tokens, max_seqs, swift_layer, acrosskv_group,
                                                   C.byref(ws), C.byref(kv)))
@@ -131,16 +135,17 @@ class SwiftKVModel:
     """
 
     def __init__(self, shape, weights, dtype: torch.dtype, max_tokens: int, max_seqs: int, swift_layer: int,
-                 acrosskv_group: int = 1, device: str = "cuda:0"):
+                 acrosskv_group: int = 1, device: str = "cuda:0", kv_format: int = KV_MODEL_DTYPE):
         self.lib = load_library()
         self.shape, self.dtype, self.device = shape, dtype, torch.device(device)
+        self.kv_format = kv_format
         self.max_tokens, self.max_seqs = max_tokens, max_seqs
         self._weights = weights           # keep the tensors alive: the library borrows their memory
-        ws_b, kv_b = workspace_bytes(shape, dtype, max_tokens, max_seqs, swift_layer, acrosskv_group)
+        ws_b, kv_b = workspace_bytes(shape, dtype, max_tokens, max_seqs, swift_layer, acrosskv_group, kv_format)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(ws_b, dtype=torch.uint8, device=self.device)
             self.kv_cache = torch.empty(kv_b, dtype=torch.uint8, device=self.device)
-            cfg = _make_config(shape, dtype)
+            cfg = _make_config(shape, dtype, kv_format)
             arr = (_LayerWeights * shape.n_layers)()
             for j, lw in enumerate(weights.layers):
                 for name, _ in _LayerWeights._fields_:
@@ -205,6 +210,7 @@ class SwiftKVModel:
         """swiftkv_kv_cache_view -> (K [n_tokens, n_kv, hd], V, owner_layer) as views into the cache tensor."""
         v = _KVView()
         _check(self.lib.swiftkv_kv_cache_view(self._h, layer, C.byref(v)))
+        assert v.dtype != DTYPE_FP8_E4M3, "FP8 cache: use kv_cache_view_fp8"
         flat = self.kv_cache.view(self.dtype)
         es = flat.element_size()
         n = v.n_tokens * v.token_stride
@@ -212,6 +218,24 @@ class SwiftKVModel:
         ko = (v.k - self.kv_cache.data_ptr()) // es
         vo = (v.v - self.kv_cache.data_ptr()) // es
         return flat[ko:ko + n].view(shape), flat[vo:vo + n].view(shape), v.owner_layer
+
+    def kv_cache_view_fp8(self, layer: int):
+        """swiftkv_kv_cache_view of an FP8 cache -> (K codes uint8 [n_tokens, n_kv, hd], V codes, K scales fp32
+        [n_tokens], V scales, owner_layer) as views into the cache tensor."""
+        v = _KVView()
+        _check(self.lib.swiftkv_kv_cache_view(self._h, layer, C.byref(v)))
+        assert v.dtype == DTYPE_FP8_E4M3
+        base = self.kv_cache.data_ptr()
+        n = v.n_tokens * v.token_stride
+        shape = (v.n_tokens, self.shape.n_kv_heads, self.shape.head_dim)
+
+        def codes(ptr):
+            return self.kv_cache[ptr - base: ptr - base + n].view(shape)
+
+        def scales(ptr):
+            return self.kv_cache[ptr - base: ptr - base + 4 * v.n_tokens].view(torch.float32)
+
+        return codes(v.k), codes(v.v), scales(v.k_scale), scales(v.v_scale), v.owner_layer
 
     def first_logits(self) -> torch.Tensor:
         """swiftkv_first_logits -> fp32 [n_seqs, vocab] view into the workspace."""
@@ -318,3 +342,36 @@ def tail_attention_noalloc(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torc
         _check(load_library().swiftkv_tail_attention_noalloc(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
                                                              out.data_ptr(), cu_seqlens.data_ptr(), b, max_seq_len, n_q, n_kv,
                                                              hd, code, _stream_ptr(stream)))
+
+
+def quantize_rows_fp8(x: torch.Tensor, want_deq: bool = True, stream: Optional[torch.cuda.Stream] = None):
+    """swiftkv_quantize_rows_fp8: x fp32 [rows, width] -> (codes uint8 [rows, width], scales fp32 [rows], deq fp32 or None)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.dim() == 2
+    rows, width = x.shape
+    codes = torch.empty((rows, width), dtype=torch.uint8, device=x.device)
+    scales = torch.empty(rows, dtype=torch.float32, device=x.device)
+    deq = torch.empty_like(x) if want_deq else None
+    with torch.cuda.device(x.device):
+        _check(load_library().swiftkv_quantize_rows_fp8(x.data_ptr(), rows, width, codes.data_ptr(), scales.data_ptr(),
+                                                        deq.data_ptr() if want_deq else None, _stream_ptr(stream)))
+    return codes, scales, deq
+
+
+def tail_attention_fp8(q: torch.Tensor, k_codes: torch.Tensor, v_codes: torch.Tensor, k_scale: torch.Tensor,
+                       v_scale: torch.Tensor, seq_lens: Sequence[int], stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_tail_attention_fp8: q fp32 [n_seqs, n_q, hd]; codes uint8 [T, n_kv, hd]; scales fp32 [T] -> fp32 [n_seqs, n_q*hd]."""
+    assert q.is_cuda and q.dtype == torch.float32 and q.is_contiguous()
+    assert k_codes.dtype == torch.uint8 and v_codes.dtype == torch.uint8 and k_codes.is_contiguous() and v_codes.is_contiguous()
+    assert k_scale.dtype == torch.float32 and v_scale.dtype == torch.float32
+    b, n_q, hd = q.shape
+    n_kv = k_codes.shape[1]
+    lib = load_library()
+    cu = _cu_seqlens(seq_lens, q.device)
+    nbytes = lib.swiftkv_tail_attention_scratch_bytes(b, n_q, hd, max(seq_lens))
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    out = torch.empty((b, n_q * hd), dtype=torch.float32, device=q.device)
+    with torch.cuda.device(q.device):
+        _check(lib.swiftkv_tail_attention_fp8(q.data_ptr(), k_codes.data_ptr(), v_codes.data_ptr(), k_scale.data_ptr(),
+                                              v_scale.data_ptr(), out.data_ptr(), cu.data_ptr(), b, max(seq_lens), n_q, n_kv, hd,
+                                              scratch.data_ptr(), nbytes, _stream_ptr(stream)))
+    return out

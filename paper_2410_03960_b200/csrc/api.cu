@@ -62,6 +62,9 @@ struct Buffers {
   void *wfold;              // folded, concatenated SingleInputKV weight [n_groups*2*d_kv, d]
   void *w16;                // bf16 models: IEEE-half compute copy of ONE layer's seven matrices (refilled per layer)
   void *kv16;               // bf16 models: half copies of the current layer's K and V, [2][T, d_kv]
+  void *kvst;               // FP8 cache: the projections' K / V rows of one layer before quantization, [2][T, d_kv] model dtype
+  void *kvdq;               // FP8 cache: dequantized K / V of one layer for the attention kernels (fp32 models; 16-bit
+                            //   models use kv16)
   float *y;                 // continuing tokens' residual [B, d]
   float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
   float *tail_scratch;
@@ -117,6 +120,7 @@ static int32_t check_cfg(const swiftkv_config *c, int max_tokens, int max_seqs, 
   if (c->n_q_heads % c->n_kv_heads) return fail(SWIFTKV_ERR_INVALID_ARG, "n_q_heads must be a multiple of n_kv_heads");
   if (c->head_dim % 2 || c->head_dim > 256) return fail(SWIFTKV_ERR_INVALID_ARG, "head_dim must be even and <= 256");
   if (c->dtype != SWIFTKV_DTYPE_F32 && c->dtype != SWIFTKV_DTYPE_BF16) return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+  if (c->kv_format != SWIFTKV_KV_MODEL_DTYPE && c->kv_format != SWIFTKV_KV_FP8) return fail(SWIFTKV_ERR_INVALID_ARG, "unknown kv_format");
   if (!(c->rope_theta > 0.f) || !(c->rms_eps >= 0.f)) return fail(SWIFTKV_ERR_INVALID_ARG, "bad rope_theta / rms_eps");
   if (max_tokens < 1 || max_seqs < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "max_tokens and max_seqs must be positive");
   if (l < 1 || l > c->n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c->n_layers);
@@ -140,6 +144,9 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   const bool bf = c.dtype == SWIFTKV_DTYPE_BF16;
   b.w16 = cv.take(bf ? 2 * (2 * d * dq + 2 * d * dkv_ + 3 * d * F) * 2 : 0);   // two layers: double buffer
   b.kv16 = cv.take(bf ? (size_t)2 * T * dkv_ * 2 : 0);
+  const bool fp8 = c.kv_format == SWIFTKV_KV_FP8;
+  b.kvst = cv.take(fp8 ? (size_t)2 * T * dkv_ * E : 0);
+  b.kvdq = cv.take(fp8 && !bf ? (size_t)2 * T * dkv_ * 4 : 0);
   b.y = (float *)cv.take((size_t)B * d * 4);
   const size_t R = std::min<size_t>(B, MAX_TAIL_ROWS);
   b.hy = (float *)cv.take(R * std::max(d, dq) * 4);
@@ -171,6 +178,13 @@ static size_t fold_elems_for(const swiftkv_config &c, int l, int g) {
   return (size_t)n_groups(c.n_layers, l, g) * 2 * c.n_kv_heads * c.head_dim * c.hidden;
 }
 static size_t slot_elems(const swiftkv_config &c, int T) { return (size_t)2 * T * c.n_kv_heads * c.head_dim; }
+// FP8 cache slot: K codes | V codes | K scales | V scales, every part padded to 256 bytes
+static size_t fp8_code_plane(const swiftkv_config &c, int T) { return ((size_t)T * c.n_kv_heads * c.head_dim + 255) & ~(size_t)255; }
+static size_t fp8_scale_plane(int T) { return ((size_t)T * 4 + 255) & ~(size_t)255; }
+static size_t slot_bytes_of(const swiftkv_config &c, int T) {
+  if (c.kv_format == SWIFTKV_KV_FP8) return 2 * fp8_code_plane(c, T) + 2 * fp8_scale_plane(T);
+  return slot_elems(c, T) * dsize(c.dtype);
+}
 
 // ---------------------------------------------------------------------------------------------------------
 extern "C" int32_t swiftkv_version(void) { return 100; }
@@ -187,7 +201,7 @@ extern "C" int32_t swiftkv_workspace_bytes(const swiftkv_config *cfg, int32_t ma
   carve_all(*cfg, max_tokens, max_seqs, fold_elems_for(*cfg, swift_layer, acrosskv_group), cv, b);
   *workspace_bytes = ((cv.off + 255) & ~(size_t)255) + 512;
   const int slots = swift_layer + n_groups(cfg->n_layers, swift_layer, acrosskv_group);
-  *kv_cache_bytes = (size_t)slots * slot_elems(*cfg, max_tokens) * dsize(cfg->dtype);
+  *kv_cache_bytes = (size_t)slots * slot_bytes_of(*cfg, max_tokens);
   return SWIFTKV_OK;
 }
 
@@ -219,7 +233,7 @@ extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_w
   const size_t base_need = (measure.off + 255) & ~(size_t)255;
   if (workspace_bytes < base_need) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "workspace %zu < %zu bytes", workspace_bytes, base_need);
   const size_t E = dsize(cfg->dtype);
-  const size_t slot_bytes = slot_elems(*cfg, max_tokens) * E;
+  const size_t slot_bytes = slot_bytes_of(*cfg, max_tokens);
   if (kv_cache_bytes < slot_bytes) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "kv cache smaller than one slot");
 
   swiftkv_model *m = new (std::nothrow) swiftkv_model();
@@ -352,6 +366,15 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const size_t plane = (size_t)m->max_tokens * dkv;          // elements of one K (or V) plane
   constexpr bool act_f16 = std::is_same<TA, __half>::value;
   T *kv = reinterpret_cast<T *>(m->kv);
+  // FP8 cache (appendix, KV quantization): projections land in a staging pair of planes, a row pass turns them into
+  // codes + per-token scales in the cache, and every attention read sees the dequantized values
+  const bool fp8 = c.kv_format == SWIFTKV_KV_FP8;
+  const size_t slot_b = slot_bytes_of(c, m->max_tokens), cp8 = fp8_code_plane(c, m->max_tokens), sp8 = fp8_scale_plane(m->max_tokens);
+  auto k_codes = [&](int slot) { return m->kv + (size_t)slot * slot_b; };
+  auto v_codes = [&](int slot) { return m->kv + (size_t)slot * slot_b + cp8; };
+  auto k_scale = [&](int slot) { return reinterpret_cast<float *>(m->kv + (size_t)slot * slot_b + 2 * cp8); };
+  auto v_scale = [&](int slot) { return reinterpret_cast<float *>(m->kv + (size_t)slot * slot_b + 2 * cp8 + sp8); };
+  T *kst = (T *)b.kvst, *vst = kst + plane;
   TA *h = (TA *)b.h, *q = (TA *)b.q, *attn = (TA *)b.attn, *act = (TA *)b.act;
   const T *no_w = nullptr;
   int32_t rc;
@@ -437,19 +460,57 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     }
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
     OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv, slot_map};
+    if (fp8) { Kj = kst; Vj = vst; qkv.seg_base = kst; qkv.slot_map = nullptr; }   // staging rows are in batch order
     bool roped = false;
     // the attention kernel reads half copies of this layer's K / V: written by the QKV epilogue for a plain prefill,
     // gathered from the cache (cached prefix + new tokens) otherwise
-    const bool want_dup = use_w16 && attn_tc && bt.plain;
+    const bool want_dup = use_w16 && attn_tc && bt.plain && !fp8;
     rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st,
                          use_w16 ? wq16 : nullptr, use_w16 ? wk16 : nullptr, use_w16 ? wv16 : nullptr, &rope, &roped,
                          want_dup ? k16 : nullptr, (long long)plane);
     if (rc) return rc;
     if (!roped) {
       { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, fp8 ? nullptr : slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
     }
-    {
+    if (fp8) {
+      // quantize this layer's rows into the cache; the attention operands are the dequantized values: written by the same
+      // pass for a whole-prompt prefill, gathered from the cache (cached prefix + new rows) otherwise
+      using TD = typename std::conditional<sizeof(T) == 2, TA, float>::type;   // operand type of the attention kernels
+      const bool tc_path = sizeof(T) == 2 && attn_tc;
+      TD *kd = sizeof(T) == 2 ? (TD *)b.kv16 : (TD *)b.kvdq, *vd = kd + plane;
+      T *kd_t = (T *)kd, *vd_t = kd_t + plane;   // (SIMT attention reads operands of the cache's element type)
+      {
+        Scope s(m, st, SWIFTKV_KC_ELEMWISE, 2);
+        if (tc_path) {
+          launch_quantize_rows_fp8<T, TD>(kst, T_tok, dkv, slot_map, k_codes(j), k_scale(j), bt.plain ? kd : nullptr, st);
+          launch_quantize_rows_fp8<T, TD>(vst, T_tok, dkv, slot_map, v_codes(j), v_scale(j), bt.plain ? vd : nullptr, st);
+        } else {
+          launch_quantize_rows_fp8<T, T>(kst, T_tok, dkv, slot_map, k_codes(j), k_scale(j), bt.plain ? kd_t : nullptr, st);
+          launch_quantize_rows_fp8<T, T>(vst, T_tok, dkv, slot_map, v_codes(j), v_scale(j), bt.plain ? vd_t : nullptr, st);
+        }
+      }
+      if (!bt.plain) {
+        Scope s(m, st, SWIFTKV_KC_ELEMWISE);
+        if (tc_path) launch_gather_dequant_fp8<TD>(k_codes(j), v_codes(j), k_scale(j), v_scale(j), kd, vd, b.kv_row0, b.kv_len, b.kcu, blk, bt.blk_stride, B, bt.max_kv, dkv, st);
+        else launch_gather_dequant_fp8<T>(k_codes(j), v_codes(j), k_scale(j), v_scale(j), kd_t, vd_t, b.kv_row0, b.kv_len, b.kcu, blk, bt.blk_stride, B, bt.max_kv, dkv, st);
+      }
+      Scope s(m, st, SWIFTKV_KC_ATTENTION);
+      const int32_t *kr0 = bt.plain ? nullptr : b.kcu;
+      bool done = false;
+      if constexpr (sizeof(T) == 2) {
+        if (tc_path) {
+          rc = launch_attention_tc(q, act_f16, kd, vd, attn, b.cu, kr0, kv_len, nullptr, 0, B, T_tok, bt.plain ? T_tok : bt.total_kv,
+                                   bt.max_new, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
+          if (rc == SWIFTKV_OK) done = true;
+          else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
+        }
+      }
+      if (!done) {
+        if (tc_path) return fail(SWIFTKV_ERR_UNSUPPORTED, "FP8 cache: tensor-core attention refused this shape");
+        launch_attention_simple<TA, T>(q, kd_t, vd_t, attn, b.cu, B, kr0, kv_len, nullptr, 0, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
+      }
+    } else {
       Scope s(m, st, SWIFTKV_KC_ATTENTION);
       bool done = false;
       if constexpr (sizeof(T) == 2) {
@@ -513,6 +574,23 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
   if (l < L) {
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
+    if (fp8) {
+      // one group at a time through the staging planes: projection (+ RoPE on K), then the quantizing row pass into the
+      // group's cache slot
+      for (int i = 0; i < ng; ++i) {
+        const size_t woff = (size_t)i * 2 * dkv * d;
+        OutDesc o{OUT_STORE, nullptr, 0, 0, kst, (long long)plane, dkv, nullptr};
+        bool roped = false;
+        rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)b.wfold + woff, 2 * dkv, no_w, 0, no_w, 0, o, st,
+                             use_w16 ? (const __half *)b.wfold + woff : nullptr, nullptr, nullptr, &rope, &roped);
+        if (rc) return rc;
+        if (use_w16 && !roped) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-folded SingleInputKV weight needs the tensor-core GEMM");
+        if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(kst, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+        Scope s(m, st, SWIFTKV_KC_ELEMWISE, 2);
+        launch_quantize_rows_fp8<T, T>(kst, T_tok, dkv, slot_map, k_codes(l + i), k_scale(l + i), (T *)nullptr, st);
+        launch_quantize_rows_fp8<T, T>(vst, T_tok, dkv, slot_map, v_codes(l + i), v_scale(l + i), (T *)nullptr, st);
+      }
+    } else {
     T *slot_l = kv + (size_t)l * 2 * plane;
     OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv, slot_map};
     bool roped = false;
@@ -521,6 +599,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     if (rc) return rc;
     if (use_w16 && !roped) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-folded SingleInputKV weight needs the tensor-core GEMM");
     if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
+    }
   }
 
   // ---- the tokens that must produce output -- the last token of a prompt (footnote of Sec. 3.2), decode tokens
@@ -537,7 +616,17 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL, 2); launch_tail_attention<T>(qy, Ks, Vs, ay, b.emit_row0 + r0, b.emit_len + r0, blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st); }
+      {
+        Scope s(m, st, SWIFTKV_KC_TAIL, 2);
+        const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
+        if (fp8)
+          launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(slot), (const fp8e4 *)v_codes(slot), k_scale(slot), v_scale(slot), ay,
+                                       b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads,
+                                       c.n_kv_heads, c.head_dim, b.tail_scratch, st);
+        else
+          launch_tail_attention<T>(qy, Ks, Vs, nullptr, nullptr, ay, b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len,
+                                   c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st);
+      }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
@@ -713,13 +802,22 @@ extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, 
   const size_t plane = (size_t)m->max_tokens * dkv;
   int slot = layer, owner = layer;
   if (layer >= l) { slot = l + (layer - l) / g; owner = l + ((layer - l) / g) * g; }
-  const uint8_t *kp = m->kv + (size_t)slot * 2 * plane * m->esize;
+  const uint8_t *kp = m->kv + (size_t)slot * slot_bytes_of(m->cfg, m->max_tokens);
   out->k = kp;
-  out->v = kp + plane * m->esize;
+  out->k_scale = out->v_scale = nullptr;
+  if (m->cfg.kv_format == SWIFTKV_KV_FP8) {
+    const size_t cp = fp8_code_plane(m->cfg, m->max_tokens), sp = fp8_scale_plane(m->max_tokens);
+    out->v = kp + cp;
+    out->k_scale = reinterpret_cast<const float *>(kp + 2 * cp);
+    out->v_scale = reinterpret_cast<const float *>(kp + 2 * cp + sp);
+    out->dtype = SWIFTKV_DTYPE_FP8_E4M3;
+  } else {
+    out->v = kp + plane * m->esize;
+    out->dtype = m->cfg.dtype;
+  }
   out->token_stride = dkv;
   out->head_stride = m->cfg.head_dim;
   out->n_tokens = m->n_tokens;
-  out->dtype = m->cfg.dtype;
   out->owner_layer = owner;
   return SWIFTKV_OK;
 }
@@ -861,13 +959,42 @@ extern "C" int32_t swiftkv_tail_attention(const float *q, const void *k_cache, c
                 tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len));
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   if (dtype == SWIFTKV_DTYPE_BF16)
-    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len, n_q_heads,
+    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, nullptr, nullptr, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len, n_q_heads,
                                 n_kv_heads, head_dim, (float *)scratch, st);
   else if (dtype == SWIFTKV_DTYPE_F32)
-    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len,
+    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, nullptr, nullptr, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len,
                                  n_q_heads, n_kv_heads, head_dim, (float *)scratch, st);
   else
     return fail(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_quantize_rows_fp8(const float *x, int32_t rows, int32_t width, uint8_t *codes, float *scales,
+                                             float *deq, void *cuda_stream) {
+  if (!x || !codes || !scales) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (rows < 1 || width < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "rows and width must be positive");
+  launch_quantize_rows_fp8<float, float>(x, rows, width, nullptr, codes, scales, deq, reinterpret_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_tail_attention_fp8(const float *q, const uint8_t *k_codes, const uint8_t *v_codes, const float *k_scale,
+                                              const float *v_scale, float *out, const int32_t *cu_seqlens, int32_t n_seqs,
+                                              int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                              void *scratch, size_t scratch_bytes, void *cuda_stream) {
+  if (!q || !k_codes || !v_codes || !k_scale || !v_scale || !out || !cu_seqlens || !scratch) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (n_seqs < 1 || n_seqs > MAX_TAIL_ROWS || max_seq_len < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
+      head_dim < 4 || head_dim > 256 || head_dim % 4)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "bad shape (n_seqs must be in [1, %d], head_dim a multiple of 4)", MAX_TAIL_ROWS);
+  if (scratch_bytes < tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len))
+    return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "scratch %zu < %zu bytes", scratch_bytes,
+                tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len));
+  launch_tail_attention<fp8e4>(q, (const fp8e4 *)k_codes, (const fp8e4 *)v_codes, k_scale, v_scale, out, cu_seqlens, nullptr, nullptr, 0,
+                               n_seqs, max_seq_len, n_q_heads, n_kv_heads, head_dim, (float *)scratch,
+                               reinterpret_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
   return SWIFTKV_OK;

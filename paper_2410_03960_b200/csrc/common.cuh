@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -27,6 +28,15 @@ template <> __device__ __forceinline__ float to_f<__half>(__half v) { return __h
 template <> __device__ __forceinline__ __half from_f<__half>(float v) {
   return __float2half_rn(fminf(fmaxf(v, -65504.f), 65504.f));
 }
+
+// one stored element of the FP8 cache (e4m3: 4 exponent bits, bias 7, 3 mantissa bits, finite only); its value is the
+// decoded number times the fp32 scale of its token row (appendix "KV quantization": per-token FP8 quantization)
+struct fp8e4 { uint8_t x; };
+template <> __device__ __forceinline__ float to_f<fp8e4>(fp8e4 v) {
+  return __half2float(__half(__nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)v.x, __NV_E4M3)));
+}
+constexpr float FP8_MAX = 448.f;
+constexpr float FP8_AMAX_FLOOR = 5.421010862427522e-20f;   // 2^-64: an all-zero row still gets a normal scale
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -107,6 +117,18 @@ void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *pos
 void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
                            const int32_t *kcu, const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv,
                            cudaStream_t st);
+// kv_fp8.cu : per-token FP8 cache rows.  One scale per row of `width` elements: scale = max(amax, 2^-64) / 448,
+// code = e4m3(x / scale) (correctly rounded fp32 divisions, round to nearest even, saturating).  Row r of `src` goes to row
+// slot_map[r] (null: r) of `codes` / `scale`; deq (nullable, row r) receives value(code) * scale in type TO.
+template <typename TI, typename TO>
+void launch_quantize_rows_fp8(const TI *src, int rows, int width, const int32_t *slot_map, uint8_t *codes, float *scale,
+                              TO *deq, cudaStream_t st);
+// dequantized, packed copies of each sequence's cache rows (K and V planes of one slot): sequence b's key p goes to row
+// kcu[b] + p of k_out / v_out.  Row addressing as in launch_gather_kv_half.
+template <typename TO>
+void launch_gather_dequant_fp8(const uint8_t *k_codes, const uint8_t *v_codes, const float *k_scale, const float *v_scale,
+                               TO *k_out, TO *v_out, const int32_t *row0, const int32_t *len, const int32_t *kcu,
+                               const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv, cudaStream_t st);
 template <typename T>
 void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
@@ -175,9 +197,10 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
 // one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
 // row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
+// T = fp8e4: kc / vc hold FP8 codes and kscale / vscale the fp32 scale of every cache row (null for other types)
 template <typename T>
-void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *row0, const int32_t *len,
-                           const int32_t *blk, int blk_stride, int n_seqs, int max_seq_len, int n_q, int n_kv, int hd,
-                           float *scratch, cudaStream_t st);
+void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
+                           const int32_t *row0, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
 
 }  // namespace skv

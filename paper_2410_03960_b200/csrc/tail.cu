@@ -273,9 +273,10 @@ __device__ __forceinline__ float dot_row(const float *__restrict__ qs, const T *
 constexpr int TA_WARPS = 4;
 template <typename T, int REP, int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
-    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    const int32_t *__restrict__ len, const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk,
-    int n_splits, float scale, float *__restrict__ scratch) {
+    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
+    const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
+    const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk, int n_splits, float scale,
+    float *__restrict__ scratch) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
   __shared__ float qs[REP][HD];
   __shared__ float w_m[TA_WARPS][REP], w_l[TA_WARPS][REP];
@@ -298,8 +299,10 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     float sc[REP];
 #pragma unroll
     for (int r = 0; r < REP; ++r) sc[r] = 0.f;
+    float v_s = 1.f;     // FP8 cache: this lane's key carries one scale for its K row and one for its V row
     if (valid) {
-      const T *kr = kc + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * HD;
+      const size_t krow = kv_row_of(blk, blk_stride, b, first, key);
+      const T *kr = kc + (krow * n_kv + kvh) * HD;
       constexpr int V = 16 / sizeof(T);
 #pragma unroll 4
       for (int i = 0; i < HD; i += V) {
@@ -312,6 +315,12 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
           for (int r = 0; r < REP; ++r) sc[r] = fmaf(qs[r][i + k], kv_, sc[r]);
         }
       }
+      if (kscale) {
+        const float k_s = kscale[krow];
+        v_s = vscale[krow];
+#pragma unroll
+        for (int r = 0; r < REP; ++r) sc[r] *= k_s;
+      }
     }
     float pe[REP];
 #pragma unroll
@@ -323,6 +332,7 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
       l[r] = l[r] * corr + warp_sum(pe[r]);
       acc[r][0] *= corr; acc[r][1] *= corr; acc[r][2] *= corr; acc[r][3] *= corr;
       m[r] = m_new;
+      pe[r] *= v_s;        // (after the row sum: the V row's scale rides on the probability)
     }
     const int n_here = min(32, k_end - c0);
     // (a 32-key chunk never straddles a 128-row page: c0 is a multiple of 32)
@@ -333,6 +343,10 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
       float v0, v1, v2, v3;
       if constexpr (sizeof(T) == 2) {
         const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
+        const T *e = reinterpret_cast<const T *>(&raw);
+        v0 = to_f(e[0]); v1 = to_f(e[1]); v2 = to_f(e[2]); v3 = to_f(e[3]);
+      } else if constexpr (sizeof(T) == 1) {
+        const uint32_t raw = *reinterpret_cast<const uint32_t *>(vr);
         const T *e = reinterpret_cast<const T *>(&raw);
         v0 = to_f(e[0]); v1 = to_f(e[1]); v2 = to_f(e[2]); v3 = to_f(e[3]);
       } else {
@@ -375,9 +389,10 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
 // K / V rows of the block's key range come from HBM once and are shared by the group's heads through L1.
 template <typename T, int MAX_E>
 __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
-    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const int32_t *__restrict__ cu,
-    const int32_t *__restrict__ len, const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int hd, int chunk,
-    int n_splits, float scale, float *__restrict__ scratch) {
+    const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
+    const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
+    const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int hd, int chunk, int n_splits, float scale,
+    float *__restrict__ scratch) {
   extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -396,12 +411,17 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     for (int e = 0; e < MAX_E; ++e) acc[e] = 0.f;
     for (int c0 = k_begin; c0 < k_end; c0 += 32) {
       const int key = c0 + lane;
-      float s = -INFINITY;
-      if (key < k_end) s = dot_row<T>(qs, kc + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * hd, hd);
+      float s = -INFINITY, v_s = 1.f;
+      if (key < k_end) {
+        const size_t krow = kv_row_of(blk, blk_stride, b, first, key);
+        s = dot_row<T>(qs, kc + (krow * n_kv + kvh) * hd, hd);
+        if (kscale) { s *= kscale[krow]; v_s = vscale[krow]; }
+      }
       const float m_new = fmaxf(m, warp_max(s));
-      const float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
+      float pe = (key < k_end) ? __expf(s - m_new) : 0.f;
       const float corr = __expf(m - m_new);
       l = l * corr + warp_sum(pe);
+      pe *= v_s;
 #pragma unroll
       for (int e = 0; e < MAX_E; ++e) acc[e] *= corr;
       m = m_new;
@@ -455,9 +475,9 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 }
 
 template <typename T>
-void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out, const int32_t *cu_seqlens,
-                           const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs, int max_seq_len, int n_q,
-                           int n_kv, int hd, float *scratch, cudaStream_t st) {
+void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
+                           const int32_t *cu_seqlens, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st) {
   if (n_seqs <= 0) return;
   const int chunk = tail_chunk(max_seq_len);
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
@@ -465,25 +485,30 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, float *out,
   const int rep = n_q / n_kv;
   if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
     dim3 grid(n_splits, n_kv, n_seqs);
-    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
     tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
     return;
   }
   const int threads = 32 * (rep < 8 ? rep : 8);
   const size_t smem = (size_t)rep * hd * sizeof(float);
   dim3 grid(n_splits, n_kv, n_seqs);
-  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
   tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
-template void launch_tail_attention<float>(const float *, const float *, const float *, float *, const int32_t *,
-                                           const int32_t *, const int32_t *, int, int, int, int, int, int, float *, cudaStream_t);
-template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, float *, const int32_t *,
-                                          const int32_t *, const int32_t *, int, int, int, int, int, int, float *, cudaStream_t);
+template void launch_tail_attention<float>(const float *, const float *, const float *, const float *, const float *, float *,
+                                           const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
+                                           float *, cudaStream_t);
+template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, const float *, const float *, float *,
+                                          const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
+                                          float *, cudaStream_t);
+template void launch_tail_attention<fp8e4>(const float *, const fp8e4 *, const fp8e4 *, const float *, const float *, float *,
+                                           const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
+                                           float *, cudaStream_t);
 
 }  // namespace skv

@@ -56,10 +56,10 @@ extern "C" int32_t swiftkv_tail_attention_noalloc(const float *q, const void *k_
   // every (prompt, head, split) entry that the merge pass reads is written by the partial pass of this same call,
   // so stale contents from an earlier call are never observed
   if (dtype == SWIFTKV_DTYPE_BF16)
-    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len, n_q_heads,
+    launch_tail_attention<bf16>(q, (const bf16 *)k_cache, (const bf16 *)v_cache, nullptr, nullptr, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len, n_q_heads,
                                 n_kv_heads, head_dim, scratch, st);
   else
-    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len,
+    launch_tail_attention<float>(q, (const float *)k_cache, (const float *)v_cache, nullptr, nullptr, out, cu_seqlens, nullptr, nullptr, 0, n_seqs, max_seq_len,
                                  n_q_heads, n_kv_heads, head_dim, scratch, st);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return report_error(SWIFTKV_ERR_CUDA, cudaGetErrorString(e));
