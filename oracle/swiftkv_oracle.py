@@ -195,11 +195,24 @@ def e4m3_encode(y: np.ndarray) -> np.ndarray:
     return (code | sign).astype(np.uint8)
 
 
-def quantize_per_token(x: np.ndarray):
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """fp32 values rounded to the nearest bfloat16 (8 significand bits; ties to even), returned as fp32."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).reshape(np.shape(x))
+
+
+def quantize_per_token(x: np.ndarray, row_dtype: str = "f32"):
     """x [n_rows, ...]: one scale per row (token).  scale = max(amax, 2^-64) / 448, code = e4m3(x / scale), every
     operation on fp32 values with one correctly rounded fp32 result (what `/` on numpy float32 arrays does).
+    row_dtype: the type in which the rows exist before they are quantized -- "bf16" for a bf16 model (its K / V rows
+    are bf16 values, so that is the precision the code decision is taken in), "f32" otherwise.
     Returns (codes uint8 like x, scale float32 [n_rows], dequantized float64 like x = value(code) * scale)."""
     x32 = np.asarray(x, dtype=np.float32)
+    if row_dtype == "bf16":
+        x32 = round_to_bf16(x32)
+    else:
+        assert row_dtype == "f32"
     flat = x32.reshape(x32.shape[0], -1)
     amax = np.maximum(np.max(np.abs(flat), axis=1), np.float32(AMAX_FLOOR)).astype(np.float32)
     scale = (amax / np.float32(E4M3_MAX)).astype(np.float32)
@@ -209,7 +222,8 @@ def quantize_per_token(x: np.ndarray):
     return codes.reshape(x32.shape), scale, deq.reshape(x32.shape)
 
 
-def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.ndarray, kv_fp8: bool = False):
+def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.ndarray, kv_fp8: bool = False,
+                  row_dtype: str = "f32"):
     """One unmodified decoder layer on all rows of one prompt.  Returns (X_out, K, V) with K after RoPE.
     kv_fp8: K (after RoPE) and V go through the cache's per-token FP8 representation before anyone attends to them."""
     n = X.shape[0]
@@ -220,7 +234,7 @@ def decoder_layer(cfg: Config, w: Dict[str, np.ndarray], X: np.ndarray, pos: np.
     q = rope(q, pos, cfg.rope_theta)
     k = rope(k, pos, cfg.rope_theta)
     if kv_fp8:
-        k, v = quantize_per_token(k)[2], quantize_per_token(v)[2]
+        k, v = quantize_per_token(k, row_dtype)[2], quantize_per_token(v, row_dtype)[2]
     a = causal_attention(q, k, v)
     X = X + a @ w["wo"].T
     m = rmsnorm(X, w["post_norm"], cfg.rms_eps)
@@ -262,13 +276,13 @@ def group_leader(l: int, g: int, j: int) -> int:
 
 
 def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int], l: int, g: int = 1,
-            kv_fp8: bool = False):
+            kv_fp8: bool = False, row_dtype: str = "f32"):
     """SwiftKV prefill.  Layers 1..l as in the unmodified model; s = x_{l+1}; for every later layer j the
     cache is  K_j = rope(rmsnorm(s, gamma_in[r]) @ W_K[r].T),  V_j = rmsnorm(s, gamma_in[r]) @ W_V[r].T
     with r the leader of j's AcrossKV group (Eq. 2, Sec. 3.3); only the last token of each prompt runs
     layers l+1..L (footnote in Sec. 3.2; Sec. 3.5), attending to those caches.
     kv_fp8: every cache row is stored as per-token FP8 codes + scale; "K", "V" are then the dequantized values and
-    "K_codes", "K_scale", "V_codes", "V_scale" the stored representation."""
+    "K_codes", "K_scale", "V_codes", "V_scale" the stored representation; row_dtype as in quantize_per_token."""
     L = cfg.n_layers
     assert 1 <= l <= L and g >= 1
     tokens = np.asarray(tokens, dtype=np.int64)
@@ -287,7 +301,7 @@ def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]
         Xn = np.empty_like(X)
         for b in range(B):
             a, e = off[b], off[b + 1]
-            Xn[a:e], Kj[a:e], Vj[a:e] = decoder_layer(cfg, w, X[a:e], pos[a:e], kv_fp8)
+            Xn[a:e], Kj[a:e], Vj[a:e] = decoder_layer(cfg, w, X[a:e], pos[a:e], kv_fp8, row_dtype)
         X, K[j], V[j] = Xn, Kj, Vj
     s = X                                                      # x_{l+1}
 
@@ -300,7 +314,7 @@ def swiftkv(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]
             K[j1 - 1] = rope(k, pos, cfg.rope_theta)
             V[j1 - 1] = (h @ w["wv"].T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
             if kv_fp8:
-                K[j1 - 1], V[j1 - 1] = quantize_per_token(K[j1 - 1])[2], quantize_per_token(V[j1 - 1])[2]
+                K[j1 - 1], V[j1 - 1] = quantize_per_token(K[j1 - 1], row_dtype)[2], quantize_per_token(V[j1 - 1], row_dtype)[2]
         else:
             K[j1 - 1] = K[r1 - 1]                              # alias: one cache per group
             V[j1 - 1] = V[r1 - 1]

@@ -44,6 +44,54 @@ __global__ void __launch_bounds__(QT) quantize_rows_kernel(const TI *__restrict_
   }
 }
 
+// 16-bit rows whose width is a multiple of 8 and at most 32 * 8 * VEC_CHUNKS: one warp per row, every lane keeps its
+// elements in registers between the maximum and the conversion (128-bit loads, 64-bit code stores, no block barrier)
+constexpr int VEC_CHUNKS = 8;
+constexpr int VEC_ROWS = 8;      // rows (warps) per block
+template <typename TO, int CHUNKS>
+__global__ void __launch_bounds__(VEC_ROWS * 32) quantize_rows_vec_kernel(const bf16 *__restrict__ src, int rows, int width,
+                                                                         const int32_t *__restrict__ slot_map,
+                                                                         uint8_t *__restrict__ codes, float *__restrict__ scale_out,
+                                                                         TO *__restrict__ deq) {
+  const int r = blockIdx.x * VEC_ROWS + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= rows) return;
+  const uint4 *x = reinterpret_cast<const uint4 *>(src + (size_t)r * width);
+  const int n_vec = width >> 3;
+  uint4 raw[CHUNKS];
+  float amax = 0.f;
+#pragma unroll
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int i = lane + c * 32;
+    if (i < n_vec) {
+      raw[c] = __ldcs(x + i);
+      const bf16 *e = reinterpret_cast<const bf16 *>(&raw[c]);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) amax = fmaxf(amax, fabsf(__bfloat162float(e[k])));
+    }
+  }
+  amax = warp_max(amax);
+  const float scale = __fdiv_rn(fmaxf(amax, FP8_AMAX_FLOOR), FP8_MAX);
+  const size_t orow = slot_map ? (size_t)slot_map[r] : (size_t)r;
+  if (lane == 0) scale_out[orow] = scale;
+  uint2 *c_out = reinterpret_cast<uint2 *>(codes + orow * width);
+#pragma unroll
+  for (int c = 0; c < CHUNKS; ++c) {
+    const int i = lane + c * 32;
+    if (i < n_vec) {
+      const bf16 *e = reinterpret_cast<const bf16 *>(&raw[c]);
+      uint8_t q[8];
+      TO d[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        q[k] = encode_e4m3(__bfloat162float(e[k]), scale);
+        d[k] = from_f<TO>(__fmul_rn(to_f(fp8e4{q[k]}), scale));
+      }
+      c_out[i] = *reinterpret_cast<const uint2 *>(q);
+      if (deq) reinterpret_cast<uint4 *>(deq + (size_t)r * width)[i] = *reinterpret_cast<const uint4 *>(d);
+    }
+  }
+}
+
 template <typename TO>
 __global__ void __launch_bounds__(QT) gather_dequant_kernel(const uint8_t *__restrict__ k_codes, const uint8_t *__restrict__ v_codes,
                                                             const float *__restrict__ k_scale, const float *__restrict__ v_scale,
@@ -68,6 +116,16 @@ template <typename TI, typename TO>
 void launch_quantize_rows_fp8(const TI *src, int rows, int width, const int32_t *slot_map, uint8_t *codes, float *scale,
                               TO *deq, cudaStream_t st) {
   if (rows <= 0) return;
+  if constexpr (sizeof(TI) == 2 && sizeof(TO) == 2) {
+    const bool aligned = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(deq)) & 15) == 0 &&
+                         (reinterpret_cast<uintptr_t>(codes) & 7) == 0;
+    if (width % 8 == 0 && width <= 32 * 8 * VEC_CHUNKS && aligned) {
+      const int blocks = (rows + VEC_ROWS - 1) / VEC_ROWS;
+      if (width <= 32 * 8 * 4) quantize_rows_vec_kernel<TO, 4><<<blocks, VEC_ROWS * 32, 0, st>>>(src, rows, width, slot_map, codes, scale, deq);
+      else quantize_rows_vec_kernel<TO, VEC_CHUNKS><<<blocks, VEC_ROWS * 32, 0, st>>>(src, rows, width, slot_map, codes, scale, deq);
+      return;
+    }
+  }
   quantize_rows_kernel<TI, TO><<<rows, QT, 0, st>>>(src, width, slot_map, codes, scale, deq);
 }
 template void launch_quantize_rows_fp8<float, float>(const float *, int, int, const int32_t *, uint8_t *, float *, float *, cudaStream_t);

@@ -5,9 +5,13 @@ per-token FP8 cache).  Three levels:
   2. single-query attention reading codes + scales, against the oracle's attention over the dequantized rows;
   3. the whole prefill / chunked steps with an FP8 cache against the oracle's quantized model.  The stored codes are
      integers decided by floating-point values that the two sides compute with different rounding, so a value that
-     sits within that rounding of a decision boundary lands on a neighbouring code: every element must agree to
-     within one code step plus the input tolerance, most codes of the large entries must be identical, and the
-     dequantized tensors and the logits are compared by norm."""
+     sits within that rounding of a decision boundary lands on a neighbouring code -- a 6-12 % jump of that cache
+     entry, which the following layers see as input noise.  fp32 model: the inputs agree to ~1e-6 and the bars are
+     tight absolute ones.  bf16 model: the oracle is run twice, with the rows quantized from bf16 (the precision the
+     kernel decides in: the reference) and from fp32; the distance between these two oracle results measures how far
+     a 2^-9 relative change of the quantizer's input moves this model, and the CUDA path -- whose arithmetic differs
+     from fp64 by about that much -- must stay within twice that distance of the reference, per layer and tensor,
+     for the code-flip rate and for the logits."""
 import numpy as np
 import pytest
 import torch
@@ -64,42 +68,61 @@ def test_tail_attention_over_fp8_rows(n_q, n_kv, hd):
         off += n
 
 
-def _check_fp8_layer(model, ref, j, rows, n, kv_bar, flip_bar, in_tol):
-    """in_tol: how far the quantizer's inputs on the two sides may be apart, as a fraction of the row maximum."""
+def _stats(codes, scales, ref, j, name, n):
+    """(rel-L2 of the dequantized rows, fraction of differing codes among the large entries, largest elementwise gap
+    beyond one code step in units of the row maximum, largest relative scale gap) against ref's layer j."""
+    ref_c = ref[name + "_codes"][j][:n]
+    ref_s = ref[name + "_scale"][j][:n].astype(np.float64)
+    got_v, ref_v = O.e4m3_decode(codes), O.e4m3_decode(ref_c)            # in units of the row's scale (max 448)
+    mag = np.maximum(np.abs(got_v), np.abs(ref_v))
+    step = np.where(mag < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(mag, 2.0 ** -6))) - 3))
+    excess = float(np.maximum(np.abs(got_v - ref_v) - step, 0).max() / 448)
+    big = np.abs(ref_v) >= 448 / 16
+    flips = float((codes[big] != ref_c[big]).mean())
+    rel = rel_l2(got_v * scales[:, None, None], ref[name][j][:n])
+    return rel, flips, excess, float(np.abs(scales / ref_s - 1).max())
+
+
+def _gpu_layer(model, j, rows):
     Kc, Vc, Ks, Vs, _ = model.kv_cache_view_fp8(j)
     rows_t = torch.as_tensor(rows, device="cuda")
-    for name, codes, scales in (("K", Kc, Ks), ("V", Vc, Vs)):
-        got_c = codes[rows_t].cpu().numpy()
-        got_s = to_np(scales[rows_t])
-        ref_c = ref[name + "_codes"][j][:n]
-        ref_s = ref[name + "_scale"][j][:n].astype(np.float64)
-        assert np.allclose(got_s, ref_s, rtol=max(kv_bar, 2 * in_tol)), (name, j)
-        got_v, ref_v = O.e4m3_decode(got_c), O.e4m3_decode(ref_c)          # in units of the row's scale (max 448)
-        # element by element: apart by at most one code step at that magnitude plus the input tolerance
-        mag = np.maximum(np.abs(got_v), np.abs(ref_v))
-        step = np.where(mag < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(mag, 2.0 ** -6))) - 3))
-        assert (np.abs(got_v - ref_v) <= step + in_tol * 448 + mag * 2 * in_tol).all(), (name, j)
-        # where a code step is large against the input tolerance (the top four binades) most codes are identical
-        big = np.abs(ref_v) >= 448 / 16
-        assert (got_c[big] != ref_c[big]).mean() <= flip_bar, (name, j, float((got_c[big] != ref_c[big]).mean()))
-        deq = got_v * got_s[:, None, None]
-        assert rel_l2(deq, ref[name][j][:n]) <= kv_bar, (name, j, rel_l2(deq, ref[name][j][:n]))
+    return {"K": (Kc[rows_t].cpu().numpy(), to_np(Ks[rows_t])), "V": (Vc[rows_t].cpu().numpy(), to_np(Vs[rows_t]))}
 
 
-# fp32 model: the inputs of the quantizer agree to ~1e-6, so hardly any code may differ.
-# bf16 model: in the first layer the inputs agree to a few 1e-3 against a code step of 6-12 % of the value, so 2-4 % of
-# the codes land on the neighbouring value (dequantized rel-L2 1.3e-2); those flips are 6-12 % perturbations of
-# individual cache entries, which the next layer sees as ~1 % input noise, so from the second layer on about a quarter
-# of the large entries sit on a neighbouring code and the dequantized tensors differ by 3.0-3.4e-2 -- a level that no
-# longer grows with depth (measured on these shapes); the logits stay within 0.04.  Layer 1 is held to the tight bars.
-@pytest.mark.parametrize("shape,dtype,act,kv_bar,flip_bar,in_tol,lg_bar", [
-    (S.TINY, torch.float32, None, 2e-3, 1e-3, 1e-5, 5e-3),
-    (S.TINY, torch.bfloat16, 1, 5e-2, 0.35, 6e-2, 0.1),
-    (MID, torch.bfloat16, 1, 5e-2, 0.35, 6e-2, 0.1),
-    (MID, torch.bfloat16, 0, 5e-2, 0.35, 6e-2, 0.1),
+def _check_fp8_layer(model, ref, j, rows, n, other=None):
+    """fp32 model (other is None): tight absolute bars.  bf16 model: within twice the distance between the two oracle
+    evaluations `ref` (rows quantized from bf16) and `other` (from fp32), plus a small floor."""
+    got = _gpu_layer(model, j, rows)
+    for name in ("K", "V"):
+        rel, flips, excess, ds = _stats(got[name][0], got[name][1], ref, j, name, n)
+        if other is None:
+            assert rel <= 2e-3 and flips <= 1e-3 and excess <= 1e-4 and ds <= 1e-4, (name, j, rel, flips, excess, ds)
+        else:
+            o_rel, o_flips, o_excess, o_ds = _stats(other[name + "_codes"][j][:n], other[name + "_scale"][j][:n].astype(np.float64),
+                                                    ref, j, name, n)
+            assert rel <= 2 * o_rel + 5e-3, (name, j, rel, o_rel)
+            assert flips <= 2 * o_flips + 0.02, (name, j, flips, o_flips)
+            assert excess <= 2 * o_excess + 0.01, (name, j, excess, o_excess)
+            assert ds <= 2 * o_ds + 0.01, (name, j, ds, o_ds)
+
+
+def _refs(cfg, ow, tok, lens, l, g, dtype):
+    """(reference, second oracle evaluation for the sensitivity bars or None, logits bar)."""
+    if dtype == torch.float32:
+        return O.swiftkv(cfg, ow, tok, lens, l, g, kv_fp8=True), None, 5e-3
+    ref = O.swiftkv(cfg, ow, tok, lens, l, g, kv_fp8=True, row_dtype="bf16")
+    other = O.swiftkv(cfg, ow, tok, lens, l, g, kv_fp8=True)
+    return ref, other, 2 * float(np.max(np.abs(other["logits"] - ref["logits"]))) + 0.02
+
+
+@pytest.mark.parametrize("shape,dtype,act", [
+    (S.TINY, torch.float32, None),
+    (S.TINY, torch.bfloat16, 1),
+    (MID, torch.bfloat16, 1),
+    (MID, torch.bfloat16, 0),
 ])
 @pytest.mark.parametrize("l,g", [(2, 1), (1, 2), (4, 1)])
-def test_prefill_with_fp8_cache(shape, dtype, act, kv_bar, flip_bar, in_tol, lg_bar, l, g):
+def test_prefill_with_fp8_cache(shape, dtype, act, l, g):
     import paper_2410_03960_b200 as P
     seed, lens = 13, [300, 77, 129]
     w = S.make_weights(shape, seed, dtype, "cuda")
@@ -110,13 +133,16 @@ def test_prefill_with_fp8_cache(shape, dtype, act, kv_bar, flip_bar, in_tol, lg_
         model.set_activation_format(act)
     model.prefill(tok, lens, l, g)
     model.status()
-    ref = O.swiftkv(cfg, ow, tok.numpy(), lens, l, g, kv_fp8=True)
+    ref, other, lg_bar = _refs(cfg, ow, tok.numpy(), lens, l, g, dtype)
+    n = sum(lens)
     for j in range(shape.n_layers):
-        _check_fp8_layer(model, ref, j, np.arange(sum(lens)), sum(lens), kv_bar, flip_bar, in_tol)
-    if dtype == torch.bfloat16:      # first layer: nothing upstream has been quantized yet
-        _check_fp8_layer(model, ref, 0, np.arange(sum(lens)), sum(lens), 2e-2, 0.06, 5e-3)
+        _check_fp8_layer(model, ref, j, np.arange(n), n, other)
+    if other is not None:            # first layer: nothing upstream has been quantized, so absolute bars hold as well
+        for name in ("K", "V"):
+            rel, flips, _, _ = _stats(*_gpu_layer(model, 0, np.arange(n))[name], ref, 0, name, n)
+            assert rel <= 2e-2 and flips <= 0.06, (name, rel, flips)
     lg = to_np(model.first_logits())
-    assert np.max(np.abs(lg - ref["logits"])) <= lg_bar, float(np.max(np.abs(lg - ref["logits"])))
+    assert np.max(np.abs(lg - ref["logits"])) <= lg_bar, (float(np.max(np.abs(lg - ref["logits"]))), lg_bar)
     # memory: codes + one fp32 scale per row and plane instead of 16-bit (32-bit) elements
     _, kv16 = P.workspace_bytes(shape, dtype, 4096, 4, l, g)
     _, kv8 = P.workspace_bytes(shape, dtype, 4096, 4, l, g, P.KV_FP8)
@@ -124,12 +150,9 @@ def test_prefill_with_fp8_cache(shape, dtype, act, kv_bar, flip_bar, in_tol, lg_
     assert kv8 * (2 if dtype == torch.bfloat16 else 4) * d_kv == kv16 * (d_kv + 4)
 
 
-@pytest.mark.parametrize("shape,dtype,act,kv_bar,flip_bar,in_tol,lg_bar", [
-    (S.TINY, torch.float32, None, 2e-3, 1e-3, 1e-5, 5e-3),
-    (MID, torch.bfloat16, 1, 5e-2, 0.35, 6e-2, 0.1),
-])
+@pytest.mark.parametrize("shape,dtype,act", [(S.TINY, torch.float32, None), (MID, torch.bfloat16, 1)])
 @pytest.mark.parametrize("paged", [False, True])
-def test_chunked_steps_with_fp8_cache(shape, dtype, act, kv_bar, flip_bar, in_tol, lg_bar, paged):
+def test_chunked_steps_with_fp8_cache(shape, dtype, act, paged):
     """Chunks and decode tokens read earlier rows back from the FP8 cache: still the oracle's one-shot quantized model."""
     import paper_2410_03960_b200 as P
     seed, lens, l, g, n_decode = 29, [260, 90], 2, 1, 2
@@ -151,9 +174,33 @@ def test_chunked_steps_with_fp8_cache(shape, dtype, act, kv_bar, flip_bar, in_to
     lg = to_np(model.first_logits())
     for b, n in enumerate(lens):
         m = n + n_decode
-        ref = O.swiftkv(cfg, ow, toks[b][:m].numpy(), [m], l, g, kv_fp8=True)
+        ref, other, lg_bar = _refs(cfg, ow, toks[b][:m].numpy(), [m], l, g, dtype)
         p = np.arange(m)
         rows = (np.asarray(pages[b])[p // 128] * 128 + p % 128) if paged else b * 384 + p
         for j in range(shape.n_layers):
-            _check_fp8_layer(model, ref, j, rows, m, kv_bar, flip_bar, in_tol)
+            _check_fp8_layer(model, ref, j, rows, m, other)
         assert np.max(np.abs(lg[b] - ref["logits"][0])) <= lg_bar, b
+
+
+def test_fp8_cache_at_8b_widths():
+    """Llama-3.1-8B layer widths (4 layers): tcgen05 GEMMs and attention, vectorized row pass, group-by-group
+    SingleInputKV projection with 2-way AcrossKV."""
+    import paper_2410_03960_b200 as P
+    shape = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-width-4-layers")
+    seed, lens, l, g = 2, [257, 130], 2, 2
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g, kv_format=P.KV_FP8)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    ref, other, lg_bar = _refs(cfg, ow, tok.numpy(), lens, l, g, torch.bfloat16)
+    n = sum(lens)
+    for j in range(shape.n_layers):
+        _check_fp8_layer(model, ref, j, np.arange(n), n, other)
+    for name in ("K", "V"):
+        rel, flips, _, _ = _stats(*_gpu_layer(model, 0, np.arange(n))[name], ref, 0, name, n)
+        assert rel <= 2e-2 and flips <= 0.06, (name, rel, flips)
+    assert model.kv_cache_view_fp8(3)[4] == 2 and model.kv_cache_view_fp8(2)[0].data_ptr() == model.kv_cache_view_fp8(3)[0].data_ptr()
+    err = float(np.max(np.abs(to_np(model.first_logits()) - ref["logits"])))
+    assert err <= lg_bar, (err, lg_bar)

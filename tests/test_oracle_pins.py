@@ -436,6 +436,19 @@ def test_quantize_per_token_properties():
     assert np.array_equal(c3[nz] ^ 0x80, codes[nz]) and np.array_equal(s3, scale)
 
 
+def test_round_to_bf16_against_library():
+    rng = np.random.default_rng(2)
+    x = np.concatenate([rng.standard_normal(100000).astype(np.float32) * 3,
+                        np.float32([0.0, -0.0, 1.0, 1.00390625, 1.001953125, 1.005859375, 3.3895314e38, 1e-38])])
+    want = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(O.round_to_bf16(x), want)
+    # ties go to the even significand: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert O.round_to_bf16(np.float32([1.00390625]))[0] == 1.0 and O.round_to_bf16(np.float32([1.01171875]))[0] == 1.015625
+    c, s, _ = O.quantize_per_token(x[:64].reshape(2, 32), "bf16")
+    c2, s2, _ = O.quantize_per_token(want[:64].reshape(2, 32))
+    assert np.array_equal(c, c2) and np.array_equal(s, s2)
+
+
 def test_kv_cache_reduction_with_fp8():
     for g, fp8, pct in _rows("kv_cache_reduction_fp8.txt"):
         got = 100 * O.kv_cache_reduction(32, 16, int(g), 0.5 if int(fp8) else 1.0)
