@@ -5,6 +5,7 @@ Runs a few SwiftKV prefills (default l = 1 of 2 layers) of a model with the Llam
 every hot kernel (the QKV / O / SwiGLU / down / SingleInputKV GEMMs, the flash-attention kernel, the norms and
 the last-token path) launches with its real shapes while the process holds only a few GB: the weights of one
 layer (436 MB) plus activations exceed the 126 MB L2, so DRAM counters stay meaningful.
+Environment: SWIFTKV_KERNEL_MASK, SWIFTKV_ACT_FORMAT (0 bf16, 1 half), SWIFTKV_KV_FORMAT=fp8 (per-token FP8 cache).
 """
 from __future__ import annotations
 
@@ -30,7 +31,8 @@ def main() -> None:
     lens = [tokens // n_prompts] * n_prompts
     tokens = sum(lens)
     tok = S.make_prompts(1, lens, shape.vocab).cuda()
-    model = P.SwiftKVModel(shape, w, torch.bfloat16, tokens, n_prompts, l, 1)
+    kv_format = P.KV_FP8 if os.environ.get("SWIFTKV_KV_FORMAT") == "fp8" else P.KV_MODEL_DTYPE
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, tokens, n_prompts, l, 1, kv_format=kv_format)
     if os.environ.get("SWIFTKV_KERNEL_MASK"):
         model.set_kernel_mask(int(os.environ["SWIFTKV_KERNEL_MASK"]))
     if os.environ.get("SWIFTKV_ACT_FORMAT"):

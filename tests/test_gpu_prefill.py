@@ -188,6 +188,33 @@ def test_config2_full_size_prefix_parity_and_determinism():
     model.prefill(tok, lens, l, g)
     model.status()
     assert torch.equal(logits1, model.first_logits())
+    _check_full_size_samples(model, lens, shape, to_np(logits1))
+
+
+def _check_full_size_samples(model, lens, shape, logits):
+    """Sampled outputs of the oracle's FULL-size run of the same workload (tests/golden/config2_full_sample.npz, written
+    by tests/golden/make_config2_full_sample.py from the oracle alone): first-token logits at 2048 vocabulary entries
+    per prompt, the arg-max, and K / V rows of layers 1, 16, 17, 32 at four positions per prompt (first, last, two
+    inside) -- the last positions and the logits depend on every token of the prompt."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "config2_full_sample.npz")
+    gold = np.load(path)
+    assert list(gold["lens"]) == list(lens)
+    for b in range(len(lens)):
+        got = logits[b][gold["vocab_idx"][b]]
+        ref = gold["logits"][b].astype(np.float64)
+        # (the norm of the sample against the sample: same 2e-2 bar as for a whole row)
+        assert rel_l2(got, ref) <= 2e-2, (b, rel_l2(got, ref))
+        assert np.max(np.abs(got - ref)) <= 0.1, (b, float(np.max(np.abs(got - ref))))
+        # the oracle's arg-max entry: within the bar of the oracle's value, and no entry beats it by more than the bar
+        assert abs(logits[b][gold["argmax"][b]] - gold["max"][b]) <= 0.1
+        assert logits[b].max() <= gold["max"][b] + 0.1
+        assert abs(np.linalg.norm(logits[b]) / gold["logits_norm"][b] - 1) <= 2e-2
+    offs = np.concatenate([[0], np.cumsum(lens)])[:-1]
+    rows = torch.as_tensor((offs[:, None] + gold["pos"]).reshape(-1), device="cuda")
+    for j in (0, 15, 16, 31):
+        K, V, _ = model.kv_cache_view(j)
+        assert rel_l2(to_np(K[rows]), gold[f"K{j}"]) <= 2e-2, (j, rel_l2(to_np(K[rows]), gold[f"K{j}"]))
+        assert rel_l2(to_np(V[rows]), gold[f"V{j}"]) <= 2e-2, (j, rel_l2(to_np(V[rows]), gold[f"V{j}"]))
 
 
 @pytest.mark.skipif(os.environ.get("SWIFTKV_RUN_SLOW") != "1",
