@@ -48,6 +48,35 @@ SWIGLU_WEIGHT_BYTES = 2 * 14336 * 4096 * 2
 SWIGLU_CAPTURE_TOKENS, SWIGLU_CAPTURE_BYTES, SWIGLU_BAND_ROWS = 8192, 1.2315e9, 2048
 
 
+def other_rooflines(prof, f_sw, lens, steps, tensor_peak, hbm_peak):
+    """Achieved rates of the remaining kernel classes against their own bounds (CUDA events over the timed steps; same
+    algorithmic-work conventions as the dominant kernel's entry)."""
+    T, d, F, dq = sum(lens), SHAPE.hidden, SHAPE.ffn, SHAPE.n_q_heads * SHAPE.head_dim
+    dkv, Lt = SHAPE.n_kv_heads * SHAPE.head_dim, SHAPE.n_layers - SWIFT_LAYER
+    out = []
+
+    def add(name, bound, work, ms, peak, unit, note):
+        if ms > 0 and peak:
+            ach = work / (ms / 1e3) / (1e12 if unit == "TFLOP/s" else 1e9)
+            out.append({"kernels": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                        "ms_per_step": ms / steps, "note": note})
+
+    proj_flops = (f_sw["gemm"] - SWIFT_LAYER * 2.0 * T * (2 * F) * d) * steps
+    add("projection GEMMs (QKV, O, down, SingleInputKV)", "tensor", proj_flops, prof["gemm"][0], tensor_peak, "TFLOP/s",
+        "2*M*N*K per launch")
+    add("attention_tc_kernel", "tensor", f_sw["attention"] * steps, prof["attention"][0], tensor_peak, "TFLOP/s",
+        "4*d_q*n*(n+1)/2 per prompt and layer (causal half only); co-limited by ex2")
+    # RMSNorm: 2 per layer + the SingleInputKV norm, read fp32 x and write 16-bit h; embedding gather: read 2 B, write 4 B
+    elem_bytes = ((2 * SWIFT_LAYER + 1) * T * d * 6.0 + T * d * 6.0) * steps
+    add("rmsnorm / embedding", "hbm", elem_bytes, prof["elementwise"][0], hbm_peak, "GB/s",
+        "6 B per element and norm; per-layer bf16->half weight copies run on a side stream and are not in this time")
+    # last-token path: every later layer's Q, O, gate, up, down weights once, the lm_head once, every later layer's cache rows once
+    tail_bytes = (Lt * (2.0 * d * dq + 3.0 * d * F) * 2 + SHAPE.vocab * d * 2.0 + Lt * T * 2.0 * dkv * 2) * steps
+    add("last-token path (weight streaming + single-query attention)", "hbm", tail_bytes, prof["tail"][0], hbm_peak, "GB/s",
+        "weights and cache rows of layers > l read once; ~150 small dependent launches per step")
+    return out
+
+
 def swiglu_traffic_bytes(tokens: int) -> float:
     per_token = (SWIGLU_CAPTURE_BYTES - (SWIGLU_CAPTURE_TOKENS // SWIGLU_BAND_ROWS) * SWIGLU_WEIGHT_BYTES) / SWIGLU_CAPTURE_TOKENS
     bands = -(-tokens // SWIGLU_BAND_ROWS)
@@ -333,6 +362,7 @@ def run_ours(args, rank, world, local_rank):
                          "all_gemms_tflops": gemm_ach, "all_gemms_ms_per_step": gemm_ms / args.steps},
             "time_share_ms_per_step": {k: v[0] / args.steps for k, v in prof.items()},
             "attention_tflops": (f_sw["attention"] * args.steps / (attn_ms / 1e3) / 1e12) if attn_ms > 0 else None,
+            "roofline_other": other_rooflines(prof, f_sw, lens, args.steps, peak, peaks.get("hbm_gbs")),
         }
         # ---- the CPU oracle, as it stands, on a bounded sample of the same workload (N = 1 only)
         if world == 1 and not args.no_cpu_baseline:
