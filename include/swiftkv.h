@@ -174,7 +174,9 @@ typedef struct {
  *   seqs   : HOST array of n_seqs entries
  * swift_layer and acrosskv_group must stay the same for all steps that share cached state.  Sum of n_new and sum of
  * (n_past + n_new) must not exceed max_tokens.  swiftkv_first_logits afterwards returns one row per emitting
- * sequence, in order; swiftkv_kv_cache_view returns whole planes (index them with cache_row + position).
+ * sequence, in order (none, n_seqs = 0, for a minibatch of inner prefill chunks in which nobody emits: such a step
+ * fills caches only and never touches layers l+1..L); swiftkv_kv_cache_view returns whole planes (index them with
+ * cache_row + position).
  * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA.
  */
 int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const swiftkv_seq_step *seqs, int32_t n_seqs,

@@ -688,7 +688,8 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
   }
   if (total > m->max_tokens || total_kv > m->max_tokens)
     return fail(SWIFTKV_ERR_INVALID_ARG, "%lld new / %lld cached+new tokens > max_tokens %d", total, total_kv, m->max_tokens);
-  if (bt.n_emit < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "no sequence is marked to emit logits");
+  // (no emitting sequence is fine: a minibatch of inner prefill chunks fills caches only and skips layers l+1..L)
+  if (plain && bt.n_emit < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "no sequence is marked to emit logits");
   bt.T_tok = (int)total; bt.total_kv = (int)total_kv;
   if (!tokens_on_device)
     for (long long t = 0; t < total; ++t)
@@ -744,10 +745,10 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
   CUDA_TRY(cudaMemcpyAsync(b.kv_row0, row0, (size_t)B * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.kv_len, klen, (size_t)B * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.kcu, kcu, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(cudaMemcpyAsync(b.last_idx, last_idx, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(cudaMemcpyAsync(b.last_pos, last_pos, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(cudaMemcpyAsync(b.emit_row0, e_row0, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(cudaMemcpyAsync(b.emit_len, e_len, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  if (ne > 0) CUDA_TRY(cudaMemcpyAsync(b.last_idx, last_idx, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  if (ne > 0) CUDA_TRY(cudaMemcpyAsync(b.last_pos, last_pos, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  if (ne > 0) CUDA_TRY(cudaMemcpyAsync(b.emit_row0, e_row0, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
+  if (ne > 0) CUDA_TRY(cudaMemcpyAsync(b.emit_len, e_len, (size_t)ne * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.tokens, tokens, (size_t)total * 4,
                            tokens_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, st));
   int32_t rc;

@@ -64,8 +64,6 @@ def main():
                 seqs.append((k, done[b], where(b, paged), int(done[b] + k == n)))
                 packed.append(toks[b][done[b]:done[b] + k])
                 done[b] += k
-            if not any(s[3] for s in seqs):
-                seqs[0] = seqs[0][:3] + (1,)
             model.step(torch.cat(packed), seqs, SWIFT_LAYER, GROUP)
             steps += 1
         return steps

@@ -58,15 +58,12 @@ def test_chunked_prefill_then_decode(shape, dtype, act, kv_bar, lg_bar, l, g):
             if emit:
                 emitting.append(b)
             done[b] += k
-        if not emitting:                       # the library wants at least one emitting sequence per step
-            seqs[0] = (seqs[0][0], seqs[0][1], seqs[0][2], 1)
-            emitting = [-1]
-        model.step(torch.cat(packed), seqs, l, g)
+        model.step(torch.cat(packed), seqs, l, g)     # (steps in which nobody emits only fill caches)
         model.status()
         lg = model.first_logits().clone()
+        assert lg.shape[0] == len(emitting)
         for i, b in enumerate(emitting):
-            if b >= 0:
-                last_logits[b] = lg[i]
+            last_logits[b] = lg[i]
     for b, n in enumerate(lens):
         ref = O.swiftkv(cfg, ow, toks[b][:n].numpy(), [n], l, g)
         _check_seq(model, shape, ref, b * cap, n, kv_bar)
@@ -116,7 +113,6 @@ def test_step_argument_checks():
     tok = S.token_ids(0, 0, 40, shape.vocab)
     for bad in ([(40, 0, 250, 1)],                      # runs past max_tokens
                 [(20, 0, 0, 1), (20, 0, 10, 1)],        # overlapping regions
-                [(40, 0, 0, 0)],                        # nobody emits
                 [(0, 0, 0, 1)]):                        # empty chunk
         n = sum(s[0] for s in bad)
         with pytest.raises(P.SwiftKVError) as e:
