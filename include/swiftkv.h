@@ -236,8 +236,10 @@ int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, float *ms_per_
 int32_t swiftkv_last_launch_count(const swiftkv_model *m);
 
 /* Select kernel families (debug / comparison): bit 0 = tensor-core GEMMs, bit 1 = tensor-core attention,
- * bit 2 = CTA-pair (cta_group::2) form of the projection GEMMs, bit 3 = CTA-pair form of the gate/up GEMM too.
- * Default 7: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
+ * bit 2 = CTA-pair (cta_group::2) form of the projection GEMMs, bit 3 = CTA-pair form of the gate/up GEMM too,
+ * bit 5 = decode minibatches (at most 8 sequences, one new token each) run every layer on the weight-streaming
+ * kernels of the last-token path instead of 128-row GEMM tiles.
+ * Default 39: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
 int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
 /* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention

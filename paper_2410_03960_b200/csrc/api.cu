@@ -67,6 +67,7 @@ struct Buffers {
                             //   models use kv16)
   float *y;                 // continuing tokens' residual [B, d]
   float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
+  float *ky, *vy;           // a decode step's new K / V rows before they go to the cache, [8, d_kv] each
   float *tail_scratch;
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
@@ -97,7 +98,7 @@ struct swiftkv_model {
   int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;   // rows in use per cache plane, sequences with logits
   int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
-  int kernel_mask = 7;
+  int kernel_mask = 39;
   int act_format = SWIFTKV_ACT_F16;
   // profiling
   bool profiling = false;
@@ -153,6 +154,8 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.qy = (float *)cv.take(R * dq * 4);
   b.ay = (float *)cv.take(R * dq * 4);
   b.acty = (float *)cv.take(R * F * 4);
+  b.ky = (float *)cv.take(R * dkv_ * 4);
+  b.vy = (float *)cv.take(R * dkv_ * 4);
   b.tail_scratch = (float *)cv.take(tail_attention_scratch_bytes(B, c.n_q_heads, c.head_dim, T));
   b.logits = (float *)cv.take((size_t)B * c.vocab * 4);
   b.tokens = (int32_t *)cv.take((size_t)T * 4);
@@ -355,6 +358,8 @@ struct Batch {
   bool plain;
   bool paged;         // sequences own lists of 128-row pages instead of one contiguous region
   int blk_stride;     // pages per sequence in the device block tables
+  bool decode;        // at most 8 sequences, one new token each, all emitting: every layer runs on the weight-streaming
+                      // kernels of the last-token path
 };
 
 template <typename TA, typename T>
@@ -410,7 +415,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     cudaEventRecord(m->ev_ready[buf], m->side);
   };
   if constexpr (sizeof(T) == 2) {
-    if (use_w16 && l > 0) {
+    if (use_w16 && l > 0 && !bt.decode) {
       cudaEventRecord(m->ev_start, st);                 // the side stream starts after everything queued before
       cudaStreamWaitEvent(m->side, m->ev_start, 0);
       convert_layer(0);
@@ -428,7 +433,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   // and stack them (Sec. 3.5)
   const int ng = n_groups(L, l, g);
   const int fold_fmt = use_w16 ? 1 : 0;
-  if (l < L && (m->fold_l != l || m->fold_g != g || m->fold_fmt != fold_fmt)) {
+  if (!bt.decode && l < L && (m->fold_l != l || m->fold_g != g || m->fold_fmt != fold_fmt)) {
     for (int i = 0; i < ng; ++i) {
       const swiftkv_layer_weights &lw = m->layers[l + i * g];
       const size_t off = (size_t)i * 2 * dkv * d;
@@ -447,8 +452,64 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     m->fold_l = l; m->fold_g = g; m->fold_fmt = fold_fmt;
   }
 
+  // ---- a minibatch of decode tokens (Sec. 3.5: "decode tokens complete all layers"): at most 8 rows, so every
+  //      projection is bound by streaming its weights once -- layers 1..l run on the last-token path's kernels too,
+  //      the new K / V rows go to the cache before the single-query attention reads it, and the rows of the later
+  //      layers' caches come from each group leader's own gain and W_K, W_V applied to the layer-l output (Eq. 2)
+  if (bt.decode) {
+    const int rows = T_tok;
+    float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
+    auto store_kv = [&](int slot) {      // ky (rotated), vy -> the cache rows of the new tokens in `slot`
+      Scope s(m, st, SWIFTKV_KC_TAIL, fp8 ? 4 : 2);
+      if (fp8) {
+        launch_scatter_rows<T>(ky, kst, nullptr, rows, dkv, st);    // rows are quantized from the model dtype
+        launch_scatter_rows<T>(vy, vst, nullptr, rows, dkv, st);
+        launch_quantize_rows_fp8<T, T>(kst, rows, dkv, b.slot, k_codes(slot), k_scale(slot), (T *)nullptr, st);
+        launch_quantize_rows_fp8<T, T>(vst, rows, dkv, b.slot, v_codes(slot), v_scale(slot), (T *)nullptr, st);
+      } else {
+        launch_scatter_rows<T>(ky, kv + (size_t)slot * 2 * plane, b.slot, rows, dkv, st);
+        launch_scatter_rows<T>(vy, kv + (size_t)slot * 2 * plane + plane, b.slot, rows, dkv, st);
+      }
+    };
+    auto project_kv = [&](const swiftkv_layer_weights &lw) {   // hy -> ky (rotated at the tokens' positions), vy
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wk, nullptr, rows, dkv, d, ky, dkv, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wv, nullptr, rows, dkv, d, vy, dkv, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(ky, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st); }
+    };
+    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx, y, rows, d, st); }
+    for (int j = 0; j < l; ++j) {
+      const swiftkv_layer_weights &lw = m->layers[j];
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
+      project_kv(lw);
+      store_kv(j);
+      {
+        Scope s(m, st, SWIFTKV_KC_TAIL, 2);
+        if (fp8)
+          launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(j), (const fp8e4 *)v_codes(j), k_scale(j), v_scale(j), ay, b.emit_row0,
+                                       b.emit_len, blk_emit, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                       b.tail_scratch, st);
+        else
+          launch_tail_attention<T>(qy, kv + (size_t)j * 2 * plane, kv + (size_t)j * 2 * plane + plane, nullptr, nullptr, ay, b.emit_row0,
+                                   b.emit_len, blk_emit, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                   b.tail_scratch, st);
+      }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, nullptr, rows, d, F, y, d, OUT_RESID_ADD_F32, st); }
+    }
+    for (int i = 0; i < ng && l < L; ++i) {      // SingleInputKV rows of the new tokens, one AcrossKV group at a time
+      const swiftkv_layer_weights &lw = m->layers[l + i * g];
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
+      project_kv(lw);
+      store_kv(l + i);
+    }
+  }
+
   // ---- layers 1..l on all prompt tokens (unmodified, Sec. 3.1)
-  for (int j = 0; j < l; ++j) {
+  for (int j = 0; j < l && !bt.decode; ++j) {
     const swiftkv_layer_weights &lw = m->layers[j];
     T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
     if constexpr (sizeof(T) == 2) {
@@ -572,7 +633,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   }
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
-  if (l < L) {
+  if (l < L && !bt.decode) {
     { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
     if (fp8) {
       // one group at a time through the staging planes: projection (+ RoPE on K), then the quantizing row pass into the
@@ -608,7 +669,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     const int rows = std::min(MAX_TAIL_ROWS, bt.n_emit - r0);
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
     float *y = b.y + (size_t)r0 * d;
-    { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
+    if (!bt.decode) { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
     for (int j = l; j < L; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
       const int slot = l + (j - l) / g;
@@ -691,6 +752,7 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
   // (no emitting sequence is fine: a minibatch of inner prefill chunks fills caches only and skips layers l+1..L)
   if (plain && bt.n_emit < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "no sequence is marked to emit logits");
   bt.T_tok = (int)total; bt.total_kv = (int)total_kv;
+  bt.decode = !plain && total == n_seqs && bt.n_emit == n_seqs && n_seqs <= MAX_TAIL_ROWS && (m->kernel_mask & 32);
   if (!tokens_on_device)
     for (long long t = 0; t < total; ++t)
       if (tokens[t] < 0 || tokens[t] >= c.vocab) return fail(SWIFTKV_ERR_INVALID_ARG, "token %lld = %d outside [0, %d)", t, tokens[t], c.vocab);
@@ -864,7 +926,7 @@ extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, flo
 extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
 extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   if (!m) return 0;
-  m->kernel_mask = mask & 15;
+  m->kernel_mask = mask & 63;
   return m->kernel_mask;
 }
 

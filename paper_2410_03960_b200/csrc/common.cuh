@@ -132,6 +132,9 @@ void launch_gather_dequant_fp8(const uint8_t *k_codes, const uint8_t *v_codes, c
 template <typename T>
 void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
+// fp32 rows -> rows slot_map[r] (null: r) of a [*, width] plane of type T
+template <typename T>
+void launch_scatter_rows(const float *src, T *dst, const int32_t *slot_map, int rows, int width, cudaStream_t st);
 void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, double theta, cudaStream_t st);
 // dst[r, c] = w[r, c] * gamma[c]   (gain of the input norm folded into a projection weight, Sec. 3.5)
 template <typename T, typename TO>

@@ -221,6 +221,22 @@ void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows
   gather_rows_kernel<<<n_rows, 256, 0, st>>>(x, idx, y, d);
 }
 
+// fp32 rows -> rows slot_map[r] (null: r) of a plane in the cache's element type (a decode step's new K / V rows)
+template <typename T>
+__global__ void scatter_rows_kernel(const float *__restrict__ src, T *__restrict__ dst, const int32_t *__restrict__ slot_map,
+                                    int width) {
+  const size_t orow = slot_map ? (size_t)slot_map[blockIdx.x] : (size_t)blockIdx.x;
+  const float *s = src + (size_t)blockIdx.x * width;
+  T *d = dst + orow * width;
+  for (int i = threadIdx.x; i < width; i += blockDim.x) d[i] = from_f<T>(s[i]);
+}
+template <typename T>
+void launch_scatter_rows(const float *src, T *dst, const int32_t *slot_map, int rows, int width, cudaStream_t st) {
+  if (rows > 0) scatter_rows_kernel<T><<<rows, 256, 0, st>>>(src, dst, slot_map, width);
+}
+template void launch_scatter_rows<float>(const float *, float *, const int32_t *, int, int, cudaStream_t);
+template void launch_scatter_rows<bf16>(const float *, bf16 *, const int32_t *, int, int, cudaStream_t);
+
 // dst[r, c] = w[r, c] * gamma[c], product in fp32, one rounding to the output type
 template <typename T, typename TO>
 __global__ void fold_kernel(const T *__restrict__ w, const T *__restrict__ gamma, TO *__restrict__ dst, long long n, int cols) {

@@ -242,8 +242,8 @@ template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *
 // ---------------------------------------------------------------------------------------------------------
 __host__ __device__ inline int tail_chunk(int max_seq_len) {
   int c = (max_seq_len + 63) / 64;          // at most 64 splits
-  c = (c + 31) / 32 * 32;
-  return c < 256 ? 256 : c;
+  c = (c + 127) / 128 * 128;                // whole rounds of the block's 4 warps x 32 keys
+  return c < 512 ? 512 : c;
 }
 
 template <typename T>
@@ -264,13 +264,31 @@ __device__ __forceinline__ float dot_row(const float *__restrict__ qs, const T *
 }
 
 // Block (split, KV head, prompt), 4 warps.  Every warp walks 32-key chunks of the block's key range for ALL query heads
-// of the KV head's group at once, so each K and V row is fetched once per group:
-//   scores : lane = key; the 256-byte K row is read with 128-bit loads and dotted with the REP query vectors (smem)
+// of the KV head's group at once, so each K and V row is fetched once per group.  The 32 K rows and 32 V rows of a chunk
+// are copied into the warp's shared-memory tiles with coalesced 16-byte cp.async (a lane-per-key read straight from
+// global memory touches 16 bytes of 32 different lines per instruction and thrashes L1), one chunk ahead of the math:
+//   scores : lane = key; its K row is read from the padded tile with 128-bit loads and dotted with the REP query vectors
 //   softmax: online, per head, warp-wide max / sum
-//   output : for each of the 32 keys the V row is read once (coalesced, lane = 4 consecutive dims) and accumulated
-//            into REP x 4 registers with the probabilities broadcast by shuffle
+//   output : for each of the 32 keys the V row is read once (lane = 4 consecutive dims) and accumulated into REP x 4
+//            registers with the probabilities broadcast by shuffle
 // then the warps are merged in shared memory and (max, sum, acc[hd]) per head goes to scratch.
 constexpr int TA_WARPS = 4;
+template <typename T>
+struct TailTile {
+  static constexpr int ROW = 128 * (int)sizeof(T);   // bytes of one K / V row of a head (head_dim 128)
+  static constexpr int KSTRIDE = ROW + 16;           // padded: lane-per-row 128-bit reads hit 32 different banks
+  static constexpr int LPR = ROW / 16;               // lanes that copy one row
+  static constexpr int RPI = 32 / LPR;               // rows per copy instruction
+  static constexpr int NI = 32 / RPI;                // copy instructions per 32-row tile
+  static constexpr int K_BYTES = 32 * KSTRIDE, V_BYTES = 32 * ROW;
+};
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 template <typename T, int REP, int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
@@ -278,35 +296,63 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk, int n_splits, float scale,
     float *__restrict__ scratch) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
-  __shared__ float qs[REP][HD];
-  __shared__ float w_m[TA_WARPS][REP], w_l[TA_WARPS][REP];
-  __shared__ float w_acc[TA_WARPS][REP][HD];
+  using TT = TailTile<T>;
+  extern __shared__ __align__(16) uint8_t ta_smem[];
+  float (*qs)[HD] = reinterpret_cast<float (*)[HD]>(ta_smem);                 // [REP][HD]
+  uint8_t *tiles = ta_smem + REP * HD * sizeof(float);
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t *kt = tiles + warp * (TT::K_BYTES + TT::V_BYTES), *vt = kt + TT::K_BYTES;
   const int first = cu[b], n = len ? len[b] : cu[b + 1] - cu[b];
   const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
+  if (k_begin >= k_end) {             // a split past the sequence's end: an empty partial for the merge pass
+    if (threadIdx.x < REP) {
+      float *dst = scratch + (((size_t)b * n_q + kvh * REP + threadIdx.x) * n_splits + split) * (HD + 2);
+      dst[0] = -INFINITY;
+      dst[1] = 0.f;
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < REP * HD; i += blockDim.x)
     qs[i / HD][i % HD] = q[((size_t)b * n_q + kvh * REP + i / HD) * HD + i % HD] * scale;
-  __syncthreads();
+
+  // copy rows [c0, c0 + 32) of this KV head into a tile (rows past k_end are skipped and never read)
+  auto issue_tile = [&](const T *base, uint8_t *tile, int stride, int c0) {
+    const int sub = lane % TT::LPR;
+#pragma unroll
+    for (int i = 0; i < TT::NI; ++i) {
+      const int r = i * TT::RPI + lane / TT::LPR, key = c0 + r;
+      if (key < k_end)
+        cp_async16(tile + r * stride + sub * 16,
+                   reinterpret_cast<const uint8_t *>(base + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * HD) + sub * 16);
+    }
+    cp_async_commit();
+  };
+  int c0 = k_begin + warp * 32;
+  if (c0 < k_end) { issue_tile(kc, kt, TT::KSTRIDE, c0); issue_tile(vc, vt, TT::ROW, c0); }
+  __syncthreads();                    // qs
 
   float m[REP], l[REP], acc[REP][4];
 #pragma unroll
   for (int r = 0; r < REP; ++r) { m[r] = -INFINITY; l[r] = 0.f; acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f; }
 
-  for (int c0 = k_begin + warp * 32; c0 < k_end; c0 += TA_WARPS * 32) {
+  for (; c0 < k_end; c0 += TA_WARPS * 32) {
+    const int next = c0 + TA_WARPS * 32;
+    const bool more = next < k_end;
     const int key = c0 + lane;
     const bool valid = key < k_end;
+    cp_async_wait<1>();               // pending groups: K(c0), V(c0) -> K(c0) has landed
+    __syncwarp();
     float sc[REP];
 #pragma unroll
     for (int r = 0; r < REP; ++r) sc[r] = 0.f;
     float v_s = 1.f;     // FP8 cache: this lane's key carries one scale for its K row and one for its V row
     if (valid) {
-      const size_t krow = kv_row_of(blk, blk_stride, b, first, key);
-      const T *kr = kc + (krow * n_kv + kvh) * HD;
+      const uint8_t *kr = kt + lane * TT::KSTRIDE;
       constexpr int V = 16 / sizeof(T);
 #pragma unroll 4
       for (int i = 0; i < HD; i += V) {
-        const uint4 raw = *reinterpret_cast<const uint4 *>(kr + i);
+        const uint4 raw = *reinterpret_cast<const uint4 *>(kr + i * sizeof(T));
         const T *e = reinterpret_cast<const T *>(&raw);
 #pragma unroll
         for (int k = 0; k < V; ++k) {
@@ -316,12 +362,15 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
         }
       }
       if (kscale) {
+        const size_t krow = kv_row_of(blk, blk_stride, b, first, key);
         const float k_s = kscale[krow];
         v_s = vscale[krow];
 #pragma unroll
         for (int r = 0; r < REP; ++r) sc[r] *= k_s;
       }
     }
+    __syncwarp();                     // every lane is done with the K tile
+    if (more) issue_tile(kc, kt, TT::KSTRIDE, next);
     float pe[REP];
 #pragma unroll
     for (int r = 0; r < REP; ++r) {
@@ -334,12 +383,12 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
       m[r] = m_new;
       pe[r] *= v_s;        // (after the row sum: the V row's scale rides on the probability)
     }
+    if (more) cp_async_wait<1>(); else cp_async_wait<0>();     // pending: V(c0) [, K(next)] -> V(c0) has landed
+    __syncwarp();
     const int n_here = min(32, k_end - c0);
-    // (a 32-key chunk never straddles a 128-row page: c0 is a multiple of 32)
-    const T *vbase = vc + (kv_row_of(blk, blk_stride, b, first, c0) * n_kv + kvh) * HD + lane * 4;
 #pragma unroll 4
     for (int i = 0; i < n_here; ++i) {
-      const T *vr = vbase + (size_t)i * n_kv * HD;
+      const T *vr = reinterpret_cast<const T *>(vt + i * TT::ROW) + lane * 4;
       float v0, v1, v2, v3;
       if constexpr (sizeof(T) == 2) {
         const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
@@ -360,24 +409,31 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
         acc[r][2] = fmaf(pi, v2, acc[r][2]); acc[r][3] = fmaf(pi, v3, acc[r][3]);
       }
     }
+    __syncwarp();                     // every lane is done with the V tile
+    if (more) issue_tile(vc, vt, TT::ROW, next);
   }
+  // merge the warps; the tiles are free now (every copy has landed and been consumed)
+  __syncthreads();
+  float *w_m = reinterpret_cast<float *>(tiles);                 // [TA_WARPS][REP]
+  float *w_l = w_m + TA_WARPS * REP;                             // [TA_WARPS][REP]
+  float *w_acc = w_l + TA_WARPS * REP;                           // [TA_WARPS][REP][HD]
 #pragma unroll
   for (int r = 0; r < REP; ++r) {
-    if (lane == 0) { w_m[warp][r] = m[r]; w_l[warp][r] = l[r]; }
-    *reinterpret_cast<float4 *>(&w_acc[warp][r][lane * 4]) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+    if (lane == 0) { w_m[warp * REP + r] = m[r]; w_l[warp * REP + r] = l[r]; }
+    *reinterpret_cast<float4 *>(&w_acc[(warp * REP + r) * HD + lane * 4]) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
   }
   __syncthreads();
   for (int idx = threadIdx.x; idx < REP * HD; idx += blockDim.x) {
     const int r = idx / HD, dd = idx % HD;
     float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < TA_WARPS; ++w) M = fmaxf(M, w_m[w][r]);
+    for (int w = 0; w < TA_WARPS; ++w) M = fmaxf(M, w_m[w * REP + r]);
     float a = 0.f, L = 0.f;
 #pragma unroll
     for (int w = 0; w < TA_WARPS; ++w) {
-      const float f = (w_m[w][r] == -INFINITY) ? 0.f : __expf(w_m[w][r] - M);
-      a += w_acc[w][r][dd] * f;
-      L += w_l[w][r] * f;
+      const float f = (w_m[w * REP + r] == -INFINITY) ? 0.f : __expf(w_m[w * REP + r] - M);
+      a += w_acc[(w * REP + r) * HD + dd] * f;
+      L += w_l[w * REP + r] * f;
     }
     float *dst = scratch + (((size_t)b * n_q + kvh * REP + r) * n_splits + split) * (HD + 2);
     if (dd == 0) { dst[0] = M; dst[1] = L; }
@@ -446,24 +502,44 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
   }
 }
 
-__global__ void tail_attention_merge_kernel(const float *__restrict__ scratch, float *__restrict__ out, int n_q, int hd,
-                                            int n_splits) {
+__global__ void __launch_bounds__(128) tail_attention_merge_kernel(const float *__restrict__ scratch, float *__restrict__ out,
+                                                                   int n_q, int hd, int n_splits) {
+  // block (head, prompt): warp 0 turns the splits' (max, sum) pairs into weights -- all loads issued together --, then
+  // every thread combines its output dims with independent loads (a serial walk over the splits costs a dependent
+  // global-memory round trip per split)
+  __shared__ float wgt[64];
+  __shared__ float inv_l;
   const int h = blockIdx.x, b = blockIdx.y;
   const float *src = scratch + ((size_t)b * n_q + h) * n_splits * (hd + 2);
-  float M = -INFINITY;
-  for (int s = 0; s < n_splits; ++s) M = fmaxf(M, src[(size_t)s * (hd + 2)]);
-  float L = 0.f;
-  for (int s = 0; s < n_splits; ++s) {
-    const float ms = src[(size_t)s * (hd + 2)];
-    L += (ms == -INFINITY) ? 0.f : src[(size_t)s * (hd + 2) + 1] * __expf(ms - M);
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x;
+    float ms[2], ls[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int s = lane + 32 * k;
+      ms[k] = s < n_splits ? src[(size_t)s * (hd + 2)] : -INFINITY;
+      ls[k] = s < n_splits ? src[(size_t)s * (hd + 2) + 1] : 0.f;
+    }
+    const float M = warp_max(fmaxf(ms[0], ms[1]));
+    float L = 0.f;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const float w = (ms[k] == -INFINITY) ? 0.f : __expf(ms[k] - M);
+      if (lane + 32 * k < 64) wgt[lane + 32 * k] = w;
+      L += ls[k] * w;
+    }
+    L = warp_sum(L);
+    if (lane == 0) inv_l = 1.f / L;
   }
+  __syncthreads();
   for (int dd = threadIdx.x; dd < hd; dd += blockDim.x) {
     float a = 0.f;
+#pragma unroll 8
     for (int s = 0; s < n_splits; ++s) {
-      const float ms = src[(size_t)s * (hd + 2)];
-      if (ms != -INFINITY) a += src[(size_t)s * (hd + 2) + 2 + dd] * __expf(ms - M);
+      const float w = wgt[s];
+      if (w != 0.f) a = fmaf(src[(size_t)s * (hd + 2) + 2 + dd], w, a);
     }
-    out[((size_t)b * n_q + h) * hd + dd] = a / L;
+    out[((size_t)b * n_q + h) * hd + dd] = a * inv_l;
   }
 }
 
@@ -485,10 +561,19 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
   const int rep = n_q / n_kv;
   if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
     dim3 grid(n_splits, n_kv, n_seqs);
-    if (rep == 1) tail_attention_group_kernel<T, 1, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 2) tail_attention_group_kernel<T, 2, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else if (rep == 4) tail_attention_group_kernel<T, 4, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
-    else tail_attention_group_kernel<T, 8, 128><<<grid, TA_WARPS * 32, 0, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch);
+    const size_t smem = (size_t)rep * 128 * sizeof(float) + (size_t)TA_WARPS * (TailTile<T>::K_BYTES + TailTile<T>::V_BYTES);
+#define SKV_LAUNCH_GROUP(R)                                                                                                   \
+    do {                                                                                                                      \
+      cudaFuncSetAttribute(tail_attention_group_kernel<T, R, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
+      tail_attention_group_kernel<T, R, 128><<<grid, TA_WARPS * 32, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, \
+                                                                                blk_stride, n_q, n_kv, chunk, n_splits, scale, \
+                                                                                scratch);                                     \
+    } while (0)
+    if (rep == 1) SKV_LAUNCH_GROUP(1);
+    else if (rep == 2) SKV_LAUNCH_GROUP(2);
+    else if (rep == 4) SKV_LAUNCH_GROUP(4);
+    else SKV_LAUNCH_GROUP(8);
+#undef SKV_LAUNCH_GROUP
     tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
     return;
   }

@@ -82,6 +82,33 @@ def test_chunked_prefill_then_decode(shape, dtype, act, kv_bar, lg_bar, l, g):
                 _check_seq(model, shape, ref, b * cap, n + t + 1, kv_bar)
 
 
+@pytest.mark.parametrize("shape,dtype,bar", [(S.TINY, torch.float32, 1e-3), (MID, torch.bfloat16, 0.1)])
+def test_decode_minibatch_on_both_paths(shape, dtype, bar):
+    """A decode-only minibatch of at most 8 sequences runs every layer on the weight-streaming kernels (kernel-mask
+    bit 5); with the bit cleared it takes the general path (128-row GEMM tiles, gathered attention operands).  Both must
+    give the oracle's logits and caches."""
+    import paper_2410_03960_b200 as P
+    seed, lens, l, g, cap = 17, [140, 33, 260], 2, 2, 384
+    w = S.make_weights(shape, seed, dtype, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    toks = [S.token_ids(seed, b, n + 2, shape.vocab) for b, n in enumerate(lens)]
+    out = {}
+    for mask in (39, 7):
+        model = P.SwiftKVModel(shape, w, dtype, cap * len(lens), len(lens), l, g)
+        assert model.set_kernel_mask(mask) == mask
+        model.step(torch.cat([t[:n] for t, n in zip(toks, lens)]), [(n, 0, b * cap, 1) for b, n in enumerate(lens)], l, g)
+        for t in range(2):
+            model.step(torch.stack([toks[b][n + t] for b, n in enumerate(lens)]),
+                       [(1, n + t, b * cap, 1) for b, n in enumerate(lens)], l, g)
+        model.status()
+        out[mask] = to_np(model.first_logits())
+        for b, n in enumerate(lens):
+            ref = O.swiftkv(cfg, ow, toks[b][:n + 2].numpy(), [n + 2], l, g)
+            assert np.max(np.abs(out[mask][b] - ref["logits"][0])) <= bar, (mask, b)
+            _check_seq(model, shape, ref, b * cap, n + 2, 1e-4 if dtype == torch.float32 else 2e-2)
+    assert np.max(np.abs(out[39] - out[7])) <= 2 * bar
+
+
 def test_mixed_minibatch_of_prefill_chunk_and_decode_token():
     """One step carries a decode token of sequence 0 and a prefill chunk of sequence 1; only sequence 0 emits."""
     import paper_2410_03960_b200 as P
