@@ -3,6 +3,7 @@
 // weights from HBM exactly once; attention is one query per (prompt, head) over the cache that the
 // SingleInputKV projection filled.  Activations of this path stay in fp32 (they are tiny), weights and the
 // cache stay in the model dtype.
+#include <cooperative_groups.h>
 #include <mma.h>
 
 #include "common.cuh"
@@ -105,6 +106,10 @@ __global__ void __launch_bounds__(256) skinny_generic_kernel(const float *__rest
 // does not care), which makes those 16 bytes exactly the lane's fragment of two MMAs.  fp32 activations are
 // split into bf16 hi + lo parts (two MMAs), so the activations keep ~16 mantissa bits.
 // A block = 8 warps works on one 16-feature tile with K split across the warps, then reduces in shared memory.
+// Matrices with few output features (N = 4096: 256 tiles) would leave most of the GPU idle and make every warp walk
+// its K range in several dependent batches of loads, so a thread-block CLUSTER of `ks` CTAs shares one tile: each CTA
+// takes 1/ks of K, the partial tiles are written into the first CTA's shared memory over DSMEM and summed there in
+// rank order (deterministic), and that CTA runs the epilogue.
 // ---------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm(
@@ -121,15 +126,19 @@ __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t &hi, ui
 }
 
 constexpr int SK_WARPS = 8;
+constexpr int SK_MAX_CLUSTER = 8;
 
 template <bool SWIGLU>
 __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *__restrict__ act, const bf16 *__restrict__ W,
                                                                    const bf16 *__restrict__ W2, int n_rows, int N, int K,
-                                                                   float *__restrict__ out, int ldo, int mode) {
+                                                                   float *__restrict__ out, int ldo, int mode, int ks) {
+  namespace cg = cooperative_groups;
   __shared__ float red[SK_WARPS][SWIGLU ? 2 : 1][32][4];
+  __shared__ float cred[SK_MAX_CLUSTER][SWIGLU ? 2 : 1][32][4];     // partial tiles of the other CTAs of the cluster
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int n0 = blockIdx.x * 16;
+  const int rank = blockIdx.x % ks;                                 // = rank in the cluster (cluster dims (ks, 1, 1))
+  const int n0 = (blockIdx.x / ks) * 16;
   const bf16 *w_lo = W + (size_t)(n0 + g) * K + 8 * t;          // row g of the tile
   const bf16 *w_hi = W + (size_t)(n0 + g + 8) * K + 8 * t;      // row g + 8
   const bf16 *u_lo = SWIGLU ? W2 + (size_t)(n0 + g) * K + 8 * t : nullptr;
@@ -137,11 +146,13 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
   const float *a_row = act + (size_t)g * K + 8 * t;              // token g
   const bool tok_ok = g < n_rows;
   float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
-  const int steps = K / 32;
+  // this CTA's share of the K steps
+  const int all_steps = K / 32;
+  const int step_lo = (int)((long long)all_steps * rank / ks), steps = (int)((long long)all_steps * (rank + 1) / ks);
   // software pipeline: the loads of U K-steps are issued together before any of their MMAs, so that each lane keeps
   // 2U (4U with SwiGLU) 16-byte weight loads in flight
   constexpr int U = SWIGLU ? 2 : 4;
-  for (int s0 = warp; s0 < steps; s0 += U * SK_WARPS) {
+  for (int s0 = step_lo + warp; s0 < steps; s0 += U * SK_WARPS) {
     uint4 wl[U], wh[U], ul[U], uh[U];
     float4 xa[U], xb[U];
 #pragma unroll
@@ -191,8 +202,8 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
     if (SWIGLU) red[warp][SWIGLU ? 1 : 0][lane][i] = c2[i];
   }
   __syncthreads();
+  float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
   if (warp == 0) {
-    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int w = 0; w < SK_WARPS; ++w)
 #pragma unroll
@@ -200,6 +211,29 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
         s[i] += red[w][0][lane][i];
         if (SWIGLU) s2[i] += red[w][SWIGLU ? 1 : 0][lane][i];
       }
+  }
+  if (ks > 1) {
+    cg::cluster_group cluster = cg::this_cluster();
+    if (warp == 0 && rank != 0) {       // hand this CTA's partial tile to the first CTA of the cluster
+      float *dst = cluster.map_shared_rank(&cred[0][0][0][0], 0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        dst[((rank * (SWIGLU ? 2 : 1) + 0) * 32 + lane) * 4 + i] = s[i];
+        if (SWIGLU) dst[((rank * 2 + 1) * 32 + lane) * 4 + i] = s2[i];
+      }
+    }
+    cluster.sync();
+    if (rank != 0) return;
+    if (warp == 0) {
+      for (int r = 1; r < ks; ++r)      // fixed order: the sum does not depend on which CTA finished first
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          s[i] += cred[r][0][lane][i];
+          if (SWIGLU) s2[i] += cred[r][SWIGLU ? 1 : 0][lane][i];
+        }
+    }
+  }
+  if (warp == 0) {
     // fragment element i: feature n0 + g + 8*(i/2), token 2t + (i%2)
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -220,8 +254,25 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
   if (n_rows <= 0 || N <= 0) return;
   if constexpr (sizeof(T) == 2) {
     if ((K % 32) == 0 && (N % 16) == 0) {
-      if (W2) skinny_mma_kernel<true><<<N / 16, SK_WARPS * 32, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
-      else skinny_mma_kernel<false><<<N / 16, SK_WARPS * 32, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
+      // cluster size: enough CTAs to fill the GPU several times over, at least 2 K steps per warp
+      const int tiles = N / 16, steps = K / 32;
+      int ks = 1;
+      while (ks < SK_MAX_CLUSTER && tiles * ks < 1024 && steps / (2 * ks) >= 2 * SK_WARPS) ks *= 2;
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3((unsigned)(tiles * ks));
+      cfg.blockDim = dim3(SK_WARPS * 32);
+      cfg.dynamicSmemBytes = 0;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = (unsigned)ks;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      const bf16 *w = reinterpret_cast<const bf16 *>(W), *w2 = reinterpret_cast<const bf16 *>(W2);
+      if (W2) cudaLaunchKernelEx(&cfg, skinny_mma_kernel<true>, act, w, w2, n_rows, N, K, out, ldo, mode, ks);
+      else cudaLaunchKernelEx(&cfg, skinny_mma_kernel<false>, act, w, w2, n_rows, N, K, out, ldo, mode, ks);
       return;
     }
   }
