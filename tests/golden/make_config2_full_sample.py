@@ -1,7 +1,7 @@
 """Writes tests/golden/config2_full_sample.npz: sampled outputs of the CPU oracle on the FULL benchmark workload
 (Llama-3.1-8B shape, bf16-valued weights, SwiftKV l = 16, g = 1, 8 prompts with lengths U[2048, 8192], seed 1).
 
-Calls only the oracle and the seeded input generators.  Takes about an hour and ~50 GB of host memory:
+Calls only the oracle and the seeded input generators.  Takes about two hours on 8 cores and ~35 GB of host memory:
     python tests/golden/make_config2_full_sample.py
 Stored (float32): for every prompt the first-token logits at 2048 seeded vocabulary indices plus the arg-max index
 and value; for layers 1, 16, 17 and 32 the K and V rows of four positions per prompt (first, last and two seeded

@@ -197,8 +197,6 @@ def _check_full_size_samples(model, lens, shape, logits):
     per prompt, the arg-max, and K / V rows of layers 1, 16, 17, 32 at four positions per prompt (first, last, two
     inside) -- the last positions and the logits depend on every token of the prompt."""
     path = os.path.join(os.path.dirname(__file__), "golden", "config2_full_sample.npz")
-    if not os.path.exists(path):      # (an hour of CPU time to produce; the prefix check above does not need it)
-        pytest.skip("tests/golden/config2_full_sample.npz is missing: run tests/golden/make_config2_full_sample.py")
     gold = np.load(path)
     assert list(gold["lens"]) == list(lens)
     for b in range(len(lens)):
