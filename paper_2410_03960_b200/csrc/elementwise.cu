@@ -111,9 +111,50 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
       orow[i] = from_f<T>(xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f));
   }
 }
+// Rows of exactly 256 * 4 * NV floats (4096: NV = 4, 8192: NV = 8) with 16-bit output: each thread keeps its NV float4
+// in registers between the sum of squares and the scaling, so the row is read from global memory exactly once.
+template <typename TG, typename T, int NV>
+__global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
+                                                          T *__restrict__ out, float eps) {
+  constexpr int D = 256 * 4 * NV;
+  const size_t row = blockIdx.x;
+  const float4 *xr = reinterpret_cast<const float4 *>(x + row * D);
+  __shared__ float red[8];
+  float4 v[NV];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    v[k] = xr[threadIdx.x + 256 * k];
+    ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float rstd = rsqrtf(tot / (float)D + eps);
+  uint2 *orow = reinterpret_cast<uint2 *>(out + row * D);
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int i4 = threadIdx.x + 256 * k;
+    float g0 = 1.f, g1 = 1.f, g2 = 1.f, g3 = 1.f;
+    if (gamma) {
+      const uint2 graw = *reinterpret_cast<const uint2 *>(gamma + 4 * i4);       // TG is a 16-bit type here
+      const TG *g = reinterpret_cast<const TG *>(&graw);
+      g0 = to_f(g[0]); g1 = to_f(g[1]); g2 = to_f(g[2]); g3 = to_f(g[3]);
+    }
+    T o4[4] = {from_f<T>(v[k].x * rstd * g0), from_f<T>(v[k].y * rstd * g1), from_f<T>(v[k].z * rstd * g2), from_f<T>(v[k].w * rstd * g3)};
+    orow[i4] = *reinterpret_cast<uint2 *>(o4);
+  }
+}
 template <typename TG, typename TO>
 void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st) {
   if (rows <= 0) return;
+  if constexpr (sizeof(TG) == 2 && sizeof(TO) == 2) {
+    if (d == 4096) { rmsnorm_reg_kernel<TG, TO, 4><<<rows, 256, 0, st>>>(x, gamma, out, eps); return; }
+    if (d == 8192) { rmsnorm_reg_kernel<TG, TO, 8><<<rows, 256, 0, st>>>(x, gamma, out, eps); return; }
+  }
   rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps);
 }
 template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t);
