@@ -1,5 +1,7 @@
 """Writes tests/golden/config2_full_sample.npz: sampled outputs of the CPU oracle on the FULL benchmark workload
 (Llama-3.1-8B shape, bf16-valued weights, SwiftKV l = 16, g = 1, 8 prompts with lengths U[2048, 8192], seed 1).
+With `--sweep N` it writes tests/golden/sweep_n<N>_full_sample.npz instead: one prompt of N tokens, seed 4, l = 16 (a
+point of the prompt-length sweep; N = 4096 takes about a quarter of an hour).
 
 Calls only the oracle and the seeded input generators.  Takes about two hours on 8 cores and ~35 GB of host memory:
     python tests/golden/make_config2_full_sample.py
@@ -34,10 +36,12 @@ def sample_plan(lens, vocab):
 
 def main():
     shape = S.LLAMA31_8B
-    lens = S.uniform_lengths(SEED, N_PROMPTS, LEN_LO, LEN_HI)
-    tok = S.make_prompts(SEED, lens, shape.vocab).numpy()
+    seed, lens, name = SEED, S.uniform_lengths(SEED, N_PROMPTS, LEN_LO, LEN_HI), "config2_full_sample.npz"
+    if len(sys.argv) > 2 and sys.argv[1] == "--sweep":
+        seed, lens, name = 4, [int(sys.argv[2])], f"sweep_n{int(sys.argv[2])}_full_sample.npz"
+    tok = S.make_prompts(seed, lens, shape.vocab).numpy()
     t0 = time.time()
-    w = S.make_weights(shape, SEED, torch.bfloat16, "cpu")
+    w = S.make_weights(shape, seed, torch.bfloat16, "cpu")
     print(f"weights {time.time() - t0:.0f} s", flush=True)
 
     def f64(t):
@@ -61,7 +65,7 @@ def main():
     for j in LAYERS:
         out[f"K{j}"] = ref["K"][j][rows].astype(np.float32)
         out[f"V{j}"] = ref["V"][j][rows].astype(np.float32)
-    np.savez(os.path.join(os.path.dirname(os.path.abspath(__file__)), "config2_full_sample.npz"), **out)
+    np.savez(os.path.join(os.path.dirname(os.path.abspath(__file__)), name), **out)
     print(f"done {time.time() - t0:.0f} s", flush=True)
 
 

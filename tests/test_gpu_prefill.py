@@ -188,16 +188,15 @@ def test_config2_full_size_prefix_parity_and_determinism():
     model.prefill(tok, lens, l, g)
     model.status()
     assert torch.equal(logits1, model.first_logits())
-    _check_full_size_samples(model, lens, shape, to_np(logits1))
+    _check_full_size_samples(model, lens, to_np(logits1), "config2_full_sample.npz")
 
 
-def _check_full_size_samples(model, lens, shape, logits):
-    """Sampled outputs of the oracle's FULL-size run of the same workload (tests/golden/config2_full_sample.npz, written
-    by tests/golden/make_config2_full_sample.py from the oracle alone): first-token logits at 2048 vocabulary entries
-    per prompt, the arg-max, and K / V rows of layers 1, 16, 17, 32 at four positions per prompt (first, last, two
-    inside) -- the last positions and the logits depend on every token of the prompt."""
-    path = os.path.join(os.path.dirname(__file__), "golden", "config2_full_sample.npz")
-    gold = np.load(path)
+def _check_full_size_samples(model, lens, logits, file):
+    """Sampled outputs of the oracle's FULL-size run of the same workload (tests/golden/*_full_sample.npz, written by
+    tests/golden/make_config2_full_sample.py from the oracle alone): first-token logits at 2048 vocabulary entries per
+    prompt, the arg-max, and K / V rows of layers 1, 16, 17, 32 at four positions per prompt (first, last, two inside)
+    -- the last positions and the logits depend on every token of the prompt."""
+    gold = np.load(os.path.join(os.path.dirname(__file__), "golden", file))
     assert list(gold["lens"]) == list(lens)
     for b in range(len(lens)):
         got = logits[b][gold["vocab_idx"][b]]
@@ -215,6 +214,18 @@ def _check_full_size_samples(model, lens, shape, logits):
         K, V, _ = model.kv_cache_view(j)
         assert rel_l2(to_np(K[rows]), gold[f"K{j}"]) <= 2e-2, (j, rel_l2(to_np(K[rows]), gold[f"K{j}"]))
         assert rel_l2(to_np(V[rows]), gold[f"V{j}"]) <= 2e-2, (j, rel_l2(to_np(V[rows]), gold[f"V{j}"]))
+
+
+def test_sweep_point_n4096_full_length_against_oracle_samples():
+    """A point of the prompt-length sweep (one prompt of 4096 tokens, seed 4, l = 16) at full length and depth."""
+    import paper_2410_03960_b200 as P
+    shape, seed, l, g, lens = S.LLAMA31_8B, 4, 16, 1, [4096]
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    _check_full_size_samples(model, lens, to_np(model.first_logits()), "sweep_n4096_full_sample.npz")
 
 
 @pytest.mark.skipif(os.environ.get("SWIFTKV_RUN_SLOW") != "1",
