@@ -366,15 +366,11 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
   if (get_tmap(&tq, q, n_tokens, (uint64_t)n_q * hd, (uint64_t)n_q * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
   if (get_tmap(&tk, k, kv_rows, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
   if (get_tmap(&tv, v, kv_rows, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attention_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM) != cudaSuccess)
-      return SWIFTKV_ERR_CUDA;
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_kernel<false, false>), ATT_SMEM) ||
+      ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_kernel<true, false>), ATT_SMEM) ||
+      ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_kernel<false, true>), ATT_SMEM) ||
+      ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_kernel<true, true>), ATT_SMEM))
+    return SWIFTKV_ERR_CUDA;
   AttnParams p{};
   p.cu = cu_seqlens; p.k_row0 = k_row0; p.kv_len = kv_len; p.blk = blk; p.blk_stride = blk_stride; p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
   p.max_tiles = (max_seq_len + BQ - 1) / BQ;

@@ -94,6 +94,10 @@ __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, fl
 }
 #endif
 
+// raises a kernel's dynamic shared-memory limit once per (device, kernel) -- the attribute belongs to the device's copy of
+// the function, so a process that drives several GPUs sets it on each; returns 0 on success
+int ensure_dynamic_smem(const void *kernel, int bytes);
+
 // sets the calling thread's swiftkv_last_error() text and returns `code` (defined with the C ABI)
 int32_t report_error(int32_t code, const char *msg);
 

@@ -98,6 +98,20 @@ int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint
   return 0;
 }
 
+int ensure_dynamic_smem(const void *kernel, int bytes) {
+  static std::mutex mu;
+  static std::unordered_map<const void *, unsigned long long> done;   // kernel -> bit mask of devices already set
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+  const unsigned long long bit = 1ull << (dev & 63);
+  std::lock_guard<std::mutex> lock(mu);
+  unsigned long long &mask = done[kernel];
+  if (mask & bit) return 0;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return -1;
+  mask |= bit;
+  return 0;
+}
+
 int num_sms() {
   static int n = 0;
   if (!n) {
@@ -609,11 +623,7 @@ int launch_pair(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &
                 const GemmTcParams &p, int tiles, cudaStream_t st) {
   using L = PairSmem<STAGES>;
   auto kern = gemm_tc_pair_kernel<STAGES, EPI>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess) return SWIFTKV_ERR_CUDA;
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem(reinterpret_cast<const void *>(kern), L::TOTAL)) return SWIFTKV_ERR_CUDA;
   int pairs = num_sms() / 2;
   if (tiles < pairs) pairs = tiles;
   kern<<<2 * pairs, GEMM_THREADS, L::TOTAL, st>>>(a, b0, b1, b2, p);
@@ -625,11 +635,7 @@ int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b
                const GemmTcParams &p, cudaStream_t st) {
   using L = SmemLayout<BN, STAGES>;
   auto kern = gemm_tc_kernel<BN, STAGES, EPI>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::TOTAL) != cudaSuccess) return SWIFTKV_ERR_CUDA;
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem(reinterpret_cast<const void *>(kern), L::TOTAL)) return SWIFTKV_ERR_CUDA;
   const int tiles = p.num_m_blocks * p.num_n_blocks;
   const int grid = tiles < num_sms() ? tiles : num_sms();
   kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(a, b0, b1, b2, p);

@@ -615,11 +615,7 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
     const size_t smem = (size_t)rep * 128 * sizeof(float) + (size_t)TA_WARPS * (TailTile<T>::K_BYTES + TailTile<T>::V_BYTES);
 #define SKV_LAUNCH_GROUP(R)                                                                                                   \
     do {                                                                                                                      \
-      static bool attr_set = false;   /* (one device per process: the attribute is set once per instantiation) */             \
-      if (!attr_set) {                                                                                                        \
-        cudaFuncSetAttribute(tail_attention_group_kernel<T, R, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-        attr_set = true;                                                                                                      \
-      }                                                                                                                       \
+      ensure_dynamic_smem(reinterpret_cast<const void *>(tail_attention_group_kernel<T, R, 128>), (int)smem);                 \
       tail_attention_group_kernel<T, R, 128><<<grid, TA_WARPS * 32, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, \
                                                                                 blk_stride, n_q, n_kv, chunk, n_splits, scale, \
                                                                                 scratch);                                     \
