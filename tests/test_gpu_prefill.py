@@ -219,6 +219,31 @@ def _check_full_size_samples(model, lens, logits, file):
         assert rel_l2(to_np(V[rows]), gold[f"V{j}"]) <= 2e-2, (j, rel_l2(to_np(V[rows]), gold[f"V{j}"]))
 
 
+def test_longest_sweep_point_65536_tokens_prefix_parity_and_determinism():
+    """The largest single prompt of the sweep (65536 tokens: 512 query tiles, 64 key splits in the last-token attention):
+    cache rows of the first tokens against the oracle's run of the truncated prompt (causality), finite logits,
+    run-to-run bitwise determinism."""
+    import paper_2410_03960_b200 as P
+    shape, seed, l, g, n, prefix = S.LLAMA31_8B, 4, 16, 1, 65536, 24
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    tok = S.make_prompts(seed, [n], shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, n, 1, l, g)
+    model.prefill(tok, [n], l, g)
+    model.status()
+    logits1 = model.first_logits().clone()
+    assert torch.isfinite(logits1).all()
+    ref = O.swiftkv(oracle_config(shape), oracle_weights(w), tok[:prefix].numpy(), [prefix], l, g)
+    for j in range(shape.n_layers):
+        K, V, _ = model.kv_cache_view(j)
+        assert K.shape[0] == n
+        assert rel_l2(to_np(K[:prefix]), ref["K"][j]) <= 2e-2, j
+        assert rel_l2(to_np(V[:prefix]), ref["V"][j]) <= 2e-2, j
+        assert torch.isfinite(K[-128:].float()).all() and torch.isfinite(V[-128:].float()).all()
+    model.prefill(tok, [n], l, g)
+    model.status()
+    assert torch.equal(logits1, model.first_logits())
+
+
 def test_sweep_point_n4096_full_length_against_oracle_samples():
     """A point of the prompt-length sweep (one prompt of 4096 tokens, seed 4, l = 16) at full length and depth."""
     import paper_2410_03960_b200 as P
