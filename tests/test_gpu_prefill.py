@@ -244,16 +244,17 @@ def test_longest_sweep_point_65536_tokens_prefix_parity_and_determinism():
     assert torch.equal(logits1, model.first_logits())
 
 
-def test_sweep_point_n4096_full_length_against_oracle_samples():
-    """A point of the prompt-length sweep (one prompt of 4096 tokens, seed 4, l = 16) at full length and depth."""
+@pytest.mark.parametrize("n", [4096, 16384])
+def test_sweep_point_full_length_against_oracle_samples(n):
+    """Points of the prompt-length sweep (one prompt of n tokens, seed 4, l = 16) at full length and depth."""
     import paper_2410_03960_b200 as P
-    shape, seed, l, g, lens = S.LLAMA31_8B, 4, 16, 1, [4096]
+    shape, seed, l, g, lens = S.LLAMA31_8B, 4, 16, 1, [n]
     w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
     tok = S.make_prompts(seed, lens, shape.vocab)
     model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
     model.prefill(tok, lens, l, g)
     model.status()
-    _check_full_size_samples(model, lens, to_np(model.first_logits()), "sweep_n4096_full_sample.npz")
+    _check_full_size_samples(model, lens, to_np(model.first_logits()), f"sweep_n{n}_full_sample.npz")
 
 
 @pytest.mark.skipif(os.environ.get("SWIFTKV_RUN_SLOW") != "1",
