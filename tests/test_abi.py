@@ -51,6 +51,16 @@ def test_workspace_bytes_validates_and_accounts_for_acrosskv(lib):
         with pytest.raises(SwiftKVError) as e:
             workspace_bytes(shape, torch.bfloat16, **args)
         assert e.value.code == -1
+    # FP8 cache (appendix, KV quantization): one byte per element plus one fp32 scale per token row and plane; with
+    # 4-way AcrossKV the paper's 68.75 % reduction against the 16-bit cache of the unmodified model (scales aside)
+    from paper_2410_03960_b200 import KV_FP8
+    _, kv8 = workspace_bytes(shape, torch.bfloat16, 4096, 4, 16, 4, KV_FP8)
+    assert kv8 == (16 + 4) * 2 * (4096 * 1024 + 4096 * 4)
+    assert abs((1 - (kv8 - (16 + 4) * 2 * 4096 * 4) / full) - 0.6875) < 1e-12
+    with pytest.raises(SwiftKVError):
+        workspace_bytes(shape, torch.bfloat16, 4096, 4, 16, 4, 7)       # unknown cache format
+    assert lib.swiftkv_quantize_rows_fp8(None, 1, 1, None, None, None, None) == -1
+    assert lib.swiftkv_tail_attention_fp8(None, None, None, None, None, None, None, 1, 1, 1, 1, 2, None, 0, None) == -1
     odd = S.ModelShape(512, 256, 4, 8, 3, 32, 688, 10000.0)
     with pytest.raises(SwiftKVError):
         workspace_bytes(odd, torch.float32, 128, 2, 2, 1)
