@@ -293,10 +293,10 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
           float4 *px = reinterpret_cast<float4 *>(reinterpret_cast<float *>(p.out.p0) + (size_t)row * p.out.ld0 + col);
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            float4 v = px[i];
+            float4 v = __ldcs(px + i);          // streamed once per projection: do not displace the weight tiles in L2
             v.x += __uint_as_float(r[4 * i]); v.y += __uint_as_float(r[4 * i + 1]);
             v.z += __uint_as_float(r[4 * i + 2]); v.w += __uint_as_float(r[4 * i + 3]);
-            px[i] = v;
+            __stcs(px + i, v);
           }
         } else {
           bf16 *dstp;
