@@ -152,25 +152,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       // ------------------------------------------------------------ MMA issuer
       constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);   // Q, K both K-major (head dim contiguous)
       constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);    // V is MN-major (head dim contiguous, keys = K)
-      const uint32_t q_addr = tc::smem_u32(smem + SM_Q);
+      // shared-memory descriptors differ only in their address field (bytes >> 4): one per buffer, plus step offsets
+      const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_Q), 16, 1024);
+      const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_K), 16, 1024);
+      const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_V), CHUNK_BYTES, 1024);
       auto issue_qk = [&](int w, int s) {   // S_w = Q_w K^T : 8 steps of 16 along the head dim
-        const uint32_t a0 = q_addr + w * TILE_BYTES, b0 = tc::smem_u32(smem + SM_K + s * TILE_BYTES);
+        const uint64_t qd = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), kd = k_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+        const uint32_t d = tmem_base + w * 128;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * CHUNK_BYTES + (kk & 3) * 32;
-          tc::umma_ss(tmem_base + w * 128, tc::umma_desc_sw128(a0 + off, 16, 1024), tc::umma_desc_sw128(b0 + off, 16, 1024),
-                      idesc_qk, kk != 0);
+          const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
+          tc::umma_ss(d, qd + off, kd + off, idesc_qk, kk != 0);
         }
       };
       // O_w (+)= P_w V : 8 steps of 16 keys, issued in two halves so that the first 64 keys can run on the tensor
       // pipe while the softmax warps still exponentiate the last 64
       auto issue_pv = [&](int w, int s, bool accumulate, int half) {
-        const uint32_t b0 = tc::smem_u32(smem + SM_V + s * TILE_BYTES);
+        const uint64_t vd = v_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+        const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4) {
           const int kk = half * 4 + k4;
-          tc::umma_ts(tmem_base + 256 + w * 128, tmem_base + w * 128 + kk * 8,
-                      tc::umma_desc_sw128(b0 + kk * 16 * 128, CHUNK_BYTES, 1024), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+          tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
         }
       };
       bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) &&
