@@ -176,48 +176,51 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
         }
       };
-      bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) &&
-                wait_or_abort(tc::smem_u32(&k_full[0]), 0, abort_flag, p.status);
+      // barrier addresses once (this thread's instruction stream is on the critical path of every key tile)
+      const uint32_t b_kf = tc::smem_u32(&k_full[0]), b_ke = tc::smem_u32(&k_empty[0]), b_vf = tc::smem_u32(&v_full[0]),
+                     b_ve = tc::smem_u32(&v_empty[0]), b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]),
+                     b_p2 = tc::smem_u32(&p_ready2[0]);
+      bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) && wait_or_abort(b_kf, 0, abort_flag, p.status);
       if (ok) {
         tc::tc_fence_after_sync();
         issue_qk(0, 0);
-        tc::umma_commit(tc::smem_u32(&s_full[0]));
+        tc::umma_commit(b_sf);
         issue_qk(1, 0);
-        tc::umma_commit(tc::smem_u32(&s_full[1]));
-        tc::umma_commit(tc::smem_u32(&k_empty[0]));
+        tc::umma_commit(b_sf + 8);
+        tc::umma_commit(b_ke);
       }
       for (int j = 0; j < n_kv_tiles && ok; ++j) {
-        const int s = j & 1, s1 = (j + 1) & 1;
-        const uint32_t ph = (j >> 1) & 1, ph1 = ((j + 1) >> 1) & 1;
+        const int s = j & 1, s1 = s ^ 1;
+        const uint32_t ph = (j >> 1) & 1, ph1 = ((j + 1) >> 1) & 1, pj = j & 1;
         const bool more = j + 1 < n_kv_tiles;
-        if (!wait_or_abort(tc::smem_u32(&v_full[s]), ph, abort_flag, p.status)) { ok = false; break; }
-        if (!wait_or_abort(tc::smem_u32(&p_ready[0]), j & 1, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_or_abort(b_vf + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_or_abort(b_p1, pj, abort_flag, p.status)) { ok = false; break; }
         tc::tc_fence_after_sync();
         issue_pv(0, s, j > 0, 0);
         if (SPLIT_P) {
-          if (!wait_or_abort(tc::smem_u32(&p_ready2[0]), j & 1, abort_flag, p.status)) { ok = false; break; }
+          if (!wait_or_abort(b_p2, pj, abort_flag, p.status)) { ok = false; break; }
           tc::tc_fence_after_sync();
         }
         issue_pv(0, s, j > 0, 1);
         if (more) {
-          if (!wait_or_abort(tc::smem_u32(&k_full[s1]), ph1, abort_flag, p.status)) { ok = false; break; }
+          if (!wait_or_abort(b_kf + 8 * s1, ph1, abort_flag, p.status)) { ok = false; break; }
           tc::tc_fence_after_sync();
           issue_qk(0, s1);
-          tc::umma_commit(tc::smem_u32(&s_full[0]));
+          tc::umma_commit(b_sf);
         }
-        if (!wait_or_abort(tc::smem_u32(&p_ready[1]), j & 1, abort_flag, p.status)) { ok = false; break; }
+        if (!wait_or_abort(b_p1 + 8, pj, abort_flag, p.status)) { ok = false; break; }
         tc::tc_fence_after_sync();
         issue_pv(1, s, j > 0, 0);
         if (SPLIT_P) {
-          if (!wait_or_abort(tc::smem_u32(&p_ready2[1]), j & 1, abort_flag, p.status)) { ok = false; break; }
+          if (!wait_or_abort(b_p2 + 8, pj, abort_flag, p.status)) { ok = false; break; }
           tc::tc_fence_after_sync();
         }
         issue_pv(1, s, j > 0, 1);
-        tc::umma_commit(tc::smem_u32(&v_empty[s]));
+        tc::umma_commit(b_ve + 8 * s);
         if (more) {
           issue_qk(1, s1);
-          tc::umma_commit(tc::smem_u32(&s_full[1]));
-          tc::umma_commit(tc::smem_u32(&k_empty[s1]));
+          tc::umma_commit(b_sf + 8);
+          tc::umma_commit(b_ke + 8 * s1);
         }
       }
       if (ok) tc::umma_commit(tc::smem_u32(o_full));
