@@ -152,12 +152,12 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
   // software pipeline: the loads of U K-steps are issued together before any of their MMAs, so that each lane keeps
   // 2U (4U with SwiGLU) 16-byte weight loads in flight
   constexpr int U = SWIGLU ? 2 : 4;
-  for (int s0 = step_lo + warp; s0 < steps; s0 += U * SK_WARPS) {
+  for (int s0 = step_lo + warp * U; s0 < steps; s0 += U * SK_WARPS) {
     uint4 wl[U], wh[U], ul[U], uh[U];
     float4 xa[U], xb[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int s = s0 + u * SK_WARPS;
+      const int s = s0 + u;
       const bool on = s < steps;
       const int kb = on ? s * 32 : 0;
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);

@@ -1,7 +1,7 @@
 """Timing of the serving-style entry point (swiftkv_step) on the benchmark model: chunked prefill, decode steps,
 paged cache rows and the FP8 cache.  Prints one JSON line per measurement (CUDA events, after a warm-up pass).
 
-    python -m paper_2410_03960_b200.step_bench [--kv-format fp8] [--chunks 8192,2048,512] [--decode-steps 6]
+    python -m paper_2410_03960_b200.step_bench [--kv-format fp8] [--chunks 8192,2048,512] [--decode-steps 6] [--kernel-mask M]
 
 Workload: the benchmark's batch (Llama-3.1-8B shape, random bf16 weights, 8 prompts with lengths U[2048, 8192],
 seed 1, l = 16, g = 1).  A chunked prefill feeds every prompt `chunk` tokens per step (all prompts that still have
@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--kv-format", choices=("model", "fp8"), default="model")
     ap.add_argument("--chunks", default="8192,2048,512")
     ap.add_argument("--decode-steps", type=int, default=6)
+    ap.add_argument("--kernel-mask", type=int, default=None, help="swiftkv_set_kernel_mask value (default: the library's)")
     args = ap.parse_args()
     shape = S.LLAMA31_8B
     lens = S.uniform_lengths(SEED, N_PROMPTS, LEN_LO, LEN_HI)
@@ -37,6 +38,8 @@ def main():
     fmt = P.KV_FP8 if args.kv_format == "fp8" else P.KV_MODEL_DTYPE
     cap = PAGES_PER_SEQ * 128
     model = P.SwiftKVModel(shape, w, torch.bfloat16, cap * n_seq, n_seq, SWIFT_LAYER, GROUP, kv_format=fmt)
+    if args.kernel_mask is not None:
+        model.set_kernel_mask(args.kernel_mask)
     # paged: sequence b owns pages b, b + 8, b + 16, ... (interleaved with the other sequences' pages)
     pages = [[b + n_seq * i for i in range(PAGES_PER_SEQ)] for b in range(n_seq)]
 
