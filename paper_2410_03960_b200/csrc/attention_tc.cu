@@ -13,6 +13,8 @@
 // Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each (all 512).  Every wait is bounded.
 #include <cstdlib>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -45,15 +47,19 @@ struct AttnParams {
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
   if (tc::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!tc::mbar_try_wait(bar, parity)) {
-    if (*abort_flag) return false;
-    if (clock64() - t0 > tc::WAIT_LIMIT_CLOCKS) {
-      *abort_flag = 1;
-      atomicOr(status, STATUS_TIMEOUT);
-      return false;
+  // try_wait itself suspends the thread for a while, so the loop is not a busy spin; the abort flag and the clock
+  // are looked at only every 32nd round to keep the time from "barrier completed" to "waiter runs" short
+  for (unsigned spins = 1;; ++spins) {
+    if (tc::mbar_try_wait(bar, parity)) return true;
+    if ((spins & 31u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > tc::WAIT_LIMIT_CLOCKS) {
+        *abort_flag = 1;
+        atomicOr(status, STATUS_TIMEOUT);
+        return false;
+      }
     }
   }
-  return true;
 }
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -148,74 +154,67 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      // ------------------------------------------------------------ MMA issuer
-      constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);   // Q, K both K-major (head dim contiguous)
-      constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);    // V is MN-major (head dim contiguous, keys = K)
-      // shared-memory descriptors differ only in their address field (bytes >> 4): one per buffer, plus step offsets
-      const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_Q), 16, 1024);
-      const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_K), 16, 1024);
-      const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_V), CHUNK_BYTES, 1024);
-      auto issue_qk = [&](int w, int s) {   // S_w = Q_w K^T : 8 steps of 16 along the head dim
-        const uint64_t qd = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), kd = k_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
-        const uint32_t d = tmem_base + w * 128;
+    // ---------------------------------------------------------------- MMA issuer
+    // The whole warp walks this code and one elected lane issues every tcgen05.mma and commit: the lane's instruction
+    // stream is on the critical path of every key tile (an MMA must leave every 64 clocks), and inside a one-lane
+    // branch each descriptor would be per-thread arithmetic.  The key-tile loop is unrolled by the two ring stages so
+    // that stage offsets and barrier parities are constants.
+    const bool leader = tc::elect_one();
+    constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);   // Q, K both K-major (head dim contiguous)
+    constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);    // V is MN-major (head dim contiguous, keys = K)
+    // shared-memory descriptors differ only in their address field (bytes >> 4): one per buffer, plus step offsets
+    const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_Q), 16, 1024);
+    const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_K), 16, 1024);
+    const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_V), CHUNK_BYTES, 1024);
+    auto issue_qk = [&](int w, int s) {   // S_w = Q_w K^T : 8 steps of 16 along the head dim
+      const uint64_t qd = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), kd = k_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+      const uint32_t d = tmem_base + w * 128;
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
-          tc::umma_ss(d, qd + off, kd + off, idesc_qk, kk != 0);
-        }
-      };
-      // O_w (+)= P_w V : 8 steps of 16 keys, issued in two halves so that the first 64 keys can run on the tensor
-      // pipe while the softmax warps still exponentiate the last 64
-      auto issue_pv = [&](int w, int s, bool accumulate, int half) {
-        const uint64_t vd = v_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
-        const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
-#pragma unroll
-        for (int k4 = 0; k4 < 4; ++k4) {
-          const int kk = half * 4 + k4;
-          tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
-        }
-      };
-      // barrier addresses once (this thread's instruction stream is on the critical path of every key tile)
-      const uint32_t b_kf = tc::smem_u32(&k_full[0]), b_ke = tc::smem_u32(&k_empty[0]), b_vf = tc::smem_u32(&v_full[0]),
-                     b_ve = tc::smem_u32(&v_empty[0]), b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]),
-                     b_p2 = tc::smem_u32(&p_ready2[0]);
-      bool ok = wait_or_abort(tc::smem_u32(q_full), 0, abort_flag, p.status) && wait_or_abort(b_kf, 0, abort_flag, p.status);
-      if (ok) {
-        tc::tc_fence_after_sync();
-        issue_qk(0, 0);
-        tc::umma_commit(b_sf);
-        issue_qk(1, 0);
-        tc::umma_commit(b_sf + 8);
-        tc::umma_commit(b_ke);
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
+        tc::umma_ss(d, qd + off, kd + off, idesc_qk, kk != 0);
       }
-      for (int j = 0; j < n_kv_tiles && ok; ++j) {
-        const int s = j & 1, s1 = s ^ 1;
-        const uint32_t ph = (j >> 1) & 1, ph1 = ((j + 1) >> 1) & 1, pj = j & 1;
-        const bool more = j + 1 < n_kv_tiles;
-        if (!wait_or_abort(b_vf + 8 * s, ph, abort_flag, p.status)) { ok = false; break; }
-        if (!wait_or_abort(b_p1, pj, abort_flag, p.status)) { ok = false; break; }
-        tc::tc_fence_after_sync();
-        issue_pv(0, s, j > 0, 0);
-        if (SPLIT_P) {
-          if (!wait_or_abort(b_p2, pj, abort_flag, p.status)) { ok = false; break; }
-          tc::tc_fence_after_sync();
-        }
-        issue_pv(0, s, j > 0, 1);
-        if (more) {
-          if (!wait_or_abort(b_kf + 8 * s1, ph1, abort_flag, p.status)) { ok = false; break; }
-          tc::tc_fence_after_sync();
+    };
+    // O_w (+)= P_w V : 8 steps of 16 keys, issued in two halves so that the first 64 keys can run on the tensor
+    // pipe while the softmax warps still exponentiate the last 64
+    auto issue_pv = [&](int w, int s, bool accumulate, int half) {
+      const uint64_t vd = v_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+      const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int kk = half * 4 + k4;
+        tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+      }
+    };
+    const uint32_t b_kf = tc::smem_u32(&k_full[0]), b_ke = tc::smem_u32(&k_empty[0]), b_vf = tc::smem_u32(&v_full[0]),
+                   b_ve = tc::smem_u32(&v_empty[0]), b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]),
+                   b_p2 = tc::smem_u32(&p_ready2[0]);
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+      const bool ok = wait_or_abort(bar, parity, abort_flag, p.status);
+      tc::tc_fence_after_sync();
+      return ok;
+    };
+    // key tile j in ring stage s = j & 1 (a compile-time constant here)
+    auto tile = [&](auto stage, int j) -> bool {
+      constexpr int s = decltype(stage)::value, s1 = s ^ 1;
+      const uint32_t ph = (j >> 1) & 1, ph1 = ph ^ s;     // fill parity of stage s for tile j, of stage s1 for tile j + 1
+      const bool more = j + 1 < n_kv_tiles, acc = j > 0;
+      if (!wait(b_vf + 8 * s, ph) || !wait(b_p1, s)) return false;
+      if (leader) issue_pv(0, s, acc, 0);
+      if (SPLIT_P && !wait(b_p2, s)) return false;
+      if (leader) issue_pv(0, s, acc, 1);
+      if (more) {
+        if (!wait(b_kf + 8 * s1, ph1)) return false;
+        if (leader) {
           issue_qk(0, s1);
           tc::umma_commit(b_sf);
         }
-        if (!wait_or_abort(b_p1 + 8, pj, abort_flag, p.status)) { ok = false; break; }
-        tc::tc_fence_after_sync();
-        issue_pv(1, s, j > 0, 0);
-        if (SPLIT_P) {
-          if (!wait_or_abort(b_p2 + 8, pj, abort_flag, p.status)) { ok = false; break; }
-          tc::tc_fence_after_sync();
-        }
-        issue_pv(1, s, j > 0, 1);
+      }
+      if (!wait(b_p1 + 8, s)) return false;
+      if (leader) issue_pv(1, s, acc, 0);
+      if (SPLIT_P && !wait(b_p2 + 8, s)) return false;
+      if (leader) {
+        issue_pv(1, s, acc, 1);
         tc::umma_commit(b_ve + 8 * s);
         if (more) {
           issue_qk(1, s1);
@@ -223,8 +222,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           tc::umma_commit(b_ke + 8 * s1);
         }
       }
-      if (ok) tc::umma_commit(tc::smem_u32(o_full));
+      return true;
+    };
+    bool ok = wait(tc::smem_u32(q_full), 0) && wait(b_kf, 0);
+    if (ok && leader) {
+      issue_qk(0, 0);
+      tc::umma_commit(b_sf);
+      issue_qk(1, 0);
+      tc::umma_commit(b_sf + 8);
+      tc::umma_commit(b_ke);
     }
+    for (int j = 0; j < n_kv_tiles && ok; j += 2) {
+      ok = tile(std::integral_constant<int, 0>{}, j);
+      if (ok && j + 1 < n_kv_tiles) ok = tile(std::integral_constant<int, 1>{}, j + 1);
+    }
+    if (ok && leader) tc::umma_commit(tc::smem_u32(o_full));
+    __syncwarp();
   } else {
     // -------------------------------------------------------------- softmax warps: head w, one row per thread
     const int w = (warp - 2) >> 2;
