@@ -459,29 +459,31 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   if (bt.decode) {
     const int rows = T_tok;
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
-    auto store_kv = [&](int slot) {      // ky (rotated), vy -> the cache rows of the new tokens in `slot`
-      Scope s(m, st, SWIFTKV_KC_TAIL, fp8 ? 4 : 2);
+    const TailRope q_rope{b.last_pos, b.cos_tab, b.sin_tab};     // the queries are rotated inside the attention kernel
+    auto store_kv = [&](int slot) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
       if (fp8) {
+        Scope s(m, st, SWIFTKV_KC_TAIL, 5);
+        launch_rope<float>(ky, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st);
         launch_scatter_rows<T>(ky, kst, nullptr, rows, dkv, st);    // rows are quantized from the model dtype
         launch_scatter_rows<T>(vy, vst, nullptr, rows, dkv, st);
         launch_quantize_rows_fp8<T, T>(kst, rows, dkv, b.slot, k_codes(slot), k_scale(slot), (T *)nullptr, st);
         launch_quantize_rows_fp8<T, T>(vst, rows, dkv, b.slot, v_codes(slot), v_scale(slot), (T *)nullptr, st);
       } else {
-        launch_scatter_rows<T>(ky, kv + (size_t)slot * 2 * plane, b.slot, rows, dkv, st);
-        launch_scatter_rows<T>(vy, kv + (size_t)slot * 2 * plane + plane, b.slot, rows, dkv, st);
+        Scope s(m, st, SWIFTKV_KC_TAIL);
+        launch_store_kv_rows<T>(ky, vy, kv + (size_t)slot * 2 * plane, kv + (size_t)slot * 2 * plane + plane, b.slot, b.last_pos,
+                                b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st);
       }
     };
-    auto project_kv = [&](const swiftkv_layer_weights &lw) {   // hy -> ky (rotated at the tokens' positions), vy
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wk, nullptr, rows, dkv, d, ky, dkv, OUT_STORE_F32, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wv, nullptr, rows, dkv, d, vy, dkv, OUT_STORE_F32, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(ky, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st); }
+    const int kv_launches = (sizeof(T) == 2 && d % 32 == 0 && dkv % 16 == 0) ? 1 : 2;
+    auto project_kv = [&](const swiftkv_layer_weights &lw) {   // hy -> ky, vy: both projections in one launch
+      Scope s(m, st, SWIFTKV_KC_TAIL, kv_launches);
+      launch_skinny_gemm_dual<T>(hy, (const T *)lw.wk, (const T *)lw.wv, rows, dkv, d, ky, vy, dkv, st);
     };
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx, y, rows, d, st); }
     for (int j = 0; j < l; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
       project_kv(lw);
       store_kv(j);
       {
@@ -489,11 +491,11 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
         if (fp8)
           launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(j), (const fp8e4 *)v_codes(j), k_scale(j), v_scale(j), ay, b.emit_row0,
                                        b.emit_len, blk_emit, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim,
-                                       b.tail_scratch, st);
+                                       b.tail_scratch, st, q_rope);
         else
           launch_tail_attention<T>(qy, kv + (size_t)j * 2 * plane, kv + (size_t)j * 2 * plane + plane, nullptr, nullptr, ay, b.emit_row0,
                                    b.emit_len, blk_emit, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim,
-                                   b.tail_scratch, st);
+                                   b.tail_scratch, st, q_rope);
       }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
@@ -676,17 +678,17 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_rope<float>(qy, 0, 1, b.last_pos + r0, nullptr, b.cos_tab, b.sin_tab, rows, c.n_q_heads, c.head_dim, st); }
       {
         Scope s(m, st, SWIFTKV_KC_TAIL, 2);
         const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
+        const TailRope q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab};    // the queries are rotated inside the attention kernel
         if (fp8)
           launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(slot), (const fp8e4 *)v_codes(slot), k_scale(slot), v_scale(slot), ay,
                                        b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads,
-                                       c.n_kv_heads, c.head_dim, b.tail_scratch, st);
+                                       c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
         else
           launch_tail_attention<T>(qy, Ks, Vs, nullptr, nullptr, ay, b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len,
-                                   c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st);
+                                   c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
       }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }

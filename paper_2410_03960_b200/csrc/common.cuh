@@ -139,6 +139,11 @@ void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows
 // fp32 rows -> rows slot_map[r] (null: r) of a [*, width] plane of type T
 template <typename T>
 void launch_scatter_rows(const float *src, T *dst, const int32_t *slot_map, int rows, int width, cudaStream_t st);
+// a decode step's new K / V rows (fp32, K not yet rotated) -> rotary embedding of K at pos[r] -> rows slot_map[r] of the
+// K and V planes in the cache's element type, one launch
+template <typename T>
+void launch_store_kv_rows(const float *ky, const float *vy, T *k_plane, T *v_plane, const int32_t *slot_map, const int32_t *pos,
+                          const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st);
 void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, double theta, cudaStream_t st);
 // dst[r, c] = w[r, c] * gamma[c]   (gain of the input norm folded into a projection weight, Sec. 3.5)
 template <typename T, typename TO>
@@ -201,6 +206,16 @@ void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, i
 template <typename T>
 void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
                         int mode, cudaStream_t st);
+// two projections of the same rows in one launch: out[r, n] = act W^T, out2[r, n] = act W2^T (a decode step's K and V)
+template <typename T>
+void launch_skinny_gemm_dual(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, float *out2,
+                             int ldo, cudaStream_t st);
+// optional rotary embedding of the query rows inside the single-query attention (row b sits at position pos[b]; the
+// tables are those of launch_rope): saves a launch per layer on the last-token path
+struct TailRope {
+  const int32_t *pos = nullptr;
+  const float *cos_tab = nullptr, *sin_tab = nullptr;
+};
 // one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
 // row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
@@ -208,6 +223,6 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
                            const int32_t *row0, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st);
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailRope rope = TailRope());
 
 }  // namespace skv

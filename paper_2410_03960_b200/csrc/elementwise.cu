@@ -278,6 +278,36 @@ void launch_scatter_rows(const float *src, T *dst, const int32_t *slot_map, int 
 template void launch_scatter_rows<float>(const float *, float *, const int32_t *, int, int, cudaStream_t);
 template void launch_scatter_rows<bf16>(const float *, bf16 *, const int32_t *, int, int, cudaStream_t);
 
+template <typename T>
+__global__ void __launch_bounds__(256) store_kv_rows_kernel(const float *__restrict__ ky, const float *__restrict__ vy,
+                                                            T *__restrict__ k_plane, T *__restrict__ v_plane,
+                                                            const int32_t *__restrict__ slot_map, const int32_t *__restrict__ pos,
+                                                            const float *__restrict__ cos_tab, const float *__restrict__ sin_tab,
+                                                            int n_heads, int hd) {
+  const int r = blockIdx.x, half = hd >> 1, width = n_heads * hd;
+  const size_t orow = slot_map ? (size_t)slot_map[r] : (size_t)r;
+  const float *k = ky + (size_t)r * width, *v = vy + (size_t)r * width;
+  T *ko = k_plane + orow * width, *vo = v_plane + orow * width;
+  const int p = pos[r];
+  for (int idx = threadIdx.x; idx < n_heads * half; idx += blockDim.x) {     // same arithmetic as rope_kernel
+    const int h = idx / half, i = idx % half;
+    const float c = cos_tab[(size_t)p * half + i], s = sin_tab[(size_t)p * half + i];
+    const float a = k[h * hd + i], b = k[h * hd + i + half];
+    ko[h * hd + i] = from_f<T>(a * c - b * s);
+    ko[h * hd + i + half] = from_f<T>(b * c + a * s);
+  }
+  for (int i = threadIdx.x; i < width; i += blockDim.x) vo[i] = from_f<T>(v[i]);
+}
+template <typename T>
+void launch_store_kv_rows(const float *ky, const float *vy, T *k_plane, T *v_plane, const int32_t *slot_map, const int32_t *pos,
+                          const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st) {
+  if (rows > 0) store_kv_rows_kernel<T><<<rows, 256, 0, st>>>(ky, vy, k_plane, v_plane, slot_map, pos, cos_tab, sin_tab, n_heads, hd);
+}
+template void launch_store_kv_rows<float>(const float *, const float *, float *, float *, const int32_t *, const int32_t *,
+                                          const float *, const float *, int, int, int, cudaStream_t);
+template void launch_store_kv_rows<bf16>(const float *, const float *, bf16 *, bf16 *, const int32_t *, const int32_t *,
+                                         const float *, const float *, int, int, int, cudaStream_t);
+
 // dst[r, c] = w[r, c] * gamma[c], product in fp32, one rounding to the output type
 template <typename T, typename TO>
 __global__ void fold_kernel(const T *__restrict__ w, const T *__restrict__ gamma, TO *__restrict__ dst, long long n, int cols) {

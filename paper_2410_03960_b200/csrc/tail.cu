@@ -128,11 +128,14 @@ __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t &hi, ui
 constexpr int SK_WARPS = 8;
 constexpr int SK_MAX_CLUSTER = 8;
 
-template <bool SWIGLU>
+// EPI: 0 = one weight matrix; 1 = two, combined as silu(act W^T) * (act W2^T); 2 = two, stored to out and out2
+template <int EPI>
 __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *__restrict__ act, const bf16 *__restrict__ W,
                                                                    const bf16 *__restrict__ W2, int n_rows, int N, int K,
-                                                                   float *__restrict__ out, int ldo, int mode, int ks) {
+                                                                   float *__restrict__ out, float *__restrict__ out2, int ldo,
+                                                                   int mode, int ks) {
   namespace cg = cooperative_groups;
+  constexpr bool SWIGLU = EPI != 0;      // (two accumulators: the name is kept from the first user)
   __shared__ float red[SK_WARPS][SWIGLU ? 2 : 1][32][4];
   __shared__ float cred[SK_MAX_CLUSTER][SWIGLU ? 2 : 1][32][4];     // partial tiles of the other CTAs of the cluster
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -240,12 +243,38 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
       const int n = n0 + g + 8 * (i >> 1), r = 2 * t + (i & 1);
       if (r < n_rows && n < N) {
         float v = s[i];
-        if (SWIGLU) v = v / (1.f + __expf(-v)) * s2[i];
+        if (EPI == 1) v = v / (1.f + __expf(-v)) * s2[i];
         float *o = out + (size_t)r * ldo + n;
         *o = (mode == OUT_RESID_ADD_F32) ? *o + v : v;
+        if (EPI == 2) out2[(size_t)r * ldo + n] = s2[i];
       }
     }
   }
+}
+
+// cluster size: enough CTAs to fill the GPU several times over, at least 2 K steps per warp
+static int skinny_cluster(int tiles, int steps) {
+  int ks = 1;
+  while (ks < SK_MAX_CLUSTER && tiles * ks < 1024 && steps / (2 * ks) >= 2 * SK_WARPS) ks *= 2;
+  return ks;
+}
+template <int EPI>
+static void launch_skinny_mma(const float *act, const bf16 *w, const bf16 *w2, int n_rows, int N, int K, float *out, float *out2,
+                              int ldo, int mode, cudaStream_t st) {
+  const int tiles = N / 16, ks = skinny_cluster(tiles, K / 32);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(tiles * ks));
+  cfg.blockDim = dim3(SK_WARPS * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)ks;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, skinny_mma_kernel<EPI>, act, w, w2, n_rows, N, K, out, out2, ldo, mode, ks);
 }
 
 template <typename T>
@@ -254,25 +283,9 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
   if (n_rows <= 0 || N <= 0) return;
   if constexpr (sizeof(T) == 2) {
     if ((K % 32) == 0 && (N % 16) == 0) {
-      // cluster size: enough CTAs to fill the GPU several times over, at least 2 K steps per warp
-      const int tiles = N / 16, steps = K / 32;
-      int ks = 1;
-      while (ks < SK_MAX_CLUSTER && tiles * ks < 1024 && steps / (2 * ks) >= 2 * SK_WARPS) ks *= 2;
-      cudaLaunchConfig_t cfg{};
-      cfg.gridDim = dim3((unsigned)(tiles * ks));
-      cfg.blockDim = dim3(SK_WARPS * 32);
-      cfg.dynamicSmemBytes = 0;
-      cfg.stream = st;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = (unsigned)ks;
-      attr[0].val.clusterDim.y = 1;
-      attr[0].val.clusterDim.z = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
       const bf16 *w = reinterpret_cast<const bf16 *>(W), *w2 = reinterpret_cast<const bf16 *>(W2);
-      if (W2) cudaLaunchKernelEx(&cfg, skinny_mma_kernel<true>, act, w, w2, n_rows, N, K, out, ldo, mode, ks);
-      else cudaLaunchKernelEx(&cfg, skinny_mma_kernel<false>, act, w, w2, n_rows, N, K, out, ldo, mode, ks);
+      if (W2) launch_skinny_mma<1>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st);
+      else launch_skinny_mma<0>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st);
       return;
     }
   }
@@ -280,6 +293,22 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
   if (blocks > 148 * 8) blocks = 148 * 8;
   skinny_generic_kernel<T><<<blocks, 256, 0, st>>>(act, W, W2, n_rows, N, K, out, ldo, mode);
 }
+template <typename T>
+void launch_skinny_gemm_dual(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, float *out2,
+                             int ldo, cudaStream_t st) {
+  if (n_rows <= 0 || N <= 0) return;
+  if constexpr (sizeof(T) == 2) {
+    if ((K % 32) == 0 && (N % 16) == 0) {
+      launch_skinny_mma<2>(act, reinterpret_cast<const bf16 *>(W), reinterpret_cast<const bf16 *>(W2), n_rows, N, K, out, out2, ldo,
+                           OUT_STORE_F32, st);
+      return;
+    }
+  }
+  launch_skinny_gemm<T>(act, W, nullptr, n_rows, N, K, out, ldo, OUT_STORE_F32, st);
+  launch_skinny_gemm<T>(act, W2, nullptr, n_rows, N, K, out2, ldo, OUT_STORE_F32, st);
+}
+template void launch_skinny_gemm_dual<float>(const float *, const float *, const float *, int, int, int, float *, float *, int, cudaStream_t);
+template void launch_skinny_gemm_dual<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, float *, int, cudaStream_t);
 template void launch_skinny_gemm<float>(const float *, const float *, const float *, int, int, int, float *, int, int, cudaStream_t);
 template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, int, int, cudaStream_t);
 
@@ -340,12 +369,22 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// element dd of a query row, rotated to the row's position when the caller asks for it (same arithmetic as rope_kernel)
+__device__ __forceinline__ float load_query(const float *__restrict__ qr, int dd, int hd, int b, const TailRope &rope) {
+  const float v = qr[dd];
+  if (!rope.pos) return v;
+  const int half = hd >> 1, i = dd < half ? dd : dd - half;
+  const size_t t = (size_t)rope.pos[b] * half + i;
+  const float c = rope.cos_tab[t], s = rope.sin_tab[t];
+  return dd < half ? v * c - qr[dd + half] * s : v * c + qr[dd - half] * s;
+}
+
 template <typename T, int REP, int HD>
 __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
     const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
     const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk, int n_splits, float scale,
-    float *__restrict__ scratch) {
+    float *__restrict__ scratch, TailRope rope) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
   using TT = TailTile<T>;
   extern __shared__ __align__(16) uint8_t ta_smem[];
@@ -365,7 +404,7 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     return;
   }
   for (int i = threadIdx.x; i < REP * HD; i += blockDim.x)
-    qs[i / HD][i % HD] = q[((size_t)b * n_q + kvh * REP + i / HD) * HD + i % HD] * scale;
+    qs[i / HD][i % HD] = load_query(q + ((size_t)b * n_q + kvh * REP + i / HD) * HD, i % HD, HD, b, rope) * scale;
 
   // copy rows [c0, c0 + 32) of this KV head into a tile (rows past k_end are skipped and never read)
   auto issue_tile = [&](const T *base, uint8_t *tile, int stride, int c0) {
@@ -499,7 +538,7 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
     const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
     const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int hd, int chunk, int n_splits, float scale,
-    float *__restrict__ scratch) {
+    float *__restrict__ scratch, TailRope rope) {
   extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -510,7 +549,7 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const int h = kvh * rep + hw;
     float *qs = sm + hw * hd;
     const float *qr = q + ((size_t)b * n_q + h) * hd;
-    for (int i = lane; i < hd; i += 32) qs[i] = qr[i] * scale;
+    for (int i = lane; i < hd; i += 32) qs[i] = load_query(qr, i, hd, b, rope) * scale;
     __syncwarp();
     float m = -INFINITY, l = 0.f;
     float acc[MAX_E];
@@ -604,7 +643,7 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
                            const int32_t *cu_seqlens, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st) {
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailRope rope) {
   if (n_seqs <= 0) return;
   const int chunk = tail_chunk(max_seq_len);
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
@@ -618,7 +657,7 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
       ensure_dynamic_smem(reinterpret_cast<const void *>(tail_attention_group_kernel<T, R, 128>), (int)smem);                 \
       tail_attention_group_kernel<T, R, 128><<<grid, TA_WARPS * 32, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, \
                                                                                 blk_stride, n_q, n_kv, chunk, n_splits, scale, \
-                                                                                scratch);                                     \
+                                                                                scratch, rope);                               \
     } while (0)
     if (rep == 1) SKV_LAUNCH_GROUP(1);
     else if (rep == 2) SKV_LAUNCH_GROUP(2);
@@ -631,20 +670,20 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
   const int threads = 32 * (rep < 8 ? rep : 8);
   const size_t smem = (size_t)rep * hd * sizeof(float);
   dim3 grid(n_splits, n_kv, n_seqs);
-  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
-  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch);
+  if (hd <= 32) tail_attention_partial_kernel<T, 1><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch, rope);
+  else if (hd <= 64) tail_attention_partial_kernel<T, 2><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch, rope);
+  else if (hd <= 128) tail_attention_partial_kernel<T, 4><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch, rope);
+  else tail_attention_partial_kernel<T, 8><<<grid, threads, smem, st>>>(q, kc, vc, kscale, vscale, cu_seqlens, len, blk, blk_stride, n_q, n_kv, hd, chunk, n_splits, scale, scratch, rope);
   tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
 }
 template void launch_tail_attention<float>(const float *, const float *, const float *, const float *, const float *, float *,
                                            const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                           float *, cudaStream_t);
+                                           float *, cudaStream_t, TailRope);
 template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, const float *, const float *, float *,
                                           const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                          float *, cudaStream_t);
+                                          float *, cudaStream_t, TailRope);
 template void launch_tail_attention<fp8e4>(const float *, const fp8e4 *, const fp8e4 *, const float *, const float *, float *,
                                            const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                           float *, cudaStream_t);
+                                           float *, cudaStream_t, TailRope);
 
 }  // namespace skv
