@@ -237,9 +237,11 @@ int32_t swiftkv_last_launch_count(const swiftkv_model *m);
 
 /* Select kernel families (debug / comparison): bit 0 = tensor-core GEMMs, bit 1 = tensor-core attention,
  * bit 2 = CTA-pair (cta_group::2) form of the projection GEMMs, bit 3 = CTA-pair form of the gate/up GEMM too,
+ * bit 4 = the tensor-core attention runs as one persistent CTA per SM over a work list that the host balances from the
+ * sequence lengths (longest item first, each to the least loaded CTA) instead of one CTA per work item,
  * bit 5 = decode minibatches (at most 8 sequences, one new token each) run every layer on the weight-streaming
  * kernels of the last-token path instead of 128-row GEMM tiles.
- * Default 39: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
+ * Default 55: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
 int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
 /* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention

@@ -71,6 +71,7 @@ struct Buffers {
   float *tail_scratch;
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
+  int32_t *att_off, *att_items;   // schedule of the persistent attention kernel: [ATT_MAX_CTAS + 1] offsets, items
   int32_t *slot;            // [T] cache row of every new token
   int32_t *kv_row0, *kv_len;   // [B] first cache row / number of cached + new tokens of every sequence
   int32_t *kcu;             // [B+1] offsets of the sequences in the gathered half K / V copy (chunked steps)
@@ -98,7 +99,8 @@ struct swiftkv_model {
   int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;   // rows in use per cache plane, sequences with logits
   int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
-  int kernel_mask = 39;
+  int kernel_mask = 55;
+  int n_sms = 0;
   int act_format = SWIFTKV_ACT_F16;
   // profiling
   bool profiling = false;
@@ -129,6 +131,11 @@ static int32_t check_cfg(const swiftkv_config *c, int max_tokens, int max_seqs, 
   return SWIFTKV_OK;
 }
 
+// persistent attention kernel: at most this many CTAs; one item per (128-query tile, pair of query heads)
+constexpr int ATT_MAX_CTAS = 1024;
+static size_t att_max_items(const swiftkv_config &c, int T, int B) {
+  return ((size_t)T / 128 + (size_t)B) * (size_t)((c.n_q_heads + 1) / 2);
+}
 static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, Carve &cv, Buffers &b) {
   const size_t E = dsize(c.dtype);
   const size_t d = c.hidden, dq = (size_t)c.n_q_heads * c.head_dim, F = c.ffn;
@@ -172,6 +179,8 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   const size_t pages = ((size_t)T + PAGE_ROWS - 1) / PAGE_ROWS;
   b.blk = (int32_t *)cv.take((size_t)B * pages * 4);
   b.blk_emit = (int32_t *)cv.take((size_t)B * pages * 4);
+  b.att_off = (int32_t *)cv.take((size_t)(ATT_MAX_CTAS + 1) * 4);
+  b.att_items = (int32_t *)cv.take(att_max_items(c, T, B) * 4);
   b.status = (unsigned int *)cv.take(256);
   b.cos_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
   b.sin_tab = (float *)cv.take((size_t)T * (c.head_dim / 2) * 4);
@@ -252,6 +261,10 @@ extern "C" int32_t swiftkv_model_load(const swiftkv_config *cfg, const swiftkv_w
   Carve cv(workspace);
   carve_all(*cfg, max_tokens, max_seqs, m->fold_capacity_elems, cv, m->b);
   if (cudaGetDevice(&m->device) != cudaSuccess) { delete m; return fail(SWIFTKV_ERR_CUDA, "cudaGetDevice failed"); }
+  if (cudaDeviceGetAttribute(&m->n_sms, cudaDevAttrMultiProcessorCount, m->device) != cudaSuccess || m->n_sms < 1) {
+    delete m;
+    return fail(SWIFTKV_ERR_CUDA, "cannot read the SM count");
+  }
   // the cache starts as zeros: attention tiles may touch rows past a sequence's end (masked to probability 0), which
   // must never hold NaN / Inf bit patterns
   cudaError_t e = cudaMemsetAsync(kv_cache, 0, (size_t)m->slot_capacity * slot_bytes, 0);
@@ -356,6 +369,7 @@ struct Batch {
   int max_kv;         // longest cached + new length
   int total_kv;       // sum of cached + new lengths
   bool plain;
+  int att_ctas;       // > 0: the device holds a schedule for that many persistent attention CTAs
   bool paged;         // sequences own lists of 128-row pages instead of one contiguous region
   int blk_stride;     // pages per sequence in the device block tables
   bool decode;        // at most 8 sequences, one new token each, all emitting: every layer runs on the weight-streaming
@@ -390,6 +404,8 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const bool use_w16 = act_f16 && (m->kernel_mask & 1) && tc_gemm_supported(T_tok, dq, d) && tc_gemm_supported(T_tok, d, dq) &&
                        tc_gemm_supported(T_tok, d, F) && (dkv % 256 == 0) && (dq % 256 == 0) && c.head_dim == 128;
   const bool attn_tc = sizeof(T) == 2 && (m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim);
+  AttnSchedule att_sched;
+  if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; }
   const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
   __half *wq16 = nullptr, *wk16 = nullptr, *wv16 = nullptr, *wo16 = nullptr, *wg16 = nullptr, *wu16 = nullptr, *wd16 = nullptr;
   auto w16_select = [&](int buf) {
@@ -564,7 +580,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       if constexpr (sizeof(T) == 2) {
         if (tc_path) {
           rc = launch_attention_tc(q, act_f16, kd, vd, attn, b.cu, kr0, kv_len, nullptr, 0, B, T_tok, bt.plain ? T_tok : bt.total_kv,
-                                   bt.max_new, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st);
+                                   bt.max_new, c.n_q_heads, c.n_kv_heads, c.head_dim, b.status, st, att_sched);
           if (rc == SWIFTKV_OK) done = true;
           else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
         }
@@ -594,7 +610,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
           // (the gathered half copies are contiguous: only a direct read of the cache follows the block tables)
           const int32_t *ablk = (act_f16 && !bt.plain) ? nullptr : blk;
           rc = launch_attention_tc(q, act_f16, kk, vv, attn, b.cu, kr0, kv_len, ablk, bt.blk_stride, B, T_tok, kv_rows, bt.max_new, c.n_q_heads,
-                                   c.n_kv_heads, c.head_dim, b.status, st);
+                                   c.n_kv_heads, c.head_dim, b.status, st, att_sched);
           if (rc == SWIFTKV_OK) done = true;
           else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "attention launch failed");
         }
@@ -802,6 +818,18 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
     }
     CUDA_TRY(cudaMemcpyAsync(b.blk, tb.data(), tb.size() * 4, cudaMemcpyHostToDevice, st));
     CUDA_TRY(cudaMemcpyAsync(b.blk_emit, te.data(), te.size() * 4, cudaMemcpyHostToDevice, st));
+  }
+  bt.att_ctas = 0;
+  if ((m->kernel_mask & 16) && (m->kernel_mask & 2) && !bt.decode && c.dtype == SWIFTKV_DTYPE_BF16 &&
+      tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim)) {
+    // the persistent attention kernel's work list, balanced here where the lengths are known
+    const int n_ctas = std::min(m->n_sms, ATT_MAX_CTAS);
+    std::vector<int32_t> n_new(B), n_past(B), off(n_ctas + 1), items(att_max_items(c, m->max_tokens, m->max_seqs));
+    for (int i = 0; i < B; ++i) { n_new[i] = seqs[i].n_new; n_past[i] = seqs[i].n_past; }
+    const int n_items = attention_schedule(n_new.data(), n_past.data(), B, c.n_q_heads, n_ctas, off.data(), items.data());
+    CUDA_TRY(cudaMemcpyAsync(b.att_off, off.data(), off.size() * 4, cudaMemcpyHostToDevice, st));
+    if (n_items > 0) CUDA_TRY(cudaMemcpyAsync(b.att_items, items.data(), (size_t)n_items * 4, cudaMemcpyHostToDevice, st));
+    bt.att_ctas = n_ctas;
   }
   CUDA_TRY(cudaMemcpyAsync(b.cu, cu, (size_t)(B + 1) * 4, cudaMemcpyHostToDevice, st));
   CUDA_TRY(cudaMemcpyAsync(b.pos, pos, (size_t)T * 4, cudaMemcpyHostToDevice, st));

@@ -11,7 +11,14 @@
 // Online softmax keeps a per-row reference max that only moves when the running max grows by more than 2^8
 // (then O_w is rescaled in tensor memory); the final O_w / l_w is exact for any such reference.
 // Tensor memory: S0 | S1 | O0 | O1, 128 fp32 columns each (all 512).  Every wait is bounded.
+// Two kernels share this design: one CTA per work item (used when only the device knows the lengths), and a persistent
+// one that walks a host-balanced list of items and overlaps an item's set-up with the previous item's epilogue.
+#include <algorithm>
 #include <cstdlib>
+#include <functional>
+#include <queue>
+#include <utility>
+#include <vector>
 
 #include <type_traits>
 
@@ -368,7 +375,371 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Persistent form: one CTA per SM walks a list of work items that the host balanced (longest first, each to the least
+// loaded CTA), so that a CTA's fixed cost -- tensor-memory allocation, barrier set-up, Q and first K loads, the first
+// Q K^T -- is paid once or hides behind the previous item's last softmax and epilogue: the producer fetches the next
+// item's Q as soon as the current item's last Q K^T has retired, and the MMA warp issues the next item's first Q K^T
+// while the softmax warps still normalise and store the current output.  Barriers, tensor memory and the K / V rings
+// live across items; every role keeps running counts of items (`it`) and key tiles (`gk`) for the barrier parities.
+//   sched_off[c] .. sched_off[c + 1] : this CTA's items in sched_items, as indices in the heavy-first item order
+// ---------------------------------------------------------------------------------------------------------
+struct AttnItem {
+  int b, qt, h0, kvh, n, past, k0, n_kv_tiles, q_row0;
+};
+__device__ __forceinline__ void decode_item(const AttnParams &p, int w, AttnItem &it) {
+  const int n_pairs = p.n_q >> 1;
+  const int per_tile = p.n_seqs * n_pairs;
+  it.qt = p.max_tiles - 1 - w / per_tile;
+  const int rem = w % per_tile;
+  it.b = rem / n_pairs;
+  const int tok0 = p.cu[it.b];
+  it.n = p.cu[it.b + 1] - tok0;
+  it.k0 = p.k_row0 ? p.k_row0[it.b] : tok0;
+  it.past = p.kv_len ? p.kv_len[it.b] - it.n : 0;
+  it.h0 = (rem % n_pairs) * 2;
+  it.kvh = it.h0 / (p.n_q / p.n_kv);
+  it.n_kv_tiles = (it.past + min(it.n, (it.qt + 1) * BQ) - 1) / BKV + 1;
+  it.q_row0 = tok0 + it.qt * BQ;
+}
+
+template <bool ACT_F16>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attention_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                               const __grid_constant__ CUtensorMap tmV, AttnParams p, const int32_t *__restrict__ sched_off,
+                               const int32_t *__restrict__ sched_items) {
+  const int i_begin = sched_off[blockIdx.x], i_end = sched_off[blockIdx.x + 1];
+  if (i_begin >= i_end) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM_BAR);
+  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7, *s_full = bars + 9,
+           *p_ready = bars + 11, *p_ready2 = bars + 13, *o_full = bars + 15;
+  uint64_t *q_empty = bars + 16;      // every Q K^T of the item has retired: Q may be overwritten
+  uint64_t *o_empty = bars + 17;      // the softmax warps have read the item's O out of tensor memory (8 arrivals)
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 18);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(q_full), 1);
+    for (int s = 0; s < 2; ++s) {
+      tc::mbar_init(tc::smem_u32(&k_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&k_empty[s]), 1);
+      tc::mbar_init(tc::smem_u32(&v_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&v_empty[s]), 1);
+      tc::mbar_init(tc::smem_u32(&s_full[s]), 1);
+      tc::mbar_init(tc::smem_u32(&p_ready[s]), 4);
+      tc::mbar_init(tc::smem_u32(&p_ready2[s]), 4);
+    }
+    tc::mbar_init(tc::smem_u32(o_full), 1);
+    tc::mbar_init(tc::smem_u32(q_empty), 1);
+    tc::mbar_init(tc::smem_u32(o_empty), 8);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmQ);
+    tc::tma_prefetch_desc(&tmK);
+    tc::tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), 512);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ TMA producer
+      int gk = 0;
+      bool ok = true;
+      AttnItem im, nx;
+      decode_item(p, sched_items[i_begin], nx);
+      for (int i = i_begin; i < i_end && ok; ++i) {
+        const int it = i - i_begin;
+        im = nx;
+        if (i + 1 < i_end) decode_item(p, sched_items[i + 1], nx);     // the next item's description: loads in flight meanwhile
+        if (!wait_or_abort(tc::smem_u32(q_empty), (it & 1) ^ 1, abort_flag, p.status)) break;
+        const uint32_t qb = tc::smem_u32(q_full);
+        tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
+        for (int w = 0; w < 2; ++w)
+          for (int c = 0; c < 2; ++c)
+            tc::tma_load_2d(tc::smem_u32(smem + SM_Q + w * TILE_BYTES + c * CHUNK_BYTES), &tmQ, qb, (im.h0 + w) * HD + c * 64, im.q_row0);
+        for (int j = 0; j < im.n_kv_tiles; ++j, ++gk) {
+          const int s = gk & 1;
+          const uint32_t ph = (gk >> 1) & 1;
+          const int krow = p.blk ? p.blk[(size_t)im.b * p.blk_stride + j] * BKV : im.k0 + j * BKV;
+          if (!wait_or_abort(tc::smem_u32(&k_empty[s]), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t kb = tc::smem_u32(&k_full[s]);
+          tc::mbar_expect_tx(kb, TILE_BYTES);
+          for (int c = 0; c < 2; ++c)
+            tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, im.kvh * HD + c * 64, krow);
+          if (!wait_or_abort(tc::smem_u32(&v_empty[s]), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t vb = tc::smem_u32(&v_full[s]);
+          tc::mbar_expect_tx(vb, TILE_BYTES);
+          for (int c = 0; c < 2; ++c)
+            tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, im.kvh * HD + c * 64, krow);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (warp-uniform, one elected lane)
+    const bool leader = tc::elect_one();
+    constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);
+    constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);
+    const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_Q), 16, 1024);
+    const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_K), 16, 1024);
+    const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_V), CHUNK_BYTES, 1024);
+    auto issue_qk = [&](int w, int s) {
+      const uint64_t qd = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), kd = k_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+      const uint32_t d = tmem_base + w * 128;
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
+        tc::umma_ss(d, qd + off, kd + off, idesc_qk, kk != 0);
+      }
+    };
+    auto issue_pv = [&](int w, int s, bool accumulate, int half) {
+      const uint64_t vd = v_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
+      const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int kk = half * 4 + k4;
+        tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+      }
+    };
+    const uint32_t b_kf = tc::smem_u32(&k_full[0]), b_ke = tc::smem_u32(&k_empty[0]), b_vf = tc::smem_u32(&v_full[0]),
+                   b_ve = tc::smem_u32(&v_empty[0]), b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]),
+                   b_p2 = tc::smem_u32(&p_ready2[0]), b_qe = tc::smem_u32(q_empty);
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+      const bool ok = wait_or_abort(bar, parity, abort_flag, p.status);
+      tc::tc_fence_after_sync();
+      return ok;
+    };
+    int gk = 0;
+    bool ok = true;
+    AttnItem im, nx;
+    decode_item(p, sched_items[i_begin], nx);
+    for (int i = i_begin; i < i_end && ok; ++i) {
+      const int it = i - i_begin;
+      im = nx;
+      if (i + 1 < i_end) decode_item(p, sched_items[i + 1], nx);
+      const int n_kv_tiles = im.n_kv_tiles;
+      // the item's first Q K^T: S_w is free as soon as the previous item's last P_w V was issued (the tensor pipe runs in
+      // order); it runs while the softmax warps still store the previous item's output
+      ok = wait(tc::smem_u32(q_full), it & 1) && wait(b_kf + 8 * (gk & 1), (gk >> 1) & 1);
+      if (!ok) break;
+      if (leader) {
+        issue_qk(0, gk & 1);
+        tc::umma_commit(b_sf);
+        issue_qk(1, gk & 1);
+        tc::umma_commit(b_sf + 8);
+        tc::umma_commit(b_ke + 8 * (gk & 1));
+        if (n_kv_tiles == 1) tc::umma_commit(b_qe);
+      }
+      // O_w is overwritten by this item's first P V: the previous item's output must have been read out
+      if (!wait(tc::smem_u32(o_empty), (it & 1) ^ 1)) { ok = false; break; }
+      for (int j = 0; j < n_kv_tiles; ++j, ++gk) {
+        const int s = gk & 1, s1 = s ^ 1;
+        const uint32_t ph = (gk >> 1) & 1, ph1 = ph ^ s, pp = gk & 1;
+        const bool more = j + 1 < n_kv_tiles, acc = j > 0;
+        if (!wait(b_vf + 8 * s, ph) || !wait(b_p1, pp)) { ok = false; break; }
+        if (leader) issue_pv(0, s, acc, 0);
+        if (!wait(b_p2, pp)) { ok = false; break; }
+        if (leader) issue_pv(0, s, acc, 1);
+        if (more) {
+          if (!wait(b_kf + 8 * s1, ph1)) { ok = false; break; }
+          if (leader) {
+            issue_qk(0, s1);
+            tc::umma_commit(b_sf);
+          }
+        }
+        if (!wait(b_p1 + 8, pp)) { ok = false; break; }
+        if (leader) issue_pv(1, s, acc, 0);
+        if (!wait(b_p2 + 8, pp)) { ok = false; break; }
+        if (leader) {
+          issue_pv(1, s, acc, 1);
+          tc::umma_commit(b_ve + 8 * s);
+          if (more) {
+            issue_qk(1, s1);
+            tc::umma_commit(b_sf + 8);
+            tc::umma_commit(b_ke + 8 * s1);
+            if (j + 2 == n_kv_tiles) tc::umma_commit(b_qe);     // the item's last Q K^T is in the pipe
+          }
+        }
+      }
+      if (ok && leader) tc::umma_commit(tc::smem_u32(o_full));
+    }
+    __syncwarp();
+  } else {
+    // -------------------------------------------------------------- softmax warps: head w, one row per thread
+    const int w = (warp - 2) >> 2;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t t_s = tmem_base + lane_base + w * 128;
+    const uint32_t t_o = tmem_base + lane_base + 256 + w * 128;
+    const float c = p.scale_log2;
+    int gk = 0;
+    bool ok = true;
+    int w_next = sched_items[i_begin];     // (only the index is fetched ahead here: these warps have no registers to spare)
+    for (int i = i_begin; i < i_end && ok; ++i) {
+      const int it = i - i_begin;
+      AttnItem im;
+      decode_item(p, w_next, im);
+      if (i + 1 < i_end) w_next = sched_items[i + 1];
+      const int n_kv_tiles = im.n_kv_tiles, past = im.past, qt = im.qt;
+      float m_ref = -INFINITY, l = 0.f;
+      for (int j = 0; j < n_kv_tiles; ++j, ++gk) {
+        if (!wait_or_abort(tc::smem_u32(&s_full[w]), gk & 1, abort_flag, p.status)) { ok = false; break; }
+        tc::tc_fence_after_sync();
+        const int shift = past + qt * BQ - j * BKV;
+        const bool diag = shift < BKV - 1;
+        const int lim = row + shift;
+        uint32_t s[128];
+        tc::tmem_ld_32x32b_x32p(t_s, s);
+        tc::tmem_ld_32x32b_x32p(t_s + 32, s + 32);
+        tc::tmem_ld_wait();
+        tc::tmem_ld_32x32b_x32p(t_s + 64, s + 64);
+        tc::tmem_ld_32x32b_x32p(t_s + 96, s + 96);
+        if (diag) {
+#pragma unroll
+          for (int e = 0; e < 64; ++e)
+            if (e > lim) s[e] = 0xff800000u;   // -inf
+        }
+        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 64; e += 8) {
+          m0 = tc::max3(m0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+          m1 = tc::max3(m1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+          m2 = tc::max3(m2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+          m3 = tc::max3(m3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
+        }
+        tc::tmem_ld_wait();
+        if (diag) {
+#pragma unroll
+          for (int e = 64; e < 128; ++e)
+            if (e > lim) s[e] = 0xff800000u;
+        }
+#pragma unroll
+        for (int e = 64; e < 128; e += 8) {
+          m0 = tc::max3(m0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+          m1 = tc::max3(m1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+          m2 = tc::max3(m2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+          m3 = tc::max3(m3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
+        }
+        const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+        const bool need = (j == 0) || ((mx - m_ref) * c > RESCALE_THRESHOLD);
+        const float m_new = need ? mx : m_ref;
+        if (j > 0 && __any_sync(0xffffffffu, need)) {
+          const float f = need ? fast_exp2((m_ref - m_new) * c) : 1.f;
+          l *= f;
+#pragma unroll 1
+          for (int ch = 0; ch < 8; ++ch) {
+            uint32_t r[16];
+            tc::tmem_ld_32x32b_x16(t_o + ch * 16, r);
+            tc::tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
+            tc::tmem_st_32x32b_x16(t_o + ch * 16, r);
+          }
+        }
+        m_ref = m_new;
+        const float neg_mc = -m_ref * c;
+        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+          for (int e = hf * 32; e < hf * 32 + 32; e += 2) {
+            const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * e]), c, neg_mc));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 1]), c, neg_mc));
+            const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 2]), c, neg_mc));
+            const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 3]), c, neg_mc));
+            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+            s[e] = ACT_F16 ? tc::pack_f16x2(p0, p1) : tc::pack_bf16x2(p0, p1);
+            s[e + 1] = ACT_F16 ? tc::pack_f16x2(p2, p3) : tc::pack_bf16x2(p2, p3);
+          }
+          tc::tmem_st_32x32b_x32(t_s + hf * 32, s + hf * 32);
+          tc::tmem_st_wait();
+          tc::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(tc::smem_u32(hf == 1 ? &p_ready2[w] : &p_ready[w]));
+        }
+        l += (l0 + l1) + (l2 + l3);
+      }
+      if (!ok) break;
+      // ---- epilogue of the item: O_w / l -> 16 bits -> out[token, head, :], then hand O_w back to the MMA warp
+      if (!wait_or_abort(tc::smem_u32(o_full), it & 1, abort_flag, p.status)) { ok = false; break; }
+      tc::tc_fence_after_sync();
+      const float inv = 1.f / l;
+      const bool valid = qt * BQ + row < im.n;
+      bf16 *dst = p.out + ((size_t)(im.q_row0 + row) * p.n_q + (im.h0 + w)) * HD;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32b_x32(t_o + ch * 32, r);
+        tc::tmem_ld_wait();
+        if (ch == 3) {               // the last read of O_w is done: the next item's first P V may overwrite it
+          tc::tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive(tc::smem_u32(o_empty));
+        }
+        if (valid) {
+          uint4 *d4 = reinterpret_cast<uint4 *>(dst + ch * 32);
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            d4[e] = make_uint4(tc::pack_act(__uint_as_float(r[8 * e]) * inv, __uint_as_float(r[8 * e + 1]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * e + 2]) * inv, __uint_as_float(r[8 * e + 3]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * e + 4]) * inv, __uint_as_float(r[8 * e + 5]) * inv, ACT_F16),
+                               tc::pack_act(__uint_as_float(r[8 * e + 6]) * inv, __uint_as_float(r[8 * e + 7]) * inv, ACT_F16));
+        }
+      }
+    }
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
 }  // namespace
+
+int attention_schedule(const int32_t *n_new, const int32_t *n_past, int n_seqs, int n_q, int n_ctas, int32_t *off, int32_t *items) {
+  const int n_pairs = n_q / 2;
+  int max_tiles = 0;
+  for (int b = 0; b < n_seqs; ++b) max_tiles = std::max(max_tiles, (n_new[b] + BQ - 1) / BQ);
+  const int per_tile = n_seqs * n_pairs;
+  // (cost in key tiles, item index); what a CTA pays per item besides its key tiles is worth about 3 of them
+  std::vector<std::pair<int, int>> work;
+  for (int qt = max_tiles - 1; qt >= 0; --qt)
+    for (int b = 0; b < n_seqs; ++b) {
+      if (qt * BQ >= n_new[b]) continue;
+      const int tiles = (n_past[b] + std::min(n_new[b], (qt + 1) * BQ) - 1) / BKV + 1;
+      for (int pr = 0; pr < n_pairs; ++pr) work.emplace_back(tiles + 3, (max_tiles - 1 - qt) * per_tile + b * n_pairs + pr);
+    }
+  std::stable_sort(work.begin(), work.end(), [](const std::pair<int, int> &x, const std::pair<int, int> &y) { return x.first > y.first; });
+  // least loaded CTA first (ties: lowest index)
+  std::priority_queue<std::pair<long long, int>, std::vector<std::pair<long long, int>>, std::greater<std::pair<long long, int>>> heap;
+  for (int c = 0; c < n_ctas; ++c) heap.emplace(0LL, c);
+  std::vector<int> owner(work.size());
+  std::vector<int32_t> count(n_ctas, 0);
+  for (size_t i = 0; i < work.size(); ++i) {
+    auto top = heap.top();
+    heap.pop();
+    owner[i] = top.second;
+    ++count[top.second];
+    heap.emplace(top.first + work[i].first, top.second);
+  }
+  off[0] = 0;
+  for (int c = 0; c < n_ctas; ++c) off[c + 1] = off[c] + count[c];
+  std::vector<int32_t> fill(off, off + n_ctas);
+  for (size_t i = 0; i < work.size(); ++i) items[fill[owner[i]]++] = work[i].second;
+  return (int)work.size();
+}
 
 bool tc_attention_supported(int n_q, int n_kv, int hd) {
   return hd == HD && n_kv >= 1 && n_q % n_kv == 0 && ((n_q / n_kv) % 2) == 0;
@@ -377,7 +748,7 @@ bool tc_attention_supported(int n_q, int n_kv, int hd) {
 int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
                         const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
                         int n_tokens, int kv_rows, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
-                        cudaStream_t st) {
+                        cudaStream_t st, AttnSchedule sched) {
   if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
   if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1 || kv_rows < 1) return SWIFTKV_ERR_INVALID_ARG;
   CUtensorMap tq, tk, tv;
@@ -397,6 +768,14 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
   p.status = status;
   const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
   if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
+  if (sched.off && sched.items && sched.n_ctas > 0) {
+    if (ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent_kernel<false>), ATT_SMEM) ||
+        ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent_kernel<true>), ATT_SMEM))
+      return SWIFTKV_ERR_CUDA;
+    if (act_f16) attention_tc_persistent_kernel<true><<<(unsigned)sched.n_ctas, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
+    else attention_tc_persistent_kernel<false><<<(unsigned)sched.n_ctas, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
+    return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+  }
   static int split = -1;
   if (split < 0) { const char *e = getenv("SWIFTKV_ATT_SPLIT_P"); split = e ? atoi(e) : 1; }
   if (act_f16) {

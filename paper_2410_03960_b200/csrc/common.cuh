@@ -192,10 +192,20 @@ bool tc_attention_supported(int n_q, int n_kv, int hd);
 // sequence -- null means a plain prefill whose K / V rows are packed like q; kv_rows: rows of k / v that hold data;
 // max_seq_len bounds the new tokens of one sequence
 // blk / blk_stride (nullable): block tables of a paged cache, see kv_row_of (then k_row0 is ignored)
+// sched (optional, device arrays): a host-balanced assignment of the work items to n_ctas persistent CTAs -- CTA c runs
+// items[off[c] .. off[c + 1]), each the item's index in the order (query tile descending, sequence, head pair) over
+// ceil(max_seq_len / 128) query tiles; see attention_schedule()
+struct AttnSchedule {
+  const int32_t *off = nullptr, *items = nullptr;
+  int n_ctas = 0;
+};
 int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
                         const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
                         int n_tokens, int kv_rows, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
-                        cudaStream_t st);
+                        cudaStream_t st, AttnSchedule sched = AttnSchedule());
+// host side of the persistent attention kernel: items of sequences with n_new[b] new tokens after n_past[b] cached ones,
+// longest first, each to the least loaded of n_ctas CTAs; writes off[n_ctas + 1] and items[], returns the item count
+int attention_schedule(const int32_t *n_new, const int32_t *n_past, int n_seqs, int n_q, int n_ctas, int32_t *off, int32_t *items);
 
 // tail.cu : the last-token path (at most MAX_TAIL_ROWS activation rows per launch, fp32 activations)
 constexpr int MAX_TAIL_ROWS = 8;

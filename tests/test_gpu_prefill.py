@@ -65,9 +65,10 @@ def test_more_prompts_than_one_tail_pass():
 
 
 @pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2), (2, 2)])
-@pytest.mark.parametrize("mask,act", [(3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
+@pytest.mark.parametrize("mask,act", [(19, 1), (19, 0), (3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
 def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask, act):
-    """The same model through the tcgen05 kernels (mask 3), the SIMT kernels (mask 0) and the two mixtures, with
+    """The same model through the tcgen05 kernels (mask 3; mask 19: attention as persistent CTAs walking a host-balanced
+    work list), the SIMT kernels (mask 0) and the two mixtures, with
     half (act 1) and bfloat16 (act 0) activations; several row tiles and a ragged tail (T = 507), prompts of 1 and
     129 tokens included."""
     lens = [300, 77, 129, 1]

@@ -93,7 +93,7 @@ def test_decode_minibatch_on_both_paths(shape, dtype, bar):
     cfg, ow = oracle_config(shape), oracle_weights(w)
     toks = [S.token_ids(seed, b, n + 2, shape.vocab) for b, n in enumerate(lens)]
     out = {}
-    for mask in (39, 7):
+    for mask in (55, 39, 7):
         model = P.SwiftKVModel(shape, w, dtype, cap * len(lens), len(lens), l, g)
         assert model.set_kernel_mask(mask) == mask
         model.step(torch.cat([t[:n] for t, n in zip(toks, lens)]), [(n, 0, b * cap, 1) for b, n in enumerate(lens)], l, g)
