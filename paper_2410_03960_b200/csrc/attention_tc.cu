@@ -49,6 +49,7 @@ struct AttnParams {
   int n_seqs, n_q, n_kv, max_tiles;
   float scale_log2;     // softmax scale * log2(e)
   unsigned int *status;
+  int store32;          // out is 32-byte aligned: 32-byte stores in the epilogue
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
@@ -73,6 +74,22 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 32 fp32 accumulators of one output row -> * inv -> 16 bits -> 64 contiguous bytes of the row
+template <bool ACT_F16>
+__device__ __forceinline__ void store_out_chunk(bf16 *dst, const uint32_t (&r)[32], float inv, bool store32) {
+  uint32_t v[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = tc::pack_act(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv, ACT_F16);
+  if (store32) {
+    tc::st_global_v8(dst, v);
+    tc::st_global_v8(dst + 16, v + 8);
+  } else {
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) d4[i] = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  }
 }
 
 // ACT_F16: q, K, V, P and the output are all IEEE halves (else all bfloat16)
@@ -354,15 +371,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         uint32_t r[32];
         tc::tmem_ld_32x32b_x32(t_o + ch * 32, r);
         tc::tmem_ld_wait();
-        if (valid) {
-          uint4 *d4 = reinterpret_cast<uint4 *>(dst + ch * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            d4[i] = make_uint4(tc::pack_act(__uint_as_float(r[8 * i]) * inv, __uint_as_float(r[8 * i + 1]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv, ACT_F16));
-        }
+        if (valid) store_out_chunk<ACT_F16>(dst + ch * 32, r, inv, p.store32 != 0);
       }
     }
   }
@@ -685,15 +694,7 @@ attention_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmQ, const __
           __syncwarp();
           if (lane == 0) tc::mbar_arrive(tc::smem_u32(o_empty));
         }
-        if (valid) {
-          uint4 *d4 = reinterpret_cast<uint4 *>(dst + ch * 32);
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            d4[e] = make_uint4(tc::pack_act(__uint_as_float(r[8 * e]) * inv, __uint_as_float(r[8 * e + 1]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * e + 2]) * inv, __uint_as_float(r[8 * e + 3]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * e + 4]) * inv, __uint_as_float(r[8 * e + 5]) * inv, ACT_F16),
-                               tc::pack_act(__uint_as_float(r[8 * e + 6]) * inv, __uint_as_float(r[8 * e + 7]) * inv, ACT_F16));
-        }
+        if (valid) store_out_chunk<ACT_F16>(dst + ch * 32, r, inv, p.store32 != 0);
       }
     }
   }
@@ -766,6 +767,7 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
   p.max_tiles = (max_seq_len + BQ - 1) / BQ;
   p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
   p.status = status;
+  p.store32 = (reinterpret_cast<uintptr_t>(out) & 31) == 0;
   const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
   if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
   if (sched.off && sched.items && sched.n_ctas > 0) {

@@ -236,6 +236,13 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32p(uint32_t taddr, uint32_t *r)
       : "r"(taddr)
       : "memory");
 }
+// 32 contiguous bytes per thread in one store (address 32-byte aligned): a whole sector per lane, where two 16-byte
+// stores of a row-per-thread pattern would each touch half of one
+__device__ __forceinline__ void st_global_v8(void *ptr, const uint32_t *v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
