@@ -64,7 +64,7 @@ def other_rooflines(prof, f_sw, lens, steps, tensor_peak, hbm_peak):
     proj_flops = (f_sw["gemm"] - SWIFT_LAYER * 2.0 * T * (2 * F) * d) * steps
     add("projection GEMMs (QKV, O, down, SingleInputKV)", "tensor", proj_flops, prof["gemm"][0], tensor_peak, "TFLOP/s",
         "2*M*N*K per launch")
-    add("attention_tc_kernel", "tensor", f_sw["attention"] * steps, prof["attention"][0], tensor_peak, "TFLOP/s",
+    add("attention_tc_persistent_kernel", "tensor", f_sw["attention"] * steps, prof["attention"][0], tensor_peak, "TFLOP/s",
         "4*d_q*n*(n+1)/2 per prompt and layer (causal half only); co-limited by ex2")
     # RMSNorm: 2 per layer + the SingleInputKV norm, read fp32 x and write 16-bit h; embedding gather: read 2 B, write 4 B
     elem_bytes = ((2 * SWIFT_LAYER + 1) * T * d * 6.0 + T * d * 6.0) * steps
@@ -73,7 +73,7 @@ def other_rooflines(prof, f_sw, lens, steps, tensor_peak, hbm_peak):
     # last-token path: every later layer's Q, O, gate, up, down weights once, the lm_head once, every later layer's cache rows once
     tail_bytes = (Lt * (2.0 * d * dq + 3.0 * d * F) * 2 + SHAPE.vocab * d * 2.0 + Lt * T * 2.0 * dkv * 2) * steps
     add("last-token path (weight streaming + single-query attention)", "hbm", tail_bytes, prof["tail"][0], hbm_peak, "GB/s",
-        "weights and cache rows of layers > l read once; ~150 small dependent launches per step")
+        "weights and cache rows of layers > l read once; ~120 small dependent launches per step")
     return out
 
 
