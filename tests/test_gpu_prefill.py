@@ -271,3 +271,25 @@ def test_config4_llama70b_full_depth_truncated_prompts():
     res = check_prefill_against_oracle(model, ref, 80, 2e-2, 2e-2, 0.15)
     assert res["logit_abs"] <= 0.15
     print("config4 truncated parity:", lens, res)
+
+
+def test_persistent_attention_gives_the_same_bits():
+    """Kernel-mask bit 4 only changes which CTA runs which (query tile, head pair) item and in what order: every item's
+    arithmetic is the same, so logits and caches must match bit for bit -- many short prompts (fewer items than SMs is the
+    other extreme, in the tests above), ragged tails, a one-token prompt, a prompt of several query tiles."""
+    import paper_2410_03960_b200 as P
+    lens = [700, 1, 129, 300, 77, 513, 128, 2, 255, 40]
+    l, g = 3, 1
+    w = S.make_weights(MID, 5, torch.bfloat16, "cuda")
+    tok = S.make_prompts(5, lens, MID.vocab)
+    out = {}
+    for mask in (55, 39):
+        model = P.SwiftKVModel(MID, w, torch.bfloat16, sum(lens), len(lens), l, g)
+        assert model.set_kernel_mask(mask) == mask
+        model.prefill(tok, lens, l, g)
+        model.status()
+        out[mask] = (model.first_logits().clone(), [t.clone() for j in range(MID.n_layers) for t in model.kv_cache_view(j)[:2]])
+        model.close()
+    assert torch.equal(out[55][0], out[39][0])
+    for a, b in zip(out[55][1], out[39][1]):
+        assert torch.equal(a, b)
