@@ -370,6 +370,7 @@ struct Batch {
   int total_kv;       // sum of cached + new lengths
   bool plain;
   int att_ctas;       // > 0: the device holds a schedule for that many persistent attention CTAs
+  std::vector<int> emit_lens;   // cached + new length of every emitting sequence, in their order (host copy)
   bool paged;         // sequences own lists of 128-row pages instead of one contiguous region
   int blk_stride;     // pages per sequence in the device block tables
   bool decode;        // at most 8 sequences, one new token each, all emitting: every layer runs on the weight-streaming
@@ -475,7 +476,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   if (bt.decode) {
     const int rows = T_tok;
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
-    const TailRope q_rope{b.last_pos, b.cos_tab, b.sin_tab};     // the queries are rotated inside the attention kernel
+    const TailOpts q_rope{b.last_pos, b.cos_tab, b.sin_tab, bt.total_kv};     // the queries are rotated inside the attention kernel
     auto store_kv = [&](int slot) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
       if (fp8) {
         Scope s(m, st, SWIFTKV_KC_TAIL, 5);
@@ -697,7 +698,9 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       {
         Scope s(m, st, SWIFTKV_KC_TAIL, 2);
         const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
-        const TailRope q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab};    // the queries are rotated inside the attention kernel
+        int emit_kv = 0;
+        for (int r = r0; r < r0 + rows; ++r) emit_kv += bt.emit_lens[r];
+        const TailOpts q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab, emit_kv};    // the queries are rotated inside the attention kernel
         if (fp8)
           launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(slot), (const fp8e4 *)v_codes(slot), k_scale(slot), v_scale(slot), ay,
                                        b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads,
@@ -805,7 +808,10 @@ static int32_t forward_common(swiftkv_model *m, const int32_t *tokens, bool toke
       pos[cu[i] + k] = pp;
       slot[cu[i] + k] = bt.paged ? s.block_table[pp / PAGE_ROWS] * PAGE_ROWS + pp % PAGE_ROWS : s.cache_row + pp;
     }
-    if (s.emit) { last_idx[ne] = cu[i + 1] - 1; last_pos[ne] = klen[i] - 1; e_row0[ne] = s.cache_row; e_len[ne] = klen[i]; ++ne; }
+    if (s.emit) {
+      last_idx[ne] = cu[i + 1] - 1; last_pos[ne] = klen[i] - 1; e_row0[ne] = s.cache_row; e_len[ne] = klen[i]; ++ne;
+      bt.emit_lens.push_back(klen[i]);
+    }
   }
   Buffers &b = m->b;
   if (bt.paged) {   // block tables of all sequences, and once more for the emitting ones in their order

@@ -220,11 +220,14 @@ void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, i
 template <typename T>
 void launch_skinny_gemm_dual(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, float *out2,
                              int ldo, cudaStream_t st);
-// optional rotary embedding of the query rows inside the single-query attention (row b sits at position pos[b]; the
-// tables are those of launch_rope): saves a launch per layer on the last-token path
-struct TailRope {
+// options of the single-query attention inside a prefill / step.  pos != null: rotary embedding of the query rows in the
+// kernel (row b sits at position pos[b]; the tables are those of launch_rope), which saves a launch per layer.
+// total_len > 0: the sum of the sequences' key counts, known to the host, from which the key split is chosen so that the
+// blocks fill whole waves of the GPU (never finer than the default split, so the scratch always suffices).
+struct TailOpts {
   const int32_t *pos = nullptr;
   const float *cos_tab = nullptr, *sin_tab = nullptr;
+  int total_len = 0;
 };
 // one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
 // row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials
@@ -233,6 +236,6 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
                            const int32_t *row0, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailRope rope = TailRope());
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailOpts rope = TailOpts());
 
 }  // namespace skv

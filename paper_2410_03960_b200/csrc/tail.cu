@@ -370,7 +370,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // element dd of a query row, rotated to the row's position when the caller asks for it (same arithmetic as rope_kernel)
-__device__ __forceinline__ float load_query(const float *__restrict__ qr, int dd, int hd, int b, const TailRope &rope) {
+__device__ __forceinline__ float load_query(const float *__restrict__ qr, int dd, int hd, int b, const TailOpts &rope) {
   const float v = qr[dd];
   if (!rope.pos) return v;
   const int half = hd >> 1, i = dd < half ? dd : dd - half;
@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
     const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
     const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk, int n_splits, float scale,
-    float *__restrict__ scratch, TailRope rope) {
+    float *__restrict__ scratch, TailOpts rope) {
   static_assert(HD == 128, "one lane owns 4 consecutive output dims");
   using TT = TailTile<T>;
   extern __shared__ __align__(16) uint8_t ta_smem[];
@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(256) tail_attention_partial_kernel(
     const float *__restrict__ q, const T *__restrict__ kc, const T *__restrict__ vc, const float *__restrict__ kscale,
     const float *__restrict__ vscale, const int32_t *__restrict__ cu, const int32_t *__restrict__ len,
     const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int hd, int chunk, int n_splits, float scale,
-    float *__restrict__ scratch, TailRope rope) {
+    float *__restrict__ scratch, TailOpts rope) {
   extern __shared__ float sm[];   // q of each warp's head: [rep][hd]
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -643,9 +643,22 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
                            const int32_t *cu_seqlens, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
-                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailRope rope) {
+                           int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailOpts rope) {
   if (n_seqs <= 0) return;
-  const int chunk = tail_chunk(max_seq_len);
+  int chunk = tail_chunk(max_seq_len);
+  if (rope.total_len > 0 && hd == 128) {
+    // blocks of `c` keys: about total_len / c + half a ragged block per sequence, times the KV heads; three blocks of the
+    // grouped kernel fit an SM.  Cost of a split = waves x keys per block; the coarsest split of the cheapest cost wins.
+    static int n_sms = 0;
+    if (n_sms == 0) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev); if (n_sms < 1) n_sms = 1; }
+    const double cap = 3.0 * n_sms;
+    double best = 1e300;
+    for (int c = chunk; c <= ((max_seq_len + 127) / 128) * 128 && c < chunk + 4096; c += 128) {
+      const double blocks = ((double)rope.total_len / c + 0.5 * n_seqs) * n_kv;
+      const double cost = ceil(blocks / cap) * (c + 64);
+      if (cost <= best) { best = cost; chunk = c; }
+    }
+  }
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
   const float scale = 1.0f / sqrtf((float)hd);
   const int rep = n_q / n_kv;
@@ -678,12 +691,12 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
 }
 template void launch_tail_attention<float>(const float *, const float *, const float *, const float *, const float *, float *,
                                            const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                           float *, cudaStream_t, TailRope);
+                                           float *, cudaStream_t, TailOpts);
 template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf16 *, const float *, const float *, float *,
                                           const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                          float *, cudaStream_t, TailRope);
+                                          float *, cudaStream_t, TailOpts);
 template void launch_tail_attention<fp8e4>(const float *, const fp8e4 *, const fp8e4 *, const float *, const float *, float *,
                                            const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
-                                           float *, cudaStream_t, TailRope);
+                                           float *, cudaStream_t, TailOpts);
 
 }  // namespace skv
