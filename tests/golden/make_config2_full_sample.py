@@ -1,7 +1,7 @@
 """Writes tests/golden/config2_full_sample.npz: sampled outputs of the CPU oracle on the FULL benchmark workload
 (Llama-3.1-8B shape, bf16-valued weights, SwiftKV l = 16, g = 1, 8 prompts with lengths U[2048, 8192], seed 1).
 With `--sweep N` it writes tests/golden/sweep_n<N>_full_sample.npz instead: one prompt of N tokens, seed 4, l = 16 (a
-point of the prompt-length sweep; N = 4096 takes about a quarter of an hour).
+point of the prompt-length sweep; N = 4096 takes about a quarter of an hour after the weights, N = 16384 about four hours).
 
 Calls only the oracle and the seeded input generators.  Takes about two hours on 8 cores and ~35 GB of host memory:
     python tests/golden/make_config2_full_sample.py
