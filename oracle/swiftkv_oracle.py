@@ -8,7 +8,9 @@ with the CUDA library and never imports it.
 Pins (see tests/test_oracle_pins.py): brute-force attention, RoPE/RMSNorm/softmax identities, the
 identity-residual and constant-prompt special cases, l = L equals the baseline, g = 1 equals a separately
 written per-layer Eq. 2 loop, the folded fused projection equals norm-then-project, Table 1's FLOP rows,
-the KV-cache reduction percentages of Sec. 4, and library routines (torch fp64) on the tiny configuration.
+the KV-cache reduction percentages of Sec. 4, library routines (torch fp64) on the tiny configuration for both the
+unmodified model and the re-wired one (every layer's cache and the logits), and, for `tail_layer`, the identity
+"last row of a causal layer = tail_layer on that row's hidden state and the layer's cache".
 The paper prints no worked numerical example of a forward pass, so K/V/logit VALUES are pinned by these
 structural facts and library cross-checks only.
 

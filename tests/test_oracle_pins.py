@@ -180,6 +180,112 @@ def test_baseline_against_torch_library_forward_on_config1():
     assert rel_l2(sk["logits"], out["logits"]) > 1e-3          # it IS a different model
 
 
+def _torch_swiftkv_forward(shape, w, tokens, seq_lens, l, g):
+    """An independent fp64 SwiftKV forward from torch library routines: layers 1..l as in the unmodified model,
+    K/V of every later layer projected from the layer-l output with that group's leading layer's norm gain and
+    W_K, W_V (Eq. 2, Sec. 3.3), and only the last token of each prompt carried through layers l+1..L
+    (footnote of Sec. 3.2, Sec. 3.5) -- written per prompt with SDPA on a one-row query, no code shared with the oracle."""
+    F = torch.nn.functional
+    dt = torch.float64
+    L, hd, half = shape.n_layers, shape.head_dim, shape.head_dim // 2
+    inv = shape.rope_theta ** (-2.0 * torch.arange(half, dtype=dt) / hd)
+    Ks, Vs, logits = [[] for _ in range(L)], [[] for _ in range(L)], []
+    lay = [{k: v.to(dt) for k, v in lw.items()} for lw in w.layers]
+    off = 0
+    for n in seq_lens:
+        ids = torch.as_tensor(tokens[off:off + n]).long()
+        off += n
+        x = w.embed.to(dt)[ids]
+        rot = torch.polar(torch.ones(n, half, dtype=dt), torch.arange(n, dtype=dt)[:, None] * inv)
+
+        def rope(t, r):
+            z = torch.complex(t[..., :half], t[..., half:]) * r[:, None, :]
+            return torch.cat([z.real, z.imag], -1)
+        for j in range(l):
+            lw = lay[j]
+            h = F.rms_norm(x, (shape.hidden,), lw["in_norm"], shape.rms_eps)
+            q = rope(F.linear(h, lw["wq"]).view(n, shape.n_q_heads, hd), rot)
+            k = rope(F.linear(h, lw["wk"]).view(n, shape.n_kv_heads, hd), rot)
+            v = F.linear(h, lw["wv"]).view(n, shape.n_kv_heads, hd)
+            Ks[j].append(k)
+            Vs[j].append(v)
+            a = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None],
+                                               v.transpose(0, 1)[None], is_causal=True, enable_gqa=True)
+            x = x + F.linear(a[0].transpose(0, 1).reshape(n, -1), lw["wo"])
+            m = F.rms_norm(x, (shape.hidden,), lw["post_norm"], shape.rms_eps)
+            x = x + F.linear(F.silu(F.linear(m, lw["w_gate"])) * F.linear(m, lw["w_up"]), lw["w_down"])
+        s = x
+        cache = {}
+        for j in range(l, L):
+            r = l + ((j - l) // g) * g                      # 0-based first layer of j's group
+            if r not in cache:
+                h = F.rms_norm(s, (shape.hidden,), lay[r]["in_norm"], shape.rms_eps)
+                cache[r] = (rope(F.linear(h, lay[r]["wk"]).view(n, shape.n_kv_heads, hd), rot),
+                            F.linear(h, lay[r]["wv"]).view(n, shape.n_kv_heads, hd))
+            Ks[j].append(cache[r][0])
+            Vs[j].append(cache[r][1])
+        y = s[n - 1:n]                                      # [1, d]: the continuing token, position n - 1
+        for j in range(l, L):
+            lw = lay[j]
+            k, v = cache[l + ((j - l) // g) * g]
+            h = F.rms_norm(y, (shape.hidden,), lw["in_norm"], shape.rms_eps)
+            q = rope(F.linear(h, lw["wq"]).view(1, shape.n_q_heads, hd), rot[n - 1:n])
+            # one query row against all n cached keys: no mask (every key is at or before position n - 1)
+            a = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None],
+                                               v.transpose(0, 1)[None], is_causal=False, enable_gqa=True)
+            y = y + F.linear(a[0].transpose(0, 1).reshape(1, -1), lw["wo"])
+            m = F.rms_norm(y, (shape.hidden,), lw["post_norm"], shape.rms_eps)
+            y = y + F.linear(F.silu(F.linear(m, lw["w_gate"])) * F.linear(m, lw["w_up"]), lw["w_down"])
+        logits.append(F.linear(F.rms_norm(y[0], (shape.hidden,), w.final_norm.to(dt), shape.rms_eps), w.lm_head.to(dt)))
+    return [torch.cat(k).numpy() for k in Ks], [torch.cat(v).numpy() for v in Vs], torch.stack(logits).numpy()
+
+
+@pytest.mark.parametrize("l,g", [(2, 1), (1, 2), (1, 3), (3, 1)])
+def test_swiftkv_against_torch_library_forward_on_config1(l, g):
+    """Config 1 with the re-wiring on: every layer's cache and the first-token logits against a SwiftKV forward
+    assembled from torch library routines.  This is what fixes the continuing token's path through layers l+1..L
+    (its own hidden state through the layer's own input norm and W_Q, rotary position n - 1, all n cached keys,
+    attention residual, post-attention norm, MLP residual)."""
+    shape = S.TINY
+    lens = [128, 96]
+    w = S.make_weights(shape, 0, torch.float32)
+    tok = S.make_prompts(0, lens, shape.vocab).numpy()
+    Kt, Vt, lt = _torch_swiftkv_forward(shape, w, tok, lens, l, g)
+    out = O.swiftkv(_cfg(shape), _weights(shape, 0), tok, lens, l, g)
+    for j in range(shape.n_layers):
+        assert rel_l2(out["K"][j], Kt[j]) < 1e-12 and rel_l2(out["V"][j], Vt[j]) < 1e-12
+    assert rel_l2(out["logits"], lt) < 1e-12
+
+
+@pytest.mark.parametrize("which", ["small", "config1"])
+def test_tail_layer_is_the_last_row_of_a_causal_layer(which):
+    """The last row of an unmodified causal layer depends only on that row's hidden state and on the layer's
+    cache, so `tail_layer` fed with the baseline's own hidden state x_j[n-1] and its own K_j, V_j must return
+    row n - 1 of `decoder_layer`'s output -- for every layer and prompt.  A wrong query position, a wrong norm
+    gain, a dropped residual or a key-range slip in `tail_layer` breaks the identity."""
+    if which == "small":
+        shape, lens, seed = SMALL, LENS, 5
+    else:
+        shape, lens, seed = S.TINY, [128, 96], 0
+    cfg, W = _cfg(shape), _weights(shape, seed)
+    tok = S.make_prompts(seed, lens, shape.vocab).numpy()
+    off = 0
+    for n in lens:
+        X = np.asarray(W.embed_rows(tok[off:off + n]), dtype=np.float64)
+        off += n
+        pos = np.arange(n)
+        for j in range(cfg.n_layers):
+            Xn, K, V = O.decoder_layer(cfg, W.layer(j), X, pos)
+            y = O.tail_layer(cfg, W.layer(j), X[n - 1], n - 1, K, V)
+            assert np.allclose(y, Xn[n - 1], rtol=1e-11, atol=1e-13)
+            if n > 2:
+                # an inner row p is the last row of the prefix 0..p: tail_layer must read keys 0..p only
+                p = n // 2
+                yp = O.tail_layer(cfg, W.layer(j), X[p], p, K, V)
+                assert np.allclose(yp, Xn[p], rtol=1e-11, atol=1e-13)
+            X = Xn
+
+
 # ------------------------------------------------------------------ SwiftKV structure -------------
 def test_layers_up_to_l_untouched_and_l_equal_L_is_baseline(small):
     cfg, W, tok = small
