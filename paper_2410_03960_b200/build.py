@@ -35,8 +35,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write(proc.stdout + proc.stderr)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed building libswiftkv.so")
-    with open(os.path.join(HERE, "build_ptxas.log"), "w") as f:
-        f.write(proc.stdout + proc.stderr)
+    # register / spill / shared-memory report of ptxas: scratch output, kept out of the source tree
+    log_dir = os.environ.get("SWIFTKV_BUILD_LOG_DIR", os.path.join(HERE, "..", "gpurun_out"))
+    try:
+        os.makedirs(log_dir, exist_ok=True)
+        with open(os.path.join(log_dir, "build_ptxas.log"), "w") as f:
+            f.write(proc.stdout + proc.stderr)
+    except OSError:
+        pass
     return LIB
 
 
