@@ -285,6 +285,9 @@ int32_t swiftkv_attention_prefill(const void *q, const void *k, const void *v, v
  * prompt b occupying rows [cu_seqlens[b], cu_seqlens[b+1]); out DEVICE fp32 [n_seqs, n_q*hd]; softmax scale
  * 1/sqrt(hd).  n_seqs <= 8.  The keys are split across CTAs; `scratch` (DEVICE, caller-owned, at least
  * swiftkv_tail_attention_scratch_bytes(...) bytes, 16-byte aligned) holds the per-split partial results.
+ * max_seq_len must bound every prompt's length: cu_seqlens lives on the device and is not checked, and keys beyond
+ * the range that max_seq_len's split covers are not read.  A prompt of length 0 gets an all-zero output row.
+ * The scratch size is valid for every call with the same n_seqs / heads and any smaller max_seq_len.
  * Errors: INVALID_ARG, WORKSPACE_SMALL (scratch too small), CUDA. */
 size_t  swiftkv_tail_attention_scratch_bytes(int32_t n_seqs, int32_t n_q_heads, int32_t head_dim, int32_t max_seq_len);
 int32_t swiftkv_tail_attention(const float *q, const void *k_cache, const void *v_cache, float *out,

@@ -232,6 +232,8 @@ struct TailOpts {
 // one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
 // row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens);
+// upper bound of the key splits of any launch whose max_seq_len is at most max_tokens (what the scratch is sized for)
+int tail_max_splits(int max_tokens);
 // T = fp8e4: kc / vc hold FP8 codes and kscale / vscale the fp32 scale of every cache row (null for other types)
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,

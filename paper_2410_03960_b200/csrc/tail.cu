@@ -619,7 +619,7 @@ __global__ void __launch_bounds__(128) tail_attention_merge_kernel(const float *
       L += ls[k] * w;
     }
     L = warp_sum(L);
-    if (lane == 0) inv_l = 1.f / L;
+    if (lane == 0) inv_l = L > 0.f ? 1.f / L : 0.f;     // a sequence without keys: every split is empty, the row is zeros
   }
   __syncthreads();
   for (int dd = threadIdx.x; dd < hd; dd += blockDim.x) {
@@ -633,11 +633,17 @@ __global__ void __launch_bounds__(128) tail_attention_merge_kernel(const float *
   }
 }
 
+// Most splits any launch with max_seq_len <= max_tokens can use.  The split count ceil(n / tail_chunk(n)) is NOT
+// monotonic in n (the chunk is rounded up to whole rounds of 128 keys), so a buffer sized from max_tokens' own split
+// count can be too small for a shorter maximum; but chunks are at least 512 keys and tail_chunk never gives more than
+// 64 splits, and a launch only ever coarsens the split it starts from.
+int tail_max_splits(int max_tokens) {
+  const int by_chunk = (max_tokens + 511) / 512;
+  return by_chunk < 64 ? by_chunk : 64;
+}
 size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_tokens) {
-  const int chunk = tail_chunk(max_tokens);
-  const int n_splits = (max_tokens + chunk - 1) / chunk;
   const int rows = max_seqs < MAX_TAIL_ROWS ? max_seqs : MAX_TAIL_ROWS;
-  return (size_t)rows * n_q * n_splits * (hd + 2) * sizeof(float);
+  return (size_t)rows * n_q * tail_max_splits(max_tokens) * (hd + 2) * sizeof(float);
 }
 
 template <typename T>

@@ -43,7 +43,7 @@ extern "C" int32_t swiftkv_tail_attention_noalloc(const float *q, const void *k_
   if (!q || !k_cache || !v_cache || !out || !cu_seqlens) return report_error(SWIFTKV_ERR_INVALID_ARG, "null argument");
   if (n_seqs < 1 || n_seqs > MAX_TAIL_ROWS || max_seq_len < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads ||
       head_dim < 2 || head_dim > 256)
-    return report_error(SWIFTKV_ERR_INVALID_ARG, "bad shape (n_seqs must be in [1, 8], head_dim even and <= 256)");
+    return report_error(SWIFTKV_ERR_INVALID_ARG, "bad shape (n_seqs must be in [1, 8], head_dim in [2, 256], n_q_heads a multiple of n_kv_heads)");
   if (dtype != SWIFTKV_DTYPE_BF16 && dtype != SWIFTKV_DTYPE_F32) return report_error(SWIFTKV_ERR_INVALID_ARG, "unknown dtype");
   const size_t need = tail_attention_scratch_bytes(n_seqs, n_q_heads, head_dim, max_seq_len);
   if (need > SWIFTKV_NOALLOC_SCRATCH_BYTES)

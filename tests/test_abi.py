@@ -66,6 +66,27 @@ def test_workspace_bytes_validates_and_accounts_for_acrosskv(lib):
         workspace_bytes(odd, torch.float32, 128, 2, 2, 1)
 
 
+def test_tail_attention_scratch_covers_every_shorter_maximum(lib):
+    """A model's split-KV scratch is sized once from max_tokens but used with each batch's own longest sequence.  The
+    split count ceil(n / chunk(n)) is not monotonic in n (chunks are whole rounds of 128 keys, at most 64 splits,
+    at least 512 keys), so the size query must cover every n <= max_tokens, not just n = max_tokens."""
+    def splits(n):
+        c = -(-n // 64)
+        c = -(-c // 128) * 128
+        c = max(c, 512)
+        return -(-n // c)
+    assert splits(32768) == 64 and splits(33000) < 64          # the non-monotonic spot: 64 splits, then fewer
+    per_split = 8 * 32 * (128 + 2) * 4
+    for T in (1, 511, 512, 513, 4096, 20000, 32768, 33000, 41123, 65536, 100000, 131072):
+        have = lib.swiftkv_tail_attention_scratch_bytes(8, 32, 128, T)
+        assert have % per_split == 0
+        worst = max(splits(n) for n in range(1, T + 1, 7)) if T > 1 else 1
+        worst = max(worst, splits(T), splits(min(T, 32768)))
+        assert have >= worst * per_split, (T, have // per_split, worst)
+    sizes = [lib.swiftkv_tail_attention_scratch_bytes(8, 32, 128, T) for T in range(1, 70000, 97)]
+    assert all(a <= b for a, b in zip(sizes, sizes[1:]))        # monotonic in the maximum length
+
+
 def test_null_arguments_return_status_codes(lib):
     assert lib.swiftkv_workspace_bytes(None, 1, 1, 1, 1, None, None) == -1
     out = C.c_void_p()

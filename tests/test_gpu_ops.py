@@ -90,3 +90,23 @@ def test_tail_attention(dtype, bar, lens, n_q, n_kv, hd):
         ref = O.single_query_attention(to_np(q[b]), to_np(k[off:off + n]), to_np(v[off:off + n]))
         assert rel_l2(to_np(out[b]), ref) < bar
         off += n
+
+
+def test_tail_attention_empty_sequence_gives_zeros_not_nan():
+    """A prompt of length 0 between two ordinary ones: no key, no probability mass -- the row is zeros (not 0/0) and
+    its neighbours are unaffected."""
+    import paper_2410_03960_b200 as P
+    lens, n_q, n_kv, hd = [40, 0, 700], 8, 2, 128
+    T, B = sum(lens), len(lens)
+    q = S.matrix(8, 1, B, n_q * hd, torch.float32, "cuda", std=1.0).view(B, n_q, hd)
+    k = S.matrix(8, 2, T, n_kv * hd, torch.bfloat16, "cuda", std=1.0).view(T, n_kv, hd)
+    v = S.matrix(8, 3, T, n_kv * hd, torch.bfloat16, "cuda", std=1.0).view(T, n_kv, hd)
+    out = P.tail_attention(q, k, v, lens)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all() and (out[1] == 0).all()
+    off = 0
+    for b, n in enumerate(lens):
+        if n:
+            ref = O.single_query_attention(to_np(q[b]), to_np(k[off:off + n]), to_np(v[off:off + n]))
+            assert rel_l2(to_np(out[b]), ref) < 1e-5
+        off += n
