@@ -44,6 +44,7 @@ extern "C" {
 #define SWIFTKV_ERR_DEVICE_TIMEOUT   -5   /* a bounded wait inside a kernel ran out                      */
 #define SWIFTKV_ERR_BAD_TOKEN        -6   /* a token id outside [0, vocab) was met on the device         */
 #define SWIFTKV_ERR_UNSUPPORTED      -7
+#define SWIFTKV_ERR_ACT_OVERFLOW     -8   /* a value beyond the IEEE-half range was clamped (SWIFTKV_ACT_F16)   */
 
 #define SWIFTKV_DTYPE_F32  0
 #define SWIFTKV_DTYPE_BF16 1
@@ -212,8 +213,9 @@ int32_t swiftkv_first_logits(const swiftkv_model *m, const float **logits, int32
 
 /*
  * Synchronises `cuda_stream` and returns the device status word latched by the kernels of earlier calls:
- * OK, DEVICE_TIMEOUT (a bounded in-kernel wait gave up; results are invalid), BAD_TOKEN, or CUDA.
- * Clears the word.
+ * OK, DEVICE_TIMEOUT (a bounded in-kernel wait gave up; results are invalid), ACT_OVERFLOW (with SWIFTKV_ACT_F16 an
+ * intermediate activation, a cached K / V value or a weight lay beyond +-65504 and was clamped: results are wrong,
+ * select SWIFTKV_ACT_BF16 for this model), BAD_TOKEN, or CUDA.  Clears the word.
  */
 int32_t swiftkv_status(swiftkv_model *m, void *cuda_stream);
 
@@ -246,7 +248,8 @@ int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
 /* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention
  * output, SwiGLU output, softmax probabilities) -- never of weights or the KV cache, which stay bf16.
- *   SWIFTKV_ACT_F16  (default): IEEE half, 8x finer rounding than bf16; conversions saturate at +-65504.  Because
+ *   SWIFTKV_ACT_F16  (default): IEEE half, 8x finer rounding than bf16; conversions saturate at +-65504 and every
+ *                      clamped store raises SWIFTKV_ERR_ACT_OVERFLOW in swiftkv_status (never silently).  Because
  *                      both operands of a tensor-core MMA must share one 16-bit type, each layer's matrices are
  *                      copied to half right before use (workspace scratch for one layer; exact for |w| >= 2^-17)
  *                      and the current layer's K / V get a half copy beside the bf16 cache.
@@ -255,6 +258,19 @@ int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 #define SWIFTKV_ACT_BF16 0
 #define SWIFTKV_ACT_F16  1
 int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format);
+
+/* Failure-detection self-check (no counterpart in the paper).  Every wait inside the kernels is bounded: when it runs out
+ * the kernel latches DEVICE_TIMEOUT in the model's status word, every role of the CTA leaves its loop and the kernel
+ * returns, so the context stays usable.  This call launches one small CTA that waits, with that same bounded wait but a
+ * limit of `limit_clocks` SM clocks (1 .. 1e8, i.e. at most ~50 ms), on a barrier that is never completed, synchronises
+ * the stream and writes to HOST outcome[2]: [0] = 1 if the waiting role gave up at its limit, [1] = 1 if a second role
+ * of the CTA left through the abort flag.  Afterwards swiftkv_status reports SWIFTKV_ERR_DEVICE_TIMEOUT once.
+ * Errors: INVALID_ARG, CUDA. */
+int32_t swiftkv_debug_bounded_wait(swiftkv_model *m, int64_t limit_clocks, int32_t *outcome, void *cuda_stream);
+
+/* Synchronises `cuda_stream`, then returns and clears the current device's status word of the stand-alone operator
+ * entry points below (swiftkv_gemm_tc, swiftkv_attention_prefill): OK, DEVICE_TIMEOUT, ACT_OVERFLOW or CUDA. */
+int32_t swiftkv_op_status(void *cuda_stream);
 
 /* Destroys the host object (never the caller's buffers).  Null is allowed. */
 void swiftkv_model_free(swiftkv_model *m);

@@ -23,6 +23,7 @@ EXPORTS = (
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
     "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
+    "swiftkv_debug_bounded_wait", "swiftkv_op_status",
 )
 
 
@@ -91,6 +92,8 @@ def load_library() -> C.CDLL:
     lib.swiftkv_set_activation_format.argtypes = [C.c_void_p, C.c_int32]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
+    lib.swiftkv_debug_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
+    lib.swiftkv_op_status.argtypes = [C.c_void_p]
     lib.swiftkv_tail_attention_scratch_bytes.argtypes = [C.c_int32] * 4
     lib.swiftkv_tail_attention_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_tail_attention.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 6 + [C.c_void_p, C.c_size_t, C.c_void_p]
@@ -248,6 +251,13 @@ class SwiftKVModel:
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> None:
         with torch.cuda.device(self.device):
             _check(self.lib.swiftkv_status(self._h, _stream_ptr(stream)))
+
+    def debug_bounded_wait(self, limit_clocks: int, stream: Optional[torch.cuda.Stream] = None) -> Tuple[bool, bool]:
+        """swiftkv_debug_bounded_wait: (the waiting role gave up at its limit, the second role left through the abort flag)."""
+        out = (C.c_int32 * 2)()
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_debug_bounded_wait(self._h, int(limit_clocks), out, _stream_ptr(stream)))
+        return bool(out[0]), bool(out[1])
 
     def profile_enable(self, on: bool) -> None:
         _check(self.lib.swiftkv_profile_enable(self._h, int(on)))

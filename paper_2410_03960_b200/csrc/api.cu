@@ -8,6 +8,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <type_traits>
 #include <vector>
@@ -353,10 +354,12 @@ static int32_t gemm_any(swiftkv_model *m, const TA *A, int M, int K, const TW *B
       if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "tensor-core GEMM launch failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
   }
-  launch_gemm_simt<TA, TW>(A, B0, M, n0, K, out, 0, st);
+  OutDesc o = out;
+  o.status = m->b.status;      // a clamped half store is reported like on the tensor-core path
+  launch_gemm_simt<TA, TW>(A, B0, M, n0, K, o, 0, st);
   m->launches += 1;
-  if (n1 > 0) { launch_gemm_simt<TA, TW>(A, B1, M, n1, K, out, n0, st); m->launches += 1; }
-  if (n2 > 0) { launch_gemm_simt<TA, TW>(A, B2, M, n2, K, out, n0 + n1, st); m->launches += 1; }
+  if (n1 > 0) { launch_gemm_simt<TA, TW>(A, B1, M, n1, K, o, n0, st); m->launches += 1; }
+  if (n2 > 0) { launch_gemm_simt<TA, TW>(A, B2, M, n2, K, o, n0 + n1, st); m->launches += 1; }
   return SWIFTKV_OK;
 }
 
@@ -421,13 +424,13 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     w16_select(buf);
     {
       Scope s(m, m->side, SWIFTKV_KC_ELEMWISE, 7, false);
-      launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, m->side);
-      launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, m->side);
+      launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, m->side, b.status);
+      launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, m->side, b.status);
     }
     cudaEventRecord(m->ev_ready[buf], m->side);
   };
@@ -538,7 +541,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
         cudaStreamWaitEvent(st, m->ev_ready[j & 1], 0);
       }
     }
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st, b.status); }
     OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv, slot_map};
     if (fp8) { Kj = kst; Vj = vst; qkv.seg_base = kst; qkv.slot_map = nullptr; }   // staging rows are in batch order
     bool roped = false;
@@ -550,7 +553,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
                          want_dup ? k16 : nullptr, (long long)plane);
     if (rc) return rc;
     if (!roped) {
-      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st); }
+      { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st, b.status); }
       { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(Kj, 0, 1, b.pos, fp8 ? nullptr : slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
     }
     if (fp8) {
@@ -603,7 +606,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
             kk = k16; vv = v16;
             if (!bt.plain) {
               Scope s2(m, st, SWIFTKV_KC_ELEMWISE);
-              launch_gather_kv_half((const bf16 *)Kj, (const bf16 *)Vj, k16, v16, b.kv_row0, b.kv_len, b.kcu, blk, bt.blk_stride, B, bt.max_kv, dkv, st);
+              launch_gather_kv_half((const bf16 *)Kj, (const bf16 *)Vj, k16, v16, b.kv_row0, b.kv_len, b.kcu, blk, bt.blk_stride, B, bt.max_kv, dkv, st, b.status);
               kr0 = b.kcu;
               kv_rows = bt.total_kv;
             }
@@ -621,7 +624,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     rc = gemm_any<TA, T>(m, attn, T_tok, dq, (const T *)lw.wo, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
                          use_w16 ? wo16 : nullptr);
     if (rc) return rc;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st, b.status); }
     bool fused = false;
     if constexpr (sizeof(T) == 2) {
       if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d) && (!act_f16 || use_w16)) {
@@ -642,7 +645,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
                              use_w16 ? wu16 : nullptr);
         if (rc) return rc;
         Scope s(m, st, SWIFTKV_KC_ELEMWISE);
-        launch_swiglu<TA>((const TA *)b.gate, (const TA *)b.up, act + (size_t)r0 * F, (long long)rows * F, st);
+        launch_swiglu<TA>((const TA *)b.gate, (const TA *)b.up, act + (size_t)r0 * F, (long long)rows * F, st, b.status);
       }
     }
     rc = gemm_any<TA, T>(m, act, T_tok, F, (const T *)lw.w_down, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
@@ -653,7 +656,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
   if (l < L && !bt.decode) {
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st, b.status); }
     if (fp8) {
       // one group at a time through the staging planes: projection (+ RoPE on K), then the quantizing row pass into the
       // group's cache slot
@@ -937,6 +940,9 @@ extern "C" int32_t swiftkv_status(swiftkv_model *m, void *cuda_stream) {
   CUDA_TRY(cudaMemsetAsync(m->b.status, 0, 4, st));
   CUDA_TRY(cudaStreamSynchronize(st));
   if (word & STATUS_TIMEOUT) return fail(SWIFTKV_ERR_DEVICE_TIMEOUT, "a bounded wait inside a kernel ran out");
+  if (word & STATUS_ACT_OVERFLOW)
+    return fail(SWIFTKV_ERR_ACT_OVERFLOW, "an activation (or weight) beyond the IEEE-half range was clamped to +-65504: results are "
+                                          "wrong; run this model with swiftkv_set_activation_format(SWIFTKV_ACT_BF16)");
   if (word & STATUS_BAD_TOKEN) return fail(SWIFTKV_ERR_BAD_TOKEN, "a token id outside [0, vocab) was clamped");
   return SWIFTKV_OK;
 }
@@ -978,13 +984,42 @@ extern "C" int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t forma
 // ---------------------------------------------------------------------------------------------------------
 // a device word for the stand-alone entry points' bounded waits
 static __device__ unsigned int g_op_status[64];
+// the word's address on the CURRENT device (every device that loads the library has its own copy of the symbol)
 static unsigned int *op_status_word() {
-  static unsigned int *ptr = nullptr;
-  if (!ptr) {
+  constexpr int MAX_DEVICES = 64;
+  static std::mutex mu;
+  static unsigned int *ptr[MAX_DEVICES] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!ptr[dev]) {
     void *p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_op_status) == cudaSuccess) ptr = reinterpret_cast<unsigned int *>(p);
+    if (cudaGetSymbolAddress(&p, g_op_status) == cudaSuccess) ptr[dev] = reinterpret_cast<unsigned int *>(p);
   }
-  return ptr;
+  return ptr[dev];
+}
+
+extern "C" int32_t swiftkv_op_status(void *cuda_stream) {
+  unsigned int *status = op_status_word();
+  if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  unsigned int word = 0;
+  CUDA_TRY(cudaMemcpyAsync(&word, status, 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(cudaMemsetAsync(status, 0, 4, st));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  if (word & STATUS_TIMEOUT) return fail(SWIFTKV_ERR_DEVICE_TIMEOUT, "a bounded wait inside a stand-alone operator ran out");
+  if (word & STATUS_ACT_OVERFLOW) return fail(SWIFTKV_ERR_ACT_OVERFLOW, "a half store of a stand-alone operator was clamped");
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_debug_bounded_wait(swiftkv_model *m, int64_t limit_clocks, int32_t *outcome, void *cuda_stream) {
+  if (!m || !outcome) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (limit_clocks < 1 || limit_clocks > 100000000LL) return fail(SWIFTKV_ERR_INVALID_ARG, "limit_clocks outside [1, 1e8]");
+  int rc = launch_bounded_wait_probe((long long)limit_clocks, m->b.status, m->b.status + 8, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  CUDA_TRY(cudaMemcpyAsync(outcome, m->b.status + 8, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, reinterpret_cast<cudaStream_t>(cuda_stream)));
+  CUDA_TRY(cudaStreamSynchronize(reinterpret_cast<cudaStream_t>(cuda_stream)));
+  return SWIFTKV_OK;
 }
 
 extern "C" int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,

@@ -12,7 +12,10 @@ namespace skv {
 
 // ---- device status word -------------------------------------------------------------------------------
 // Kernels never trap: a bounded wait that runs out, or a bad token id, sets a bit here and carries on.
-enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BAD_TOKEN = 2u };
+// STATUS_ACT_OVERFLOW: a value that had to be stored as IEEE half lay beyond the half range (|v| >= 65520 would round to
+// infinity) and was clamped to +-65504.
+enum : unsigned int { STATUS_TIMEOUT = 1u, STATUS_BAD_TOKEN = 2u, STATUS_ACT_OVERFLOW = 4u };
+constexpr float HALF_OVERFLOW = 65520.f;
 
 // ---- element types ---------------------------------------------------------------------------------------
 using bf16 = __nv_bfloat16;
@@ -63,8 +66,11 @@ struct OutDesc {
   long long seg_stride;   // elements
   int seg_w;
   const int32_t *slot_map;   // optional: GEMM row r lands in row slot_map[r] of a segment (cache row of token r)
+  unsigned int *status;      // optional: receives STATUS_ACT_OVERFLOW when a half store had to clamp
 };
-inline OutDesc out_plain(int mode, void *p, long long ld, int n) { return OutDesc{mode, p, ld, n, nullptr, 0, 1, nullptr}; }
+inline OutDesc out_plain(int mode, void *p, long long ld, int n, unsigned int *status = nullptr) {
+  return OutDesc{mode, p, ld, n, nullptr, 0, 1, nullptr, status};
+}
 
 // ---- paged cache rows ------------------------------------------------------------------------------------
 // A sequence's token p lives in cache row first + p (contiguous region), or -- with a block table -- in row
@@ -84,6 +90,9 @@ __device__ __forceinline__ void store_out(const OutDesc &o, int row, int col, fl
   } else if (o.mode == OUT_STORE_F32) {
     reinterpret_cast<float *>(o.p0)[(size_t)row * o.ld0 + col] = acc;
   } else if (col < o.n0) {
+    if constexpr (sizeof(TP) == 2 && !__is_same(TP, bf16)) {
+      if (fabsf(acc) >= HALF_OVERFLOW && o.status) atomicOr(o.status, STATUS_ACT_OVERFLOW);
+    }
     reinterpret_cast<TP *>(o.p0)[(size_t)row * o.ld0 + col] = from_f<TP>(acc);
   } else {
     const int c = col - o.n0;
@@ -109,18 +118,22 @@ void launch_embed(const T *embed, const int32_t *tokens, float *x, int n_tokens,
 void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions, int32_t *last_idx, int n_tokens,
                       cudaStream_t st);
 // y = x * rsqrt(mean(x^2)+eps) * gamma (gamma may be null: unit-rms only).  x fp32 [rows, d] -> out TO [rows, d]
+// status (nullable): receives STATUS_ACT_OVERFLOW when TO is IEEE half and a value had to be clamped (the same holds for
+// the other launches below that take a status word)
 template <typename TG, typename TO>
-void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st);
+void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st,
+                    unsigned int *status = nullptr);
 // in-place rotary embedding on `n_batches` tensors [*, n_heads, hd] spaced batch_stride elements apart; logical row r
 // (position positions[r]) lives in tensor row slot_map[r] (null: row r)
 template <typename T>
 void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const int32_t *slot_map,
-                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st);
+                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st,
+                 unsigned int *status = nullptr);
 // packs each sequence's cache rows [row0[b], row0[b] + len[b]) of one layer's K and V planes (bf16) into contiguous half
 // copies starting at row kcu[b]: the tensor-core attention kernel's operands in a chunked step with half activations
 void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
                            const int32_t *kcu, const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv,
-                           cudaStream_t st);
+                           cudaStream_t st, unsigned int *status = nullptr);
 // kv_fp8.cu : per-token FP8 cache rows.  One scale per row of `width` elements: scale = max(amax, 2^-64) / 448,
 // code = e4m3(x / scale) (correctly rounded fp32 divisions, round to nearest even, saturating).  Row r of `src` goes to row
 // slot_map[r] (null: r) of `codes` / `scale`; deq (nullable, row r) receives value(code) * scale in type TO.
@@ -134,7 +147,7 @@ void launch_gather_dequant_fp8(const uint8_t *k_codes, const uint8_t *v_codes, c
                                TO *k_out, TO *v_out, const int32_t *row0, const int32_t *len, const int32_t *kcu,
                                const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv, cudaStream_t st);
 template <typename T>
-void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st);
+void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st, unsigned int *status = nullptr);
 void launch_gather_rows(const float *x, const int32_t *idx, float *y, int n_rows, int d, cudaStream_t st);
 // fp32 rows -> rows slot_map[r] (null: r) of a [*, width] plane of type T
 template <typename T>
@@ -149,7 +162,7 @@ void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, doub
 template <typename T, typename TO>
 void launch_fold(const T *w, const T *gamma, TO *dst, int rows, int cols, cudaStream_t st);
 // IEEE-half copy of a bf16 matrix (the compute copy of a layer's weights when activations are kept in half)
-void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st);
+void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st, unsigned int *status = nullptr);
 
 // gemm_simt.cu : C = A[M,K] * B[N,K]^T with fp32 accumulation, any shape; result column c is written as
 // column col0 + c of `out` (p0 region in the activation type TA, segments in the weight / cache type TW)
@@ -179,6 +192,11 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
 int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg, const void *Wu, int F, void *act,
                           unsigned int *status, cudaStream_t st);
 bool tc_swiglu_supported(int M, int F, int K);
+// Failure-detection self-check: one CTA whose consumer role waits -- with the GEMM kernels' own bounded wait, but a
+// limit of `limit_clocks` -- on a barrier that nothing ever completes, and whose second role watches the CTA's abort
+// flag.  The wait runs out, STATUS_TIMEOUT is set in *status, both roles leave their loops, the kernel returns.
+// outcome[0] = 1 if the waiting role gave up at its limit, outcome[1] = 1 if the second role left through the abort flag.
+int launch_bounded_wait_probe(long long limit_clocks, unsigned int *status, unsigned int *outcome, cudaStream_t st);
 
 // attention.cu
 // k_row0 / kv_len as for launch_attention_tc

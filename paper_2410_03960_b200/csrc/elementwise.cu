@@ -1,9 +1,20 @@
 // Memory-bound kernels of the SwiftKV prefill path: embedding gather, RMSNorm, rotary embedding, SwiGLU,
 // last-token gather, RoPE table, and the one-time gain fold of the SingleInputKV weight (Sec. 3.5).
 // All use 128-bit global accesses where the row length allows and warp-shuffle reductions.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace skv {
+
+// a thread's running "had to clamp a half store" note: `hit` collects, `report` raises the status bit once per thread
+template <typename T>
+__device__ __forceinline__ void note_overflow(float v, bool &hit) {
+  if constexpr (std::is_same<T, __half>::value) hit |= fabsf(v) >= HALF_OVERFLOW;
+}
+__device__ __forceinline__ void report_overflow(bool hit, unsigned int *status) {
+  if (hit && status) atomicOr(status, STATUS_ACT_OVERFLOW);
+}
 
 // ---------------------------------------------------------------------------------------------------------
 // embedding gather: x[t, :] = float(E[tok[t], :])      (Sec. 3.1: X are the input embeddings)
@@ -72,7 +83,8 @@ void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions,
 // ---------------------------------------------------------------------------------------------------------
 template <typename TG, typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
-                                                      T *__restrict__ out, int d, float eps) {
+                                                      T *__restrict__ out, int d, float eps, unsigned int *status) {
+  bool hit = false;
   const size_t row = blockIdx.x;
   const float *xr = x + row * d;
   T *orow = out + row * d;
@@ -100,22 +112,29 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
       float g0 = 1.f, g1 = 1.f, g2 = 1.f, g3 = 1.f;
       if (gamma) { g0 = to_f(gamma[i]); g1 = to_f(gamma[i + 1]); g2 = to_f(gamma[i + 2]); g3 = to_f(gamma[i + 3]); }
       if constexpr (sizeof(T) == 2) {
-        T o4[4] = {from_f<T>(v.x * rstd * g0), from_f<T>(v.y * rstd * g1), from_f<T>(v.z * rstd * g2), from_f<T>(v.w * rstd * g3)};
+        const float y0 = v.x * rstd * g0, y1 = v.y * rstd * g1, y2 = v.z * rstd * g2, y3 = v.w * rstd * g3;
+        note_overflow<T>(y0, hit); note_overflow<T>(y1, hit); note_overflow<T>(y2, hit); note_overflow<T>(y3, hit);
+        T o4[4] = {from_f<T>(y0), from_f<T>(y1), from_f<T>(y2), from_f<T>(y3)};
         *reinterpret_cast<uint2 *>(orow + i) = *reinterpret_cast<uint2 *>(o4);
       } else {
         *reinterpret_cast<float4 *>(orow + i) = make_float4(v.x * rstd * g0, v.y * rstd * g1, v.z * rstd * g2, v.w * rstd * g3);
       }
     }
   } else {
-    for (int i = threadIdx.x; i < d; i += blockDim.x)
-      orow[i] = from_f<T>(xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f));
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+      const float y = xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f);
+      note_overflow<T>(y, hit);
+      orow[i] = from_f<T>(y);
+    }
   }
+  report_overflow(hit, status);
 }
 // Rows of exactly 256 * 4 * NV floats (4096: NV = 4, 8192: NV = 8) with 16-bit output: each thread keeps its NV float4
 // in registers between the sum of squares and the scaling, so the row is read from global memory exactly once.
 template <typename TG, typename T, int NV>
 __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
-                                                          T *__restrict__ out, float eps) {
+                                                          T *__restrict__ out, float eps, unsigned int *status) {
+  bool hit = false;
   constexpr int D = 256 * 4 * NV;
   const size_t row = blockIdx.x;
   const float4 *xr = reinterpret_cast<const float4 *>(x + row * D);
@@ -144,22 +163,25 @@ __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restric
       const TG *g = reinterpret_cast<const TG *>(&graw);
       g0 = to_f(g[0]); g1 = to_f(g[1]); g2 = to_f(g[2]); g3 = to_f(g[3]);
     }
-    T o4[4] = {from_f<T>(v[k].x * rstd * g0), from_f<T>(v[k].y * rstd * g1), from_f<T>(v[k].z * rstd * g2), from_f<T>(v[k].w * rstd * g3)};
+    const float y0 = v[k].x * rstd * g0, y1 = v[k].y * rstd * g1, y2 = v[k].z * rstd * g2, y3 = v[k].w * rstd * g3;
+    note_overflow<T>(y0, hit); note_overflow<T>(y1, hit); note_overflow<T>(y2, hit); note_overflow<T>(y3, hit);
+    T o4[4] = {from_f<T>(y0), from_f<T>(y1), from_f<T>(y2), from_f<T>(y3)};
     orow[i4] = *reinterpret_cast<uint2 *>(o4);
   }
+  report_overflow(hit, status);
 }
 template <typename TG, typename TO>
-void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st) {
+void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st, unsigned int *status) {
   if (rows <= 0) return;
   if constexpr (sizeof(TG) == 2 && sizeof(TO) == 2) {
-    if (d == 4096) { rmsnorm_reg_kernel<TG, TO, 4><<<rows, 256, 0, st>>>(x, gamma, out, eps); return; }
-    if (d == 8192) { rmsnorm_reg_kernel<TG, TO, 8><<<rows, 256, 0, st>>>(x, gamma, out, eps); return; }
+    if (d == 4096) { rmsnorm_reg_kernel<TG, TO, 4><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
+    if (d == 8192) { rmsnorm_reg_kernel<TG, TO, 8><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
   }
-  rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps);
+  rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps, status);
 }
-template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t);
-template void launch_rmsnorm<bf16, bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t);
-template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *, int, int, float, cudaStream_t);
+template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t, unsigned int *);
+template void launch_rmsnorm<bf16, bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t, unsigned int *);
+template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *, int, int, float, cudaStream_t, unsigned int *);
 
 // ---------------------------------------------------------------------------------------------------------
 // Rotary embedding, rotate-half pairing (i, i + hd/2), in place.  One thread per pair.
@@ -167,7 +189,7 @@ template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *
 template <typename T>
 __global__ void rope_kernel(T *__restrict__ x, long long batch_stride, const int32_t *__restrict__ positions,
                             const int32_t *__restrict__ slot_map, const float *__restrict__ cos_tab,
-                            const float *__restrict__ sin_tab, int rows, int n_heads, int hd) {
+                            const float *__restrict__ sin_tab, int rows, int n_heads, int hd, unsigned int *status) {
   const int half = hd >> 1;
   const long long per_row = (long long)n_heads * half;
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -180,20 +202,24 @@ __global__ void rope_kernel(T *__restrict__ x, long long batch_stride, const int
   const size_t trow = slot_map ? (size_t)slot_map[row] : (size_t)row;
   T *base = x + (size_t)blockIdx.y * batch_stride + (trow * n_heads + h) * hd;
   const float a = to_f(base[i]), b = to_f(base[i + half]);
+  bool hit = false;
+  note_overflow<T>(a * c - b * s, hit);
+  note_overflow<T>(b * c + a * s, hit);
   base[i] = from_f<T>(a * c - b * s);
   base[i + half] = from_f<T>(b * c + a * s);
+  report_overflow(hit, status);
 }
 template <typename T>
 void launch_rope(T *x, long long batch_stride, int n_batches, const int32_t *positions, const int32_t *slot_map,
-                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st) {
+                 const float *cos_tab, const float *sin_tab, int rows, int n_heads, int hd, cudaStream_t st, unsigned int *status) {
   const long long n = (long long)rows * n_heads * (hd / 2);
   if (n <= 0 || n_batches <= 0) return;
   dim3 grid((unsigned)((n + 255) / 256), (unsigned)n_batches);
-  rope_kernel<T><<<grid, 256, 0, st>>>(x, batch_stride, positions, slot_map, cos_tab, sin_tab, rows, n_heads, hd);
+  rope_kernel<T><<<grid, 256, 0, st>>>(x, batch_stride, positions, slot_map, cos_tab, sin_tab, rows, n_heads, hd, status);
 }
-template void launch_rope<float>(float *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
-template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
-template void launch_rope<__half>(__half *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t);
+template void launch_rope<float>(float *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t, unsigned int *);
+template void launch_rope<bf16>(bf16 *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t, unsigned int *);
+template void launch_rope<__half>(__half *, long long, int, const int32_t *, const int32_t *, const float *, const float *, int, int, int, cudaStream_t, unsigned int *);
 
 // cos/sin of p * theta^(-2i/hd), evaluated in double precision and rounded once to fp32.
 __global__ void rope_table_kernel(float *cos_tab, float *sin_tab, int max_pos, int half, double log_theta, int hd) {
@@ -216,7 +242,9 @@ void launch_rope_table(float *cos_tab, float *sin_tab, int max_pos, int hd, doub
 // SwiGLU: out = silu(gate) * up      (Sec. 3.1 MLP; fp32 arithmetic, model-dtype storage)
 // ---------------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void swiglu_kernel(const T *__restrict__ gate, const T *__restrict__ up, T *__restrict__ out, long long n) {
+__global__ void swiglu_kernel(const T *__restrict__ gate, const T *__restrict__ up, T *__restrict__ out, long long n,
+                              unsigned int *status) {
+  bool hit = false;
   const long long stride = (long long)gridDim.x * blockDim.x;
   constexpr int V = 16 / sizeof(T);
   const long long nv = n / V;
@@ -230,26 +258,31 @@ __global__ void swiglu_kernel(const T *__restrict__ gate, const T *__restrict__ 
 #pragma unroll
     for (int k = 0; k < V; ++k) {
       const float z = to_f(ge[k]);
-      oe[k] = from_f<T>(z / (1.f + __expf(-z)) * to_f(ue[k]));
+      const float y = z / (1.f + __expf(-z)) * to_f(ue[k]);
+      note_overflow<T>(y, hit);
+      oe[k] = from_f<T>(y);
     }
     reinterpret_cast<uint4 *>(out)[i] = o;
   }
   for (long long i = nv * V + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     const float z = to_f(gate[i]);
-    out[i] = from_f<T>(z / (1.f + __expf(-z)) * to_f(up[i]));
+    const float y = z / (1.f + __expf(-z)) * to_f(up[i]);
+    note_overflow<T>(y, hit);
+    out[i] = from_f<T>(y);
   }
+  report_overflow(hit, status);
 }
 template <typename T>
-void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st) {
+void launch_swiglu(const T *gate, const T *up, T *out, long long n, cudaStream_t st, unsigned int *status) {
   if (n <= 0) return;
   long long blocks = (n / (16 / sizeof(T)) + 255) / 256;
   if (blocks < 1) blocks = 1;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  swiglu_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(gate, up, out, n);
+  swiglu_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(gate, up, out, n, status);
 }
-template void launch_swiglu<float>(const float *, const float *, float *, long long, cudaStream_t);
-template void launch_swiglu<bf16>(const bf16 *, const bf16 *, bf16 *, long long, cudaStream_t);
-template void launch_swiglu<__half>(const __half *, const __half *, __half *, long long, cudaStream_t);
+template void launch_swiglu<float>(const float *, const float *, float *, long long, cudaStream_t, unsigned int *);
+template void launch_swiglu<bf16>(const bf16 *, const bf16 *, bf16 *, long long, cudaStream_t, unsigned int *);
+template void launch_swiglu<__half>(const __half *, const __half *, __half *, long long, cudaStream_t, unsigned int *);
 
 // y[b, :] = x[idx[b], :]   (the tokens that continue past layer l: the last token of each prompt)
 __global__ void gather_rows_kernel(const float *__restrict__ x, const int32_t *__restrict__ idx, float *__restrict__ y, int d) {
@@ -330,9 +363,17 @@ template void launch_fold<bf16, __half>(const bf16 *, const bf16 *, __half *, in
 __global__ void gather_kv_half_kernel(const bf16 *__restrict__ k, const bf16 *__restrict__ v, __half *__restrict__ k16,
                                       __half *__restrict__ v16, const int32_t *__restrict__ row0,
                                       const int32_t *__restrict__ len, const int32_t *__restrict__ kcu,
-                                      const int32_t *__restrict__ blk, int blk_stride, int dkv) {
+                                      const int32_t *__restrict__ blk, int blk_stride, int dkv, unsigned int *status) {
   const int b = blockIdx.y, r = blockIdx.x;
   if (r >= len[b]) return;
+  bool hit = false;
+  auto cvt = [&](__nv_bfloat162 x) {       // bf16 pair -> half pair, clamped to the half range (a bf16 may lie beyond it)
+    float2 f = __bfloat1622float2(x);
+    hit |= fabsf(f.x) >= HALF_OVERFLOW || fabsf(f.y) >= HALF_OVERFLOW;
+    f.x = fminf(fmaxf(f.x, -65504.f), 65504.f);
+    f.y = fminf(fmaxf(f.y, -65504.f), 65504.f);
+    return __float22half2_rn(f);
+  };
   const size_t src = kv_row_of(blk, blk_stride, b, row0[b], r) * dkv, dst = ((size_t)kcu[b] + r) * dkv;
   for (int i = threadIdx.x * 8; i < dkv; i += blockDim.x * 8) {
     const uint4 kr = *reinterpret_cast<const uint4 *>(k + src + i), vr = *reinterpret_cast<const uint4 *>(v + src + i);
@@ -340,20 +381,22 @@ __global__ void gather_kv_half_kernel(const bf16 *__restrict__ k, const bf16 *__
     uint4 ko, vo;
     __half2 *ko2 = reinterpret_cast<__half2 *>(&ko), *vo2 = reinterpret_cast<__half2 *>(&vo);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) { ko2[q] = __float22half2_rn(__bfloat1622float2(k2[q])); vo2[q] = __float22half2_rn(__bfloat1622float2(v2[q])); }
+    for (int q = 0; q < 4; ++q) { ko2[q] = cvt(k2[q]); vo2[q] = cvt(v2[q]); }
     *reinterpret_cast<uint4 *>(k16 + dst + i) = ko;
     *reinterpret_cast<uint4 *>(v16 + dst + i) = vo;
   }
+  report_overflow(hit, status);
 }
 void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v16, const int32_t *row0, const int32_t *len,
                            const int32_t *kcu, const int32_t *blk, int blk_stride, int n_seqs, int max_len, int dkv,
-                           cudaStream_t st) {
+                           cudaStream_t st, unsigned int *status) {
   if (n_seqs <= 0 || max_len <= 0) return;
-  gather_kv_half_kernel<<<dim3(max_len, n_seqs), 128, 0, st>>>(k, v, k16, v16, row0, len, kcu, blk, blk_stride, dkv);
+  gather_kv_half_kernel<<<dim3(max_len, n_seqs), 128, 0, st>>>(k, v, k16, v16, row0, len, kcu, blk, blk_stride, dkv, status);
 }
 
 // bfloat16 -> IEEE half copy of a weight matrix (exact for |w| >= 2^-17, absolute error <= 2^-25 below), 128-bit accesses
-__global__ void bf16_to_f16_kernel(const bf16 *__restrict__ src, __half *__restrict__ dst, long long n) {
+__global__ void bf16_to_f16_kernel(const bf16 *__restrict__ src, __half *__restrict__ dst, long long n, unsigned int *status) {
+  bool hit = false;
   const long long stride = (long long)gridDim.x * blockDim.x;
   const long long nv = n / 8;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += stride) {
@@ -362,18 +405,28 @@ __global__ void bf16_to_f16_kernel(const bf16 *__restrict__ src, __half *__restr
     uint4 o;
     __half2 *o2 = reinterpret_cast<__half2 *>(&o);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) o2[k] = __float22half2_rn(__bfloat1622float2(in2[k]));
+    for (int k = 0; k < 4; ++k) {
+      float2 f = __bfloat1622float2(in2[k]);
+      hit |= fabsf(f.x) >= HALF_OVERFLOW || fabsf(f.y) >= HALF_OVERFLOW;     // a weight beyond the half range: clamped
+      f.x = fminf(fmaxf(f.x, -65504.f), 65504.f);
+      f.y = fminf(fmaxf(f.y, -65504.f), 65504.f);
+      o2[k] = __float22half2_rn(f);
+    }
     reinterpret_cast<uint4 *>(dst)[i] = o;
   }
-  for (long long i = nv * 8 + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
-    dst[i] = __float2half_rn(__bfloat162float(src[i]));
+  for (long long i = nv * 8 + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const float f = __bfloat162float(src[i]);
+    hit |= fabsf(f) >= HALF_OVERFLOW;
+    dst[i] = __float2half_rn(fminf(fmaxf(f, -65504.f), 65504.f));
+  }
+  report_overflow(hit, status);
 }
-void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st) {
+void launch_bf16_to_f16(const bf16 *src, __half *dst, long long n, cudaStream_t st, unsigned int *status) {
   if (n <= 0) return;
   long long blocks = (n / 8 + 255) / 256;
   if (blocks < 1) blocks = 1;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  bf16_to_f16_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, dst, n);
+  bf16_to_f16_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, dst, n, status);
 }
 
 }  // namespace skv

@@ -166,12 +166,13 @@ __device__ __forceinline__ void tile_coords(int tile, int num_m_blocks, int num_
   m_blk = band * group_m + (r - n_blk * band_h);
 }
 
-__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status) {
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int *abort_flag, unsigned int *status,
+                                              long long limit = tc::WAIT_LIMIT_CLOCKS) {
   if (tc::mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (!tc::mbar_try_wait(bar, parity)) {
     if (*abort_flag) return false;
-    if (clock64() - t0 > tc::WAIT_LIMIT_CLOCKS) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       atomicOr(status, STATUS_TIMEOUT);
       return false;
@@ -182,8 +183,10 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
 
 // One thread = one accumulator row (TMEM lane): apply the epilogue to the BN columns at t_row and write them out.
 // Warp-collective (tcgen05.ld): every lane of the warp must call it, also for rows beyond M.
+// amax: running maximum magnitude of the values this thread stored as IEEE halves (checked against the half range once,
+// when the CTA is done)
 template <int BN, int EPI>
-__device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_row, int row, int n_blk) {
+__device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_row, int row, int n_blk, float &amax) {
   constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
   if constexpr (SWIGLU) {
     constexpr int HALF = BN / 2;
@@ -199,7 +202,9 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
         for (int i = 0; i < 16; ++i) {
           const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
           const float u0 = __uint_as_float(u[2 * i]), u1 = __uint_as_float(u[2 * i + 1]);
-          pk[i] = tc::pack_act(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1, p.f16 != 0);
+          const float y0 = g0 / (1.f + __expf(-g0)) * u0, y1 = g1 / (1.f + __expf(-g1)) * u1;
+          amax = fmaxf(amax, fmaxf(fabsf(y0), fabsf(y1)));
+          pk[i] = tc::pack_act(y0, y1, p.f16 != 0);
         }
         uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * p.F + (size_t)n_blk * HALF + c * 32);
 #pragma unroll
@@ -249,6 +254,10 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
                 bq[4 * i + e] = __float_as_uint(y * cc4[e] + x * ss4[e]);
               }
             }
+          }
+          if (f16 || dupp) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fmaxf(fabsf(__uint_as_float(a[i])), fabsf(__uint_as_float(bq[i]))));
           }
           uint4 *d0 = reinterpret_cast<uint4 *>(dstp + c * 32);
           uint4 *d1 = reinterpret_cast<uint4 *>(dstp + 64 + c * 32);
@@ -309,6 +318,10 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
             const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
             const size_t srow = p.out.slot_map ? (size_t)p.out.slot_map[row] : (size_t)row;
             dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + srow * p.out.seg_w + within;
+          }
+          if (f16) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(r[i])));
           }
           uint4 *dst = reinterpret_cast<uint4 *>(dstp);
 #pragma unroll
@@ -428,6 +441,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // -------------------------------------------------- epilogue warps (2..5)
     const int quarter = warp & 3;   // the TMEM lane quarter this warp may read
     int it = 0;
+    float amax = 0.f;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
       int m_blk, n_blk;
       tile_coords(tile, p.num_m_blocks, p.num_n_blocks, p.group_m, m_blk, n_blk);
@@ -437,11 +451,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc::tc_fence_after_sync();
       const int row = m_blk * BM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-      epilogue_rows<BN, EPI>(p, t_row, row, n_blk);
+      epilogue_rows<BN, EPI>(p, t_row, row, n_blk, amax);
       tc::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(tc::smem_u32(&tempty_bar[acc]));
     }
+    if ((p.f16 || p.dup_base) && amax >= HALF_OVERFLOW) atomicOr(p.status, STATUS_ACT_OVERFLOW);   // a half store was clamped
   }
   tc::tc_fence_before_sync();
   __syncthreads();
@@ -593,6 +608,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t leader_tempty0 = tc::mapa_shared(tc::smem_u32(&tempty_bar[0]), 0);
     const uint32_t leader_tempty1 = tc::mapa_shared(tc::smem_u32(&tempty_bar[1]), 0);
     int it = 0;
+    float amax = 0.f;
     for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
       int m2, n_blk;
       coords(tile, m2, n_blk);
@@ -602,11 +618,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tc::tc_fence_after_sync();
       const int row = m2 * 2 * BM + rank * BM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * PAIR_BN;
-      epilogue_rows<PAIR_BN, EPI>(p, t_row, row, n_blk);
+      epilogue_rows<PAIR_BN, EPI>(p, t_row, row, n_blk, amax);
       tc::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive_cluster(acc ? leader_tempty1 : leader_tempty0);
     }
+    if ((p.f16 || p.dup_base) && amax >= HALF_OVERFLOW) atomicOr(p.status, STATUS_ACT_OVERFLOW);
   }
   tc::tc_fence_before_sync();
   __syncthreads();
@@ -615,6 +632,29 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncwarp();
     tc::tc_fence_after_sync();
     tc::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+// see launch_bounded_wait_probe
+__global__ void __launch_bounds__(64) bounded_wait_probe_kernel(long long limit, unsigned int *status, unsigned int *outcome) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  volatile int *abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(&bar), 1);      // one arrival expected; nobody will ever arrive
+    abort_word = 0;
+    tc::fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    // the role that runs out of patience: same wait as every role of the GEMM kernels, short limit
+    const bool ok = wait_or_abort(tc::smem_u32(&bar), 0, abort_flag, status, limit);
+    outcome[0] = ok ? 0u : 1u;
+  } else if (threadIdx.x == 32) {
+    // a role with the full limit: it must leave because the first role raised the abort flag, not by its own clock
+    const long long t0 = clock64();
+    const bool ok = wait_or_abort(tc::smem_u32(&bar), 0, abort_flag, status);
+    outcome[1] = (!ok && clock64() - t0 < 2 * limit + 10000000) ? 1u : 0u;
   }
 }
 
@@ -643,6 +683,11 @@ int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b
 }
 
 }  // namespace
+
+int launch_bounded_wait_probe(long long limit_clocks, unsigned int *status, unsigned int *outcome, cudaStream_t st) {
+  bounded_wait_probe_kernel<<<1, 64, 0, st>>>(limit_clocks, status, outcome);
+  return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+}
 
 bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (N % 128) == 0 && N >= 128; }
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }

@@ -46,3 +46,21 @@ def test_reference_arm_is_rank0_only():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                         "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+def test_gpus_flag_without_a_launcher_starts_local_ranks():
+    """`bench.py --gpus 2` with no WORLD_SIZE in the environment starts itself as two local ranks (one process per GPU on
+    a GPU machine; here the host-only arm over gloo): rank 0 prints one line with the whole-job figures."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "hostcheck", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    sys.path.insert(0, ROOT)
+    import bench
+    assert out["n_gpus"] == 2 and out["max_time"] == 2.0
+    assert out["tokens"] == float(sum(bench.rank_batch(0)[1]) + sum(bench.rank_batch(1)[1]))
+    assert out["seq_lens_rank0"] == bench.rank_batch(0)[1]
