@@ -257,7 +257,30 @@ int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
  * Ignored by fp32 models.  Takes effect at the next prefill. */
 #define SWIFTKV_ACT_BF16 0
 #define SWIFTKV_ACT_F16  1
+/*   SWIFTKV_ACT_F16_SPLIT     : SWIFTKV_ACT_F16 with the error-critical operands of a whole-prompt prefill carried as PAIRS
+ *                      of halves, value = hi + lo (~22 significant bits), at the price of extra tensor-core passes:
+ *                      a GEMM whose A operand is a pair runs its K loop twice (A_hi B^T + A_lo B^T in one fp32
+ *                      accumulator), the attention scores take three passes (Q_hi K_hi^T + Q_lo K_hi^T + Q_hi K_lo^T).
+ *                      Which operands: swiftkv_set_split_mask, default SWIFTKV_SPLIT_DEFAULT.  For deep models whose
+ *                      softmax is so sharp that the 2^-12 rounding of h, q and K dominates the error of the logits (the
+ *                      80-layer 70B shape with random weights misses the 0.1 max-abs bar with plain halves).  Chunked /
+ *                      decode steps and the FP8 cache run as SWIFTKV_ACT_F16. */
+#define SWIFTKV_ACT_F16_SPLIT 2
 int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format);
+
+/* Operands that travel as half pairs under SWIFTKV_ACT_F16_SPLIT (bits; call after swiftkv_set_activation_format):
+ *   QKV_INPUT : the normed hidden state that feeds the Q/K/V projections and the SingleInputKV projection (those GEMMs x2)
+ *   SCORES    : q and K inside the attention kernel (Q K^T x3)
+ *   ATTN_OUT  : the attention output that feeds the O projection (x2; implies the half-pair attention kernel)
+ *   MLP_INPUT : the normed hidden state that feeds the gate / up projections (x2)
+ *   MLP_ACT   : the SwiGLU output that feeds the down projection (x2) */
+#define SWIFTKV_SPLIT_QKV_INPUT 1
+#define SWIFTKV_SPLIT_SCORES    2
+#define SWIFTKV_SPLIT_ATTN_OUT  4
+#define SWIFTKV_SPLIT_MLP_INPUT 8
+#define SWIFTKV_SPLIT_MLP_ACT   16
+#define SWIFTKV_SPLIT_DEFAULT   (SWIFTKV_SPLIT_QKV_INPUT | SWIFTKV_SPLIT_SCORES | SWIFTKV_SPLIT_ATTN_OUT)
+int32_t swiftkv_set_split_mask(swiftkv_model *m, int32_t mask);
 
 /* Failure-detection self-check (no counterpart in the paper).  Every wait inside the kernels is bounded: when it runs out
  * the kernel latches DEVICE_TIMEOUT in the model's status word, every role of the CTA leaves its loop and the kernel
@@ -285,6 +308,20 @@ void swiftkv_model_free(swiftkv_model *m);
  * Needs K % 64 == 0, N % 128 == 0, 16-byte aligned pointers.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
 int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K, int32_t dtype,
                         void *cuda_stream);
+
+/* The half-pair operand format of SWIFTKV_ACT_F16_SPLIT, stand-alone.  C[M,N] (DEVICE fp32, row-major, ldc = N) +=
+ * (A_hi + A_lo) B^T with A2 DEVICE IEEE half [M, 2K], each row [hi(K) | lo(K)], B IEEE half [N, K]; two tensor-core passes
+ * into one fp32 accumulator.  Same shape rules as swiftkv_gemm_tc.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_gemm_tc_split(const void *A2, const void *B, float *C, int32_t M, int32_t N, int32_t K, void *cuda_stream);
+
+/* Causal varlen GQA attention (Sec. 3.1) with the scores computed from half pairs: q = q_hi + q_lo [T, n_q, hd] and
+ * K = k_hi + k_lo [T, n_kv, hd] (all IEEE half), S = Q_hi K_hi^T + Q_lo K_hi^T + Q_hi K_lo^T; v and out IEEE half;
+ * out_split != 0: out is [T, 2 * n_q * hd], each row [hi | lo].  head_dim 128, even n_q / n_kv.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_attention_prefill_split(const void *q_hi, const void *q_lo, const void *k_hi, const void *k_lo, const void *v,
+                                        void *out, int32_t out_split, const int32_t *cu_seqlens, int32_t n_seqs,
+                                        int32_t total_tokens, int32_t max_seq_len, int32_t n_q_heads, int32_t n_kv_heads,
+                                        int32_t head_dim, void *cuda_stream);
 
 /* Causal varlen grouped-query attention (Sec. 3.1) on packed prompts.  q [T, n_q, hd] and out [T, n_q*hd] in
  * q_dtype, k, v [T, n_kv, hd] in kv_dtype; cu_seqlens DEVICE int32 [n_seqs+1]; softmax scale 1/sqrt(hd).

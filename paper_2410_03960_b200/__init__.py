@@ -6,12 +6,20 @@ PyTorch is used for device memory and streams.
 from .binding import (  # noqa: F401
     ACT_BF16,
     ACT_F16,
+    ACT_F16_SPLIT,
+    SPLIT_ATTN_OUT,
+    SPLIT_MLP_ACT,
+    SPLIT_MLP_INPUT,
+    SPLIT_QKV_INPUT,
+    SPLIT_SCORES,
     KC_NAMES,
     KV_FP8,
     KV_MODEL_DTYPE,
     SwiftKVError,
     SwiftKVModel,
     attention_prefill,
+    attention_prefill_split,
+    gemm_tc_split,
     gemm_tc,
     library_path,
     load_library,

@@ -11,7 +11,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB: Optional[C.CDLL] = None
 
 DTYPE_F32, DTYPE_BF16, DTYPE_F16, DTYPE_FP8_E4M3 = 0, 1, 2, 3
-ACT_BF16, ACT_F16 = 0, 1
+ACT_BF16, ACT_F16, ACT_F16_SPLIT = 0, 1, 2
+SPLIT_QKV_INPUT, SPLIT_SCORES, SPLIT_ATTN_OUT, SPLIT_MLP_INPUT, SPLIT_MLP_ACT = 1, 2, 4, 8, 16
 KV_MODEL_DTYPE, KV_FP8 = 0, 1
 _DTYPE_CODE = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 KC_NAMES = ("gemm", "attention", "elementwise", "tail", "gemm_swiglu")
@@ -23,7 +24,8 @@ EXPORTS = (
     "swiftkv_profile_enable", "swiftkv_profile_read", "swiftkv_last_launch_count", "swiftkv_set_kernel_mask",
     "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
-    "swiftkv_debug_bounded_wait", "swiftkv_op_status",
+    "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
+    "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split",
 )
 
 
@@ -90,6 +92,9 @@ def load_library() -> C.CDLL:
     lib.swiftkv_model_free.argtypes = [C.c_void_p]
     lib.swiftkv_model_free.restype = None
     lib.swiftkv_set_activation_format.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_set_split_mask.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_gemm_tc_split.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+    lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
     lib.swiftkv_debug_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
@@ -276,8 +281,50 @@ class SwiftKVModel:
         return int(self.lib.swiftkv_set_kernel_mask(self._h, mask))
 
     def set_activation_format(self, fmt: int) -> None:
-        """swiftkv_set_activation_format: ACT_F16 (default) or ACT_BF16."""
+        """swiftkv_set_activation_format: ACT_F16 (default), ACT_BF16 or ACT_F16_SPLIT (half pairs)."""
         _check(self.lib.swiftkv_set_activation_format(self._h, fmt))
+
+    def set_split_mask(self, mask: int) -> None:
+        """swiftkv_set_split_mask: which operands travel as half pairs (SPLIT_* bits)."""
+        _check(self.lib.swiftkv_set_split_mask(self._h, mask))
+
+
+def split_halves(x: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """fp32 tensor -> (hi, lo) IEEE halves with hi + lo ~ x (marshalling of the half-pair operand format)."""
+    hi = x.to(torch.float16)
+    return hi, (x - hi.float()).to(torch.float16)
+
+
+def gemm_tc_split(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_gemm_tc_split: a fp32 [M, K] (sent as half pairs), b IEEE half [N, K] -> fp32 [M, N]."""
+    assert a.is_cuda and a.dtype == torch.float32 and b.dtype == torch.float16
+    hi, lo = split_halves(a)
+    a2 = torch.cat([hi, lo], dim=1).contiguous()
+    c = torch.zeros((a.shape[0], b.shape[0]), dtype=torch.float32, device=a.device)
+    with torch.cuda.device(a.device):
+        _check(load_library().swiftkv_gemm_tc_split(a2.data_ptr(), b.contiguous().data_ptr(), c.data_ptr(), a.shape[0],
+                                                    b.shape[0], a.shape[1], _stream_ptr(stream)))
+    return c
+
+
+def attention_prefill_split(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens: Sequence[int], out_split: bool = False,
+                            stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_attention_prefill_split: q fp32 [T, n_q, hd], k fp32 [T, n_kv, hd] (sent as half pairs), v IEEE half.
+    Returns fp32 [T, n_q*hd]: the half output, or hi + lo of the pair output when out_split."""
+    T, n_q, hd = q.shape
+    n_kv = k.shape[1]
+    qh, ql = split_halves(q.contiguous())
+    kh, kl = split_halves(k.contiguous())
+    cu = _cu_seqlens(seq_lens, q.device)
+    out = torch.zeros((T, (2 if out_split else 1) * n_q * hd), dtype=torch.float16, device=q.device)
+    with torch.cuda.device(q.device):
+        _check(load_library().swiftkv_attention_prefill_split(qh.data_ptr(), ql.data_ptr(), kh.data_ptr(), kl.data_ptr(),
+                                                              v.contiguous().data_ptr(), out.data_ptr(), int(out_split),
+                                                              cu.data_ptr(), len(seq_lens), T, max(seq_lens), n_q, n_kv, hd,
+                                                              _stream_ptr(stream)))
+    if out_split:
+        return out[:, :n_q * hd].float() + out[:, n_q * hd:].float()
+    return out.float()
 
 
 def gemm_tc(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

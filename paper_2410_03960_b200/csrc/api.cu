@@ -103,6 +103,7 @@ struct swiftkv_model {
   int kernel_mask = 55;
   int n_sms = 0;
   int act_format = SWIFTKV_ACT_F16;
+  int split_mask = 0;           // SWIFTKV_SPLIT_* bits: which operands travel as half pairs (SWIFTKV_ACT_F16_SPLIT)
   // profiling
   bool profiling = false;
   std::vector<cudaEvent_t> pool;
@@ -141,18 +142,20 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   const size_t E = dsize(c.dtype);
   const size_t d = c.hidden, dq = (size_t)c.n_q_heads * c.head_dim, F = c.ffn;
   const size_t chunk = std::min<size_t>(T, MLP_CHUNK_ROWS);
+  // (a 16-bit model's activation buffers hold two halves per element, so that the half-pair format fits)
+  const size_t P2 = c.dtype == SWIFTKV_DTYPE_BF16 ? 2 : 1;
   b.x = (float *)cv.take((size_t)T * d * 4);
-  b.h = cv.take((size_t)T * d * E);
-  b.q = cv.take((size_t)T * dq * E);
-  b.attn = cv.take((size_t)T * dq * E);
+  b.h = cv.take((size_t)T * d * E * P2);
+  b.q = cv.take((size_t)T * dq * E * P2);
+  b.attn = cv.take((size_t)T * dq * E * P2);
   b.gate = cv.take(chunk * F * E);
   b.up = cv.take(chunk * F * E);
-  b.act = cv.take((size_t)T * F * E);
+  b.act = cv.take((size_t)T * F * E * P2);
   b.wfold = cv.take(fold_elems * E);
   const size_t dkv_ = (size_t)c.n_kv_heads * c.head_dim;
   const bool bf = c.dtype == SWIFTKV_DTYPE_BF16;
   b.w16 = cv.take(bf ? 2 * (2 * d * dq + 2 * d * dkv_ + 3 * d * F) * 2 : 0);   // two layers: double buffer
-  b.kv16 = cv.take(bf ? (size_t)2 * T * dkv_ * 2 : 0);
+  b.kv16 = cv.take(bf ? (size_t)3 * T * dkv_ * 2 : 0);      // K, V and (half pairs) the low halves of K
   const bool fp8 = c.kv_format == SWIFTKV_KV_FP8;
   b.kvst = cv.take(fp8 ? (size_t)2 * T * dkv_ * E : 0);
   b.kvdq = cv.take(fp8 && !bf ? (size_t)2 * T * dkv_ * 4 : 0);
@@ -334,9 +337,10 @@ template <typename TA, typename TW>
 static int32_t gemm_any(swiftkv_model *m, const TA *A, int M, int K, const TW *B0, int n0, const TW *B1, int n1,
                         const TW *B2, int n2, const OutDesc &out, cudaStream_t st, const __half *Bh0 = nullptr,
                         const __half *Bh1 = nullptr, const __half *Bh2 = nullptr, const RopeSpec *rope = nullptr,
-                        bool *rope_fused = nullptr, void *dup = nullptr, long long dup_stride = 0) {
+                        bool *rope_fused = nullptr, void *dup = nullptr, long long dup_stride = 0, const GemmSplit *split = nullptr) {
   Scope sc(m, st, SWIFTKV_KC_GEMM, 0);
   if (rope_fused) *rope_fused = false;
+  if (split && !split->a_split && !split->lo_p0 && !split->lo_dup) split = nullptr;
   if constexpr (sizeof(TW) == 2) {
     constexpr bool f16 = std::is_same<TA, __half>::value;
     const bool have_b = !f16 || (Bh0 && (n1 == 0 || Bh1) && (n2 == 0 || Bh2));
@@ -346,14 +350,17 @@ static int32_t gemm_any(swiftkv_model *m, const TA *A, int M, int K, const TW *B
       const void *b2 = f16 ? (const void *)Bh2 : (const void *)B2;
       int rc = SWIFTKV_ERR_UNSUPPORTED;
       if (rope && rope_fused) {
-        rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, dup, dup_stride, rope, m->b.status, st);
+        rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, dup, dup_stride, rope, m->b.status, st, split);
         if (rc == SWIFTKV_OK) *rope_fused = true;
       }
-      if (rc == SWIFTKV_ERR_UNSUPPORTED) rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, nullptr, 0, nullptr, m->b.status, st);
+      const bool split_out = split && (split->lo_p0 || split->lo_dup);      // low halves come from the rotary epilogue only
+      if (rc == SWIFTKV_ERR_UNSUPPORTED && !split_out)
+        rc = launch_gemm_tc(A, f16, M, K, b0, n0, b1, n1, b2, n2, out, nullptr, 0, nullptr, m->b.status, st, split);
       if (rc == SWIFTKV_OK) { m->launches += 1; return rc; }
       if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "tensor-core GEMM launch failed: %s", cudaGetErrorString(cudaGetLastError()));
     }
   }
+  if (split) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-pair operands need the tensor-core GEMM (shape %d x %d x %d)", M, n0 + n1 + n2, K);
   OutDesc o = out;
   o.status = m->b.status;      // a clamped half store is reported like on the tensor-core path
   launch_gemm_simt<TA, TW>(A, B0, M, n0, K, o, 0, st);
@@ -408,6 +415,11 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const bool use_w16 = act_f16 && (m->kernel_mask & 1) && tc_gemm_supported(T_tok, dq, d) && tc_gemm_supported(T_tok, d, dq) &&
                        tc_gemm_supported(T_tok, d, F) && (dkv % 256 == 0) && (dq % 256 == 0) && c.head_dim == 128;
   const bool attn_tc = sizeof(T) == 2 && (m->kernel_mask & 2) && tc_attention_supported(c.n_q_heads, c.n_kv_heads, c.head_dim);
+  // half pairs (SWIFTKV_ACT_F16_SPLIT): which operands carry hi + lo halves in this pass.  Only the whole-prompt prefill on
+  // the tensor-core kernels has them; chunked / decode steps and the FP8 cache run as plain SWIFTKV_ACT_F16.
+  const int sm = (use_w16 && attn_tc && bt.plain && !fp8 && !bt.decode) ? m->split_mask : 0;
+  const bool sp_hin = sm & SWIFTKV_SPLIT_QKV_INPUT, sp_qk = (sm & (SWIFTKV_SPLIT_SCORES | SWIFTKV_SPLIT_ATTN_OUT)) != 0,
+             sp_ao = sm & SWIFTKV_SPLIT_ATTN_OUT, sp_hpost = sm & SWIFTKV_SPLIT_MLP_INPUT, sp_act = sm & SWIFTKV_SPLIT_MLP_ACT;
   AttnSchedule att_sched;
   if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; }
   const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
@@ -441,7 +453,8 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       convert_layer(0);
     }
   }
-  __half *k16 = (__half *)b.kv16, *v16 = k16 + plane;
+  __half *k16 = (__half *)b.kv16, *v16 = k16 + plane, *k_lo = v16 + plane;
+  __half *q_lo = (__half *)b.q + (size_t)m->max_tokens * dq;         // low halves of the queries: a second plane
 
   const int32_t *slot_map = bt.plain ? nullptr : b.slot;        // cache row of each new token (identity when plain)
   const int32_t *k_row0 = bt.plain ? nullptr : b.kv_row0;
@@ -541,8 +554,9 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
         cudaStreamWaitEvent(st, m->ev_ready[j & 1], 0);
       }
     }
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st, b.status); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.in_norm, h, T_tok, d, c.rms_eps, st, b.status, sp_hin); }
     OutDesc qkv{OUT_STORE, q, dq, dq, Kj, (long long)plane, dkv, slot_map};
+    const GemmSplit qkv_split{sp_hin, sp_qk ? (void *)q_lo : nullptr, sp_qk ? (void *)k_lo : nullptr};
     if (fp8) { Kj = kst; Vj = vst; qkv.seg_base = kst; qkv.slot_map = nullptr; }   // staging rows are in batch order
     bool roped = false;
     // the attention kernel reads half copies of this layer's K / V: written by the QKV epilogue for a plain prefill,
@@ -550,7 +564,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     const bool want_dup = use_w16 && attn_tc && bt.plain && !fp8;
     rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)lw.wq, dq, (const T *)lw.wk, dkv, (const T *)lw.wv, dkv, qkv, st,
                          use_w16 ? wq16 : nullptr, use_w16 ? wk16 : nullptr, use_w16 ? wv16 : nullptr, &rope, &roped,
-                         want_dup ? k16 : nullptr, (long long)plane);
+                         want_dup ? k16 : nullptr, (long long)plane, &qkv_split);
     if (rc) return rc;
     if (!roped) {
       { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<TA>(q, 0, 1, b.pos, nullptr, b.cos_tab, b.sin_tab, T_tok, c.n_q_heads, c.head_dim, st, b.status); }
@@ -597,8 +611,14 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       Scope s(m, st, SWIFTKV_KC_ATTENTION);
       bool done = false;
       if constexpr (sizeof(T) == 2) {
+        if (sp_qk) {     // scores from half pairs of q and K (three passes); output rows as [hi | lo] if the O projection wants them
+          rc = launch_attention_tc_split(q, q_lo, k16, k_lo, v16, attn, sp_ao, b.cu, B, T_tok, bt.max_new, c.n_q_heads, c.n_kv_heads,
+                                         c.head_dim, b.status, st);
+          if (rc) return fail(rc, "half-pair attention launch failed");
+          done = true;
+        }
         // (half activations: the kernel needs half copies of K and V -- from the QKV epilogue, or gathered here)
-        if (attn_tc && (!act_f16 || (use_w16 && roped))) {
+        if (!done && attn_tc && (!act_f16 || (use_w16 && roped))) {
           const void *kk = Kj, *vv = Vj;
           const int32_t *kr0 = k_row0;
           int kv_rows = bt.plain ? T_tok : m->max_tokens;
@@ -621,20 +641,22 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       }
       if (!done) launch_attention_simple<TA, T>(q, Kj, Vj, attn, b.cu, B, k_row0, kv_len, blk, bt.blk_stride, T_tok, c.n_q_heads, c.n_kv_heads, c.head_dim, st);
     }
+    const GemmSplit o_split{sp_ao, nullptr, nullptr}, down_split{sp_act, nullptr, nullptr};
     rc = gemm_any<TA, T>(m, attn, T_tok, dq, (const T *)lw.wo, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
-                         use_w16 ? wo16 : nullptr);
+                         use_w16 ? wo16 : nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, &o_split);
     if (rc) return rc;
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st, b.status); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)lw.post_norm, h, T_tok, d, c.rms_eps, st, b.status, sp_hpost); }
     bool fused = false;
     if constexpr (sizeof(T) == 2) {
       if ((m->kernel_mask & 1) && tc_swiglu_supported(T_tok, F, d) && (!act_f16 || use_w16)) {
         Scope s(m, st, SWIFTKV_KC_SWIGLU);
         const void *wg = act_f16 ? (const void *)wg16 : lw.w_gate, *wu = act_f16 ? (const void *)wu16 : lw.w_up;
-        rc = launch_gemm_tc_swiglu(h, act_f16, T_tok, d, wg, wu, F, act, b.status, st);
+        rc = launch_gemm_tc_swiglu(h, act_f16, T_tok, d, wg, wu, F, act, b.status, st, sp_hpost, sp_act);
         if (rc == SWIFTKV_OK) fused = true;
         else if (rc != SWIFTKV_ERR_UNSUPPORTED) return fail(rc, "SwiGLU GEMM launch failed");
       }
     }
+    if (!fused && (sp_hpost || sp_act)) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-pair MLP operands need the fused gate/up kernel");
     if (!fused) {
       for (int r0 = 0; r0 < T_tok; r0 += MLP_CHUNK_ROWS) {
         const int rows = std::min(MLP_CHUNK_ROWS, T_tok - r0);
@@ -649,14 +671,15 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       }
     }
     rc = gemm_any<TA, T>(m, act, T_tok, F, (const T *)lw.w_down, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
-                         use_w16 ? wd16 : nullptr);
+                         use_w16 ? wd16 : nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, &down_split);
     if (rc) return rc;
     if (use_w16) cudaEventRecord(m->ev_free[j & 1], st);   // this layer's half copies may be overwritten
   }
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
   if (l < L && !bt.decode) {
-    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st, b.status); }
+    { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rmsnorm<T, TA>(b.x, (const T *)nullptr, h, T_tok, d, c.rms_eps, st, b.status, sp_hin); }
+    const GemmSplit kv_split{sp_hin, nullptr, nullptr};
     if (fp8) {
       // one group at a time through the staging planes: projection (+ RoPE on K), then the quantizing row pass into the
       // group's cache slot
@@ -678,7 +701,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     OutDesc o{OUT_STORE, nullptr, 0, 0, slot_l, (long long)plane, dkv, slot_map};
     bool roped = false;
     rc = gemm_any<TA, T>(m, h, T_tok, d, (const T *)b.wfold, ng * 2 * dkv, no_w, 0, no_w, 0, o, st,
-                         use_w16 ? (const __half *)b.wfold : nullptr, nullptr, nullptr, &rope, &roped);
+                         use_w16 ? (const __half *)b.wfold : nullptr, nullptr, nullptr, &rope, &roped, nullptr, 0, &kv_split);
     if (rc) return rc;
     if (use_w16 && !roped) return fail(SWIFTKV_ERR_UNSUPPORTED, "half-folded SingleInputKV weight needs the tensor-core GEMM");
     if (!roped) { Scope s(m, st, SWIFTKV_KC_ELEMWISE); launch_rope<T>(slot_l, (long long)(2 * plane), ng, b.pos, slot_map, b.cos_tab, b.sin_tab, T_tok, c.n_kv_heads, c.head_dim, st); }
@@ -974,8 +997,18 @@ extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
 
 extern "C" int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format) {
   if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
-  if (format != SWIFTKV_ACT_BF16 && format != SWIFTKV_ACT_F16) return fail(SWIFTKV_ERR_INVALID_ARG, "unknown activation format");
-  m->act_format = format;
+  if (format != SWIFTKV_ACT_BF16 && format != SWIFTKV_ACT_F16 && format != SWIFTKV_ACT_F16_SPLIT)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "unknown activation format");
+  m->act_format = format == SWIFTKV_ACT_F16_SPLIT ? SWIFTKV_ACT_F16 : format;
+  m->split_mask = format == SWIFTKV_ACT_F16_SPLIT ? SWIFTKV_SPLIT_DEFAULT : 0;
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_set_split_mask(swiftkv_model *m, int32_t mask) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if (mask < 0 || mask > 31) return fail(SWIFTKV_ERR_INVALID_ARG, "split mask outside [0, 31]");
+  if (mask && m->act_format != SWIFTKV_ACT_F16) return fail(SWIFTKV_ERR_INVALID_ARG, "half pairs need IEEE-half activations");
+  m->split_mask = mask;
   return SWIFTKV_OK;
 }
 
@@ -1035,6 +1068,37 @@ extern "C" int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_
   int rc = launch_gemm_tc(A, f16, M, K, B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N), nullptr, 0, nullptr,
                           status, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_gemm_tc_split(const void *A2, const void *B, float *C, int32_t M, int32_t N, int32_t K,
+                                         void *cuda_stream) {
+  if (!A2 || !B || !C || M < 1 || N < 1 || K < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "bad argument");
+  if (((uintptr_t)A2 | (uintptr_t)B | (uintptr_t)C) & 15) return fail(SWIFTKV_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  if (!tc_gemm_supported(M, N, K)) return fail(SWIFTKV_ERR_UNSUPPORTED, "needs K %% 64 == 0 and N %% 128 == 0");
+  unsigned int *status = op_status_word();
+  if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+  const GemmSplit split{true, nullptr, nullptr};
+  int rc = launch_gemm_tc(A2, true, M, K, B, N, nullptr, 0, nullptr, 0, out_plain(OUT_RESID_ADD_F32, C, N, N), nullptr, 0, nullptr,
+                          status, reinterpret_cast<cudaStream_t>(cuda_stream), &split);
+  if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_attention_prefill_split(const void *q_hi, const void *q_lo, const void *k_hi, const void *k_lo,
+                                                   const void *v, void *out, int32_t out_split, const int32_t *cu_seqlens,
+                                                   int32_t n_seqs, int32_t total_tokens, int32_t max_seq_len, int32_t n_q_heads,
+                                                   int32_t n_kv_heads, int32_t head_dim, void *cuda_stream) {
+  if (!q_hi || !q_lo || !k_hi || !k_lo || !v || !out || !cu_seqlens) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (n_seqs < 1 || total_tokens < 1 || max_seq_len < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "bad shape");
+  if (!tc_attention_supported(n_q_heads, n_kv_heads, head_dim))
+    return fail(SWIFTKV_ERR_UNSUPPORTED, "needs head_dim 128 and an even number of query heads per KV head");
+  unsigned int *status = op_status_word();
+  if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+  int rc = launch_attention_tc_split(q_hi, q_lo, k_hi, k_lo, v, out, out_split != 0, cu_seqlens, n_seqs, total_tokens, max_seq_len,
+                                     n_q_heads, n_kv_heads, head_dim, status, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (rc) return fail(rc, "attention launch failed");
   return SWIFTKV_OK;
 }
 

@@ -707,6 +707,293 @@ attention_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmQ, const __
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Extended-precision scores (activation format "half pairs"): q and K each arrive as a pair of half tensors, value =
+// hi + lo, and S = Q K^T is accumulated from three tensor-core passes  Q_hi K_hi^T + Q_lo K_hi^T + Q_hi K_lo^T  (the
+// lo-lo term is below fp32 rounding), so the scores carry ~22 significant bits of q and K instead of 11.  This is for
+// models whose softmax is so sharp that the 2^-12 rounding of q and K dominates the end-to-end error (the 80-layer
+// 70B shape with random weights).  Everything else is attention_tc_kernel: same roles, same softmax, P and V as single
+// halves.  Shared memory: Q 4 tiles (hi, lo of two heads) + K 2 tiles (hi, lo) + V 1 tile = 224 KB, so the K and V
+// rings have one stage each: the next key tile's K lands while the softmax warps work on the current scores, the next V
+// while they work on the next scores.  out_split: output rows are [hi | lo] pairs, 2 * n_q * hd elements apart.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int SPL_SM_Q = 0, SPL_SM_K = 4 * TILE_BYTES, SPL_SM_V = 6 * TILE_BYTES, SPL_SM_BAR = 7 * TILE_BYTES;
+constexpr int SPL_SMEM = SPL_SM_BAR + 256 + 1024;
+
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attention_tc_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmQlo,
+                          const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmKlo,
+                          const __grid_constant__ CUtensorMap tmV, AttnParams p, int out_split) {
+  const int n_pairs = p.n_q >> 1;
+  const int per_tile = p.n_seqs * n_pairs;
+  const int qt = p.max_tiles - 1 - (int)(blockIdx.x / per_tile);
+  const int rem = blockIdx.x % per_tile;
+  const int b = rem / n_pairs, pair = rem % n_pairs;
+  const int tok0 = p.cu[b], n = p.cu[b + 1] - tok0;
+  if (qt * BQ >= n) return;
+  const int k0 = p.k_row0 ? p.k_row0[b] : tok0;
+  const int past = p.kv_len ? p.kv_len[b] - n : 0;
+  const int h0 = pair * 2;
+  const int kvh = h0 / (p.n_q / p.n_kv);
+  const int n_kv_tiles = (past + min(n, (qt + 1) * BQ) - 1) / BKV + 1;
+  const int q_row0 = tok0 + qt * BQ;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SPL_SM_BAR);
+  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 2, *v_full = bars + 3, *v_empty = bars + 4;
+  uint64_t *s_full = bars + 5;        // [2]
+  uint64_t *p_ready = bars + 7;       // [2]
+  uint64_t *p_ready2 = bars + 9;      // [2]
+  uint64_t *o_full = bars + 11;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 12);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(tc::smem_u32(q_full), 1);
+    tc::mbar_init(tc::smem_u32(k_full), 1);
+    tc::mbar_init(tc::smem_u32(k_empty), 1);
+    tc::mbar_init(tc::smem_u32(v_full), 1);
+    tc::mbar_init(tc::smem_u32(v_empty), 1);
+    for (int w = 0; w < 2; ++w) {
+      tc::mbar_init(tc::smem_u32(&s_full[w]), 1);
+      tc::mbar_init(tc::smem_u32(&p_ready[w]), 4);
+      tc::mbar_init(tc::smem_u32(&p_ready2[w]), 4);
+    }
+    tc::mbar_init(tc::smem_u32(o_full), 1);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+    tc::tma_prefetch_desc(&tmQ);
+    tc::tma_prefetch_desc(&tmQlo);
+    tc::tma_prefetch_desc(&tmK);
+    tc::tma_prefetch_desc(&tmKlo);
+    tc::tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), 512);
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  tc::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ TMA producer
+      const uint32_t qb = tc::smem_u32(q_full);
+      tc::mbar_expect_tx(qb, 4 * TILE_BYTES);
+      for (int w = 0; w < 2; ++w)
+        for (int c = 0; c < 2; ++c) {
+          tc::tma_load_2d(tc::smem_u32(smem + SPL_SM_Q + w * TILE_BYTES + c * CHUNK_BYTES), &tmQ, qb, (h0 + w) * HD + c * 64, q_row0);
+          tc::tma_load_2d(tc::smem_u32(smem + SPL_SM_Q + (2 + w) * TILE_BYTES + c * CHUNK_BYTES), &tmQlo, qb, (h0 + w) * HD + c * 64, q_row0);
+        }
+      for (int j = 0; j < n_kv_tiles; ++j) {
+        const uint32_t ph = j & 1;
+        const int krow = p.blk ? p.blk[(size_t)b * p.blk_stride + j] * BKV : k0 + j * BKV;
+        if (!wait_or_abort(tc::smem_u32(k_empty), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t kb = tc::smem_u32(k_full);
+        tc::mbar_expect_tx(kb, 2 * TILE_BYTES);
+        for (int c = 0; c < 2; ++c) {
+          tc::tma_load_2d(tc::smem_u32(smem + SPL_SM_K + c * CHUNK_BYTES), &tmK, kb, kvh * HD + c * 64, krow);
+          tc::tma_load_2d(tc::smem_u32(smem + SPL_SM_K + TILE_BYTES + c * CHUNK_BYTES), &tmKlo, kb, kvh * HD + c * 64, krow);
+        }
+        if (!wait_or_abort(tc::smem_u32(v_empty), ph ^ 1, abort_flag, p.status)) break;
+        const uint32_t vb = tc::smem_u32(v_full);
+        tc::mbar_expect_tx(vb, TILE_BYTES);
+        for (int c = 0; c < 2; ++c)
+          tc::tma_load_2d(tc::smem_u32(smem + SPL_SM_V + c * CHUNK_BYTES), &tmV, vb, kvh * HD + c * 64, krow);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (warp-uniform, one elected lane)
+    const bool leader = tc::elect_one();
+    constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, 1, 1);
+    constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, 1, 1);
+    const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SPL_SM_Q), 16, 1024);
+    const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SPL_SM_K), 16, 1024);
+    const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SPL_SM_V), CHUNK_BYTES, 1024);
+    auto issue_qk = [&](int w) {   // S_w = Q_hi K_hi^T + Q_lo K_hi^T + Q_hi K_lo^T, 8 steps of 16 along the head dim each
+      const uint64_t qh = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), ql = q_desc0 + (uint64_t)((2 + w) * (TILE_BYTES >> 4));
+      const uint64_t kh = k_desc0, kl = k_desc0 + (uint64_t)(TILE_BYTES >> 4);
+      const uint32_t d = tmem_base + w * 128;
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
+        tc::umma_ss(d, qh + off, kh + off, idesc_qk, kk != 0);
+        tc::umma_ss(d, ql + off, kh + off, idesc_qk, 1u);
+        tc::umma_ss(d, qh + off, kl + off, idesc_qk, 1u);
+      }
+    };
+    auto issue_pv = [&](int w, bool accumulate, int half) {
+      const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
+#pragma unroll
+      for (int k4 = 0; k4 < 4; ++k4) {
+        const int kk = half * 4 + k4;
+        tc::umma_ts(d, a_t + kk * 8, v_desc0 + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
+      }
+    };
+    const uint32_t b_kf = tc::smem_u32(k_full), b_ke = tc::smem_u32(k_empty), b_vf = tc::smem_u32(v_full), b_ve = tc::smem_u32(v_empty),
+                   b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]), b_p2 = tc::smem_u32(&p_ready2[0]);
+    auto wait = [&](uint32_t bar, uint32_t parity) {
+      const bool ok = wait_or_abort(bar, parity, abort_flag, p.status);
+      tc::tc_fence_after_sync();
+      return ok;
+    };
+    bool ok = wait(tc::smem_u32(q_full), 0) && wait(b_kf, 0);
+    if (ok && leader) {
+      issue_qk(0);
+      tc::umma_commit(b_sf);
+      issue_qk(1);
+      tc::umma_commit(b_sf + 8);
+      tc::umma_commit(b_ke);
+    }
+    for (int j = 0; j < n_kv_tiles && ok; ++j) {
+      const uint32_t ph = j & 1;
+      const bool more = j + 1 < n_kv_tiles, acc = j > 0;
+      if (!wait(b_vf, ph) || !wait(b_p1, ph)) { ok = false; break; }
+      if (leader) issue_pv(0, acc, 0);
+      if (!wait(b_p2, ph)) { ok = false; break; }
+      if (leader) issue_pv(0, acc, 1);
+      if (more) {
+        if (!wait(b_kf, ph ^ 1)) { ok = false; break; }
+        if (leader) {
+          issue_qk(0);
+          tc::umma_commit(b_sf);
+        }
+      }
+      if (!wait(b_p1 + 8, ph)) { ok = false; break; }
+      if (leader) issue_pv(1, acc, 0);
+      if (!wait(b_p2 + 8, ph)) { ok = false; break; }
+      if (leader) {
+        issue_pv(1, acc, 1);
+        tc::umma_commit(b_ve);
+        if (more) {
+          issue_qk(1);
+          tc::umma_commit(b_sf + 8);
+          tc::umma_commit(b_ke);
+        }
+      }
+    }
+    if (ok && leader) tc::umma_commit(tc::smem_u32(o_full));
+    __syncwarp();
+  } else {
+    // -------------------------------------------------------------- softmax warps: head w, one row per thread
+    const int w = (warp - 2) >> 2;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t t_s = tmem_base + lane_base + w * 128;
+    const uint32_t t_o = tmem_base + lane_base + 256 + w * 128;
+    const float c = p.scale_log2;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv_tiles; ++j) {
+      if (!wait_or_abort(tc::smem_u32(&s_full[w]), j & 1, abort_flag, p.status)) { ok = false; break; }
+      tc::tc_fence_after_sync();
+      const int shift = past + qt * BQ - j * BKV;
+      const bool diag = shift < BKV - 1;
+      const int lim = row + shift;
+      uint32_t s[128];
+      tc::tmem_ld_32x32b_x32p(t_s, s);
+      tc::tmem_ld_32x32b_x32p(t_s + 32, s + 32);
+      tc::tmem_ld_32x32b_x32p(t_s + 64, s + 64);
+      tc::tmem_ld_32x32b_x32p(t_s + 96, s + 96);
+      tc::tmem_ld_wait();
+      if (diag) {
+#pragma unroll
+        for (int i = 0; i < 128; ++i)
+          if (i > lim) s[i] = 0xff800000u;   // -inf
+      }
+      float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 8) {
+        m0 = tc::max3(m0, __uint_as_float(s[i]), __uint_as_float(s[i + 1]));
+        m1 = tc::max3(m1, __uint_as_float(s[i + 2]), __uint_as_float(s[i + 3]));
+        m2 = tc::max3(m2, __uint_as_float(s[i + 4]), __uint_as_float(s[i + 5]));
+        m3 = tc::max3(m3, __uint_as_float(s[i + 6]), __uint_as_float(s[i + 7]));
+      }
+      const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+      const bool need = (j == 0) || ((mx - m_ref) * c > RESCALE_THRESHOLD);
+      const float m_new = need ? mx : m_ref;
+      if (j > 0 && __any_sync(0xffffffffu, need)) {
+        const float f = need ? fast_exp2((m_ref - m_new) * c) : 1.f;
+        l *= f;
+#pragma unroll 1
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t r[16];
+          tc::tmem_ld_32x32b_x16(t_o + ch * 16, r);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+          tc::tmem_st_32x32b_x16(t_o + ch * 16, r);
+        }
+      }
+      m_ref = m_new;
+      const float neg_mc = -m_ref * c;
+      float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+#pragma unroll
+        for (int i = hf * 32; i < hf * 32 + 32; i += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * i]), c, neg_mc));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 1]), c, neg_mc));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 2]), c, neg_mc));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * i + 3]), c, neg_mc));
+          l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+          s[i] = tc::pack_f16x2(p0, p1);
+          s[i + 1] = tc::pack_f16x2(p2, p3);
+        }
+        tc::tmem_st_32x32b_x32(t_s + hf * 32, s + hf * 32);
+        tc::tmem_st_wait();
+        tc::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(tc::smem_u32(hf == 1 ? &p_ready2[w] : &p_ready[w]));
+      }
+      l += (l0 + l1) + (l2 + l3);
+    }
+    // ---- epilogue: O_w / l -> half (and the low halves, if asked for) -> out[token, head, :]
+    if (ok && wait_or_abort(tc::smem_u32(o_full), 0, abort_flag, p.status)) {
+      tc::tc_fence_after_sync();
+      const float inv = 1.f / l;
+      const bool valid = qt * BQ + row < n;
+      const size_t dq = (size_t)p.n_q * HD;
+      const size_t o_off = (size_t)(q_row0 + row) * (out_split ? 2 * dq : dq) + (size_t)(h0 + w) * HD;
+      __half *out_lo = out_split ? reinterpret_cast<__half *>(p.out) + dq : nullptr;
+#pragma unroll 1
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t r[32];
+        tc::tmem_ld_32x32b_x32(t_o + ch * 32, r);
+        tc::tmem_ld_wait();
+        if (valid) {
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float a = __uint_as_float(r[2 * i]) * inv, bq = __uint_as_float(r[2 * i + 1]) * inv;
+            hi[i] = tc::pack_f16x2(a, bq);
+            const float2 hf2 = __half22float2(*reinterpret_cast<const __half2 *>(&hi[i]));
+            lo[i] = tc::pack_f16x2(a - hf2.x, bq - hf2.y);
+          }
+          uint4 *d4 = reinterpret_cast<uint4 *>(p.out + o_off + ch * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) d4[i] = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+          if (out_lo) {
+            uint4 *l4 = reinterpret_cast<uint4 *>(out_lo + o_off + ch * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) l4[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+          }
+        }
+      }
+    }
+  }
+  tc::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tc_fence_after_sync();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
 }  // namespace
 
 int attention_schedule(const int32_t *n_new, const int32_t *n_past, int n_seqs, int n_q, int n_ctas, int32_t *off, int32_t *items) {
@@ -787,6 +1074,31 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
     if (split) attention_tc_kernel<false, true><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
     else attention_tc_kernel<false, false><<<(unsigned)grid, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p);
   }
+  return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+}
+
+int launch_attention_tc_split(const void *q_hi, const void *q_lo, const void *k_hi, const void *k_lo, const void *v, void *out,
+                              bool out_split, const int32_t *cu_seqlens, int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv,
+                              int hd, unsigned int *status, cudaStream_t st) {
+  if (!tc_attention_supported(n_q, n_kv, hd)) return SWIFTKV_ERR_UNSUPPORTED;
+  if (n_tokens < 1 || n_seqs < 1 || max_seq_len < 1) return SWIFTKV_ERR_INVALID_ARG;
+  CUtensorMap tq, tql, tk, tkl, tv;
+  if (get_tmap(&tq, q_hi, n_tokens, (uint64_t)n_q * hd, (uint64_t)n_q * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tql, q_lo, n_tokens, (uint64_t)n_q * hd, (uint64_t)n_q * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tk, k_hi, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tkl, k_lo, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (get_tmap(&tv, v, n_tokens, (uint64_t)n_kv * hd, (uint64_t)n_kv * hd, 128, 64)) return SWIFTKV_ERR_CUDA;
+  if (ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_split_kernel), SPL_SMEM)) return SWIFTKV_ERR_CUDA;
+  AttnParams p{};
+  p.cu = cu_seqlens; p.k_row0 = nullptr; p.kv_len = nullptr; p.blk = nullptr; p.blk_stride = 0;
+  p.out = reinterpret_cast<bf16 *>(out); p.n_seqs = n_seqs; p.n_q = n_q; p.n_kv = n_kv;
+  p.max_tiles = (max_seq_len + BQ - 1) / BQ;
+  p.scale_log2 = (1.0f / sqrtf((float)hd)) * 1.4426950408889634f;
+  p.status = status;
+  p.store32 = 0;
+  const long long grid = (long long)p.max_tiles * n_seqs * (n_q / 2);
+  if (grid > 0x7fffffffLL) return SWIFTKV_ERR_UNSUPPORTED;
+  attention_tc_split_kernel<<<(unsigned)grid, ATT_THREADS, SPL_SMEM, st>>>(tq, tql, tk, tkl, tv, p, out_split ? 1 : 0);
   return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
 }
 

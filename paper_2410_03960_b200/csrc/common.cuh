@@ -121,8 +121,10 @@ void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions,
 // status (nullable): receives STATUS_ACT_OVERFLOW when TO is IEEE half and a value had to be clamped (the same holds for
 // the other launches below that take a status word)
 template <typename TG, typename TO>
+// split (TO = IEEE half only): out is [rows, 2d], each row [hi(d) | lo(d)] with lo = y - float(hi): the A operand of a
+// GEMM launched with GemmSplit::a_split
 void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st,
-                    unsigned int *status = nullptr);
+                    unsigned int *status = nullptr, bool split = false);
 // in-place rotary embedding on `n_batches` tensors [*, n_heads, hd] spaced batch_stride elements apart; logical row r
 // (position positions[r]) lives in tensor row slot_map[r] (null: row r)
 template <typename T>
@@ -185,12 +187,23 @@ struct RopeSpec {
 // f16: A, every B and the columns below out.n0 hold IEEE halves instead of bfloat16 (same type on both operands);
 // columns routed to segments (the K / V cache planes) are always stored as bfloat16, and -- if dup_base is given --
 // stored a second time as halves at dup_base + segment * dup_stride (the attention kernel's operand copy)
+// split (optional, IEEE-half operands only): extended-precision activations as pairs of halves, value = hi + lo.
+//   a_split : A is [M, 2K], each row [hi(K) | lo(K)]; the product is A_hi B^T + A_lo B^T in one accumulator (the K loop
+//             runs twice over B), so A enters with ~22 significant bits at twice the tensor-core time;
+//   lo_p0   : the epilogue also writes the low halves of the columns below out.n0 (same layout as out.p0);
+//   lo_dup  : ... and the low halves of segment 0's half copy (a layer's K plane), row stride out.seg_w.
+struct GemmSplit {
+  bool a_split = false;
+  void *lo_p0 = nullptr, *lo_dup = nullptr;
+};
 int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB0, const void *B1, int nB1, const void *B2,
                    int nB2, OutDesc out, void *dup_base, long long dup_stride, const RopeSpec *rope, unsigned int *status,
-                   cudaStream_t st);
+                   cudaStream_t st, const GemmSplit *split = nullptr);
 // act[M, F] = silu(A Wg^T) * (A Wu^T), gate/up tiles paired inside one CTA tile; f16: all three in IEEE half
+// a_split: A is [M, 2K] = [hi | lo] as above; out_split: act is [M, 2F], each row [hi(F) | lo(F)] (the split A operand of
+// the down projection)
 int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg, const void *Wu, int F, void *act,
-                          unsigned int *status, cudaStream_t st);
+                          unsigned int *status, cudaStream_t st, bool a_split = false, bool out_split = false);
 bool tc_swiglu_supported(int M, int F, int K);
 // Failure-detection self-check: one CTA whose consumer role waits -- with the GEMM kernels' own bounded wait, but a
 // limit of `limit_clocks` -- on a barrier that nothing ever completes, and whose second role watches the CTA's abort
@@ -221,6 +234,12 @@ int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, v
                         const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
                         int n_tokens, int kv_rows, int max_seq_len, int n_q, int n_kv, int hd, unsigned int *status,
                         cudaStream_t st, AttnSchedule sched = AttnSchedule());
+// Plain prefill (every sequence starts at position 0, K / V rows packed like q) with extended-precision scores: q and K
+// as pairs of half tensors (value = hi + lo), S = Q K^T from three tensor-core passes; v, out in IEEE half.  out_split: out
+// is [T, 2 * n_q * hd], each row [hi | lo] (the split A operand of the O projection); else [T, n_q * hd].  One CTA per item.
+int launch_attention_tc_split(const void *q_hi, const void *q_lo, const void *k_hi, const void *k_lo, const void *v, void *out,
+                              bool out_split, const int32_t *cu_seqlens, int n_seqs, int n_tokens, int max_seq_len, int n_q, int n_kv,
+                              int hd, unsigned int *status, cudaStream_t st);
 // host side of the persistent attention kernel: items of sequences with n_new[b] new tokens after n_past[b] cached ones,
 // longest first, each to the least loaded of n_ctas CTAs; writes off[n_ctas + 1] and items[], returns the item count
 int attention_schedule(const int32_t *n_new, const int32_t *n_past, int n_seqs, int n_q, int n_ctas, int32_t *off, int32_t *items);

@@ -83,11 +83,12 @@ void launch_positions(const int32_t *cu_seqlens, int n_seqs, int32_t *positions,
 // ---------------------------------------------------------------------------------------------------------
 template <typename TG, typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
-                                                      T *__restrict__ out, int d, float eps, unsigned int *status) {
+                                                      T *__restrict__ out, int d, float eps, unsigned int *status, int split) {
   bool hit = false;
   const size_t row = blockIdx.x;
   const float *xr = x + row * d;
-  T *orow = out + row * d;
+  // split (IEEE-half output only): the row is written as [hi(d) | lo(d)], lo = what the rounding to half left over
+  T *orow = out + row * d * (split ? 2 : 1);
   __shared__ float red[8];
   float ss = 0.f;
   const bool vec = (d & 3) == 0;
@@ -116,6 +117,10 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
         note_overflow<T>(y0, hit); note_overflow<T>(y1, hit); note_overflow<T>(y2, hit); note_overflow<T>(y3, hit);
         T o4[4] = {from_f<T>(y0), from_f<T>(y1), from_f<T>(y2), from_f<T>(y3)};
         *reinterpret_cast<uint2 *>(orow + i) = *reinterpret_cast<uint2 *>(o4);
+        if (split) {
+          T l4[4] = {from_f<T>(y0 - to_f(o4[0])), from_f<T>(y1 - to_f(o4[1])), from_f<T>(y2 - to_f(o4[2])), from_f<T>(y3 - to_f(o4[3]))};
+          *reinterpret_cast<uint2 *>(orow + d + i) = *reinterpret_cast<uint2 *>(l4);
+        }
       } else {
         *reinterpret_cast<float4 *>(orow + i) = make_float4(v.x * rstd * g0, v.y * rstd * g1, v.z * rstd * g2, v.w * rstd * g3);
       }
@@ -125,13 +130,14 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *__restrict__ 
       const float y = xr[i] * rstd * (gamma ? to_f(gamma[i]) : 1.f);
       note_overflow<T>(y, hit);
       orow[i] = from_f<T>(y);
+      if (split) orow[d + i] = from_f<T>(y - to_f(orow[i]));
     }
   }
   report_overflow(hit, status);
 }
 // Rows of exactly 256 * 4 * NV floats (4096: NV = 4, 8192: NV = 8) with 16-bit output: each thread keeps its NV float4
 // in registers between the sum of squares and the scaling, so the row is read from global memory exactly once.
-template <typename TG, typename T, int NV>
+template <typename TG, typename T, int NV, bool SPLIT>
 __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restrict__ x, const TG *__restrict__ gamma,
                                                           T *__restrict__ out, float eps, unsigned int *status) {
   bool hit = false;
@@ -153,7 +159,7 @@ __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restric
 #pragma unroll
   for (int w = 0; w < 8; ++w) tot += red[w];
   const float rstd = rsqrtf(tot / (float)D + eps);
-  uint2 *orow = reinterpret_cast<uint2 *>(out + row * D);
+  uint2 *orow = reinterpret_cast<uint2 *>(out + row * D * (SPLIT ? 2 : 1));
 #pragma unroll
   for (int k = 0; k < NV; ++k) {
     const int i4 = threadIdx.x + 256 * k;
@@ -167,21 +173,31 @@ __global__ void __launch_bounds__(256) rmsnorm_reg_kernel(const float *__restric
     note_overflow<T>(y0, hit); note_overflow<T>(y1, hit); note_overflow<T>(y2, hit); note_overflow<T>(y3, hit);
     T o4[4] = {from_f<T>(y0), from_f<T>(y1), from_f<T>(y2), from_f<T>(y3)};
     orow[i4] = *reinterpret_cast<uint2 *>(o4);
+    if constexpr (SPLIT) {           // [hi(D) | lo(D)]: the low halves follow the row's high halves
+      T l4[4] = {from_f<T>(y0 - to_f(o4[0])), from_f<T>(y1 - to_f(o4[1])), from_f<T>(y2 - to_f(o4[2])), from_f<T>(y3 - to_f(o4[3]))};
+      orow[D / 4 + i4] = *reinterpret_cast<uint2 *>(l4);
+    }
   }
   report_overflow(hit, status);
 }
 template <typename TG, typename TO>
-void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st, unsigned int *status) {
+void launch_rmsnorm(const float *x, const TG *gamma, TO *out, int rows, int d, float eps, cudaStream_t st, unsigned int *status,
+                    bool split) {
   if (rows <= 0) return;
+  if constexpr (!std::is_same<TO, __half>::value) split = false;      // hi + lo pairs exist for IEEE halves only
   if constexpr (sizeof(TG) == 2 && sizeof(TO) == 2) {
-    if (d == 4096) { rmsnorm_reg_kernel<TG, TO, 4><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
-    if (d == 8192) { rmsnorm_reg_kernel<TG, TO, 8><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
+    if constexpr (std::is_same<TO, __half>::value) {
+      if (split && d == 4096) { rmsnorm_reg_kernel<TG, TO, 4, true><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
+      if (split && d == 8192) { rmsnorm_reg_kernel<TG, TO, 8, true><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
+    }
+    if (!split && d == 4096) { rmsnorm_reg_kernel<TG, TO, 4, false><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
+    if (!split && d == 8192) { rmsnorm_reg_kernel<TG, TO, 8, false><<<rows, 256, 0, st>>>(x, gamma, out, eps, status); return; }
   }
-  rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps, status);
+  rmsnorm_kernel<TG, TO><<<rows, 256, 0, st>>>(x, gamma, out, d, eps, status, split ? 1 : 0);
 }
-template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t, unsigned int *);
-template void launch_rmsnorm<bf16, bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t, unsigned int *);
-template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *, int, int, float, cudaStream_t, unsigned int *);
+template void launch_rmsnorm<float, float>(const float *, const float *, float *, int, int, float, cudaStream_t, unsigned int *, bool);
+template void launch_rmsnorm<bf16, bf16>(const float *, const bf16 *, bf16 *, int, int, float, cudaStream_t, unsigned int *, bool);
+template void launch_rmsnorm<bf16, __half>(const float *, const bf16 *, __half *, int, int, float, cudaStream_t, unsigned int *, bool);
 
 // ---------------------------------------------------------------------------------------------------------
 // Rotary embedding, rotate-half pairing (i, i + hd/2), in place.  One thread per pair.

@@ -140,6 +140,11 @@ struct GemmTcParams {
   bf16 *act;             // SwiGLU output [M, F]
   int F;
   int f16;               // A, B and the columns below out.n0 (and the SwiGLU output) hold IEEE halves (else bfloat16)
+  int kb_wrap;           // K blocks of B.  Equal to K / 64 normally; half of it when A holds [hi | lo] halves side by side
+                         // along K (K = 2 x B's K): the second half of the K loop multiplies A's lo part with B again
+  __half *lo_p0;         // split output: the low halves (value - float(high half)) of the columns below out.n0 ...
+  __half *lo_dup;        // ... and of the even-numbered segments' half copies (K planes), row stride out.seg_w
+  int lo_act;            // ... and of the SwiGLU output: its rows are then [hi(F) | lo(F)], 2F elements apart
   __half *dup_base;      // optional second copy (halves) of the columns routed to segments
   long long dup_stride;
   const int32_t *rope_pos;   // EPI_ROPE: position of every row; cos/sin tables [pos][64]
@@ -181,6 +186,12 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
   return true;
 }
 
+// low halves of a pair: what the high halves (already packed) left of a and b, as halves again
+__device__ __forceinline__ uint32_t pack_f16x2_lo(float a, float b, uint32_t hi_packed) {
+  const float2 h = __half22float2(*reinterpret_cast<const __half2 *>(&hi_packed));
+  return tc::pack_f16x2(a - h.x, b - h.y);
+}
+
 // One thread = one accumulator row (TMEM lane): apply the epilogue to the BN columns at t_row and write them out.
 // Warp-collective (tcgen05.ld): every lane of the warp must call it, also for rows beyond M.
 // amax: running maximum magnitude of the values this thread stored as IEEE halves (checked against the half range once,
@@ -206,9 +217,22 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
           amax = fmaxf(amax, fmaxf(fabsf(y0), fabsf(y1)));
           pk[i] = tc::pack_act(y0, y1, p.f16 != 0);
         }
-        uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * p.F + (size_t)n_blk * HALF + c * 32);
+        const size_t act_ld = p.lo_act ? 2 * (size_t)p.F : (size_t)p.F;
+        uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * act_ld + (size_t)n_blk * HALF + c * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+        if (p.lo_act) {      // split output: the low halves, recomputed from the same fp32 values
+          uint32_t lo[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[2 * i]), g1 = __uint_as_float(g[2 * i + 1]);
+            const float u0 = __uint_as_float(u[2 * i]), u1 = __uint_as_float(u[2 * i + 1]);
+            lo[i] = pack_f16x2_lo(g0 / (1.f + __expf(-g0)) * u0, g1 / (1.f + __expf(-g1)) * u1, pk[i]);
+          }
+          uint4 *dl = reinterpret_cast<uint4 *>(p.act + (size_t)row * act_ld + p.F + (size_t)n_blk * HALF + c * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dl[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+        }
       }
     }
   } else if constexpr (EPI == EPI_ROPE) {
@@ -221,12 +245,13 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
     for (int hh = 0; hh < BN / 128; ++hh) {
       const int col_h = n_blk * BN + hh * 128;
       bf16 *dstp;
-      __half *dupp = nullptr;
+      __half *dupp = nullptr, *lop = nullptr;      // lop: where the low halves of this head go (split output), if anywhere
       bool rope, f16 = false;
       if (col_h < p.out.n0) {
         dstp = reinterpret_cast<bf16 *>(p.out.p0) + (size_t)row * p.out.ld0 + col_h;
         rope = true;
         f16 = p.f16 != 0;
+        if (p.lo_p0) lop = p.lo_p0 + (size_t)row * p.out.ld0 + col_h;
       } else {
         const int cc = col_h - p.out.n0;
         const int seg = cc / p.out.seg_w, within = cc - seg * p.out.seg_w;
@@ -234,6 +259,7 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
         dstp = reinterpret_cast<bf16 *>(p.out.seg_base) + (size_t)seg * p.out.seg_stride + srow * p.out.seg_w + within;
         if (p.dup_base) dupp = p.dup_base + (size_t)seg * p.dup_stride + (size_t)row * p.out.seg_w + within;
         rope = (seg & 1) == 0;      // segments alternate K (rotated) and V (not)
+        if (p.lo_dup && dupp && seg == 0) lop = p.lo_dup + (size_t)row * p.out.seg_w + within;
       }
 #pragma unroll 1
       for (int c = 0; c < 2; ++c) {
@@ -271,6 +297,23 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
                                tc::pack_act(__uint_as_float(bq[8 * i + 2]), __uint_as_float(bq[8 * i + 3]), f16),
                                tc::pack_act(__uint_as_float(bq[8 * i + 4]), __uint_as_float(bq[8 * i + 5]), f16),
                                tc::pack_act(__uint_as_float(bq[8 * i + 6]), __uint_as_float(bq[8 * i + 7]), f16));
+          }
+          if (lop) {    // low halves of q (or of K's half copy): value - float(high half), from the same fp32 accumulators
+            uint4 *l0 = reinterpret_cast<uint4 *>(lop + c * 32);
+            uint4 *l1 = reinterpret_cast<uint4 *>(lop + 64 + c * 32);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t wa[4], wb[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float a0 = __uint_as_float(a[8 * i + 2 * e]), a1 = __uint_as_float(a[8 * i + 2 * e + 1]);
+                const float b0 = __uint_as_float(bq[8 * i + 2 * e]), b1 = __uint_as_float(bq[8 * i + 2 * e + 1]);
+                wa[e] = pack_f16x2_lo(a0, a1, tc::pack_f16x2(a0, a1));
+                wb[e] = pack_f16x2_lo(b0, b1, tc::pack_f16x2(b0, b1));
+              }
+              l0[i] = make_uint4(wa[0], wa[1], wa[2], wa[3]);
+              l1[i] = make_uint4(wb[0], wb[1], wb[2], wb[3]);
+            }
           }
           if (dupp) {   // the same values once more as halves, straight from the fp32 accumulators
             uint4 *e0 = reinterpret_cast<uint4 *>(dupp + c * 32);
@@ -396,11 +439,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           uint8_t *sb = sa + L::A_BYTES;
           tc::mbar_expect_tx(fb, L::STAGE_BYTES);
           tc::tma_load_2d(tc::smem_u32(sa), &tmA, fb, kb * BK, m_blk * BM);
+          const int kx = (kb >= p.kb_wrap ? kb - p.kb_wrap : kb) * BK;      // B's K coordinate (wraps for a split A)
           if constexpr (SWIGLU) {
-            tc::tma_load_2d(tc::smem_u32(sb), &tmB0, fb, kb * BK, b_row);                     // gate rows
-            tc::tma_load_2d(tc::smem_u32(sb + L::B_BYTES / 2), &tmB1, fb, kb * BK, b_row);   // up rows
+            tc::tma_load_2d(tc::smem_u32(sb), &tmB0, fb, kx, b_row);                     // gate rows
+            tc::tma_load_2d(tc::smem_u32(sb + L::B_BYTES / 2), &tmB1, fb, kx, b_row);   // up rows
           } else {
-            tc::tma_load_2d(tc::smem_u32(sb), tb, fb, kb * BK, b_row);
+            tc::tma_load_2d(tc::smem_u32(sb), tb, fb, kx, b_row);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -566,7 +610,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           uint8_t *sb = sa + L::A_BYTES;
           if (leader) tc::mbar_expect_tx(own_full, 2 * L::STAGE_BYTES);   // bytes of both CTAs' loads
           tc::tma_load_2d_pair(tc::smem_u32(sa), &tmA, leader_full, kb * BK, a_row);
-          tc::tma_load_2d_pair(tc::smem_u32(sb), tb, leader_full, kb * BK, b_row);
+          tc::tma_load_2d_pair(tc::smem_u32(sb), tb, leader_full, (kb >= p.kb_wrap ? kb - p.kb_wrap : kb) * BK, b_row);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -706,8 +750,11 @@ void tc_gemm_use_cta_pairs(bool on, bool swiglu_too) { g_use_pairs = on; g_swigl
 
 int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB0, const void *B1, int nB1, const void *B2,
                    int nB2, OutDesc out, void *dup_base, long long dup_stride, const RopeSpec *rope, unsigned int *status,
-                   cudaStream_t st) {
+                   cudaStream_t st, const GemmSplit *split) {
   const int N = nB0 + nB1 + nB2;
+  const bool a_split = split && split->a_split;
+  if (split && !f16) return SWIFTKV_ERR_UNSUPPORTED;            // hi + lo pairs exist for IEEE halves only
+  if (split && (split->lo_p0 || split->lo_dup) && !rope) return SWIFTKV_ERR_UNSUPPORTED;
   if (!tc_gemm_supported(M, N, K)) return SWIFTKV_ERR_UNSUPPORTED;
   if (out.mode == OUT_STORE_F32) return SWIFTKV_ERR_UNSUPPORTED;
   int BN = 256;
@@ -715,13 +762,18 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
   if (nB1 + nB2 > 0 && ((nB0 % BN) || (nB1 % BN))) return SWIFTKV_ERR_UNSUPPORTED;
   if (out.mode == OUT_STORE && ((out.n0 % 32) || (out.n0 < N && (out.seg_w % 32)))) return SWIFTKV_ERR_UNSUPPORTED;
   CUtensorMap ta, tb0, tb1, tb2;
-  if (get_tmap(&ta, A, M, K, K, BM, BK)) return SWIFTKV_ERR_CUDA;
+  const int KA = a_split ? 2 * K : K;      // A's row: [hi | lo] side by side along K when split
+  if (get_tmap(&ta, A, M, KA, KA, BM, BK)) return SWIFTKV_ERR_CUDA;
   if (get_tmap(&tb0, B0, nB0, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
   tb1 = tb0; tb2 = tb0;
   if (nB1 > 0 && get_tmap(&tb1, B1, nB1, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
   if (nB2 > 0 && get_tmap(&tb2, B2, nB2, K, K, BN, BK)) return SWIFTKV_ERR_CUDA;
   GemmTcParams p{};
-  p.M = M; p.N = N; p.K = K; p.nB0 = nB0; p.nB1 = nB1;
+  p.M = M; p.N = N; p.K = KA; p.nB0 = nB0; p.nB1 = nB1;
+  p.kb_wrap = K / BK;
+  p.lo_p0 = split ? reinterpret_cast<__half *>(split->lo_p0) : nullptr;
+  p.lo_dup = split ? reinterpret_cast<__half *>(split->lo_dup) : nullptr;
+  p.lo_act = 0;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = N / BN;
   p.out = out; p.act = nullptr; p.F = 0; p.status = status; p.group_m = group_m_setting();
@@ -751,14 +803,18 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
 }
 
 int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg, const void *Wu, int F, void *act,
-                          unsigned int *status, cudaStream_t st) {
+                          unsigned int *status, cudaStream_t st, bool a_split, bool out_split) {
   if (!tc_swiglu_supported(M, F, K)) return SWIFTKV_ERR_UNSUPPORTED;
+  if ((a_split || out_split) && !f16) return SWIFTKV_ERR_UNSUPPORTED;
   CUtensorMap ta, tg, tu;
-  if (get_tmap(&ta, A, M, K, K, BM, BK)) return SWIFTKV_ERR_CUDA;
+  const int KA = a_split ? 2 * K : K;
+  if (get_tmap(&ta, A, M, KA, KA, BM, BK)) return SWIFTKV_ERR_CUDA;
   if (get_tmap(&tg, Wg, F, K, K, 128, BK)) return SWIFTKV_ERR_CUDA;
   if (get_tmap(&tu, Wu, F, K, K, 128, BK)) return SWIFTKV_ERR_CUDA;
   GemmTcParams p{};
-  p.M = M; p.N = 2 * F; p.K = K; p.nB0 = F; p.nB1 = F;
+  p.M = M; p.N = 2 * F; p.K = KA; p.nB0 = F; p.nB1 = F;
+  p.kb_wrap = K / BK;
+  p.lo_p0 = nullptr; p.lo_dup = nullptr; p.lo_act = out_split ? 1 : 0;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = F / 128;
   p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status; p.group_m = group_m_setting();

@@ -214,3 +214,80 @@ def test_paged_argument_checks():
         with pytest.raises(P.SwiftKVError) as e:
             model.step(tok[:n], bad, 2, 1)
         assert e.value.code == -1
+
+
+W8B_4L = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-width-4-layers")
+
+
+@pytest.mark.parametrize("act", [1, 0])
+@pytest.mark.parametrize("paged", [False, True])
+def test_chunked_prefill_and_decode_at_8b_widths(act, paged):
+    """The deployment path at the real Llama-3.1-8B widths (hidden 4096, 32 / 8 heads, FFN 14336; 4 layers, l = 2):
+    chunks that are not multiples of the 128-row tiles and attend to a cached prefix, then three decode steps on the
+    weight-streaming decode path (kernel-mask bit 5) and, on a second model, on the general path -- contiguous regions and
+    scattered pages, both activation formats -- against the oracle's one-shot prefill of the same token sequences."""
+    import paper_2410_03960_b200 as P
+    shape, dtype, seed, l, g = W8B_4L, torch.bfloat16, 13, 2, 1
+    lens, n_decode, chunk = [333, 128, 1, 200], 3, 150          # chunks of 150: 333 = 150 + 150 + 33
+    cap_pages = 3                                                # 384 cache rows per sequence
+    w = S.make_weights(shape, seed, dtype, "cuda")
+    cfg, ow = oracle_config(shape), oracle_weights(w)
+    toks = [S.token_ids(seed, b, n + n_decode, shape.vocab) for b, n in enumerate(lens)]
+    refs = {}
+
+    def ref_of(b, m):
+        if (b, m) not in refs:
+            refs[(b, m)] = O.swiftkv(cfg, ow, toks[b][:m].numpy(), [m], l, g)
+        return refs[(b, m)]
+
+    # scattered, interleaved pages for the paged variant; contiguous regions otherwise
+    perm = [5, 0, 9, 2, 11, 7, 1, 10, 4, 8, 3, 6]
+    pages = [perm[b::4][:cap_pages] for b in range(4)]
+    where = (lambda b: pages[b]) if paged else (lambda b: b * cap_pages * 128)
+
+    def rows_of(b, m):
+        if paged:
+            return torch.as_tensor(_paged_rows(pages[b], m), device="cuda")
+        return torch.arange(b * cap_pages * 128, b * cap_pages * 128 + m, device="cuda")
+
+    for mask in (55, 23):                                        # decode steps on the weight-streaming path / the general path
+        model = P.SwiftKVModel(shape, w, dtype, 4 * cap_pages * 128, len(lens), l, g)
+        model.set_kernel_mask(mask)
+        model.set_activation_format(act)
+        done, last = [0] * len(lens), {}
+        while any(d < n for d, n in zip(done, lens)):
+            seqs, packed, emitting = [], [], []
+            for b, n in enumerate(lens):
+                if done[b] >= n:
+                    continue
+                k = min(chunk, n - done[b])
+                emit = int(done[b] + k == n)
+                seqs.append((k, done[b], where(b), emit))
+                packed.append(toks[b][done[b]:done[b] + k])
+                if emit:
+                    emitting.append(b)
+                done[b] += k
+            model.step(torch.cat(packed), seqs, l, g)
+            model.status()
+            lg = model.first_logits().clone()
+            for i, b in enumerate(emitting):
+                last[b] = lg[i]
+        for b, n in enumerate(lens):
+            assert np.max(np.abs(to_np(last[b]) - ref_of(b, n)["logits"][0])) <= 0.1, (mask, b)
+        for t in range(n_decode):
+            model.step(torch.stack([toks[b][n + t] for b, n in enumerate(lens)]),
+                       [(1, n + t, where(b), 1) for b, n in enumerate(lens)], l, g)
+            model.status()
+            lg = to_np(model.first_logits())
+            for b, n in enumerate(lens):
+                ref = ref_of(b, n + t + 1)
+                assert rel_l2(lg[b], ref["logits"][0]) <= 2e-2, (mask, t, b)
+                assert np.max(np.abs(lg[b] - ref["logits"][0])) <= 0.1, (mask, t, b)
+        for b, n in enumerate(lens):
+            m = n + n_decode
+            rows = rows_of(b, m)
+            for j in range(shape.n_layers):
+                K, V, _ = model.kv_cache_view(j)
+                assert rel_l2(to_np(K[rows]), ref_of(b, m)["K"][j]) <= 2e-2, (mask, b, j)
+                assert rel_l2(to_np(V[rows]), ref_of(b, m)["V"][j]) <= 2e-2, (mask, b, j)
+        model.close()
