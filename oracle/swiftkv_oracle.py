@@ -21,6 +21,9 @@ every token's K row and V row of a layer one fp32 scale (row maximum mapped to 4
 decided by floating point, so that decision is taken in fp32 exactly as the kernel takes it: fp32 inputs,
 correctly rounded fp32 divisions, round-to-nearest-even, saturation.  With `kv_fp8=True` the cache IS the
 quantized representation: every attention read (prefill of layers <= l included) sees code * scale.
+SimScore (Sec. 3.2, Eq. 1): `similarity`, `layer_inputs`, `simscore`; pins: hand values, torch's cosine_similarity,
+the identity-residual model (every layer input equal, SimScore = 1), invariance to per-token rescaling.
+
 Pins: the format's defining values and torch's float8_e4m3fn (decode table, encode of random values and of
 every midpoint), a pure-Python nearest-value search, the half-step error bound, scale equivariance, and the
 paper's combined cache reductions (62.5 % and 68.75 %).
@@ -367,6 +370,30 @@ def hidden_after(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence
             Xn[a:e], _, _ = decoder_layer(cfg, w, X[a:e], pos[a:e])
         X = Xn
     return X
+
+
+# ---------------------------------------------------------------------------------------------------
+# SimScore (Sec. 3.2, Eq. 1): how similar a layer's input is to the inputs of all later layers
+# ---------------------------------------------------------------------------------------------------
+def similarity(Xa: np.ndarray, Xb: np.ndarray) -> float:
+    """Average over tokens i of the cosine similarity between Xa[i] and Xb[i]  (Xa, Xb: [n_tokens, hidden])."""
+    dots = np.sum(Xa * Xb, axis=-1)
+    return float(np.mean(dots / (np.linalg.norm(Xa, axis=-1) * np.linalg.norm(Xb, axis=-1))))
+
+
+def layer_inputs(cfg: Config, W: Weights, tokens: np.ndarray, seq_lens: Sequence[int]) -> List[np.ndarray]:
+    """x_1 .. x_L of the unmodified model: element l-1 is the input of (1-based) layer l, all tokens."""
+    return [hidden_after(cfg, W, tokens, seq_lens, n) for n in range(cfg.n_layers)]
+
+
+def simscore(xs: Sequence[np.ndarray]) -> np.ndarray:
+    """Eq. 1 for every layer that has a later one.  xs[l-1] = x_l (input of layer l), l = 1..L.
+    Returns s with s[l-1] = SimScore(x_l) = sum_{j=l+1..L} Similarity(x_l, x_j) / (L - l), l = 1..L-1."""
+    L = len(xs)
+    out = np.empty(L - 1, dtype=F64)
+    for l in range(1, L):
+        out[l - 1] = sum(similarity(xs[l - 1], xs[j - 1]) for j in range(l + 1, L + 1)) / (L - l)
+    return out
 
 
 # ---------------------------------------------------------------------------------------------------

@@ -415,6 +415,52 @@ def test_causality_and_batch_independence(small):
             assert np.allclose(tr["V"][j], full["V"][j][:6], rtol=1e-12, atol=1e-14)
 
 
+# ------------------------------------------------------------------ SimScore (Eq. 1) --------------
+def test_simscore_definition():
+    """Eq. 1: SimScore(x_l) = average over the later layers j of Similarity(x_l, x_j), Similarity = average over tokens
+    of the cosine.  Hand values, a library routine, and the facts a cosine obeys."""
+    e1, e2 = np.array([1.0, 0.0, 0.0]), np.array([0.0, 1.0, 0.0])
+    d45 = np.array([1.0, 1.0, 0.0])
+    # two tokens; x_1 = (e1, e1); x_2 = (e1, e2) -> cosines 1 and 0; x_3 = (d45, -e1) -> cosines 1/sqrt2 and -1
+    x1, x2, x3 = np.stack([e1, e1]), np.stack([e1, e2]), np.stack([d45, -e1])
+    assert O.similarity(x1, x2) == pytest.approx(0.5)
+    assert O.similarity(x1, x3) == pytest.approx((1 / math.sqrt(2) - 1) / 2)
+    s = O.simscore([x1, x2, x3])
+    assert s.shape == (2,)
+    assert s[0] == pytest.approx((0.5 + (1 / math.sqrt(2) - 1) / 2) / 2)       # layers 2 and 3 follow layer 1
+    assert s[1] == pytest.approx((1 / math.sqrt(2) + 0.0) / 2)                 # only layer 3 follows layer 2: cos 1/sqrt2, 0
+    rng = np.random.default_rng(4)
+    xs = [rng.standard_normal((9, 16)) for _ in range(5)]
+    got = O.simscore(xs)
+    for l in range(1, 5):
+        want = np.mean([torch.nn.functional.cosine_similarity(torch.from_numpy(xs[l - 1]), torch.from_numpy(xs[j - 1]), dim=-1).mean().item()
+                        for j in range(l + 1, 6)])
+        assert got[l - 1] == pytest.approx(want, rel=1e-12)
+    # a cosine ignores positive per-token scales and is 1 between equal inputs
+    scaled = [x * np.exp(rng.uniform(-3, 3, (9, 1))) for x in xs]
+    assert np.allclose(O.simscore(scaled), got, rtol=1e-12)
+    assert np.allclose(O.simscore([xs[0]] * 4), 1.0)
+    assert np.allclose(O.simscore([xs[0], -xs[0]]), -1.0)
+
+
+def test_simscore_of_the_identity_residual_model_is_one():
+    """W_O = W_down = 0: every layer is the identity on the residual stream, all layer inputs are equal (the paper's
+    premise "inputs of deeper layers are similar" made exact), so SimScore(x_l) = 1 for every l; with the ordinary
+    random weights it lies strictly between 0 and 1 and the layer inputs are what `decoder_layer` chains."""
+    cfg = _cfg(SMALL)
+    tok = S.make_prompts(9, LENS, SMALL.vocab).numpy()
+    xs = O.layer_inputs(cfg, _weights(SMALL, seed=9, zero_out=True), tok, LENS)
+    assert len(xs) == cfg.n_layers and np.allclose(O.simscore(xs), 1.0, rtol=0, atol=1e-12)
+    W = _weights(SMALL, seed=9)
+    xs = O.layer_inputs(cfg, W, tok, LENS)
+    assert np.array_equal(xs[0], W.embed_rows(tok))                             # x_1 is the embedding
+    pos = np.concatenate([np.arange(n) for n in LENS])
+    a, e = 0, LENS[0]
+    assert np.allclose(O.decoder_layer(cfg, W.layer(2), xs[2][a:e], pos[a:e])[0], xs[3][a:e], rtol=1e-12, atol=1e-14)
+    s = O.simscore(xs)
+    assert ((s > 0) & (s < 1)).all()
+
+
 # ------------------------------------------------------------------ closed forms the paper prints --
 def _rows(name):
     with open(os.path.join(GOLD, name)) as f:
