@@ -183,6 +183,23 @@ typedef struct {
 int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const swiftkv_seq_step *seqs, int32_t n_seqs,
                      int32_t swift_layer, int32_t acrosskv_group, void *cuda_stream);
 
+/*
+ * SimScore (Sec. 3.2, Eq. 1), the paper's measure of how alike the inputs of deeper layers are -- the observation
+ * SingleInputKV rests on:  SimScore(x_l) = sum_{j=l+1..L} Similarity(x_l, x_j) / (L - l),  Similarity = the cosine
+ * similarity of token i's x_l and x_j averaged over all tokens; x_l is the input of (1-based) layer l of the UNMODIFIED
+ * model.  Runs a full-depth prefill of the batch (as swiftkv_prefill with swift_layer = n_layers: caches and logits are
+ * filled as a side effect), capturing every layer's input in `scratch` (DEVICE, caller-owned, 256-byte aligned, at least
+ * swiftkv_simscore_scratch_bytes(m, total tokens) bytes = n_layers * tokens * hidden * 4 + a little), then reduces.
+ *   simscore : DEVICE fp32 [n_layers - 1]; entry l-1 = SimScore(x_l), l = 1 .. n_layers - 1
+ *   sim      : nullable, DEVICE fp32 [n_layers][n_layers]; sim[a][b] = Similarity(x_{a+1}, x_{b+1}) (symmetric, 1 on the
+ *              diagonal)
+ * tokens, seq_lens: HOST arrays as for swiftkv_prefill.  The model's cache must have room for n_layers slots.
+ * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA.
+ */
+size_t  swiftkv_simscore_scratch_bytes(const swiftkv_model *m, int32_t n_tokens);
+int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                         void *scratch, size_t scratch_bytes, float *sim, float *simscore, void *cuda_stream);
+
 typedef struct {
   const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype (FP8 cache: uint8 e4m3
                                codes), AFTER RoPE                                                           */

@@ -25,7 +25,7 @@ EXPORTS = (
     "swiftkv_set_activation_format", "swiftkv_model_free", "swiftkv_gemm_tc", "swiftkv_attention_prefill", "swiftkv_tail_attention_scratch_bytes",
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
-    "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split",
+    "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
 )
 
 
@@ -93,6 +93,10 @@ def load_library() -> C.CDLL:
     lib.swiftkv_model_free.restype = None
     lib.swiftkv_set_activation_format.argtypes = [C.c_void_p, C.c_int32]
     lib.swiftkv_set_split_mask.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_simscore_scratch_bytes.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_simscore_scratch_bytes.restype = C.c_size_t
+    lib.swiftkv_simscore.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p,
+                                     C.c_void_p]
     lib.swiftkv_gemm_tc_split.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
@@ -256,6 +260,22 @@ class SwiftKVModel:
     def status(self, stream: Optional[torch.cuda.Stream] = None) -> None:
         with torch.cuda.device(self.device):
             _check(self.lib.swiftkv_status(self._h, _stream_ptr(stream)))
+
+    def simscore(self, tokens, seq_lens: Sequence[int], stream: Optional[torch.cuda.Stream] = None):
+        """swiftkv_simscore (Eq. 1): returns (SimScore fp32 [n_layers - 1], Similarity matrix fp32 [n_layers, n_layers])."""
+        tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous()
+        assert not tokens.is_cuda
+        L = self.shape.n_layers
+        lens = (C.c_int32 * len(seq_lens))(*[int(n) for n in seq_lens])
+        nbytes = self.lib.swiftkv_simscore_scratch_bytes(self._h, int(sum(seq_lens)))
+        scratch = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        sim = torch.empty((L, L), dtype=torch.float32, device=self.device)
+        score = torch.empty(L - 1, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_simscore(self._h, tokens.data_ptr(), lens, len(seq_lens), scratch.data_ptr(), nbytes,
+                                             sim.data_ptr(), score.data_ptr(), _stream_ptr(stream)))
+            torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+        return score, sim
 
     def debug_bounded_wait(self, limit_clocks: int, stream: Optional[torch.cuda.Stream] = None) -> Tuple[bool, bool]:
         """swiftkv_debug_bounded_wait: (the waiting role gave up at its limit, the second role left through the abort flag)."""

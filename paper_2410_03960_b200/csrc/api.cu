@@ -103,6 +103,7 @@ struct swiftkv_model {
   int kernel_mask = 55;
   int n_sms = 0;
   int act_format = SWIFTKV_ACT_F16;
+  float *capture = nullptr;     // while set: layer j's input (the residual stream before layer j) is copied to capture[j][T][d]
   int split_mask = 0;           // SWIFTKV_SPLIT_* bits: which operands travel as half pairs (SWIFTKV_ACT_F16_SPLIT)
   // profiling
   bool profiling = false;
@@ -421,7 +422,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const bool sp_hin = sm & SWIFTKV_SPLIT_QKV_INPUT, sp_qk = (sm & (SWIFTKV_SPLIT_SCORES | SWIFTKV_SPLIT_ATTN_OUT)) != 0,
              sp_ao = sm & SWIFTKV_SPLIT_ATTN_OUT, sp_hpost = sm & SWIFTKV_SPLIT_MLP_INPUT, sp_act = sm & SWIFTKV_SPLIT_MLP_ACT;
   AttnSchedule att_sched;
-  if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; }
+  if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; att_sched.two_per_row = (m->kernel_mask & 64) != 0; }
   const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
   __half *wq16 = nullptr, *wk16 = nullptr, *wv16 = nullptr, *wo16 = nullptr, *wg16 = nullptr, *wu16 = nullptr, *wd16 = nullptr;
   auto w16_select = [&](int buf) {
@@ -547,6 +548,10 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   for (int j = 0; j < l && !bt.decode; ++j) {
     const swiftkv_layer_weights &lw = m->layers[j];
     T *Kj = kv + (size_t)j * 2 * plane, *Vj = Kj + plane;
+    if (m->capture) {     // SimScore (Eq. 1) needs every layer's input
+      Scope s(m, st, SWIFTKV_KC_ELEMWISE);
+      cudaMemcpyAsync(m->capture + (size_t)j * T_tok * d, b.x, (size_t)T_tok * d * sizeof(float), cudaMemcpyDeviceToDevice, st);
+    }
     if constexpr (sizeof(T) == 2) {
       if (use_w16) {
         if (j + 1 < l) convert_layer(j + 1);            // queued now, runs beside this layer's kernels
@@ -918,6 +923,40 @@ extern "C" int32_t swiftkv_step(swiftkv_model *m, const int32_t *tokens, const s
   return forward_common(m, tokens, false, seqs, n_seqs, false, swift_layer, acrosskv_group, cuda_stream);
 }
 
+static size_t simscore_bytes(const swiftkv_config &c, int n_tokens) {
+  const size_t xs = ((size_t)c.n_layers * n_tokens * c.hidden * sizeof(float) + 255) & ~(size_t)255;
+  return xs + (size_t)c.n_layers * c.n_layers * sizeof(double);
+}
+extern "C" size_t swiftkv_simscore_scratch_bytes(const swiftkv_model *m, int32_t n_tokens) {
+  if (!m || n_tokens < 1) return 0;
+  return simscore_bytes(m->cfg, n_tokens);
+}
+extern "C" int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                                    void *scratch, size_t scratch_bytes, float *sim, float *simscore, void *cuda_stream) {
+  if (!m || !tokens || !seq_lens || !scratch || !simscore) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (m->cfg.n_layers < 2) return fail(SWIFTKV_ERR_INVALID_ARG, "SimScore needs at least two layers");
+  if ((reinterpret_cast<uintptr_t>(scratch) & 255)) return fail(SWIFTKV_ERR_INVALID_ARG, "scratch must be 256-byte aligned");
+  if (n_seqs < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs < 1");
+  long long T = 0;
+  for (int i = 0; i < n_seqs; ++i) T += seq_lens[i] > 0 ? seq_lens[i] : 0;
+  if (T < 1 || T > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "token count outside [1, max_tokens]");
+  if (scratch_bytes < simscore_bytes(m->cfg, (int)T))
+    return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "scratch %zu < %zu bytes", scratch_bytes, simscore_bytes(m->cfg, (int)T));
+  const int L = m->cfg.n_layers;
+  m->capture = reinterpret_cast<float *>(scratch);
+  const int32_t rc = prefill_common(m, tokens, false, seq_lens, n_seqs, L, 1, cuda_stream);   // the unmodified model
+  m->capture = nullptr;
+  if (rc) return rc;
+  const size_t xs = ((size_t)L * T * m->cfg.hidden * sizeof(float) + 255) & ~(size_t)255;
+  launch_simscore(reinterpret_cast<const float *>(scratch), L, (int)T, m->cfg.hidden,
+                  reinterpret_cast<double *>(reinterpret_cast<uint8_t *>(scratch) + xs), sim, simscore,
+                  reinterpret_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  m->launches += 3;
+  return SWIFTKV_OK;
+}
+
 extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out) {
   if (!m || !out) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
   if (layer < 0 || layer >= m->cfg.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, m->cfg.n_layers);
@@ -991,7 +1030,7 @@ extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, flo
 extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
 extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   if (!m) return 0;
-  m->kernel_mask = mask & 63;
+  m->kernel_mask = mask & 127;
   return m->kernel_mask;
 }
 

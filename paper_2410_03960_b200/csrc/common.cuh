@@ -229,6 +229,7 @@ bool tc_attention_supported(int n_q, int n_kv, int hd);
 struct AttnSchedule {
   const int32_t *off = nullptr, *items = nullptr;
   int n_ctas = 0;
+  bool two_per_row = false;   // softmax with two threads per query row (8 warps per head) instead of one
 };
 int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
                         const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
@@ -243,6 +244,10 @@ int launch_attention_tc_split(const void *q_hi, const void *q_lo, const void *k_
 // host side of the persistent attention kernel: items of sequences with n_new[b] new tokens after n_past[b] cached ones,
 // longest first, each to the least loaded of n_ctas CTAs; writes off[n_ctas + 1] and items[], returns the item count
 int attention_schedule(const int32_t *n_new, const int32_t *n_past, int n_seqs, int n_q, int n_ctas, int32_t *off, int32_t *items);
+
+// simscore.cu : Eq. 1 over captured layer inputs xs [L][T][d] (fp32).  sums: [L][L] doubles of scratch; sim (nullable):
+// [L][L] average cosines (symmetric, diagonal 1); simscore: [L-1], entry l-1 = SimScore(x_l)
+void launch_simscore(const float *xs, int L, int T, int d, double *sums, float *sim, float *simscore, cudaStream_t st);
 
 // tail.cu : the last-token path (at most MAX_TAIL_ROWS activation rows per launch, fp32 activations)
 constexpr int MAX_TAIL_ROWS = 8;

@@ -10,8 +10,10 @@ per-token FP8 cache).  Three levels:
      tight absolute ones.  bf16 model: the oracle is run twice, with the rows quantized from bf16 (the precision the
      kernel decides in: the reference) and from fp32; the distance between these two oracle results measures how far
      a 2^-9 relative change of the quantizer's input moves this model, and the CUDA path -- whose arithmetic differs
-     from fp64 by about that much -- must stay within twice that distance of the reference, per layer and tensor,
-     for the code-flip rate and for the logits."""
+     from fp64 by about that much -- must stay within 1.25 times that distance of the reference (rel-L2 of the
+     dequantized rows; 1.5 times for the code-flip rate, twice for the scales and the logits), per layer and tensor.
+     Whatever happened upstream, every stored row must be a valid representation: row maximum on the largest code,
+     scale * 448 = that maximum, and re-quantizing the dequantized row with the oracle returns the stored codes."""
 import numpy as np
 import pytest
 import torch
@@ -89,7 +91,9 @@ def _gpu_layer(model, j, rows):
     return {"K": (Kc[rows_t].cpu().numpy(), to_np(Ks[rows_t])), "V": (Vc[rows_t].cpu().numpy(), to_np(Vs[rows_t]))}
 
 
-RATIO_CAP = 2.0      # GPU-to-reference distance over oracle-to-oracle distance (see the module docstring)
+# GPU-to-reference distance over oracle-to-oracle distance (see the module docstring).  Measured: rel-L2 ratios 0.27 .. 1.07,
+# code-flip ratios 0.15 .. 1.30 (tiny, mid and 8B-width shapes, both activation formats)
+RATIO_CAP, FLIP_CAP, LOOSE_CAP = 1.25, 1.5, 2.0
 RATIOS = []          # (layer, tensor, measured ratio) of the last checks, for the record (printed with -s)
 
 
@@ -129,9 +133,9 @@ def _check_fp8_layer(model, ref, j, rows, n, other=None):
                                                     ref, j, name, n)
             RATIOS.append((j, name, round(rel / max(o_rel, 1e-12), 3), round(flips / max(o_flips, 1e-12), 3)))
             assert rel <= RATIO_CAP * o_rel + 5e-3, (name, j, rel, o_rel)
-            assert flips <= RATIO_CAP * o_flips + 0.02, (name, j, flips, o_flips)
-            assert excess <= RATIO_CAP * o_excess + 0.01, (name, j, excess, o_excess)
-            assert ds <= RATIO_CAP * o_ds + 0.01, (name, j, ds, o_ds)
+            assert flips <= FLIP_CAP * o_flips + 0.02, (name, j, flips, o_flips)
+            assert excess <= LOOSE_CAP * o_excess + 0.01, (name, j, excess, o_excess)
+            assert ds <= LOOSE_CAP * o_ds + 0.01, (name, j, ds, o_ds)
 
 
 def _refs(cfg, ow, tok, lens, l, g, dtype):
@@ -170,7 +174,8 @@ def test_prefill_with_fp8_cache(shape, dtype, act, l, g):
             rel, flips, _, _ = _stats(*_gpu_layer(model, 0, np.arange(n))[name], ref, 0, name, n)
             assert rel <= 2e-2 and flips <= 0.06, (name, rel, flips)
     lg = to_np(model.first_logits())
-    print("fp8 prefill", shape.name, dtype, act, l, g, "GPU/oracle distance ratios (layer, tensor, rel-L2, flips):", RATIOS[-2 * shape.n_layers:],
+    print("fp8 prefill", shape.name, dtype, act, l, g, "GPU/oracle distance ratios (layer, tensor, rel-L2, flips):",
+          RATIOS[-2 * shape.n_layers:] if other is not None else "n/a (fp32: absolute bars)",
           "logits", float(np.max(np.abs(lg - ref["logits"]))), "bar", lg_bar)
     assert np.max(np.abs(lg - ref["logits"])) <= lg_bar, (float(np.max(np.abs(lg - ref["logits"]))), lg_bar)
     # memory: codes + one fp32 scale per row and plane instead of 16-bit (32-bit) elements
