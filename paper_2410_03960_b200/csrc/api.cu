@@ -422,7 +422,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   const bool sp_hin = sm & SWIFTKV_SPLIT_QKV_INPUT, sp_qk = (sm & (SWIFTKV_SPLIT_SCORES | SWIFTKV_SPLIT_ATTN_OUT)) != 0,
              sp_ao = sm & SWIFTKV_SPLIT_ATTN_OUT, sp_hpost = sm & SWIFTKV_SPLIT_MLP_INPUT, sp_act = sm & SWIFTKV_SPLIT_MLP_ACT;
   AttnSchedule att_sched;
-  if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; att_sched.two_per_row = (m->kernel_mask & 64) != 0; }
+  if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; }
   const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
   __half *wq16 = nullptr, *wk16 = nullptr, *wv16 = nullptr, *wo16 = nullptr, *wg16 = nullptr, *wu16 = nullptr, *wd16 = nullptr;
   auto w16_select = [&](int buf) {
@@ -1030,7 +1030,7 @@ extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, flo
 extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
 extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   if (!m) return 0;
-  m->kernel_mask = mask & 127;
+  m->kernel_mask = mask & 63;
   return m->kernel_mask;
 }
 

@@ -710,308 +710,6 @@ attention_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmQ, const __
 
 
 // ---------------------------------------------------------------------------------------------------------
-// The persistent kernel with the softmax of a head spread over 8 warps (two threads per query row, 18 warps per CTA):
-// producer, MMA issue order, barriers and tensor-memory layout are those of attention_tc_persistent_kernel; only the
-// S -> P step and the epilogue change (see the comment at the softmax warps).
-// ---------------------------------------------------------------------------------------------------------
-constexpr int ATT2_THREADS = 576;
-constexpr int SM_XCH = SM_BAR + 256;                 // 8 KB of row maxima / row sums exchanged between the two threads of a row
-constexpr int ATT2_SMEM = SM_BAR + 256 + 8192 + 1024;
-
-template <bool ACT_F16>
-__global__ void __maxnreg__(112)
-attention_tc_persistent2_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                               const __grid_constant__ CUtensorMap tmV, AttnParams p, const int32_t *__restrict__ sched_off,
-                               const int32_t *__restrict__ sched_items) {
-  const int i_begin = sched_off[blockIdx.x], i_end = sched_off[blockIdx.x + 1];
-  if (i_begin >= i_end) return;
-
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + SM_BAR);
-  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 3, *v_full = bars + 5, *v_empty = bars + 7, *s_full = bars + 9,
-           *p_ready = bars + 11, *p_ready2 = bars + 13, *o_full = bars + 15;
-  uint64_t *q_empty = bars + 16;      // every Q K^T of the item has retired: Q may be overwritten
-  uint64_t *o_empty = bars + 17;      // the softmax warps have read the item's O out of tensor memory (16 arrivals)
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 18);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x == 0) {
-    tc::mbar_init(tc::smem_u32(q_full), 1);
-    for (int s = 0; s < 2; ++s) {
-      tc::mbar_init(tc::smem_u32(&k_full[s]), 1);
-      tc::mbar_init(tc::smem_u32(&k_empty[s]), 1);
-      tc::mbar_init(tc::smem_u32(&v_full[s]), 1);
-      tc::mbar_init(tc::smem_u32(&v_empty[s]), 1);
-      tc::mbar_init(tc::smem_u32(&s_full[s]), 1);
-      tc::mbar_init(tc::smem_u32(&p_ready[s]), 4);
-      tc::mbar_init(tc::smem_u32(&p_ready2[s]), 4);
-    }
-    tc::mbar_init(tc::smem_u32(o_full), 1);
-    tc::mbar_init(tc::smem_u32(q_empty), 1);
-    tc::mbar_init(tc::smem_u32(o_empty), 16);
-    *abort_flag = 0;
-    tc::fence_barrier_init();
-    tc::tma_prefetch_desc(&tmQ);
-    tc::tma_prefetch_desc(&tmK);
-    tc::tma_prefetch_desc(&tmV);
-  }
-  if (warp == 1) tc::tmem_alloc(tc::smem_u32(tmem_slot), 512);
-  tc::tc_fence_before_sync();
-  __syncthreads();
-  tc::tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_slot;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      // ------------------------------------------------------------ TMA producer
-      int gk = 0;
-      bool ok = true;
-      AttnItem im, nx;
-      decode_item(p, sched_items[i_begin], nx);
-      for (int i = i_begin; i < i_end && ok; ++i) {
-        const int it = i - i_begin;
-        im = nx;
-        if (i + 1 < i_end) decode_item(p, sched_items[i + 1], nx);     // the next item's description: loads in flight meanwhile
-        if (!wait_or_abort(tc::smem_u32(q_empty), (it & 1) ^ 1, abort_flag, p.status)) break;
-        const uint32_t qb = tc::smem_u32(q_full);
-        tc::mbar_expect_tx(qb, 2 * TILE_BYTES);
-        for (int w = 0; w < 2; ++w)
-          for (int c = 0; c < 2; ++c)
-            tc::tma_load_2d(tc::smem_u32(smem + SM_Q + w * TILE_BYTES + c * CHUNK_BYTES), &tmQ, qb, (im.h0 + w) * HD + c * 64, im.q_row0);
-        for (int j = 0; j < im.n_kv_tiles; ++j, ++gk) {
-          const int s = gk & 1;
-          const uint32_t ph = (gk >> 1) & 1;
-          const int krow = p.blk ? p.blk[(size_t)im.b * p.blk_stride + j] * BKV : im.k0 + j * BKV;
-          if (!wait_or_abort(tc::smem_u32(&k_empty[s]), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t kb = tc::smem_u32(&k_full[s]);
-          tc::mbar_expect_tx(kb, TILE_BYTES);
-          for (int c = 0; c < 2; ++c)
-            tc::tma_load_2d(tc::smem_u32(smem + SM_K + s * TILE_BYTES + c * CHUNK_BYTES), &tmK, kb, im.kvh * HD + c * 64, krow);
-          if (!wait_or_abort(tc::smem_u32(&v_empty[s]), ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t vb = tc::smem_u32(&v_full[s]);
-          tc::mbar_expect_tx(vb, TILE_BYTES);
-          for (int c = 0; c < 2; ++c)
-            tc::tma_load_2d(tc::smem_u32(smem + SM_V + s * TILE_BYTES + c * CHUNK_BYTES), &tmV, vb, im.kvh * HD + c * 64, krow);
-        }
-      }
-    }
-  } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer (warp-uniform, one elected lane)
-    const bool leader = tc::elect_one();
-    constexpr uint32_t idesc_qk = tc::umma_idesc(BQ, BKV, 0, 0, ACT_F16, ACT_F16);
-    constexpr uint32_t idesc_pv = tc::umma_idesc(BQ, HD, 0, 1, ACT_F16, ACT_F16);
-    const uint64_t q_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_Q), 16, 1024);
-    const uint64_t k_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_K), 16, 1024);
-    const uint64_t v_desc0 = tc::umma_desc_sw128(tc::smem_u32(smem + SM_V), CHUNK_BYTES, 1024);
-    auto issue_qk = [&](int w, int s) {
-      const uint64_t qd = q_desc0 + (uint64_t)(w * (TILE_BYTES >> 4)), kd = k_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
-      const uint32_t d = tmem_base + w * 128;
-#pragma unroll
-      for (int kk = 0; kk < HD / 16; ++kk) {
-        const uint32_t off = ((kk >> 2) * CHUNK_BYTES + (kk & 3) * 32) >> 4;
-        tc::umma_ss(d, qd + off, kd + off, idesc_qk, kk != 0);
-      }
-    };
-    auto issue_pv = [&](int w, int s, bool accumulate, int half) {
-      const uint64_t vd = v_desc0 + (uint64_t)(s * (TILE_BYTES >> 4));
-      const uint32_t d = tmem_base + 256 + w * 128, a_t = tmem_base + w * 128;
-#pragma unroll
-      for (int k4 = 0; k4 < 4; ++k4) {
-        const int kk = half * 4 + k4;
-        tc::umma_ts(d, a_t + kk * 8, vd + (uint64_t)((kk * 16 * 128) >> 4), idesc_pv, (accumulate || kk != 0) ? 1u : 0u);
-      }
-    };
-    const uint32_t b_kf = tc::smem_u32(&k_full[0]), b_ke = tc::smem_u32(&k_empty[0]), b_vf = tc::smem_u32(&v_full[0]),
-                   b_ve = tc::smem_u32(&v_empty[0]), b_sf = tc::smem_u32(&s_full[0]), b_p1 = tc::smem_u32(&p_ready[0]),
-                   b_p2 = tc::smem_u32(&p_ready2[0]), b_qe = tc::smem_u32(q_empty);
-    auto wait = [&](uint32_t bar, uint32_t parity) {
-      const bool ok = wait_or_abort(bar, parity, abort_flag, p.status);
-      tc::tc_fence_after_sync();
-      return ok;
-    };
-    int gk = 0;
-    bool ok = true;
-    AttnItem im, nx;
-    decode_item(p, sched_items[i_begin], nx);
-    for (int i = i_begin; i < i_end && ok; ++i) {
-      const int it = i - i_begin;
-      im = nx;
-      if (i + 1 < i_end) decode_item(p, sched_items[i + 1], nx);
-      const int n_kv_tiles = im.n_kv_tiles;
-      // the item's first Q K^T: S_w is free as soon as the previous item's last P_w V was issued (the tensor pipe runs in
-      // order); it runs while the softmax warps still store the previous item's output
-      ok = wait(tc::smem_u32(q_full), it & 1) && wait(b_kf + 8 * (gk & 1), (gk >> 1) & 1);
-      if (!ok) break;
-      if (leader) {
-        issue_qk(0, gk & 1);
-        tc::umma_commit(b_sf);
-        issue_qk(1, gk & 1);
-        tc::umma_commit(b_sf + 8);
-        tc::umma_commit(b_ke + 8 * (gk & 1));
-        if (n_kv_tiles == 1) tc::umma_commit(b_qe);
-      }
-      // O_w is overwritten by this item's first P V: the previous item's output must have been read out
-      if (!wait(tc::smem_u32(o_empty), (it & 1) ^ 1)) { ok = false; break; }
-      for (int j = 0; j < n_kv_tiles; ++j, ++gk) {
-        const int s = gk & 1, s1 = s ^ 1;
-        const uint32_t ph = (gk >> 1) & 1, ph1 = ph ^ s, pp = gk & 1;
-        const bool more = j + 1 < n_kv_tiles, acc = j > 0;
-        if (!wait(b_vf + 8 * s, ph) || !wait(b_p1, pp)) { ok = false; break; }
-        if (leader) issue_pv(0, s, acc, 0);
-        if (!wait(b_p2, pp)) { ok = false; break; }
-        if (leader) issue_pv(0, s, acc, 1);
-        if (more) {
-          if (!wait(b_kf + 8 * s1, ph1)) { ok = false; break; }
-          if (leader) {
-            issue_qk(0, s1);
-            tc::umma_commit(b_sf);
-          }
-        }
-        if (!wait(b_p1 + 8, pp)) { ok = false; break; }
-        if (leader) issue_pv(1, s, acc, 0);
-        if (!wait(b_p2 + 8, pp)) { ok = false; break; }
-        if (leader) {
-          issue_pv(1, s, acc, 1);
-          tc::umma_commit(b_ve + 8 * s);
-          if (more) {
-            issue_qk(1, s1);
-            tc::umma_commit(b_sf + 8);
-            tc::umma_commit(b_ke + 8 * s1);
-            if (j + 2 == n_kv_tiles) tc::umma_commit(b_qe);     // the item's last Q K^T is in the pipe
-          }
-        }
-      }
-      if (ok && leader) tc::umma_commit(tc::smem_u32(o_full));
-    }
-    __syncwarp();
-  } else {
-    // -------------------------------------------------------------- softmax warps: 8 per head, TWO threads per query row
-    // Warp group g = (warp - 2) / 4: head w = g / 2, column half hf = g % 2; the warp's TMEM lane quarter is warp % 4.
-    // Thread (row, hf) owns keys [64 hf, 64 hf + 64) of its row's scores and dims [64 hf, 64 hf + 64) of its row's output.
-    // The two threads of a row exchange their partial row maximum (and, once per item, their partial row sum) through
-    // shared memory behind a 64-thread named barrier; that barrier also orders "both have read S" before either
-    // overwrites it with P.  Halving the per-thread work halves the latency of the S -> P step, which is what the tensor
-    // pipe waits for between a head's Q K^T and its P V.
-    const int g = (warp - 2) >> 2;
-    const int w = g >> 1, hf = g & 1;
-    const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;
-    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t t_s = tmem_base + lane_base + w * 128;
-    const uint32_t t_o = tmem_base + lane_base + 256 + w * 128;
-    float *xch = reinterpret_cast<float *>(smem + SM_XCH) + w * 1024;      // [2 parities][2 halves][128 rows] max, then the same for sums
-    const int pair_bar = 1 + w * 4 + quarter;                               // named barrier of the 64 threads that share 32 rows
-    const float c = p.scale_log2;
-    int gk = 0;
-    bool ok = true;
-    int w_next = sched_items[i_begin];
-    for (int i = i_begin; i < i_end && ok; ++i) {
-      const int it = i - i_begin;
-      AttnItem im;
-      decode_item(p, w_next, im);
-      if (i + 1 < i_end) w_next = sched_items[i + 1];
-      const int n_kv_tiles = im.n_kv_tiles, past = im.past, qt = im.qt;
-      float m_ref = -INFINITY, l = 0.f;
-      for (int j = 0; j < n_kv_tiles; ++j, ++gk) {
-        if (!wait_or_abort(tc::smem_u32(&s_full[w]), gk & 1, abort_flag, p.status)) { ok = false; break; }
-        tc::tc_fence_after_sync();
-        const int shift = past + qt * BQ - j * BKV;
-        const bool diag = shift < BKV - 1;
-        const int lim = row + shift - hf * 64;            // local column e of this thread is visible iff e <= lim
-        uint32_t s[64];
-        tc::tmem_ld_32x32b_x32p(t_s + hf * 64, s);
-        tc::tmem_ld_32x32b_x32p(t_s + hf * 64 + 32, s + 32);
-        tc::tmem_ld_wait();
-        if (diag) {
-#pragma unroll
-          for (int e = 0; e < 64; ++e)
-            if (e > lim) s[e] = 0xff800000u;   // -inf
-        }
-        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-        for (int e = 0; e < 64; e += 8) {
-          m0 = tc::max3(m0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
-          m1 = tc::max3(m1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
-          m2 = tc::max3(m2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
-          m3 = tc::max3(m3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
-        }
-        const float m_loc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-        float *xm = xch + (gk & 1) * 256;
-        xm[hf * 128 + row] = m_loc;
-        asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-        const float mx = fmaxf(m_loc, xm[(hf ^ 1) * 128 + row]);
-        const bool need = (j == 0) || ((mx - m_ref) * c > RESCALE_THRESHOLD);
-        const float m_new = need ? mx : m_ref;
-        if (j > 0 && __any_sync(0xffffffffu, need)) {
-          const float f = need ? fast_exp2((m_ref - m_new) * c) : 1.f;
-          l *= f;
-#pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t r[16];
-            tc::tmem_ld_32x32b_x16(t_o + hf * 64 + ch * 16, r);
-            tc::tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * f);
-            tc::tmem_st_32x32b_x16(t_o + hf * 64 + ch * 16, r);
-          }
-        }
-        m_ref = m_new;
-        const float neg_mc = -m_ref * c;
-        float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * e]), c, neg_mc));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 1]), c, neg_mc));
-          const float p2 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 2]), c, neg_mc));
-          const float p3 = fast_exp2(fmaf(__uint_as_float(s[2 * e + 3]), c, neg_mc));
-          l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-          s[e] = ACT_F16 ? tc::pack_f16x2(p0, p1) : tc::pack_bf16x2(p0, p1);
-          s[e + 1] = ACT_F16 ? tc::pack_f16x2(p2, p3) : tc::pack_bf16x2(p2, p3);
-        }
-        tc::tmem_st_32x32b_x32(t_s + hf * 32, s);          // this half's P: 64 keys packed into 32 columns
-        tc::tmem_st_wait();
-        tc::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) tc::mbar_arrive(tc::smem_u32(hf == 1 ? &p_ready2[w] : &p_ready[w]));
-        l += (l0 + l1) + (l2 + l3);
-      }
-      if (!ok) break;
-      // ---- epilogue of the item: the row sum is the two threads' partial sums; each stores its 64 dims of O_w / l
-      float *xl = xch + 512 + (it & 1) * 256;
-      xl[hf * 128 + row] = l;
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_bar) : "memory");
-      const float inv = 1.f / (l + xl[(hf ^ 1) * 128 + row]);
-      if (!wait_or_abort(tc::smem_u32(o_full), it & 1, abort_flag, p.status)) { ok = false; break; }
-      tc::tc_fence_after_sync();
-      const bool valid = qt * BQ + row < im.n;
-      bf16 *dst = p.out + ((size_t)(im.q_row0 + row) * p.n_q + (im.h0 + w)) * HD + hf * 64;
-#pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t r[32];
-        tc::tmem_ld_32x32b_x32(t_o + hf * 64 + ch * 32, r);
-        tc::tmem_ld_wait();
-        if (ch == 1) {               // the last read of O_w is done: the next item's first P V may overwrite it
-          tc::tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) tc::mbar_arrive(tc::smem_u32(o_empty));
-        }
-        if (valid) store_out_chunk<ACT_F16>(dst + ch * 32, r, inv, p.store32 != 0);
-      }
-    }
-  }
-  tc::tc_fence_before_sync();
-  __syncthreads();
-  if (warp == 1) {
-    __syncwarp();
-    tc::tc_fence_after_sync();
-    tc::tmem_dealloc(tmem_base, 512);
-  }
-}
-
-
-// ---------------------------------------------------------------------------------------------------------
 // Extended-precision scores (activation format "half pairs"): q and K each arrive as a pair of half tensors, value =
 // hi + lo, and S = Q K^T is accumulated from three tensor-core passes  Q_hi K_hi^T + Q_lo K_hi^T + Q_hi K_lo^T  (the
 // lo-lo term is below fp32 rounding), so the scores carry ~22 significant bits of q and K instead of 11.  This is for
@@ -1364,14 +1062,6 @@ int launch_attention_tc(const void *q, bool act_f16, const void *k, const void *
     if (ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent_kernel<false>), ATT_SMEM) ||
         ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent_kernel<true>), ATT_SMEM))
       return SWIFTKV_ERR_CUDA;
-    if (sched.two_per_row) {
-      if (ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent2_kernel<false>), ATT2_SMEM) ||
-          ensure_dynamic_smem(reinterpret_cast<const void *>(attention_tc_persistent2_kernel<true>), ATT2_SMEM))
-        return SWIFTKV_ERR_CUDA;
-      if (act_f16) attention_tc_persistent2_kernel<true><<<(unsigned)sched.n_ctas, ATT2_THREADS, ATT2_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
-      else attention_tc_persistent2_kernel<false><<<(unsigned)sched.n_ctas, ATT2_THREADS, ATT2_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
-      return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
-    }
     if (act_f16) attention_tc_persistent_kernel<true><<<(unsigned)sched.n_ctas, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
     else attention_tc_persistent_kernel<false><<<(unsigned)sched.n_ctas, ATT_THREADS, ATT_SMEM, st>>>(tq, tk, tv, p, sched.off, sched.items);
     return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;

@@ -229,7 +229,6 @@ bool tc_attention_supported(int n_q, int n_kv, int hd);
 struct AttnSchedule {
   const int32_t *off = nullptr, *items = nullptr;
   int n_ctas = 0;
-  bool two_per_row = false;   // softmax with two threads per query row (8 warps per head) instead of one
 };
 int launch_attention_tc(const void *q, bool f16, const void *k, const void *v, void *out, const int32_t *cu_seqlens,
                         const int32_t *k_row0, const int32_t *kv_len, const int32_t *blk, int blk_stride, int n_seqs,
