@@ -65,10 +65,10 @@ def test_more_prompts_than_one_tail_pass():
 
 
 @pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2), (2, 2)])
-@pytest.mark.parametrize("mask,act", [(19, 1), (19, 0), (83, 1), (83, 0), (3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
+@pytest.mark.parametrize("mask,act", [(19, 1), (19, 0), (3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
 def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask, act):
     """The same model through the tcgen05 kernels (mask 3; mask 19: attention as persistent CTAs walking a host-balanced
-    work list; mask 83: the same with two softmax threads per query row), the SIMT kernels (mask 0) and the two mixtures, with
+    work list), the SIMT kernels (mask 0) and the two mixtures, with
     half (act 1) and bfloat16 (act 0) activations; several row tiles and a ragged tail (T = 507), prompts of 1 and
     129 tokens included."""
     lens = [300, 77, 129, 1]
@@ -318,7 +318,7 @@ def test_persistent_attention_gives_the_same_bits():
     w = S.make_weights(MID, 5, torch.bfloat16, "cuda")
     tok = S.make_prompts(5, lens, MID.vocab)
     out = {}
-    for mask in (55, 39, 119):
+    for mask in (55, 39):
         model = P.SwiftKVModel(MID, w, torch.bfloat16, sum(lens), len(lens), l, g)
         assert model.set_kernel_mask(mask) == mask
         model.prefill(tok, lens, l, g)
@@ -328,8 +328,3 @@ def test_persistent_attention_gives_the_same_bits():
     assert torch.equal(out[55][0], out[39][0])
     for a, b in zip(out[55][1], out[39][1]):
         assert torch.equal(a, b)
-    # kernel-mask bit 6 (two softmax threads per query row) adds each row's probabilities in another order, so the row sum
-    # differs in its last bits: equal to fp32 rounding, not bit for bit
-    assert (out[119][0] - out[55][0]).abs().max().item() <= 2e-3
-    for a, b in zip(out[119][1], out[55][1]):
-        assert (a.float() - b.float()).abs().max().item() <= 0.05 and (a != b).float().mean().item() <= 0.01
