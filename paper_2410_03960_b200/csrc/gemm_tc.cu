@@ -218,9 +218,11 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
           pk[i] = tc::pack_act(y0, y1, p.f16 != 0);
         }
         const size_t act_ld = p.lo_act ? 2 * (size_t)p.F : (size_t)p.F;
+        // (streaming stores: the [T, F] output is far larger than the L2 and is read once, by the next kernel; kept out of the
+        // way, the band of A rows that every column block re-reads stays resident)
         uint4 *dst = reinterpret_cast<uint4 *>(p.act + (size_t)row * act_ld + (size_t)n_blk * HALF + c * 32);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+        for (int i = 0; i < 4; ++i) __stcs(dst + i, make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]));
         if (p.lo_act) {      // split output: the low halves, recomputed from the same fp32 values
           uint32_t lo[16];
 #pragma unroll

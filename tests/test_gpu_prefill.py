@@ -192,6 +192,42 @@ def test_config2_full_size_prefix_parity_and_determinism():
     _check_full_size_samples(model, lens, to_np(logits1), "config2_full_sample.npz")
 
 
+@pytest.mark.parametrize("name,seed,lens,l,g", [
+    ("config3", 2, [16384] * 4, 24, 2),                 # config 3 at full size: 4 x 16384 tokens, l = 24, 2-way AcrossKV
+    ("sweep-l24-g4", 4, [16384], 24, 4),                # a sweep point with 4-way AcrossKV
+    ("sweep-l24-g2", 4, [16384], 24, 2),
+])
+def test_full_size_prefix_parity_and_determinism_with_acrosskv(name, seed, lens, l, g):
+    """Full-size runs whose complete oracle evaluation is out of reach (hours of host time): by causality the cache rows of
+    the first P tokens of every prompt equal those of the P-token prompts, which the oracle affords -- every layer, the
+    shared AcrossKV slots included; the full-length logits must be finite and bitwise reproducible; layers of one group
+    must return the same cache pointers."""
+    import paper_2410_03960_b200 as P
+    shape, prefix = S.LLAMA31_8B, 24
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    logits1 = model.first_logits().clone()
+    assert torch.isfinite(logits1).all()
+    short = [prefix] * len(lens)
+    ref = O.swiftkv(oracle_config(shape), oracle_weights(w), S.make_prompts(seed, short, shape.vocab).numpy(), short, l, g)
+    offs = np.concatenate([[0], np.cumsum(lens)])[:-1]
+    idx = torch.as_tensor(np.concatenate([np.arange(o, o + prefix) for o in offs]), device="cuda")
+    for j in range(shape.n_layers):
+        K, V, owner = model.kv_cache_view(j)
+        assert rel_l2(to_np(K[idx]), ref["K"][j]) <= 2e-2, (name, j)
+        assert rel_l2(to_np(V[idx]), ref["V"][j]) <= 2e-2, (name, j)
+        if j >= l:
+            leader = l + ((j - l) // g) * g
+            assert owner == leader and K.data_ptr() == model.kv_cache_view(leader)[0].data_ptr()
+    model.prefill(tok, lens, l, g)
+    model.status()
+    assert torch.equal(logits1, model.first_logits())
+    model.close()
+
+
 def _check_full_size_samples(model, lens, logits, file):
     """Sampled outputs of the oracle's FULL-size run of the same workload (tests/golden/*_full_sample.npz, written by
     tests/golden/make_config2_full_sample.py from the oracle alone): first-token logits at 2048 vocabulary entries per
@@ -305,6 +341,27 @@ def test_config4_llama70b_full_depth_truncated_prompts():
     model.prefill(tok, lens, l, g)
     model.status()
     print("config4 truncated parity (plain halves):", _check_config4_samples(model, lens, "config4_truncated_sample.npz"))
+    model.close()
+
+
+def test_config4_full_size_against_oracle_samples():
+    """Config 4 at FULL size -- the 80-layer 70B shape, the complete seed-3 batch of 7 prompts totalling 16384 tokens,
+    l = 40 -- in the half-pair format, against stored outputs of the oracle's run of the same batch: all first-token
+    logits of every prompt, and K / V rows of ten layers at the first, the last and an inner position of every prompt."""
+    import paper_2410_03960_b200 as P
+    if not os.path.exists(os.path.join(os.path.dirname(__file__), "golden", "config4_full_sample.npz")):
+        pytest.skip("tests/golden/config4_full_sample.npz has not been generated (tests/golden/make_config4_sample.py --full)")
+    lens = S.lengths_to_total(3, 16384, 1024, 4096)
+    shape, seed, l, g = S.LLAMA31_70B, 3, 40, 1
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
+    model.set_activation_format(P.ACT_F16_SPLIT)
+    model.prefill(tok, lens, l, g)
+    model.status()
+    res = _check_config4_samples(model, lens, "config4_full_sample.npz")
+    print("config4 full-size parity (half pairs):", lens, res)
+    assert res["logit_rel"] <= 2e-2 and res["logit_abs"] <= 0.1, res
     model.close()
 
 

@@ -219,8 +219,7 @@ def test_paged_argument_checks():
 W8B_4L = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-width-4-layers")
 
 
-@pytest.mark.parametrize("act", [1, 0])
-@pytest.mark.parametrize("paged", [False, True])
+@pytest.mark.parametrize("act,paged", [(1, False), (1, True), (0, False)])
 def test_chunked_prefill_and_decode_at_8b_widths(act, paged):
     """The deployment path at the real Llama-3.1-8B widths (hidden 4096, 32 / 8 heads, FFN 14336; 4 layers, l = 2):
     chunks that are not multiples of the 128-row tiles and attend to a cached prefix, then three decode steps on the
