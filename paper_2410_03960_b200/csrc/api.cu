@@ -721,21 +721,12 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
     float *y = b.y + (size_t)r0 * d;
     if (!bt.decode) { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
-    // each weight-streaming launch asks the L2 for the head of the next launch's matrix (at most PF_CAP bytes in all)
-    static const long pf_mb = [] { const char *e = getenv("SWIFTKV_TAIL_PREFETCH_MB"); return e ? atol(e) : 40L; }();
-    const size_t PF_CAP = (size_t)(pf_mb < 0 ? 0 : pf_mb) << 20, E = sizeof(T);
-    auto head = [&](const void *p, size_t bytes) { return std::min(bytes, PF_CAP); };
     for (int j = l; j < L; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
       const int slot = l + (j - l) / g;
       const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
-      const Prefetch pf_o{lw.wo, head(lw.wo, (size_t)d * dq * E), nullptr, 0};
-      const Prefetch pf_gu{lw.w_gate, head(lw.w_gate, (size_t)F * d * E) / 2, lw.w_up, head(lw.w_up, (size_t)F * d * E) / 2};
-      const Prefetch pf_d{lw.w_down, head(lw.w_down, (size_t)d * F * E), nullptr, 0};
-      const void *nq = j + 1 < L ? m->layers[j + 1].wq : m->lm_head;
-      const Prefetch pf_n{nq, head(nq, j + 1 < L ? (size_t)dq * d * E : (size_t)c.vocab * d * E), nullptr, 0};
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st, pf_o); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
       {
         Scope s(m, st, SWIFTKV_KC_TAIL, 2);
         const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
@@ -750,10 +741,10 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
           launch_tail_attention<T>(qy, Ks, Vs, nullptr, nullptr, ay, b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len,
                                    c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
       }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st, pf_gu); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st, pf_d); }
-      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, nullptr, rows, d, F, y, d, OUT_RESID_ADD_F32, st, pf_n); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
+      { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, nullptr, rows, d, F, y, d, OUT_RESID_ADD_F32, st); }
     }
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)m->final_norm, hy, rows, d, c.rms_eps, st); }
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)m->lm_head, nullptr, rows, c.vocab, d,

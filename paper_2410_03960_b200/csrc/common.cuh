@@ -254,17 +254,9 @@ template <typename T>
 void launch_tail_rmsnorm(const float *y, const T *gamma, float *out, int rows, int d, float eps, cudaStream_t st);
 // out[r, n] = sum_k act[r, k] * W[n, k]  (mode OUT_STORE_F32 or OUT_RESID_ADD_F32);
 // with W2: out[r, n] = silu(act W^T) * (act W2^T)
-// pf (optional): memory the NEXT launch will stream (the heads of its one or two weight matrices); this launch asks the L2
-// to fetch it, spread over its CTAs, so that HBM keeps streaming between the two dependent kernels
-struct Prefetch {
-  const void *a = nullptr;
-  size_t a_bytes = 0;
-  const void *b = nullptr;
-  size_t b_bytes = 0;
-};
 template <typename T>
 void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
-                        int mode, cudaStream_t st, Prefetch pf = Prefetch());
+                        int mode, cudaStream_t st);
 // two projections of the same rows in one launch: out[r, n] = act W^T, out2[r, n] = act W2^T (a decode step's K and V)
 template <typename T>
 void launch_skinny_gemm_dual(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, float *out2,

@@ -3,8 +3,6 @@
 // weights from HBM exactly once; attention is one query per (prompt, head) over the cache that the
 // SingleInputKV projection filled.  Activations of this path stay in fp32 (they are tiny), weights and the
 // cache stay in the model dtype.
-#include <cstdlib>
-
 #include <cooperative_groups.h>
 #include <mma.h>
 
@@ -130,36 +128,12 @@ __device__ __forceinline__ void split_hi_lo(float x0, float x1, uint32_t &hi, ui
 constexpr int SK_WARPS = 8;
 constexpr int SK_MAX_CLUSTER = 8;
 
-// Ask the L2 to fetch [p, p + bytes) from HBM (16-byte granularity; nothing waits for it).  The weight-streaming kernels
-// use it twice: a CTA requests its own tile's rows at once when it starts -- so its K loop reads from L2 instead of
-// paying one HBM round trip per batch of loads -- and every launch requests the head of the NEXT launch's weights, so
-// that HBM keeps streaming across the gap between two dependent kernels.
-__device__ __forceinline__ void l2_prefetch(const void *p, unsigned bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-}
-constexpr unsigned PF_CHUNK = 4096;
-// this CTA's share (CTA `part` of `parts`) of a region, issued by the threads from `first_thread` on
-__device__ __forceinline__ void l2_prefetch_share(const uint8_t *base, unsigned long long bytes, unsigned part, unsigned parts,
-                                                  int first_thread) {
-  if (!base || bytes == 0 || (int)threadIdx.x < first_thread) return;
-  const unsigned long long per = ((bytes + parts - 1) / parts + PF_CHUNK - 1) / PF_CHUNK * PF_CHUNK;
-  const unsigned long long lo = per * part, hi = lo + per < bytes ? lo + per : bytes;
-  for (unsigned long long off = lo + (unsigned long long)(threadIdx.x - first_thread) * PF_CHUNK; off < hi;
-       off += (unsigned long long)(blockDim.x - first_thread) * PF_CHUNK) {
-    const unsigned long long left = hi - off;
-    const unsigned n = (unsigned)(left < PF_CHUNK ? left : PF_CHUNK) & ~15u;
-    if (n) l2_prefetch(base + off, n);
-  }
-}
-
 // EPI: 0 = one weight matrix; 1 = two, combined as silu(act W^T) * (act W2^T); 2 = two, stored to out and out2
 template <int EPI>
 __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *__restrict__ act, const bf16 *__restrict__ W,
                                                                    const bf16 *__restrict__ W2, int n_rows, int N, int K,
                                                                    float *__restrict__ out, float *__restrict__ out2, int ldo,
-                                                                   int mode, int ks, const uint8_t *__restrict__ pf,
-                                                                   unsigned long long pf_bytes, const uint8_t *__restrict__ pf2,
-                                                                   unsigned long long pf2_bytes, int own_pf) {
+                                                                   int mode, int ks) {
   namespace cg = cooperative_groups;
   constexpr bool SWIGLU = EPI != 0;      // (two accumulators: the name is kept from the first user)
   __shared__ float red[SK_WARPS][SWIGLU ? 2 : 1][32][4];
@@ -178,14 +152,6 @@ __global__ void __launch_bounds__(SK_WARPS * 32) skinny_mma_kernel(const float *
   // this CTA's share of the K steps
   const int all_steps = K / 32;
   const int step_lo = (int)((long long)all_steps * rank / ks), steps = (int)((long long)all_steps * (rank + 1) / ks);
-  // the whole share of this CTA -- 16 rows (32 with a second matrix) x its K range -- is requested from HBM right away
-  if (own_pf && threadIdx.x < (SWIGLU ? 32 : 16)) {
-    const bf16 *rowp = (threadIdx.x < 16 ? W : W2) + (size_t)(n0 + (threadIdx.x & 15)) * K + (size_t)step_lo * 32;
-    const unsigned row_bytes = (unsigned)(steps - step_lo) * 64u;
-    for (unsigned off = 0; off < row_bytes; off += 8192u) l2_prefetch(reinterpret_cast<const uint8_t *>(rowp) + off, min(8192u, row_bytes - off));
-  }
-  l2_prefetch_share(pf, pf_bytes, blockIdx.x, gridDim.x, 32);        // the head of the next launch's weights
-  l2_prefetch_share(pf2, pf2_bytes, blockIdx.x, gridDim.x, 32);
   // software pipeline: the loads of U K-steps are issued together before any of their MMAs, so that each lane keeps
   // 2U (4U with SwiGLU) 16-byte weight loads in flight
   constexpr int U = SWIGLU ? 2 : 4;
@@ -292,13 +258,9 @@ static int skinny_cluster(int tiles, int steps) {
   while (ks < SK_MAX_CLUSTER && tiles * ks < 1024 && steps / (2 * ks) >= 2 * SK_WARPS) ks *= 2;
   return ks;
 }
-static int own_tile_prefetch() {
-  static const int v = [] { const char *e = getenv("SWIFTKV_TAIL_OWN_PREFETCH"); return e ? atoi(e) : 1; }();
-  return v;
-}
 template <int EPI>
 static void launch_skinny_mma(const float *act, const bf16 *w, const bf16 *w2, int n_rows, int N, int K, float *out, float *out2,
-                              int ldo, int mode, cudaStream_t st, Prefetch pf = Prefetch()) {
+                              int ldo, int mode, cudaStream_t st) {
   const int tiles = N / 16, ks = skinny_cluster(tiles, K / 32);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(tiles * ks));
@@ -312,20 +274,18 @@ static void launch_skinny_mma(const float *act, const bf16 *w, const bf16 *w2, i
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, skinny_mma_kernel<EPI>, act, w, w2, n_rows, N, K, out, out2, ldo, mode, ks,
-                     reinterpret_cast<const uint8_t *>(pf.a), (unsigned long long)pf.a_bytes,
-                     reinterpret_cast<const uint8_t *>(pf.b), (unsigned long long)pf.b_bytes, own_tile_prefetch());
+  cudaLaunchKernelEx(&cfg, skinny_mma_kernel<EPI>, act, w, w2, n_rows, N, K, out, out2, ldo, mode, ks);
 }
 
 template <typename T>
 void launch_skinny_gemm(const float *act, const T *W, const T *W2, int n_rows, int N, int K, float *out, int ldo,
-                        int mode, cudaStream_t st, Prefetch pf) {
+                        int mode, cudaStream_t st) {
   if (n_rows <= 0 || N <= 0) return;
   if constexpr (sizeof(T) == 2) {
     if ((K % 32) == 0 && (N % 16) == 0) {
       const bf16 *w = reinterpret_cast<const bf16 *>(W), *w2 = reinterpret_cast<const bf16 *>(W2);
-      if (W2) launch_skinny_mma<1>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st, pf);
-      else launch_skinny_mma<0>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st, pf);
+      if (W2) launch_skinny_mma<1>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st);
+      else launch_skinny_mma<0>(act, w, w2, n_rows, N, K, out, nullptr, ldo, mode, st);
       return;
     }
   }
@@ -349,10 +309,8 @@ void launch_skinny_gemm_dual(const float *act, const T *W, const T *W2, int n_ro
 }
 template void launch_skinny_gemm_dual<float>(const float *, const float *, const float *, int, int, int, float *, float *, int, cudaStream_t);
 template void launch_skinny_gemm_dual<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, float *, int, cudaStream_t);
-template void launch_skinny_gemm<float>(const float *, const float *, const float *, int, int, int, float *, int, int, cudaStream_t,
-                                        Prefetch);
-template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, int, int, cudaStream_t,
-                                       Prefetch);
+template void launch_skinny_gemm<float>(const float *, const float *, const float *, int, int, int, float *, int, int, cudaStream_t);
+template void launch_skinny_gemm<bf16>(const float *, const bf16 *, const bf16 *, int, int, int, float *, int, int, cudaStream_t);
 
 // ---------------------------------------------------------------------------------------------------------
 // single-query attention over the cache, split along the keys.
