@@ -259,8 +259,12 @@ int32_t swiftkv_last_launch_count(const swiftkv_model *m);
  * bit 4 = the tensor-core attention runs as one persistent CTA per SM over a work list that the host balances from the
  * sequence lengths (longest item first, each to the least loaded CTA) instead of one CTA per work item,
  * bit 5 = decode minibatches (at most 8 sequences, one new token each) run every layer on the weight-streaming
- * kernels of the last-token path instead of 128-row GEMM tiles.
- * Default 55: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
+ * kernels of the last-token path instead of 128-row GEMM tiles,
+ * bit 6 = the projections of the last-token path between two attention calls (O, gate/up + SwiGLU, down, the next
+ * layer's Q or the lm_head, norms folded in) run as ONE persistent cooperative launch (weight rows streamed through a
+ * shared-memory ring, grid-wide barriers between the stages) instead of one launch per operator; bf16 models whose
+ * hidden, query and FFN widths are multiples of 512.
+ * Default 55: everything that the model's shape and dtype support except bits 3 and 6.  Returns the mask in effect. */
 int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
 /* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention

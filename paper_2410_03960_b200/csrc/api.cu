@@ -716,31 +716,64 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
 
   // ---- the tokens that must produce output -- the last token of a prompt (footnote of Sec. 3.2), decode tokens
   //      (Sec. 3.5) -- continue through layers l+1..L
+  // kernel-mask bit 6: the dependent projections between two attention calls -- O, gate/up, down and the next layer's Q, or
+  // the lm_head at the end -- run as ONE persistent cooperative launch with the norms folded in
+  bool fused_tail = false;
+  if constexpr (sizeof(T) == 2) {
+    fused_tail = (m->kernel_mask & 64) && bt.n_emit > 0 && tail_fused_supported(std::min(MAX_TAIL_ROWS, bt.n_emit), d, dq, F, c.vocab);
+  }
+  unsigned int fused_arrivals = 0;
+  if (fused_tail && cudaMemsetAsync(b.status + 32, 0, 32 * sizeof(unsigned int), st) != cudaSuccess)
+    return fail(SWIFTKV_ERR_CUDA, "clearing the grid-barrier words failed");
   for (int r0 = 0; r0 < bt.n_emit; r0 += MAX_TAIL_ROWS) {
     const int rows = std::min(MAX_TAIL_ROWS, bt.n_emit - r0);
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
     float *y = b.y + (size_t)r0 * d;
     if (!bt.decode) { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx + r0, y, rows, d, st); }
+    const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
+    int emit_kv = 0;
+    for (int r = r0; r < r0 + rows; ++r) emit_kv += bt.emit_lens[r];
+    const TailOpts q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab, emit_kv};    // the queries are rotated inside the attention kernel
+    auto attention = [&](int slot) {
+      Scope s(m, st, SWIFTKV_KC_TAIL, 2);
+      if (fp8)
+        launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(slot), (const fp8e4 *)v_codes(slot), k_scale(slot), v_scale(slot), ay,
+                                     b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads,
+                                     c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
+      else
+        launch_tail_attention<T>(qy, kv + (size_t)slot * 2 * plane, kv + (size_t)slot * 2 * plane + plane, nullptr, nullptr, ay,
+                                 b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads,
+                                 c.head_dim, b.tail_scratch, st, q_rope);
+    };
+    if (fused_tail) {
+      TailStage list[6];
+      int n_list = 0;
+      auto flush = [&]() -> int32_t {
+        if (n_list == 0) return SWIFTKV_OK;
+        Scope s(m, st, SWIFTKV_KC_TAIL);
+        const int frc = launch_tail_fused(list, n_list, rows, c.rms_eps, b.status + 32, &fused_arrivals, b.status, st);
+        n_list = 0;
+        return frc == SWIFTKV_OK ? SWIFTKV_OK : fail(frc, "fused last-token launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+      };
+      for (int j = l; j < L; ++j) {
+        const swiftkv_layer_weights &lw = m->layers[j];
+        list[n_list++] = TailStage{y, lw.in_norm, lw.wq, nullptr, qy, dq, d, dq, 0};
+        if ((rc = flush())) return rc;
+        attention(l + (j - l) / g);
+        list[n_list++] = TailStage{ay, nullptr, lw.wo, nullptr, y, d, dq, d, 1};
+        list[n_list++] = TailStage{y, lw.post_norm, lw.w_gate, lw.w_up, acty, F, d, F, 2};
+        list[n_list++] = TailStage{acty, nullptr, lw.w_down, nullptr, y, d, F, d, 1};
+        if (j + 1 == L) list[n_list++] = TailStage{y, m->final_norm, m->lm_head, nullptr, b.logits + (size_t)r0 * c.vocab, c.vocab, d, c.vocab, 0};
+      }
+      if (l == L) list[n_list++] = TailStage{y, m->final_norm, m->lm_head, nullptr, b.logits + (size_t)r0 * c.vocab, c.vocab, d, c.vocab, 0};
+      if ((rc = flush())) return rc;
+      continue;
+    }
     for (int j = l; j < L; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
-      const int slot = l + (j - l) / g;
-      const T *Ks = kv + (size_t)slot * 2 * plane, *Vs = Ks + plane;
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
-      {
-        Scope s(m, st, SWIFTKV_KC_TAIL, 2);
-        const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
-        int emit_kv = 0;
-        for (int r = r0; r < r0 + rows; ++r) emit_kv += bt.emit_lens[r];
-        const TailOpts q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab, emit_kv};    // the queries are rotated inside the attention kernel
-        if (fp8)
-          launch_tail_attention<fp8e4>(qy, (const fp8e4 *)k_codes(slot), (const fp8e4 *)v_codes(slot), k_scale(slot), v_scale(slot), ay,
-                                       b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len, c.n_q_heads,
-                                       c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
-        else
-          launch_tail_attention<T>(qy, Ks, Vs, nullptr, nullptr, ay, b.emit_row0 + r0, b.emit_len + r0, be, bt.blk_stride, rows, max_len,
-                                   c.n_q_heads, c.n_kv_heads, c.head_dim, b.tail_scratch, st, q_rope);
-      }
+      attention(l + (j - l) / g);
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
@@ -1031,7 +1064,7 @@ extern "C" int32_t swiftkv_profile_read(swiftkv_model *m, void *cuda_stream, flo
 extern "C" int32_t swiftkv_last_launch_count(const swiftkv_model *m) { return m ? m->launches : 0; }
 extern "C" int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask) {
   if (!m) return 0;
-  m->kernel_mask = mask & 63;
+  m->kernel_mask = mask & 127;
   return m->kernel_mask;
 }
 

@@ -281,4 +281,20 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
                            const int32_t *row0, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
                            int max_seq_len, int n_q, int n_kv, int hd, float *scratch, cudaStream_t st, TailOpts rope = TailOpts());
 
+// Several dependent projections of the last-token path (at most 6) as one persistent cooperative launch with grid-wide
+// barriers between them (bf16 weights).  Stage: out (+)= A W^T with A [rows, K] fp32, W [N, K]; epi 0 store, 1 accumulate
+// into out, 2 out = silu(A W^T) * (A W2^T); gamma != null: A is RMS-normalised on the fly (the norm that precedes the
+// projection is folded in).  sync: two words of device scratch; status: the model's status word.
+struct TailStage {
+  const float *A;
+  const void *gamma, *W, *W2;
+  float *out;
+  int N, K, ldo, epi;
+};
+bool tail_fused_supported(int rows, int d, int dq, int F, int vocab);
+// arrivals: the host's count of barrier arrivals on sync[0] so far (the counter is never reset between launches; zero both
+// together).
+int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
+                      unsigned int *status, cudaStream_t st);
+
 }  // namespace skv

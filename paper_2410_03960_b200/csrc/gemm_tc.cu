@@ -53,12 +53,12 @@ int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_
   return r == CUDA_SUCCESS ? 0 : -2;
 }
 int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1,
-                      uint64_t s2, uint32_t b0, uint32_t b1) {
+                      uint64_t s2, uint32_t b0, uint32_t b1, uint32_t b2) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return -1;
   cuuint64_t dims[3] = {d0, d1, d2};
   cuuint64_t strides[2] = {s1 * 2, s2 * 2};
-  cuuint32_t box[3] = {b0, b1, 1};
+  cuuint32_t box[3] = {b0, b1, b2};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -92,6 +92,22 @@ int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint
   if (g_tmaps.size() > 65536) g_tmaps.clear();
   CUtensorMap m;
   int rc = make_tmap_2d_bf16(&m, p, rows, cols, ld, br, bc);
+  if (rc) return rc;
+  g_tmaps.emplace(k, m);
+  *out = m;
+  return 0;
+}
+
+// A weight matrix [N, K] seen as [K / 64][N][64]: one copy brings 16 rows x (64 * chunks) columns as `chunks` blocks of
+// 16 swizzled 128-byte lines (the weight-streaming kernels' ring stage).  Cached like the 2D maps.
+int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uint32_t chunks) {
+  TmapKey k{p, N, K, 0xFFFFFFFFull, 16, chunks};
+  std::lock_guard<std::mutex> g(g_tmap_mu);
+  auto it = g_tmaps.find(k);
+  if (it != g_tmaps.end()) { *out = it->second; return 0; }
+  if (g_tmaps.size() > 65536) g_tmaps.clear();
+  CUtensorMap m;
+  int rc = make_tmap_3d_bf16(&m, p, 64, N, K / 64, K, 64, 64, 16, chunks);
   if (rc) return rc;
   g_tmaps.emplace(k, m);
   *out = m;

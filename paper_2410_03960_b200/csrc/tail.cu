@@ -3,10 +3,12 @@
 // weights from HBM exactly once; attention is one query per (prompt, head) over the cache that the
 // SingleInputKV projection filled.  Activations of this path stay in fp32 (they are tiny), weights and the
 // cache stay in the model dtype.
+
 #include <cooperative_groups.h>
 #include <mma.h>
 
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace skv {
 
@@ -704,5 +706,440 @@ template void launch_tail_attention<bf16>(const float *, const bf16 *, const bf1
 template void launch_tail_attention<fp8e4>(const float *, const fp8e4 *, const fp8e4 *, const float *, const float *, float *,
                                            const int32_t *, const int32_t *, const int32_t *, int, int, int, int, int, int,
                                            float *, cudaStream_t, TailOpts);
+
+// ---------------------------------------------------------------------------------------------------------
+// Several dependent weight-streaming projections of the last-token path in ONE launch (bf16 weights): a persistent
+// cooperative kernel, one CTA per SM, walks a short list of stages -- per layer
+//     O projection + residual | [RMSNorm +] gate/up + SwiGLU | down projection + residual | [next layer's RMSNorm +] Q projection
+// (the single-query attention between a Q and an O projection stays its own kernel) -- separated by grid-wide barriers
+// instead of kernel boundaries.  Why: each stage moves 30 - 240 MB, i.e. 5 - 40 us at the HBM roofline, and a separate
+// launch adds its ramp, its tail and a dependent round trip to HBM to every one of them.  Here a producer warp streams
+// each CTA's weight rows AND the matching K-slice of the (at most 8) activation rows through a shared-memory ring with bulk
+// asynchronous copies (row segments of 1 - 2 KB, ~170 KB in flight per SM), so the HBM pipe stays full across tiles and --
+// the ring is refilled while the CTA waits at a barrier -- across stages, and the MMA warps never wait for L2.
+//   * work split of a projection: 16-feature tiles, tile t belongs to CTA t % gridDim; the 8 MMA warps split every K
+//     chunk of the tile (swap-AB mma.m16n8k16 as in skinny_mma_kernel, fp32 activations as bf16 hi + lo), are summed in
+//     shared memory in warp order (deterministic), and warp 0 runs the epilogue;
+//   * RMSNorm is folded into the projection that consumes it: every CTA recomputes the row statistics from the fp32
+//     residual rows (128 KB of L2 reads, while the ring fills) and scales the activation fragments by rstd * gain;
+//   * data produced inside the kernel is read with ld.global.cg or by the bulk copies, never through L1.
+// Every wait -- ring barriers, the grid barrier -- is bounded: on timeout the kernel latches STATUS_TIMEOUT, raises a
+// global abort word that every later wait sees at once, waits (bounded) for its own copies in flight and returns.
+// ---------------------------------------------------------------------------------------------------------
+namespace fused {
+
+constexpr int CONSUMERS = 8;
+constexpr int THREADS = (CONSUMERS + 1) * 32;
+constexpr int STAGES = 5;
+// one matrix: 16 rows x 512 columns per ring stage; two matrices (gate / up): 2 x (16 rows x 256 columns).  A stage is
+// filled by ONE tiled bulk copy per matrix (a copy per row segment costs the copy engine ~60 clocks each and capped the
+// stream at a third of the HBM rate): blocks of 16 lines of 128 bytes, 128-byte swizzle.
+constexpr int KC1 = 512, KC2 = 256;
+constexpr int STAGE_BYTES = 16 * KC1 * 2;             // 16384
+constexpr int RING_BYTES = STAGES * STAGE_BYTES;      // 81920
+constexpr int RES_BYTES = 131072;                     // resident activations: 8 row slots x K x (bf16 hi + bf16 lo), K <= 4096
+constexpr int RED_FLOATS = 2 * CONSUMERS * 2 * 32 * 4;   // two buffers of [warp][matrix][lane][4]
+constexpr int SM_RES = RING_BYTES, SM_RED = SM_RES + RES_BYTES, SM_BAR = SM_RED + RED_FLOATS * 4, SM_MISC = SM_BAR + 128;
+constexpr int SMEM_BYTES = SM_MISC + 256 + 1024;      // 230784 incl. the slack to align the ring to 1024 bytes
+constexpr long long WAIT_LIMIT = 4000000000LL;
+constexpr int MAX_STAGE_LIST = 6;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// one row segment: global -> this CTA's shared memory, completion bytes credited to `bar` (both addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// epi 0: out = A W^T (store); 1: out += A W^T; 2: out = silu(A W^T) * (A W2^T)
+struct Stage {
+  CUtensorMap tmW, tmW2;   // [N, K] as [K / 64][N][64], box (64, 16, KC / 64)
+  const float *A;          // [rows, K] fp32 (produced earlier, possibly in this launch)
+  const bf16 *gamma;       // non-null: A is RMS-normalised on the fly (row statistic * gain)
+  float *out;
+  int N, K, ldo, epi;
+};
+struct Params {
+  Stage st[MAX_STAGE_LIST];
+  int n_stages, rows;
+  float eps;
+  unsigned int sync_base;   // arrivals counted by earlier launches (the counter is never reset)
+  unsigned int *sync;       // [0] arrivals at the grid barrier, [1] abort word
+  unsigned int *status;
+};
+
+struct Ctx {
+  uint8_t *smem;
+  volatile int *abort_s;    // this CTA's copy of "give up"
+  unsigned epoch;           // grid barriers passed
+  unsigned chunk_no;        // ring chunks produced / consumed so far (same sequence in every role)
+};
+
+__device__ __forceinline__ bool aborted(const Params &p, Ctx &c) {
+  if (*c.abort_s) return true;
+  if (*reinterpret_cast<volatile unsigned int *>(p.sync + 1)) { *c.abort_s = 1; return true; }
+  return false;
+}
+__device__ __forceinline__ void give_up(const Params &p, Ctx &c) {
+  *c.abort_s = 1;
+  atomicOr(p.status, STATUS_TIMEOUT);
+  atomicExch(p.sync + 1, 1u);
+}
+__device__ __forceinline__ bool ring_wait(const Params &p, Ctx &c, uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (unsigned spins = 1;; ++spins) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spins & 63u) == 0u) {
+      if (aborted(p, c)) return false;
+      if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); return false; }
+    }
+  }
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// all CTAs of the (cooperative, hence co-resident) grid -- their MMA warps; the producer warps never stop here, they
+// keep the rings full with the next stage's weights.  Returns false when the kernel is giving up.
+__device__ __forceinline__ bool grid_barrier(const Params &p, Ctx &c) {
+  consumer_sync();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned target = p.sync_base + (c.epoch + 1) * gridDim.x;
+    atomicAdd(p.sync, 1u);
+    const long long t0 = clock64();
+    for (unsigned spins = 1;; ++spins) {
+      if ((int)(*reinterpret_cast<volatile unsigned int *>(p.sync) - target) >= 0) break;
+      if ((spins & 15u) == 0u) {
+        if (aborted(p, c)) break;
+        if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); break; }
+      }
+    }
+    __threadfence();
+  }
+  consumer_sync();
+  c.epoch += 1;
+  return !*c.abort_s;
+}
+
+// ---- producer warp: every stage's weight rows, tile by tile, chunk by chunk, through the ring
+__device__ void produce(const Params &p, Ctx &c) {
+  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES;
+  if ((threadIdx.x & 31) != 0) return;
+  for (int i = 0; i < p.n_stages; ++i) {
+    const Stage &sg = p.st[i];
+    const bool dual = sg.epi == 2;
+    const int kc_len = dual ? KC2 : KC1;
+    const int n_tiles = sg.N / 16, n_chunks = sg.K / kc_len;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      for (int kc = 0; kc < n_chunks; ++kc, ++c.chunk_no) {
+        const int st = c.chunk_no % STAGES;
+        const uint32_t ph = (c.chunk_no / STAGES) & 1;
+        if (!ring_wait(p, c, smem_u32(&empty[st]), ph ^ 1)) return;
+        const uint32_t fb = smem_u32(&full[st]);
+        mbar_expect_tx(fb, STAGE_BYTES);
+        const uint32_t dst = smem_u32(c.smem + st * STAGE_BYTES);
+        tc::tma_load_3d(dst, &sg.tmW, fb, 0, tile * 16, kc * (kc_len / 64));
+        if (dual) tc::tma_load_3d(dst + STAGE_BYTES / 2, &sg.tmW2, fb, 0, tile * 16, kc * (kc_len / 64));
+      }
+    }
+  }
+}
+
+// ---- MMA warps, one stage.  RESIDENT: the (normalised) activations sit in shared memory as bf16 hi / lo fragments, split
+//      once per stage; otherwise (rows * K too large) every chunk's fragments come from L2, one chunk ahead of their use
+template <bool DUAL, bool RESIDENT>
+__device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
+  constexpr int KC = DUAL ? KC2 : KC1;
+  constexpr int STEPS = KC / (CONSUMERS * 32);         // 32-wide K steps per warp and chunk: 2 (one matrix) or 1 (two)
+  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES;
+  float *red = reinterpret_cast<float *>(c.smem + SM_RED);
+  float *rstd_s = reinterpret_cast<float *>(c.smem + SM_MISC) + 8;
+  uint8_t *res = c.smem + SM_RES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int K = sg.K, n_tiles = sg.N / 16, n_chunks = K / KC;
+  const int g = lane >> 2, t = lane & 3;
+  const bool tok_ok = g < p.rows;
+  // RMSNorm folded in: activations are multiplied by the gain on the way in, the row statistic 1 / rms scales the OUTPUT
+  // row in the epilogue (it is a per-row scalar), so it can be accumulated in the same pass that brings the activations in
+  float ss[MAX_TAIL_ROWS];
+#pragma unroll
+  for (int r = 0; r < MAX_TAIL_ROWS; ++r) ss[r] = 0.f;
+  if (RESIDENT) {
+    // 8 consecutive K elements of one row -> 4 + 4 packed words at [K step][hi | lo][row][quarter]; loads in batches of 4
+    // (every CTA reads the same rows at the same moment: each starts at its own offset, so that at any instant the
+    // requests of the grid spread over the whole array instead of queueing on the same L2 lines)
+    const int octets_per_row = K / 8, n_oct = p.rows * octets_per_row;
+    const int rot = (int)(((long long)blockIdx.x * n_oct) / gridDim.x) & ~31;
+    for (int o0 = threadIdx.x; o0 < n_oct; o0 += 4 * CONSUMERS * 32) {
+      float4 xa[4], xb[4];
+      uint4 gm[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int ol = o0 + q * CONSUMERS * 32;
+        xa[q] = xb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        gm[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (ol < n_oct) {
+          const int o = ol + rot < n_oct ? ol + rot : ol + rot - n_oct;
+          const int r = o / octets_per_row, k8 = o - r * octets_per_row;
+          const float *src = sg.A + (size_t)r * K + (size_t)k8 * 8;
+          xa[q] = __ldcg(reinterpret_cast<const float4 *>(src));
+          xb[q] = __ldcg(reinterpret_cast<const float4 *>(src + 4));
+          if (sg.gamma) gm[q] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)k8 * 8));
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int ol = o0 + q * CONSUMERS * 32;
+        if (ol >= n_oct) continue;
+        const int o = ol + rot < n_oct ? ol + rot : ol + rot - n_oct;
+        const int r = o / octets_per_row, k8 = o - r * octets_per_row;
+        float x[8] = {xa[q].x, xa[q].y, xa[q].z, xa[q].w, xb[q].x, xb[q].y, xb[q].z, xb[q].w};
+        if (sg.gamma) {
+          float sq = 0.f;
+          const bf16 *ge = reinterpret_cast<const bf16 *>(&gm[q]);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) { sq = fmaf(x[e], x[e], sq); x[e] *= to_f(ge[e]); }
+#pragma unroll
+          for (int rr = 0; rr < MAX_TAIL_ROWS; ++rr) ss[rr] += (rr == r) ? sq : 0.f;
+        }
+        uint4 hi, lo;
+        split_hi_lo(x[0], x[1], hi.x, lo.x);
+        split_hi_lo(x[2], x[3], hi.y, lo.y);
+        split_hi_lo(x[4], x[5], hi.z, lo.z);
+        split_hi_lo(x[6], x[7], hi.w, lo.w);
+        uint8_t *dst = res + (size_t)(k8 >> 2) * 1024 + (size_t)(4 * r + (k8 & 3)) * 16;
+        *reinterpret_cast<uint4 *>(dst) = hi;
+        *reinterpret_cast<uint4 *>(dst + 512) = lo;
+      }
+    }
+  } else if (sg.gamma) {
+    for (int i = threadIdx.x * 4; i < K; i += CONSUMERS * 32 * 4) {
+#pragma unroll
+      for (int r = 0; r < MAX_TAIL_ROWS; ++r)
+        if (r < p.rows) {
+          const float4 v = __ldcg(reinterpret_cast<const float4 *>(sg.A + (size_t)r * K + i));
+          ss[r] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+    }
+  }
+  if (sg.gamma) {
+    float *part = red + 2 * CONSUMERS * 2 * 32 * 4 - CONSUMERS * MAX_TAIL_ROWS;      // the tail of the second buffer: [8 warps][8 rows]
+#pragma unroll
+    for (int r = 0; r < MAX_TAIL_ROWS; ++r) {
+      const float v = warp_sum(ss[r]);
+      if (lane == 0) part[warp * MAX_TAIL_ROWS + r] = v;
+    }
+    consumer_sync();
+    if (threadIdx.x < MAX_TAIL_ROWS) {
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < CONSUMERS; ++w) tot += part[w * MAX_TAIL_ROWS + threadIdx.x];
+      rstd_s[threadIdx.x] = rsqrtf(tot / (float)K + p.eps);
+    }
+  }
+  consumer_sync();
+  const int k_lane = warp * (STEPS * 32) + 8 * t;          // this lane's first K index inside a chunk
+  const float *a_row = sg.A + (size_t)g * K + k_lane;
+  // direct mode: the next chunk's activation fragments (and gains) are requested before the current chunk is multiplied
+  float4 nxa[STEPS], nxb[STEPS];
+  uint4 ngm[STEPS];
+  auto fetch = [&](int kc) {
+#pragma unroll
+    for (int u = 0; u < STEPS; ++u) {
+      nxa[u] = nxb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      ngm[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (tok_ok) {
+        nxa[u] = __ldcg(reinterpret_cast<const float4 *>(a_row + (size_t)kc * KC + u * 32));
+        nxb[u] = __ldcg(reinterpret_cast<const float4 *>(a_row + (size_t)kc * KC + u * 32 + 4));
+      }
+      if (sg.gamma) ngm[u] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)kc * KC + k_lane + u * 32));
+    }
+  };
+  int tile_no = 0;
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_no) {
+    // four independent accumulator chains per matrix
+    float acc[4][4] = {}, acc2[4][4] = {};
+    if (!RESIDENT) fetch(0);
+    for (int kc = 0; kc < n_chunks; ++kc, ++c.chunk_no) {
+      const int st = c.chunk_no % STAGES;
+      const uint32_t ph = (c.chunk_no / STAGES) & 1;
+      float4 xa[STEPS], xb[STEPS];
+      uint4 gm[STEPS];
+      if (!RESIDENT) {
+#pragma unroll
+        for (int u = 0; u < STEPS; ++u) { xa[u] = nxa[u]; xb[u] = nxb[u]; gm[u] = ngm[u]; }
+        if (kc + 1 < n_chunks) fetch(kc + 1);
+      }
+      if (!ring_wait(p, c, smem_u32(&full[st]), ph)) return;
+      const uint8_t *sw = c.smem + st * STAGE_BYTES;
+#pragma unroll
+      for (int u = 0; u < STEPS; ++u) {
+        uint32_t bh[4], bl[4];
+        if (RESIDENT) {
+          const uint8_t *fr = res + (size_t)(kc * (KC / 32) + warp * STEPS + u) * 1024 + (size_t)lane * 16;
+          const uint4 h4 = *reinterpret_cast<const uint4 *>(fr), l4 = *reinterpret_cast<const uint4 *>(fr + 512);
+          bh[0] = h4.x; bh[1] = h4.y; bh[2] = h4.z; bh[3] = h4.w;
+          bl[0] = l4.x; bl[1] = l4.y; bl[2] = l4.z; bl[3] = l4.w;
+          if (!tok_ok) { bh[0] = bh[1] = bh[2] = bh[3] = 0u; bl[0] = bl[1] = bl[2] = bl[3] = 0u; }
+        } else {
+          float x[8] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+          if (sg.gamma) {
+            const bf16 *ge = reinterpret_cast<const bf16 *>(&gm[u]);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) x[e] *= to_f(ge[e]);
+          }
+          split_hi_lo(x[0], x[1], bh[0], bl[0]);
+          split_hi_lo(x[2], x[3], bh[1], bl[1]);
+          split_hi_lo(x[4], x[5], bh[2], bl[2]);
+          split_hi_lo(x[6], x[7], bh[3], bl[3]);
+        }
+        // K index inside the chunk -> block of 64 columns (16 lines of 128 bytes) and 16-byte unit inside the line, swizzled
+        // by the line number (rows g and g + 8 share g & 7)
+        const int kk = k_lane + u * 32;
+        const uint32_t off = (uint32_t)(kk >> 6) * 2048u + (uint32_t)((((kk & 63) >> 3) ^ g) << 4);
+        const uint4 wl = *reinterpret_cast<const uint4 *>(sw + off + g * 128);
+        const uint4 wh = *reinterpret_cast<const uint4 *>(sw + off + (g + 8) * 128);
+        const uint32_t a1[4] = {wl.x, wh.x, wl.y, wh.y}, a2[4] = {wl.z, wh.z, wl.w, wh.w};
+        mma_bf16_16816(acc[0], a1, bh[0], bh[1]);
+        mma_bf16_16816(acc[1], a1, bl[0], bl[1]);
+        mma_bf16_16816(acc[2], a2, bh[2], bh[3]);
+        mma_bf16_16816(acc[3], a2, bl[2], bl[3]);
+        if (DUAL) {
+          const uint4 ul = *reinterpret_cast<const uint4 *>(sw + STAGE_BYTES / 2 + off + g * 128);
+          const uint4 uh = *reinterpret_cast<const uint4 *>(sw + STAGE_BYTES / 2 + off + (g + 8) * 128);
+          const uint32_t d1[4] = {ul.x, uh.x, ul.y, uh.y}, d2[4] = {ul.z, uh.z, ul.w, uh.w};
+          mma_bf16_16816(acc2[0], d1, bh[0], bh[1]);
+          mma_bf16_16816(acc2[1], d1, bl[0], bl[1]);
+          mma_bf16_16816(acc2[2], d2, bh[2], bh[3]);
+          mma_bf16_16816(acc2[3], d2, bl[2], bl[3]);
+        }
+      }
+      // Releasing the stage: every lane first fences its own reads of the stage (they must have been PERFORMED, not just
+      // issued, before the producer may overwrite it).  __syncwarp() + one arrive alone, and also one arrive per lane, were
+      // not enough: with reads still outstanding when the next copy landed, a few weight rows of a tile came out wrong
+      // once in ~20 steps at the 8B widths (seen on the down projection, whose MMA warps also wait on L2 loads).
+      __threadfence_block();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
+    }
+    // the 8 warps' partial tiles, summed in warp order by warp 0 (two buffers: one barrier per tile)
+    float *buf = red + (tile_no & 1) * (CONSUMERS * 2 * 32 * 4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      buf[((warp * 2 + 0) * 32 + lane) * 4 + i] = (acc[0][i] + acc[1][i]) + (acc[2][i] + acc[3][i]);
+      if (DUAL) buf[((warp * 2 + 1) * 32 + lane) * 4 + i] = (acc2[0][i] + acc2[1][i]) + (acc2[2][i] + acc2[3][i]);
+    }
+    consumer_sync();
+    if (warp == (tile_no & (CONSUMERS - 1))) {      // (the warps take turns, so that none falls a whole epilogue behind per tile)
+      float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int w = 0; w < CONSUMERS; ++w)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          s1[i] += buf[((w * 2 + 0) * 32 + lane) * 4 + i];
+          if (DUAL) s2[i] += buf[((w * 2 + 1) * 32 + lane) * 4 + i];
+        }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {      // fragment element i: feature 16 tile + g + 8 (i / 2), token 2 t + (i % 2)
+        const int n = tile * 16 + g + 8 * (i >> 1), r = 2 * t + (i & 1);
+        if (r < p.rows) {
+          const float rs = sg.gamma ? rstd_s[r] : 1.f;       // the folded norm's row statistic
+          float v = s1[i] * rs;
+          if (DUAL) v = v / (1.f + __expf(-v)) * (s2[i] * rs);
+          float *o = sg.out + (size_t)r * sg.ldo + n;
+          if (sg.epi == 1) v += __ldcg(o);
+          *o = v;
+        }
+      }
+    }
+  }
+  consumer_sync();       // the statistics / resident buffers may be rewritten by the next stage
+}
+
+__global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_constant__ Params p) {
+  extern __shared__ uint8_t fsmem_raw[];
+  uint8_t *fsmem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fsmem_raw) + 1023) & ~(uintptr_t)1023);
+  Ctx c;
+  c.smem = fsmem;
+  c.abort_s = reinterpret_cast<volatile int *>(fsmem + SM_MISC);
+  c.epoch = 0;
+  c.chunk_no = 0;
+  uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + SM_BAR), *empty = full + STAGES;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), CONSUMERS); }
+    *c.abort_s = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if ((threadIdx.x >> 5) == CONSUMERS) {
+    produce(p, c);
+    // giving up: copies still in flight must land before this CTA's shared memory is released
+    if (*c.abort_s && (threadIdx.x & 31) == 0) {
+      const unsigned issued = c.chunk_no;
+      for (unsigned q = issued > STAGES ? issued - STAGES : 0; q < issued; ++q) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(smem_u32(&full[q % STAGES]), (q / STAGES) & 1) && clock64() - t0 < 100000000LL) {}
+      }
+    }
+  } else {
+    for (int i = 0; i < p.n_stages; ++i) {
+      if (i > 0 && !grid_barrier(p, c)) break;
+      const Stage &sg = p.st[i];
+      const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
+      if (sg.epi == 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
+      else { if (resident) consume<false, true>(p, c, sg); else consume<false, false>(p, c, sg); }
+      if (*c.abort_s) break;
+    }
+  }
+  __syncthreads();
+}
+
+}  // namespace fused
+
+bool tail_fused_supported(int rows, int d, int dq, int F, int vocab) {
+  return rows >= 1 && rows <= MAX_TAIL_ROWS && d % fused::KC1 == 0 && dq % fused::KC1 == 0 && F % fused::KC1 == 0 && vocab % 16 == 0;
+}
+
+int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
+                      unsigned int *status, cudaStream_t st) {
+  if (n_stages < 1 || n_stages > fused::MAX_STAGE_LIST || rows < 1 || rows > MAX_TAIL_ROWS) return SWIFTKV_ERR_UNSUPPORTED;
+  fused::Params p{};
+  for (int i = 0; i < n_stages; ++i) {
+    const TailStage &s = stages[i];
+    const int kc = s.W2 ? fused::KC2 : fused::KC1;
+    if (s.N % 16 || s.K % kc || (s.W2 != nullptr) != (s.epi == 2)) return SWIFTKV_ERR_UNSUPPORTED;
+    fused::Stage &d = p.st[i];
+    if (get_tmap_rows16(&d.tmW, s.W, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
+    d.tmW2 = d.tmW;
+    if (s.W2 && get_tmap_rows16(&d.tmW2, s.W2, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
+    d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
+  }
+  p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
+  p.sync_base = *arrivals;
+  int dev = 0, n_sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
+    return SWIFTKV_ERR_CUDA;
+  const void *kern = (const void *)fused::tail_fused_kernel;
+  if (ensure_dynamic_smem(kern, fused::SMEM_BYTES)) return SWIFTKV_ERR_CUDA;
+  void *args[] = {&p};
+  if (cudaLaunchCooperativeKernel(kern, dim3((unsigned)n_sms), dim3(fused::THREADS), args, (size_t)fused::SMEM_BYTES, st) != cudaSuccess)
+    return SWIFTKV_ERR_CUDA;
+  *arrivals += (unsigned)(n_stages - 1) * (unsigned)n_sms;
+  return SWIFTKV_OK;
+}
 
 }  // namespace skv

@@ -273,9 +273,11 @@ __device__ __forceinline__ uint32_t pack_act(float lo, float hi, bool f16) {
 // (box_cols must be 64), out-of-range rows/cols read as zero.  Returns 0 on success.
 int make_tmap_2d_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
                       uint32_t box_rows, uint32_t box_cols);
-// bf16 tensor [d2][d1][d0] with element strides (s2, s1, 1); box (b0, b1, 1), 128-byte swizzle.
+// bf16 tensor [d2][d1][d0] with element strides (s2, s1, 1); box (b0, b1, b2), 128-byte swizzle.
 int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t s1,
-                      uint64_t s2, uint32_t b0, uint32_t b1);
+                      uint64_t s2, uint32_t b0, uint32_t b1, uint32_t b2);
+// cached map of a weight matrix [N, K] (K % 64 == 0) as [K / 64][N][64] with box (64, 16, chunks), 128-byte swizzle
+int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uint32_t chunks);
 
 // cached make_tmap_2d_bf16 (tensor maps are pure functions of pointer, shape and box)
 int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, uint32_t box_cols);

@@ -65,10 +65,11 @@ def test_more_prompts_than_one_tail_pass():
 
 
 @pytest.mark.parametrize("l,g", [(2, 1), (4, 1), (1, 2), (2, 2)])
-@pytest.mark.parametrize("mask,act", [(19, 1), (19, 0), (3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
+@pytest.mark.parametrize("mask,act", [(83, 1), (83, 0), (64, 1), (19, 1), (19, 0), (3, 1), (3, 0), (0, 1), (0, 0), (1, 1), (2, 1)])
 def test_mid_shape_bf16_tensor_core_and_simt_paths(l, g, mask, act):
     """The same model through the tcgen05 kernels (mask 3; mask 19: attention as persistent CTAs walking a host-balanced
-    work list), the SIMT kernels (mask 0) and the two mixtures, with
+    work list; mask 83: plus the last-token path as one persistent launch, mask 64: that launch after SIMT kernels), the SIMT
+    kernels (mask 0) and the two mixtures, with
     half (act 1) and bfloat16 (act 0) activations; several row tiles and a ragged tail (T = 507), prompts of 1 and
     129 tokens included."""
     lens = [300, 77, 129, 1]
@@ -362,6 +363,65 @@ def test_config4_full_size_against_oracle_samples():
     res = _check_config4_samples(model, lens, "config4_full_sample.npz")
     print("config4 full-size parity (half pairs):", lens, res)
     assert res["logit_rel"] <= 2e-2 and res["logit_abs"] <= 0.1, res
+    model.close()
+
+
+def test_fused_last_token_launch_against_oracle_and_the_per_operator_path():
+    """Kernel-mask bit 6: layers l+1..L and the lm_head of the continuing tokens in one persistent cooperative launch.
+    Eleven prompts (two passes of at most 8 rows), ragged lengths incl. 1 token, AcrossKV groups with a short last group;
+    against the oracle at the bf16 bars, against the per-operator path to fp32 summation-order noise, and bitwise
+    reproducible."""
+    import paper_2410_03960_b200 as P
+    lens = [300, 1, 129, 77, 513, 128, 2, 255, 40, 700, 9]
+    l, g = 1, 2
+    w = S.make_weights(MID, 6, torch.bfloat16, "cuda")
+    tok = S.make_prompts(6, lens, MID.vocab)
+    ref = O.swiftkv(oracle_config(MID), oracle_weights(w), tok.numpy(), lens, l, g)
+    out = {}
+    for mask in (119, 55):
+        model = P.SwiftKVModel(MID, w, torch.bfloat16, sum(lens), len(lens), l, g)
+        assert model.set_kernel_mask(mask) == mask
+        model.prefill(tok, lens, l, g)
+        model.status()
+        check_prefill_against_oracle(model, ref, MID.n_layers, 2e-2, 2e-2, 0.1)
+        out[mask] = model.first_logits().clone()
+        if mask == 119:
+            n_fused = model.last_launch_count()
+            model.prefill(tok, lens, l, g)
+            model.status()
+            assert torch.equal(out[119], model.first_logits())
+        else:
+            assert model.last_launch_count() > n_fused + 20          # the fused form really replaces ~10 launches per layer
+        model.close()
+    assert (out[119] - out[55]).abs().max().item() <= 2e-3
+
+
+def test_fused_last_token_launch_repeats_bit_for_bit_at_8b_widths():
+    """The fused launch streams weights through a shared-memory ring that a producer warp refills as soon as the MMA warps
+    release a stage; a release that comes before every lane has read the stage shows up as a few wrong weight rows in a
+    tile, rarely (one step in ~20 at these widths), so: 8 prompts (8 activation rows, the widest form), the 8B widths
+    (down projection K = 14336, the stage that reads activations from L2 while it multiplies), 60 repeats, equal bits."""
+    import paper_2410_03960_b200 as P
+    shape = S.LLAMA31_8B
+    lens = [700, 300, 512, 900, 411, 650, 1000, 257]
+    l, g = 16, 1
+    w = S.make_weights(shape, 1, torch.bfloat16, "cuda")
+    tok = S.make_prompts(1, lens, shape.vocab).cuda()
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, sum(lens), len(lens), l, g)
+    assert model.set_kernel_mask(119) == 119
+    first = None
+    for it in range(60):
+        model.prefill_device_tokens(tok, lens, l, g)
+        model.status()
+        lg = model.first_logits()
+        if first is None:
+            first = lg.clone()
+        else:
+            assert torch.equal(lg, first), f"repeat {it}: max difference {(lg - first).abs().max().item():.3e}"
+    model.set_kernel_mask(55)
+    model.prefill_device_tokens(tok, lens, l, g)
+    model.status()
+    assert (model.first_logits() - first).abs().max().item() <= 2e-3
     model.close()
 
 
