@@ -114,6 +114,29 @@ int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uin
   return 0;
 }
 
+// fp32 activations [rows, K] (rows <= 8) seen as [K / 32][rows][32]: one copy brings `steps` blocks of [row_slots][32
+// floats], rows beyond `rows` zero-filled (the fused last-token kernel's activation blocks).
+int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t row_slots, uint64_t K, uint32_t steps) {
+  TmapKey k{p, rows, K, 0xFFFFFFFEull, row_slots, steps};
+  std::lock_guard<std::mutex> g(g_tmap_mu);
+  auto it = g_tmaps.find(k);
+  if (it != g_tmaps.end()) { *out = it->second; return 0; }
+  if (g_tmaps.size() > 65536) g_tmaps.clear();
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return -1;
+  CUtensorMap m;
+  cuuint64_t dims[3] = {32, rows, K / 32};
+  cuuint64_t strides[2] = {K * 4, 128};
+  cuuint32_t box[3] = {32, row_slots, steps};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(p), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return -2;
+  g_tmaps.emplace(k, m);
+  *out = m;
+  return 0;
+}
+
 int ensure_dynamic_smem(const void *kernel, int bytes) {
   static std::mutex mu;
   static std::unordered_map<const void *, unsigned long long> done;   // kernel -> bit mask of devices already set

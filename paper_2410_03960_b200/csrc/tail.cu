@@ -737,12 +737,19 @@ constexpr int STAGES = 5;
 constexpr int KC1 = 512, KC2 = 256;
 constexpr int STAGE_BYTES = 16 * KC1 * 2;             // 16384
 constexpr int RING_BYTES = STAGES * STAGE_BYTES;      // 81920
-constexpr int RES_BYTES = 131072;                     // resident activations: 8 row slots x K x (bf16 hi + bf16 lo), K <= 4096
+// Activations come in blocks of one 32-wide K step: [row slots][32 floats], row slots = the launch's rows rounded up to a
+// power of two (1, 2, 4, 8; the padding rows are zero-filled), brought by tiled bulk copies.  K <= 4096: all K / 32 blocks
+// are resident and converted IN PLACE, once per stage, into the MMA fragments [bf16 hi | bf16 lo][row][quarter]; larger K:
+// the blocks of a K chunk travel with the chunk's weights through a ring of their own and are converted as they are used.
+constexpr int ACT_BLOCK = 1024;                       // the largest block: 8 row slots
+constexpr int RES_BYTES = 131072;
+constexpr int ACT_SLOT = (KC1 / 32) * ACT_BLOCK;      // 16384; STAGES of them fit RES_BYTES
 constexpr int RED_FLOATS = 2 * CONSUMERS * 2 * 32 * 4;   // two buffers of [warp][matrix][lane][4]
 constexpr int SM_RES = RING_BYTES, SM_RED = SM_RES + RES_BYTES, SM_BAR = SM_RED + RED_FLOATS * 4, SM_MISC = SM_BAR + 128;
 constexpr int SMEM_BYTES = SM_MISC + 256 + 1024;      // 230784 incl. the slack to align the ring to 1024 bytes
 constexpr long long WAIT_LIMIT = 4000000000LL;
 constexpr int MAX_STAGE_LIST = 6;
+static_assert(STAGES * ACT_SLOT <= RES_BYTES, "the activation ring lives in the resident area");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -760,15 +767,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// one row segment: global -> this CTA's shared memory, completion bytes credited to `bar` (both addresses 16-byte aligned)
-__device__ __forceinline__ void bulk_copy(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
+// data written with ordinary stores (by any SM, made visible by a barrier) is about to be read by a bulk copy
+__device__ __forceinline__ void fence_generic_to_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // epi 0: out = A W^T (store); 1: out += A W^T; 2: out = silu(A W^T) * (A W2^T)
 struct Stage {
   CUtensorMap tmW, tmW2;   // [N, K] as [K / 64][N][64], box (64, 16, KC / 64)
+  CUtensorMap tmA;         // [rows, K] fp32 as [K / 32][rows][32], box (32, row slots, KC / 32)
   const float *A;          // [rows, K] fp32 (produced earlier, possibly in this launch)
   const bf16 *gamma;       // non-null: A is RMS-normalised on the fly (row statistic * gain)
   float *out;
@@ -777,6 +782,7 @@ struct Stage {
 struct Params {
   Stage st[MAX_STAGE_LIST];
   int n_stages, rows;
+  int rs;                   // log2 of the row slots per activation block
   float eps;
   unsigned int sync_base;   // arrivals counted by earlier launches (the counter is never reset)
   unsigned int *sync;       // [0] arrivals at the grid barrier, [1] abort word
@@ -786,8 +792,10 @@ struct Params {
 struct Ctx {
   uint8_t *smem;
   volatile int *abort_s;    // this CTA's copy of "give up"
+  volatile int *open_s;     // the last stage whose inputs are complete (written by the MMA warps after the grid barrier)
   unsigned epoch;           // grid barriers passed
   unsigned chunk_no;        // ring chunks produced / consumed so far (same sequence in every role)
+  unsigned fill_no;         // resident fills so far
 };
 
 __device__ __forceinline__ bool aborted(const Params &p, Ctx &c) {
@@ -835,7 +843,9 @@ __device__ __forceinline__ bool grid_barrier(const Params &p, Ctx &c) {
   return !*c.abort_s;
 }
 
-// ---- producer warp: every stage's weight rows, tile by tile, chunk by chunk, through the ring
+// ---- producer warp (one lane): every stage's weight rows, tile by tile, chunk by chunk, through the ring -- as far ahead
+//      as the ring allows, across stage boundaries.  A stage whose K is too large for resident activations also gets each
+//      chunk's activation blocks, but those are requested only once the stage's inputs are complete (open_s).
 __device__ void produce(const Params &p, Ctx &c) {
   uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES;
   if ((threadIdx.x & 31) != 0) return;
@@ -844,107 +854,157 @@ __device__ void produce(const Params &p, Ctx &c) {
     const bool dual = sg.epi == 2;
     const int kc_len = dual ? KC2 : KC1;
     const int n_tiles = sg.N / 16, n_chunks = sg.K / kc_len;
+    const bool resident = (long long)sg.K * 32 <= RES_BYTES;
+    const uint32_t act_bytes = resident ? 0u : (uint32_t)(kc_len / 32) * (128u << p.rs);
+    const unsigned my_tiles = (int)blockIdx.x < n_tiles ? (unsigned)(n_tiles - 1 - (int)blockIdx.x) / gridDim.x + 1u : 0u;
+    const unsigned total = my_tiles * (unsigned)n_chunks, base = c.chunk_no;
+    unsigned act_j = resident ? total : 0u;       // next chunk of the stage whose activation blocks are still to be requested
+    int act_kc = 0;
+    bool open = i == 0;
+    auto request_activations = [&](unsigned issued) {
+      if (act_j >= issued) return;
+      if (!open) {
+        if (*c.open_s < i) return;
+        __threadfence();
+        fence_generic_to_async();
+        open = true;
+      }
+      for (; act_j < issued; ++act_j) {
+        const unsigned slot = (base + act_j) % STAGES;
+        tc::tma_load_3d(smem_u32(c.smem + SM_RES + slot * ACT_SLOT), &sg.tmA, smem_u32(&full[slot]), 0, 0, act_kc * (kc_len / 32));
+        if (++act_kc == n_chunks) act_kc = 0;
+      }
+    };
+    unsigned j = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-      for (int kc = 0; kc < n_chunks; ++kc, ++c.chunk_no) {
-        const int st = c.chunk_no % STAGES;
-        const uint32_t ph = (c.chunk_no / STAGES) & 1;
-        if (!ring_wait(p, c, smem_u32(&empty[st]), ph ^ 1)) return;
-        const uint32_t fb = smem_u32(&full[st]);
-        mbar_expect_tx(fb, STAGE_BYTES);
-        const uint32_t dst = smem_u32(c.smem + st * STAGE_BYTES);
+      for (int kc = 0; kc < n_chunks; ++kc, ++j) {
+        const unsigned slot = (base + j) % STAGES;
+        const uint32_t ph = ((base + j) / STAGES) & 1;
+        const uint32_t eb = smem_u32(&empty[slot]);
+        if (!mbar_try_wait(eb, ph ^ 1)) {
+          const long long t0 = clock64();
+          for (unsigned spins = 1; !mbar_try_wait(eb, ph ^ 1); ++spins) {
+            request_activations(j);
+            if ((spins & 63u) == 0u) {
+              if (aborted(p, c)) { c.chunk_no = base + j; return; }
+              if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); c.chunk_no = base + j; return; }
+            }
+          }
+        }
+        const uint32_t fb = smem_u32(&full[slot]);
+        mbar_expect_tx(fb, STAGE_BYTES + act_bytes);
+        const uint32_t dst = smem_u32(c.smem + slot * STAGE_BYTES);
         tc::tma_load_3d(dst, &sg.tmW, fb, 0, tile * 16, kc * (kc_len / 64));
         if (dual) tc::tma_load_3d(dst + STAGE_BYTES / 2, &sg.tmW2, fb, 0, tile * 16, kc * (kc_len / 64));
+        request_activations(j + 1);
+      }
+    }
+    c.chunk_no = base + total;
+    if (act_j < total) {
+      const long long t0 = clock64();
+      for (unsigned spins = 1; act_j < total; ++spins) {
+        request_activations(total);
+        if ((spins & 63u) == 0u) {
+          if (aborted(p, c)) return;
+          if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); return; }
+        }
       }
     }
   }
 }
 
-// ---- MMA warps, one stage.  RESIDENT: the (normalised) activations sit in shared memory as bf16 hi / lo fragments, split
-//      once per stage; otherwise (rows * K too large) every chunk's fragments come from L2, one chunk ahead of their use
+// ---- MMA warps, one stage.  RESIDENT: the (gain-scaled) activations sit in shared memory as bf16 hi / lo fragments, made
+//      once per stage; otherwise every chunk's fp32 blocks arrive with its weights and are split as they are used
 template <bool DUAL, bool RESIDENT>
 __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
   constexpr int KC = DUAL ? KC2 : KC1;
   constexpr int STEPS = KC / (CONSUMERS * 32);         // 32-wide K steps per warp and chunk: 2 (one matrix) or 1 (two)
-  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES;
+  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES, *afull = empty + STAGES;
   float *red = reinterpret_cast<float *>(c.smem + SM_RED);
   float *rstd_s = reinterpret_cast<float *>(c.smem + SM_MISC) + 8;
   uint8_t *res = c.smem + SM_RES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = sg.K, n_tiles = sg.N / 16, n_chunks = K / KC;
   const int g = lane >> 2, t = lane & 3;
-  const bool tok_ok = g < p.rows;
+  const int rs = p.rs, RP = 1 << rs, AB = 128 << rs;   // row slots, bytes per activation block
+  const bool row_ok = g < RP;
   // RMSNorm folded in: activations are multiplied by the gain on the way in, the row statistic 1 / rms scales the OUTPUT
   // row in the epilogue (it is a per-row scalar), so it can be accumulated in the same pass that brings the activations in
-  float ss[MAX_TAIL_ROWS];
-#pragma unroll
-  for (int r = 0; r < MAX_TAIL_ROWS; ++r) ss[r] = 0.f;
+  float ss = 0.f;                                      // RESIDENT: this lane's row (g); else row (lane & 7)
   if (RESIDENT) {
-    // 8 consecutive K elements of one row -> 4 + 4 packed words at [K step][hi | lo][row][quarter]; loads in batches of 4
-    // (every CTA reads the same rows at the same moment: each starts at its own offset, so that at any instant the
-    // requests of the grid spread over the whole array instead of queueing on the same L2 lines)
-    const int octets_per_row = K / 8, n_oct = p.rows * octets_per_row;
-    const int rot = (int)(((long long)blockIdx.x * n_oct) / gridDim.x) & ~31;
-    for (int o0 = threadIdx.x; o0 < n_oct; o0 += 4 * CONSUMERS * 32) {
-      float4 xa[4], xb[4];
-      uint4 gm[4];
+    if (threadIdx.x == 0) {
+      fence_generic_to_async();
+      mbar_expect_tx(smem_u32(afull), (uint32_t)(K / 32) * (uint32_t)AB);
+      for (int part = 0; part < K / KC1; ++part)
+        tc::tma_load_3d(smem_u32(res + part * (KC1 / 32) * AB), &sg.tmA, smem_u32(afull), 0, 0, part * (KC1 / 32));
+    }
+    if (!ring_wait(p, c, smem_u32(afull), c.fill_no & 1)) return;
+    c.fill_no += 1;
+    // every warp converts, in place, exactly the blocks it will multiply with, 8 / RP blocks at a time:
+    // lane = (block of the group, row, quarter)
+    const int grp = g >> rs, r = g & (RP - 1), G = 8 >> rs;
+    const int n_blk = K / (32 * CONSUMERS);
+    for (int b = 0; b < n_blk; b += 2 * G) {
+      uint8_t *blk[2];
+      float x[2][8];
+      uint4 gm[2];
+      bool live[2];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int ol = o0 + q * CONSUMERS * 32;
-        xa[q] = xb[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        gm[q] = make_uint4(0u, 0u, 0u, 0u);
-        if (ol < n_oct) {
-          const int o = ol + rot < n_oct ? ol + rot : ol + rot - n_oct;
-          const int r = o / octets_per_row, k8 = o - r * octets_per_row;
-          const float *src = sg.A + (size_t)r * K + (size_t)k8 * 8;
-          xa[q] = __ldcg(reinterpret_cast<const float4 *>(src));
-          xb[q] = __ldcg(reinterpret_cast<const float4 *>(src + 4));
-          if (sg.gamma) gm[q] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)k8 * 8));
+      for (int h = 0; h < 2; ++h) {
+        const int bb = b + h * G + grp;
+        live[h] = bb < n_blk;
+        const int s = (bb / STEPS) * (CONSUMERS * STEPS) + warp * STEPS + (bb % STEPS);
+        blk[h] = res + (size_t)s * AB;
+        float4 xa = make_float4(0.f, 0.f, 0.f, 0.f), xb = xa;
+        if (live[h]) {
+          xa = *reinterpret_cast<const float4 *>(blk[h] + r * 128 + t * 32);
+          xb = *reinterpret_cast<const float4 *>(blk[h] + r * 128 + t * 32 + 16);
         }
+        x[h][0] = xa.x; x[h][1] = xa.y; x[h][2] = xa.z; x[h][3] = xa.w;
+        x[h][4] = xb.x; x[h][5] = xb.y; x[h][6] = xb.z; x[h][7] = xb.w;
+        gm[h] = make_uint4(0u, 0u, 0u, 0u);
+        if (sg.gamma && live[h]) gm[h] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)s * 32 + t * 8));
       }
+      __syncwarp();
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int ol = o0 + q * CONSUMERS * 32;
-        if (ol >= n_oct) continue;
-        const int o = ol + rot < n_oct ? ol + rot : ol + rot - n_oct;
-        const int r = o / octets_per_row, k8 = o - r * octets_per_row;
-        float x[8] = {xa[q].x, xa[q].y, xa[q].z, xa[q].w, xb[q].x, xb[q].y, xb[q].z, xb[q].w};
+      for (int h = 0; h < 2; ++h) {
         if (sg.gamma) {
-          float sq = 0.f;
-          const bf16 *ge = reinterpret_cast<const bf16 *>(&gm[q]);
+          const bf16 *ge = reinterpret_cast<const bf16 *>(&gm[h]);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) { sq = fmaf(x[e], x[e], sq); x[e] *= to_f(ge[e]); }
-#pragma unroll
-          for (int rr = 0; rr < MAX_TAIL_ROWS; ++rr) ss[rr] += (rr == r) ? sq : 0.f;
+          for (int e = 0; e < 8; ++e) { ss = fmaf(x[h][e], x[h][e], ss); x[h][e] *= to_f(ge[e]); }
         }
         uint4 hi, lo;
-        split_hi_lo(x[0], x[1], hi.x, lo.x);
-        split_hi_lo(x[2], x[3], hi.y, lo.y);
-        split_hi_lo(x[4], x[5], hi.z, lo.z);
-        split_hi_lo(x[6], x[7], hi.w, lo.w);
-        uint8_t *dst = res + (size_t)(k8 >> 2) * 1024 + (size_t)(4 * r + (k8 & 3)) * 16;
-        *reinterpret_cast<uint4 *>(dst) = hi;
-        *reinterpret_cast<uint4 *>(dst + 512) = lo;
-      }
-    }
-  } else if (sg.gamma) {
-    for (int i = threadIdx.x * 4; i < K; i += CONSUMERS * 32 * 4) {
-#pragma unroll
-      for (int r = 0; r < MAX_TAIL_ROWS; ++r)
-        if (r < p.rows) {
-          const float4 v = __ldcg(reinterpret_cast<const float4 *>(sg.A + (size_t)r * K + i));
-          ss[r] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        split_hi_lo(x[h][0], x[h][1], hi.x, lo.x);
+        split_hi_lo(x[h][2], x[h][3], hi.y, lo.y);
+        split_hi_lo(x[h][4], x[h][5], hi.z, lo.z);
+        split_hi_lo(x[h][6], x[h][7], hi.w, lo.w);
+        if (live[h]) {
+          *reinterpret_cast<uint4 *>(blk[h] + (4 * r + t) * 16) = hi;
+          *reinterpret_cast<uint4 *>(blk[h] + (AB >> 1) + (4 * r + t) * 16) = lo;
         }
+      }
+      __syncwarp();
     }
+    // row r's sum: over the quarters and over the blocks of a group, in a fixed order
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    for (int m = 4 << rs; m < 32; m <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+  } else if (sg.gamma) {
+    // 4 lanes per row: quarters of the row, from L2 (the blocks in shared memory pass by only once)
+    const int r = lane >> 2;
+    if (r < p.rows)
+      for (int i = (warp * 4 + t) * 4; i < K; i += CONSUMERS * 4 * 4) {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(sg.A + (size_t)r * K + i));
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+      }
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
   }
   if (sg.gamma) {
     float *part = red + 2 * CONSUMERS * 2 * 32 * 4 - CONSUMERS * MAX_TAIL_ROWS;      // the tail of the second buffer: [8 warps][8 rows]
-#pragma unroll
-    for (int r = 0; r < MAX_TAIL_ROWS; ++r) {
-      const float v = warp_sum(ss[r]);
-      if (lane == 0) part[warp * MAX_TAIL_ROWS + r] = v;
-    }
+    if (t == 0 && g < (RESIDENT ? RP : MAX_TAIL_ROWS)) part[warp * MAX_TAIL_ROWS + g] = ss;
     consumer_sync();
-    if (threadIdx.x < MAX_TAIL_ROWS) {
+    if (threadIdx.x < p.rows) {
       float tot = 0.f;
 #pragma unroll
       for (int w = 0; w < CONSUMERS; ++w) tot += part[w * MAX_TAIL_ROWS + threadIdx.x];
@@ -953,36 +1013,20 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
   }
   consumer_sync();
   const int k_lane = warp * (STEPS * 32) + 8 * t;          // this lane's first K index inside a chunk
-  const float *a_row = sg.A + (size_t)g * K + k_lane;
-  // direct mode: the next chunk's activation fragments (and gains) are requested before the current chunk is multiplied
-  float4 nxa[STEPS], nxb[STEPS];
-  uint4 ngm[STEPS];
-  auto fetch = [&](int kc) {
-#pragma unroll
-    for (int u = 0; u < STEPS; ++u) {
-      nxa[u] = nxb[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-      ngm[u] = make_uint4(0u, 0u, 0u, 0u);
-      if (tok_ok) {
-        nxa[u] = __ldcg(reinterpret_cast<const float4 *>(a_row + (size_t)kc * KC + u * 32));
-        nxb[u] = __ldcg(reinterpret_cast<const float4 *>(a_row + (size_t)kc * KC + u * 32 + 4));
-      }
-      if (sg.gamma) ngm[u] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)kc * KC + k_lane + u * 32));
-    }
-  };
   int tile_no = 0;
   for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_no) {
     // four independent accumulator chains per matrix
     float acc[4][4] = {}, acc2[4][4] = {};
-    if (!RESIDENT) fetch(0);
     for (int kc = 0; kc < n_chunks; ++kc, ++c.chunk_no) {
       const int st = c.chunk_no % STAGES;
       const uint32_t ph = (c.chunk_no / STAGES) & 1;
-      float4 xa[STEPS], xb[STEPS];
       uint4 gm[STEPS];
       if (!RESIDENT) {
 #pragma unroll
-        for (int u = 0; u < STEPS; ++u) { xa[u] = nxa[u]; xb[u] = nxb[u]; gm[u] = ngm[u]; }
-        if (kc + 1 < n_chunks) fetch(kc + 1);
+        for (int u = 0; u < STEPS; ++u) {
+          gm[u] = make_uint4(0u, 0u, 0u, 0u);
+          if (sg.gamma) gm[u] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)kc * KC + k_lane + u * 32));
+        }
       }
       if (!ring_wait(p, c, smem_u32(&full[st]), ph)) return;
       const uint8_t *sw = c.smem + st * STAGE_BYTES;
@@ -990,13 +1034,22 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
       for (int u = 0; u < STEPS; ++u) {
         uint32_t bh[4], bl[4];
         if (RESIDENT) {
-          const uint8_t *fr = res + (size_t)(kc * (KC / 32) + warp * STEPS + u) * 1024 + (size_t)lane * 16;
-          const uint4 h4 = *reinterpret_cast<const uint4 *>(fr), l4 = *reinterpret_cast<const uint4 *>(fr + 512);
+          uint4 h4 = make_uint4(0u, 0u, 0u, 0u), l4 = h4;
+          if (row_ok) {
+            const uint8_t *fr = res + (size_t)(kc * (KC / 32) + warp * STEPS + u) * AB + (size_t)lane * 16;
+            h4 = *reinterpret_cast<const uint4 *>(fr);
+            l4 = *reinterpret_cast<const uint4 *>(fr + (AB >> 1));
+          }
           bh[0] = h4.x; bh[1] = h4.y; bh[2] = h4.z; bh[3] = h4.w;
           bl[0] = l4.x; bl[1] = l4.y; bl[2] = l4.z; bl[3] = l4.w;
-          if (!tok_ok) { bh[0] = bh[1] = bh[2] = bh[3] = 0u; bl[0] = bl[1] = bl[2] = bl[3] = 0u; }
         } else {
-          float x[8] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+          float4 xa = make_float4(0.f, 0.f, 0.f, 0.f), xb = xa;
+          if (row_ok) {
+            const uint8_t *fa = res + (size_t)st * ACT_SLOT + (size_t)(warp * STEPS + u) * AB + g * 128 + t * 32;
+            xa = *reinterpret_cast<const float4 *>(fa);
+            xb = *reinterpret_cast<const float4 *>(fa + 16);
+          }
+          float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
           if (sg.gamma) {
             const bf16 *ge = reinterpret_cast<const bf16 *>(&gm[u]);
 #pragma unroll
@@ -1031,12 +1084,12 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
       // Releasing the stage: every lane first fences its own reads of the stage (they must have been PERFORMED, not just
       // issued, before the producer may overwrite it).  __syncwarp() + one arrive alone, and also one arrive per lane, were
       // not enough: with reads still outstanding when the next copy landed, a few weight rows of a tile came out wrong
-      // once in ~20 steps at the 8B widths (seen on the down projection, whose MMA warps also wait on L2 loads).
+      // once in ~20 steps at the 8B widths.
       __threadfence_block();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
     }
-    // the 8 warps' partial tiles, summed in warp order by warp 0 (two buffers: one barrier per tile)
+    // the 8 warps' partial tiles, summed in warp order by one warp (two buffers: one barrier per tile)
     float *buf = red + (tile_no & 1) * (CONSUMERS * 2 * 32 * 4);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -1076,12 +1129,16 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
   Ctx c;
   c.smem = fsmem;
   c.abort_s = reinterpret_cast<volatile int *>(fsmem + SM_MISC);
+  c.open_s = c.abort_s + 1;
   c.epoch = 0;
   c.chunk_no = 0;
-  uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + SM_BAR), *empty = full + STAGES;
+  c.fill_no = 0;
+  uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + SM_BAR), *empty = full + STAGES, *afull = empty + STAGES;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), CONSUMERS); }
+    mbar_init(smem_u32(afull), 1);
     *c.abort_s = 0;
+    *c.open_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -1097,7 +1154,10 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
     }
   } else {
     for (int i = 0; i < p.n_stages; ++i) {
-      if (i > 0 && !grid_barrier(p, c)) break;
+      if (i > 0) {
+        if (!grid_barrier(p, c)) break;
+        if (threadIdx.x == 0) *c.open_s = i;
+      }
       const Stage &sg = p.st[i];
       const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
       if (sg.epi == 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
@@ -1118,6 +1178,9 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
                       unsigned int *status, cudaStream_t st) {
   if (n_stages < 1 || n_stages > fused::MAX_STAGE_LIST || rows < 1 || rows > MAX_TAIL_ROWS) return SWIFTKV_ERR_UNSUPPORTED;
   fused::Params p{};
+  int rs = 0;
+  while ((1 << rs) < rows) ++rs;
+  p.rs = rs;
   for (int i = 0; i < n_stages; ++i) {
     const TailStage &s = stages[i];
     const int kc = s.W2 ? fused::KC2 : fused::KC1;
@@ -1126,6 +1189,8 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
     if (get_tmap_rows16(&d.tmW, s.W, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
     d.tmW2 = d.tmW;
     if (s.W2 && get_tmap_rows16(&d.tmW2, s.W2, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
+    const bool resident = (long long)s.K * 32 <= fused::RES_BYTES;
+    if (get_tmap_act_f32(&d.tmA, s.A, rows, 1u << rs, s.K, resident ? fused::KC1 / 32 : kc / 32)) return SWIFTKV_ERR_CUDA;
     d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
   }
   p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
