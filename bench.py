@@ -76,7 +76,7 @@ def other_rooflines(prof, f_sw, lens, steps, tensor_peak, hbm_peak):
     # last-token path: every later layer's Q, O, gate, up, down weights once, the lm_head once, every later layer's cache rows once
     tail_bytes = (Lt * (2.0 * d * dq + 3.0 * d * F) * 2 + SHAPE.vocab * d * 2.0 + Lt * T * 2.0 * dkv * 2) * steps
     add("last-token path (weight streaming + single-query attention)", "hbm", tail_bytes, prof["tail"][0], hbm_peak, "GB/s",
-        "weights and cache rows of layers > l read once; ~120 small dependent launches per step")
+        "weights and cache rows of layers > l read once; per layer one fused persistent launch (O, gate/up, down, next Q) + the single-query attention")
     return out
 
 

@@ -264,7 +264,7 @@ int32_t swiftkv_last_launch_count(const swiftkv_model *m);
  * layer's Q or the lm_head, norms folded in) run as ONE persistent cooperative launch (weight rows streamed through a
  * shared-memory ring, grid-wide barriers between the stages) instead of one launch per operator; bf16 models whose
  * hidden, query and FFN widths are multiples of 512.
- * Default 55: everything that the model's shape and dtype support except bits 3 and 6.  Returns the mask in effect. */
+ * Default 119: everything that the model's shape and dtype support except bit 3.  Returns the mask in effect. */
 int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 
 /* Storage format of the intermediate activations of a bf16 model (normed hidden states, queries, attention

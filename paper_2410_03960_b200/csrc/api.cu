@@ -101,7 +101,7 @@ struct swiftkv_model {
   int n_tokens = 0, n_seqs = 0, cur_l = 0, cur_g = 1;   // rows in use per cache plane, sequences with logits
   int fold_l = -1, fold_g = -1, fold_fmt = -1;
   int launches = 0;
-  int kernel_mask = 55;
+  int kernel_mask = 119;
   int n_sms = 0;
   int act_format = SWIFTKV_ACT_F16;
   float *capture = nullptr;     // while set: layer j's input (the residual stream before layer j) is copied to capture[j][T][d]
