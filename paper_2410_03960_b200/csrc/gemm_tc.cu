@@ -777,14 +777,18 @@ int launch_bounded_wait_probe(long long limit_clocks, unsigned int *status, unsi
 bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (N % 128) == 0 && N >= 128; }
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
 
-static int group_m_setting() {
-  static int v = 0;
+// Raster band height in 128-row blocks.  A band's A rows (band x K x 2 bytes) are re-walked for every column block, so they
+// must stay in L2 next to the streaming weights and output: 4096 rows for K <= 8192, 2048 rows for longer K.
+static int group_m_setting(int K) {
+  static int v = 0, v_long = 0;
   if (!v) {
-    const char *e = getenv("SWIFTKV_GROUP_M");
-    v = e ? atoi(e) : 16;
-    if (v < 1) v = 16;
+    const char *e = getenv("SWIFTKV_GROUP_M"), *el = getenv("SWIFTKV_GROUP_M_LONGK");
+    v_long = el ? atoi(el) : (e ? atoi(e) : 16);
+    if (v_long < 1) v_long = 16;
+    v = e ? atoi(e) : 32;
+    if (v < 1) v = 32;
   }
-  return v;
+  return K > 8192 ? v_long : v;
 }
 static bool g_use_pairs = true, g_swiglu_pairs = false;
 void tc_gemm_use_cta_pairs(bool on, bool swiglu_too) { g_use_pairs = on; g_swiglu_pairs = swiglu_too; }
@@ -817,7 +821,7 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
   p.lo_act = 0;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = N / BN;
-  p.out = out; p.act = nullptr; p.F = 0; p.status = status; p.group_m = group_m_setting();
+  p.out = out; p.act = nullptr; p.F = 0; p.status = status; p.group_m = group_m_setting(K);
   p.f16 = f16; p.dup_base = reinterpret_cast<__half *>(dup_base); p.dup_stride = dup_stride;
   if (dup_base && !rope) return SWIFTKV_ERR_UNSUPPORTED;
   const bool pairs = g_use_pairs && BN == 256 && M > 128;
@@ -858,7 +862,7 @@ int launch_gemm_tc_swiglu(const void *A, bool f16, int M, int K, const void *Wg,
   p.lo_p0 = nullptr; p.lo_dup = nullptr; p.lo_act = out_split ? 1 : 0;
   p.num_m_blocks = (M + BM - 1) / BM;
   p.num_n_blocks = F / 128;
-  p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status; p.group_m = group_m_setting();
+  p.out = OutDesc{}; p.act = reinterpret_cast<bf16 *>(act); p.F = F; p.status = status; p.group_m = group_m_setting(K);
   p.f16 = f16; p.dup_base = nullptr; p.dup_stride = 0;
   // measured on the 8B shape under the power cap: the single-CTA form is 3 % faster for this launch (it already keeps
   // the tensor pipe 85 % busy), while the pair form wins 7-10 % on the N = 4096 / 6144 projections
