@@ -43,9 +43,9 @@ ORACLE_SAMPLE_TOKENS_PER_PROMPT = 32
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0
-# DRAM traffic of one fused gate/up GEMM launch.  The committed ncu capture (profiles/gemm_tc_kernel_8b_widths.md)
-# measured 1.2315 GB at T = 8192 tokens: the two weight matrices (235 MB) are re-streamed once per band of 2048
-# rows (4 bands), A (67 MB) and the SwiGLU output (235 MB, 225 MB seen at capture end) move once.  The full
+# DRAM traffic of one fused gate/up GEMM launch.  The committed ncu capture (profiles/gemm_tc_kernel_8b_widths.md, band
+# height 32) measured 0.7636 GB at T = 8192 tokens: the two weight matrices (235 MB) are re-streamed once per band of
+# 4096 rows (2 bands), A (67 MB) and the SwiGLU output (235 MB, 224 MB seen at capture end) move once.  The full
 # workload cannot be captured under the profiling size rule, so the capture is scaled with that model:
 SWIGLU_WEIGHT_BYTES = 2 * 14336 * 4096 * 2
 SWIGLU_CAPTURE_TOKENS, SWIGLU_CAPTURE_BYTES, SWIGLU_BAND_ROWS = 8192, 0.7636e9, 4096

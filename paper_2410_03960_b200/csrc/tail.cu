@@ -1171,7 +1171,18 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
 }  // namespace fused
 
 bool tail_fused_supported(int rows, int d, int dq, int F, int vocab) {
-  return rows >= 1 && rows <= MAX_TAIL_ROWS && d % fused::KC1 == 0 && dq % fused::KC1 == 0 && F % fused::KC1 == 0 && vocab % 16 == 0;
+  // the grid barriers need every CTA resident at once: a device (or context) that cannot promise that keeps the
+  // per-operator kernels
+  static int coop = -1;
+  if (coop < 0) {
+    int dev = 0, v = 0, per_sm = 0;
+    coop = cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v &&
+           ensure_dynamic_smem((const void *)fused::tail_fused_kernel, fused::SMEM_BYTES) == 0 &&
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused::tail_fused_kernel, fused::THREADS, fused::SMEM_BYTES) == cudaSuccess &&
+           per_sm >= 1;
+  }
+  return coop == 1 && rows >= 1 && rows <= MAX_TAIL_ROWS && d % fused::KC1 == 0 && dq % fused::KC1 == 0 && F % fused::KC1 == 0 &&
+         vocab % 16 == 0;
 }
 
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
