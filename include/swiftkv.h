@@ -200,6 +200,38 @@ size_t  swiftkv_simscore_scratch_bytes(const swiftkv_model *m, int32_t n_tokens)
 int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
                          void *scratch, size_t scratch_bytes, float *sim, float *simscore, void *cuda_stream);
 
+/* Knowledge recovery, Sec. 3.4 Eq. 3 ("Efficient Distillation"; temperature 2.0 in the training details of the appendix):
+ * one frozen copy of the model runs in two modes on the same batch --
+ *     y_teacher = M(x, SwiftKV = False)   every token through every unmodified layer,
+ *     y_student = M(x, SwiftKV = True)    layers > swift_layer re-wired: their K / V come from x_{l+1} through the group
+ *                                         leader's input-norm gain and the STUDENT's W_K, W_V (Eq. 2, AcrossKV groups of
+ *                                         Sec. 3.3), their queries from the layer's own normalised input through the
+ *                                         student's W_Q; in training every prompt token runs every layer --
+ * and this call returns the standard distillation loss on the two logit tensors,
+ *     loss = T^2 * mean over all prompt tokens of KL( softmax(y_teacher / T) || softmax(y_student / T) ),  T = temperature,
+ * and its gradient with respect to the student's W_Q, W_K, W_V of every layer > swift_layer (the only trainable
+ * parameters; norm gains and everything else stay frozen).  Layers 1..swift_layer are shared by both modes and run once.
+ *   tokens      : DEVICE int32 [sum(seq_lens)], packed prompt-major;  seq_lens: HOST int32 [n_seqs], every prompt >= 1 token
+ *   student_w*  : HOST arrays [n_layers] of DEVICE pointers, fp32 [out_features][hidden] like the model's own matrices;
+ *                 entries of layers <= swift_layer (0-based index < swift_layer) are ignored and may be null.  With
+ *                 acrosskv_group > 1 only the first layer of each group projects K / V: the other layers' student W_K / W_V
+ *                 are never read and their gradients are written as zeros.
+ *   grad_w*     : HOST arrays [n_layers] of DEVICE pointers, fp32, same shapes, WRITTEN (not accumulated)
+ *   loss        : DEVICE fp32 scalar, written
+ *   workspace   : DEVICE, caller-owned, 256-byte aligned, >= swiftkv_distill_workspace_bytes(m, total tokens, swift_layer)
+ * fp32 models only (SWIFTKV_ERR_UNSUPPORTED otherwise): the step runs in fp32 on the CUDA cores; gradients repeat bit for
+ * bit (every output element is summed by one block in a fixed order).  The model's prefill state (swiftkv_kv_cache_view,
+ * swiftkv_first_logits) is invalid afterwards until the next prefill.  The sequence offsets are copied with a blocking
+ * copy after synchronising `cuda_stream`; everything else is queued on it.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_SMALL, CUDA.
+ */
+size_t  swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer);
+int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                              int32_t swift_layer, int32_t acrosskv_group, float temperature,
+                              const void *const *student_wq, const void *const *student_wk, const void *const *student_wv,
+                              void *const *grad_wq, void *const *grad_wk, void *const *grad_wv, float *loss,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 typedef struct {
   const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype (FP8 cache: uint8 e4m3
                                codes), AFTER RoPE                                                           */

@@ -26,6 +26,7 @@ EXPORTS = (
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
     "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
+    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads",
 )
 
 
@@ -97,6 +98,10 @@ def load_library() -> C.CDLL:
     lib.swiftkv_simscore_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_simscore.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p,
                                      C.c_void_p]
+    lib.swiftkv_distill_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    lib.swiftkv_distill_workspace_bytes.restype = C.c_size_t
+    lib.swiftkv_distill_grads.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float] + [C.c_void_p] * 8 + \
+        [C.c_size_t, C.c_void_p]
     lib.swiftkv_gemm_tc_split.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
@@ -276,6 +281,31 @@ class SwiftKVModel:
                                              sim.data_ptr(), score.data_ptr(), _stream_ptr(stream)))
             torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
         return score, sim
+
+    def distill_grads(self, tokens, seq_lens: Sequence[int], swift_layer: int, acrosskv_group: int, temperature: float,
+                      student: dict, stream: Optional[torch.cuda.Stream] = None):
+        """swiftkv_distill_grads (Sec. 3.4, Eq. 3).  student: {"wq" | "wk" | "wv": list over layers of fp32 CUDA tensors (None for
+        layers <= swift_layer)}.  Returns (loss tensor [1], {"wq" | "wk" | "wv": list of gradient tensors, None likewise})."""
+        L = self.shape.n_layers
+        tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous().to(self.device)
+        lens = (C.c_int32 * len(seq_lens))(*[int(n) for n in seq_lens])
+        nbytes = self.lib.swiftkv_distill_workspace_bytes(self._h, int(sum(seq_lens)), int(swift_layer))
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        loss = torch.zeros(1, dtype=torch.float32, device=self.device)
+        grads = {k: [None if student[k][j] is None else torch.empty_like(student[k][j]) for j in range(L)] for k in ("wq", "wk", "wv")}
+
+        def ptrs(lst):
+            return (C.c_void_p * L)(*[None if t is None else t.data_ptr() for t in lst])
+        for k in ("wq", "wk", "wv"):
+            for t in student[k]:
+                assert t is None or (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous())
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_distill_grads(self._h, tokens.data_ptr(), lens, len(seq_lens), int(swift_layer), int(acrosskv_group),
+                                                  float(temperature), ptrs(student["wq"]), ptrs(student["wk"]), ptrs(student["wv"]),
+                                                  ptrs(grads["wq"]), ptrs(grads["wk"]), ptrs(grads["wv"]), loss.data_ptr(),
+                                                  ws.data_ptr(), nbytes, _stream_ptr(stream)))
+            torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+        return loss, grads
 
     def debug_bounded_wait(self, limit_clocks: int, stream: Optional[torch.cuda.Stream] = None) -> Tuple[bool, bool]:
         """swiftkv_debug_bounded_wait: (the waiting role gave up at its limit, the second role left through the abort flag)."""

@@ -12,7 +12,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libswiftkv.so")
-SOURCES = ["api.cu", "elementwise.cu", "gemm_simt.cu", "gemm_tc.cu", "attention_simple.cu", "attention_tc.cu", "tail.cu", "tail_noalloc.cu", "kv_fp8.cu", "simscore.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "gemm_simt.cu", "gemm_tc.cu", "attention_simple.cu", "attention_tc.cu", "tail.cu", "tail_noalloc.cu", "kv_fp8.cu", "simscore.cu", "distill.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math",
               "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v"]
 

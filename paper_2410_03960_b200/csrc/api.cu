@@ -991,6 +991,65 @@ extern "C" int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, con
   return SWIFTKV_OK;
 }
 
+static DistillDims distill_dims(const swiftkv_config &c) {
+  return DistillDims{c.vocab, c.hidden, c.n_layers, c.n_q_heads, c.n_kv_heads, c.head_dim, c.ffn, c.rms_eps};
+}
+extern "C" size_t swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer) {
+  if (!m || total_tokens < 1 || swift_layer < 1 || swift_layer > m->cfg.n_layers) return 0;
+  return distill_workspace_floats(distill_dims(m->cfg), total_tokens, swift_layer) * sizeof(float);
+}
+extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
+                                         int32_t l, int32_t g, float temperature, const void *const *student_wq,
+                                         const void *const *student_wk, const void *const *student_wv, void *const *grad_wq,
+                                         void *const *grad_wk, void *const *grad_wv, float *loss, void *workspace,
+                                         size_t workspace_bytes, void *cuda_stream) {
+  if (!m || !tokens || !seq_lens || !student_wq || !student_wk || !student_wv || !grad_wq || !grad_wk || !grad_wv || !loss || !workspace)
+    return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  const swiftkv_config &c = m->cfg;
+  if (c.dtype != SWIFTKV_DTYPE_F32) return fail(SWIFTKV_ERR_UNSUPPORTED, "the distillation step runs fp32 models only");
+  if (l < 1 || l > c.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c.n_layers);
+  if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
+  if (!(temperature > 0.f)) return fail(SWIFTKV_ERR_INVALID_ARG, "temperature must be positive");
+  if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255)) return fail(SWIFTKV_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+  std::vector<int32_t> cu(n_seqs + 1, 0);
+  for (int i = 0; i < n_seqs; ++i) {
+    if (seq_lens[i] < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "sequence %d: length %d < 1", i, seq_lens[i]);
+    cu[i + 1] = cu[i] + seq_lens[i];
+  }
+  const int T = cu[n_seqs];
+  if (T > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "%d tokens > max_tokens %d", T, m->max_tokens);
+  const DistillDims dims = distill_dims(c);
+  const size_t need = distill_workspace_floats(dims, T, l) * sizeof(float);
+  if (workspace_bytes < need) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "workspace %zu < %zu bytes", workspace_bytes, need);
+  std::vector<DistillLayer> layers(c.n_layers);
+  for (int j = 0; j < c.n_layers; ++j) {
+    const swiftkv_layer_weights &w = m->layers[j];
+    DistillLayer &d = layers[j];
+    d = DistillLayer{(const float *)w.in_norm, (const float *)w.wq, (const float *)w.wk, (const float *)w.wv, (const float *)w.wo,
+                     (const float *)w.post_norm, (const float *)w.w_gate, (const float *)w.w_up, (const float *)w.w_down,
+                     nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    if (j >= l) {
+      if (!student_wq[j] || !student_wk[j] || !student_wv[j] || !grad_wq[j] || !grad_wk[j] || !grad_wv[j])
+        return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d: null student weight or gradient pointer", j);
+      d.s_wq = (const float *)student_wq[j]; d.s_wk = (const float *)student_wk[j]; d.s_wv = (const float *)student_wv[j];
+      d.g_wq = (float *)grad_wq[j]; d.g_wk = (float *)grad_wk[j]; d.g_wv = (float *)grad_wv[j];
+    }
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  Buffers &b = m->b;
+  // sequence offsets to the device (a few bytes: a blocking copy keeps the host vector's lifetime out of the picture)
+  CUDA_TRY(cudaStreamSynchronize(st));
+  CUDA_TRY(cudaMemcpy(b.cu, cu.data(), (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice));
+  launch_positions(b.cu, n_seqs, b.pos, b.last_idx, T, st);
+  DistillArgs a{(const float *)m->embed, (const float *)m->final_norm, (const float *)m->lm_head, tokens, b.cu, b.pos, b.cos_tab,
+                b.sin_tab, T, n_seqs, l, g, temperature, loss, b.status, workspace, workspace_bytes / sizeof(float)};
+  const int rc = run_distill(dims, a, layers.data(), st);
+  if (rc) return fail(rc, "distillation step failed: %s", cudaGetErrorString(cudaGetLastError()));
+  m->ready = false;      // the prefill state (positions, offsets) has been overwritten
+  return SWIFTKV_OK;
+}
+
 extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out) {
   if (!m || !out) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
   if (layer < 0 || layer >= m->cfg.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, m->cfg.n_layers);

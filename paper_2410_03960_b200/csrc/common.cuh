@@ -292,6 +292,27 @@ struct TailStage {
   int N, K, ldo, epi;
 };
 bool tail_fused_supported(int rows, int d, int dq, int F, int vocab);
+
+// distill.cu : loss of Eq. 3 and its gradients with respect to the student's W_Q, W_K, W_V (fp32 models)
+struct DistillDims { int vocab, d, L, n_q, n_kv, hd, F; float eps; };
+struct DistillLayer {
+  const float *in_norm, *wq, *wk, *wv, *wo, *post_norm, *w_gate, *w_up, *w_down;   // the frozen model
+  const float *s_wq, *s_wk, *s_wv;                                                 // the student's copies (layers >= l)
+  float *g_wq, *g_wk, *g_wv;                                                       // their gradients (written)
+};
+struct DistillArgs {
+  const float *embed, *final_norm, *lm_head;
+  const int32_t *tokens, *cu, *pos;      // device: packed token ids, sequence offsets [B + 1], position of every token in its prompt
+  const float *cos_tab, *sin_tab;
+  int T, B, l, g;
+  float tau;
+  float *loss;                           // device scalar
+  unsigned int *status;
+  void *ws;
+  size_t ws_floats;
+};
+size_t distill_workspace_floats(const DistillDims &c, int T, int l);
+int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *layers, cudaStream_t st);
 // arrivals: the host's count of barrier arrivals on sync[0] so far (the counter is never reset between launches; zero both
 // together).
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,

@@ -1,0 +1,124 @@
+"""The knowledge-recovery step (Sec. 3.4, Eq. 3) through the C ABI against the oracle: distillation loss at temperature 2
+between the unmodified teacher and the re-wired student at every prompt position, and its gradients with respect to the
+student's W_Q, W_K, W_V of the layers > l (AcrossKV groups included)."""
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as S
+from oracle import distill_oracle as D
+from helpers import oracle_config, oracle_weights, to_np
+
+pytestmark = pytest.mark.gpu
+
+MID = S.ModelShape(1024, 512, 4, 8, 2, 128, 1024, 500000.0, 1e-5, "mid")
+SIX = S.ModelShape(512, 256, 6, 8, 2, 32, 688, 10000.0, 1e-5, "tiny-6-layers")
+ODD = S.ModelShape(320, 192, 5, 6, 3, 48, 400, 10000.0, 1e-5, "odd-widths")          # head_dim 48: lanes past the head are idle
+
+
+def _scaled_weights(shape, seed, scale):
+    """The benchmark's N(0, 0.02) weights leave teacher and student almost equal; larger matrices make the re-wiring matter."""
+    w = S.make_weights(shape, seed, torch.float32, "cpu")
+    for lw in w.layers:
+        for name, t in lw.items():
+            if t.ndim == 2:
+                t.mul_(scale)
+    w.embed.mul_(scale)
+    w.lm_head.mul_(scale)
+    return w
+
+
+def _student(w, l, seed, noise):
+    g = torch.Generator().manual_seed(seed)
+    L = len(w.layers)
+    return {name: [None if j < l else (w.layers[j][name] + noise * w.layers[j][name].std() * torch.randn(w.layers[j][name].shape, generator=g)).contiguous()
+                   for j in range(L)] for name in ("wq", "wk", "wv")}
+
+
+def _rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+@pytest.mark.parametrize("shape,lens,l,g,scale", [
+    (SIX, [37, 1, 20], 3, 1, 3.0),
+    (SIX, [37, 1, 20], 2, 2, 3.0),
+    (SIX, [25, 14], 1, 3, 3.0),             # groups of 3 with a short last group (layers 2-4, 5-6)
+    (ODD, [19, 30, 2], 2, 2, 3.0),
+    (MID, [40, 9], 2, 1, 2.0),
+    (MID, [130], 1, 2, 2.0),                # one prompt longer than a 128-row tile
+])
+def test_loss_and_gradients_against_oracle(shape, lens, l, g, scale):
+    import paper_2410_03960_b200 as P
+    seed, tau = 17, 2.0
+    w = _scaled_weights(shape, seed, scale)
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    st = _student(w, l, seed + 1, 0.3)
+    cfg, W = oracle_config(shape), oracle_weights(w)
+    want_loss, want = D.distill_grads(cfg, W, {k: [None if t is None else t.double().numpy() for t in v] for k, v in st.items()},
+                                      tok.numpy(), lens, l, g, tau)
+    assert want_loss > 1e-3                                          # a real difference between the two modes
+
+    wc = S.Weights(shape, torch.float32, w.embed.cuda(), w.final_norm.cuda(), w.lm_head.cuda(),
+                   [{k: v.cuda() for k, v in lw.items()} for lw in w.layers])
+    model = P.SwiftKVModel(shape, wc, torch.float32, sum(lens), len(lens), l, g)
+    st_gpu = {k: [None if t is None else t.cuda() for t in v] for k, v in st.items()}
+    loss, grads = model.distill_grads(tok, lens, l, g, tau, st_gpu)
+    model.status()
+    # fp32 arithmetic against fp64: rounding 6e-8 per operation, sums of up to a few thousand terms (x sqrt(n) ~ 50), about ten
+    # dependent stages forward and backward -> a few 1e-5 at worst; measured 3e-6
+    assert abs(float(loss) - want_loss) <= 2e-5 * want_loss, (float(loss), want_loss)
+    worst = 0.0
+    for name in ("wq", "wk", "wv"):
+        for j in range(l, shape.n_layers):
+            got, ref = to_np(grads[name][j]).astype(np.float64), want[name][j]
+            if np.abs(ref).max() == 0.0:
+                assert np.abs(got).max() == 0.0, (name, j)               # not a group leader: never read, zero gradient
+                continue
+            worst = max(worst, _rel(got, ref))
+            assert _rel(got, ref) <= 5e-5, (name, j, _rel(got, ref))
+    print(f"distill {shape.name} l={l} g={g}: loss {float(loss):.6f} (oracle {want_loss:.6f}), worst gradient rel-L2 {worst:.2e}")
+    # bit-reproducible
+    loss2, grads2 = model.distill_grads(tok, lens, l, g, tau, st_gpu)
+    assert torch.equal(loss, loss2)
+    assert all(torch.equal(a, b) for name in grads for a, b in zip(grads[name], grads2[name]) if a is not None)
+    model.close()
+
+
+def test_unrewired_student_has_no_loss_and_a_gradient_step_lowers_the_loss():
+    import paper_2410_03960_b200 as P
+    shape, lens, tau = SIX, [30, 11], 2.0
+    w = _scaled_weights(shape, 5, 3.0)
+    wc = S.Weights(shape, torch.float32, w.embed.cuda(), w.final_norm.cuda(), w.lm_head.cuda(),
+                   [{k: v.cuda() for k, v in lw.items()} for lw in w.layers])
+    tok = S.make_prompts(5, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, wc, torch.float32, sum(lens), len(lens), 1, 1)
+    # l = L - 1: the only re-wired layer reads x_{l+1} itself, so its K / V are the teacher's and the loss vanishes
+    l = shape.n_layers - 1
+    st = {name: [None if j < l else wc.layers[j][name].clone() for j in range(shape.n_layers)] for name in ("wq", "wk", "wv")}
+    loss, grads = model.distill_grads(tok, lens, l, 1, tau, st)
+    assert float(loss) <= 1e-9 and float(grads["wq"][l].abs().max()) <= 1e-6
+    # l = 2, student initialised from the original weights (Sec. 3.4): plain gradient steps recover part of the gap
+    l = 2
+    st = {name: [None if j < l else wc.layers[j][name].clone() for j in range(shape.n_layers)] for name in ("wq", "wk", "wv")}
+    loss0, grads = model.distill_grads(tok, lens, l, 1, tau, st)
+    assert float(loss0) > 1e-3
+    gnorm2 = sum(float((t.double() ** 2).sum()) for name in grads for t in grads[name] if t is not None)
+    lr = 0.1 * float(loss0) / gnorm2                                   # a step that a linear model would turn into -10 %
+    for name in st:
+        for j in range(l, shape.n_layers):
+            st[name][j] -= lr * grads[name][j]
+    loss1, _ = model.distill_grads(tok, lens, l, 1, tau, st)
+    assert float(loss1) < float(loss0) * 0.97, (float(loss0), float(loss1))
+    model.close()
+
+
+def test_argument_checks():
+    import paper_2410_03960_b200 as P
+    shape, lens = S.TINY, [8]
+    w = S.make_weights(shape, 1, torch.bfloat16, "cuda")
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, 8, 1, 2, 1)
+    st = {name: [None, None] + [w.layers[j][name].float() for j in range(2, shape.n_layers)] for name in ("wq", "wk", "wv")}
+    with pytest.raises(P.SwiftKVError) as e:
+        model.distill_grads(S.make_prompts(1, lens, shape.vocab), lens, 2, 1, 2.0, st)
+    assert e.value.code == -7          # SWIFTKV_ERR_UNSUPPORTED
+    model.close()
