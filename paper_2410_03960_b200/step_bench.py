@@ -1,7 +1,7 @@
 """Timing of the serving-style entry point (swiftkv_step) on the benchmark model: chunked prefill, decode steps,
 paged cache rows and the FP8 cache.  Prints one JSON line per measurement (CUDA events, after a warm-up pass).
 
-    python -m paper_2410_03960_b200.step_bench [--kv-format fp8] [--chunks 8192,2048,512] [--decode-steps 6] [--kernel-mask M]
+    python -m paper_2410_03960_b200.step_bench [--kv-format fp8] [--chunks 8192,2048,512] [--decode-steps 12] [--kernel-mask M]
 
 Workload: the benchmark's batch (Llama-3.1-8B shape, random bf16 weights, 8 prompts with lengths U[2048, 8192],
 seed 1, l = 16, g = 1).  A chunked prefill feeds every prompt `chunk` tokens per step (all prompts that still have
@@ -20,19 +20,20 @@ import paper_2410_03960_b200 as P                 # noqa: E402
 
 SEED, N_PROMPTS, LEN_LO, LEN_HI, SWIFT_LAYER, GROUP = 1, 8, 2048, 8192, 16, 1
 PAGES_PER_SEQ = 65
+DECODE_WARMUP = 8
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--kv-format", choices=("model", "fp8"), default="model")
     ap.add_argument("--chunks", default="8192,2048,512")
-    ap.add_argument("--decode-steps", type=int, default=6)
+    ap.add_argument("--decode-steps", type=int, default=12)
     ap.add_argument("--kernel-mask", type=int, default=None, help="swiftkv_set_kernel_mask value (default: the library's)")
     args = ap.parse_args()
     shape = S.LLAMA31_8B
     lens = S.uniform_lengths(SEED, N_PROMPTS, LEN_LO, LEN_HI)
     total, n_seq = sum(lens), len(lens)
-    extra = args.decode_steps + 2
+    extra = args.decode_steps + DECODE_WARMUP
     toks = [S.token_ids(SEED, b, n + extra, shape.vocab) for b, n in enumerate(lens)]
     w = S.make_weights(shape, SEED, torch.bfloat16, "cuda")
     fmt = P.KV_FP8 if args.kv_format == "fp8" else P.KV_MODEL_DTYPE
@@ -88,8 +89,8 @@ def main():
                            [(1, n + t, where(b, paged), 1) for b, n in enumerate(lens)], SWIFT_LAYER, GROUP)
             return t1 - t0
 
-        decode(0, 2)
-        ms, n = timed(lambda: decode(2, 2 + args.decode_steps))
+        decode(0, DECODE_WARMUP)       # (the first steps after a prefill run ~30 % slower: clocks and caches settle)
+        ms, n = timed(lambda: decode(DECODE_WARMUP, DECODE_WARMUP + args.decode_steps))
         print(json.dumps(dict(base, what="decode_step", paged=paged, batch=n_seq, context=total // n_seq,
                               ms_per_step=round(ms / n, 3), tokens_per_s=round(n_seq * n / ms * 1e3, 1))), flush=True)
 
