@@ -69,7 +69,7 @@ struct Buffers {
                             //   models use kv16)
   float *y;                 // continuing tokens' residual [B, d]
   float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
-  float *ky, *vy;           // a decode step's new K / V rows before they go to the cache, [8, d_kv] each
+  float *ky, *vy;           // a decode step's new K / V rows before they go to the cache, KV_STAGE_SLOTS x [8, d_kv] each
   float *tail_scratch;
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
@@ -137,6 +137,8 @@ static int32_t check_cfg(const swiftkv_config *c, int max_tokens, int max_seqs, 
 
 // persistent attention kernel: at most this many CTAs; one item per (128-query tile, pair of query heads)
 constexpr int ATT_MAX_CTAS = 1024;
+// staging rows for the K / V projections of a decode step: this many AcrossKV groups' rows per fused launch
+constexpr int KV_STAGE_SLOTS = 6;
 static size_t att_max_items(const swiftkv_config &c, int T, int B) {
   return ((size_t)T / 128 + (size_t)B) * (size_t)((c.n_q_heads + 1) / 2);
 }
@@ -167,8 +169,8 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.qy = (float *)cv.take(R * dq * 4);
   b.ay = (float *)cv.take(R * dq * 4);
   b.acty = (float *)cv.take(R * F * 4);
-  b.ky = (float *)cv.take(R * dkv_ * 4);
-  b.vy = (float *)cv.take(R * dkv_ * 4);
+  b.ky = (float *)cv.take(KV_STAGE_SLOTS * R * dkv_ * 4);      // (several AcrossKV groups' rows per fused launch)
+  b.vy = (float *)cv.take(KV_STAGE_SLOTS * R * dkv_ * 4);
   b.tail_scratch = (float *)cv.take(tail_attention_scratch_bytes(B, c.n_q_heads, c.head_dim, T));
   b.logits = (float *)cv.take((size_t)B * c.vocab * 4);
   b.tokens = (int32_t *)cv.take((size_t)T * 4);
@@ -487,6 +489,27 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     m->fold_l = l; m->fold_g = g; m->fold_fmt = fold_fmt;
   }
 
+  // kernel-mask bit 6: the dependent projections between two attention calls of the last-token / decode path -- O, gate/up,
+  // down and the next layer's Q (and K / V of a decode token), or the lm_head at the end -- run as ONE persistent cooperative
+  // launch with the norms folded in
+  bool fused_tail = false;
+  if constexpr (sizeof(T) == 2) {
+    fused_tail = (m->kernel_mask & 64) && bt.n_emit > 0 && dkv % 16 == 0 &&
+                 tail_fused_supported(std::min(MAX_TAIL_ROWS, bt.n_emit), d, dq, F, c.vocab);
+  }
+  unsigned int fused_arrivals = 0;
+  if (fused_tail && cudaMemsetAsync(b.status + 32, 0, 32 * sizeof(unsigned int), st) != cudaSuccess)
+    return fail(SWIFTKV_ERR_CUDA, "clearing the grid-barrier words failed");
+  TailStage list[6];
+  int n_list = 0;
+  auto flush = [&](int rows) -> int32_t {
+    if (n_list == 0) return SWIFTKV_OK;
+    Scope s(m, st, SWIFTKV_KC_TAIL);
+    const int frc = launch_tail_fused(list, n_list, rows, c.rms_eps, b.status + 32, &fused_arrivals, b.status, st);
+    n_list = 0;
+    return frc == SWIFTKV_OK ? SWIFTKV_OK : fail(frc, "fused last-token launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  };
+
   // ---- a minibatch of decode tokens (Sec. 3.5: "decode tokens complete all layers"): at most 8 rows, so every
   //      projection is bound by streaming its weights once -- layers 1..l run on the last-token path's kernels too,
   //      the new K / V rows go to the cache before the single-query attention reads it, and the rows of the later
@@ -495,7 +518,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     const int rows = T_tok;
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
     const TailOpts q_rope{b.last_pos, b.cos_tab, b.sin_tab, bt.total_kv};     // the queries are rotated inside the attention kernel
-    auto store_kv = [&](int slot) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
+    auto store_kv = [&](int slot, float *ky, float *vy) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
       if (fp8) {
         Scope s(m, st, SWIFTKV_KC_TAIL, 5);
         launch_rope<float>(ky, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st);
@@ -517,10 +540,16 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     { Scope s(m, st, SWIFTKV_KC_TAIL); launch_gather_rows(b.x, b.last_idx, y, rows, d, st); }
     for (int j = 0; j < l; ++j) {
       const swiftkv_layer_weights &lw = m->layers[j];
+      if (fused_tail) {      // [O, gate/up, down of the previous layer,] Q, K / V of this one: one launch
+        list[n_list++] = TailStage{y, lw.in_norm, lw.wq, nullptr, qy, dq, d, dq, 0};
+        list[n_list++] = TailStage{y, lw.in_norm, lw.wk, lw.wv, ky, dkv, d, dkv, 3, vy};
+        if ((rc = flush(rows))) return rc;
+      } else {
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.wq, nullptr, rows, dq, d, qy, dq, OUT_STORE_F32, st); }
       project_kv(lw);
-      store_kv(j);
+      }
+      store_kv(j, ky, vy);
       {
         Scope s(m, st, SWIFTKV_KC_TAIL, 2);
         if (fp8)
@@ -532,16 +561,38 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
                                    b.emit_len, blk_emit, bt.blk_stride, rows, max_len, c.n_q_heads, c.n_kv_heads, c.head_dim,
                                    b.tail_scratch, st, q_rope);
       }
+      if (fused_tail) {      // (launched with the next layer's Q / K / V, or with the first SingleInputKV rows below)
+        list[n_list++] = TailStage{ay, nullptr, lw.wo, nullptr, y, d, dq, d, 1};
+        list[n_list++] = TailStage{y, lw.post_norm, lw.w_gate, lw.w_up, acty, F, d, F, 2};
+        list[n_list++] = TailStage{acty, nullptr, lw.w_down, nullptr, y, d, F, d, 1};
+        continue;
+      }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(ay, (const T *)lw.wo, nullptr, rows, d, dq, y, d, OUT_RESID_ADD_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.post_norm, hy, rows, d, c.rms_eps, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(hy, (const T *)lw.w_gate, (const T *)lw.w_up, rows, F, d, acty, F, OUT_STORE_F32, st); }
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_skinny_gemm<T>(acty, (const T *)lw.w_down, nullptr, rows, d, F, y, d, OUT_RESID_ADD_F32, st); }
     }
+    if (fused_tail) {
+      // SingleInputKV rows of the new tokens (Eq. 2, unfused: each group leader's own gain and W_K, W_V on the layer-l output):
+      // as many groups per launch as the stage list and the staging rows hold, then their cache stores
+      int first = 0;
+      for (int i = 0; i < ng && l < L; ++i) {
+        const swiftkv_layer_weights &lw = m->layers[l + i * g];
+        const int k_slot = i - first;
+        list[n_list++] = TailStage{y, lw.in_norm, lw.wk, lw.wv, ky + (size_t)k_slot * rows * dkv, dkv, d, dkv, 3, vy + (size_t)k_slot * rows * dkv};
+        if (n_list == 6 || k_slot + 1 == KV_STAGE_SLOTS || i + 1 == ng) {
+          if ((rc = flush(rows))) return rc;
+          for (int q = first; q <= i; ++q) store_kv(l + q, ky + (size_t)(q - first) * rows * dkv, vy + (size_t)(q - first) * rows * dkv);
+          first = i + 1;
+        }
+      }
+      if ((rc = flush(rows))) return rc;      // (l == L: the last layer's O / gate-up / down are still pending)
+    } else
     for (int i = 0; i < ng && l < L; ++i) {      // SingleInputKV rows of the new tokens, one AcrossKV group at a time
       const swiftkv_layer_weights &lw = m->layers[l + i * g];
       { Scope s(m, st, SWIFTKV_KC_TAIL); launch_tail_rmsnorm<T>(y, (const T *)lw.in_norm, hy, rows, d, c.rms_eps, st); }
       project_kv(lw);
-      store_kv(l + i);
+      store_kv(l + i, ky, vy);
     }
   }
 
@@ -716,15 +767,6 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
 
   // ---- the tokens that must produce output -- the last token of a prompt (footnote of Sec. 3.2), decode tokens
   //      (Sec. 3.5) -- continue through layers l+1..L
-  // kernel-mask bit 6: the dependent projections between two attention calls -- O, gate/up, down and the next layer's Q, or
-  // the lm_head at the end -- run as ONE persistent cooperative launch with the norms folded in
-  bool fused_tail = false;
-  if constexpr (sizeof(T) == 2) {
-    fused_tail = (m->kernel_mask & 64) && bt.n_emit > 0 && tail_fused_supported(std::min(MAX_TAIL_ROWS, bt.n_emit), d, dq, F, c.vocab);
-  }
-  unsigned int fused_arrivals = 0;
-  if (fused_tail && cudaMemsetAsync(b.status + 32, 0, 32 * sizeof(unsigned int), st) != cudaSuccess)
-    return fail(SWIFTKV_ERR_CUDA, "clearing the grid-barrier words failed");
   for (int r0 = 0; r0 < bt.n_emit; r0 += MAX_TAIL_ROWS) {
     const int rows = std::min(MAX_TAIL_ROWS, bt.n_emit - r0);
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty;
@@ -746,19 +788,10 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
                                  c.head_dim, b.tail_scratch, st, q_rope);
     };
     if (fused_tail) {
-      TailStage list[6];
-      int n_list = 0;
-      auto flush = [&]() -> int32_t {
-        if (n_list == 0) return SWIFTKV_OK;
-        Scope s(m, st, SWIFTKV_KC_TAIL);
-        const int frc = launch_tail_fused(list, n_list, rows, c.rms_eps, b.status + 32, &fused_arrivals, b.status, st);
-        n_list = 0;
-        return frc == SWIFTKV_OK ? SWIFTKV_OK : fail(frc, "fused last-token launch failed: %s", cudaGetErrorString(cudaGetLastError()));
-      };
       for (int j = l; j < L; ++j) {
         const swiftkv_layer_weights &lw = m->layers[j];
         list[n_list++] = TailStage{y, lw.in_norm, lw.wq, nullptr, qy, dq, d, dq, 0};
-        if ((rc = flush())) return rc;
+        if ((rc = flush(rows))) return rc;
         attention(l + (j - l) / g);
         list[n_list++] = TailStage{ay, nullptr, lw.wo, nullptr, y, d, dq, d, 1};
         list[n_list++] = TailStage{y, lw.post_norm, lw.w_gate, lw.w_up, acty, F, d, F, 2};
@@ -766,7 +799,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
         if (j + 1 == L) list[n_list++] = TailStage{y, m->final_norm, m->lm_head, nullptr, b.logits + (size_t)r0 * c.vocab, c.vocab, d, c.vocab, 0};
       }
       if (l == L) list[n_list++] = TailStage{y, m->final_norm, m->lm_head, nullptr, b.logits + (size_t)r0 * c.vocab, c.vocab, d, c.vocab, 0};
-      if ((rc = flush())) return rc;
+      if ((rc = flush(rows))) return rc;
       continue;
     }
     for (int j = l; j < L; ++j) {

@@ -283,13 +283,14 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
 
 // Several dependent projections of the last-token path (at most 6) as one persistent cooperative launch with grid-wide
 // barriers between them (bf16 weights).  Stage: out (+)= A W^T with A [rows, K] fp32, W [N, K]; epi 0 store, 1 accumulate
-// into out, 2 out = silu(A W^T) * (A W2^T); gamma != null: A is RMS-normalised on the fly (the norm that precedes the
+// into out, 2 out = silu(A W^T) * (A W2^T), 3 out = A W^T and out2 = A W2^T; gamma != null: A is RMS-normalised on the fly (the norm that precedes the
 // projection is folded in).  sync: two words of device scratch; status: the model's status word.
 struct TailStage {
   const float *A;
   const void *gamma, *W, *W2;
   float *out;
   int N, K, ldo, epi;
+  float *out2 = nullptr;     // epi 3 (two projections of the same input, e.g. K and V of a decode token): W2's result
 };
 bool tail_fused_supported(int rows, int d, int dq, int F, int vocab);
 

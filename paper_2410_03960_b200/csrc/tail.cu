@@ -7,6 +7,8 @@
 #include <cooperative_groups.h>
 #include <mma.h>
 
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_common.cuh"
 
@@ -392,7 +394,9 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
   extern __shared__ __align__(16) uint8_t ta_smem[];
   float (*qs)[HD] = reinterpret_cast<float (*)[HD]>(ta_smem);                 // [REP][HD]
   uint8_t *tiles = ta_smem + REP * HD * sizeof(float);
-  const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+  // (the KV heads of one key range are neighbours in the grid: their blocks run at the same time and together read whole
+  //  cache rows -- all heads of a token are contiguous -- instead of one 256-byte piece per 2 KB row each at its own time)
+  const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   uint8_t *kt = tiles + warp * (TT::K_BYTES + TT::V_BYTES), *vt = kt + TT::K_BYTES;
   const int first = cu[b], n = len ? len[b] : cu[b + 1] - cu[b];
@@ -533,6 +537,186 @@ __global__ void __launch_bounds__(TA_WARPS * 32) tail_attention_group_kernel(
   }
 }
 
+// The same block / warp / tile structure with the arithmetic on the tensor cores (bf16 cache, head_dim 128, <= 8 query heads
+// per KV head): the scalar form above spends ~1400 issue slots per 32-key tile and is bound by the latency of its FMA chains
+// at the occupancy its shared memory allows; here a tile is 64 + 64 mma.sync.m16n8k16 plus ~100 loads.
+//   scores : S[head, key] = Q K^T with the group's query rows as the A operand (rows >= REP are zero; fp32 queries as bf16
+//            hi + lo, so the products carry ~16 significant bits of q against the exact bf16 keys), K rows straight from
+//            the padded tile as the B operand;
+//   softmax: a lane holds 8 scores of one head (row g = lane / 4), quad reductions give the row maximum and sum;
+//   output : O[head, dim] += P V with the probabilities (bf16 hi + lo) re-used from the score accumulators as the A operand
+//            and V read through ldmatrix.trans from a padded tile.
+constexpr int TM_VSTRIDE = 256 + 16;
+constexpr int TM_TILE_BYTES = 32 * (256 + 16) + 32 * TM_VSTRIDE;
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, const void *p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+}
+template <int REP>
+__global__ void __launch_bounds__(TA_WARPS * 32, 3) tail_attention_mma_kernel(
+    const float *__restrict__ q, const bf16 *__restrict__ kc, const bf16 *__restrict__ vc, const int32_t *__restrict__ cu,
+    const int32_t *__restrict__ len, const int32_t *__restrict__ blk, int blk_stride, int n_q, int n_kv, int chunk, int n_splits,
+    float scale, float *__restrict__ scratch, TailOpts rope) {
+  constexpr int HD = 128, KSTRIDE = 256 + 16;
+  extern __shared__ __align__(16) uint8_t ta_smem[];
+  float (*qs)[HD] = reinterpret_cast<float (*)[HD]>(ta_smem);                 // [REP][HD]
+  uint8_t *tiles = ta_smem + REP * HD * sizeof(float);
+  const int kvh = blockIdx.x, split = blockIdx.y, b = blockIdx.z;      // (KV heads fastest: see tail_attention_group_kernel)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  uint8_t *kt = tiles + warp * TM_TILE_BYTES, *vt = kt + 32 * KSTRIDE;
+  const int first = cu[b], n = len ? len[b] : cu[b + 1] - cu[b];
+  const int k_begin = split * chunk, k_end = min(n, k_begin + chunk);
+  if (k_begin >= k_end) {             // a split past the sequence's end: an empty partial for the merge pass
+    if (threadIdx.x < REP) {
+      float *dst = scratch + (((size_t)b * n_q + kvh * REP + threadIdx.x) * n_splits + split) * (HD + 2);
+      dst[0] = -INFINITY;
+      dst[1] = 0.f;
+    }
+    return;
+  }
+  for (int i = threadIdx.x; i < REP * HD; i += blockDim.x)
+    qs[i / HD][i % HD] = load_query(q + ((size_t)b * n_q + kvh * REP + i / HD) * HD, i % HD, HD, b, rope) * scale;
+
+  auto issue_tile = [&](const bf16 *base, uint8_t *tile, int c0) {      // rows [c0, c0 + 32) of this KV head; 16 lanes copy one row
+    const int sub = lane & 15;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int r = i * 2 + (lane >> 4), key = c0 + r;
+      if (key < k_end)
+        cp_async16(tile + r * KSTRIDE + sub * 16,
+                   reinterpret_cast<const uint8_t *>(base + (kv_row_of(blk, blk_stride, b, first, key) * n_kv + kvh) * HD) + sub * 16);
+      else
+        *reinterpret_cast<uint4 *>(tile + r * KSTRIDE + sub * 16) = make_uint4(0u, 0u, 0u, 0u);      // (keeps NaN bit patterns out of P V)
+    }
+    cp_async_commit();
+  };
+  int c0 = k_begin + warp * 32;
+  if (c0 < k_end) { issue_tile(kc, kt, c0); issue_tile(vc, vt, c0); }
+  __syncthreads();                    // qs
+
+  // the group's queries as A fragments (row g of the 16 x 16 tile; rows 8..15 and rows >= REP are zero)
+  uint32_t qh[8][2], ql[8][2];
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
+    if (g < REP) {
+      x0 = qs[g][kk * 16 + 2 * t]; x1 = qs[g][kk * 16 + 2 * t + 1];
+      x2 = qs[g][kk * 16 + 8 + 2 * t]; x3 = qs[g][kk * 16 + 8 + 2 * t + 1];
+    }
+    split_hi_lo(x0, x1, qh[kk][0], ql[kk][0]);
+    split_hi_lo(x2, x3, qh[kk][1], ql[kk][1]);
+  }
+  float m = -INFINITY, l = 0.f;       // of head g (the four lanes of a quad hold the same values)
+  float acc[16][4];
+#pragma unroll
+  for (int nd = 0; nd < 16; ++nd) acc[nd][0] = acc[nd][1] = acc[nd][2] = acc[nd][3] = 0.f;
+
+  for (; c0 < k_end; c0 += TA_WARPS * 32) {
+    const int next = c0 + TA_WARPS * 32;
+    const bool more = next < k_end;
+    cp_async_wait<1>();               // pending groups: K(c0), V(c0) -> K(c0) has landed
+    __syncwarp();
+    float sc[4][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+      // one ldmatrix brings the B fragments of two 16-dim steps: 8 key rows x (4 x 16 bytes)
+      const uint8_t *kr = kt + (nt * 8 + (lane & 7)) * KSTRIDE + (lane >> 3) * 16;
+#pragma unroll
+      for (int kp = 0; kp < 4; ++kp) {
+        uint32_t b[4];
+        ldmatrix_x4(b[0], b[1], b[2], b[3], kr + kp * 64);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int kk = 2 * kp + h;
+          const uint32_t ah[4] = {qh[kk][0], 0u, qh[kk][1], 0u}, al[4] = {ql[kk][0], 0u, ql[kk][1], 0u};
+          mma_bf16_16816(sc[nt], ah, b[2 * h], b[2 * h + 1]);
+          mma_bf16_16816(sc[nt], al, b[2 * h], b[2 * h + 1]);
+        }
+      }
+    }
+    __syncwarp();                     // every lane is done with the K tile
+    if (more) issue_tile(kc, kt, next);
+    // online softmax of head g over the tile's 32 keys: this lane holds keys nt * 8 + 2 t, + 1
+    float mx = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      if (c0 + nt * 8 + 2 * t >= k_end) sc[nt][0] = -INFINITY;
+      if (c0 + nt * 8 + 2 * t + 1 >= k_end) sc[nt][1] = -INFINITY;
+      mx = fmaxf(mx, fmaxf(sc[nt][0], sc[nt][1]));
+    }
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float m_new = fmaxf(m, mx);
+    const float corr = __expf(m - m_new);
+    float sum = 0.f;
+    uint32_t ph[4], pl[4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const float p0 = __expf(sc[nt][0] - m_new), p1 = __expf(sc[nt][1] - m_new);
+      sum += p0 + p1;
+      split_hi_lo(p0, p1, ph[nt], pl[nt]);
+    }
+    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+    l = l * corr + sum;
+    m = m_new;
+#pragma unroll
+    for (int nd = 0; nd < 16; ++nd) { acc[nd][0] *= corr; acc[nd][1] *= corr; }
+    if (more) cp_async_wait<1>(); else cp_async_wait<0>();     // pending: V(c0) [, K(next)] -> V(c0) has landed
+    __syncwarp();
+    // P V: keys in two steps of 16; ldmatrix.trans brings, per instruction, both key halves of two 8-dim column blocks
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks) {
+      const uint32_t ah[4] = {ph[2 * ks], 0u, ph[2 * ks + 1], 0u}, al[4] = {pl[2 * ks], 0u, pl[2 * ks + 1], 0u};
+      const uint8_t *vrow = vt + (ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * TM_VSTRIDE + (lane >> 4) * 16;
+#pragma unroll
+      for (int np = 0; np < 8; ++np) {
+        uint32_t b00, b01, b10, b11;
+        ldmatrix_x4_trans(b00, b01, b10, b11, vrow + np * 32);
+        mma_bf16_16816(acc[2 * np], ah, b00, b01);
+        mma_bf16_16816(acc[2 * np], al, b00, b01);
+        mma_bf16_16816(acc[2 * np + 1], ah, b10, b11);
+        mma_bf16_16816(acc[2 * np + 1], al, b10, b11);
+      }
+    }
+    __syncwarp();                     // every lane is done with the V tile
+    if (more) issue_tile(vc, vt, next);
+  }
+  // merge the warps; the tiles are free now (every copy has landed and been consumed)
+  __syncthreads();
+  float *w_m = reinterpret_cast<float *>(tiles);                 // [TA_WARPS][REP]
+  float *w_l = w_m + TA_WARPS * REP;                             // [TA_WARPS][REP]
+  float *w_acc = w_l + TA_WARPS * REP;                           // [TA_WARPS][REP][HD]
+  if (g < REP) {
+    if (t == 0) { w_m[warp * REP + g] = m; w_l[warp * REP + g] = l; }
+#pragma unroll
+    for (int nd = 0; nd < 16; ++nd)
+      *reinterpret_cast<float2 *>(&w_acc[(warp * REP + g) * HD + nd * 8 + 2 * t]) = make_float2(acc[nd][0], acc[nd][1]);
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < REP * HD; idx += blockDim.x) {
+    const int r = idx / HD, dd = idx % HD;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < TA_WARPS; ++w) M = fmaxf(M, w_m[w * REP + r]);
+    float a = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < TA_WARPS; ++w) {
+      const float f = (w_m[w * REP + r] == -INFINITY) ? 0.f : __expf(w_m[w * REP + r] - M);
+      a += w_acc[(w * REP + r) * HD + dd] * f;
+      L += w_l[w * REP + r] * f;
+    }
+    float *dst = scratch + (((size_t)b * n_q + kvh * REP + r) * n_splits + split) * (HD + 2);
+    if (dd == 0) { dst[0] = M; dst[1] = L; }
+    dst[2 + dd] = a;
+  }
+}
+
 // Shape-generic form: block (split, KV head, prompt); warp w = query head kvh*rep + w of that KV head's group, so the
 // K / V rows of the block's key range come from HBM once and are shared by the group's heads through L1.
 template <typename T, int MAX_E>
@@ -648,6 +832,13 @@ size_t tail_attention_scratch_bytes(int max_seqs, int n_q, int hd, int max_token
   return (size_t)rows * n_q * tail_max_splits(max_tokens) * (hd + 2) * sizeof(float);
 }
 
+// (SWIFTKV_TAIL_ATTENTION_SCALAR=1 keeps the scalar kernel: A/B and debugging)
+static bool tail_attention_use_mma() {
+  static int v = -1;
+  if (v < 0) { const char *e = getenv("SWIFTKV_TAIL_ATTENTION_SCALAR"); v = (e && e[0] == '1') ? 0 : 1; }
+  return v == 1;
+}
+
 template <typename T>
 void launch_tail_attention(const float *q, const T *kc, const T *vc, const float *kscale, const float *vscale, float *out,
                            const int32_t *cu_seqlens, const int32_t *len, const int32_t *blk, int blk_stride, int n_seqs,
@@ -670,8 +861,28 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
   const int n_splits = (max_seq_len + chunk - 1) / chunk;
   const float scale = 1.0f / sqrtf((float)hd);
   const int rep = n_q / n_kv;
+  if constexpr (sizeof(T) == 2) {
+    if (hd == 128 && !kscale && (rep == 1 || rep == 2 || rep == 4 || rep == 8) && tail_attention_use_mma()) {
+      dim3 grid(n_kv, n_splits, n_seqs);
+      const size_t smem = (size_t)rep * 128 * sizeof(float) + (size_t)TA_WARPS * TM_TILE_BYTES;
+#define SKV_LAUNCH_MMA(R)                                                                                                     \
+      do {                                                                                                                    \
+        ensure_dynamic_smem(reinterpret_cast<const void *>(tail_attention_mma_kernel<R>), (int)smem);                         \
+        tail_attention_mma_kernel<R><<<grid, TA_WARPS * 32, smem, st>>>(q, reinterpret_cast<const bf16 *>(kc),                \
+                                                                        reinterpret_cast<const bf16 *>(vc), cu_seqlens, len, blk, \
+                                                                        blk_stride, n_q, n_kv, chunk, n_splits, scale, scratch, rope); \
+      } while (0)
+      if (rep == 1) SKV_LAUNCH_MMA(1);
+      else if (rep == 2) SKV_LAUNCH_MMA(2);
+      else if (rep == 4) SKV_LAUNCH_MMA(4);
+      else SKV_LAUNCH_MMA(8);
+#undef SKV_LAUNCH_MMA
+      tail_attention_merge_kernel<<<dim3(n_q, n_seqs), 128, 0, st>>>(scratch, out, n_q, hd, n_splits);
+      return;
+    }
+  }
   if (hd == 128 && (rep == 1 || rep == 2 || rep == 4 || rep == 8)) {
-    dim3 grid(n_splits, n_kv, n_seqs);
+    dim3 grid(n_kv, n_splits, n_seqs);
     const size_t smem = (size_t)rep * 128 * sizeof(float) + (size_t)TA_WARPS * (TailTile<T>::K_BYTES + TailTile<T>::V_BYTES);
 #define SKV_LAUNCH_GROUP(R)                                                                                                   \
     do {                                                                                                                      \
@@ -770,13 +981,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // data written with ordinary stores (by any SM, made visible by a barrier) is about to be read by a bulk copy
 __device__ __forceinline__ void fence_generic_to_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// epi 0: out = A W^T (store); 1: out += A W^T; 2: out = silu(A W^T) * (A W2^T)
+// epi 0: out = A W^T (store); 1: out += A W^T; 2: out = silu(A W^T) * (A W2^T); 3: out = A W^T and out2 = A W2^T
 struct Stage {
   CUtensorMap tmW, tmW2;   // [N, K] as [K / 64][N][64], box (64, 16, KC / 64)
   CUtensorMap tmA;         // [rows, K] fp32 as [K / 32][rows][32], box (32, row slots, KC / 32)
   const float *A;          // [rows, K] fp32 (produced earlier, possibly in this launch)
   const bf16 *gamma;       // non-null: A is RMS-normalised on the fly (row statistic * gain)
-  float *out;
+  float *out, *out2;
   int N, K, ldo, epi;
 };
 struct Params {
@@ -851,7 +1062,7 @@ __device__ void produce(const Params &p, Ctx &c) {
   if ((threadIdx.x & 31) != 0) return;
   for (int i = 0; i < p.n_stages; ++i) {
     const Stage &sg = p.st[i];
-    const bool dual = sg.epi == 2;
+    const bool dual = sg.epi >= 2;
     const int kc_len = dual ? KC2 : KC1;
     const int n_tiles = sg.N / 16, n_chunks = sg.K / kc_len;
     const bool resident = (long long)sg.K * 32 <= RES_BYTES;
@@ -1112,7 +1323,10 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
         if (r < p.rows) {
           const float rs = sg.gamma ? rstd_s[r] : 1.f;       // the folded norm's row statistic
           float v = s1[i] * rs;
-          if (DUAL) v = v / (1.f + __expf(-v)) * (s2[i] * rs);
+          if (DUAL) {
+            if (sg.epi == 2) v = v / (1.f + __expf(-v)) * (s2[i] * rs);
+            else sg.out2[(size_t)r * sg.ldo + n] = s2[i] * rs;
+          }
           float *o = sg.out + (size_t)r * sg.ldo + n;
           if (sg.epi == 1) v += __ldcg(o);
           *o = v;
@@ -1160,7 +1374,7 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
       }
       const Stage &sg = p.st[i];
       const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
-      if (sg.epi == 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
+      if (sg.epi >= 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
       else { if (resident) consume<false, true>(p, c, sg); else consume<false, false>(p, c, sg); }
       if (*c.abort_s) break;
     }
@@ -1195,14 +1409,14 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
   for (int i = 0; i < n_stages; ++i) {
     const TailStage &s = stages[i];
     const int kc = s.W2 ? fused::KC2 : fused::KC1;
-    if (s.N % 16 || s.K % kc || (s.W2 != nullptr) != (s.epi == 2)) return SWIFTKV_ERR_UNSUPPORTED;
+    if (s.N % 16 || s.K % kc || (s.W2 != nullptr) != (s.epi >= 2) || (s.epi == 3 && !s.out2)) return SWIFTKV_ERR_UNSUPPORTED;
     fused::Stage &d = p.st[i];
     if (get_tmap_rows16(&d.tmW, s.W, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
     d.tmW2 = d.tmW;
     if (s.W2 && get_tmap_rows16(&d.tmW2, s.W2, s.N, s.K, kc / 64)) return SWIFTKV_ERR_CUDA;
     const bool resident = (long long)s.K * 32 <= fused::RES_BYTES;
     if (get_tmap_act_f32(&d.tmA, s.A, rows, 1u << rs, s.K, resident ? fused::KC1 / 32 : kc / 32)) return SWIFTKV_ERR_CUDA;
-    d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
+    d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.out2 = s.out2; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
   }
   p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
   p.sync_base = *arrivals;
