@@ -363,7 +363,7 @@ def run_ours(args, rank, world, local_rank):
                               "frac_of_measured_sustained": f_sw["total"] / (t_bf16 / args.steps) / 1e12 / peak,
                               "note": "swiftkv_set_activation_format(SWIFTKV_ACT_BF16): every MMA operand bfloat16; meets the "
                                       "2e-2 / 0.1 parity bars on models of a few layers only (rounding 2^-9 per stored "
-                                      "activation), see DESIGN.md"},
+                                      "activation)"},
             "e2e": {"value": tokens_all / t_e2e, "unit": "tokens/s", "h2d_bytes_per_step": T * 4 + (N_PROMPTS + 1) * 4 + N_PROMPTS * 4,
                     "d2h_bytes_per_step": N_PROMPTS * SHAPE.vocab * 4},
             "gpu_launches": launches,

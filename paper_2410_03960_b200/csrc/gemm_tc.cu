@@ -778,7 +778,7 @@ bool tc_gemm_supported(int M, int N, int K) { return M >= 1 && K >= 64 && (K % 6
 bool tc_swiglu_supported(int M, int F, int K) { return M >= 1 && K >= 64 && (K % 64) == 0 && (F % 128) == 0 && F >= 128; }
 
 // Raster band height in 128-row blocks.  A band's A rows (band x K x 2 bytes) are re-walked for every column block, so they
-// must stay in L2 next to the streaming weights and output: 4096 rows for K <= 8192, 2048 rows for longer K.
+// must stay in L2 next to the streaming weights and output: 4096 rows for K <= 4096 (33 MB of A), 2048 rows for longer K.
 static int group_m_setting(int K) {
   static int v = 0, v_long = 0;
   if (!v) {
@@ -788,7 +788,7 @@ static int group_m_setting(int K) {
     v = e ? atoi(e) : 32;
     if (v < 1) v = 32;
   }
-  return K > 8192 ? v_long : v;
+  return K > 4096 ? v_long : v;
 }
 static bool g_use_pairs = true, g_swiglu_pairs = false;
 void tc_gemm_use_cta_pairs(bool on, bool swiglu_too) { g_use_pairs = on; g_swiglu_pairs = swiglu_too; }
