@@ -517,7 +517,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   if (bt.decode) {
     const int rows = T_tok;
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
-    const TailOpts q_rope{b.last_pos, b.cos_tab, b.sin_tab, bt.total_kv, bt.emit_lens.data()};     // the queries are rotated inside the attention kernel
+    const TailOpts q_rope{b.last_pos, b.cos_tab, b.sin_tab, bt.total_kv};     // the queries are rotated inside the attention kernel
     auto store_kv = [&](int slot, float *ky, float *vy) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
       if (fp8) {
         Scope s(m, st, SWIFTKV_KC_TAIL, 5);
@@ -775,7 +775,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     const int32_t *be = blk_emit ? blk_emit + (size_t)r0 * bt.blk_stride : nullptr;
     int emit_kv = 0;
     for (int r = r0; r < r0 + rows; ++r) emit_kv += bt.emit_lens[r];
-    const TailOpts q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab, emit_kv, bt.emit_lens.data() + r0};    // the queries are rotated inside the attention kernel
+    const TailOpts q_rope{b.last_pos + r0, b.cos_tab, b.sin_tab, emit_kv};    // the queries are rotated inside the attention kernel
     auto attention = [&](int slot) {
       Scope s(m, st, SWIFTKV_KC_TAIL, 2);
       if (fp8)

@@ -269,7 +269,6 @@ struct TailOpts {
   const int32_t *pos = nullptr;
   const float *cos_tab = nullptr, *sin_tab = nullptr;
   int total_len = 0;
-  const int *host_lens = nullptr;     // HOST copy of the sequences' key counts (optional): the key split is then chosen from exact block counts
 };
 // one query token per sequence against that sequence's cache rows [row0[b], row0[b] + len[b]); len == nullptr means
 // row0 is a cu_seqlens array (len[b] = row0[b+1] - row0[b]); scratch holds split partials

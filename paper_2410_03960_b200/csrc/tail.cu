@@ -853,12 +853,7 @@ void launch_tail_attention(const float *q, const T *kc, const T *vc, const float
     const double cap = 3.0 * n_sms;
     double best = 1e300;
     for (int c = chunk; c <= ((max_seq_len + 127) / 128) * 128 && c < chunk + 4096; c += 128) {
-      double blocks = ((double)rope.total_len / c + 0.5 * n_seqs) * n_kv;
-      if (rope.host_lens) {      // exact: a block past its sequence's end leaves at once and does not count
-        long long nb = 0;
-        for (int b = 0; b < n_seqs; ++b) nb += (rope.host_lens[b] + c - 1) / c;
-        blocks = (double)nb * n_kv;
-      }
+      const double blocks = ((double)rope.total_len / c + 0.5 * n_seqs) * n_kv;
       const double cost = ceil(blocks / cap) * (c + 64);
       if (cost <= best) { best = cost; chunk = c; }
     }
