@@ -219,11 +219,13 @@ int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t 
  *   grad_w*     : HOST arrays [n_layers] of DEVICE pointers, fp32, same shapes, WRITTEN (not accumulated)
  *   loss        : DEVICE fp32 scalar, written
  *   workspace   : DEVICE, caller-owned, 256-byte aligned, >= swiftkv_distill_workspace_bytes(m, total tokens, swift_layer)
- * fp32 models only (SWIFTKV_ERR_UNSUPPORTED otherwise): the step runs in fp32 on the CUDA cores; gradients repeat bit for
- * bit (every output element is summed by one block in a fixed order).  The model's prefill state (swiftkv_kv_cache_view,
+ * The step runs in fp32 on the CUDA cores whatever the model's dtype: a bf16 model's frozen weights are widened into fp32
+ * copies inside `workspace` first (its size accounts for them: 4 bytes per model parameter), the student's matrices and
+ * the gradients are fp32 either way (master weights).  Gradients repeat bit for bit (every output element is summed by one
+ * block in a fixed order).  The model's prefill state (swiftkv_kv_cache_view,
  * swiftkv_first_logits) is invalid afterwards until the next prefill.  The sequence offsets are copied with a blocking
  * copy after synchronising `cuda_stream`; everything else is queued on it.
- * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_SMALL, CUDA.
+ * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA.
  */
 size_t  swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer);
 int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,

@@ -1027,9 +1027,18 @@ extern "C" int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, con
 static DistillDims distill_dims(const swiftkv_config &c) {
   return DistillDims{c.vocab, c.hidden, c.n_layers, c.n_q_heads, c.n_kv_heads, c.head_dim, c.ffn, c.rms_eps};
 }
+// fp32 copies of a bf16 model's frozen weights (the step computes in fp32): floats per layer / for embedding, final norm, lm_head
+static size_t distill_layer_weight_floats(const swiftkv_config &c) {
+  const size_t d = c.hidden, dq = (size_t)c.n_q_heads * c.head_dim, dkv = (size_t)c.n_kv_heads * c.head_dim, F = c.ffn;
+  return 2 * d + 2 * dq * d + 2 * dkv * d + 3 * F * d + 9 * 4;
+}
+static size_t distill_weight_floats(const swiftkv_config &c) {
+  if (c.dtype != SWIFTKV_DTYPE_BF16) return 0;
+  return (size_t)c.n_layers * distill_layer_weight_floats(c) + 2 * (size_t)c.vocab * c.hidden + c.hidden + 3 * 4;
+}
 extern "C" size_t swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer) {
   if (!m || total_tokens < 1 || swift_layer < 1 || swift_layer > m->cfg.n_layers) return 0;
-  return distill_workspace_floats(distill_dims(m->cfg), total_tokens, swift_layer) * sizeof(float);
+  return (distill_workspace_floats(distill_dims(m->cfg), total_tokens, swift_layer) + distill_weight_floats(m->cfg)) * sizeof(float);
 }
 extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
                                          int32_t l, int32_t g, float temperature, const void *const *student_wq,
@@ -1039,7 +1048,6 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
   if (!m || !tokens || !seq_lens || !student_wq || !student_wk || !student_wv || !grad_wq || !grad_wk || !grad_wv || !loss || !workspace)
     return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
   const swiftkv_config &c = m->cfg;
-  if (c.dtype != SWIFTKV_DTYPE_F32) return fail(SWIFTKV_ERR_UNSUPPORTED, "the distillation step runs fp32 models only");
   if (l < 1 || l > c.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c.n_layers);
   if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
   if (!(temperature > 0.f)) return fail(SWIFTKV_ERR_INVALID_ARG, "temperature must be positive");
@@ -1053,14 +1061,27 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
   const int T = cu[n_seqs];
   if (T > m->max_tokens) return fail(SWIFTKV_ERR_INVALID_ARG, "%d tokens > max_tokens %d", T, m->max_tokens);
   const DistillDims dims = distill_dims(c);
-  const size_t need = distill_workspace_floats(dims, T, l) * sizeof(float);
+  const size_t main_floats = distill_workspace_floats(dims, T, l);
+  const size_t need = (main_floats + distill_weight_floats(c)) * sizeof(float);
   if (workspace_bytes < need) return fail(SWIFTKV_ERR_WORKSPACE_SMALL, "workspace %zu < %zu bytes", workspace_bytes, need);
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // a bf16 model: fp32 copies of the frozen weights behind the step's own workspace
+  const bool widen = c.dtype == SWIFTKV_DTYPE_BF16;
+  float *wcopy = reinterpret_cast<float *>(workspace) + main_floats;
+  auto f32 = [&](const void *p, size_t n) -> const float * {
+    if (!widen) return reinterpret_cast<const float *>(p);
+    float *dst = wcopy;
+    wcopy += (n + 3) & ~(size_t)3;
+    distill_upcast(p, dst, (long long)n, st);
+    return dst;
+  };
+  const size_t dd = c.hidden, dq_ = (size_t)c.n_q_heads * c.head_dim, dkv_ = (size_t)c.n_kv_heads * c.head_dim, F_ = c.ffn;
   std::vector<DistillLayer> layers(c.n_layers);
   for (int j = 0; j < c.n_layers; ++j) {
     const swiftkv_layer_weights &w = m->layers[j];
     DistillLayer &d = layers[j];
-    d = DistillLayer{(const float *)w.in_norm, (const float *)w.wq, (const float *)w.wk, (const float *)w.wv, (const float *)w.wo,
-                     (const float *)w.post_norm, (const float *)w.w_gate, (const float *)w.w_up, (const float *)w.w_down,
+    d = DistillLayer{f32(w.in_norm, dd), f32(w.wq, dq_ * dd), f32(w.wk, dkv_ * dd), f32(w.wv, dkv_ * dd), f32(w.wo, dd * dq_),
+                     f32(w.post_norm, dd), f32(w.w_gate, F_ * dd), f32(w.w_up, F_ * dd), f32(w.w_down, dd * F_),
                      nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     if (j >= l) {
       if (!student_wq[j] || !student_wk[j] || !student_wv[j] || !grad_wq[j] || !grad_wk[j] || !grad_wv[j])
@@ -1069,13 +1090,12 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
       d.g_wq = (float *)grad_wq[j]; d.g_wk = (float *)grad_wk[j]; d.g_wv = (float *)grad_wv[j];
     }
   }
-  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   Buffers &b = m->b;
   // sequence offsets to the device (a few bytes: a blocking copy keeps the host vector's lifetime out of the picture)
   CUDA_TRY(cudaStreamSynchronize(st));
   CUDA_TRY(cudaMemcpy(b.cu, cu.data(), (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice));
   launch_positions(b.cu, n_seqs, b.pos, b.last_idx, T, st);
-  DistillArgs a{(const float *)m->embed, (const float *)m->final_norm, (const float *)m->lm_head, tokens, b.cu, b.pos, b.cos_tab,
+  DistillArgs a{f32(m->embed, (size_t)c.vocab * dd), f32(m->final_norm, dd), f32(m->lm_head, (size_t)c.vocab * dd), tokens, b.cu, b.pos, b.cos_tab,
                 b.sin_tab, T, n_seqs, l, g, temperature, loss, b.status, workspace, workspace_bytes / sizeof(float)};
   const int rc = run_distill(dims, a, layers.data(), st);
   if (rc) return fail(rc, "distillation step failed: %s", cudaGetErrorString(cudaGetLastError()));

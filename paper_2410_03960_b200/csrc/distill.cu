@@ -4,7 +4,8 @@
 // at temperature tau (tau^2 * mean over tokens of KL(softmax(y_t / tau) || softmax(y_s / tau))), and the gradient is taken
 // with respect to the student's W_Q, W_K, W_V only.  Layers 1..l are identical in both modes and run once.
 //
-// fp32 models, fp32 arithmetic throughout (forward with the library's SIMT operators, the backward operators below): this
+// fp32 arithmetic throughout (forward with the library's SIMT operators, the backward operators below; a bf16 model's frozen
+// weights are widened to fp32 copies in the workspace first, the student's copies and the gradients are fp32 either way): this
 // is the functional form of the step; the tensor-core GEMMs of the prefill path take 16-bit operands and are not used here.
 // Every output element is owned by one thread block and summed in a fixed order, so gradients repeat bit for bit.
 #include <algorithm>
@@ -270,7 +271,15 @@ __global__ void seq_end_kernel(const int32_t *__restrict__ cu, int n_seqs, int32
 
 inline int grid_for(long long n) { return (int)std::min<long long>((n + 255) / 256, 148 * 8); }
 
+__global__ void upcast_kernel(const bf16 *__restrict__ src, float *__restrict__ dst, long long n) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) dst[i] = to_f(src[i]);
+}
+
 }  // namespace
+
+void distill_upcast(const void *src_bf16, float *dst, long long n, cudaStream_t st) {
+  if (n > 0) upcast_kernel<<<grid_for(n), 256, 0, st>>>(reinterpret_cast<const bf16 *>(src_bf16), dst, n);
+}
 
 size_t distill_workspace_floats(const DistillDims &c, int T, int l) {
   const size_t d = c.d, dq = (size_t)c.n_q * c.hd, dkv = (size_t)c.n_kv * c.hd, F = c.F, V = c.vocab;

@@ -112,13 +112,55 @@ def test_unrewired_student_has_no_loss_and_a_gradient_step_lowers_the_loss():
     model.close()
 
 
+def test_bf16_model_with_fp32_student_copies():
+    """A bf16 model's frozen weights are widened to fp32 inside the step (exactly), the student's copies and the gradients are
+    fp32: same bars against the oracle run on the bf16 values."""
+    import paper_2410_03960_b200 as P
+    shape, lens, l, g, tau = MID, [33, 9, 70], 2, 2, 2.0
+    w = _scaled_weights(shape, 23, 2.0)
+    wb = S.Weights(shape, torch.bfloat16, w.embed.bfloat16(), w.final_norm.bfloat16(), w.lm_head.bfloat16(),
+                   [{k: v.bfloat16() for k, v in lw.items()} for lw in w.layers])
+    w32 = S.Weights(shape, torch.float32, wb.embed.float(), wb.final_norm.float(), wb.lm_head.float(),
+                    [{k: v.float() for k, v in lw.items()} for lw in wb.layers])
+    tok = S.make_prompts(23, lens, shape.vocab)
+    st = _student(w32, l, 24, 0.3)
+    want_loss, want = D.distill_grads(oracle_config(shape), oracle_weights(w32),
+                                      {k: [None if t is None else t.double().numpy() for t in v] for k, v in st.items()},
+                                      tok.numpy(), lens, l, g, tau)
+    wc = S.Weights(shape, torch.bfloat16, wb.embed.cuda(), wb.final_norm.cuda(), wb.lm_head.cuda(),
+                   [{k: v.cuda() for k, v in lw.items()} for lw in wb.layers])
+    model = P.SwiftKVModel(shape, wc, torch.bfloat16, sum(lens), len(lens), l, g)
+    loss, grads = model.distill_grads(tok, lens, l, g, tau, {k: [None if t is None else t.cuda() for t in v] for k, v in st.items()})
+    model.status()
+    assert abs(float(loss) - want_loss) <= 2e-5 * want_loss, (float(loss), want_loss)
+    for name in ("wq", "wk", "wv"):
+        for j in range(l, shape.n_layers):
+            got, ref = to_np(grads[name][j]).astype(np.float64), want[name][j]
+            if np.abs(ref).max() == 0.0:
+                assert np.abs(got).max() == 0.0
+            else:
+                assert _rel(got, ref) <= 5e-5, (name, j, _rel(got, ref))
+    # the prefill path of the same handle still works afterwards
+    model.prefill(tok, lens, l, g)
+    model.status()
+    assert torch.isfinite(model.first_logits()).all()
+    model.close()
+
+
 def test_argument_checks():
     import paper_2410_03960_b200 as P
     shape, lens = S.TINY, [8]
-    w = S.make_weights(shape, 1, torch.bfloat16, "cuda")
-    model = P.SwiftKVModel(shape, w, torch.bfloat16, 8, 1, 2, 1)
-    st = {name: [None, None] + [w.layers[j][name].float() for j in range(2, shape.n_layers)] for name in ("wq", "wk", "wv")}
-    with pytest.raises(P.SwiftKVError) as e:
-        model.distill_grads(S.make_prompts(1, lens, shape.vocab), lens, 2, 1, 2.0, st)
-    assert e.value.code == -7          # SWIFTKV_ERR_UNSUPPORTED
+    w = S.make_weights(shape, 1, torch.float32, "cuda")
+    model = P.SwiftKVModel(shape, w, torch.float32, 8, 1, 2, 1)
+    st = {name: [None, None] + [w.layers[j][name].clone() for j in range(2, shape.n_layers)] for name in ("wq", "wk", "wv")}
+    tok = S.make_prompts(1, lens, shape.vocab)
+    for bad in (dict(swift_layer=0), dict(swift_layer=shape.n_layers + 1), dict(acrosskv_group=0), dict(temperature=0.0)):
+        args = dict(swift_layer=2, acrosskv_group=1, temperature=2.0)
+        args.update(bad)
+        with pytest.raises(P.SwiftKVError) as e:
+            model.distill_grads(tok, lens, args["swift_layer"], args["acrosskv_group"], args["temperature"], st)
+        assert e.value.code == -1, bad          # SWIFTKV_ERR_INVALID_ARG
+    st["wk"][3] = None                          # a missing student matrix of a re-wired layer
+    with pytest.raises((P.SwiftKVError, AssertionError)):
+        model.distill_grads(tok, lens, 2, 1, 2.0, st)
     model.close()
