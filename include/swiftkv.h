@@ -345,6 +345,14 @@ int32_t swiftkv_set_split_mask(swiftkv_model *m, int32_t mask);
  * of the CTA left through the abort flag.  Afterwards swiftkv_status reports SWIFTKV_ERR_DEVICE_TIMEOUT once.
  * Errors: INVALID_ARG, CUDA. */
 int32_t swiftkv_debug_bounded_wait(swiftkv_model *m, int64_t limit_clocks, int32_t *outcome, void *cuda_stream);
+/* The same self-check for the persistent cooperative launch of the last-token path (kernel-mask bit 6): two stages of layer
+ * 1 are launched on one zero row with every in-kernel wait limited to `limit_clocks` SM clocks (1 .. 1e8) and a grid barrier
+ * between them that cannot complete (the host claims one arrival that never happened).  Every CTA's wait runs out, the kernel
+ * latches DEVICE_TIMEOUT, raises its abort word, lets the copies in flight land, and returns; the call synchronises the
+ * stream.  Afterwards swiftkv_status reports SWIFTKV_ERR_DEVICE_TIMEOUT once and the model needs a new prefill before its
+ * cache / logits are read.  bf16 models whose widths the fused launch supports (UNSUPPORTED otherwise).
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_debug_fused_barrier_wait(swiftkv_model *m, int64_t limit_clocks, void *cuda_stream);
 
 /* Synchronises `cuda_stream`, then returns and clears the current device's status word of the stand-alone operator
  * entry points below (swiftkv_gemm_tc, swiftkv_attention_prefill): OK, DEVICE_TIMEOUT, ACT_OVERFLOW or CUDA. */

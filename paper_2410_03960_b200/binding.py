@@ -26,7 +26,7 @@ EXPORTS = (
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
     "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
-    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads",
+    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait",
 )
 
 
@@ -106,6 +106,7 @@ def load_library() -> C.CDLL:
     lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
+    lib.swiftkv_debug_fused_barrier_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.swiftkv_debug_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
     lib.swiftkv_op_status.argtypes = [C.c_void_p]
     lib.swiftkv_tail_attention_scratch_bytes.argtypes = [C.c_int32] * 4
@@ -281,6 +282,11 @@ class SwiftKVModel:
                                              sim.data_ptr(), score.data_ptr(), _stream_ptr(stream)))
             torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
         return score, sim
+
+    def debug_fused_barrier_wait(self, limit_clocks: int, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """swiftkv_debug_fused_barrier_wait: makes the fused last-token launch's grid barrier run out; status() raises afterwards."""
+        with torch.cuda.device(self.device):
+            _check(self.lib.swiftkv_debug_fused_barrier_wait(self._h, int(limit_clocks), _stream_ptr(stream)))
 
     def distill_grads(self, tokens, seq_lens: Sequence[int], swift_layer: int, acrosskv_group: int, temperature: float,
                       student: dict, stream: Optional[torch.cuda.Stream] = None):

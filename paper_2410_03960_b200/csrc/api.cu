@@ -1240,6 +1240,31 @@ extern "C" int32_t swiftkv_debug_bounded_wait(swiftkv_model *m, int64_t limit_cl
   return SWIFTKV_OK;
 }
 
+extern "C" int32_t swiftkv_debug_fused_barrier_wait(swiftkv_model *m, int64_t limit_clocks, void *cuda_stream) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (limit_clocks < 1 || limit_clocks > 100000000LL) return fail(SWIFTKV_ERR_INVALID_ARG, "limit_clocks outside [1, 1e8]");
+  const swiftkv_config &c = m->cfg;
+  const int d = c.hidden, dq = c.n_q_heads * c.head_dim, F = c.ffn;
+  if (c.dtype != SWIFTKV_DTYPE_BF16 || !tail_fused_supported(1, d, dq, F, c.vocab))
+    return fail(SWIFTKV_ERR_UNSUPPORTED, "the fused last-token launch does not run this model");
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  Buffers &b = m->b;
+  const swiftkv_layer_weights &lw = m->layers[0];
+  CUDA_TRY(cudaMemsetAsync(b.status + 32, 0, 32 * sizeof(unsigned int), st));
+  CUDA_TRY(cudaMemsetAsync(b.ay, 0, (size_t)dq * sizeof(float), st));
+  CUDA_TRY(cudaMemsetAsync(b.y, 0, (size_t)d * sizeof(float), st));
+  // two stages of layer 1 on one zero row; the host claims one barrier arrival that never happened, so the grid barrier
+  // between the stages can never complete and every CTA's wait runs out at the limit
+  TailStage list[2] = {TailStage{b.ay, nullptr, lw.wo, nullptr, b.y, d, dq, d, 1},
+                       TailStage{b.y, lw.post_norm, lw.w_gate, lw.w_up, b.acty, F, d, F, 2}};
+  unsigned int arrivals = 1;
+  const int rc = launch_tail_fused(list, 2, 1, c.rms_eps, b.status + 32, &arrivals, b.status, st, (long long)limit_clocks);
+  if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  CUDA_TRY(cudaStreamSynchronize(st));
+  m->ready = false;
+  return SWIFTKV_OK;
+}
+
 extern "C" int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K,
                                    int32_t dtype, void *cuda_stream) {
   const int32_t act_dtype = dtype;

@@ -317,7 +317,9 @@ void distill_upcast(const void *src_bf16, float *dst, long long n, cudaStream_t 
 int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *layers, cudaStream_t st);
 // arrivals: the host's count of barrier arrivals on sync[0] so far (the counter is never reset between launches; zero both
 // together).
+// wait_limit_clocks: how long any single wait inside the kernel (ring stage, grid barrier) may take before the kernel latches
+// STATUS_TIMEOUT and every role leaves (0: the default of about two seconds).
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
-                      unsigned int *status, cudaStream_t st);
+                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks = 0);
 
 }  // namespace skv

@@ -995,6 +995,7 @@ struct Params {
   int n_stages, rows;
   int rs;                   // log2 of the row slots per activation block
   float eps;
+  long long wait_limit;     // clocks any single wait may take before the kernel gives up
   unsigned int sync_base;   // arrivals counted by earlier launches (the counter is never reset)
   unsigned int *sync;       // [0] arrivals at the grid barrier, [1] abort word
   unsigned int *status;
@@ -1004,6 +1005,7 @@ struct Ctx {
   uint8_t *smem;
   volatile int *abort_s;    // this CTA's copy of "give up"
   volatile int *open_s;     // the last stage whose inputs are complete (written by the MMA warps after the grid barrier)
+  volatile int *decide_s;   // "give up", as published to all MMA warps at one point (so that they leave together)
   unsigned epoch;           // grid barriers passed
   unsigned chunk_no;        // ring chunks produced / consumed so far (same sequence in every role)
   unsigned fill_no;         // resident fills so far
@@ -1026,7 +1028,7 @@ __device__ __forceinline__ bool ring_wait(const Params &p, Ctx &c, uint32_t bar,
     if (mbar_try_wait(bar, parity)) return true;
     if ((spins & 63u) == 0u) {
       if (aborted(p, c)) return false;
-      if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); return false; }
+      if (clock64() - t0 > p.wait_limit) { give_up(p, c); return false; }
     }
   }
 }
@@ -1044,14 +1046,15 @@ __device__ __forceinline__ bool grid_barrier(const Params &p, Ctx &c) {
       if ((int)(*reinterpret_cast<volatile unsigned int *>(p.sync) - target) >= 0) break;
       if ((spins & 15u) == 0u) {
         if (aborted(p, c)) break;
-        if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); break; }
+        if (clock64() - t0 > p.wait_limit) { give_up(p, c); break; }
       }
     }
     __threadfence();
+    *c.decide_s = *c.abort_s;
   }
   consumer_sync();
   c.epoch += 1;
-  return !*c.abort_s;
+  return !*c.decide_s;
 }
 
 // ---- producer warp (one lane): every stage's weight rows, tile by tile, chunk by chunk, through the ring -- as far ahead
@@ -1098,7 +1101,7 @@ __device__ void produce(const Params &p, Ctx &c) {
             request_activations(j);
             if ((spins & 63u) == 0u) {
               if (aborted(p, c)) { c.chunk_no = base + j; return; }
-              if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); c.chunk_no = base + j; return; }
+              if (clock64() - t0 > p.wait_limit) { give_up(p, c); c.chunk_no = base + j; return; }
             }
           }
         }
@@ -1117,7 +1120,7 @@ __device__ void produce(const Params &p, Ctx &c) {
         request_activations(total);
         if ((spins & 63u) == 0u) {
           if (aborted(p, c)) return;
-          if (clock64() - t0 > WAIT_LIMIT) { give_up(p, c); return; }
+          if (clock64() - t0 > p.wait_limit) { give_up(p, c); return; }
         }
       }
     }
@@ -1142,6 +1145,7 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
   // RMSNorm folded in: activations are multiplied by the gain on the way in, the row statistic 1 / rms scales the OUTPUT
   // row in the epilogue (it is a per-row scalar), so it can be accumulated in the same pass that brings the activations in
   float ss = 0.f;                                      // RESIDENT: this lane's row (g); else row (lane & 7)
+  bool dead = false;
   if (RESIDENT) {
     if (threadIdx.x == 0) {
       fence_generic_to_async();
@@ -1149,13 +1153,15 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
       for (int part = 0; part < K / KC1; ++part)
         tc::tma_load_3d(smem_u32(res + part * (KC1 / 32) * AB), &sg.tmA, smem_u32(afull), 0, 0, part * (KC1 / 32));
     }
-    if (!ring_wait(p, c, smem_u32(afull), c.fill_no & 1)) return;
+    // (a wait that runs out never makes a warp leave early: the named barriers below count all 256 threads, so a warp that
+    //  gave up keeps walking the same barriers and only skips the work)
+    dead = !ring_wait(p, c, smem_u32(afull), c.fill_no & 1);
     c.fill_no += 1;
     // every warp converts, in place, exactly the blocks it will multiply with, 8 / RP blocks at a time:
     // lane = (block of the group, row, quarter)
     const int grp = g >> rs, r = g & (RP - 1), G = 8 >> rs;
     const int n_blk = K / (32 * CONSUMERS);
-    for (int b = 0; b < n_blk; b += 2 * G) {
+    for (int b = 0; b < n_blk && !dead; b += 2 * G) {
       uint8_t *blk[2];
       float x[2][8];
       uint4 gm[2];
@@ -1239,7 +1245,8 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
           if (sg.gamma) gm[u] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)kc * KC + k_lane + u * 32));
         }
       }
-      if (!ring_wait(p, c, smem_u32(&full[st]), ph)) return;
+      if (!dead && !ring_wait(p, c, smem_u32(&full[st]), ph)) dead = true;
+      if (dead) continue;
       const uint8_t *sw = c.smem + st * STAGE_BYTES;
 #pragma unroll
       for (int u = 0; u < STEPS; ++u) {
@@ -1308,7 +1315,7 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
       if (DUAL) buf[((warp * 2 + 1) * 32 + lane) * 4 + i] = (acc2[0][i] + acc2[1][i]) + (acc2[2][i] + acc2[3][i]);
     }
     consumer_sync();
-    if (warp == (tile_no & (CONSUMERS - 1))) {      // (the warps take turns, so that none falls a whole epilogue behind per tile)
+    if (warp == (tile_no & (CONSUMERS - 1)) && !*c.abort_s) {      // (the warps take turns, so that none falls a whole epilogue behind per tile)
       float s1[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int w = 0; w < CONSUMERS; ++w)
@@ -1344,6 +1351,7 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
   c.smem = fsmem;
   c.abort_s = reinterpret_cast<volatile int *>(fsmem + SM_MISC);
   c.open_s = c.abort_s + 1;
+  c.decide_s = c.abort_s + 2;
   c.epoch = 0;
   c.chunk_no = 0;
   c.fill_no = 0;
@@ -1353,6 +1361,7 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
     mbar_init(smem_u32(afull), 1);
     *c.abort_s = 0;
     *c.open_s = 0;
+    *c.decide_s = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -1376,7 +1385,9 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
       const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
       if (sg.epi >= 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
       else { if (resident) consume<false, true>(p, c, sg); else consume<false, false>(p, c, sg); }
-      if (*c.abort_s) break;
+      if (threadIdx.x == 0) *c.decide_s = *c.abort_s;      // (consume ended with a barrier of the MMA warps)
+      consumer_sync();
+      if (*c.decide_s) break;
     }
   }
   __syncthreads();
@@ -1400,7 +1411,7 @@ bool tail_fused_supported(int rows, int d, int dq, int F, int vocab) {
 }
 
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
-                      unsigned int *status, cudaStream_t st) {
+                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks) {
   if (n_stages < 1 || n_stages > fused::MAX_STAGE_LIST || rows < 1 || rows > MAX_TAIL_ROWS) return SWIFTKV_ERR_UNSUPPORTED;
   fused::Params p{};
   int rs = 0;
@@ -1420,6 +1431,7 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
   }
   p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
   p.sync_base = *arrivals;
+  p.wait_limit = wait_limit_clocks > 0 ? wait_limit_clocks : fused::WAIT_LIMIT;
   int dev = 0, n_sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
     return SWIFTKV_ERR_CUDA;

@@ -44,6 +44,35 @@ def test_bounded_wait_runs_out_and_is_reported_once():
     model.close()
 
 
+def test_fused_launch_grid_barrier_runs_out_and_is_reported():
+    """The persistent cooperative launch of the last-token path waits at its own grid barrier and ring barriers; all are
+    bounded.  A launch whose barrier cannot complete (the host claims an arrival that never happened), with a limit of one
+    million clocks: every CTA gives up, the kernel returns, DEVICE_TIMEOUT is reported once, and the next prefill -- which
+    uses the same kernel with the default limit -- gives the same bits as before."""
+    import paper_2410_03960_b200 as P
+    lens = [70, 9, 300]
+    w = S.make_weights(MID, 6, torch.bfloat16, "cuda")
+    tok = S.make_prompts(6, lens, MID.vocab)
+    model = _model(MID, w, lens)
+    assert model.set_kernel_mask(119) == 119
+    model.prefill(tok, lens, 2, 1)
+    model.status()
+    want = model.first_logits().clone()
+    model.debug_fused_barrier_wait(1_000_000)
+    with pytest.raises(P.SwiftKVError) as e:
+        model.status()
+    assert e.value.code == -5
+    model.status()
+    for _ in range(2):
+        model.prefill(tok, lens, 2, 1)
+        model.status()
+        assert torch.equal(model.first_logits(), want)
+    with pytest.raises(P.SwiftKVError) as e:
+        model.debug_fused_barrier_wait(10 ** 12)
+    assert e.value.code == -1
+    model.close()
+
+
 @pytest.mark.parametrize("mask", [55, 0])
 def test_half_activation_overflow_is_reported_not_silent(mask):
     """With IEEE-half activations a value beyond +-65504 is clamped -- and reported: one layer's up-projection is scaled
