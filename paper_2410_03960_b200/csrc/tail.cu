@@ -941,26 +941,27 @@ namespace fused {
 
 constexpr int CONSUMERS = 8;
 constexpr int THREADS = (CONSUMERS + 1) * 32;
-constexpr int STAGES = 5;
+// ring depth: 5 stages beside 8 rows of resident activations; fewer rows leave room for more (up to 11), so that the
+// producer can run further ahead while the MMA warps stand at a grid barrier or fill their activations
+constexpr int MIN_STAGES = 5, MAX_STAGES = 12;
 // one matrix: 16 rows x 512 columns per ring stage; two matrices (gate / up): 2 x (16 rows x 256 columns).  A stage is
 // filled by ONE tiled bulk copy per matrix (a copy per row segment costs the copy engine ~60 clocks each and capped the
 // stream at a third of the HBM rate): blocks of 16 lines of 128 bytes, 128-byte swizzle.
 constexpr int KC1 = 512, KC2 = 256;
 constexpr int STAGE_BYTES = 16 * KC1 * 2;             // 16384
-constexpr int RING_BYTES = STAGES * STAGE_BYTES;      // 81920
+constexpr int POOL_BYTES = 212992;                    // the ring (n x 16 KB) followed by the activation area
 // Activations come in blocks of one 32-wide K step: [row slots][32 floats], row slots = the launch's rows rounded up to a
 // power of two (1, 2, 4, 8; the padding rows are zero-filled), brought by tiled bulk copies.  K <= 4096: all K / 32 blocks
 // are resident and converted IN PLACE, once per stage, into the MMA fragments [bf16 hi | bf16 lo][row][quarter]; larger K:
 // the blocks of a K chunk travel with the chunk's weights through a ring of their own and are converted as they are used.
 constexpr int ACT_BLOCK = 1024;                       // the largest block: 8 row slots
-constexpr int RES_BYTES = 131072;
-constexpr int ACT_SLOT = (KC1 / 32) * ACT_BLOCK;      // 16384; STAGES of them fit RES_BYTES
+constexpr int RES_BYTES = 131072;                     // K * 32 <= RES_BYTES: resident (K <= 4096)
 constexpr int RED_FLOATS = 2 * CONSUMERS * 2 * 32 * 4;   // two buffers of [warp][matrix][lane][4]
-constexpr int SM_RES = RING_BYTES, SM_RED = SM_RES + RES_BYTES, SM_BAR = SM_RED + RED_FLOATS * 4, SM_MISC = SM_BAR + 128;
-constexpr int SMEM_BYTES = SM_MISC + 256 + 1024;      // 230784 incl. the slack to align the ring to 1024 bytes
+constexpr int SM_RED = POOL_BYTES, SM_BAR = SM_RED + RED_FLOATS * 4, SM_MISC = SM_BAR + 256;
+constexpr int SMEM_BYTES = SM_MISC + 256 + 1024;      // 230912 incl. the slack to align the ring to 1024 bytes
+static_assert(MIN_STAGES * STAGE_BYTES + RES_BYTES <= POOL_BYTES, "8 rows: 5 ring stages + 128 KB of resident activations");
 constexpr long long WAIT_LIMIT = 4000000000LL;
 constexpr int MAX_STAGE_LIST = 6;
-static_assert(STAGES * ACT_SLOT <= RES_BYTES, "the activation ring lives in the resident area");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -994,6 +995,7 @@ struct Params {
   Stage st[MAX_STAGE_LIST];
   int n_stages, rows;
   int rs;                   // log2 of the row slots per activation block
+  int n_ring;               // ring depth of this launch (MIN_STAGES .. MAX_STAGES - 1)
   float eps;
   long long wait_limit;     // clocks any single wait may take before the kernel gives up
   unsigned int sync_base;   // arrivals counted by earlier launches (the counter is never reset)
@@ -1008,6 +1010,7 @@ struct Ctx {
   volatile int *decide_s;   // "give up", as published to all MMA warps at one point (so that they leave together)
   unsigned epoch;           // grid barriers passed
   unsigned chunk_no;        // ring chunks produced / consumed so far (same sequence in every role)
+  unsigned slot, phase;     // ring slot of chunk chunk_no and the parity of its use
   unsigned fill_no;         // resident fills so far
 };
 
@@ -1061,8 +1064,10 @@ __device__ __forceinline__ bool grid_barrier(const Params &p, Ctx &c) {
 //      as the ring allows, across stage boundaries.  A stage whose K is too large for resident activations also gets each
 //      chunk's activation blocks, but those are requested only once the stage's inputs are complete (open_s).
 __device__ void produce(const Params &p, Ctx &c) {
-  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES;
+  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + MAX_STAGES;
   if ((threadIdx.x & 31) != 0) return;
+  const unsigned n_ring = (unsigned)p.n_ring;
+  uint8_t *res = c.smem + n_ring * STAGE_BYTES;
   for (int i = 0; i < p.n_stages; ++i) {
     const Stage &sg = p.st[i];
     const bool dual = sg.epi >= 2;
@@ -1070,9 +1075,11 @@ __device__ void produce(const Params &p, Ctx &c) {
     const int n_tiles = sg.N / 16, n_chunks = sg.K / kc_len;
     const bool resident = (long long)sg.K * 32 <= RES_BYTES;
     const uint32_t act_bytes = resident ? 0u : (uint32_t)(kc_len / 32) * (128u << p.rs);
+    const uint32_t act_slot_bytes = (uint32_t)(KC1 / 32) * (128u << p.rs);
     const unsigned my_tiles = (int)blockIdx.x < n_tiles ? (unsigned)(n_tiles - 1 - (int)blockIdx.x) / gridDim.x + 1u : 0u;
     const unsigned total = my_tiles * (unsigned)n_chunks, base = c.chunk_no;
     unsigned act_j = resident ? total : 0u;       // next chunk of the stage whose activation blocks are still to be requested
+    unsigned act_slot = c.slot;                   // ... and its ring slot
     int act_kc = 0;
     bool open = i == 0;
     auto request_activations = [&](unsigned issued) {
@@ -1084,16 +1091,16 @@ __device__ void produce(const Params &p, Ctx &c) {
         open = true;
       }
       for (; act_j < issued; ++act_j) {
-        const unsigned slot = (base + act_j) % STAGES;
-        tc::tma_load_3d(smem_u32(c.smem + SM_RES + slot * ACT_SLOT), &sg.tmA, smem_u32(&full[slot]), 0, 0, act_kc * (kc_len / 32));
+        tc::tma_load_3d(smem_u32(res + act_slot * act_slot_bytes), &sg.tmA, smem_u32(&full[act_slot]), 0, 0, act_kc * (kc_len / 32));
         if (++act_kc == n_chunks) act_kc = 0;
+        if (++act_slot == n_ring) act_slot = 0;
       }
     };
     unsigned j = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       for (int kc = 0; kc < n_chunks; ++kc, ++j) {
-        const unsigned slot = (base + j) % STAGES;
-        const uint32_t ph = ((base + j) / STAGES) & 1;
+        const unsigned slot = c.slot;
+        const uint32_t ph = c.phase;
         const uint32_t eb = smem_u32(&empty[slot]);
         if (!mbar_try_wait(eb, ph ^ 1)) {
           const long long t0 = clock64();
@@ -1110,6 +1117,7 @@ __device__ void produce(const Params &p, Ctx &c) {
         const uint32_t dst = smem_u32(c.smem + slot * STAGE_BYTES);
         tc::tma_load_3d(dst, &sg.tmW, fb, 0, tile * 16, kc * (kc_len / 64));
         if (dual) tc::tma_load_3d(dst + STAGE_BYTES / 2, &sg.tmW2, fb, 0, tile * 16, kc * (kc_len / 64));
+        if (++c.slot == n_ring) { c.slot = 0; c.phase ^= 1; }
         request_activations(j + 1);
       }
     }
@@ -1133,10 +1141,11 @@ template <bool DUAL, bool RESIDENT>
 __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
   constexpr int KC = DUAL ? KC2 : KC1;
   constexpr int STEPS = KC / (CONSUMERS * 32);         // 32-wide K steps per warp and chunk: 2 (one matrix) or 1 (two)
-  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + STAGES, *afull = empty + STAGES;
+  uint64_t *full = reinterpret_cast<uint64_t *>(c.smem + SM_BAR), *empty = full + MAX_STAGES, *afull = empty + MAX_STAGES;
   float *red = reinterpret_cast<float *>(c.smem + SM_RED);
   float *rstd_s = reinterpret_cast<float *>(c.smem + SM_MISC) + 8;
-  uint8_t *res = c.smem + SM_RES;
+  const unsigned n_ring = (unsigned)p.n_ring;
+  uint8_t *res = c.smem + n_ring * STAGE_BYTES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int K = sg.K, n_tiles = sg.N / 16, n_chunks = K / KC;
   const int g = lane >> 2, t = lane & 3;
@@ -1235,8 +1244,9 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
     // four independent accumulator chains per matrix
     float acc[4][4] = {}, acc2[4][4] = {};
     for (int kc = 0; kc < n_chunks; ++kc, ++c.chunk_no) {
-      const int st = c.chunk_no % STAGES;
-      const uint32_t ph = (c.chunk_no / STAGES) & 1;
+      const int st = (int)c.slot;
+      const uint32_t ph = c.phase;
+      if (++c.slot == n_ring) { c.slot = 0; c.phase ^= 1; }
       uint4 gm[STEPS];
       if (!RESIDENT) {
 #pragma unroll
@@ -1263,7 +1273,7 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
         } else {
           float4 xa = make_float4(0.f, 0.f, 0.f, 0.f), xb = xa;
           if (row_ok) {
-            const uint8_t *fa = res + (size_t)st * ACT_SLOT + (size_t)(warp * STEPS + u) * AB + g * 128 + t * 32;
+            const uint8_t *fa = res + (size_t)st * ((KC1 / 32) * AB) + (size_t)(warp * STEPS + u) * AB + g * 128 + t * 32;
             xa = *reinterpret_cast<const float4 *>(fa);
             xb = *reinterpret_cast<const float4 *>(fa + 16);
           }
@@ -1354,10 +1364,12 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
   c.decide_s = c.abort_s + 2;
   c.epoch = 0;
   c.chunk_no = 0;
+  c.slot = 0;
+  c.phase = 0;
   c.fill_no = 0;
-  uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + SM_BAR), *empty = full + STAGES, *afull = empty + STAGES;
+  uint64_t *full = reinterpret_cast<uint64_t *>(fsmem + SM_BAR), *empty = full + MAX_STAGES, *afull = empty + MAX_STAGES;
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), CONSUMERS); }
+    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(smem_u32(&full[s]), 1); mbar_init(smem_u32(&empty[s]), CONSUMERS); }
     mbar_init(smem_u32(afull), 1);
     *c.abort_s = 0;
     *c.open_s = 0;
@@ -1369,10 +1381,10 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
     produce(p, c);
     // giving up: copies still in flight must land before this CTA's shared memory is released
     if (*c.abort_s && (threadIdx.x & 31) == 0) {
-      const unsigned issued = c.chunk_no;
-      for (unsigned q = issued > STAGES ? issued - STAGES : 0; q < issued; ++q) {
+      const unsigned issued = c.chunk_no, n_ring = (unsigned)p.n_ring;
+      for (unsigned q = issued > n_ring ? issued - n_ring : 0; q < issued; ++q) {
         const long long t0 = clock64();
-        while (!mbar_try_wait(smem_u32(&full[q % STAGES]), (q / STAGES) & 1) && clock64() - t0 < 100000000LL) {}
+        while (!mbar_try_wait(smem_u32(&full[q % n_ring]), (q / n_ring) & 1) && clock64() - t0 < 100000000LL) {}
       }
     }
   } else {
@@ -1430,6 +1442,23 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
     d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.out2 = s.out2; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
   }
   p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
+  // ring depth: as many 16 KB stages as fit beside the activation area this launch needs (resident blocks of its widest
+  // resident stage, or one activation slot per ring stage for a stage that streams them)
+  {
+    const size_t ab = (size_t)128 << rs;
+    size_t resident_need = 0;
+    bool streams = false;
+    for (int i = 0; i < n_stages; ++i) {
+      if ((long long)stages[i].K * 32 <= fused::RES_BYTES) resident_need = std::max(resident_need, (size_t)(stages[i].K / 32) * ab);
+      else streams = true;
+    }
+    int n = fused::MIN_STAGES;
+    for (int cand = fused::MAX_STAGES - 1; cand > fused::MIN_STAGES; --cand) {
+      const size_t act = std::max(resident_need, streams ? (size_t)cand * (fused::KC1 / 32) * ab : (size_t)0);
+      if ((size_t)cand * fused::STAGE_BYTES + act <= (size_t)fused::POOL_BYTES) { n = cand; break; }
+    }
+    p.n_ring = n;
+  }
   p.sync_base = *arrivals;
   p.wait_limit = wait_limit_clocks > 0 ? wait_limit_clocks : fused::WAIT_LIMIT;
   int dev = 0, n_sms = 0;
