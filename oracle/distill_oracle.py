@@ -15,7 +15,11 @@ the output logits of the original model"), with the usual tau^2 factor, averaged
 RMSNorm gains stay frozen (they are not part of W_QKV); with AcrossKV only a group leader's W_K, W_V are used, so the
 other layers' W_K, W_V receive zero gradient.
 
-`distill_grads` is the analytic backward pass written out operator by operator.  Pins (tests/test_oracle_pins.py):
+The update rule: the paper's training details give a learning rate (3e-4), a weight decay (0.05) and a warm-up ratio but do
+not name the optimiser; `adamw_update` is AdamW with decoupled weight decay (the usual choice for exactly that set of
+hyper-parameters), pinned against torch.optim.AdamW.
+
+`distill_grads` is the analytic backward pass written out operator by operator.  Pins (tests/test_distill_oracle_pins.py):
 central finite differences of `distill_loss`, torch autograd (fp64) through a torch-assembled student, loss = 0 and zero
 gradients when the student is not re-wired (l = L), KL >= 0, zero gradient for non-leader W_K / W_V.
 
@@ -197,3 +201,16 @@ def distill_grads(cfg: Config, W: Weights, S, tokens, seq_lens, l: int, g: int =
             grads["wk"][j] = np.zeros_like(S["wk"][j])
             grads["wv"][j] = np.zeros_like(S["wv"][j])
     return loss, grads
+
+
+def adamw_update(param, grad, m, v, step: int, lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                 weight_decay: float = 0.05):
+    """One AdamW step (decoupled weight decay), `step` counted from 1.  Returns (param, m, v), all new arrays.
+        p <- p (1 - lr wd);  m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;
+        p <- p - lr (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)."""
+    param = np.asarray(param, dtype=F64) * (1.0 - lr * weight_decay)
+    m = beta1 * np.asarray(m, dtype=F64) + (1.0 - beta1) * grad
+    v = beta2 * np.asarray(v, dtype=F64) + (1.0 - beta2) * grad * grad
+    m_hat = m / (1.0 - beta1 ** step)
+    v_hat = v / (1.0 - beta2 ** step)
+    return param - lr * m_hat / (np.sqrt(v_hat) + eps), m, v

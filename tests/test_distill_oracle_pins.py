@@ -169,3 +169,21 @@ def test_loss_definition_and_temperature():
         assert abs(got - lib) <= 1e-12
     assert abs(D.distill_loss_from_logits(yt, yt, 2.0)) <= 1e-15
     assert abs(D.distill_loss_from_logits(yt, yt + 3.0, 2.0)) <= 1e-15          # logits are shift-invariant
+
+
+def test_adamw_update_against_the_library():
+    rng = np.random.default_rng(4)
+    p0 = rng.standard_normal((7, 5))
+    grads = [rng.standard_normal((7, 5)) * (10.0 ** -k) for k in range(4)]
+    for wd in (0.05, 0.0):
+        t = torch.tensor(p0, dtype=torch.float64, requires_grad=True)
+        opt = torch.optim.AdamW([t], lr=3e-4, betas=(0.9, 0.999), eps=1e-8, weight_decay=wd)
+        p, m, v = p0.copy(), np.zeros_like(p0), np.zeros_like(p0)
+        for step, g in enumerate(grads, 1):
+            t.grad = torch.tensor(g)
+            opt.step()
+            p, m, v = D.adamw_update(p, g, m, v, step, 3e-4, 0.9, 0.999, 1e-8, wd)
+            assert np.abs(p - t.detach().numpy()).max() <= 1e-14
+    # first step of a zero-decay run moves every weight by lr against the sign of its gradient (up to eps)
+    p, _, _ = D.adamw_update(p0, grads[0], np.zeros_like(p0), np.zeros_like(p0), 1, 3e-4, weight_decay=0.0)
+    assert np.allclose(p0 - p, 3e-4 * np.sign(grads[0]), rtol=1e-6)
