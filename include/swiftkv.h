@@ -234,6 +234,16 @@ int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int
                               void *const *grad_wq, void *const *grad_wk, void *const *grad_wv, float *loss,
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* The update that goes with swiftkv_distill_grads.  The training details of the paper give a learning rate (3e-4), a weight
+ * decay (0.05) and a warm-up ratio (5 %) but do not name the optimiser; this is AdamW with decoupled weight decay, one
+ * elementwise pass over a parameter tensor (all DEVICE fp32 arrays of n elements; exp_avg / exp_avg_sq are the optimiser
+ * state, zero before step 1; step counts from 1; the learning-rate schedule is the caller's):
+ *     p <- p (1 - lr wd);  m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;
+ *     p <- p - lr (m / (1 - b1^step)) / (sqrt(v / (1 - b2^step)) + eps).
+ * Errors: INVALID_ARG, CUDA. */
+int32_t swiftkv_adamw_update(float *param, const float *grad, float *exp_avg, float *exp_avg_sq, int64_t n, int32_t step,
+                             float lr, float beta1, float beta2, float eps, float weight_decay, void *cuda_stream);
+
 typedef struct {
   const void *k;            /* device, [n_tokens][n_kv_heads][head_dim], model dtype (FP8 cache: uint8 e4m3
                                codes), AFTER RoPE                                                           */

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     KV_MODEL_DTYPE,
     SwiftKVError,
     SwiftKVModel,
+    adamw_update,
     attention_prefill,
     attention_prefill_split,
     gemm_tc_split,

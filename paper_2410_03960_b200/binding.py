@@ -26,7 +26,7 @@ EXPORTS = (
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
     "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
-    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait",
+    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait", "swiftkv_adamw_update",
 )
 
 
@@ -106,6 +106,7 @@ def load_library() -> C.CDLL:
     lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
+    lib.swiftkv_adamw_update.argtypes = [C.c_void_p] * 4 + [C.c_int64, C.c_int32] + [C.c_float] * 5 + [C.c_void_p]
     lib.swiftkv_debug_fused_barrier_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.swiftkv_debug_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
     lib.swiftkv_op_status.argtypes = [C.c_void_p]
@@ -343,6 +344,17 @@ class SwiftKVModel:
     def set_split_mask(self, mask: int) -> None:
         """swiftkv_set_split_mask: which operands travel as half pairs (SPLIT_* bits)."""
         _check(self.lib.swiftkv_set_split_mask(self._h, mask))
+
+
+def adamw_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor, step: int,
+                 lr: float = 3e-4, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.05,
+                 stream: Optional[torch.cuda.Stream] = None) -> None:
+    """swiftkv_adamw_update: one in-place AdamW step on an fp32 CUDA tensor (defaults: the paper's lr and weight decay)."""
+    for t in (param, grad, exp_avg, exp_avg_sq):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.numel() == param.numel()
+    with torch.cuda.device(param.device):
+        _check(load_library().swiftkv_adamw_update(param.data_ptr(), grad.data_ptr(), exp_avg.data_ptr(), exp_avg_sq.data_ptr(),
+                                                  param.numel(), int(step), lr, beta1, beta2, eps, weight_decay, _stream_ptr(stream)))
 
 
 def split_halves(x: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:

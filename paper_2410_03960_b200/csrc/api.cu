@@ -1103,6 +1103,18 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
   return SWIFTKV_OK;
 }
 
+extern "C" int32_t swiftkv_adamw_update(float *param, const float *grad, float *exp_avg, float *exp_avg_sq, int64_t n, int32_t step,
+                                        float lr, float beta1, float beta2, float eps, float weight_decay, void *cuda_stream) {
+  if (!param || !grad || !exp_avg || !exp_avg_sq) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
+  if (n < 0 || step < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "n must be >= 0 and step >= 1");
+  if (!(lr >= 0.f) || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f) || !(weight_decay >= 0.f))
+    return fail(SWIFTKV_ERR_INVALID_ARG, "bad hyper-parameter");
+  launch_adamw(param, grad, exp_avg, exp_avg_sq, (long long)n, lr, beta1, beta2, eps, weight_decay, step, reinterpret_cast<cudaStream_t>(cuda_stream));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(SWIFTKV_ERR_CUDA, "launch failed: %s", cudaGetErrorString(e));
+  return SWIFTKV_OK;
+}
+
 extern "C" int32_t swiftkv_kv_cache_view(const swiftkv_model *m, int32_t layer, swiftkv_kv_view *out) {
   if (!m || !out) return fail(SWIFTKV_ERR_INVALID_ARG, "null argument");
   if (layer < 0 || layer >= m->cfg.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, m->cfg.n_layers);

@@ -314,6 +314,8 @@ struct DistillArgs {
 };
 size_t distill_workspace_floats(const DistillDims &c, int T, int l);
 void distill_upcast(const void *src_bf16, float *dst, long long n, cudaStream_t st);
+void launch_adamw(float *p, const float *g, float *m, float *v, long long n, float lr, float b1, float b2, float eps, float wd,
+                  int step, cudaStream_t st);
 int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *layers, cudaStream_t st);
 // arrivals: the host's count of barrier arrivals on sync[0] so far (the counter is never reset between launches; zero both
 // together).

@@ -9,6 +9,7 @@
 // is the functional form of the step; the tensor-core GEMMs of the prefill path take 16-bit operands and are not used here.
 // Every output element is owned by one thread block and summed in a fixed order, so gradients repeat bit for bit.
 #include <algorithm>
+#include <cmath>
 #include <vector>
 
 #include "common.cuh"
@@ -279,6 +280,31 @@ __global__ void upcast_kernel(const bf16 *__restrict__ src, float *__restrict__ 
 
 void distill_upcast(const void *src_bf16, float *dst, long long n, cudaStream_t st) {
   if (n > 0) upcast_kernel<<<grid_for(n), 256, 0, st>>>(reinterpret_cast<const bf16 *>(src_bf16), dst, n);
+}
+
+// AdamW with decoupled weight decay, step counted from 1 (bias corrections computed on the host in double):
+//   p <- p (1 - lr wd);  m <- b1 m + (1 - b1) g;  v <- b2 v + (1 - b2) g^2;  p <- p - lr (m / c1) / (sqrt(v / c2) + eps)
+namespace {
+__global__ void adamw_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ m, float *__restrict__ v,
+                             long long n, float lr, float b1, float b2, float nb1, float nb2, float eps, float decay, float inv_c1,
+                             float inv_c2) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const float gi = g[i];
+    const float mi = b1 * m[i] + nb1 * gi;
+    const float vi = b2 * v[i] + nb2 * gi * gi;
+    m[i] = mi;
+    v[i] = vi;
+    p[i] = p[i] * decay - lr * (mi * inv_c1) / (sqrtf(vi * inv_c2) + eps);
+  }
+}
+}  // namespace
+void launch_adamw(float *p, const float *g, float *m, float *v, long long n, float lr, float b1, float b2, float eps, float wd,
+                  int step, cudaStream_t st) {
+  if (n <= 0) return;
+  const double c1 = 1.0 - pow((double)b1, (double)step), c2 = 1.0 - pow((double)b2, (double)step);
+  // (1 - beta as a float subtraction would lose half of beta2's significant digits: everything derived is rounded once, from double)
+  adamw_kernel<<<grid_for(n), 256, 0, st>>>(p, g, m, v, n, lr, b1, b2, (float)(1.0 - (double)b1), (float)(1.0 - (double)b2), eps,
+                                            (float)(1.0 - (double)lr * wd), (float)(1.0 / c1), (float)(1.0 / c2));
 }
 
 size_t distill_workspace_floats(const DistillDims &c, int T, int l) {

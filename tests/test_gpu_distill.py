@@ -164,3 +164,43 @@ def test_argument_checks():
     with pytest.raises((P.SwiftKVError, AssertionError)):
         model.distill_grads(tok, lens, 2, 1, 2.0, st)
     model.close()
+
+
+def test_adamw_update_against_oracle_and_a_short_training_run():
+    """The update that goes with the gradients (AdamW, the paper's lr 3e-4 / weight decay 0.05): elementwise parity with the
+    oracle's formula over three steps, then eight distillation steps on one batch with the student initialised from the
+    original weights -- the loss must fall steadily (knowledge recovery at toy scale, Sec. 3.4)."""
+    import paper_2410_03960_b200 as P
+    rng = np.random.default_rng(9)
+    p0 = rng.standard_normal(10007).astype(np.float32)
+    p, m, v = p0.astype(np.float64), np.zeros(10007), np.zeros(10007)
+    tp, tm, tv = torch.tensor(p0).cuda(), torch.zeros(10007, device="cuda"), torch.zeros(10007, device="cuda")
+    for step in range(1, 4):
+        g = (rng.standard_normal(10007) * 10.0 ** -step).astype(np.float32)
+        f32 = lambda x: float(np.float32(x))                           # the C ABI takes the hyper-parameters as floats  # noqa: E731
+        p, m, v = D.adamw_update(p, g.astype(np.float64), m, v, step, f32(3e-4), f32(0.9), f32(0.999), f32(1e-8), f32(0.05))
+        P.adamw_update(tp, torch.tensor(g).cuda(), tm, tv, step)
+        assert np.abs(to_np(tp) - p).max() <= 2e-6 * np.abs(p).max()
+        assert _rel(to_np(tm).astype(np.float64), m) <= 1e-6 and _rel(to_np(tv).astype(np.float64), v) <= 1e-6
+
+    shape, lens, l, tau = SIX, [40, 23], 2, 2.0
+    w = _scaled_weights(shape, 5, 3.0)
+    wc = S.Weights(shape, torch.float32, w.embed.cuda(), w.final_norm.cuda(), w.lm_head.cuda(),
+                   [{k: t.cuda() for k, t in lw.items()} for lw in w.layers])
+    tok = S.make_prompts(5, lens, shape.vocab)
+    model = P.SwiftKVModel(shape, wc, torch.float32, sum(lens), len(lens), l, 1)
+    st = {name: [None if j < l else wc.layers[j][name].clone() for j in range(shape.n_layers)] for name in ("wq", "wk", "wv")}
+    state = {name: [None if t is None else (torch.zeros_like(t), torch.zeros_like(t)) for t in st[name]] for name in st}
+    losses = []
+    for step in range(1, 9):
+        loss, grads = model.distill_grads(tok, lens, l, 1, tau, st)
+        losses.append(float(loss))
+        for name in st:
+            for j in range(l, shape.n_layers):
+                P.adamw_update(st[name][j].view(-1), grads[name][j].view(-1), state[name][j][0].view(-1), state[name][j][1].view(-1),
+                               step, lr=3e-3, weight_decay=0.05)
+    torch.cuda.synchronize()
+    assert all(b < a for a, b in zip(losses, losses[1:])), losses
+    assert losses[-1] < 0.7 * losses[0], losses
+    print("distillation losses over 8 AdamW steps:", [round(x, 5) for x in losses])
+    model.close()
