@@ -219,17 +219,24 @@ int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t 
  *   grad_w*     : HOST arrays [n_layers] of DEVICE pointers, fp32, same shapes, WRITTEN (not accumulated)
  *   loss        : DEVICE fp32 scalar, written
  *   workspace   : DEVICE, caller-owned, 256-byte aligned, >= swiftkv_distill_workspace_bytes(m, total tokens, swift_layer)
- * The step runs in fp32 on the CUDA cores whatever the model's dtype: a bf16 model's frozen weights are widened into fp32
- * copies inside `workspace` first (its size accounts for them: 4 bytes per model parameter), the student's matrices and
- * the gradients are fp32 either way (master weights).  Gradients repeat bit for bit (every output element is summed by one
- * block in a fixed order).  The model's prefill state (swiftkv_kv_cache_view,
+ * All data is fp32 whatever the model's dtype: a bf16 model's frozen weights are widened into fp32 copies inside `workspace`
+ * first (its size accounts for them: 4 bytes per model parameter), the student's matrices and the gradients are fp32 either
+ * way (master weights).  `precision` selects where the GEMMs (projections, data gradients, weight gradients) run:
+ * SWIFTKV_DISTILL_FP32 on the CUDA cores; SWIFTKV_DISTILL_TF32X3 on the tensor cores (tcgen05 kind::tf32) with every operand
+ * split into an exact sum of two tf32 numbers and three products per GEMM -- results at fp32 accuracy; SWIFTKV_DISTILL_TF32 one
+ * tf32 product per GEMM (operands cut to 10 mantissa bits, gradients good to ~1e-3).  GEMM shapes the tensor-core kernel does
+ * not tile (it needs out-features % 128 == 0 and inner dimension % 32 == 0) stay on the CUDA cores.  Attention, norms, SwiGLU,
+ * RoPE and the loss are fp32 CUDA-core kernels in every mode.  Gradients repeat bit for bit (no atomics).  The model's prefill state (swiftkv_kv_cache_view,
  * swiftkv_first_logits) is invalid afterwards until the next prefill.  The sequence offsets are copied with a blocking
  * copy after synchronising `cuda_stream`; everything else is queued on it.
  * Errors: INVALID_ARG, WORKSPACE_SMALL, CUDA.
  */
 size_t  swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer);
+#define SWIFTKV_DISTILL_FP32   0   /* every GEMM in fp32 on the CUDA cores */
+#define SWIFTKV_DISTILL_TF32X3 1   /* GEMMs on the tensor cores, operands as exact sums of two tf32 numbers (three products): fp32-grade */
+#define SWIFTKV_DISTILL_TF32   2   /* GEMMs on the tensor cores, one tf32 product (10 mantissa bits per operand) */
 int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
-                              int32_t swift_layer, int32_t acrosskv_group, float temperature,
+                              int32_t swift_layer, int32_t acrosskv_group, float temperature, int32_t precision,
                               const void *const *student_wq, const void *const *student_wk, const void *const *student_wv,
                               void *const *grad_wq, void *const *grad_wk, void *const *grad_wv, float *loss,
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
@@ -381,6 +388,13 @@ void swiftkv_model_free(swiftkv_model *m);
  * Needs K % 64 == 0, N % 128 == 0, 16-byte aligned pointers.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
 int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_t M, int32_t N, int32_t K, int32_t dtype,
                         void *cuda_stream);
+
+/* C[M,N] (+)= A[M,K] * B[N,K]^T with fp32 operands on the tensor cores (tcgen05 kind::tf32: sign, exponent and 10 mantissa
+ * bits of every operand enter the product; fp32 accumulation), row-major, ldc = N; accumulate != 0 adds to C.  The GEMM
+ * form of the knowledge-recovery step's tensor-core mode.  Needs K % 32 == 0, N % 128 == 0, 16-byte aligned pointers.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int32_t swiftkv_gemm_tf32(const float *A, const float *B, float *C, int32_t M, int32_t N, int32_t K, int32_t accumulate,
+                          void *cuda_stream);
 
 /* The half-pair operand format of SWIFTKV_ACT_F16_SPLIT, stand-alone.  C[M,N] (DEVICE fp32, row-major, ldc = N) +=
  * (A_hi + A_lo) B^T with A2 DEVICE IEEE half [M, 2K], each row [hi(K) | lo(K)], B IEEE half [N, K]; two tensor-core passes

@@ -5,6 +5,9 @@ PyTorch is used for device memory and streams.
 """
 from .binding import (  # noqa: F401
     ACT_BF16,
+    DISTILL_FP32,
+    DISTILL_TF32,
+    DISTILL_TF32X3,
     ACT_F16,
     ACT_F16_SPLIT,
     SPLIT_ATTN_OUT,
@@ -22,6 +25,7 @@ from .binding import (  # noqa: F401
     attention_prefill_split,
     gemm_tc_split,
     gemm_tc,
+    gemm_tf32,
     library_path,
     load_library,
     quantize_rows_fp8,

@@ -26,8 +26,11 @@ EXPORTS = (
     "swiftkv_tail_attention", "swiftkv_tail_attention_noalloc", "swiftkv_quantize_rows_fp8", "swiftkv_tail_attention_fp8",
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
     "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
-    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait", "swiftkv_adamw_update",
+    "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait", "swiftkv_adamw_update", "swiftkv_gemm_tf32",
 )
+
+
+DISTILL_FP32, DISTILL_TF32X3, DISTILL_TF32 = 0, 1, 2
 
 
 class SwiftKVError(RuntimeError):
@@ -100,12 +103,13 @@ def load_library() -> C.CDLL:
                                      C.c_void_p]
     lib.swiftkv_distill_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
     lib.swiftkv_distill_workspace_bytes.restype = C.c_size_t
-    lib.swiftkv_distill_grads.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float] + [C.c_void_p] * 8 + \
+    lib.swiftkv_distill_grads.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_int32] + [C.c_void_p] * 8 + \
         [C.c_size_t, C.c_void_p]
     lib.swiftkv_gemm_tc_split.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill_split.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_void_p] + [C.c_int32] * 6 + [C.c_void_p]
     lib.swiftkv_gemm_tc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_attention_prefill.argtypes = [C.c_void_p] * 5 + [C.c_int32] * 9 + [C.c_void_p]
+    lib.swiftkv_gemm_tf32.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
     lib.swiftkv_adamw_update.argtypes = [C.c_void_p] * 4 + [C.c_int64, C.c_int32] + [C.c_float] * 5 + [C.c_void_p]
     lib.swiftkv_debug_fused_barrier_wait.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
     lib.swiftkv_debug_bounded_wait.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int32), C.c_void_p]
@@ -290,9 +294,9 @@ class SwiftKVModel:
             _check(self.lib.swiftkv_debug_fused_barrier_wait(self._h, int(limit_clocks), _stream_ptr(stream)))
 
     def distill_grads(self, tokens, seq_lens: Sequence[int], swift_layer: int, acrosskv_group: int, temperature: float,
-                      student: dict, stream: Optional[torch.cuda.Stream] = None):
+                      student: dict, stream: Optional[torch.cuda.Stream] = None, precision: int = 0):
         """swiftkv_distill_grads (Sec. 3.4, Eq. 3).  student: {"wq" | "wk" | "wv": list over layers of fp32 CUDA tensors (None for
-        layers <= swift_layer)}.  Returns (loss tensor [1], {"wq" | "wk" | "wv": list of gradient tensors, None likewise})."""
+        layers <= swift_layer)}; precision: DISTILL_FP32 / DISTILL_TF32X3 / DISTILL_TF32.  Returns (loss tensor [1], {"wq" | "wk" | "wv": list of gradient tensors, None likewise})."""
         L = self.shape.n_layers
         tokens = torch.as_tensor(tokens, dtype=torch.int32).contiguous().to(self.device)
         lens = (C.c_int32 * len(seq_lens))(*[int(n) for n in seq_lens])
@@ -308,7 +312,7 @@ class SwiftKVModel:
                 assert t is None or (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous())
         with torch.cuda.device(self.device):
             _check(self.lib.swiftkv_distill_grads(self._h, tokens.data_ptr(), lens, len(seq_lens), int(swift_layer), int(acrosskv_group),
-                                                  float(temperature), ptrs(student["wq"]), ptrs(student["wk"]), ptrs(student["wv"]),
+                                                  float(temperature), int(precision), ptrs(student["wq"]), ptrs(student["wk"]), ptrs(student["wv"]),
                                                   ptrs(grads["wq"]), ptrs(grads["wk"]), ptrs(grads["wv"]), loss.data_ptr(),
                                                   ws.data_ptr(), nbytes, _stream_ptr(stream)))
             torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
@@ -393,6 +397,18 @@ def attention_prefill_split(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, s
     if out_split:
         return out[:, :n_q * hd].float() + out[:, n_q * hd:].float()
     return out.float()
+
+
+def gemm_tf32(a: torch.Tensor, b: torch.Tensor, out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """swiftkv_gemm_tf32: a [M, K] x b [N, K]^T with fp32 operands on the tensor cores; `out` given: accumulated into."""
+    assert a.is_cuda and b.is_cuda and a.dtype == b.dtype == torch.float32 and a.is_contiguous() and b.is_contiguous()
+    M, K = a.shape
+    N = b.shape[0]
+    acc = out is not None
+    c = out if acc else torch.empty((M, N), dtype=torch.float32, device=a.device)
+    with torch.cuda.device(a.device):
+        _check(load_library().swiftkv_gemm_tf32(a.data_ptr(), b.data_ptr(), c.data_ptr(), M, N, K, int(acc), _stream_ptr(stream)))
+    return c
 
 
 def gemm_tc(a: torch.Tensor, b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:

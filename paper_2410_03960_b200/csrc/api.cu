@@ -1041,7 +1041,7 @@ extern "C" size_t swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_
   return (distill_workspace_floats(distill_dims(m->cfg), total_tokens, swift_layer) + distill_weight_floats(m->cfg)) * sizeof(float);
 }
 extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
-                                         int32_t l, int32_t g, float temperature, const void *const *student_wq,
+                                         int32_t l, int32_t g, float temperature, int32_t precision, const void *const *student_wq,
                                          const void *const *student_wk, const void *const *student_wv, void *const *grad_wq,
                                          void *const *grad_wk, void *const *grad_wv, float *loss, void *workspace,
                                          size_t workspace_bytes, void *cuda_stream) {
@@ -1051,6 +1051,7 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
   if (l < 1 || l > c.n_layers) return fail(SWIFTKV_ERR_INVALID_ARG, "swift_layer %d outside [1, %d]", l, c.n_layers);
   if (g < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "acrosskv_group must be >= 1");
   if (!(temperature > 0.f)) return fail(SWIFTKV_ERR_INVALID_ARG, "temperature must be positive");
+  if (precision < 0 || precision > 2) return fail(SWIFTKV_ERR_INVALID_ARG, "precision must be SWIFTKV_DISTILL_FP32, _TF32X3 or _TF32");
   if (n_seqs < 1 || n_seqs > m->max_seqs) return fail(SWIFTKV_ERR_INVALID_ARG, "n_seqs %d outside [1, %d]", n_seqs, m->max_seqs);
   if ((reinterpret_cast<uintptr_t>(workspace) & 255)) return fail(SWIFTKV_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
   std::vector<int32_t> cu(n_seqs + 1, 0);
@@ -1096,7 +1097,7 @@ extern "C" int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens
   CUDA_TRY(cudaMemcpy(b.cu, cu.data(), (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice));
   launch_positions(b.cu, n_seqs, b.pos, b.last_idx, T, st);
   DistillArgs a{f32(m->embed, (size_t)c.vocab * dd), f32(m->final_norm, dd), f32(m->lm_head, (size_t)c.vocab * dd), tokens, b.cu, b.pos, b.cos_tab,
-                b.sin_tab, T, n_seqs, l, g, temperature, loss, b.status, workspace, workspace_bytes / sizeof(float)};
+                b.sin_tab, T, n_seqs, l, g, precision, temperature, loss, b.status, workspace, main_floats};
   const int rc = run_distill(dims, a, layers.data(), st);
   if (rc) return fail(rc, "distillation step failed: %s", cudaGetErrorString(cudaGetLastError()));
   m->ready = false;      // the prefill state (positions, offsets) has been overwritten
@@ -1289,6 +1290,18 @@ extern "C" int32_t swiftkv_gemm_tc(const void *A, const void *B, void *C, int32_
   const bool f16 = act_dtype == SWIFTKV_DTYPE_F16;
   int rc = launch_gemm_tc(A, f16, M, K, B, N, nullptr, 0, nullptr, 0, out_plain(OUT_STORE, C, N, N), nullptr, 0, nullptr,
                           status, reinterpret_cast<cudaStream_t>(cuda_stream));
+  if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
+  return SWIFTKV_OK;
+}
+
+extern "C" int32_t swiftkv_gemm_tf32(const float *A, const float *B, float *C, int32_t M, int32_t N, int32_t K, int32_t accumulate,
+                                     void *cuda_stream) {
+  if (!A || !B || !C || M < 1 || N < 1 || K < 1) return fail(SWIFTKV_ERR_INVALID_ARG, "bad argument");
+  if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 15) return fail(SWIFTKV_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+  if (!tc_gemm_tf32_supported(M, N, K)) return fail(SWIFTKV_ERR_UNSUPPORTED, "needs K %% 32 == 0 and N %% 128 == 0");
+  unsigned int *status = op_status_word();
+  if (!status) return fail(SWIFTKV_ERR_CUDA, "no status word");
+  int rc = launch_gemm_tc_tf32(A, B, M, N, K, C, accumulate != 0, status, reinterpret_cast<cudaStream_t>(cuda_stream));
   if (rc) return fail(rc, "launch failed: %s", cudaGetErrorString(cudaGetLastError()));
   return SWIFTKV_OK;
 }

@@ -174,6 +174,10 @@ void launch_gemm_simt(const TA *A, const TW *B, int M, int N, int K, OutDesc out
 // gemm_tc.cu : tcgen05 / TMEM / TMA GEMMs (bf16)
 struct TcGemmPlan;   // host object holding tensor maps
 bool tc_gemm_supported(int M, int N, int K);
+// fp32 operands on the tensor cores (kind::tf32, 10 mantissa bits of each operand): out[M, N] (+)= A[M, K] B[N, K]^T
+bool tc_gemm_tf32_supported(int M, int N, int K);
+int launch_gemm_tc_tf32(const float *A, const float *B, int M, int N, int K, float *out, bool accumulate, unsigned int *status,
+                        cudaStream_t st);
 // CTA-pair (cta_group::2) kernels on / off (default on)
 void tc_gemm_use_cta_pairs(bool on, bool swiglu_too);
 // generic: B rows come from up to three matrices stacked along N: [0,nB0) from B0, [nB0, nB0+nB1) from B1, rest B2
@@ -306,6 +310,7 @@ struct DistillArgs {
   const int32_t *tokens, *cu, *pos;      // device: packed token ids, sequence offsets [B + 1], position of every token in its prompt
   const float *cos_tab, *sin_tab;
   int T, B, l, g;
+  int precision;                         // 0 fp32 CUDA cores; 1 tensor cores, split tf32 operands (fp32-grade); 2 tensor cores, plain tf32
   float tau;
   float *loss;                           // device scalar
   unsigned int *status;

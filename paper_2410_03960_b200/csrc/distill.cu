@@ -4,9 +4,11 @@
 // at temperature tau (tau^2 * mean over tokens of KL(softmax(y_t / tau) || softmax(y_s / tau))), and the gradient is taken
 // with respect to the student's W_Q, W_K, W_V only.  Layers 1..l are identical in both modes and run once.
 //
-// fp32 arithmetic throughout (forward with the library's SIMT operators, the backward operators below; a bf16 model's frozen
-// weights are widened to fp32 copies in the workspace first, the student's copies and the gradients are fp32 either way): this
-// is the functional form of the step; the tensor-core GEMMs of the prefill path take 16-bit operands and are not used here.
+// fp32 data throughout (a bf16 model's frozen weights are widened to fp32 copies in the workspace first, the student's copies
+// and the gradients are fp32 either way).  The GEMMs -- every projection forward, every data gradient, the three weight
+// gradients -- run on the CUDA cores (precision 0) or on the tensor cores through the tcgen05 GEMM's kind::tf32 form
+// (precision 1: operands as exact sums of two tf32 numbers, three products, fp32-grade; precision 2: one product, 10
+// mantissa bits per operand); attention forward / backward, norms, SwiGLU, RoPE and the loss stay fp32 CUDA-core kernels.
 // Every output element is owned by one thread block and summed in a fixed order, so gradients repeat bit for bit.
 #include <algorithm>
 #include <cmath>
@@ -272,6 +274,14 @@ __global__ void seq_end_kernel(const int32_t *__restrict__ cu, int n_seqs, int32
 
 inline int grid_for(long long n) { return (int)std::min<long long>((n + 255) / 256, 148 * 8); }
 
+// x = hi + lo exactly, hi = x with the 13 low mantissa bits cleared (what kind::tf32 keeps of an operand), lo = x - hi
+__global__ void split_tf32_kernel(const float *__restrict__ x, float *__restrict__ hi, float *__restrict__ lo, long long n) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    const float v = x[i], h = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
+    hi[i] = h;
+    lo[i] = v - h;
+  }
+}
 __global__ void upcast_kernel(const bf16 *__restrict__ src, float *__restrict__ dst, long long n) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) dst[i] = to_f(src[i]);
 }
@@ -311,8 +321,10 @@ size_t distill_workspace_floats(const DistillDims &c, int T, int l) {
   const size_t d = c.d, dq = (size_t)c.n_q * c.hd, dkv = (size_t)c.n_kv * c.hd, F = c.F, V = c.vocab;
   const size_t per_layer = (size_t)T * (4 * d + 2 * dq + 2 * dkv + 2 * F + d);       // X, h, X1, m, q, att, k, v, gate, up, hs
   const size_t wmax = std::max(std::max(V * d, F * d), dq * d);
+  const size_t amax = (size_t)T * std::max(std::max(d, dq), std::max(F, V));
   const size_t common = (size_t)T * (3 * d + 2 * V + 3 * F + 3 * dq + 4 * dkv + 3 * (size_t)c.n_q + 2 * std::max(std::max(d, dq), F)) + wmax + 2 * T +
-                        128 + 48 * (size_t)(c.L - l + 1);        // (+ the rounding of every piece to 16 bytes)
+                        2 * amax + 2 * wmax +                    // operand halves of the tensor-core modes
+                        160 + 48 * (size_t)(c.L - l + 1);        // (+ the rounding of every piece to 16 bytes)
   return common + (size_t)(c.L - l) * per_layer + (size_t)T * (6 * d + 2 * dq + 2 * dkv + 3 * F);   // (+ the teacher's scratch layer)
 }
 
@@ -339,6 +351,9 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
   const size_t tmax = (size_t)T * std::max(std::max(d, dq), F);
   float *trA = ws.take(tmax), *trB = ws.take(tmax);
   float *wT = ws.take(std::max(std::max((size_t)V * d, (size_t)F * d), (size_t)dq * d));
+  const size_t amax = (size_t)T * std::max(std::max(d, dq), std::max(F, V));
+  const size_t wmax = std::max(std::max((size_t)V * d, (size_t)F * d), (size_t)dq * d);
+  float *a_hi = ws.take(amax), *a_lo = ws.take(amax), *b_hi = ws.take(wmax), *b_lo = ws.take(wmax);
   float *row_loss = ws.take(T);
   int32_t *seq_end = reinterpret_cast<int32_t *>(ws.take(T));
   std::vector<LayerSave> save(L + 1);
@@ -352,7 +367,19 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
   }
   if (ws.p > ws.end) return SWIFTKV_ERR_WORKSPACE_SMALL;
 
+  // out[M, N] (+)= A[M, K] B[N, K]^T.  precision 0: fp32 on the CUDA cores.  1: tensor cores with every operand as an exact sum
+  // of two tf32 numbers, three products (the lo x lo term is below fp32 resolution) -- fp32-grade results.  2: one tf32 product
+  // (operands cut to 10 mantissa bits).  Shapes the tensor-core kernel does not tile keep the CUDA-core kernel.
   auto gemm = [&](const float *A, const float *Bm, int M, int N, int K, float *out, bool accumulate) {
+    if (a.precision != 0 && tc_gemm_tf32_supported(M, N, K) && (size_t)M * K <= amax && (size_t)N * K <= wmax) {
+      if (a.precision == 2) { launch_gemm_tc_tf32(A, Bm, M, N, K, out, accumulate, a.status, st); return; }
+      split_tf32_kernel<<<grid_for((long long)M * K), 256, 0, st>>>(A, a_hi, a_lo, (long long)M * K);
+      split_tf32_kernel<<<grid_for((long long)N * K), 256, 0, st>>>(Bm, b_hi, b_lo, (long long)N * K);
+      launch_gemm_tc_tf32(a_lo, b_hi, M, N, K, out, accumulate, a.status, st);
+      launch_gemm_tc_tf32(a_hi, b_lo, M, N, K, out, true, a.status, st);
+      launch_gemm_tc_tf32(a_hi, b_hi, M, N, K, out, true, a.status, st);
+      return;
+    }
     launch_gemm_simt<float, float>(A, Bm, M, N, K, out_plain(accumulate ? OUT_RESID_ADD_F32 : OUT_STORE_F32, out, N, N), 0, st);
   };
   auto copy = [&](float *dst, const float *src, size_t n) { cudaMemcpyAsync(dst, src, n * sizeof(float), cudaMemcpyDeviceToDevice, st); };

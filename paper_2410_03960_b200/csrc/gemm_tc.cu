@@ -137,6 +137,28 @@ int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t r
   return 0;
 }
 
+// fp32 matrix [rows, cols] row-major: tiles of box_rows x 32 elements (128 bytes), 128-byte swizzle (the tf32 GEMM's operands)
+int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  TmapKey k{p, rows, cols, 0xFFFFFFFDull, box_rows, 32};
+  std::lock_guard<std::mutex> g(g_tmap_mu);
+  auto it = g_tmaps.find(k);
+  if (it != g_tmaps.end()) { *out = it->second; return 0; }
+  if (g_tmaps.size() > 65536) g_tmaps.clear();
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return -1;
+  CUtensorMap m;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 4};
+  cuuint32_t box[2] = {32, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(p), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return -2;
+  g_tmaps.emplace(k, m);
+  *out = m;
+  return 0;
+}
+
 int ensure_dynamic_smem(const void *kernel, int bytes) {
   static std::mutex mu;
   static std::unordered_map<const void *, unsigned long long> done;   // kernel -> bit mask of devices already set
@@ -420,11 +442,14 @@ __device__ __forceinline__ void epilogue_rows(const GemmTcParams &p, uint32_t t_
   }
 }
 
-template <int BN, int STAGES, int EPI>
+// TF32: A and B hold fp32 (tensor maps of fp32 elements, 32 per 128-byte tile row instead of 64; p.K counts 16-bit units, i.e.
+// twice the fp32 K), the MMAs are kind::tf32; everything else -- tile bytes, descriptors, ring, epilogues -- is the same.
+template <int BN, int STAGES, int EPI, bool TF32 = false>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmTcParams p) {
   using L = SmemLayout<BN, STAGES>;
+  constexpr int KSTEP = TF32 ? BK / 2 : BK;      // elements of the operand type per K block
   constexpr bool SWIGLU = (EPI == EPI_SWIGLU);
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -479,8 +504,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           uint8_t *sa = smem + stage * L::STAGE_BYTES;
           uint8_t *sb = sa + L::A_BYTES;
           tc::mbar_expect_tx(fb, L::STAGE_BYTES);
-          tc::tma_load_2d(tc::smem_u32(sa), &tmA, fb, kb * BK, m_blk * BM);
-          const int kx = (kb >= p.kb_wrap ? kb - p.kb_wrap : kb) * BK;      // B's K coordinate (wraps for a split A)
+          tc::tma_load_2d(tc::smem_u32(sa), &tmA, fb, kb * KSTEP, m_blk * BM);
+          const int kx = (kb >= p.kb_wrap ? kb - p.kb_wrap : kb) * KSTEP;      // B's K coordinate (wraps for a split A)
           if constexpr (SWIGLU) {
             tc::tma_load_2d(tc::smem_u32(sb), &tmB0, fb, kx, b_row);                     // gate rows
             tc::tma_load_2d(tc::smem_u32(sb + L::B_BYTES / 2), &tmB1, fb, kx, b_row);   // up rows
@@ -494,7 +519,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     if (lane == 0) {
       // ------------------------------------------------ MMA issuer
-      const uint32_t idesc = tc::umma_idesc(BM, BN, 0, 0, p.f16, p.f16);
+      const uint32_t idesc = TF32 ? tc::umma_idesc_tf32(BM, BN) : tc::umma_idesc(BM, BN, 0, 0, p.f16, p.f16);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
@@ -514,7 +539,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t ad = tc::umma_desc_sw128(a_addr + k * UMMA_K * 2, 16, 1024);
             const uint64_t bd = tc::umma_desc_sw128(b_addr + k * UMMA_K * 2, 16, 1024);
-            tc::umma_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            if constexpr (TF32) tc::umma_ss_tf32(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            else tc::umma_ss(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           tc::umma_commit(tc::smem_u32(&empty_bar[stage]));   // frees the ring slot when these MMAs retire
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -768,6 +794,31 @@ int launch_cfg(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b
 }
 
 }  // namespace
+
+// fp32 operands on the tensor cores (kind::tf32): out[M, N] (+)= A[M, K] B[N, K]^T, fp32 in and out.  N % 128 == 0, K % 32 == 0.
+bool tc_gemm_tf32_supported(int M, int N, int K) { return M >= 1 && K >= 32 && (K % 32) == 0 && (N % 128) == 0; }
+int launch_gemm_tc_tf32(const float *A, const float *B, int M, int N, int K, float *out, bool accumulate, unsigned int *status,
+                        cudaStream_t st) {
+  if (!tc_gemm_tf32_supported(M, N, K)) return SWIFTKV_ERR_UNSUPPORTED;
+  constexpr int BN = 128, STAGES = 6;
+  CUtensorMap ta, tb;
+  if (get_tmap_f32(&ta, A, M, K, BM) || get_tmap_f32(&tb, B, N, K, BN)) return SWIFTKV_ERR_CUDA;
+  if (!accumulate && cudaMemsetAsync(out, 0, (size_t)M * N * sizeof(float), st) != cudaSuccess) return SWIFTKV_ERR_CUDA;
+  GemmTcParams p{};
+  p.M = M; p.N = N; p.K = 2 * K; p.nB0 = N; p.nB1 = 0;
+  p.kb_wrap = 2 * K / BK;
+  p.num_m_blocks = (M + BM - 1) / BM; p.num_n_blocks = N / BN;
+  p.group_m = 32;
+  p.out = out_plain(OUT_RESID_ADD_F32, out, N, N, status);
+  p.status = status;
+  using L = SmemLayout<BN, STAGES>;
+  auto kern = gemm_tc_kernel<BN, STAGES, EPI_PLAIN, true>;
+  if (ensure_dynamic_smem(reinterpret_cast<const void *>(kern), L::TOTAL)) return SWIFTKV_ERR_CUDA;
+  const int tiles = p.num_m_blocks * p.num_n_blocks;
+  const int grid = tiles < num_sms() ? tiles : num_sms();
+  kern<<<grid, GEMM_THREADS, L::TOTAL, st>>>(ta, tb, tb, tb, p);
+  return cudaGetLastError() == cudaSuccess ? SWIFTKV_OK : SWIFTKV_ERR_CUDA;
+}
 
 int launch_bounded_wait_probe(long long limit_clocks, unsigned int *status, unsigned int *outcome, cudaStream_t st) {
   bounded_wait_probe_kernel<<<1, 64, 0, st>>>(limit_clocks, status, outcome);

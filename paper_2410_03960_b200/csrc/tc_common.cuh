@@ -113,6 +113,19 @@ __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// kind::tf32: both operands are fp32 words in shared memory of which the tensor core uses sign, exponent and 10 mantissa bits;
+// one instruction covers K = 8 (32 bytes per row, like K = 16 of the 16-bit kinds), fp32 accumulation
+__host__ __device__ constexpr uint32_t umma_idesc_tf32(int M, int N) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // D[tmem] (+)= A[tmem] * B[smem]; A is read from tensor memory (bf16 packed two per 32-bit column).
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -278,6 +291,7 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t 
                       uint64_t s2, uint32_t b0, uint32_t b1, uint32_t b2);
 // cached map of a weight matrix [N, K] (K % 64 == 0) as [K / 64][N][64] with box (64, 16, chunks), 128-byte swizzle
 int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uint32_t chunks);
+int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows);
 int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t row_slots, uint64_t K, uint32_t steps);
 
 // cached make_tmap_2d_bf16 (tensor maps are pure functions of pointer, shape and box)

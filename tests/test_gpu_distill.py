@@ -84,6 +84,44 @@ def test_loss_and_gradients_against_oracle(shape, lens, l, g, scale):
     model.close()
 
 
+@pytest.mark.parametrize("precision,loss_bar,grad_bar", [(1, 2e-5, 5e-5), (2, 5e-3, 2e-2)])
+@pytest.mark.parametrize("lens,l,g", [([64, 32], 2, 1), ([96, 31, 1], 1, 2)])
+def test_tensor_core_modes_against_oracle(precision, loss_bar, grad_bar, lens, l, g):
+    """The GEMMs of the step on the tensor cores (tcgen05 kind::tf32).  Split operands (each an exact sum of two tf32 numbers,
+    three products): the same bars as the fp32 mode.  Plain tf32 (operands cut to 10 mantissa bits, 2^-10 relative each,
+    systematic because the hardware truncates): gradients to 2e-2.  MID's widths are multiples of 128, so every projection and
+    data gradient runs on the tensor-core kernel; the weight gradients do when the token count is a multiple of 32 (96), and
+    fall back to the CUDA-core kernel otherwise (128)."""
+    import paper_2410_03960_b200 as P
+    shape, seed, tau = MID, 29, 2.0
+    w = _scaled_weights(shape, seed, 2.0)
+    tok = S.make_prompts(seed, lens, shape.vocab)
+    st = _student(w, l, seed + 1, 0.3)
+    want_loss, want = D.distill_grads(oracle_config(shape), oracle_weights(w),
+                                      {k: [None if t is None else t.double().numpy() for t in v] for k, v in st.items()},
+                                      tok.numpy(), lens, l, g, tau)
+    wc = S.Weights(shape, torch.float32, w.embed.cuda(), w.final_norm.cuda(), w.lm_head.cuda(),
+                   [{k: v.cuda() for k, v in lw.items()} for lw in w.layers])
+    model = P.SwiftKVModel(shape, wc, torch.float32, sum(lens), len(lens), l, g)
+    st_gpu = {k: [None if t is None else t.cuda() for t in v] for k, v in st.items()}
+    loss, grads = model.distill_grads(tok, lens, l, g, tau, st_gpu, precision=precision)
+    model.status()
+    assert abs(float(loss) - want_loss) <= loss_bar * want_loss, (float(loss), want_loss)
+    worst = 0.0
+    for name in ("wq", "wk", "wv"):
+        for j in range(l, shape.n_layers):
+            got, ref = to_np(grads[name][j]).astype(np.float64), want[name][j]
+            if np.abs(ref).max() == 0.0:
+                assert np.abs(got).max() == 0.0
+                continue
+            worst = max(worst, _rel(got, ref))
+            assert _rel(got, ref) <= grad_bar, (name, j, _rel(got, ref))
+    print(f"distill precision {precision} lens {lens}: loss rel {abs(float(loss) - want_loss) / want_loss:.2e}, worst gradient rel-L2 {worst:.2e}")
+    loss2, grads2 = model.distill_grads(tok, lens, l, g, tau, st_gpu, precision=precision)
+    assert torch.equal(loss, loss2) and all(torch.equal(a, b) for n_ in grads for a, b in zip(grads[n_], grads2[n_]) if a is not None)
+    model.close()
+
+
 def test_unrewired_student_has_no_loss_and_a_gradient_step_lowers_the_loss():
     import paper_2410_03960_b200 as P
     shape, lens, tau = SIX, [30, 11], 2.0

@@ -30,6 +30,33 @@ def test_gemm_tcgen05(M, N, K, act):
     assert np.max(np.abs(got - ref)) <= ulp * np.max(np.abs(ref)) + 1e-3
 
 
+@pytest.mark.parametrize("M,N,K", [(200, 128, 32), (1000, 384, 4096), (77, 1024, 160), (4096, 256, 2048)])
+def test_gemm_tf32_tcgen05(M, N, K):
+    """fp32 operands on the tensor cores (kind::tf32): each operand enters with 10 mantissa bits, the products are summed in
+    fp32.  Against the fp64 product of the fp32 inputs the error of one term is at most 2 * 2^-10 relative (two truncated or
+    rounded operands); against the fp64 product of inputs whose low 13 mantissa bits are cleared it is fp32 summation noise
+    if the hardware truncates -- either way bounded by the first figure, and far from a 16-bit operand's 2^-8."""
+    import paper_2410_03960_b200 as P
+    a = S.matrix(12, 1, M, K, torch.float32, "cuda", std=1.0)
+    b = S.matrix(12, 2, N, K, torch.float32, "cuda", std=1.0)
+    c = P.gemm_tf32(a, b)
+    torch.cuda.synchronize()
+    ref = to_np(a) @ to_np(b).T
+    got = to_np(c)
+    assert np.isfinite(got).all()
+    assert rel_l2(got, ref) <= 1.5e-3, rel_l2(got, ref)
+    # accumulate form
+    c2 = P.gemm_tf32(a, b, out=c.clone())
+    torch.cuda.synchronize()
+    assert rel_l2(to_np(c2), 2.0 * ref) <= 1.5e-3
+    # the product of the truncated inputs pins the operand handling more tightly (either rounding mode gives < 6e-4)
+    def trunc(x):
+        return (x.view(torch.int32) & ~0x1FFF).view(torch.float32)
+    ref_t = to_np(trunc(a)) @ to_np(trunc(b)).T
+    print(f"tf32 gemm {M}x{N}x{K}: rel-L2 vs exact {rel_l2(got, ref):.2e}, vs truncated operands {rel_l2(got, ref_t):.2e}")
+    assert min(rel_l2(got, ref), rel_l2(got, ref_t)) <= 6e-4
+
+
 @pytest.mark.parametrize("qdtype,dtype,bar", [(torch.float32, torch.float32, 1e-5), (torch.bfloat16, torch.bfloat16, 1e-2),
                                               (torch.float16, torch.bfloat16, 1e-3)])
 @pytest.mark.parametrize("lens,n_q,n_kv,hd", [([5, 1, 70], 8, 2, 32), ([33, 64], 4, 4, 64), ([130], 8, 2, 128)])
