@@ -113,8 +113,50 @@ __global__ void add_kernel(float *__restrict__ dst, const float *__restrict__ sr
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) dst[i] += src[i];
 }
 
-// One warp per (query token, query head).  Recomputes the row's scores against its prompt's keys (two passes: maximum and
-// sum, then the gradient), writes dq and the row's (max, sum, D = dO . O) for the key-side kernel.
+// Causal attention forward, one warp per (query token, query head): a single pass over the prompt's keys with a running
+// maximum, sum and output (the library's generic fp32 attention kernel took half of the step).  Writes the output row and
+// the row's (maximum, sum) for the backward pass.
+template <int MAX_E>
+__global__ void __launch_bounds__(128) attn_fwd_kernel(const float *__restrict__ q, const float *__restrict__ k,
+                                                       const float *__restrict__ v, float *__restrict__ o, float *__restrict__ stat,
+                                                       const int32_t *__restrict__ pos, int n_tokens, int n_q, int n_kv, int hd,
+                                                       float scale) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long item = (long long)blockIdx.x * 4 + warp;
+  if (item >= (long long)n_tokens * n_q) return;
+  const int tok = (int)(item / n_q), h = (int)(item % n_q), kvh = h / (n_q / n_kv);
+  const int p = pos[tok], first = tok - p;                  // the prompt's first packed row
+  float qe[MAX_E], acc[MAX_E];
+#pragma unroll
+  for (int e = 0; e < MAX_E; ++e) {
+    const int dd = lane + 32 * e;
+    qe[e] = dd < hd ? q[((size_t)tok * n_q + h) * hd + dd] * scale : 0.f;
+    acc[e] = 0.f;
+  }
+  float m = -INFINITY, l = 0.f;
+  for (int j = 0; j <= p; ++j) {
+    const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd, *vr = v + ((size_t)(first + j) * n_kv + kvh) * hd;
+    float s = 0.f;
+#pragma unroll
+    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) s = fmaf(qe[e], kr[dd], s); }
+    s = warp_sum(s);
+    const float m_new = fmaxf(m, s), corr = expf(m - m_new), pj = expf(s - m_new);
+    l = l * corr + pj;
+#pragma unroll
+    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) acc[e] = fmaf(pj, vr[dd], acc[e] * corr); }
+    m = m_new;
+  }
+  const float inv = 1.f / l;
+#pragma unroll
+  for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) o[((size_t)tok * n_q + h) * hd + dd] = acc[e] * inv; }
+  if (lane == 0 && stat) {
+    float *st = stat + ((size_t)tok * n_q + h) * 3;
+    st[0] = m; st[1] = l;
+  }
+}
+
+// Backward, query side: one warp per (query token, query head), with the forward pass's (maximum, sum) of the row; writes dq
+// and D = dO . O next to them for the key-side kernel.
 template <int MAX_E>
 __global__ void __launch_bounds__(128) attn_bwd_q_kernel(const float *__restrict__ q, const float *__restrict__ k,
                                                          const float *__restrict__ v, const float *__restrict__ o,
@@ -138,22 +180,8 @@ __global__ void __launch_bounds__(128) attn_bwd_q_kernel(const float *__restrict
     acc[e] = 0.f;
   }
   D = warp_sum(D);
-  float m = -INFINITY;
-  for (int j = 0; j <= p; ++j) {
-    const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd;
-    float s = 0.f;
-#pragma unroll
-    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) s = fmaf(qe[e], kr[dd], s); }
-    m = fmaxf(m, warp_sum(s) * scale);
-  }
-  float l = 0.f;
-  for (int j = 0; j <= p; ++j) {
-    const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd;
-    float s = 0.f;
-#pragma unroll
-    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) s = fmaf(qe[e], kr[dd], s); }
-    l += expf(warp_sum(s) * scale - m);
-  }
+  float *st = stat + ((size_t)tok * n_q + h) * 3;
+  const float m = st[0], inv_l = 1.f / st[1];
   for (int j = 0; j <= p; ++j) {
     const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd, *vr = v + ((size_t)(first + j) * n_kv + kvh) * hd;
     float s = 0.f, dp = 0.f;
@@ -162,17 +190,14 @@ __global__ void __launch_bounds__(128) attn_bwd_q_kernel(const float *__restrict
       const int dd = lane + 32 * e;
       if (dd < hd) { s = fmaf(qe[e], kr[dd], s); dp = fmaf(doe[e], vr[dd], dp); }
     }
-    const float pij = expf(warp_sum(s) * scale - m) / l;
+    const float pij = expf(warp_sum(s) * scale - m) * inv_l;
     const float ds = pij * (warp_sum(dp) - D) * scale;
 #pragma unroll
     for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) acc[e] = fmaf(ds, kr[dd], acc[e]); }
   }
 #pragma unroll
   for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) dq[((size_t)tok * n_q + h) * hd + dd] = acc[e]; }
-  if (lane == 0) {
-    float *st = stat + ((size_t)tok * n_q + h) * 3;
-    st[0] = m; st[1] = l; st[2] = D;
-  }
+  if (lane == 0) st[2] = D;
 }
 
 // One warp per (key token, KV head): every later query of the prompt, every query head of the group, in a fixed order.
@@ -319,13 +344,13 @@ void launch_adamw(float *p, const float *g, float *m, float *v, long long n, flo
 
 size_t distill_workspace_floats(const DistillDims &c, int T, int l) {
   const size_t d = c.d, dq = (size_t)c.n_q * c.hd, dkv = (size_t)c.n_kv * c.hd, F = c.F, V = c.vocab;
-  const size_t per_layer = (size_t)T * (4 * d + 2 * dq + 2 * dkv + 2 * F + d);       // X, h, X1, m, q, att, k, v, gate, up, hs
+  const size_t per_layer = (size_t)T * (4 * d + 2 * dq + 2 * dkv + 2 * F + d + 3 * (size_t)c.n_q);   // X, h, X1, m, q, att, k, v, gate, up, hs, row statistics
   const size_t wmax = std::max(std::max(V * d, F * d), dq * d);
   const size_t amax = (size_t)T * std::max(std::max(d, dq), std::max(F, V));
   const size_t common = (size_t)T * (3 * d + 2 * V + 3 * F + 3 * dq + 4 * dkv + 3 * (size_t)c.n_q + 2 * std::max(std::max(d, dq), F)) + wmax + 2 * T +
                         2 * amax + 2 * wmax +                    // operand halves of the tensor-core modes
                         160 + 48 * (size_t)(c.L - l + 1);        // (+ the rounding of every piece to 16 bytes)
-  return common + (size_t)(c.L - l) * per_layer + (size_t)T * (6 * d + 2 * dq + 2 * dkv + 3 * F);   // (+ the teacher's scratch layer)
+  return common + (size_t)(c.L - l) * per_layer + (size_t)T * (6 * d + 2 * dq + 2 * dkv + 3 * F + 3 * (size_t)c.n_q);   // (+ the teacher's scratch layer)
 }
 
 namespace {
@@ -333,7 +358,7 @@ struct Bump {
   float *p, *end;
   float *take(size_t n) { float *r = p; p += (n + 3) & ~(size_t)3; return p <= end ? r : nullptr; }
 };
-struct LayerSave { float *X, *h, *q, *att, *X1, *m, *gate, *up, *hs, *k, *v; };
+struct LayerSave { float *X, *h, *q, *att, *X1, *m, *gate, *up, *hs, *k, *v, *stat; };
 }  // namespace
 
 int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *layers, cudaStream_t st) {
@@ -347,7 +372,6 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
   float *t_F0 = ws.take((size_t)T * F), *t_F1 = ws.take((size_t)T * F), *t_F2 = ws.take((size_t)T * F);
   float *da = ws.take((size_t)T * dq), *dqb = ws.take((size_t)T * dq), *t_q = ws.take((size_t)T * dq);
   float *dk = ws.take((size_t)T * dkv), *dv = ws.take((size_t)T * dkv), *dks = ws.take((size_t)T * dkv), *dvs = ws.take((size_t)T * dkv);
-  float *stat = ws.take((size_t)T * nq * 3);
   const size_t tmax = (size_t)T * std::max(std::max(d, dq), F);
   float *trA = ws.take(tmax), *trB = ws.take(tmax);
   float *wT = ws.take(std::max(std::max((size_t)V * d, (size_t)F * d), (size_t)dq * d));
@@ -364,6 +388,7 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
     s.q = ws.take((size_t)T * dq); s.att = ws.take((size_t)T * dq);
     s.k = ws.take((size_t)T * dkv); s.v = ws.take((size_t)T * dkv);
     s.gate = ws.take((size_t)T * F); s.up = ws.take((size_t)T * F);
+    s.stat = ws.take((size_t)T * nq * 3);
   }
   if (ws.p > ws.end) return SWIFTKV_ERR_WORKSPACE_SMALL;
 
@@ -419,7 +444,13 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
       launch_rope<float>(s.k, 0, 1, a.pos, nullptr, a.cos_tab, a.sin_tab, T, nkv, hd, st);
       kk = s.k; vv = s.v;
     }
-    launch_attention_simple<float, float>(s.q, kk, vv, s.att, a.cu, B, nullptr, nullptr, nullptr, 0, T, nq, nkv, hd, st);
+    {
+      const unsigned blocks = (unsigned)(((long long)T * nq + 3) / 4);
+      if (hd <= 32) attn_fwd_kernel<1><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
+      else if (hd <= 64) attn_fwd_kernel<2><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
+      else if (hd <= 128) attn_fwd_kernel<4><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
+      else attn_fwd_kernel<8><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
+    }
     gemm(s.att, w.wo, T, d, dq, x, true);
     copy(s.X1, x, (size_t)T * d);
     launch_rmsnorm<float, float>(x, w.post_norm, s.m, T, d, c.eps, st);
@@ -470,9 +501,9 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
     const LayerSave &ld = save[r];
 #define SKV_ATT_BWD(E)                                                                                                          \
     do {                                                                                                                        \
-      attn_bwd_q_kernel<E><<<(unsigned)(((long long)T * nq + 3) / 4), 128, 0, st>>>(s.q, ld.k, ld.v, s.att, da, dqb, stat, a.pos, T, nq, \
+      attn_bwd_q_kernel<E><<<(unsigned)(((long long)T * nq + 3) / 4), 128, 0, st>>>(s.q, ld.k, ld.v, s.att, da, dqb, s.stat, a.pos, T, nq, \
                                                                                      nkv, hd, scale);                           \
-      attn_bwd_kv_kernel<E><<<(unsigned)(((long long)T * nkv + 3) / 4), 128, 0, st>>>(s.q, ld.k, ld.v, da, stat, dks, dvs, a.pos,  \
+      attn_bwd_kv_kernel<E><<<(unsigned)(((long long)T * nkv + 3) / 4), 128, 0, st>>>(s.q, ld.k, ld.v, da, s.stat, dks, dvs, a.pos,  \
                                                                                        seq_end, T, nq, nkv, hd, scale);         \
     } while (0)
     if (hd <= 32) SKV_ATT_BWD(1); else if (hd <= 64) SKV_ATT_BWD(2); else if (hd <= 128) SKV_ATT_BWD(4); else SKV_ATT_BWD(8);
