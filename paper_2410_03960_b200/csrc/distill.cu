@@ -113,45 +113,93 @@ __global__ void add_kernel(float *__restrict__ dst, const float *__restrict__ sr
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) dst[i] += src[i];
 }
 
-// Causal attention forward, one warp per (query token, query head): a single pass over the prompt's keys with a running
-// maximum, sum and output (the library's generic fp32 attention kernel took half of the step).  Writes the output row and
-// the row's (maximum, sum) for the backward pass.
+// Causal attention forward: one warp per (four consecutive query tokens, query head), a single pass over the prompt's keys
+// with a running maximum, sum and output per row.  Every K / V row is read once for the four queries (a warp per single query
+// re-read the whole prefix from L2 and was bound by that); rows of the group that belong to another prompt than its first
+// row are done in a pass of their own.  Writes the output rows and each row's (maximum, sum) for the backward pass.
 template <int MAX_E>
 __global__ void __launch_bounds__(128) attn_fwd_kernel(const float *__restrict__ q, const float *__restrict__ k,
                                                        const float *__restrict__ v, float *__restrict__ o, float *__restrict__ stat,
                                                        const int32_t *__restrict__ pos, int n_tokens, int n_q, int n_kv, int hd,
                                                        float scale) {
+  constexpr int R = 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_groups = (n_tokens + R - 1) / R;
   const long long item = (long long)blockIdx.x * 4 + warp;
-  if (item >= (long long)n_tokens * n_q) return;
-  const int tok = (int)(item / n_q), h = (int)(item % n_q), kvh = h / (n_q / n_kv);
-  const int p = pos[tok], first = tok - p;                  // the prompt's first packed row
-  float qe[MAX_E], acc[MAX_E];
+  if (item >= (long long)n_groups * n_q) return;
+  const int grp = (int)(item / n_q), h = (int)(item % n_q), kvh = h / (n_q / n_kv);
+  const int tok0 = grp * R;
+  int p_r[R], first_r[R];
 #pragma unroll
-  for (int e = 0; e < MAX_E; ++e) {
-    const int dd = lane + 32 * e;
-    qe[e] = dd < hd ? q[((size_t)tok * n_q + h) * hd + dd] * scale : 0.f;
-    acc[e] = 0.f;
+  for (int r = 0; r < R; ++r) {
+    const int tok = tok0 + r;
+    p_r[r] = tok < n_tokens ? pos[tok] : -1;
+    first_r[r] = tok - p_r[r];
   }
-  float m = -INFINITY, l = 0.f;
-  for (int j = 0; j <= p; ++j) {
-    const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd, *vr = v + ((size_t)(first + j) * n_kv + kvh) * hd;
-    float s = 0.f;
+  unsigned todo = 0;
 #pragma unroll
-    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) s = fmaf(qe[e], kr[dd], s); }
-    s = warp_sum(s);
-    const float m_new = fmaxf(m, s), corr = expf(m - m_new), pj = expf(s - m_new);
-    l = l * corr + pj;
+  for (int r = 0; r < R; ++r) if (p_r[r] >= 0) todo |= 1u << r;
+  while (todo) {
+    const int lead = __ffs(todo) - 1;
+    const int first = first_r[lead];
+    unsigned act = 0;
+    int p_max = 0;
 #pragma unroll
-    for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) acc[e] = fmaf(pj, vr[dd], acc[e] * corr); }
-    m = m_new;
-  }
-  const float inv = 1.f / l;
+    for (int r = 0; r < R; ++r)
+      if (((todo >> r) & 1u) && first_r[r] == first) { act |= 1u << r; p_max = max(p_max, p_r[r]); }
+    todo &= ~act;
+    float qe[R][MAX_E], acc[R][MAX_E], m[R], l[R];
 #pragma unroll
-  for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) o[((size_t)tok * n_q + h) * hd + dd] = acc[e] * inv; }
-  if (lane == 0 && stat) {
-    float *st = stat + ((size_t)tok * n_q + h) * 3;
-    st[0] = m; st[1] = l;
+    for (int r = 0; r < R; ++r) {
+      m[r] = -INFINITY; l[r] = 0.f;
+#pragma unroll
+      for (int e = 0; e < MAX_E; ++e) {
+        const int dd = lane + 32 * e;
+        qe[r][e] = (((act >> r) & 1u) && dd < hd) ? q[((size_t)(tok0 + r) * n_q + h) * hd + dd] * scale : 0.f;
+        acc[r][e] = 0.f;
+      }
+    }
+    for (int j = 0; j <= p_max; ++j) {
+      const float *kr = k + ((size_t)(first + j) * n_kv + kvh) * hd, *vr = v + ((size_t)(first + j) * n_kv + kvh) * hd;
+      float ke[MAX_E], ve[MAX_E], s[R];
+#pragma unroll
+      for (int e = 0; e < MAX_E; ++e) {
+        const int dd = lane + 32 * e;
+        ke[e] = dd < hd ? kr[dd] : 0.f;
+        ve[e] = dd < hd ? vr[dd] : 0.f;
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        s[r] = 0.f;
+#pragma unroll
+        for (int e = 0; e < MAX_E; ++e) s[r] = fmaf(qe[r][e], ke[e], s[r]);
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) s[r] = warp_sum(s[r]);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (((act >> r) & 1u) && j <= p_r[r]) {
+          const float m_new = fmaxf(m[r], s[r]), corr = expf(m[r] - m_new), pj = expf(s[r] - m_new);
+          l[r] = l[r] * corr + pj;
+#pragma unroll
+          for (int e = 0; e < MAX_E; ++e) acc[r][e] = fmaf(pj, ve[e], acc[r][e] * corr);
+          m[r] = m_new;
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if ((act >> r) & 1u) {
+        const int tok = tok0 + r;
+        const float inv = 1.f / l[r];
+#pragma unroll
+        for (int e = 0; e < MAX_E; ++e) { const int dd = lane + 32 * e; if (dd < hd) o[((size_t)tok * n_q + h) * hd + dd] = acc[r][e] * inv; }
+        if (lane == 0 && stat) {
+          float *st = stat + ((size_t)tok * n_q + h) * 3;
+          st[0] = m[r]; st[1] = l[r];
+        }
+      }
+    }
   }
 }
 
@@ -445,7 +493,7 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
       kk = s.k; vv = s.v;
     }
     {
-      const unsigned blocks = (unsigned)(((long long)T * nq + 3) / 4);
+      const unsigned blocks = (unsigned)(((long long)((T + 3) / 4) * nq + 3) / 4);      // a warp per (4 tokens, head), 4 warps per block
       if (hd <= 32) attn_fwd_kernel<1><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
       else if (hd <= 64) attn_fwd_kernel<2><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
       else if (hd <= 128) attn_fwd_kernel<4><<<blocks, 128, 0, st>>>(s.q, kk, vv, s.att, s.stat, a.pos, T, nq, nkv, hd, scale);
