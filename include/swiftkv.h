@@ -223,7 +223,7 @@ int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t 
  * first (its size accounts for them: 4 bytes per model parameter), the student's matrices and the gradients are fp32 either
  * way (master weights).  `precision` selects where the GEMMs (projections, data gradients, weight gradients) run:
  * SWIFTKV_DISTILL_FP32 on the CUDA cores; SWIFTKV_DISTILL_TF32X3 on the tensor cores (tcgen05 kind::tf32) with every operand
- * split into an exact sum of two tf32 numbers and three products per GEMM -- results at fp32 accuracy; SWIFTKV_DISTILL_TF32 one
+ * split into two tf32 numbers (x rounded to nearest, and the rounded remainder) and three products per GEMM -- results at fp32 accuracy; SWIFTKV_DISTILL_TF32 one
  * tf32 product per GEMM (operands cut to 10 mantissa bits, gradients good to ~1e-3).  GEMM shapes the tensor-core kernel does
  * not tile (it needs out-features % 128 == 0 and inner dimension % 32 == 0) stay on the CUDA cores.  Attention, norms, SwiGLU,
  * RoPE and the loss are fp32 CUDA-core kernels in every mode.  Gradients repeat bit for bit (no atomics).  The model's prefill state (swiftkv_kv_cache_view,
@@ -233,7 +233,7 @@ int32_t swiftkv_simscore(swiftkv_model *m, const int32_t *tokens, const int32_t 
  */
 size_t  swiftkv_distill_workspace_bytes(const swiftkv_model *m, int32_t total_tokens, int32_t swift_layer);
 #define SWIFTKV_DISTILL_FP32   0   /* every GEMM in fp32 on the CUDA cores */
-#define SWIFTKV_DISTILL_TF32X3 1   /* GEMMs on the tensor cores, operands as exact sums of two tf32 numbers (three products): fp32-grade */
+#define SWIFTKV_DISTILL_TF32X3 1   /* GEMMs on the tensor cores, operands as sums of two tf32 numbers (three products): fp32-grade */
 #define SWIFTKV_DISTILL_TF32   2   /* GEMMs on the tensor cores, one tf32 product (10 mantissa bits per operand) */
 int32_t swiftkv_distill_grads(swiftkv_model *m, const int32_t *tokens, const int32_t *seq_lens, int32_t n_seqs,
                               int32_t swift_layer, int32_t acrosskv_group, float temperature, int32_t precision,

@@ -176,8 +176,10 @@ struct TcGemmPlan;   // host object holding tensor maps
 bool tc_gemm_supported(int M, int N, int K);
 // fp32 operands on the tensor cores (kind::tf32, 10 mantissa bits of each operand): out[M, N] (+)= A[M, K] B[N, K]^T
 bool tc_gemm_tf32_supported(int M, int N, int K);
+// k_chunk > 0 (a multiple of 32): one launch per k_chunk of the inner dimension, summed by the epilogue's fp32 add -- the tensor
+// core's own accumulation cuts instead of rounding, an error that grows with the length of the chain
 int launch_gemm_tc_tf32(const float *A, const float *B, int M, int N, int K, float *out, bool accumulate, unsigned int *status,
-                        cudaStream_t st);
+                        cudaStream_t st, int k_chunk = 0);
 // CTA-pair (cta_group::2) kernels on / off (default on)
 void tc_gemm_use_cta_pairs(bool on, bool swiglu_too);
 // generic: B rows come from up to three matrices stacked along N: [0,nB0) from B0, [nB0, nB0+nB1) from B1, rest B2

@@ -347,12 +347,19 @@ __global__ void seq_end_kernel(const int32_t *__restrict__ cu, int n_seqs, int32
 
 inline int grid_for(long long n) { return (int)std::min<long long>((n + 255) / 256, 148 * 8); }
 
-// x = hi + lo exactly, hi = x with the 13 low mantissa bits cleared (what kind::tf32 keeps of an operand), lo = x - hi
+// x ~ hi + lo, both representable in tf32 (10 mantissa bits): hi = x rounded to nearest, lo = (x - hi) rounded to nearest, so
+// that the tensor core's own cut of the 13 low bits changes neither.  What is lost is at most 2^-22 |x| and has no preferred
+// sign (cutting instead of rounding loses up to 2^-20 |x|, always toward zero, which adds up over sums of thousands of terms).
+__device__ __forceinline__ float round_tf32(float v) {
+  const uint32_t u = __float_as_uint(v);
+  if ((u & 0x7F800000u) == 0x7F800000u) return v;      // inf / nan pass
+  return __uint_as_float((u + 0x1000u) & 0xFFFFE000u);
+}
 __global__ void split_tf32_kernel(const float *__restrict__ x, float *__restrict__ hi, float *__restrict__ lo, long long n) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-    const float v = x[i], h = __uint_as_float(__float_as_uint(v) & 0xFFFFE000u);
+    const float v = x[i], h = round_tf32(v);
     hi[i] = h;
-    lo[i] = v - h;
+    lo[i] = round_tf32(v - h);
   }
 }
 __global__ void upcast_kernel(const bf16 *__restrict__ src, float *__restrict__ dst, long long n) {
@@ -448,9 +455,10 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
       if (a.precision == 2) { launch_gemm_tc_tf32(A, Bm, M, N, K, out, accumulate, a.status, st); return; }
       split_tf32_kernel<<<grid_for((long long)M * K), 256, 0, st>>>(A, a_hi, a_lo, (long long)M * K);
       split_tf32_kernel<<<grid_for((long long)N * K), 256, 0, st>>>(Bm, b_hi, b_lo, (long long)N * K);
+      // (accumulation chains of at most 1024: longer ones lose more to the tensor core's cut-off add than the split gains)
       launch_gemm_tc_tf32(a_lo, b_hi, M, N, K, out, accumulate, a.status, st);
       launch_gemm_tc_tf32(a_hi, b_lo, M, N, K, out, true, a.status, st);
-      launch_gemm_tc_tf32(a_hi, b_hi, M, N, K, out, true, a.status, st);
+      launch_gemm_tc_tf32(a_hi, b_hi, M, N, K, out, true, a.status, st, 1024);
       return;
     }
     launch_gemm_simt<float, float>(A, Bm, M, N, K, out_plain(accumulate ? OUT_RESID_ADD_F32 : OUT_STORE_F32, out, N, N), 0, st);

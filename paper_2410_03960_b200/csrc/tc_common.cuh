@@ -291,7 +291,7 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t 
                       uint64_t s2, uint32_t b0, uint32_t b1, uint32_t b2);
 // cached map of a weight matrix [N, K] (K % 64 == 0) as [K / 64][N][64] with box (64, 16, chunks), 128-byte swizzle
 int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uint32_t chunks);
-int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t ld = 0);      // ld: row stride in elements (0: cols)
 int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t row_slots, uint64_t K, uint32_t steps);
 
 // cached make_tmap_2d_bf16 (tensor maps are pure functions of pointer, shape and box)
