@@ -340,6 +340,18 @@ int32_t swiftkv_set_kernel_mask(swiftkv_model *m, int32_t mask);
 #define SWIFTKV_ACT_F16_SPLIT 2
 int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t format);
 
+/* Optional room for the half copies of the weights (SWIFTKV_ACT_F16 on a bf16 model).  Without it every prefill / chunk step
+ * copies each of its layers' seven matrices to half right before use (one layer of scratch, on a side stream): 2 x 2 bytes
+ * per parameter of layers 1..l of HBM traffic per step, noticeable when steps are small (chunks of a few thousand tokens).
+ * With a DEVICE buffer of swiftkv_half_weight_cache_bytes(cfg, n) bytes (256-byte aligned, owned by the caller, alive until
+ * the model is destroyed or the cache is replaced) the copies of the first n layers are made once, by the first step that
+ * needs them, and reused by every later step whose SwiftKV layer l is <= n; a step with l > n falls back to per-step copies.
+ * The library cannot see the caller changing the model's weights: call swiftkv_set_half_weight_cache again (same buffer is
+ * fine) after updating them, which marks every copy stale.  buffer = NULL, bytes = 0 removes the cache.  The results are
+ * bit-identical with and without it.  swiftkv_half_weight_cache_bytes returns -1 for a bad config. */
+int64_t swiftkv_half_weight_cache_bytes(const swiftkv_config *cfg, int32_t n_layers);
+int32_t swiftkv_set_half_weight_cache(swiftkv_model *m, void *buffer, int64_t bytes);
+
 /* Operands that travel as half pairs under SWIFTKV_ACT_F16_SPLIT (bits; call after swiftkv_set_activation_format):
  *   QKV_INPUT : the normed hidden state that feeds the Q/K/V projections and the SingleInputKV projection (those GEMMs x2)
  *   SCORES    : q and K inside the attention kernel (Q K^T x3)

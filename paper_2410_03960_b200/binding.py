@@ -27,6 +27,7 @@ EXPORTS = (
     "swiftkv_debug_bounded_wait", "swiftkv_op_status", "swiftkv_set_split_mask",
     "swiftkv_gemm_tc_split", "swiftkv_attention_prefill_split", "swiftkv_simscore_scratch_bytes", "swiftkv_simscore",
     "swiftkv_distill_workspace_bytes", "swiftkv_distill_grads", "swiftkv_debug_fused_barrier_wait", "swiftkv_adamw_update", "swiftkv_gemm_tf32",
+    "swiftkv_half_weight_cache_bytes", "swiftkv_set_half_weight_cache",
 )
 
 
@@ -97,6 +98,9 @@ def load_library() -> C.CDLL:
     lib.swiftkv_model_free.restype = None
     lib.swiftkv_set_activation_format.argtypes = [C.c_void_p, C.c_int32]
     lib.swiftkv_set_split_mask.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_half_weight_cache_bytes.argtypes = [C.c_void_p, C.c_int32]
+    lib.swiftkv_half_weight_cache_bytes.restype = C.c_int64
+    lib.swiftkv_set_half_weight_cache.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
     lib.swiftkv_simscore_scratch_bytes.argtypes = [C.c_void_p, C.c_int32]
     lib.swiftkv_simscore_scratch_bytes.restype = C.c_size_t
     lib.swiftkv_simscore.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p,
@@ -348,6 +352,19 @@ class SwiftKVModel:
     def set_split_mask(self, mask: int) -> None:
         """swiftkv_set_split_mask: which operands travel as half pairs (SPLIT_* bits)."""
         _check(self.lib.swiftkv_set_split_mask(self._h, mask))
+
+    def set_half_weight_cache(self, n_layers: int) -> int:
+        """swiftkv_set_half_weight_cache: room (a torch tensor owned by this object) for the half copies of the first
+        `n_layers` layers' matrices, made once and kept from step to step; 0 removes it.  Call again after changing the
+        model's weights.  Returns the bytes held."""
+        cfg = _make_config(self.shape, self.dtype, self.kv_format)
+        need = int(self.lib.swiftkv_half_weight_cache_bytes(C.byref(cfg), n_layers))
+        if need < 0:
+            raise SwiftKVError(-1, "swiftkv_half_weight_cache_bytes rejected the config")
+        with torch.cuda.device(self.device):
+            self._w16_cache = torch.empty(need, dtype=torch.uint8, device=self.device) if need else None
+            _check(self.lib.swiftkv_set_half_weight_cache(self._h, self._w16_cache.data_ptr() if need else None, need))
+        return need
 
 
 def adamw_update(param: torch.Tensor, grad: torch.Tensor, exp_avg: torch.Tensor, exp_avg_sq: torch.Tensor, step: int,

@@ -115,6 +115,10 @@ struct swiftkv_model {
   // side stream on which the next layer's weights are copied to half while the current layer computes
   cudaStream_t side = nullptr;
   cudaEvent_t ev_start = nullptr, ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
+  // optional caller-owned room for the half copies of the first layers' matrices, kept from step to step
+  // (swiftkv_set_half_weight_cache): capacity and number of layers whose copies are current
+  __half *w16_cache = nullptr;
+  int w16_cache_cap = 0, w16_cache_valid = 0;
 };
 
 static size_t dsize(int dtype) { return dtype == SWIFTKV_DTYPE_BF16 ? 2 : 4; }
@@ -428,30 +432,35 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   if (bt.att_ctas > 0) { att_sched.off = b.att_off; att_sched.items = b.att_items; att_sched.n_ctas = bt.att_ctas; }
   const size_t w16_layer = (size_t)2 * d * dq + (size_t)2 * d * dkv + (size_t)3 * d * F;   // halves of one layer's copy
   __half *wq16 = nullptr, *wk16 = nullptr, *wv16 = nullptr, *wo16 = nullptr, *wg16 = nullptr, *wu16 = nullptr, *wd16 = nullptr;
-  auto w16_select = [&](int buf) {
-    wq16 = (__half *)b.w16 + (size_t)buf * w16_layer; wk16 = wq16 + (size_t)dq * d; wv16 = wk16 + (size_t)dkv * d;
+  auto w16_at = [&](__half *base) {
+    wq16 = base; wk16 = wq16 + (size_t)dq * d; wv16 = wk16 + (size_t)dkv * d;
     wo16 = wv16 + (size_t)dkv * d; wg16 = wo16 + (size_t)d * dq; wu16 = wg16 + (size_t)F * d; wd16 = wu16 + (size_t)F * d;
+  };
+  auto w16_select = [&](int buf) { w16_at((__half *)b.w16 + (size_t)buf * w16_layer); };
+  // layer j's seven matrices -> the selected half copies, on stream `s`
+  auto convert_into = [&](int j, cudaStream_t s, bool timed) {
+    const swiftkv_layer_weights &lw = m->layers[j];
+    Scope sc(m, s, SWIFTKV_KC_ELEMWISE, 7, timed);
+    launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, s, b.status);
+    launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, s, b.status);
   };
   // layer j's copy is made on the side stream into buffer j % 2 while layer j - 1 computes on `st`
   auto convert_layer = [&](int j) {
-    const swiftkv_layer_weights &lw = m->layers[j];
     const int buf = j & 1;
     if (j >= 2) cudaStreamWaitEvent(m->side, m->ev_free[buf], 0);   // layer j - 2 has finished with this buffer
     w16_select(buf);
-    {
-      Scope s(m, m->side, SWIFTKV_KC_ELEMWISE, 7, false);
-      launch_bf16_to_f16((const bf16 *)lw.wq, wq16, (long long)dq * d, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.wk, wk16, (long long)dkv * d, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.wv, wv16, (long long)dkv * d, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.wo, wo16, (long long)d * dq, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.w_gate, wg16, (long long)F * d, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.w_up, wu16, (long long)F * d, m->side, b.status);
-      launch_bf16_to_f16((const bf16 *)lw.w_down, wd16, (long long)d * F, m->side, b.status);
-    }
+    convert_into(j, m->side, false);
     cudaEventRecord(m->ev_ready[buf], m->side);
   };
+  // with room for them the copies of layers 1..l stay from step to step: made once, on `st`, by the first step that needs them
+  const bool w16_resident = use_w16 && m->w16_cache && l <= m->w16_cache_cap && !bt.decode;
   if constexpr (sizeof(T) == 2) {
-    if (use_w16 && l > 0 && !bt.decode) {
+    if (use_w16 && l > 0 && !bt.decode && !w16_resident) {
       cudaEventRecord(m->ev_start, st);                 // the side stream starts after everything queued before
       cudaStreamWaitEvent(m->side, m->ev_start, 0);
       convert_layer(0);
@@ -605,7 +614,10 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
       cudaMemcpyAsync(m->capture + (size_t)j * T_tok * d, b.x, (size_t)T_tok * d * sizeof(float), cudaMemcpyDeviceToDevice, st);
     }
     if constexpr (sizeof(T) == 2) {
-      if (use_w16) {
+      if (w16_resident) {
+        w16_at(m->w16_cache + (size_t)j * w16_layer);
+        if (j >= m->w16_cache_valid) convert_into(j, st, true);
+      } else if (use_w16) {
         if (j + 1 < l) convert_layer(j + 1);            // queued now, runs beside this layer's kernels
         w16_select(j & 1);
         cudaStreamWaitEvent(st, m->ev_ready[j & 1], 0);
@@ -730,7 +742,8 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     rc = gemm_any<TA, T>(m, act, T_tok, F, (const T *)lw.w_down, d, no_w, 0, no_w, 0, out_plain(OUT_RESID_ADD_F32, b.x, d, d), st,
                          use_w16 ? wd16 : nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, &down_split);
     if (rc) return rc;
-    if (use_w16) cudaEventRecord(m->ev_free[j & 1], st);   // this layer's half copies may be overwritten
+    if (w16_resident) m->w16_cache_valid = std::max(m->w16_cache_valid, j + 1);
+    else if (use_w16) cudaEventRecord(m->ev_free[j & 1], st);   // this layer's half copies may be overwritten
   }
 
   // ---- SingleInputKV (+ AcrossKV): one projection of s = x_{l+1} fills the caches of layers l+1..L (Eq. 2)
@@ -1199,6 +1212,23 @@ extern "C" int32_t swiftkv_set_activation_format(swiftkv_model *m, int32_t forma
     return fail(SWIFTKV_ERR_INVALID_ARG, "unknown activation format");
   m->act_format = format == SWIFTKV_ACT_F16_SPLIT ? SWIFTKV_ACT_F16 : format;
   m->split_mask = format == SWIFTKV_ACT_F16_SPLIT ? SWIFTKV_SPLIT_DEFAULT : 0;
+  return SWIFTKV_OK;
+}
+
+extern "C" int64_t swiftkv_half_weight_cache_bytes(const swiftkv_config *cfg, int32_t n_layers) {
+  if (!cfg || n_layers < 0 || cfg->hidden < 1 || cfg->ffn < 1 || cfg->head_dim < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1) return -1;
+  const long long d = cfg->hidden, dq = (long long)cfg->n_q_heads * cfg->head_dim, dkv = (long long)cfg->n_kv_heads * cfg->head_dim, F = cfg->ffn;
+  return (int64_t)((2 * d * dq + 2 * d * dkv + 3 * d * F) * 2 * n_layers);
+}
+
+extern "C" int32_t swiftkv_set_half_weight_cache(swiftkv_model *m, void *buffer, int64_t bytes) {
+  if (!m) return fail(SWIFTKV_ERR_INVALID_ARG, "model is null");
+  if ((buffer == nullptr) != (bytes == 0) || bytes < 0) return fail(SWIFTKV_ERR_INVALID_ARG, "buffer and bytes must both be given or both be zero");
+  if (reinterpret_cast<uintptr_t>(buffer) & 255) return fail(SWIFTKV_ERR_INVALID_ARG, "buffer must be 256-byte aligned");
+  const int64_t per_layer = swiftkv_half_weight_cache_bytes(&m->cfg, 1);
+  m->w16_cache = reinterpret_cast<__half *>(buffer);
+  m->w16_cache_cap = buffer ? (int)std::min<int64_t>(bytes / per_layer, m->cfg.n_layers) : 0;
+  m->w16_cache_valid = 0;
   return SWIFTKV_OK;
 }
 

@@ -28,6 +28,8 @@ def main():
     ap.add_argument("--kv-format", choices=("model", "fp8"), default="model")
     ap.add_argument("--chunks", default="8192,2048,512")
     ap.add_argument("--decode-steps", type=int, default=12)
+    ap.add_argument("--no-half-weight-cache", action="store_true",
+                    help="copy the layers' matrices to half in every step instead of once (swiftkv_set_half_weight_cache)")
     ap.add_argument("--kernel-mask", type=int, default=None, help="swiftkv_set_kernel_mask value (default: the library's)")
     args = ap.parse_args()
     shape = S.LLAMA31_8B
@@ -41,6 +43,8 @@ def main():
     model = P.SwiftKVModel(shape, w, torch.bfloat16, cap * n_seq, n_seq, SWIFT_LAYER, GROUP, kv_format=fmt)
     if args.kernel_mask is not None:
         model.set_kernel_mask(args.kernel_mask)
+    if not args.no_half_weight_cache:
+        model.set_half_weight_cache(SWIFT_LAYER)
     # paged: sequence b owns pages b, b + 8, b + 16, ... (interleaved with the other sequences' pages)
     pages = [[b + n_seq * i for i in range(PAGES_PER_SEQ)] for b in range(n_seq)]
 
@@ -73,7 +77,8 @@ def main():
         return steps
 
     base = {"model": "llama-3.1-8b shape bf16", "l": SWIFT_LAYER, "g": GROUP, "prompts": n_seq, "tokens": total,
-            "kv_format": args.kv_format, "data": "synthetic"}
+            "kv_format": args.kv_format, "data": "synthetic",
+            "half_weight_cache": not args.no_half_weight_cache}
     for chunk in [int(c) for c in args.chunks.split(",")]:
         for paged in (False, True):
             chunked(chunk, paged)

@@ -294,3 +294,64 @@ def test_chunked_prefill_and_decode_at_8b_widths(act, paged):
                 assert rel_l2(to_np(K[rows]), ref_of(b, m)["K"][j]) <= 2e-2, (mask, b, j)
                 assert rel_l2(to_np(V[rows]), ref_of(b, m)["V"][j]) <= 2e-2, (mask, b, j)
         model.close()
+
+
+def test_half_weight_cache_gives_the_same_bits_and_follows_weight_updates():
+    """swiftkv_set_half_weight_cache: the half copies of the first layers' matrices made once and kept, instead of once per
+    step.  Same conversion kernel, same GEMMs: logits and caches of chunked steps and of a one-shot prefill are bit-identical
+    with and without it; a cache too small for the step's l falls back to per-step copies; after the caller changes a weight
+    and sets the cache again, the result follows the new weight (and differs from the stale one)."""
+    import paper_2410_03960_b200 as P
+    shape, l, g, seed = MID, 3, 1, 23
+    lens, cap, chunk = [300, 130], 384, 128
+    w = S.make_weights(shape, seed, torch.bfloat16, "cuda")
+    toks = [S.token_ids(seed, b, n, shape.vocab) for b, n in enumerate(lens)]
+
+    def run(model):
+        done = [0] * len(lens)
+        while any(d < n for d, n in zip(done, lens)):
+            seqs, packed = [], []
+            for b, n in enumerate(lens):
+                if done[b] < n:
+                    k = min(chunk, n - done[b])
+                    seqs.append((k, done[b], b * cap, int(done[b] + k == n)))
+                    packed.append(toks[b][done[b]:done[b] + k])
+                    done[b] += k
+            model.step(torch.cat(packed), seqs, l, g)
+        model.status()
+        out = [model.first_logits().clone()]
+        for j in range(shape.n_layers):
+            K, V, _ = model.kv_cache_view(j)
+            out += [K.clone(), V.clone()]
+        return out
+
+    model = P.SwiftKVModel(shape, w, torch.bfloat16, cap * len(lens), len(lens), l, g)
+    plain = run(model)
+    launches_plain = model.last_launch_count()
+    assert model.set_half_weight_cache(l) == 2 * l * (2 * shape.hidden * shape.n_q_heads * shape.head_dim +
+                                                      2 * shape.hidden * shape.n_kv_heads * shape.head_dim + 3 * shape.hidden * shape.ffn)
+    first = run(model)          # makes the copies
+    again = run(model)          # reuses them
+    assert model.last_launch_count() == launches_plain - 7 * l          # the last step no longer copies 7 matrices per layer
+    for a, b_, c in zip(plain, first, again):
+        assert torch.equal(a, b_) and torch.equal(a, c)
+    model.set_half_weight_cache(l - 1)                                   # too small for l: per-step copies again
+    for a, b_ in zip(plain, run(model)):
+        assert torch.equal(a, b_)
+    assert model.last_launch_count() == launches_plain
+    # a weight update: stale copies until the cache is set again
+    model.set_half_weight_cache(l)
+    run(model)
+    w.layers[0]["w_down"].mul_(0.5)
+    stale = run(model)
+    assert all(torch.equal(a, b_) for a, b_ in zip(plain, stale))        # (documented: the library cannot see the change)
+    model.set_half_weight_cache(l)
+    fresh = run(model)
+    model.set_half_weight_cache(0)
+    uncached = run(model)
+    assert not torch.equal(fresh[0], plain[0])
+    for a, b_ in zip(fresh, uncached):
+        assert torch.equal(a, b_)
+    with pytest.raises(P.SwiftKVError):
+        P.binding._check(model.lib.swiftkv_set_half_weight_cache(model._h, None, 256))
+    model.close()
