@@ -28,6 +28,7 @@ def main():
     ap.add_argument("--kv-format", choices=("model", "fp8"), default="model")
     ap.add_argument("--chunks", default="8192,2048,512")
     ap.add_argument("--decode-steps", type=int, default=12)
+    ap.add_argument("--profile", action="store_true", help="also print the kernel classes' CUDA-event times of each chunked run")
     ap.add_argument("--no-half-weight-cache", action="store_true",
                     help="copy the layers' matrices to half in every step instead of once (swiftkv_set_half_weight_cache)")
     ap.add_argument("--kernel-mask", type=int, default=None, help="swiftkv_set_kernel_mask value (default: the library's)")
@@ -85,6 +86,14 @@ def main():
             ms, steps = timed(lambda: chunked(chunk, paged))
             print(json.dumps(dict(base, what="chunked_prefill", chunk=chunk, paged=paged, steps=steps, ms=round(ms, 2),
                                   tokens_per_s=round(total / ms * 1e3, 1))), flush=True)
+            if args.profile:
+                model.profile_enable(True)
+                model.profile_read()
+                chunked(chunk, paged)
+                prof = model.profile_read()
+                model.profile_enable(False)
+                print(json.dumps(dict(what="kernel_classes_ms", chunk=chunk, paged=paged,
+                                      **{k: [round(v[0], 2), v[1]] for k, v in prof.items()})), flush=True)
     for paged in (False, True):
         chunked(8192, paged)
 
