@@ -959,6 +959,7 @@ constexpr int RES_BYTES = 131072;                     // K * 32 <= RES_BYTES: re
 constexpr int RED_FLOATS = 2 * CONSUMERS * 2 * 32 * 4;   // two buffers of [warp][matrix][lane][4]
 constexpr int SM_RED = POOL_BYTES, SM_BAR = SM_RED + RED_FLOATS * 4, SM_MISC = SM_BAR + 256;
 constexpr int SMEM_BYTES = SM_MISC + 256 + 1024;      // 230912 incl. the slack to align the ring to 1024 bytes
+static_assert(RES_BYTES / 32 * 2 <= RED_FLOATS * 2, "a resident stage's norm gains (2 bytes per K) fit the first reduction buffer");
 static_assert(MIN_STAGES * STAGE_BYTES + RES_BYTES <= POOL_BYTES, "8 rows: 5 ring stages + 128 KB of resident activations");
 constexpr long long WAIT_LIMIT = 4000000000LL;
 constexpr int MAX_STAGE_LIST = 6;
@@ -1166,6 +1167,10 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
     //  gave up keeps walking the same barriers and only skips the work)
     dead = !ring_wait(p, c, smem_u32(afull), c.fill_no & 1);
     c.fill_no += 1;
+    // the norm gains were requested into the (idle) reduction area before the grid barrier: fetched from global memory one
+    // pair per conversion step they cost a dependent L2 round trip per step -- 0.7 ms of a 6.4 ms decode step, measured
+    cp_async_wait<0>();
+    consumer_sync();
     // every warp converts, in place, exactly the blocks it will multiply with, 8 / RP blocks at a time:
     // lane = (block of the group, row, quarter)
     const int grp = g >> rs, r = g & (RP - 1), G = 8 >> rs;
@@ -1189,7 +1194,7 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
         x[h][0] = xa.x; x[h][1] = xa.y; x[h][2] = xa.z; x[h][3] = xa.w;
         x[h][4] = xb.x; x[h][5] = xb.y; x[h][6] = xb.z; x[h][7] = xb.w;
         gm[h] = make_uint4(0u, 0u, 0u, 0u);
-        if (sg.gamma && live[h]) gm[h] = __ldg(reinterpret_cast<const uint4 *>(sg.gamma + (size_t)s * 32 + t * 8));
+        if (sg.gamma && live[h]) gm[h] = *reinterpret_cast<const uint4 *>(reinterpret_cast<const uint8_t *>(red) + ((size_t)s * 32 + t * 8) * 2);
       }
       __syncwarp();
 #pragma unroll
@@ -1389,18 +1394,25 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
     }
   } else {
     for (int i = 0; i < p.n_stages; ++i) {
+      const Stage &sg = p.st[i];
+      const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
+      // a resident stage's norm gains (at most 8 KB, constants) travel while the CTA waits at the barrier: the reduction
+      // area is idle between the previous stage's last epilogue and this stage's first
+      if (resident && sg.gamma)
+        for (int o = (int)threadIdx.x * 16; o < sg.K * 2; o += CONSUMERS * 32 * 16)
+          cp_async16(fsmem + SM_RED + o, reinterpret_cast<const uint8_t *>(sg.gamma) + o);
+      cp_async_commit();
       if (i > 0) {
         if (!grid_barrier(p, c)) break;
         if (threadIdx.x == 0) *c.open_s = i;
       }
-      const Stage &sg = p.st[i];
-      const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
       if (sg.epi >= 2) { if (resident) consume<true, true>(p, c, sg); else consume<true, false>(p, c, sg); }
       else { if (resident) consume<false, true>(p, c, sg); else consume<false, false>(p, c, sg); }
       if (threadIdx.x == 0) *c.decide_s = *c.abort_s;      // (consume ended with a barrier of the MMA warps)
       consumer_sync();
       if (*c.decide_s) break;
     }
+    cp_async_wait<0>();      // (a gain request of a stage that was never reached)
   }
   __syncthreads();
 }
