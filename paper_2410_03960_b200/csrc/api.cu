@@ -71,6 +71,7 @@ struct Buffers {
   float *hy, *qy, *ay, *acty;  // the continuing tokens' activations stay in fp32
   float *ky, *vy;           // a decode step's new K / V rows before they go to the cache, KV_STAGE_SLOTS x [8, d_kv] each
   float *tail_scratch;
+  void *tail_handover;      // the fused last-token launch: rows published pre-split from one stage to the next
   float *logits;            // [B, vocab]
   int32_t *tokens, *cu, *pos, *last_idx, *last_pos;
   int32_t *att_off, *att_items;   // schedule of the persistent attention kernel: [ATT_MAX_CTAS + 1] offsets, items
@@ -176,6 +177,7 @@ static void carve_all(const swiftkv_config &c, int T, int B, size_t fold_elems, 
   b.ky = (float *)cv.take(KV_STAGE_SLOTS * R * dkv_ * 4);      // (several AcrossKV groups' rows per fused launch)
   b.vy = (float *)cv.take(KV_STAGE_SLOTS * R * dkv_ * 4);
   b.tail_scratch = (float *)cv.take(tail_attention_scratch_bytes(B, c.n_q_heads, c.head_dim, T));
+  b.tail_handover = cv.take(TAIL_HANDOVER_BYTES);
   b.logits = (float *)cv.take((size_t)B * c.vocab * 4);
   b.tokens = (int32_t *)cv.take((size_t)T * 4);
   b.cu = (int32_t *)cv.take((size_t)(B + 1) * 4);
@@ -514,7 +516,7 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
   auto flush = [&](int rows) -> int32_t {
     if (n_list == 0) return SWIFTKV_OK;
     Scope s(m, st, SWIFTKV_KC_TAIL);
-    const int frc = launch_tail_fused(list, n_list, rows, c.rms_eps, b.status + 32, &fused_arrivals, b.status, st);
+    const int frc = launch_tail_fused(list, n_list, rows, c.rms_eps, b.status + 32, &fused_arrivals, b.status, st, 0, b.tail_handover);
     n_list = 0;
     return frc == SWIFTKV_OK ? SWIFTKV_OK : fail(frc, "fused last-token launch failed: %s", cudaGetErrorString(cudaGetLastError()));
   };

@@ -328,7 +328,11 @@ int run_distill(const DistillDims &c, const DistillArgs &a, const DistillLayer *
 // together).
 // wait_limit_clocks: how long any single wait inside the kernel (ring stage, grid barrier) may take before the kernel latches
 // STATUS_TIMEOUT and every role leaves (0: the default of about two seconds).
+// handover: TAIL_HANDOVER_BYTES of device scratch (or null): where a stage publishes its output rows pre-split for the resident,
+// normed stage that follows it in the same launch (SWIFTKV_TAIL_HANDOVER=0 keeps every stage converting for itself).
+constexpr size_t TAIL_HANDOVER_IMAGE_BYTES = 131072;                       // K <= 4096, 8 row slots, hi + lo
+constexpr size_t TAIL_HANDOVER_BYTES = TAIL_HANDOVER_IMAGE_BYTES + 256 * MAX_TAIL_ROWS * sizeof(float);
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
-                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks = 0);
+                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks = 0, void *handover = nullptr);
 
 }  // namespace skv

@@ -137,6 +137,28 @@ int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t r
   return 0;
 }
 
+// the same blocks already laid out as the kernel keeps them in shared memory: [K / 32][row slots][32 words], contiguous
+int get_tmap_act_image(CUtensorMap *out, const void *p, uint32_t row_slots, uint64_t K, uint32_t steps) {
+  TmapKey k{p, row_slots, K, 0xFFFFFFFCull, row_slots, steps};
+  std::lock_guard<std::mutex> g(g_tmap_mu);
+  auto it = g_tmaps.find(k);
+  if (it != g_tmaps.end()) { *out = it->second; return 0; }
+  if (g_tmaps.size() > 65536) g_tmaps.clear();
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return -1;
+  CUtensorMap m;
+  cuuint64_t dims[3] = {32, row_slots, K / 32};
+  cuuint64_t strides[2] = {128, (cuuint64_t)row_slots * 128};
+  cuuint32_t box[3] = {32, row_slots, steps};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(p), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return -2;
+  g_tmaps.emplace(k, m);
+  *out = m;
+  return 0;
+}
+
 // fp32 matrix [rows, cols] row-major: tiles of box_rows x 32 elements (128 bytes), 128-byte swizzle (the tf32 GEMM's operands)
 int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t ld) {
   if (ld == 0) ld = cols;

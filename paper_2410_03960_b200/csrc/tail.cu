@@ -991,6 +991,16 @@ struct Stage {
   const bf16 *gamma;       // non-null: A is RMS-normalised on the fly (row statistic * gain)
   float *out, *out2;
   int N, K, ldo, epi;
+  // Hand-over between two adjacent stages of one launch (the second one resident and normed, reading the first one's output):
+  // the first stage's epilogue also publishes its rows as the second one needs them in shared memory -- multiplied by the
+  // second stage's gain, split into bf16 hi / lo, in the fragment layout of one block per 32-wide K step -- and the sum of
+  // squares of each row over its 16 features; the second stage's fill is then its whole set-up (otherwise all 148 CTAs
+  // repeat the same fp32 -> hi / lo pass over the whole activation vector for themselves).
+  uint8_t *pub_image;          // producer: where to publish (null: do not)
+  float *pub_ss;               // producer: [N / 16][8] partial sums of squares
+  const bf16 *pub_gamma;       // producer: the consuming stage's gain
+  int presplit;                // consumer: tmA points at the published image; the row statistics come from pre_ss
+  const float *pre_ss;
 };
 struct Params {
   Stage st[MAX_STAGE_LIST];
@@ -1156,7 +1166,25 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
   // row in the epilogue (it is a per-row scalar), so it can be accumulated in the same pass that brings the activations in
   float ss = 0.f;                                      // RESIDENT: this lane's row (g); else row (lane & 7)
   bool dead = false;
-  if (RESIDENT) {
+  if (RESIDENT && sg.presplit) {
+    // the producing stage published hi / lo fragments and per-tile sums of squares: fill, row statistics, done
+    if (threadIdx.x == 0) {
+      fence_generic_to_async();
+      mbar_expect_tx(smem_u32(afull), (uint32_t)(K / 32) * (uint32_t)AB);
+      for (int part = 0; part < K / KC1; ++part)
+        tc::tma_load_3d(smem_u32(res + part * (KC1 / 32) * AB), &sg.tmA, smem_u32(afull), 0, 0, part * (KC1 / 32));
+    }
+    if (warp < p.rows) {            // warp w: row w, the producer's K / 16 tiles in a fixed order
+      float tot = 0.f;
+      for (int tl = lane; tl < K / 16; tl += 32) tot += __ldcg(sg.pre_ss + (size_t)tl * MAX_TAIL_ROWS + warp);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+      if (lane == 0) rstd_s[warp] = rsqrtf(tot / (float)K + p.eps);
+    }
+    dead = !ring_wait(p, c, smem_u32(afull), c.fill_no & 1);
+    c.fill_no += 1;
+    cp_async_wait<0>();
+  } else if (RESIDENT) {
     if (threadIdx.x == 0) {
       fence_generic_to_async();
       mbar_expect_tx(smem_u32(afull), (uint32_t)(K / 32) * (uint32_t)AB);
@@ -1231,7 +1259,7 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
     ss += __shfl_xor_sync(0xffffffffu, ss, 1);
     ss += __shfl_xor_sync(0xffffffffu, ss, 2);
   }
-  if (sg.gamma) {
+  if (sg.gamma && !(RESIDENT && sg.presplit)) {
     float *part = red + 2 * CONSUMERS * 2 * 32 * 4 - CONSUMERS * MAX_TAIL_ROWS;      // the tail of the second buffer: [8 warps][8 rows]
     if (t == 0 && g < (RESIDENT ? RP : MAX_TAIL_ROWS)) part[warp * MAX_TAIL_ROWS + g] = ss;
     consumer_sync();
@@ -1339,6 +1367,11 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
           s1[i] += buf[((w * 2 + 0) * 32 + lane) * 4 + i];
           if (DUAL) s2[i] += buf[((w * 2 + 1) * 32 + lane) * 4 + i];
         }
+      float pg[2] = {0.f, 0.f}, sq[2] = {0.f, 0.f};
+      if (!DUAL && sg.pub_image) {
+        pg[0] = to_f(sg.pub_gamma[tile * 16 + g]);
+        pg[1] = to_f(sg.pub_gamma[tile * 16 + g + 8]);
+      }
 #pragma unroll
       for (int i = 0; i < 4; ++i) {      // fragment element i: feature 16 tile + g + 8 (i / 2), token 2 t + (i % 2)
         const int n = tile * 16 + g + 8 * (i >> 1), r = 2 * t + (i & 1);
@@ -1352,6 +1385,26 @@ __device__ void consume(const Params &p, Ctx &c, const Stage &sg) {
           float *o = sg.out + (size_t)r * sg.ldo + n;
           if (sg.epi == 1) v += __ldcg(o);
           *o = v;
+          if (!DUAL && sg.pub_image) {
+            // element n of row r in the consumer's block n / 32: quarter (n % 32) / 8 of the row, 16-bit slot n % 8; hi half of
+            // the block, then lo half
+            sq[i & 1] = fmaf(v, v, sq[i & 1]);
+            const float x = v * pg[i >> 1];
+            const bf16 hi = __float2bfloat16_rn(x);
+            const bf16 lo = __float2bfloat16_rn(x - to_f(hi));
+            uint8_t *dst = sg.pub_image + (size_t)(n >> 5) * AB + (4 * r + ((n & 31) >> 3)) * 16 + (n & 7) * 2;
+            *reinterpret_cast<bf16 *>(dst) = hi;
+            *reinterpret_cast<bf16 *>(dst + (AB >> 1)) = lo;
+          }
+        }
+      }
+      if (!DUAL && sg.pub_image) {       // rows 2 t, 2 t + 1: sum over the tile's 16 features (the 8 lanes that share t, two each)
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {
+          sq[rr] += __shfl_xor_sync(0xffffffffu, sq[rr], 4);
+          sq[rr] += __shfl_xor_sync(0xffffffffu, sq[rr], 8);
+          sq[rr] += __shfl_xor_sync(0xffffffffu, sq[rr], 16);
+          if (g == 0 && 2 * t + rr < p.rows) sg.pub_ss[(size_t)tile * MAX_TAIL_ROWS + 2 * t + rr] = sq[rr];
         }
       }
     }
@@ -1398,7 +1451,7 @@ __global__ void __launch_bounds__(THREADS, 1) tail_fused_kernel(const __grid_con
       const bool resident = (long long)sg.K * 32 <= RES_BYTES;      // 1 KB per 32-wide K step (8 row slots x (hi + lo))
       // a resident stage's norm gains (at most 8 KB, constants) travel while the CTA waits at the barrier: the reduction
       // area is idle between the previous stage's last epilogue and this stage's first
-      if (resident && sg.gamma)
+      if (resident && sg.gamma && !sg.presplit)
         for (int o = (int)threadIdx.x * 16; o < sg.K * 2; o += CONSUMERS * 32 * 16)
           cp_async16(fsmem + SM_RED + o, reinterpret_cast<const uint8_t *>(sg.gamma) + o);
       cp_async_commit();
@@ -1435,7 +1488,7 @@ bool tail_fused_supported(int rows, int d, int dq, int F, int vocab) {
 }
 
 int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps, unsigned int *sync, unsigned int *arrivals,
-                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks) {
+                      unsigned int *status, cudaStream_t st, long long wait_limit_clocks, void *handover) {
   if (n_stages < 1 || n_stages > fused::MAX_STAGE_LIST || rows < 1 || rows > MAX_TAIL_ROWS) return SWIFTKV_ERR_UNSUPPORTED;
   fused::Params p{};
   int rs = 0;
@@ -1452,6 +1505,25 @@ int launch_tail_fused(const TailStage *stages, int n_stages, int rows, float eps
     const bool resident = (long long)s.K * 32 <= fused::RES_BYTES;
     if (get_tmap_act_f32(&d.tmA, s.A, rows, 1u << rs, s.K, resident ? fused::KC1 / 32 : kc / 32)) return SWIFTKV_ERR_CUDA;
     d.A = s.A; d.gamma = reinterpret_cast<const bf16 *>(s.gamma); d.out = s.out; d.out2 = s.out2; d.N = s.N; d.K = s.K; d.ldo = s.ldo; d.epi = s.epi;
+  }
+  // a resident, normed stage that reads the output of the stage right before it takes that output pre-split from the
+  // producer's epilogue (one hand-over area serves every such pair of the launch: a pair's fill is over before the next
+  // producer's first epilogue, two grid barriers later)
+  static int handover_on = -1;
+  if (handover_on < 0) { const char *e = getenv("SWIFTKV_TAIL_HANDOVER"); handover_on = (e && e[0] == '0') ? 0 : 1; }
+  if (handover && handover_on) {
+    uint8_t *image = reinterpret_cast<uint8_t *>(handover);
+    float *ss = reinterpret_cast<float *>(image + TAIL_HANDOVER_IMAGE_BYTES);
+    for (int i = 1; i < n_stages; ++i) {
+      const TailStage &a = stages[i - 1], &b = stages[i];
+      const bool resident = (long long)b.K * 32 <= fused::RES_BYTES;
+      if (!resident || !b.gamma || b.A != a.out || a.epi > 1 || a.N != b.K || a.ldo != b.K) continue;
+      fused::Stage &pa = p.st[i - 1], &pb = p.st[i];
+      if (pa.presplit) continue;      // (it still fills from the area while its own fastest CTAs would already publish into it)
+      if (get_tmap_act_image(&pb.tmA, image, 1u << rs, b.K, fused::KC1 / 32)) return SWIFTKV_ERR_CUDA;
+      pa.pub_image = image; pa.pub_ss = ss; pa.pub_gamma = reinterpret_cast<const bf16 *>(b.gamma);
+      pb.presplit = 1; pb.pre_ss = ss;
+    }
   }
   p.n_stages = n_stages; p.rows = rows; p.eps = eps; p.sync = sync; p.status = status;
   // ring depth: as many 16 KB stages as fit beside the activation area this launch needs (resident blocks of its widest

@@ -293,6 +293,7 @@ int make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t 
 int get_tmap_rows16(CUtensorMap *out, const void *p, uint64_t N, uint64_t K, uint32_t chunks);
 int get_tmap_f32(CUtensorMap *out, const float *p, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t ld = 0);      // ld: row stride in elements (0: cols)
 int get_tmap_act_f32(CUtensorMap *out, const float *p, uint32_t rows, uint32_t row_slots, uint64_t K, uint32_t steps);
+int get_tmap_act_image(CUtensorMap *out, const void *p, uint32_t row_slots, uint64_t K, uint32_t steps);
 
 // cached make_tmap_2d_bf16 (tensor maps are pure functions of pointer, shape and box)
 int get_tmap(CUtensorMap *out, const void *p, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows, uint32_t box_cols);
