@@ -917,6 +917,22 @@ int launch_gemm_tc(const void *A, bool f16, int M, int K, const void *B0, int nB
     if (nB2 > 0 && get_tmap(&tb2h, B2, nB2, K, K, 128, BK)) return SWIFTKV_ERR_CUDA;
   }
   const int pair_tiles = ((M + 255) / 256) * (N / 256);
+  // Few rows: a launch whose CTA pairs would cover less than half of the SMs runs as single CTAs on 128 x 128 tiles instead
+  // (four times as many CTAs, each with a quarter of a pair's work) -- e.g. 512 rows x 4096 features: 128 CTAs instead of 64;
+  // same accumulation order, same bits.  Only for long inner dimensions, where the launch is bound by streaming the weights
+  // (a 256-token prompt at the 8B widths: 7.5 -> 7.2 ms); short ones are launch-latency either way.
+  static int small_m_single = -1;
+  if (small_m_single < 0) { const char *e = getenv("SWIFTKV_SMALL_M_SINGLE"); small_m_single = (e && e[0] == '0') ? 0 : 1; }
+  if (pairs && small_m_single && K >= 2048 && 4 * pair_tiles <= num_sms()) {
+    p.num_n_blocks = N / 128;
+    if (rope) {
+      if (rope->hd != 128 || out.mode != OUT_STORE || (out.n0 % 128) || (out.n0 < N && (out.seg_w % 128)))
+        return SWIFTKV_ERR_UNSUPPORTED;
+      p.rope_pos = rope->positions; p.cos_tab = rope->cos_tab; p.sin_tab = rope->sin_tab;
+      return launch_cfg<128, 6, EPI_ROPE>(ta, tb0h, tb1h, tb2h, p, st);
+    }
+    return launch_cfg<128, 6, EPI_PLAIN>(ta, tb0h, tb1h, tb2h, p, st);
+  }
   if (rope) {
     // fused rotary embedding needs head-aligned tiles of 128-wide heads and a bf16 store
     if (rope->hd != 128 || out.mode != OUT_STORE || (out.n0 % 128) || (out.n0 < N && (out.seg_w % 128)))
