@@ -223,7 +223,8 @@ W8B_4L = S.ModelShape(128256, 4096, 4, 32, 8, 128, 14336, 500000.0, 1e-5, "8b-wi
 def test_chunked_prefill_and_decode_at_8b_widths(act, paged):
     """The deployment path at the real Llama-3.1-8B widths (hidden 4096, 32 / 8 heads, FFN 14336; 4 layers, l = 2):
     chunks that are not multiples of the 128-row tiles and attend to a cached prefix, then three decode steps on the
-    weight-streaming decode path (kernel-mask bit 5) and, on a second model, on the general path -- contiguous regions and
+    fused persistent launch (kernel-mask bits 5 and 6, the default), on the per-operator weight-streaming kernels (bit 5) and on
+    the general path, each on a model of its own -- contiguous regions and
     scattered pages, both activation formats -- against the oracle's one-shot prefill of the same token sequences."""
     import paper_2410_03960_b200 as P
     shape, dtype, seed, l, g = W8B_4L, torch.bfloat16, 13, 2, 1
@@ -253,7 +254,10 @@ def test_chunked_prefill_and_decode_at_8b_widths(act, paged):
             return torch.as_tensor(_paged_rows(pages[b], m), device="cuda")
         return torch.arange(b * cap_pages * 128, b * cap_pages * 128 + m, device="cuda")
 
-    for mask in (55, 23):                                        # decode steps on the weight-streaming path / the general path
+    # decode steps on the fused persistent launch (the default: one launch per layer, K / V of the new token from the same
+    # launch as Q, rows handed over pre-split between its stages), on the per-operator weight-streaming kernels, and on the
+    # general path
+    for mask in (119, 55, 23):
         model = P.SwiftKVModel(shape, w, dtype, 4 * cap_pages * 128, len(lens), l, g)
         model.set_kernel_mask(mask)
         model.set_activation_format(act)
