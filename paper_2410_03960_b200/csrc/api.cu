@@ -530,13 +530,10 @@ static int32_t run_prefill(swiftkv_model *m, const Batch &bt, int l, int g, cuda
     float *hy = b.hy, *qy = b.qy, *ay = b.ay, *acty = b.acty, *ky = b.ky, *vy = b.vy, *y = b.y;
     const TailOpts q_rope{b.last_pos, b.cos_tab, b.sin_tab, bt.total_kv};     // the queries are rotated inside the attention kernel
     auto store_kv = [&](int slot, float *ky, float *vy) {      // ky -> rotary embedding, vy -> the cache rows of the new tokens in `slot`
-      if (fp8) {
-        Scope s(m, st, SWIFTKV_KC_TAIL, 5);
-        launch_rope<float>(ky, 0, 1, b.last_pos, nullptr, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim, st);
-        launch_scatter_rows<T>(ky, kst, nullptr, rows, dkv, st);    // rows are quantized from the model dtype
-        launch_scatter_rows<T>(vy, vst, nullptr, rows, dkv, st);
-        launch_quantize_rows_fp8<T, T>(kst, rows, dkv, b.slot, k_codes(slot), k_scale(slot), (T *)nullptr, st);
-        launch_quantize_rows_fp8<T, T>(vst, rows, dkv, b.slot, v_codes(slot), v_scale(slot), (T *)nullptr, st);
+      if (fp8) {        // (rows are quantized from the model dtype)
+        Scope s(m, st, SWIFTKV_KC_TAIL);
+        launch_store_kv_rows_fp8<T>(ky, vy, b.slot, b.last_pos, b.cos_tab, b.sin_tab, rows, c.n_kv_heads, c.head_dim,
+                                    k_codes(slot), k_scale(slot), v_codes(slot), v_scale(slot), st);
       } else {
         Scope s(m, st, SWIFTKV_KC_TAIL);
         launch_store_kv_rows<T>(ky, vy, kv + (size_t)slot * 2 * plane, kv + (size_t)slot * 2 * plane + plane, b.slot, b.last_pos,

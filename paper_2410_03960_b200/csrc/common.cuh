@@ -139,6 +139,12 @@ void launch_gather_kv_half(const bf16 *k, const bf16 *v, __half *k16, __half *v1
 // kv_fp8.cu : per-token FP8 cache rows.  One scale per row of `width` elements: scale = max(amax, 2^-64) / 448,
 // code = e4m3(x / scale) (correctly rounded fp32 divisions, round to nearest even, saturating).  Row r of `src` goes to row
 // slot_map[r] (null: r) of `codes` / `scale`; deq (nullable, row r) receives value(code) * scale in type TO.
+// the new K / V rows of a decode minibatch (fp32, one per sequence) -> FP8 cache rows slot_map[r]: rotary embedding on K, rounding
+// to the model dtype T, per-row scale, codes -- one launch
+template <typename T>
+void launch_store_kv_rows_fp8(const float *ky, const float *vy, const int32_t *slot_map, const int32_t *positions, const float *cos_tab,
+                              const float *sin_tab, int rows, int n_heads, int hd, uint8_t *k_codes, float *k_scale, uint8_t *v_codes,
+                              float *v_scale, cudaStream_t st);
 template <typename TI, typename TO>
 void launch_quantize_rows_fp8(const TI *src, int rows, int width, const int32_t *slot_map, uint8_t *codes, float *scale,
                               TO *deq, cudaStream_t st);

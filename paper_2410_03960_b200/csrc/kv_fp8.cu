@@ -110,7 +110,63 @@ __global__ void __launch_bounds__(QT) gather_dequant_kernel(const uint8_t *__res
   for (int i = threadIdx.x; i < dkv; i += QT) o[i] = from_f<TO>(__fmul_rn(to_f(fp8e4{c[i]}), s));
 }
 
+// A decode minibatch's new K / V rows (fp32, one row per sequence) into the FP8 cache in one pass: rotary embedding on K (the
+// arithmetic of rope_kernel), rounding to the model dtype (the cache is defined as the quantized model-dtype row), per-row
+// scale and codes (the arithmetic of quantize_rows_kernel).  Block (row, K or V); the rounded row waits in shared memory
+// between the maximum and the encoding.
+template <typename T>
+__global__ void __launch_bounds__(QT) store_kv_rows_fp8_kernel(const float *__restrict__ ky, const float *__restrict__ vy,
+                                                               const int32_t *__restrict__ slot_map, const int32_t *__restrict__ positions,
+                                                               const float *__restrict__ cos_tab, const float *__restrict__ sin_tab,
+                                                               int n_heads, int hd, uint8_t *__restrict__ k_codes,
+                                                               float *__restrict__ k_scale, uint8_t *__restrict__ v_codes,
+                                                               float *__restrict__ v_scale) {
+  extern __shared__ float row_s[];
+  __shared__ float red[QT / 32];
+  const int r = blockIdx.x, width = n_heads * hd, half = hd >> 1;
+  const bool is_v = blockIdx.y != 0;
+  const float *src = (is_v ? vy : ky) + (size_t)r * width;
+  float amax = 0.f;
+  if (!is_v) {
+    const int p = positions[r];
+    for (int idx = threadIdx.x; idx < n_heads * half; idx += QT) {
+      const int h = idx / half, i = idx % half;
+      const float c = cos_tab[(size_t)p * half + i], s = sin_tab[(size_t)p * half + i];
+      const float a = src[h * hd + i], b = src[h * hd + i + half];
+      const float x0 = to_f(from_f<T>(a * c - b * s)), x1 = to_f(from_f<T>(b * c + a * s));
+      row_s[h * hd + i] = x0;
+      row_s[h * hd + i + half] = x1;
+      amax = fmaxf(amax, fmaxf(fabsf(x0), fabsf(x1)));
+    }
+  } else {
+    for (int i = threadIdx.x; i < width; i += QT) {
+      const float x = to_f(from_f<T>(src[i]));
+      row_s[i] = x;
+      amax = fmaxf(amax, fabsf(x));
+    }
+  }
+  amax = block_max(amax, red);      // (its barrier also publishes row_s)
+  const float scale = __fdiv_rn(fmaxf(amax, FP8_AMAX_FLOOR), FP8_MAX);
+  const size_t orow = (size_t)slot_map[r];
+  if (threadIdx.x == 0) (is_v ? v_scale : k_scale)[orow] = scale;
+  uint8_t *c = (is_v ? v_codes : k_codes) + orow * width;
+  for (int i = threadIdx.x; i < width; i += QT) c[i] = encode_e4m3(row_s[i], scale);
+}
+
 }  // namespace
+
+template <typename T>
+void launch_store_kv_rows_fp8(const float *ky, const float *vy, const int32_t *slot_map, const int32_t *positions, const float *cos_tab,
+                              const float *sin_tab, int rows, int n_heads, int hd, uint8_t *k_codes, float *k_scale, uint8_t *v_codes,
+                              float *v_scale, cudaStream_t st) {
+  if (rows <= 0) return;
+  store_kv_rows_fp8_kernel<T><<<dim3((unsigned)rows, 2), QT, (size_t)n_heads * hd * sizeof(float), st>>>(
+      ky, vy, slot_map, positions, cos_tab, sin_tab, n_heads, hd, k_codes, k_scale, v_codes, v_scale);
+}
+template void launch_store_kv_rows_fp8<bf16>(const float *, const float *, const int32_t *, const int32_t *, const float *, const float *, int,
+                                             int, int, uint8_t *, float *, uint8_t *, float *, cudaStream_t);
+template void launch_store_kv_rows_fp8<float>(const float *, const float *, const int32_t *, const int32_t *, const float *, const float *, int,
+                                              int, int, uint8_t *, float *, uint8_t *, float *, cudaStream_t);
 
 template <typename TI, typename TO>
 void launch_quantize_rows_fp8(const TI *src, int rows, int width, const int32_t *slot_map, uint8_t *codes, float *scale,
